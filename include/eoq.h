@@ -1,0 +1,176 @@
+/*
+ * eoq.h -- C ABI of the EOQ 8-bit integer training layer on NVIDIA sm_100a.
+ *
+ * The library implements the quantized convolution layer of the BN-free Fixup
+ * residual network of "Towards Efficient Full 8-bit Integer DNN Online Training
+ * on Resource-limited Devices without Batch Normalization" (arXiv 2105.13890):
+ * forward, error back-propagation and weight gradient, each an int8 x int8 ->
+ * int32 implicit GEMM, fused with the paper's quantizers, plus the 8-bit update.
+ *
+ * Conventions for every entry point
+ *   - A quantized tensor is (integer codes, exponent p): real value = code * 2^p.
+ *     Forward-side tensors (activations, weights, gamma, biases) sit on the grid
+ *     of Q(., 8), p = -7, and carry no exponent.  Outputs of the scale quantizer
+ *     SQ carry one int32 exponent per tensor, kept in DEVICE memory so that no
+ *     host round trip separates producer and consumer.
+ *   - All bit widths are 8 (Sec. 5.1).  R(.) rounds to nearest, ties to even.
+ *   - Layouts: activations and errors NHWC int8; weights [c_out][kh][kw][c_in]
+ *     int8.  c_in and c_out must be multiples of 16 (pad with zero channels).
+ *   - Pointers named in a "device" list are device pointers the caller owns; the
+ *     library never allocates or frees tensor memory.  Tensor pointers must be
+ *     16-byte aligned.  Scratch memory is the caller's `workspace` (device, 256-byte
+ *     aligned, at least eoq_workspace_size() bytes; contents are undefined on
+ *     entry and on return).  The handle owns only a few hundred bytes of device
+ *     state (status word, small reduction cells).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls enqueue work and return without synchronising, except
+ *     eoq_create, eoq_destroy and eoq_last_status.
+ *   - Every function returns an eoq_status_t.  Nothing throws, traps or aborts.
+ *     Conditions only the device can see (a wait that ran out, a non-finite
+ *     input, an all-zero SQ input) are OR-ed into the handle's device status
+ *     word; eoq_last_status() reads and clears it.
+ */
+#ifndef EOQ_H
+#define EOQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define EOQ_API __attribute__((visibility("default")))
+#else
+#define EOQ_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct eoq_handle_s *eoq_handle_t;
+
+typedef enum {
+    EOQ_OK = 0,
+    EOQ_ERR_BAD_ARG = 1,     /* null pointer, non-positive size, inconsistent geometry */
+    EOQ_ERR_ALIGNMENT = 2,   /* pointer not 16-byte aligned, channel count not a multiple of 16 */
+    EOQ_ERR_UNSUPPORTED = 3, /* geometry outside what the kernels cover */
+    EOQ_ERR_WORKSPACE = 4,   /* workspace missing, misaligned or too small */
+    EOQ_ERR_RANGE = 5,       /* a scalar code outside its range */
+    EOQ_ERR_CUDA = 6         /* a CUDA call failed; see eoq_last_cuda_error() */
+} eoq_status_t;
+
+/* Bits of the device status word returned by eoq_last_status(). */
+#define EOQ_DEV_TIMEOUT 1u   /* a bounded wait inside a kernel ran out; results of that call are invalid */
+#define EOQ_DEV_NONFINITE 2u /* eoq_quantize met a NaN or an infinity */
+#define EOQ_DEV_SQ_ZERO 4u   /* a scale quantizer saw an all-zero tensor (codes 0, exponent passed through) */
+#define EOQ_DEV_RANGE 8u     /* an input exponent outside the supported range */
+
+typedef enum { EOQ_Q = 0, EOQ_CQ = 1, EOQ_SQ = 2 } eoq_qmode_t;
+typedef enum { EOQ_ROUND_RNE = 0, EOQ_ROUND_STOCHASTIC = 1 } eoq_round_t;
+typedef enum { EOQ_PASS_FWD = 0, EOQ_PASS_DGRAD = 1, EOQ_PASS_WGRAD = 2 } eoq_pass_t;
+
+/* Geometry of one convolution: input [n,h,w,c_in], filter kh x kw, square stride and padding.
+ * Output spatial size is (h + 2 pad - kh) / stride + 1 by (w + 2 pad - kw) / stride + 1. */
+typedef struct {
+    int n, h, w, c_in, c_out, kh, kw, stride, pad;
+} eoq_conv_desc_t;
+
+/* Creates a handle on CUDA device `device` (makes it current).  Synchronises. */
+EOQ_API int eoq_create(eoq_handle_t *handle, int device);
+EOQ_API int eoq_destroy(eoq_handle_t handle);
+
+/* Bytes of workspace a pass needs for this geometry (a multiple of 256; may be 0). */
+EOQ_API int eoq_workspace_size(const eoq_conv_desc_t *desc, int pass, size_t *bytes);
+
+/*
+ * Forward chain of one layer (Sec. 3.2.1, first equation block):
+ *   x1 = x0 + Q_b(b1)         (zero halo: padding applies to x1)
+ *   x2 = Q_a1(conv(x1, Q_w(w)))  code = sat16(R(acc / 2^s)), s = -x_exp (7 when x_exp is NULL)
+ *   x3 = Q_gamma(gamma) * x2
+ *   x4 = x3 + Q_b(b2) [+ shortcut]
+ *   x5 = Q_a2(relu(x4))       code = sat(R(max(x4,0) / 2^7), -127, 127);  relu = 0 keeps x4's sign
+ * device in : x [n,h,w,c_in] int8; x_exp (int32, exponent of x; NULL means -7); w; shortcut
+ *             [n,ho,wo,c_out] int8 at p = -7 or NULL.
+ * host in   : b1_c, gamma_c, b2_c integer codes at p = -7 (gamma = 1 is 128), each within int16.
+ * device out: x5 [n,ho,wo,c_out] int8; optional x2 (int16, same shape), relu_mask (bit i of the
+ *             NHWC-linear element index i in byte i/8, bit i%8: [x4 > 0]) and acc_dump (int32 conv
+ *             accumulators including the b1 term) -- each may be NULL.
+ * Errors: BAD_ARG, ALIGNMENT, UNSUPPORTED (kh*kw > 64 taps), RANGE, WORKSPACE, CUDA.
+ */
+EOQ_API int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *x, const int32_t *x_exp,
+                 int32_t b1_c, const int8_t *w, int32_t gamma_c, int32_t b2_c, const int8_t *shortcut, int relu,
+                 int8_t *x5, int16_t *x2, uint8_t *relu_mask, int32_t *acc_dump, void *workspace,
+                 size_t workspace_bytes, void *stream);
+
+/*
+ * Error back-propagation through the convolution (Sec. 3.2.1, second equation block):
+ *   e4 = Q_e(e3 * Q_w(w)), the transposed convolution followed by SQ over the whole tensor.
+ * device in : e3 [n,ho,wo,c_out] int8 with exponent *e3_exp; w.
+ * device out: e4 [n,h,w,c_in] int8; *e4_exp = *e3_exp - 7 + t - 7 with 2^t the scale of SQ;
+ *             optional sum_e4 (int64: sum of the e4 codes, the argument of g_b1 = Q_g(e4)) and
+ *             acc_dump (int32 accumulators [n,h,w,c_in]).
+ */
+EOQ_API int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                   const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4, int32_t *acc_dump,
+                   void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Weight gradient (Sec. 3.2.1, third equation block): g_w = Q_g(e3 * x1), the correlation of the
+ * error with x1 = x0 + Q_b(b1) (zero halo), summed exactly over batch and space, followed by SQ.
+ * device in : e3 and *e3_exp as above; x = x0 [n,h,w,c_in] int8.   host in: b1_c.
+ * device out: g [c_out,kh,kw,c_in] int8; *g_exp; optional acc_dump (int64, same shape as g).
+ */
+EOQ_API int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                   const int8_t *x, int32_t b1_c, int8_t *g, int32_t *g_exp, int64_t *acc_dump,
+                   void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The three quantization functions (Sec. 3.2.2) on a flat tensor of n elements.
+ *   src_is_float = 1: src is fp32.  Q -> int16 codes R(x * 2^7) (saturated to int16);
+ *                     CQ -> int8 codes in [-127,127]; SQ -> int8 codes and *dst_exp.
+ *   src_is_float = 0: src is int32 codes with exponent *src_exp (device); only SQ is defined:
+ *                     int8 codes and *dst_exp = *src_exp + t - 7.
+ * dst_exp may be NULL for Q and CQ.  Uses no workspace (pass NULL, 0).
+ */
+EOQ_API int eoq_quantize(eoq_handle_t handle, int mode, const void *src, int src_is_float, const int32_t *src_exp,
+                 size_t n, void *dst, int32_t *dst_exp, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Head of the error chain (Sec. 3.2.1): e1 = e0 * [x4 > 0], e2 = e1, e3 = Q_e(e2 * Q_gamma(gamma)),
+ * with the sums behind g_b2 = Q_g(sum e1) and g_gamma = Q_g(sum e2 * x2).
+ * device in : e0 (int8, n_el elements) with exponent *e0_exp; relu_mask as written by eoq_conv_fwd
+ *             (NULL = all ones); x2 int16 or NULL.   host in: gamma_c.
+ * device out: e3 int8, *e3_exp = *e0_exp - 7 + t - 7; optional sum_e1, sum_e1x2 (int64).
+ * n_el must be a multiple of 16.
+ */
+EOQ_API int eoq_err_prescale(eoq_handle_t handle, const int8_t *e0, const int32_t *e0_exp, const uint8_t *relu_mask,
+                     const int16_t *x2, size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp,
+                     int64_t *sum_e1, int64_t *sum_e1x2, void *stream);
+
+/*
+ * The 8-bit update (Sec. 3.2.3, update quantization) on `num` weight tensors in one call:
+ *   u = Q_u(lr * g) = SQ(lr * g, 8), lr = lr_mant * 2^lr_exp, lr_mant in [1, 255];
+ *   w <- Q_w(w - u): code = sat(R((w - u) * 2^7), -127, 127), in place on the int8 codes.
+ * host in   : arrays (host memory, num entries) of device pointers w[i], g[i], g_exp[i] and sizes n[i].
+ * EOQ_ROUND_STOCHASTIC (an extension, not in the paper) replaces R by floor((v + r) / 2^s) with r
+ * drawn from a counter hash of (seed, step, tensor index, element index).  num <= 256 per call.
+ */
+EOQ_API int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const int8_t *const *g,
+               const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp, int round_mode,
+               uint64_t seed, uint64_t step, void *stream);
+
+/* int8 layout change between NCHW and NHWC ([n,c,h,w] <-> [n,h,w,c]); to_nhwc = 1 reads NCHW. */
+EOQ_API int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t *dst, int n, int c, int h, int w,
+                       int to_nhwc, void *stream);
+
+/* Synchronises `stream`, returns the OR of the EOQ_DEV_* bits raised since the last call, clears them. */
+EOQ_API int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits);
+
+/* The last cudaError_t a call on this handle recorded (0 if none). */
+EOQ_API int eoq_last_cuda_error(eoq_handle_t handle);
+
+EOQ_API const char *eoq_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EOQ_H */

@@ -1,0 +1,596 @@
+// C ABI of libeoq: argument checks, TMA descriptors, launch plans.  Declarations and their contract: eoq.h.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <string.h>
+
+#include <new>
+
+#include "eoq_internal.h"
+
+using namespace eoq;
+
+namespace {
+
+// --------------------------------------------------------------------------------- driver entry points
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const int *, const int *, cuuint32_t, cuuint32_t,
+                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn g_encode_tiled = nullptr;
+EncodeIm2colFn g_encode_im2col = nullptr;
+
+bool load_driver_entry_points()
+{
+    if (g_encode_tiled && g_encode_im2col) return true;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return false;
+    g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return false;
+    g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(fn);
+    return true;
+}
+
+CUtensorMapSwizzle swizzle_for(int row_bytes)
+{
+    switch (row_bytes) {
+        case 128: return CU_TENSOR_MAP_SWIZZLE_128B;
+        case 64: return CU_TENSOR_MAP_SWIZZLE_64B;
+        case 32: return CU_TENSOR_MAP_SWIZZLE_32B;
+        default: return CU_TENSOR_MAP_SWIZZLE_NONE;
+    }
+}
+
+// Widest of 128/64/32/16 channel bytes that divides c (c is a multiple of 16).
+int chunk_bytes(int c)
+{
+    for (int k = 128; k > 16; k >>= 1)
+        if (c % k == 0) return k;
+    return 16;
+}
+
+// im2col view of an NHWC int8 tensor [n][h][w][c]: `pixels` consecutive positions of the walk that starts at
+// (lower_w, lower_h) and advances by `stride`, `box_c` channels each.  count_w/h = positions per row/column.
+bool make_im2col_map(CUtensorMap *map, const void *ptr, int n, int h, int w, int c, int lower_w, int lower_h,
+                     int count_w, int count_h, int stride, int box_c, int pixels)
+{
+    cuuint64_t dims[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
+    cuuint64_t strides[3] = {(cuuint64_t)c, (cuuint64_t)c * w, (cuuint64_t)c * w * h};
+    int lower[2] = {lower_w, lower_h};
+    // the walk covers count positions: (extent + upper - lower - 1) / stride + 1 = count
+    int upper[2] = {(count_w - 1) * stride + 1 + lower_w - w, (count_h - 1) * stride + 1 + lower_h - h};
+    for (int i = 0; i < 2; ++i)
+        if (lower[i] < -128 || lower[i] > 127 || upper[i] < -128 || upper[i] > 127) return false;
+    cuuint32_t estr[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
+    return g_encode_im2col(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(ptr), dims, strides, lower, upper,
+                           (cuuint32_t)box_c, (cuuint32_t)pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           swizzle_for(box_c), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tiled view of a [rows][taps][c] int8 tensor with a (box_c, 1, box_rows) box.
+bool make_weight_map(CUtensorMap *map, const void *ptr, int rows, int taps, int c, int box_c, int box_rows)
+{
+    cuuint64_t dims[3] = {(cuuint64_t)c, (cuuint64_t)taps, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)c, (cuuint64_t)c * taps};
+    cuuint32_t box[3] = {(cuuint32_t)box_c, 1, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(box_c), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tiled view of a [rows][c] int8 matrix with a (box_c, box_rows) box.
+bool make_matrix_map(CUtensorMap *map, const void *ptr, size_t rows, int c, int box_c, int box_rows)
+{
+    cuuint64_t dims[2] = {(cuuint64_t)c, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)c};
+    cuuint32_t box[2] = {(cuuint32_t)box_c, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(box_c), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// --------------------------------------------------------------------------------- checks and geometry
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+inline size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+struct Geometry {
+    int ho, wo, taps;
+    size_t in_elems, out_elems, w_elems;
+};
+
+int check_desc(const eoq_conv_desc_t *d, Geometry *g)
+{
+    if (!d) return EOQ_ERR_BAD_ARG;
+    if (d->n <= 0 || d->h <= 0 || d->w <= 0 || d->c_in <= 0 || d->c_out <= 0 || d->kh <= 0 || d->kw <= 0 ||
+        d->stride <= 0 || d->pad < 0)
+        return EOQ_ERR_BAD_ARG;
+    if (d->h + 2 * d->pad < d->kh || d->w + 2 * d->pad < d->kw) return EOQ_ERR_BAD_ARG;
+    if (d->c_in % 16 || d->c_out % 16) return EOQ_ERR_ALIGNMENT;
+    if (d->kh * d->kw > kMaxTaps || d->kh > 16 || d->kw > 16 || d->stride > 8 || d->pad > 64) return EOQ_ERR_UNSUPPORTED;
+    g->ho = (d->h + 2 * d->pad - d->kh) / d->stride + 1;
+    g->wo = (d->w + 2 * d->pad - d->kw) / d->stride + 1;
+    g->taps = d->kh * d->kw;
+    g->in_elems = (size_t)d->n * d->h * d->w * d->c_in;
+    g->out_elems = (size_t)d->n * g->ho * g->wo * d->c_out;
+    g->w_elems = (size_t)d->c_out * g->taps * d->c_in;
+    if ((size_t)d->n * d->h * d->w >= (1u << 31) || (size_t)d->n * g->ho * g->wo >= (1u << 31)) return EOQ_ERR_UNSUPPORTED;
+    return EOQ_OK;
+}
+
+// Rows (or columns) whose filter window leaves the image at the low / high end.
+void border_counts(int extent_in, int extent_out, int k, int stride, int pad, int *nlo, int *nhi, int *ncls)
+{
+    int lo = 0, hi = 0;
+    for (int y = 0; y < extent_out; ++y) {
+        if (y * stride - pad < 0) ++lo;
+        if (y * stride - pad + k - 1 > extent_in - 1) ++hi;
+    }
+    *nlo = lo;
+    *nhi = hi;
+    *ncls = (lo + hi + 1 >= extent_out) ? extent_out : lo + hi + 1;
+}
+
+BorderClasses border_classes(const eoq_conv_desc_t &d, const Geometry &g)
+{
+    BorderClasses bc;
+    border_counts(d.h, g.ho, d.kh, d.stride, d.pad, &bc.nlo_h, &bc.nhi_h, &bc.nrc);
+    border_counts(d.w, g.wo, d.kw, d.stride, d.pad, &bc.nlo_w, &bc.nhi_w, &bc.ncc);
+    return bc;
+}
+
+int record(Handle *h, cudaError_t e)
+{
+    if (e == cudaSuccess) return EOQ_OK;
+    h->last_cuda_error = (int)e;
+    return EOQ_ERR_CUDA;
+}
+
+// Shared tiling choices of the implicit GEMM: K sub-tiles, pipeline depth, column tile.
+void plan_igemm(IgemmParams &p, int src_channels, int ntaps, int sm_count)
+{
+    p.kc = chunk_bytes(src_channels);
+    p.chunks_per_tap = src_channels / p.kc;
+    p.ntaps = ntaps;
+    p.real_sub = ntaps * p.chunks_per_tap;
+    p.num_sub = (p.kc == 16 && (p.real_sub & 1)) ? p.real_sub + 1 : p.real_sub;
+    p.subs_per_stage = 128 / p.kc;
+    if (p.subs_per_stage > p.num_sub) p.subs_per_stage = p.num_sub;
+    p.num_m_tiles = (p.M + kTileM - 1) / kTileM;
+    // widest column tile that still gives every SM a tile; narrow ones only when the grid would starve
+    int tn = p.N < 256 ? p.N : 256;
+    while (tn > 64 && tn % 32 == 0 && (long long)p.num_m_tiles * ((p.N + tn - 1) / tn) < sm_count) tn /= 2;
+    p.tile_n = tn;
+    p.num_n_tiles = (p.N + tn - 1) / tn;
+    const size_t stage = (size_t)p.subs_per_stage * (kTileM + tn) * p.kc;
+    int stages = (int)((200 * 1024) / stage);
+    p.num_stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
+}
+
+}  // namespace
+
+// ================================================================================= handle
+
+extern "C" int eoq_create(eoq_handle_t *handle, int device)
+{
+    if (!handle) return EOQ_ERR_BAD_ARG;
+    *handle = nullptr;
+    if (cudaSetDevice(device) != cudaSuccess) return EOQ_ERR_CUDA;
+    if (!load_driver_entry_points()) return EOQ_ERR_CUDA;
+    Handle *h = new (std::nothrow) Handle();
+    if (!h) return EOQ_ERR_BAD_ARG;
+    h->device = device;
+    h->last_cuda_error = 0;
+    h->dev = nullptr;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, device);
+    if (e == cudaSuccess) {
+        h->sm_count = prop.multiProcessorCount;
+        if (prop.major != 10) {
+            delete h;
+            return EOQ_ERR_UNSUPPORTED;  // the kernels are sm_100a only
+        }
+        e = cudaMalloc(reinterpret_cast<void **>(&h->dev), sizeof(DeviceState));
+    }
+    if (e == cudaSuccess) e = cudaMemset(h->dev, 0, sizeof(DeviceState));
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        if (h->dev) cudaFree(h->dev);
+        delete h;
+        return EOQ_ERR_CUDA;
+    }
+    *handle = reinterpret_cast<eoq_handle_t>(h);
+    return EOQ_OK;
+}
+
+extern "C" int eoq_destroy(eoq_handle_t handle)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h) return EOQ_ERR_BAD_ARG;
+    cudaSetDevice(h->device);
+    cudaDeviceSynchronize();
+    if (h->dev) cudaFree(h->dev);
+    delete h;
+    return EOQ_OK;
+}
+
+extern "C" int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !bits) return EOQ_ERR_BAD_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    unsigned v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, &h->dev->status, sizeof(unsigned), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(&h->dev->status, 0, sizeof(unsigned), s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    *bits = v;
+    return record(h, e);
+}
+
+extern "C" int eoq_last_cuda_error(eoq_handle_t handle)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    return h ? h->last_cuda_error : 0;
+}
+
+extern "C" const char *eoq_status_string(int status)
+{
+    switch (status) {
+        case EOQ_OK: return "ok";
+        case EOQ_ERR_BAD_ARG: return "bad argument";
+        case EOQ_ERR_ALIGNMENT: return "alignment (16-byte pointers, channels in multiples of 16)";
+        case EOQ_ERR_UNSUPPORTED: return "unsupported geometry or device";
+        case EOQ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case EOQ_ERR_RANGE: return "scalar code out of range";
+        case EOQ_ERR_CUDA: return "CUDA error";
+        default: return "unknown status";
+    }
+}
+
+// ================================================================================= workspace
+
+extern "C" int eoq_workspace_size(const eoq_conv_desc_t *desc, int pass, size_t *bytes)
+{
+    Geometry g;
+    if (!bytes) return EOQ_ERR_BAD_ARG;
+    int st = check_desc(desc, &g);
+    if (st != EOQ_OK) return st;
+    const BorderClasses bc = border_classes(*desc, g);
+    switch (pass) {
+        case EOQ_PASS_FWD:  // b1 table
+            *bytes = round256((size_t)bc.nrc * bc.ncc * desc->c_out * sizeof(int32_t));
+            return EOQ_OK;
+        case EOQ_PASS_DGRAD:  // transposed weights + int32 sums
+            *bytes = round256(g.w_elems) + round256(g.in_elems * sizeof(int32_t));
+            return EOQ_OK;
+        case EOQ_PASS_WGRAD:  // int64 sums + per-tap error sums
+            *bytes = round256(g.w_elems * sizeof(long long)) + round256((size_t)desc->c_out * g.taps * sizeof(long long));
+            return EOQ_OK;
+        default: return EOQ_ERR_BAD_ARG;
+    }
+}
+
+static int check_workspace(const eoq_conv_desc_t *desc, int pass, const void *ws, size_t ws_bytes)
+{
+    size_t need = 0;
+    int st = eoq_workspace_size(desc, pass, &need);
+    if (st != EOQ_OK) return st;
+    if (need == 0) return EOQ_OK;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) || ws_bytes < need) return EOQ_ERR_WORKSPACE;
+    return EOQ_OK;
+}
+
+// ================================================================================= forward
+
+extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *x, const int32_t *x_exp,
+                            int32_t b1_c, const int8_t *w, int32_t gamma_c, int32_t b2_c, const int8_t *shortcut,
+                            int relu, int8_t *x5, int16_t *x2, uint8_t *relu_mask, int32_t *acc_dump, void *workspace,
+                            size_t workspace_bytes, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    Geometry g;
+    if (!h || !x || !w || !x5) return EOQ_ERR_BAD_ARG;
+    int st = check_desc(desc, &g);
+    if (st != EOQ_OK) return st;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(x5) || !aligned16(shortcut) || !aligned16(x2) ||
+        !aligned16(relu_mask) || !aligned16(acc_dump))
+        return EOQ_ERR_ALIGNMENT;
+    if (b1_c < -32768 || b1_c > 32767 || gamma_c < -32768 || gamma_c > 32767 || b2_c < -32768 || b2_c > 32767)
+        return EOQ_ERR_RANGE;
+    const eoq_conv_desc_t &d = *desc;
+    // the accumulator with its b1 term must fit int32: taps * c_in * (127 + |b1|) * 127 < 2^31
+    if ((double)g.taps * d.c_in * (127.0 + (b1_c < 0 ? -b1_c : b1_c)) * 127.0 >= 2147483647.0) return EOQ_ERR_RANGE;
+    if (b1_c != 0 && (st = check_workspace(desc, EOQ_PASS_FWD, workspace, workspace_bytes)) != EOQ_OK) return st;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+    IgemmParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = d.n * g.ho * g.wo;
+    p.N = d.c_out;
+    p.hq = g.ho;
+    p.wq = g.wo;
+    plan_igemm(p, d.c_in, g.taps, h->sm_count);
+    p.src_stride = d.stride;
+    p.base_h = -d.pad;
+    p.base_w = -d.pad;
+    for (int t = 0; t < g.taps; ++t) {
+        p.tap_dh[t] = (unsigned char)(t / d.kw);
+        p.tap_dw[t] = (unsigned char)(t % d.kw);
+        p.tap_b[t] = (unsigned char)t;
+    }
+    p.out_h = g.ho;
+    p.out_w = g.wo;
+    p.out_step = 1;
+    p.epilogue = kEpiForward;
+    p.x_exp = x_exp;
+    p.b1_c = b1_c;
+    p.gamma_c = gamma_c;
+    p.b2_c = b2_c;
+    p.shortcut = shortcut;
+    p.relu = relu ? 1 : 0;
+    p.x5 = x5;
+    p.x2 = x2;
+    p.relu_mask = relu_mask;
+    p.acc_out = acc_dump;
+    p.dev = h->dev;
+    if (b1_c != 0) {
+        const BorderClasses bc = border_classes(d, g);
+        p.b1_table = reinterpret_cast<const int32_t *>(workspace);
+        p.b1_nlo_h = bc.nlo_h; p.b1_nhi_h = bc.nhi_h; p.b1_nrc = bc.nrc;
+        p.b1_nlo_w = bc.nlo_w; p.b1_nhi_w = bc.nhi_w; p.b1_ncc = bc.ncc;
+        cudaError_t e = launch_b1_weight_table(w, reinterpret_cast<int32_t *>(workspace), d, bc, s);
+        if (e != cudaSuccess) return record(h, e);
+    }
+    CUtensorMap map_a, map_b;
+    if (!make_im2col_map(&map_a, x, d.n, d.h, d.w, d.c_in, -d.pad, -d.pad, g.wo, g.ho, d.stride, p.kc, kTileM) ||
+        !make_weight_map(&map_b, w, d.c_out, g.taps, d.c_in, p.kc, p.tile_n))
+        return EOQ_ERR_UNSUPPORTED;
+    const int tiles = p.num_m_tiles * p.num_n_tiles;
+    return record(h, launch_igemm(p, map_a, map_b, tiles < h->sm_count ? tiles : h->sm_count, s));
+}
+
+// ================================================================================= error back-propagation
+
+extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3,
+                              const int32_t *e3_exp, const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4,
+                              int32_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    Geometry g;
+    if (!h || !e3 || !e3_exp || !w || !e4 || !e4_exp) return EOQ_ERR_BAD_ARG;
+    int st = check_desc(desc, &g);
+    if (st != EOQ_OK) return st;
+    if (!aligned16(e3) || !aligned16(w) || !aligned16(e4) || !aligned16(acc_dump)) return EOQ_ERR_ALIGNMENT;
+    if ((st = check_workspace(desc, EOQ_PASS_DGRAD, workspace, workspace_bytes)) != EOQ_OK) return st;
+    const eoq_conv_desc_t &d = *desc;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+    int8_t *wt = reinterpret_cast<int8_t *>(workspace);
+    int32_t *sums = acc_dump ? acc_dump : reinterpret_cast<int32_t *>(reinterpret_cast<char *>(workspace) + round256(g.w_elems));
+    cudaError_t e = launch_reset_cells(h->dev, s);
+    if (e == cudaSuccess) e = launch_weight_transpose(w, wt, d.c_out, g.taps, d.c_in, s);
+    if (e != cudaSuccess) return record(h, e);
+
+    // One GEMM per residue class (y mod stride, x mod stride) of the input pixels: within a class the taps
+    // kh with (y + pad - kh) divisible by the stride form a unit-stride correlation over e3.
+    bool cleared = false;
+    for (int py = 0; py < d.stride && py < d.h; ++py)
+        for (int px = 0; px < d.stride && px < d.w; ++px) {
+            IgemmParams p;
+            memset(&p, 0, sizeof(p));
+            int dh[16], dw[16], kh_of[16], kw_of[16], nh = 0, nw = 0, min_h = 0, min_w = 0;
+            for (int kh = 0; kh < d.kh; ++kh)
+                if ((py + d.pad - kh) % d.stride == 0) {
+                    // floor division is exact here; negative quotients are rows above the image
+                    dh[nh] = (py + d.pad - kh) / d.stride;
+                    kh_of[nh] = kh;
+                    if (dh[nh] < min_h) min_h = dh[nh];
+                    ++nh;
+                }
+            for (int kw = 0; kw < d.kw; ++kw)
+                if ((px + d.pad - kw) % d.stride == 0) {
+                    dw[nw] = (px + d.pad - kw) / d.stride;
+                    kw_of[nw] = kw;
+                    if (dw[nw] < min_w) min_w = dw[nw];
+                    ++nw;
+                }
+            const int hq = (d.h - py + d.stride - 1) / d.stride, wq = (d.w - px + d.stride - 1) / d.stride;
+            if (nh == 0 || nw == 0) {
+                // no tap reaches this class: its sums are zero
+                if (!cleared) {
+                    e = cudaMemsetAsync(sums, 0, g.in_elems * sizeof(int32_t), s);
+                    if (e != cudaSuccess) return record(h, e);
+                    cleared = true;
+                }
+                continue;
+            }
+            p.M = d.n * hq * wq;
+            p.N = d.c_in;
+            p.hq = hq;
+            p.wq = wq;
+            plan_igemm(p, d.c_out, nh * nw, h->sm_count);
+            p.src_stride = 1;
+            p.base_h = min_h;
+            p.base_w = min_w;
+            for (int a = 0; a < nh; ++a)
+                for (int b = 0; b < nw; ++b) {
+                    const int t = a * nw + b;
+                    if (dh[a] - min_h > 255 || dw[b] - min_w > 255) return EOQ_ERR_UNSUPPORTED;
+                    p.tap_dh[t] = (unsigned char)(dh[a] - min_h);
+                    p.tap_dw[t] = (unsigned char)(dw[b] - min_w);
+                    p.tap_b[t] = (unsigned char)(kh_of[a] * d.kw + kw_of[b]);
+                }
+            p.out_h = d.h;
+            p.out_w = d.w;
+            p.out_step = d.stride;
+            p.out_off_h = py;
+            p.out_off_w = px;
+            p.epilogue = kEpiDgrad;
+            p.acc_out = sums;
+            p.dev = h->dev;
+            CUtensorMap map_a, map_b;
+            if (!make_im2col_map(&map_a, e3, d.n, g.ho, g.wo, d.c_out, min_w, min_h, wq, hq, 1, p.kc, kTileM) ||
+                !make_weight_map(&map_b, wt, d.c_in, g.taps, d.c_out, p.kc, p.tile_n))
+                return EOQ_ERR_UNSUPPORTED;
+            const int tiles = p.num_m_tiles * p.num_n_tiles;
+            e = launch_igemm(p, map_a, map_b, tiles < h->sm_count ? tiles : h->sm_count, s);
+            if (e != cudaSuccess) return record(h, e);
+        }
+    // Q_e over the whole tensor: the maximum is complete only now
+    e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
+                      h->sm_count, s);
+    return record(h, e);
+}
+
+// ================================================================================= weight gradient
+
+extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3,
+                              const int32_t *e3_exp, const int8_t *x, int32_t b1_c, int8_t *gq, int32_t *g_exp,
+                              int64_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    Geometry g;
+    if (!h || !e3 || !e3_exp || !x || !gq || !g_exp) return EOQ_ERR_BAD_ARG;
+    int st = check_desc(desc, &g);
+    if (st != EOQ_OK) return st;
+    if (!aligned16(e3) || !aligned16(x) || !aligned16(gq) || !aligned16(acc_dump)) return EOQ_ERR_ALIGNMENT;
+    if (b1_c < -32768 || b1_c > 32767) return EOQ_ERR_RANGE;
+    if ((st = check_workspace(desc, EOQ_PASS_WGRAD, workspace, workspace_bytes)) != EOQ_OK) return st;
+    const eoq_conv_desc_t &d = *desc;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+    long long *acc = reinterpret_cast<long long *>(workspace);
+    long long *tap_sums = reinterpret_cast<long long *>(reinterpret_cast<char *>(workspace) + round256(g.w_elems * sizeof(long long)));
+
+    WgradParams p;
+    memset(&p, 0, sizeof(p));
+    p.P = d.n * g.ho * g.wo;
+    p.ho = g.ho;
+    p.wo = g.wo;
+    p.c_in = d.c_in;
+    p.c_out = d.c_out;
+    p.ntaps = g.taps;
+    p.kc = chunk_bytes(d.c_in);
+    p.nc = chunk_bytes(d.c_out);
+    p.chunks_per_tap = d.c_in / p.kc;
+    p.rows_total = g.taps * d.c_in;
+    p.subs_per_mtile = kTileM / p.kc;
+    p.num_m_tiles = (p.rows_total + kTileM - 1) / kTileM;
+    p.tile_n = d.c_out < 256 ? d.c_out : 256;
+    if (p.tile_n % p.nc) p.tile_n = (p.tile_n / p.nc) * p.nc;
+    p.num_n_tiles = (d.c_out + p.tile_n - 1) / p.tile_n;
+    p.pixels_per_stage = 64;
+    const int total_stages = (p.P + p.pixels_per_stage - 1) / p.pixels_per_stage;
+    // a 64-pixel stage adds at most 64 * 127 * 255 to an int32 partial sum: cap the stages one CTA runs
+    const int max_stages_exact = 1024;
+    const int tiles = p.num_m_tiles * p.num_n_tiles;
+    int splits = (2 * h->sm_count + tiles - 1) / tiles;
+    const int max_splits = (total_stages + 7) / 8;  // at least 8 stages of work per CTA
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    int per = (total_stages + splits - 1) / splits;
+    if (per > max_stages_exact) per = max_stages_exact;
+    splits = (total_stages + per - 1) / per;
+    p.stages_per_split = per;
+    p.num_k_splits = splits;
+    const size_t stage_bytes = (size_t)p.subs_per_mtile * p.pixels_per_stage * p.kc + (size_t)p.tile_n * p.pixels_per_stage;
+    int stages = (int)((200 * 1024) / stage_bytes);
+    p.num_stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
+    p.src_stride = d.stride;
+    p.base_h = -d.pad;
+    p.base_w = -d.pad;
+    for (int t = 0; t < g.taps; ++t) {
+        p.tap_dh[t] = (unsigned char)(t / d.kw);
+        p.tap_dw[t] = (unsigned char)(t % d.kw);
+    }
+    p.acc = acc;
+    p.dev = h->dev;
+
+    cudaError_t e = cudaMemsetAsync(acc, 0, g.w_elems * sizeof(long long), s);
+    if (e == cudaSuccess && b1_c != 0) e = launch_b1_error_sums(e3, tap_sums, d, g.ho, g.wo, s);
+    if (e != cudaSuccess) return record(h, e);
+    CUtensorMap map_x, map_e;
+    if (!make_im2col_map(&map_x, x, d.n, d.h, d.w, d.c_in, -d.pad, -d.pad, g.wo, g.ho, d.stride, p.kc, p.pixels_per_stage) ||
+        !make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage))
+        return EOQ_ERR_UNSUPPORTED;
+    e = launch_wgrad(p, map_x, map_e, s);
+    if (e != cudaSuccess) return record(h, e);
+    // the kernel leaves sums as [oc][tap][ic], which is the layout of g
+    e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
+                      b1_c != 0 ? tap_sums : nullptr, b1_c, g.taps, d.c_in, h->dev, h->sm_count, s);
+    return record(h, e);
+}
+
+// ================================================================================= elementwise entry points
+
+extern "C" int eoq_quantize(eoq_handle_t handle, int mode, const void *src, int src_is_float, const int32_t *src_exp,
+                            size_t n, void *dst, int32_t *dst_exp, void *workspace, size_t workspace_bytes,
+                            void *stream)
+{
+    (void)workspace;
+    (void)workspace_bytes;
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !src || !dst || n == 0) return EOQ_ERR_BAD_ARG;
+    if (mode != EOQ_Q && mode != EOQ_CQ && mode != EOQ_SQ) return EOQ_ERR_BAD_ARG;
+    if (mode == EOQ_SQ && !dst_exp) return EOQ_ERR_BAD_ARG;
+    if (!aligned16(src) || !aligned16(dst)) return EOQ_ERR_ALIGNMENT;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (src_is_float)
+        return record(h, launch_quantize_f32(mode, reinterpret_cast<const float *>(src), n, dst, dst_exp, h->dev, h->sm_count, s));
+    if (mode != EOQ_SQ || !src_exp) return EOQ_ERR_UNSUPPORTED;
+    return record(h, launch_sq_i32(reinterpret_cast<const int32_t *>(src), src_exp, 0, n, reinterpret_cast<int8_t *>(dst),
+                                   dst_exp, nullptr, false, h->dev, h->sm_count, s));
+}
+
+extern "C" int eoq_err_prescale(eoq_handle_t handle, const int8_t *e0, const int32_t *e0_exp, const uint8_t *relu_mask,
+                                const int16_t *x2, size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp,
+                                int64_t *sum_e1, int64_t *sum_e1x2, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !e0 || !e0_exp || !e3 || !e3_exp || n_el == 0 || (n_el % 16)) return EOQ_ERR_BAD_ARG;
+    if (!aligned16(e0) || !aligned16(e3) || !aligned16(x2) || (reinterpret_cast<uintptr_t>(relu_mask) & 1)) return EOQ_ERR_ALIGNMENT;
+    if (gamma_c < -32768 || gamma_c > 32767) return EOQ_ERR_RANGE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    return record(h, launch_err_prescale(e0, e0_exp, relu_mask, x2, n_el, gamma_c, e3, e3_exp,
+                                         reinterpret_cast<long long *>(sum_e1), reinterpret_cast<long long *>(sum_e1x2),
+                                         h->dev, h->sm_count, s));
+}
+
+extern "C" int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const int8_t *const *g,
+                          const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp,
+                          int round_mode, uint64_t seed, uint64_t step, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || num <= 0 || !w || !g || !g_exp || !n) return EOQ_ERR_BAD_ARG;
+    if (num > 256) return EOQ_ERR_UNSUPPORTED;
+    if (lr_mant < 1 || lr_mant > 255 || lr_exp < -64 || lr_exp > 64) return EOQ_ERR_RANGE;
+    if (round_mode != EOQ_ROUND_RNE && round_mode != EOQ_ROUND_STOCHASTIC) return EOQ_ERR_BAD_ARG;
+    UpdateTensor t[256];
+    for (int i = 0; i < num; ++i) {
+        if (!w[i] || !g[i] || !g_exp[i] || n[i] == 0) return EOQ_ERR_BAD_ARG;
+        t[i].w = w[i];
+        t[i].g = g[i];
+        t[i].g_exp = g_exp[i];
+        t[i].n = n[i];
+    }
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    return record(h, launch_update(t, num, lr_mant, lr_exp, round_mode == EOQ_ROUND_STOCHASTIC, seed, step, h->dev, h->sm_count, s));
+}
+
+extern "C" int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t *dst, int n, int c, int hh, int ww,
+                                  int to_nhwc, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !src || !dst || n <= 0 || c <= 0 || hh <= 0 || ww <= 0 || n > 65535) return EOQ_ERR_BAD_ARG;
+    return record(h, launch_layout_convert(src, dst, n, c, hh, ww, to_nhwc, reinterpret_cast<cudaStream_t>(stream)));
+}

@@ -1,0 +1,656 @@
+// Bandwidth-bound kernels of the EOQ layer (arXiv 2105.13890): the standalone quantizers Q / CQ / SQ
+// (Sec. 3.2.2), the second phase of the scale quantizer after a convolution, the head of the error
+// chain (Sec. 3.2.1), the 8-bit update (Sec. 3.2.3) and small layout helpers.
+// Reductions run warp-shuffle -> one atomic per warp; 16 elements per thread with 128-bit accesses.
+#include "eoq_device.cuh"
+#include "eoq_internal.h"
+
+namespace eoq {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d)
+{
+    return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) | ((uint32_t)(d & 0xff) << 24);
+}
+
+inline int grid_for(size_t work_items, int sm_count, int per_sm = 8)
+{
+    size_t blocks = (work_items + kThreads - 1) / kThreads;
+    size_t cap = (size_t)sm_count * per_sm;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+// ------------------------------------------------------------------ fp32 -> Q / CQ / SQ
+
+// R(log2 M) for a positive finite float given by its bit pattern.
+__device__ __forceinline__ int round_log2_f32bits(uint32_t bits)
+{
+    const int eb = (int)((bits >> 23) & 0xffu);
+    const uint32_t frac = bits & 0x7fffffu;
+    if (eb == 0) return round_log2_u32(frac) - 149;  // subnormal: frac * 2^-149
+    const unsigned long long m = (1ull << 23) | frac;  // M = m * 2^(eb - 150), m in [2^23, 2^24)
+    return (eb - 127) + ((m * m >= (1ull << 47)) ? 1 : 0);
+}
+
+__global__ void absmax_f32_kernel(const float *__restrict__ src, size_t n, DeviceState *dev)
+{
+    uint32_t mx = 0;
+    bool bad = false;
+    const size_t n4 = n / 4;
+    const float4 *s4 = reinterpret_cast<const float4 *>(src);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 v = __ldg(s4 + i);
+        uint32_t b[4] = {__float_as_uint(v.x), __float_as_uint(v.y), __float_as_uint(v.z), __float_as_uint(v.w)};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            uint32_t a = b[k] & 0x7fffffffu;
+            bad |= a >= 0x7f800000u;
+            mx = max(mx, a);
+        }
+    }
+    for (size_t i = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        uint32_t a = __float_as_uint(src[i]) & 0x7fffffffu;
+        bad |= a >= 0x7f800000u;
+        mx = max(mx, a);
+    }
+    mx = warp_max_u32(mx);
+    bad = __any_sync(0xffffffffu, bad);
+    if ((threadIdx.x & 31) == 0) {
+        if (mx) atomicMax(&dev->absmax_u32, mx);
+        if (bad) atomicOr(&dev->status, EOQ_DEV_NONFINITE);
+    }
+}
+
+// mode 0: Q -> int16, mode 1: CQ -> int8, mode 2: SQ -> int8 under the already reduced maximum.
+__global__ void quantize_f32_kernel(int mode, const float *__restrict__ src, size_t n, void *dst, int32_t *dst_exp,
+                                    DeviceState *dev)
+{
+    int up = 7;  // codes = R(x * 2^up)
+    if (mode == 2) {
+        const uint32_t mbits = dev->absmax_u32;
+        if (mbits == 0 || mbits >= 0x7f800000u) {
+            up = 7;
+            if (blockIdx.x == 0 && threadIdx.x == 0) {
+                if (mbits == 0) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+                *dst_exp = -7;
+            }
+        } else {
+            const int t = round_log2_f32bits(mbits);
+            up = 7 - t;
+            if (blockIdx.x == 0 && threadIdx.x == 0) *dst_exp = t - 7;
+        }
+    } else if (dst_exp && blockIdx.x == 0 && threadIdx.x == 0) {
+        *dst_exp = -7;
+    }
+    const int lim = (mode == 0) ? 32767 : 127;
+    const int lo = (mode == 0) ? -32768 : -127;
+    auto code = [&](float x) -> int {
+        float y = scalbnf(x, up);  // exact: a power-of-two scaling of a value that stays far from overflow
+        if (!(fabsf(y) < 1.0e9f)) return (y > 0.f) ? lim : ((y < 0.f) ? lo : 0);
+        return clampi(__float2int_rn(y), lo, lim);
+    };
+    const size_t n16 = n / 16;
+    const float4 *s4 = reinterpret_cast<const float4 *>(src);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
+        int c[16];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float4 v = __ldg(s4 + i * 4 + k);
+            c[4 * k + 0] = code(v.x);
+            c[4 * k + 1] = code(v.y);
+            c[4 * k + 2] = code(v.z);
+            c[4 * k + 3] = code(v.w);
+        }
+        if (mode == 0) {
+            int4 *d = reinterpret_cast<int4 *>(dst) + i * 2;
+            d[0] = make_int4((c[0] & 0xffff) | (c[1] << 16), (c[2] & 0xffff) | (c[3] << 16),
+                             (c[4] & 0xffff) | (c[5] << 16), (c[6] & 0xffff) | (c[7] << 16));
+            d[1] = make_int4((c[8] & 0xffff) | (c[9] << 16), (c[10] & 0xffff) | (c[11] << 16),
+                             (c[12] & 0xffff) | (c[13] << 16), (c[14] & 0xffff) | (c[15] << 16));
+        } else {
+            reinterpret_cast<int4 *>(dst)[i] =
+                make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
+                          (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+        }
+    }
+    for (size_t i = n16 * 16 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = code(src[i]);
+        if (mode == 0) reinterpret_cast<int16_t *>(dst)[i] = (int16_t)c;
+        else reinterpret_cast<int8_t *>(dst)[i] = (int8_t)c;
+    }
+}
+
+// ------------------------------------------------------------------ int32 -> SQ (phase 2 of Q_e after dgrad)
+
+__global__ void absmax_i32_kernel(const int32_t *__restrict__ src, size_t n, DeviceState *dev)
+{
+    uint32_t mx = 0;
+    const size_t n4 = n / 4;
+    const int4 *s4 = reinterpret_cast<const int4 *>(src);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        int4 v = __ldg(s4 + i);
+        mx = max(max(mx, (uint32_t)abs(v.x)), max((uint32_t)abs(v.y), max((uint32_t)abs(v.z), (uint32_t)abs(v.w))));
+    }
+    for (size_t i = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        mx = max(mx, (uint32_t)abs(src[i]));
+    mx = warp_max_u32(mx);
+    if ((threadIdx.x & 31) == 0 && mx) atomicMax(&dev->absmax_u32, mx);
+}
+
+__global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *src_exp, int exp_bias, size_t n,
+                              int8_t *dst, int32_t *dst_exp, long long *sum_codes, DeviceState *dev)
+{
+    const uint32_t M = dev->absmax_u32;
+    const int t = M ? round_log2_u32(M) : 7;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const int p_in = (src_exp ? *src_exp : 0) + exp_bias;
+        *dst_exp = M ? p_in + t - 7 : p_in;
+        if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+    }
+    long long sum = 0;
+    const size_t n16 = n / 16;
+    const int4 *s4 = reinterpret_cast<const int4 *>(src);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
+        int c[16];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            int4 v = __ldcs(s4 + i * 4 + k);
+            c[4 * k + 0] = sq_code32(v.x, t);
+            c[4 * k + 1] = sq_code32(v.y, t);
+            c[4 * k + 2] = sq_code32(v.z, t);
+            c[4 * k + 3] = sq_code32(v.w, t);
+        }
+        int s = 0;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) s += c[k];
+        sum += s;
+        reinterpret_cast<int4 *>(dst)[i] =
+            make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
+                      (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+    }
+    for (size_t i = n16 * 16 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = sq_code32(src[i], t);
+        sum += c;
+        dst[i] = (int8_t)c;
+    }
+    if (sum_codes) {
+        sum = warp_sum_i64(sum);
+        if ((threadIdx.x & 31) == 0 && sum) atomicAdd(reinterpret_cast<unsigned long long *>(sum_codes), (unsigned long long)sum);
+    }
+}
+
+// ------------------------------------------------------------------ int64 -> SQ (Q_g after the weight gradient)
+
+// Adds the b1 term of x1 = x0 + b1 (b1 times the sum of the error over the pixels whose tap falls inside
+// the image), optionally copies the exact sums out, and reduces max |.|.
+__global__ void wgrad_fix_absmax_kernel(long long *acc, size_t n, const long long *tap_sums, int32_t b1_c, int taps,
+                                        int c_in, long long *copy_out, DeviceState *dev)
+{
+    unsigned long long mx = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        long long v = acc[i];
+        if (tap_sums) {
+            v += (long long)b1_c * tap_sums[i / c_in];  // index of (oc, tap)
+            acc[i] = v;
+        }
+        if (copy_out) copy_out[i] = v;
+        const unsigned long long a = (unsigned long long)(v < 0 ? -v : v);
+        mx = a > mx ? a : mx;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        unsigned long long other = __shfl_xor_sync(0xffffffffu, mx, o);
+        mx = other > mx ? other : mx;
+    }
+    if ((threadIdx.x & 31) == 0 && mx) atomicMax(&dev->absmax_u64, mx);
+    (void)taps;
+}
+
+__global__ void sq_i64_kernel(const long long *__restrict__ src, const int32_t *src_exp, int exp_bias, size_t n,
+                              int8_t *dst, int32_t *dst_exp, DeviceState *dev)
+{
+    const unsigned long long M = dev->absmax_u64;
+    const int t = M ? round_log2_u64(M) : 7;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const int p_in = (src_exp ? *src_exp : 0) + exp_bias;
+        *dst_exp = M ? p_in + t - 7 : p_in;
+        if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+    }
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = (int8_t)sq_code64(src[i], t);
+}
+
+// ------------------------------------------------------------------ head of the error chain
+
+__device__ __forceinline__ void unpack16(const int4 &v, int (&o)[16])
+{
+    const int8_t *b = reinterpret_cast<const int8_t *>(&v);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) o[k] = b[k];
+}
+
+// Pass 1: max |e1| and the sums behind g_b2 and g_gamma, with e1 = e0 * [x4 > 0].
+__global__ void prescale_reduce_kernel(const int8_t *__restrict__ e0, const uint8_t *__restrict__ mask,
+                                       const int16_t *__restrict__ x2, size_t n16, DeviceState *dev)
+{
+    uint32_t mx = 0;
+    long long s1 = 0, s2 = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
+        int e[16];
+        unpack16(__ldg(reinterpret_cast<const int4 *>(e0) + i), e);
+        const uint32_t m = mask ? (uint32_t) __ldg(reinterpret_cast<const uint16_t *>(mask) + i) : 0xffffu;
+        int a1 = 0, a2 = 0;
+        int xv[16];
+        if (x2) {
+            const int4 lo = __ldg(reinterpret_cast<const int4 *>(x2) + 2 * i);
+            const int4 hi = __ldg(reinterpret_cast<const int4 *>(x2) + 2 * i + 1);
+            const int16_t *pl = reinterpret_cast<const int16_t *>(&lo), *ph = reinterpret_cast<const int16_t *>(&hi);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { xv[k] = pl[k]; xv[8 + k] = ph[k]; }
+        }
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const int e1 = ((m >> k) & 1u) ? e[k] : 0;
+            mx = max(mx, (uint32_t)abs(e1));
+            a1 += e1;
+            if (x2) a2 += e1 * xv[k];  // |e1 * x2| < 2^22, 16 terms
+        }
+        s1 += a1;
+        s2 += a2;
+    }
+    mx = warp_max_u32(mx);
+    s1 = warp_sum_i64(s1);
+    s2 = warp_sum_i64(s2);
+    if ((threadIdx.x & 31) == 0) {
+        if (mx) atomicMax(&dev->absmax_u32, mx);
+        if (s1) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum0), (unsigned long long)s1);
+        if (s2) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum1), (unsigned long long)s2);
+    }
+}
+
+// Pass 2: e3 = Q_e(gamma * e1) under the reduced maximum.
+__global__ void prescale_apply_kernel(const int8_t *__restrict__ e0, const int32_t *e0_exp,
+                                      const uint8_t *__restrict__ mask, size_t n16, int32_t gamma_c, int8_t *e3,
+                                      int32_t *e3_exp, long long *sum_e1, long long *sum_e1x2, DeviceState *dev)
+{
+    const uint32_t M = dev->absmax_u32 * (uint32_t)abs(gamma_c);  // max |gamma * e1| < 2^7 * 2^15
+    const int t = M ? round_log2_u32(M) : 7;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const int p_in = *e0_exp - 7;
+        *e3_exp = M ? p_in + t - 7 : p_in;
+        if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+        if (sum_e1) *sum_e1 = dev->sum0;
+        if (sum_e1x2) *sum_e1x2 = dev->sum1;
+    }
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
+        int e[16], c[16];
+        unpack16(__ldg(reinterpret_cast<const int4 *>(e0) + i), e);
+        const uint32_t m = mask ? (uint32_t) __ldg(reinterpret_cast<const uint16_t *>(mask) + i) : 0xffffu;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) c[k] = ((m >> k) & 1u) ? sq_code32(gamma_c * e[k], t) : 0;
+        reinterpret_cast<int4 *>(e3)[i] =
+            make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
+                      (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+    }
+}
+
+// ------------------------------------------------------------------ 8-bit update
+
+constexpr int kUpdChunk = 64;           // tensors per launch
+constexpr int kUpdElemsPerBlock = 8192;  // elements one block covers
+
+struct UpdateBatch {
+    UpdateTensor t[kUpdChunk];
+    int first_block[kUpdChunk + 1];
+    int num;
+    int tensor_base;  // index of t[0] in the whole call (cell of its maximum, counter of the hash)
+};
+
+__device__ __forceinline__ int find_tensor(const UpdateBatch &b, int block)
+{
+    int k = 0;
+    while (k + 1 < b.num && block >= b.first_block[k + 1]) ++k;
+    return k;
+}
+
+__global__ void update_absmax_kernel(const __grid_constant__ UpdateBatch b, DeviceState *dev)
+{
+    const int k = find_tensor(b, blockIdx.x);
+    const UpdateTensor &T = b.t[k];
+    const size_t begin = (size_t)(blockIdx.x - b.first_block[k]) * kUpdElemsPerBlock;
+    const size_t end = min((size_t)T.n, begin + kUpdElemsPerBlock);
+    uint32_t mx = 0;
+    if (begin < end) {
+        // 16-byte path when the tensor base allows it (it always does for 16-byte aligned tensors)
+        const bool vec = (reinterpret_cast<uintptr_t>(T.g) & 15) == 0;
+        size_t i = begin + (size_t)threadIdx.x * 16;
+        if (vec) {
+            for (; i + 16 <= end; i += (size_t)blockDim.x * 16) {
+                int e[16];
+                unpack16(__ldg(reinterpret_cast<const int4 *>(T.g + i)), e);
+#pragma unroll
+                for (int q = 0; q < 16; ++q) mx = max(mx, (uint32_t)abs(e[q]));
+            }
+        }
+        // remaining elements of this block's range
+        const size_t tail = vec ? begin + ((end - begin) / 16) * 16 : begin;
+        for (size_t j = tail + threadIdx.x; j < end; j += blockDim.x) mx = max(mx, (uint32_t)abs((int)T.g[j]));
+    }
+    mx = warp_max_u32(mx);
+    if ((threadIdx.x & 31) == 0 && mx) atomicMax(&dev->tensor_absmax[b.tensor_base + k], mx);
+}
+
+// SplitMix64 output function (Steele, Lea, Flood 2014) as a counter hash.
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z)
+{
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// w <- Q_w(w - Q_u(lr * g)) on int8 codes (Sec. 3.2.3).
+__device__ __forceinline__ int update_one(int w, int g, int lr_mant, int t, int d, int stochastic,
+                                          unsigned long long key, unsigned long long idx)
+{
+    const int u = sq_code32(lr_mant * g, t);
+    long long next;
+    if (d >= 0) {
+        next = (long long)w - (long long)u * (1ll << min(d, 40));
+    } else if (-d > 40) {
+        next = w;
+    } else {
+        const int s = -d;
+        const long long v = (long long)w * (1ll << s) - u;
+        if (!stochastic) {
+            next = rne_shr64(v, s);
+        } else {
+            const unsigned long long r = mix64(key + 0x9E3779B97F4A7C15ull * (idx + 1)) & ((1ull << s) - 1ull);
+            next = (v + (long long)r) >> s;
+        }
+    }
+    return (int)(next < -127 ? -127 : (next > 127 ? 127 : next));
+}
+
+__global__ void update_apply_kernel(const __grid_constant__ UpdateBatch b, int32_t lr_mant, int32_t lr_exp,
+                                    int stochastic, unsigned long long seed, unsigned long long step,
+                                    DeviceState *dev)
+{
+    const int k = find_tensor(b, blockIdx.x);
+    const UpdateTensor &T = b.t[k];
+    const uint32_t M = dev->tensor_absmax[b.tensor_base + k] * (uint32_t)lr_mant;  // max |lr_mant * g| < 2^15
+    if (M == 0) {
+        if (threadIdx.x == 0 && blockIdx.x == b.first_block[k]) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+        return;  // u = 0: the weights keep their codes
+    }
+    const int t = round_log2_u32(M);
+    const int d = (__ldg(T.g_exp) + lr_exp + t - 7) + 7;  // exponent of u, relative to the weight grid 2^-7
+    unsigned long long key = 0;
+    if (stochastic) {
+        key = mix64(seed + 0x9E3779B97F4A7C15ull * (step + 1));
+        key = mix64(key + 0x9E3779B97F4A7C15ull * ((unsigned long long)(b.tensor_base + k) + 1));
+    }
+    const size_t begin = (size_t)(blockIdx.x - b.first_block[k]) * kUpdElemsPerBlock;
+    const size_t end = min((size_t)T.n, begin + kUpdElemsPerBlock);
+    if (begin >= end) return;
+    const bool vec = ((reinterpret_cast<uintptr_t>(T.g) | reinterpret_cast<uintptr_t>(T.w)) & 15) == 0;
+    if (vec) {
+        for (size_t i = begin + (size_t)threadIdx.x * 16; i + 16 <= end; i += (size_t)blockDim.x * 16) {
+            int gv[16], wv[16], c[16];
+            unpack16(__ldg(reinterpret_cast<const int4 *>(T.g + i)), gv);
+            unpack16(*reinterpret_cast<const int4 *>(T.w + i), wv);
+#pragma unroll
+            for (int q = 0; q < 16; ++q) c[q] = update_one(wv[q], gv[q], lr_mant, t, d, stochastic, key, i + q);
+            *reinterpret_cast<int4 *>(T.w + i) =
+                make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
+                          (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+        }
+    }
+    const size_t tail = vec ? begin + ((end - begin) / 16) * 16 : begin;
+    for (size_t j = tail + threadIdx.x; j < end; j += blockDim.x)
+        T.w[j] = (int8_t)update_one(T.w[j], T.g[j], lr_mant, t, d, stochastic, key, j);
+}
+
+// ------------------------------------------------------------------ layout helpers
+
+// [n][rows][cols] -> [n][cols][rows] on bytes, 32 x 32 tiles through shared memory.
+__global__ void transpose_bytes_kernel(const int8_t *__restrict__ src, int8_t *__restrict__ dst, int rows, int cols)
+{
+    __shared__ int8_t tile[32][33];
+    const size_t img = (size_t)blockIdx.z * rows * cols;
+    const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+        const int rr = r0 + r, cc = c0 + threadIdx.x;
+        if (rr < rows && cc < cols) tile[r][threadIdx.x] = src[img + (size_t)rr * cols + cc];
+    }
+    __syncthreads();
+    for (int c = threadIdx.y; c < 32; c += blockDim.y) {
+        const int cc = c0 + c, rr = r0 + threadIdx.x;
+        if (rr < rows && cc < cols) dst[img + (size_t)cc * rows + rr] = tile[threadIdx.x][c];
+    }
+}
+
+// w[oc][tap][ic] -> wt[ic][tap][oc]
+__global__ void weight_transpose_kernel(const int8_t *__restrict__ w, int8_t *__restrict__ wt, int c_out, int taps,
+                                        int c_in)
+{
+    const size_t total = (size_t)c_out * taps * c_in;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int oc = (int)(i % c_out);
+        const int tap = (int)((i / c_out) % taps);
+        const int ic = (int)(i / ((size_t)c_out * taps));
+        wt[i] = w[((size_t)oc * taps + tap) * c_in + ic];
+    }
+}
+
+// ------------------------------------------------------------------ b1 support
+
+// Is filter tap k inside the image for the rows of class `cls`?
+__device__ __forceinline__ bool tap_valid(int cls, int k, int extent_out, int extent_in, int nlo, int nhi, int ncls,
+                                          int stride, int pad)
+{
+    int y;
+    if (ncls == extent_out) y = cls;
+    else if (cls < nlo) y = cls;
+    else if (cls == nlo) y = nlo;
+    else y = extent_out - nhi + (cls - nlo - 1);
+    const int src = y * stride - pad + k;
+    return src >= 0 && src < extent_in;
+}
+
+// table[class][oc] = sum over the taps valid for the class, and over ic, of w[oc][tap][ic]  (the forward
+// pass adds b1 times this: conv(x0 + b1) = conv(x0) + b1 * conv(indicator of the image)).
+__global__ void b1_weight_table_kernel(const int8_t *__restrict__ w, int32_t *table, eoq_conv_desc_t d, int ho, int wo,
+                                       BorderClasses bc)
+{
+    const int oc = blockIdx.x * blockDim.x + threadIdx.x;
+    const int cls = blockIdx.y;
+    if (oc >= d.c_out) return;
+    const int rc = cls / bc.ncc, cc = cls % bc.ncc;
+    int32_t sum = 0;
+    for (int kh = 0; kh < d.kh; ++kh) {
+        if (!tap_valid(rc, kh, ho, d.h, bc.nlo_h, bc.nhi_h, bc.nrc, d.stride, d.pad)) continue;
+        for (int kw = 0; kw < d.kw; ++kw) {
+            if (!tap_valid(cc, kw, wo, d.w, bc.nlo_w, bc.nhi_w, bc.ncc, d.stride, d.pad)) continue;
+            const int8_t *p = w + (((size_t)oc * d.kh + kh) * d.kw + kw) * d.c_in;
+            for (int ic = 0; ic < d.c_in; ++ic) sum += p[ic];
+        }
+    }
+    table[(size_t)cls * d.c_out + oc] = sum;
+}
+
+// tap_sums[oc][tap] = sum of e3[n,y,x,oc] over the pixels whose tap falls inside the image (the weight
+// gradient adds b1 times this to every input channel).  One block per (tap, channel group).
+__global__ void b1_error_sums_kernel(const int8_t *__restrict__ e3, long long *tap_sums, eoq_conv_desc_t d, int ho, int wo)
+{
+    const int tap = blockIdx.y;
+    const int kh = tap / d.kw, kw = tap % d.kw;
+    const int oc = blockIdx.x * 32 + (threadIdx.x & 31);
+    const int lanes = blockDim.x >> 5, slot = threadIdx.x >> 5;
+    long long sum = 0;
+    if (oc < d.c_out) {
+        const size_t pixels = (size_t)d.n * ho * wo;
+        for (size_t p = (size_t)blockIdx.z * lanes + slot; p < pixels; p += (size_t)gridDim.z * lanes) {
+            const int x = (int)(p % wo), y = (int)((p / wo) % ho);
+            const int sy = y * d.stride - d.pad + kh, sx = x * d.stride - d.pad + kw;
+            if (sy >= 0 && sy < d.h && sx >= 0 && sx < d.w) sum += e3[p * d.c_out + oc];
+        }
+    }
+    __shared__ long long part[32][33];
+    part[slot][threadIdx.x & 31] = sum;
+    __syncthreads();
+    if (slot == 0 && oc < d.c_out) {
+        long long s = 0;
+        for (int k = 0; k < lanes; ++k) s += part[k][threadIdx.x & 31];
+        if (s) atomicAdd(reinterpret_cast<unsigned long long *>(tap_sums + (size_t)oc * (d.kh * d.kw) + tap), (unsigned long long)s);
+    }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ launchers
+
+cudaError_t launch_reset_cells(DeviceState *dev, cudaStream_t s)
+{
+    // every cell after the status word
+    return cudaMemsetAsync(reinterpret_cast<char *>(dev) + offsetof(DeviceState, absmax_u32), 0,
+                           offsetof(DeviceState, tensor_absmax) - offsetof(DeviceState, absmax_u32), s);
+}
+
+cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst, int32_t *dst_exp, DeviceState *dev,
+                                int sm_count, cudaStream_t s)
+{
+    if (mode == 2) {
+        cudaError_t e = launch_reset_cells(dev, s);
+        if (e != cudaSuccess) return e;
+        absmax_f32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
+    }
+    quantize_f32_kernel<<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(mode, src, n, dst, dst_exp, dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
+                          int32_t *dst_exp, long long *sum_codes, bool max_already_reduced, DeviceState *dev,
+                          int sm_count, cudaStream_t s)
+{
+    if (!max_already_reduced) {
+        cudaError_t e = launch_reset_cells(dev, s);
+        if (e != cudaSuccess) return e;
+        absmax_i32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
+    }
+    if (sum_codes) {
+        cudaError_t e = cudaMemsetAsync(sum_codes, 0, sizeof(long long), s);
+        if (e != cudaSuccess) return e;
+    }
+    sq_i32_kernel<<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes, dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
+                          int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int taps,
+                          int c_in, DeviceState *dev, int sm_count, cudaStream_t s)
+{
+    cudaError_t e = launch_reset_cells(dev, s);
+    if (e != cudaSuccess) return e;
+    wgrad_fix_absmax_kernel<<<grid_for(n, sm_count), kThreads, 0, s>>>(const_cast<long long *>(src), n, tap_sums, b1_c,
+                                                                       taps, c_in, copy_out, dev);
+    sq_i64_kernel<<<grid_for(n, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const uint8_t *mask, const int16_t *x2,
+                                size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
+                                long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s)
+{
+    cudaError_t e = launch_reset_cells(dev, s);
+    if (e != cudaSuccess) return e;
+    const size_t n16 = n_el / 16;
+    prescale_reduce_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, mask, x2, n16, dev);
+    prescale_apply_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, e0_exp, mask, n16, gamma_c, e3, e3_exp,
+                                                                       sum_e1, sum_e1x2, dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_update(const UpdateTensor *t, int num, int32_t lr_mant, int32_t lr_exp, int stochastic,
+                          uint64_t seed, uint64_t step, DeviceState *dev, int sm_count, cudaStream_t s)
+{
+    (void)sm_count;
+    cudaError_t e = cudaMemsetAsync(dev->tensor_absmax, 0, sizeof(unsigned) * 256, s);
+    if (e != cudaSuccess) return e;
+    for (int base = 0; base < num; base += kUpdChunk) {
+        UpdateBatch b;
+        b.num = num - base < kUpdChunk ? num - base : kUpdChunk;
+        b.tensor_base = base;
+        int blocks = 0;
+        for (int k = 0; k < b.num; ++k) {
+            b.t[k] = t[base + k];
+            b.first_block[k] = blocks;
+            blocks += (int)((t[base + k].n + kUpdElemsPerBlock - 1) / kUpdElemsPerBlock);
+        }
+        b.first_block[b.num] = blocks;
+        if (blocks == 0) continue;
+        update_absmax_kernel<<<blocks, kThreads, 0, s>>>(b, dev);
+    }
+    for (int base = 0; base < num; base += kUpdChunk) {
+        UpdateBatch b;
+        b.num = num - base < kUpdChunk ? num - base : kUpdChunk;
+        b.tensor_base = base;
+        int blocks = 0;
+        for (int k = 0; k < b.num; ++k) {
+            b.t[k] = t[base + k];
+            b.first_block[k] = blocks;
+            blocks += (int)((t[base + k].n + kUpdElemsPerBlock - 1) / kUpdElemsPerBlock);
+        }
+        b.first_block[b.num] = blocks;
+        if (blocks == 0) continue;
+        update_apply_kernel<<<blocks, kThreads, 0, s>>>(b, lr_mant, lr_exp, stochastic, seed, step, dev);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_layout_convert(const int8_t *src, int8_t *dst, int n, int c, int h, int w, int to_nhwc,
+                                  cudaStream_t s)
+{
+    // NCHW is [n][c][hw]; NHWC is [n][hw][c]
+    const int rows = to_nhwc ? c : h * w, cols = to_nhwc ? h * w : c;
+    dim3 grid((cols + 31) / 32, (rows + 31) / 32, n), block(32, 8);
+    transpose_bytes_kernel<<<grid, block, 0, s>>>(src, dst, rows, cols);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_weight_transpose(const int8_t *w, int8_t *wt, int c_out, int taps, int c_in, cudaStream_t s)
+{
+    const size_t total = (size_t)c_out * taps * c_in;
+    int blocks = (int)((total + kThreads - 1) / kThreads);
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    weight_transpose_kernel<<<blocks, kThreads, 0, s>>>(w, wt, c_out, taps, c_in);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_b1_weight_table(const int8_t *w, int32_t *table, const eoq_conv_desc_t &d, const BorderClasses &bc,
+                                   cudaStream_t s)
+{
+    const int ho = (d.h + 2 * d.pad - d.kh) / d.stride + 1, wo = (d.w + 2 * d.pad - d.kw) / d.stride + 1;
+    dim3 grid((d.c_out + 127) / 128, bc.nrc * bc.ncc);
+    b1_weight_table_kernel<<<grid, 128, 0, s>>>(w, table, d, ho, wo, bc);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, const eoq_conv_desc_t &d, int ho, int wo,
+                                 cudaStream_t s)
+{
+    cudaError_t e = cudaMemsetAsync(tap_sums, 0, sizeof(long long) * d.c_out * d.kh * d.kw, s);
+    if (e != cudaSuccess) return e;
+    const size_t pixels = (size_t)d.n * ho * wo;
+    int zs = (int)((pixels + 4095) / 4096);
+    zs = zs < 1 ? 1 : (zs > 64 ? 64 : zs);
+    dim3 grid((d.c_out + 31) / 32, d.kh * d.kw, zs);
+    b1_error_sums_kernel<<<grid, 1024, 0, s>>>(e3, tap_sums, d, ho, wo);
+    return cudaGetLastError();
+}
+
+}  // namespace eoq

@@ -1,0 +1,142 @@
+// Internal declarations shared by the translation units of libeoq (not part of the public ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "eoq.h"
+
+namespace eoq {
+
+constexpr int kMaxTaps = 64;        // kh * kw of any supported filter
+constexpr int kTileM = 128;         // GEMM rows per CTA tile (TMEM lanes)
+constexpr int kGemmThreads = 192;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr uint32_t kSpinLimit = 1u << 22;  // polls before a wait gives up (normal waits end within microseconds)
+
+// Device state a handle owns.
+struct DeviceState {
+    unsigned status;       // EOQ_DEV_* bits
+    unsigned absmax_u32;   // reduction cell for |.| maxima (int32 sources, float bit patterns)
+    unsigned long long absmax_u64;
+    long long sum0, sum1;  // reduction cells for integer sums
+    unsigned tensor_absmax[256];  // per-tensor maxima of the multi-tensor update
+};
+
+struct Handle {
+    int device;
+    int sm_count;
+    int last_cuda_error;
+    DeviceState *dev;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Implicit-GEMM kernel used by the forward pass and by error back-propagation.
+//   D[m, j] = sum over sub-tiles s of  A_s[m, 0..kc) . B_s[j, 0..kc)
+// A_s is fetched by TMA in im2col mode from an NHWC int8 tensor (tap offset + channel chunk),
+// B_s by a tiled TMA from a [rows][taps][channels] int8 tensor.
+// ---------------------------------------------------------------------------------------------
+enum EpilogueKind { kEpiForward = 0, kEpiDgrad = 1 };
+
+struct IgemmParams {
+    // GEMM extent
+    int M;              // rows: n_img * hq * wq
+    int N;              // columns (multiple of 16)
+    int hq, wq;         // pixel grid per image walked by the rows
+    int tile_n;         // columns per CTA tile (multiple of 16, <= 256)
+    int num_m_tiles, num_n_tiles;
+    // K structure
+    int kc;             // channel bytes per sub-tile: 16, 32, 64 or 128 (= TMA swizzle span, 16 = none)
+    int chunks_per_tap; // source channels / kc
+    int num_sub;        // taps * chunks_per_tap (padded to even when kc == 16)
+    int real_sub;       // sub-tiles that carry data
+    int subs_per_stage;
+    int num_stages;
+    int src_stride;     // TMA traversal stride in source pixels
+    int base_h, base_w; // source coordinate of tap offset (0,0) for pixel (0,0)
+    unsigned char tap_dh[kMaxTaps], tap_dw[kMaxTaps];  // im2col offsets of each tap
+    unsigned char tap_b[kMaxTaps];                     // tap coordinate of each tap in the B tensor
+    int ntaps;
+    // output mapping: GEMM row (n, y, x) -> pixel (n, y*out_step + out_off_h, x*out_step + out_off_w)
+    int out_h, out_w, out_step, out_off_h, out_off_w;
+    int epilogue;       // EpilogueKind
+    // forward epilogue
+    const int32_t *x_exp;     // device exponent of the input or null
+    int32_t b1_c, gamma_c, b2_c;
+    const int32_t *b1_table;  // [classes][N] tap-validity sums of the weights (null when b1_c == 0)
+    int b1_nlo_h, b1_nhi_h, b1_nrc, b1_nlo_w, b1_nhi_w, b1_ncc;
+    const int8_t *shortcut;
+    int relu;
+    int8_t *x5;
+    int16_t *x2;
+    uint8_t *relu_mask;
+    int32_t *acc_out;         // forward: optional dump; dgrad: the int32 scratch (required)
+    DeviceState *dev;
+};
+
+size_t igemm_smem_bytes(const IgemmParams &p);
+cudaError_t launch_igemm(const IgemmParams &p, const CUtensorMap &map_a, const CUtensorMap &map_b, int grid,
+                         cudaStream_t stream);
+
+// ---------------------------------------------------------------------------------------------
+// Weight-gradient kernel: D[(tap, ic), oc] = sum over pixels of x1[pixel + tap, ic] * e3[pixel, oc]
+// ---------------------------------------------------------------------------------------------
+struct WgradParams {
+    int P;               // reduction length: n * ho * wo error pixels
+    int ho, wo;
+    int c_in, c_out;
+    int ntaps;
+    int kc;              // c_in bytes per A sub-tile (16..128)
+    int nc;              // c_out bytes per B sub-tile (16..128)
+    int chunks_per_tap;  // c_in / kc
+    int rows_total;      // ntaps * c_in (GEMM M)
+    int subs_per_mtile;  // 128 / kc
+    int tile_n;          // c_out columns per CTA (multiple of 16, <= 256)
+    int num_m_tiles, num_n_tiles, num_k_splits;
+    int pixels_per_stage;   // 64
+    int stages_per_split;   // pipeline iterations each CTA runs
+    int num_stages;
+    int src_stride, base_h, base_w;
+    unsigned char tap_dh[kMaxTaps], tap_dw[kMaxTaps];
+    long long *acc;      // [c_out][taps][c_in] int64, zeroed before launch
+    DeviceState *dev;
+};
+
+size_t wgrad_smem_bytes(const WgradParams &p);
+cudaError_t launch_wgrad(const WgradParams &p, const CUtensorMap &map_x, const CUtensorMap &map_e, cudaStream_t stream);
+
+// ---------------------------------------------------------------------------------------------
+// Elementwise / reduction kernels
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_reset_cells(DeviceState *dev, cudaStream_t s);
+cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst, int32_t *dst_exp, DeviceState *dev,
+                                int sm_count, cudaStream_t s);
+cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
+                          int32_t *dst_exp, long long *sum_codes, bool max_already_reduced, DeviceState *dev,
+                          int sm_count, cudaStream_t s);
+cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
+                          int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int taps,
+                          int c_in, DeviceState *dev, int sm_count, cudaStream_t s);
+cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const uint8_t *mask, const int16_t *x2,
+                                size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
+                                long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s);
+struct UpdateTensor {
+    int8_t *w;
+    const int8_t *g;
+    const int32_t *g_exp;
+    unsigned long long n;
+};
+cudaError_t launch_update(const UpdateTensor *t, int num, int32_t lr_mant, int32_t lr_exp, int stochastic,
+                          uint64_t seed, uint64_t step, DeviceState *dev, int sm_count, cudaStream_t s);
+cudaError_t launch_layout_convert(const int8_t *src, int8_t *dst, int n, int c, int h, int w, int to_nhwc,
+                                  cudaStream_t s);
+cudaError_t launch_weight_transpose(const int8_t *w, int8_t *wt, int c_out, int taps, int c_in, cudaStream_t s);
+// b1 support: class tables of weight sums (forward) and of error sums (weight gradient)
+struct BorderClasses {
+    int nlo_h, nhi_h, nrc, nlo_w, nhi_w, ncc;
+};
+cudaError_t launch_b1_weight_table(const int8_t *w, int32_t *table, const eoq_conv_desc_t &d, const BorderClasses &bc,
+                                   cudaStream_t s);
+cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, const eoq_conv_desc_t &d, int ho, int wo,
+                                 cudaStream_t s);
+
+}  // namespace eoq

@@ -1,0 +1,209 @@
+"""Thin ctypes binding over libeoq.so (the C ABI declared in include/eoq.h).
+
+Each function has the name and argument order of its C counterpart and only
+marshals arguments: torch tensors (device memory owned by the caller) become raw
+pointers, the current torch CUDA stream becomes the ``stream`` argument.  All
+arithmetic runs in the CUDA kernels; there is no CPU fallback, and a missing
+library raises at first use.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libeoq.so")
+
+EOQ_OK, EOQ_ERR_BAD_ARG, EOQ_ERR_ALIGNMENT, EOQ_ERR_UNSUPPORTED, EOQ_ERR_WORKSPACE, EOQ_ERR_RANGE, EOQ_ERR_CUDA = range(7)
+EOQ_DEV_TIMEOUT, EOQ_DEV_NONFINITE, EOQ_DEV_SQ_ZERO, EOQ_DEV_RANGE = 1, 2, 4, 8
+EOQ_Q, EOQ_CQ, EOQ_SQ = 0, 1, 2
+EOQ_ROUND_RNE, EOQ_ROUND_STOCHASTIC = 0, 1
+EOQ_PASS_FWD, EOQ_PASS_DGRAD, EOQ_PASS_WGRAD = 0, 1, 2
+
+EXPORTS = [
+    "eoq_create", "eoq_destroy", "eoq_workspace_size", "eoq_conv_fwd", "eoq_conv_dgrad", "eoq_conv_wgrad",
+    "eoq_quantize", "eoq_err_prescale", "eoq_update", "eoq_layout_convert", "eoq_last_status",
+    "eoq_last_cuda_error", "eoq_status_string",
+]
+
+
+class EoqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class eoq_conv_desc_t(C.Structure):
+    _fields_ = [(k, C.c_int) for k in ("n", "h", "w", "c_in", "c_out", "kh", "kw", "stride", "pad")]
+
+    @property
+    def ho(self) -> int:
+        return (self.h + 2 * self.pad - self.kh) // self.stride + 1
+
+    @property
+    def wo(self) -> int:
+        return (self.w + 2 * self.pad - self.kw) // self.stride + 1
+
+
+def conv_desc(n, h, w, c_in, c_out, kh, kw, stride=1, pad=0) -> eoq_conv_desc_t:
+    return eoq_conv_desc_t(n, h, w, c_in, c_out, kh, kw, stride, pad)
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libeoq.so; raises if it has not been built (python -m paper_2105_13890_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2105_13890_b200.build` "
+                               "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, sz, u64 = C.c_void_p, C.c_int32, C.c_size_t, C.c_uint64
+        dp = C.POINTER(eoq_conv_desc_t)
+        L.eoq_create.argtypes = [C.POINTER(vp), C.c_int]
+        L.eoq_destroy.argtypes = [vp]
+        L.eoq_workspace_size.argtypes = [dp, C.c_int, C.POINTER(sz)]
+        L.eoq_conv_fwd.argtypes = [vp, dp, vp, vp, i32, vp, i32, i32, vp, C.c_int, vp, vp, vp, vp, vp, sz, vp]
+        L.eoq_conv_dgrad.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.eoq_conv_wgrad.argtypes = [vp, dp, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+        L.eoq_quantize.argtypes = [vp, C.c_int, vp, C.c_int, vp, sz, vp, vp, vp, sz, vp]
+        L.eoq_err_prescale.argtypes = [vp, vp, vp, vp, vp, sz, i32, vp, vp, vp, vp, vp]
+        L.eoq_update.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), i32, i32,
+                                 C.c_int, u64, u64, vp]
+        L.eoq_layout_convert.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp]
+        L.eoq_last_status.argtypes = [vp, vp, C.POINTER(C.c_uint)]
+        L.eoq_last_cuda_error.argtypes = [vp]
+        L.eoq_status_string.argtypes = [C.c_int]
+        L.eoq_status_string.restype = C.c_char_p
+        for name in EXPORTS:
+            if name != "eoq_status_string":
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().eoq_status_string(int(status)).decode()
+
+
+def _ptr(t) -> Optional[int]:
+    """Raw address of a torch tensor (or of an int already holding one); None stays NULL."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is not None:
+        return stream if isinstance(stream, int) else stream.cuda_stream
+    import torch
+
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _nbytes(t) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def _check(status: int, where: str) -> None:
+    if status != EOQ_OK:
+        raise EoqError(status, where)
+
+
+# ------------------------------------------------------------------------------- entry points
+
+def eoq_create(device: int = 0) -> int:
+    h = C.c_void_p()
+    _check(lib().eoq_create(C.byref(h), int(device)), "eoq_create")
+    return h.value
+
+
+def eoq_destroy(handle: int) -> None:
+    _check(lib().eoq_destroy(handle), "eoq_destroy")
+
+
+def eoq_workspace_size(desc: eoq_conv_desc_t, pass_: int) -> int:
+    out = C.c_size_t(0)
+    _check(lib().eoq_workspace_size(C.byref(desc), int(pass_), C.byref(out)), "eoq_workspace_size")
+    return out.value
+
+
+def eoq_conv_fwd(handle, desc, x, x_exp, b1_c, w, gamma_c, b2_c, shortcut, relu, x5, x2=None, relu_mask=None,
+                 acc_dump=None, workspace=None, stream=None, check: bool = True) -> int:
+    st = lib().eoq_conv_fwd(handle, C.byref(desc), _ptr(x), _ptr(x_exp), int(b1_c), _ptr(w), int(gamma_c), int(b2_c),
+                            _ptr(shortcut), 1 if relu else 0, _ptr(x5), _ptr(x2), _ptr(relu_mask), _ptr(acc_dump),
+                            _ptr(workspace), _nbytes(workspace), _stream(stream))
+    if check:
+        _check(st, "eoq_conv_fwd")
+    return st
+
+
+def eoq_conv_dgrad(handle, desc, e3, e3_exp, w, e4, e4_exp, sum_e4=None, acc_dump=None, workspace=None, stream=None,
+                   check: bool = True) -> int:
+    st = lib().eoq_conv_dgrad(handle, C.byref(desc), _ptr(e3), _ptr(e3_exp), _ptr(w), _ptr(e4), _ptr(e4_exp),
+                              _ptr(sum_e4), _ptr(acc_dump), _ptr(workspace), _nbytes(workspace), _stream(stream))
+    if check:
+        _check(st, "eoq_conv_dgrad")
+    return st
+
+
+def eoq_conv_wgrad(handle, desc, e3, e3_exp, x, b1_c, g, g_exp, acc_dump=None, workspace=None, stream=None,
+                   check: bool = True) -> int:
+    st = lib().eoq_conv_wgrad(handle, C.byref(desc), _ptr(e3), _ptr(e3_exp), _ptr(x), int(b1_c), _ptr(g), _ptr(g_exp),
+                              _ptr(acc_dump), _ptr(workspace), _nbytes(workspace), _stream(stream))
+    if check:
+        _check(st, "eoq_conv_wgrad")
+    return st
+
+
+def eoq_quantize(handle, mode, src, src_is_float, src_exp, n, dst, dst_exp=None, workspace=None, stream=None,
+                 check: bool = True) -> int:
+    st = lib().eoq_quantize(handle, int(mode), _ptr(src), 1 if src_is_float else 0, _ptr(src_exp), int(n), _ptr(dst),
+                            _ptr(dst_exp), _ptr(workspace), _nbytes(workspace), _stream(stream))
+    if check:
+        _check(st, "eoq_quantize")
+    return st
+
+
+def eoq_err_prescale(handle, e0, e0_exp, relu_mask, x2, n_el, gamma_c, e3, e3_exp, sum_e1=None, sum_e1x2=None,
+                     stream=None, check: bool = True) -> int:
+    st = lib().eoq_err_prescale(handle, _ptr(e0), _ptr(e0_exp), _ptr(relu_mask), _ptr(x2), int(n_el), int(gamma_c),
+                                _ptr(e3), _ptr(e3_exp), _ptr(sum_e1), _ptr(sum_e1x2), _stream(stream))
+    if check:
+        _check(st, "eoq_err_prescale")
+    return st
+
+
+def eoq_update(handle, w: Sequence, g: Sequence, g_exp: Sequence, lr_mant: int, lr_exp: int,
+               round_mode: int = EOQ_ROUND_RNE, seed: int = 0, step: int = 0, stream=None, check: bool = True) -> int:
+    num = len(w)
+    arr = C.c_void_p * num
+    sizes = (C.c_size_t * num)(*[t.numel() for t in w])
+    st = lib().eoq_update(handle, num, arr(*[_ptr(t) for t in w]), arr(*[_ptr(t) for t in g]),
+                          arr(*[_ptr(t) for t in g_exp]), sizes, int(lr_mant), int(lr_exp), int(round_mode),
+                          int(seed), int(step), _stream(stream))
+    if check:
+        _check(st, "eoq_update")
+    return st
+
+
+def eoq_layout_convert(handle, src, dst, n, c, h, w, to_nhwc: bool, stream=None, check: bool = True) -> int:
+    st = lib().eoq_layout_convert(handle, _ptr(src), _ptr(dst), n, c, h, w, 1 if to_nhwc else 0, _stream(stream))
+    if check:
+        _check(st, "eoq_layout_convert")
+    return st
+
+
+def eoq_last_status(handle, stream=None) -> int:
+    bits = C.c_uint(0)
+    _check(lib().eoq_last_status(handle, _stream(stream), C.byref(bits)), "eoq_last_status")
+    return bits.value
+
+
+def eoq_last_cuda_error(handle) -> int:
+    return lib().eoq_last_cuda_error(handle)
