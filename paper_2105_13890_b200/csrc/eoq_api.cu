@@ -383,7 +383,18 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
 
     // One GEMM per residue class (y mod stride, x mod stride) of the input pixels: within a class the taps
     // kh with (y + pad - kh) divisible by the stride form a unit-stride correlation over e3.
-    bool cleared = false;
+    // a class no tap reaches (e.g. the odd pixels of a strided 1x1 filter) keeps zero sums: clear first
+    bool any_empty = false;
+    for (int r = 0; r < d.stride; ++r) {
+        bool hit_h = false, hit_w = false;
+        for (int kh = 0; kh < d.kh; ++kh) hit_h |= (r + d.pad - kh) % d.stride == 0;
+        for (int kw = 0; kw < d.kw; ++kw) hit_w |= (r + d.pad - kw) % d.stride == 0;
+        any_empty |= (r < d.h && !hit_h) || (r < d.w && !hit_w);
+    }
+    if (any_empty) {
+        e = cudaMemsetAsync(sums, 0, g.in_elems * sizeof(int32_t), s);
+        if (e != cudaSuccess) return record(h, e);
+    }
     for (int py = 0; py < d.stride && py < d.h; ++py)
         for (int px = 0; px < d.stride && px < d.w; ++px) {
             IgemmParams p;
@@ -405,15 +416,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                     ++nw;
                 }
             const int hq = (d.h - py + d.stride - 1) / d.stride, wq = (d.w - px + d.stride - 1) / d.stride;
-            if (nh == 0 || nw == 0) {
-                // no tap reaches this class: its sums are zero
-                if (!cleared) {
-                    e = cudaMemsetAsync(sums, 0, g.in_elems * sizeof(int32_t), s);
-                    if (e != cudaSuccess) return record(h, e);
-                    cleared = true;
-                }
-                continue;
-            }
+            if (nh == 0 || nw == 0) continue;  // no tap reaches this class: its sums stay zero
             p.M = d.n * hq * wq;
             p.N = d.c_in;
             p.hq = hq;

@@ -1,0 +1,239 @@
+"""GPU parity: every C-ABI entry point against the oracle, element by element, on seeded synthetic inputs.
+Integer tensors must match bit for bit; exponents are integers and must be equal."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import ConvDesc
+from paper_2105_13890_b200 import eoq, synth
+
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+# geometry sweep: several tiles, ragged tails, every swizzle width, strides, 1x1 and 7x7, tiny images
+SHAPES = [
+    ConvDesc(8, 32, 32, 16, 16, 3, 3, 1, 1),      # the single-layer configuration
+    ConvDesc(2, 8, 8, 64, 64, 3, 3, 1, 1),
+    ConvDesc(3, 13, 11, 32, 48, 3, 3, 1, 1),      # ragged last tile, 48 columns
+    ConvDesc(2, 10, 10, 128, 128, 3, 3, 1, 1),
+    ConvDesc(1, 14, 14, 256, 512, 3, 3, 1, 1),    # two column tiles
+    ConvDesc(3, 9, 7, 64, 48, 3, 3, 2, 1),        # stride 2, odd extents
+    ConvDesc(2, 16, 16, 64, 128, 3, 3, 2, 1),
+    ConvDesc(2, 8, 8, 64, 128, 1, 1, 1, 0),
+    ConvDesc(2, 16, 16, 64, 128, 1, 1, 2, 0),     # projection shortcut
+    ConvDesc(2, 20, 20, 16, 64, 7, 7, 2, 3),      # stem-like
+    ConvDesc(1, 2, 2, 16, 16, 3, 3, 1, 1),        # every pixel touches the border
+    ConvDesc(1, 1, 1, 32, 16, 1, 1, 1, 0),        # degenerate: one pixel
+    ConvDesc(5, 7, 7, 512, 512, 3, 3, 1, 1),      # K = 4608
+    ConvDesc(2, 12, 12, 192, 80, 3, 3, 1, 1),     # channel counts that are not powers of two
+]
+IDS = [f"n{d.n}_{d.h}x{d.w}_c{d.c_in}-{d.c_out}_k{d.kh}s{d.stride}p{d.pad}" for d in SHAPES]
+
+
+def layer_data(d, seed, wrange=30):
+    x0 = synth.relu_codes((d.n, d.h, d.w, d.c_in), seed, 0) if seed % 2 else synth.int8_uniform((d.n, d.h, d.w, d.c_in), seed, 0)
+    w = synth.int8_uniform((d.c_out, d.kh, d.kw, d.c_in), seed, 1, -wrange, wrange)
+    sc = synth.int8_uniform((d.n, d.ho, d.wo, d.c_out), seed, 2)
+    e3 = synth.normal_codes((d.n, d.ho, d.wo, d.c_out), seed, 3)
+    return x0, w, sc, e3
+
+
+@pytest.mark.parametrize("d", SHAPES, ids=IDS)
+@pytest.mark.parametrize("scal", [(0, 128, 0, False, True), (-3, 90, 5, True, True), (7, -200, -40, True, False)],
+                         ids=["init", "b1neg_sc", "b1pos_norelu"])
+def test_conv_fwd(d, scal):
+    b1, gamma, b2, use_sc, relu = scal
+    x0, w, sc, _ = layer_data(d, 100 + d.c_in + d.h)
+    ref = oracle.layer_forward(d, x0, b1, w, gamma, b2, sc if use_sc else None, relu)
+    gd = G.gdesc(d)
+    shape = ref["x5"].shape
+    x5, x2, acc = G.zeros(shape, torch.int8), G.zeros(shape, torch.int16), G.zeros(shape, torch.int32)
+    mask = G.zeros((ref["x5"].size + 7) // 8, torch.uint8)
+    eoq.eoq_conv_fwd(G.handle(), gd, G.dev(x0), None, b1, G.dev(w), gamma, b2, G.dev(sc) if use_sc else None, relu,
+                     x5, x2, mask, acc, G.workspace(gd, eoq.EOQ_PASS_FWD))
+    assert G.status_clear() == 0
+    assert np.array_equal(G.host(acc).astype(np.int64), ref["acc"])
+    assert np.array_equal(G.host(x2).astype(np.int32), ref["x2"])
+    assert np.array_equal(G.host(x5), ref["x5"])
+    assert np.array_equal(G.unpack_mask(mask, shape), ref["mask"])
+
+
+def test_conv_fwd_without_optional_outputs_and_with_input_exponent():
+    d = ConvDesc(2, 12, 12, 16, 32, 3, 3, 1, 1)
+    x0, w, _, _ = layer_data(d, 7)
+    gd = G.gdesc(d)
+    for p_in in (-5, -9, -7):
+        ref = oracle.layer_forward(d, x0, 0, w, 128, 3, None, True, x_exp=p_in)
+        x5 = G.zeros(ref["x5"].shape, torch.int8)
+        eoq.eoq_conv_fwd(G.handle(), gd, G.dev(x0), G.dev(np.array([p_in], dtype=np.int32)), 0, G.dev(w), 128, 3, None,
+                         True, x5)
+        assert G.status_clear() == 0
+        assert np.array_equal(G.host(x5), ref["x5"])
+
+
+@pytest.mark.parametrize("d", SHAPES, ids=IDS)
+def test_conv_dgrad(d):
+    _, w, _, e3 = layer_data(d, 200 + d.c_out + d.w)
+    p3 = -11
+    B = oracle.conv_dgrad_acc(d, e3, w)
+    e4, p4, z = oracle.sq_int(B, p3 - 7)
+    gd = G.gdesc(d)
+    e4_d, acc = G.zeros(B.shape, torch.int8), G.zeros(B.shape, torch.int32)
+    e4_exp, s4 = G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+    eoq.eoq_conv_dgrad(G.handle(), gd, G.dev(e3), G.dev(np.array([p3], dtype=np.int32)), G.dev(w), e4_d, e4_exp, s4,
+                       acc, G.workspace(gd, eoq.EOQ_PASS_DGRAD))
+    assert G.status_clear() == (eoq.EOQ_DEV_SQ_ZERO if z else 0)
+    assert np.array_equal(G.host(acc).astype(np.int64), B)
+    assert e4_exp.item() == p4
+    assert np.array_equal(G.host(e4_d).astype(np.int32), e4)
+    assert s4.item() == int(e4.astype(np.int64).sum())
+    # same call with the sums kept in the workspace
+    e4_b, exp_b = G.zeros(B.shape, torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_conv_dgrad(G.handle(), gd, G.dev(e3), G.dev(np.array([p3], dtype=np.int32)), G.dev(w), e4_b, exp_b, None,
+                       None, G.workspace(gd, eoq.EOQ_PASS_DGRAD))
+    G.status_clear()
+    assert torch.equal(e4_b, e4_d) and exp_b.item() == p4
+
+
+@pytest.mark.parametrize("d", SHAPES, ids=IDS)
+@pytest.mark.parametrize("b1", [0, -5])
+def test_conv_wgrad(d, b1):
+    x0, _, _, e3 = layer_data(d, 300 + d.c_in + d.w)
+    p3 = -9
+    Gacc = oracle.conv_wgrad_acc(d, e3, x0, b1)
+    g, pg, z = oracle.sq_int(Gacc, p3 - 7)
+    gd = G.gdesc(d)
+    g_d, acc = G.zeros(Gacc.shape, torch.int8), G.zeros(Gacc.shape, torch.int64)
+    g_exp = G.zeros(1, torch.int32)
+    eoq.eoq_conv_wgrad(G.handle(), gd, G.dev(e3), G.dev(np.array([p3], dtype=np.int32)), G.dev(x0), b1, g_d, g_exp, acc,
+                       G.workspace(gd, eoq.EOQ_PASS_WGRAD))
+    assert G.status_clear() == (eoq.EOQ_DEV_SQ_ZERO if z else 0)
+    assert np.array_equal(G.host(acc), Gacc)
+    assert g_exp.item() == pg
+    assert np.array_equal(G.host(g_d).astype(np.int32), g)
+
+
+def test_wgrad_long_reduction_needs_more_than_int32():
+    """All-extreme operands over 2^17+ pixels overflow an int32 sum; the split-K partials must still be exact."""
+    d = ConvDesc(9, 128, 128, 16, 16, 1, 1, 1, 0)
+    x0 = np.full((d.n, d.h, d.w, d.c_in), 127, dtype=np.int8)
+    e3 = np.full((d.n, d.ho, d.wo, d.c_out), -127, dtype=np.int8)
+    gd = G.gdesc(d)
+    acc, g_d, g_exp = G.zeros((16, 1, 1, 16), torch.int64), G.zeros((16, 1, 1, 16), torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_conv_wgrad(G.handle(), gd, G.dev(e3), G.dev(np.array([0], dtype=np.int32)), G.dev(x0), 0, g_d, g_exp, acc,
+                       G.workspace(gd, eoq.EOQ_PASS_WGRAD))
+    assert G.status_clear() == 0
+    want = -127 * 127 * d.n * d.h * d.w
+    assert abs(want) > 2**31
+    assert (G.host(acc) == want).all()
+
+
+@pytest.mark.parametrize("n", [1, 15, 16, 4099, 1 << 20])
+@pytest.mark.parametrize("mode", [eoq.EOQ_Q, eoq.EOQ_CQ, eoq.EOQ_SQ])
+def test_quantize_f32(n, mode):
+    x = synth.normal_f32(n, 400 + n % 97, mode, std=2.5 if mode != eoq.EOQ_SQ else 1e-3)
+    c, p, flag = oracle.quantize_f32(mode, x)
+    if mode == eoq.EOQ_Q:
+        c = np.clip(c, -32768, 32767)
+    out = G.zeros(n, torch.int16 if mode == eoq.EOQ_Q else torch.int8)
+    ex = G.zeros(1, torch.int32)
+    eoq.eoq_quantize(G.handle(), mode, G.dev(x), True, None, n, out, ex)
+    assert G.status_clear() == 0
+    assert np.array_equal(G.host(out).astype(np.int32), c) and ex.item() == p
+
+
+def test_quantize_edge_cases():
+    h = G.handle()
+    out, ex = G.zeros(64, torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_quantize(h, eoq.EOQ_SQ, G.zeros(64, torch.float32), True, None, 64, out, ex)
+    assert G.status_clear() == eoq.EOQ_DEV_SQ_ZERO and not out.any() and ex.item() == -7
+    x = np.ones(64, dtype=np.float32)
+    x[5] = np.inf
+    eoq.eoq_quantize(h, eoq.EOQ_SQ, G.dev(x), True, None, 64, out, ex)
+    assert G.status_clear() & eoq.EOQ_DEV_NONFINITE
+    # ties, saturation and subnormal magnitudes
+    x = np.array([0.5 / 128, 1.5 / 128, -2.5 / 128, 300.0, -300.0, 1e-45, 0.99609375, 1.0] * 2, dtype=np.float32)
+    for mode in (eoq.EOQ_Q, eoq.EOQ_CQ):
+        c, _, _ = oracle.quantize_f32(mode, x)
+        o = G.zeros(16, torch.int16 if mode == eoq.EOQ_Q else torch.int8)
+        eoq.eoq_quantize(h, mode, G.dev(x), True, None, 16, o, None)
+        assert np.array_equal(G.host(o).astype(np.int32), np.clip(c, -32768, 32767))
+    tiny = (synth.normal_f32(333, 9, 9) * 1e-41).astype(np.float32)
+    c, p, _ = oracle.quantize_f32(eoq.EOQ_SQ, tiny)
+    o = G.zeros(333, torch.int8)
+    eoq.eoq_quantize(h, eoq.EOQ_SQ, G.dev(tiny), True, None, 333, o, ex)
+    assert G.status_clear() == 0 and np.array_equal(G.host(o).astype(np.int32), c) and ex.item() == p
+
+
+@pytest.mark.parametrize("n", [16, 1000, 1 << 18])
+def test_quantize_int32_source(n):
+    a = synth.rng(500, n).integers(-2**27, 2**27, size=n).astype(np.int32)
+    c, p, _ = oracle.sq_int(a.astype(np.int64), -19)
+    out, ex = G.zeros(n, torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_quantize(G.handle(), eoq.EOQ_SQ, G.dev(a), False, G.dev(np.array([-19], dtype=np.int32)), n, out, ex)
+    assert G.status_clear() == 0
+    assert np.array_equal(G.host(out).astype(np.int32), c) and ex.item() == p
+
+
+@pytest.mark.parametrize("n_el", [16, 4096 + 16, 1 << 19])
+@pytest.mark.parametrize("gamma", [128, -77, 3])
+def test_err_prescale(n_el, gamma):
+    e0 = synth.normal_codes(n_el, 600, gamma & 0xff)
+    mask = synth.bits(n_el, 601, 0)
+    x2 = synth.rng(602, 0).integers(-3000, 3001, size=n_el).astype(np.int16)
+    p0 = -13
+    e3, p3, s1, s2, z = oracle.err_prescale(e0, p0, mask, x2.astype(np.int32), gamma)
+    e3_d, e3_exp = G.zeros(n_el, torch.int8), G.zeros(1, torch.int32)
+    s1_d, s2_d = G.zeros(1, torch.int64), G.zeros(1, torch.int64)
+    eoq.eoq_err_prescale(G.handle(), G.dev(e0), G.dev(np.array([p0], dtype=np.int32)), G.dev(G.pack_mask(mask)),
+                         G.dev(x2), n_el, gamma, e3_d, e3_exp, s1_d, s2_d)
+    assert G.status_clear() == 0
+    assert np.array_equal(G.host(e3_d), e3) and e3_exp.item() == p3
+    assert s1_d.item() == s1 and s2_d.item() == s2
+
+
+@pytest.mark.parametrize("stochastic", [False, True])
+def test_update_multi_tensor(stochastic):
+    sizes = [16, 2304, 36864 + 5, 100000, 1, 8192, 8193]
+    r = synth.rng(700, int(stochastic))
+    ws = [synth.int8_uniform(n, 701, i) for i, n in enumerate(sizes)]
+    gs = [synth.normal_codes(n, 702, i, std_codes=40) for i, n in enumerate(sizes)]
+    pgs = [int(v) for v in r.integers(-16, -4, size=len(sizes))]
+    gs[4][:] = 0  # an all-zero gradient leaves its tensor untouched
+    for lr_mant, lr_exp in ((1, -3), (37, -8), (255, 2)):
+        w_d = [G.dev(w) for w in ws]
+        eoq.eoq_update(G.handle(), w_d, [G.dev(g) for g in gs], [G.dev(np.array([p], dtype=np.int32)) for p in pgs],
+                       lr_mant, lr_exp, eoq.EOQ_ROUND_STOCHASTIC if stochastic else eoq.EOQ_ROUND_RNE, seed=11, step=3)
+        assert G.status_clear() == eoq.EOQ_DEV_SQ_ZERO
+        changed = 0
+        for i, (w, g, p) in enumerate(zip(ws, gs, pgs)):
+            want, _, _ = oracle.update(w, g, p, lr_mant, lr_exp, stochastic=stochastic, seed=11, step=3, tensor_id=i)
+            got = G.host(w_d[i]).astype(np.int32)
+            assert np.array_equal(got, want), (i, lr_mant, lr_exp)
+            changed += int((got != w).sum())
+        assert changed > 0
+
+
+def test_layout_convert_round_trip():
+    x = synth.int8_uniform((3, 20, 7, 9), 800, 0)  # NCHW
+    nhwc, back = G.zeros((3, 7, 9, 20), torch.int8), G.zeros((3, 20, 7, 9), torch.int8)
+    eoq.eoq_layout_convert(G.handle(), G.dev(x), nhwc, 3, 20, 7, 9, True)
+    eoq.eoq_layout_convert(G.handle(), nhwc, back, 3, 20, 7, 9, False)
+    assert np.array_equal(G.host(nhwc), x.transpose(0, 2, 3, 1)) and np.array_equal(G.host(back), x)
+
+
+def test_argument_errors_launch_nothing():
+    h = G.handle()
+    d = eoq.conv_desc(1, 8, 8, 16, 16, 3, 3, 1, 1)
+    x, w, y = G.zeros((1, 8, 8, 16), torch.int8), G.zeros((16, 3, 3, 16), torch.int8), G.zeros((1, 8, 8, 16), torch.int8)
+    assert eoq.eoq_conv_fwd(h, eoq.conv_desc(1, 8, 8, 12, 16, 3, 3, 1, 1), x, None, 0, w, 128, 0, None, True, y, check=False) == eoq.EOQ_ERR_ALIGNMENT
+    assert eoq.eoq_conv_fwd(h, d, x, None, 0, w, 1 << 20, 0, None, True, y, check=False) == eoq.EOQ_ERR_RANGE
+    assert eoq.eoq_conv_fwd(h, d, x, None, 4, w, 128, 0, None, True, y, check=False) == eoq.EOQ_ERR_WORKSPACE
+    assert eoq.eoq_conv_fwd(h, d, None, None, 0, w, 128, 0, None, True, y, check=False) == eoq.EOQ_ERR_BAD_ARG
+    assert eoq.eoq_conv_fwd(h, d, x.data_ptr() + 1, None, 0, w, 128, 0, None, True, y, check=False) == eoq.EOQ_ERR_ALIGNMENT
+    ex = G.zeros(1, torch.int32)
+    assert eoq.eoq_conv_dgrad(h, d, y, ex, w, x, ex, check=False) == eoq.EOQ_ERR_WORKSPACE
+    assert eoq.eoq_conv_fwd(h, eoq.conv_desc(1, 8, 8, 16, 16, 9, 9, 1, 4), x, None, 0, w, 128, 0, None, True, y, check=False) == eoq.EOQ_ERR_UNSUPPORTED
+    assert G.status_clear() == 0
