@@ -1,0 +1,331 @@
+#!/usr/bin/env python
+"""Benchmark of the EOQ int8 convolution training path (arXiv 2105.13890) on B200.
+
+One step = one pass of the whole hot path over one synthetic batch: input quantizer, then for every quantized
+convolution of Fixup ResNet-18 (batch 64, 224x224) forward + error head + dgrad + wgrad, then the 8-bit
+update of all weights.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet18|resnet20|resnet50|single] [--batch B]
+  python bench.py --impl reference ...     # the CPU oracle on host cores, same metric, bounded sample per step
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "int8 conv TOPS per train step (fwd+dgrad+wgrad) and img/s, % of INT8 roofline"
+INT8_OVER_BF16 = 2.0  # nominal dense ratio (4.5 / 2.25 PFLOP/s)
+
+
+def peaks():
+    """Measured denominators (generated file) or the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"],
+                "bf16_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc, self.lines = None, []
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def window(self, t0, t1):
+        return [l for (t, l) in self.lines if t0 <= t <= t1]
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    @staticmethod
+    def summarize(lines):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------- CPU oracle arm
+
+def oracle_step(wl, seed, scal):
+    """One step of the same path on the CPU oracle, as it stands.  Returns seconds."""
+    import numpy as np
+
+    import oracle
+    from oracle import ConvDesc
+    from paper_2105_13890_b200 import synth
+    from paper_2105_13890_b200.workloads import init_weight_f32
+
+    b1_c, gamma_c, b2_c = scal
+    # inputs first (not timed: the GPU arm's inputs are resident before its timed region too)
+    data = []
+    first = wl.layers[0]
+    image = synth.normal_f32((first.n, first.h, first.w, 3), seed, 0)
+    for i, l in enumerate(wl.layers):
+        d = ConvDesc(l.n, l.h, l.w, l.c_in, l.c_out, l.k, l.k, l.stride, l.pad)
+        x0 = synth.relu_codes((l.n, l.h, l.w, l.c_in), seed, 1) if i else None
+        e0 = synth.normal_codes((l.n, l.ho, l.wo, l.c_out), seed, 2)
+        sc = synth.relu_codes((l.n, l.ho, l.wo, l.c_out), seed, 3) if l.shortcut else None
+        w = oracle.q_w(init_weight_f32(l, wl, synth.normal_f64((l.c_out, l.k, l.k, l.c_in), seed, 100 + i)))
+        data.append((l, d, x0, e0, sc, w))
+    t0 = time.perf_counter()
+    img = np.zeros((first.n, first.h, first.w, first.c_in), dtype=np.float32)
+    img[..., :3] = image
+    codes, p_in, _ = oracle.quantize_f32(oracle.MODE_SQ, img)
+    saved = []
+    for i, (l, d, x0, e0, sc, w) in enumerate(data):
+        if i == 0:
+            x0 = codes.astype(np.int8)
+        gamma = gamma_c if l.gamma_trainable else 128
+        fwd = oracle.layer_forward(d, x0, 0 if i == 0 else b1_c, w, gamma, b2_c if l.relu else 0, sc, l.relu,
+                                   x_exp=p_in if i == 0 else -7)
+        saved.append((x0, fwd))
+    grads = []
+    for i in range(len(data) - 1, -1, -1):
+        l, d, _, e0, sc, w = data[i]
+        x0, fwd = saved[i]
+        gamma = gamma_c if l.gamma_trainable else 128
+        mask = fwd["mask"] if l.relu else np.ones_like(fwd["mask"])
+        e3, p3, s1, s2, _ = oracle.err_prescale(e0, -12, mask, fwd["x2"] if l.gamma_trainable else None, gamma)
+        if l.has_dgrad:
+            oracle.sq_int(oracle.conv_dgrad_acc(d, e3, w), p3 - 7)
+        g, pg, _ = oracle.sq_int(oracle.conv_wgrad_acc(d, e3, x0, 0 if i == 0 else b1_c), p3 - 7)
+        grads.append((i, g.astype(np.int8), pg))
+    for i, g, pg in grads:
+        oracle.update(data[i][5], g, pg, 1, -6, stochastic=True, seed=seed, step=0, tensor_id=i)
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    """--impl reference: the oracle timed on the host cores, each step a bounded sample (small batch) of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2105_13890_b200 import workloads
+
+    oracle.build()
+    sample_batch = args.ref_arm_batch
+    wl = workloads.get(args.workload, sample_batch)
+    full = workloads.get(args.workload, args.batch)
+    cores = os.cpu_count() or 1
+    for _ in range(args.warmup):
+        oracle_step(wl, 1, (-2, 118, 3))
+    secs = [oracle_step(wl, 1, (-2, 118, 3)) for _ in range(args.steps)]
+    t = sum(secs) / len(secs)
+    tops = wl.total_ops / t / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "img_per_s": wl.batch / t,
+        "config": {"workload": full.name, "sample": f"batch {sample_batch} of {full.batch} per step, all layers"},
+        "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": cores, "kind": "oracle",
+                         "sample": f"{wl.name}: every layer of the workload at batch {sample_batch}"},
+        "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------- GPU arm
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2105_13890_b200 import eoq, workloads
+    from paper_2105_13890_b200.step import Scalars, TrainStep
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    wl = workloads.get(args.workload, args.batch)
+    handle = eoq.eoq_create(local)
+    step = TrainStep(wl, handle, f"cuda:{local}", scalars=Scalars())
+    stream = torch.cuda.current_stream()
+
+    for _ in range(args.warmup):
+        step.run()
+    barrier()
+    status = eoq.eoq_last_status(handle)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    time.sleep(0.3)
+    # ---- timed region: K steps, inputs resident
+    l0 = eoq.eoq_launch_count(handle)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step.run()
+    ev1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    ms = ev0.elapsed_time(ev1)
+    launches = eoq.eoq_launch_count(handle) - l0
+    status |= eoq.eoq_last_status(handle)
+
+    # ---- end to end: host image in (pinned), results out, every step
+    host_img = torch.from_numpy(step.host_image(12345)).pin_memory()
+    results = step.result_tensors()
+    host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in results]
+    h2d = host_img.numel() * host_img.element_size()
+    d2h = sum(t.numel() * t.element_size() for t in results)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step.image.copy_(host_img, non_blocking=True)
+        step.run()
+        for src, dst in zip(results, host_out):
+            dst.copy_(src, non_blocking=True)
+    e1.record(stream)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+
+    # ---- per-kernel timing of the tensor-core kernels (events around each launch, same stream)
+    eoq.eoq_profile_start(handle)
+    for _ in range(args.steps):
+        step.run()
+    prof_n, prof_ms = eoq.eoq_profile_stop(handle)
+    clocks = ClockSampler.summarize(sampler.window(t_wall0, t_wall1)) if sampler else None
+    if sampler:
+        sampler.stop()
+
+    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=f"cuda:{local}")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, ms_e2e = t.tolist()
+
+    if rank == 0:
+        pk = peaks()
+        ops_step = wl.total_ops
+        sec = ms / 1e3 / args.steps
+        tops = world * ops_step / sec / 1e12
+        tops_e2e = world * ops_step / (ms_e2e / 1e3 / args.steps) / 1e12
+        int8_peak = pk["bf16_sustained"] * INT8_OVER_BF16
+        fwd_ops = sum(2 * l.macs for l in wl.layers) * args.steps
+        dgrad_ops = sum(2 * l.macs for l in wl.layers if l.has_dgrad) * args.steps
+        igemm_ms = prof_ms[0] + prof_ms[1]
+        igemm_n = prof_n[0] + prof_n[1]
+        achieved = (fwd_ops + dgrad_ops) / (igemm_ms / 1e3) / 1e12 if igemm_ms > 0 else None
+        line = {
+            "metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "img_per_s": world * wl.batch / sec,
+            "pct_of_int8_peak": 100.0 * tops / world / int8_peak,
+            "config": {"workload": wl.name, "layers": len(wl.layers), "global_batch": world * wl.batch,
+                       "gop_per_step": ops_step / 1e9, "l2": "working set larger than L2; no flush between steps",
+                       "scalars": "b1=-2 gamma=118 b2=3 codes", "parallelism": f"replicas x{world}"},
+            "clocks": clocks,
+            "e2e": {"value": tops_e2e, "unit": "TOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": int(launches),
+            "device_status": int(status),
+            "roofline": {
+                "kernel": "igemm_kernel (forward + dgrad implicit GEMM, tcgen05 kind::i8)", "bound": "tensor",
+                "achieved": achieved, "peak": int8_peak, "unit": "TOPS",
+                "frac": (achieved / int8_peak) if achieved else None, "traffic": None,
+                "peak_source": f"{pk['source']} sustained bf16 {pk['bf16_sustained']} TFLOP/s x {INT8_OVER_BF16} (nominal int8:bf16)",
+                "launches": igemm_n, "avg_launch_ms": igemm_ms / igemm_n if igemm_n else None,
+            },
+            "kernels": {
+                "igemm_fwd": {"launches": prof_n[0], "ms": prof_ms[0], "tops": fwd_ops / (prof_ms[0] / 1e3) / 1e12 if prof_ms[0] else None},
+                "igemm_dgrad": {"launches": prof_n[1], "ms": prof_ms[1], "tops": dgrad_ops / (prof_ms[1] / 1e3) / 1e12 if prof_ms[1] else None},
+                "wgrad": {"launches": prof_n[2], "ms": prof_ms[2], "tops": fwd_ops / (prof_ms[2] / 1e3) / 1e12 if prof_ms[2] else None},
+            },
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+
+            oracle.build()
+            small = workloads.get(args.workload, args.ref_batch)
+            secs = oracle_step(small, 1, (-2, 118, 3))
+            line["cpu_baseline"] = {"value": small.total_ops / secs / 1e12, "unit": "TOPS", "cores": os.cpu_count(),
+                                    "kind": "oracle", "seconds": secs,
+                                    "sample": f"{small.name}: every layer of the workload at batch {args.ref_batch}, one step"}
+        print(json.dumps(line), flush=True)
+    eoq.eoq_destroy(handle)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="eoq", choices=["eoq", "reference"])
+    ap.add_argument("--workload", default="resnet18")
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--ref-batch", type=int, default=4, help="batch of the CPU-oracle sample timed beside the GPU run")
+    ap.add_argument("--ref-arm-batch", type=int, default=1, help="batch of each step of --impl reference")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

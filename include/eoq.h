@@ -158,12 +158,35 @@ EOQ_API int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const int
                const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp, int round_mode,
                uint64_t seed, uint64_t step, void *stream);
 
+/*
+ * Q_e-style input quantizer for the network input (Sec. 5.1 quantizes every layer but the last): SQ(., 8)
+ * of an fp32 NHWC image with c_src channels per pixel, written as int8 with c_dst >= c_src channels per
+ * pixel (the extra channels are zero), so that the first convolution sees a multiple of 16 channels.
+ * device in : src [pixels][c_src] fp32.   device out: dst [pixels][c_dst] int8 (c_dst a multiple of 16, <= 64),
+ *             *dst_exp.  The maximum runs over the whole tensor.
+ */
+EOQ_API int eoq_quantize_image(eoq_handle_t handle, const float *src, size_t pixels, int c_src, int c_dst, int8_t *dst,
+                       int32_t *dst_exp, void *stream);
+
 /* int8 layout change between NCHW and NHWC ([n,c,h,w] <-> [n,h,w,c]); to_nhwc = 1 reads NCHW. */
 EOQ_API int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t *dst, int n, int c, int h, int w,
                        int to_nhwc, void *stream);
 
 /* Synchronises `stream`, returns the OR of the EOQ_DEV_* bits raised since the last call, clears them. */
 EOQ_API int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits);
+
+/*
+ * Instrumentation (off by default).  Between eoq_profile_start and eoq_profile_stop every launch of the two
+ * tensor-core kernels is bracketed by CUDA events on its stream.  eoq_profile_stop synchronises the device,
+ * and reports per kind (EOQ_PROF_*) the number of launches and their summed duration in milliseconds; it
+ * keeps at most 8192 launches.  eoq_launch_count returns how many kernels this handle has launched so far.
+ */
+#define EOQ_PROF_IGEMM_FWD 0
+#define EOQ_PROF_IGEMM_DGRAD 1
+#define EOQ_PROF_WGRAD 2
+EOQ_API int eoq_profile_start(eoq_handle_t handle);
+EOQ_API int eoq_profile_stop(eoq_handle_t handle, int launches[3], double milliseconds[3]);
+EOQ_API unsigned long long eoq_launch_count(eoq_handle_t handle);
 
 /* The last cudaError_t a call on this handle recorded (0 if none). */
 EOQ_API int eoq_last_cuda_error(eoq_handle_t handle);

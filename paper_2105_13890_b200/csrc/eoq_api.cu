@@ -192,6 +192,10 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
     h->device = device;
     h->last_cuda_error = 0;
     h->dev = nullptr;
+    h->launches = 0;
+    h->profiling = false;
+    h->num_records = 0;
+    h->records = nullptr;
     cudaDeviceProp prop;
     cudaError_t e = cudaGetDeviceProperties(&prop, device);
     if (e == cudaSuccess) {
@@ -220,9 +224,87 @@ extern "C" int eoq_destroy(eoq_handle_t handle)
     cudaSetDevice(h->device);
     cudaDeviceSynchronize();
     if (h->dev) cudaFree(h->dev);
+    if (h->records) {
+        for (int i = 0; i < h->num_records; ++i) {
+            cudaEventDestroy(h->records[i].begin);
+            cudaEventDestroy(h->records[i].end);
+        }
+        delete[] h->records;
+    }
     delete h;
     return EOQ_OK;
 }
+
+extern "C" int eoq_profile_start(eoq_handle_t handle)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h) return EOQ_ERR_BAD_ARG;
+    if (!h->records) {
+        h->records = new (std::nothrow) ProfRecord[kMaxProfRecords];
+        if (!h->records) return EOQ_ERR_BAD_ARG;
+    }
+    for (int i = 0; i < h->num_records; ++i) {
+        cudaEventDestroy(h->records[i].begin);
+        cudaEventDestroy(h->records[i].end);
+    }
+    h->num_records = 0;
+    h->profiling = true;
+    return EOQ_OK;
+}
+
+extern "C" int eoq_profile_stop(eoq_handle_t handle, int launches[3], double milliseconds[3])
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !launches || !milliseconds) return EOQ_ERR_BAD_ARG;
+    h->profiling = false;
+    cudaError_t e = cudaDeviceSynchronize();
+    for (int k = 0; k < 3; ++k) {
+        launches[k] = 0;
+        milliseconds[k] = 0.0;
+    }
+    for (int i = 0; i < h->num_records && e == cudaSuccess; ++i) {
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, h->records[i].begin, h->records[i].end);
+        launches[h->records[i].kind] += 1;
+        milliseconds[h->records[i].kind] += ms;
+    }
+    return record(h, e);
+}
+
+extern "C" unsigned long long eoq_launch_count(eoq_handle_t handle)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    return h ? h->launches : 0ull;
+}
+
+namespace {
+
+// Brackets one tensor-core kernel launch with events while profiling is on.
+struct ProfScope {
+    Handle *h;
+    cudaStream_t s;
+    ProfRecord *r;
+    ProfScope(Handle *h_, int kind, cudaStream_t s_) : h(h_), s(s_), r(nullptr)
+    {
+        if (!h->profiling || h->num_records >= kMaxProfRecords) return;
+        ProfRecord *c = &h->records[h->num_records];
+        if (cudaEventCreate(&c->begin) != cudaSuccess) return;
+        if (cudaEventCreate(&c->end) != cudaSuccess) {
+            cudaEventDestroy(c->begin);
+            return;
+        }
+        c->kind = kind;
+        ++h->num_records;
+        r = c;
+        cudaEventRecord(r->begin, s);
+    }
+    ~ProfScope()
+    {
+        if (r) cudaEventRecord(r->end, s);
+    }
+};
+
+}  // namespace
 
 extern "C" int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits)
 {
@@ -350,12 +432,15 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
         p.b1_nlo_w = bc.nlo_w; p.b1_nhi_w = bc.nhi_w; p.b1_ncc = bc.ncc;
         cudaError_t e = launch_b1_weight_table(w, reinterpret_cast<int32_t *>(workspace), d, bc, s);
         if (e != cudaSuccess) return record(h, e);
+        count_launches(h, 1);
     }
     CUtensorMap map_a, map_b;
     if (!make_im2col_map(&map_a, x, d.n, d.h, d.w, d.c_in, -d.pad, -d.pad, g.wo, g.ho, d.stride, p.kc, kTileM) ||
         !make_weight_map(&map_b, w, d.c_out, g.taps, d.c_in, p.kc, p.tile_n))
         return EOQ_ERR_UNSUPPORTED;
     const int tiles = p.num_m_tiles * p.num_n_tiles;
+    count_launches(h, 1);
+    ProfScope prof(h, EOQ_PROF_IGEMM_FWD, s);
     return record(h, launch_igemm(p, map_a, map_b, tiles < h->sm_count ? tiles : h->sm_count, s));
 }
 
@@ -380,6 +465,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     cudaError_t e = launch_reset_cells(h->dev, s);
     if (e == cudaSuccess) e = launch_weight_transpose(w, wt, d.c_out, g.taps, d.c_in, s);
     if (e != cudaSuccess) return record(h, e);
+    count_launches(h, 1);
 
     // One GEMM per residue class (y mod stride, x mod stride) of the input pixels: within a class the taps
     // kh with (y + pad - kh) divisible by the stride form a unit-stride correlation over e3.
@@ -446,12 +532,17 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                 !make_weight_map(&map_b, wt, d.c_in, g.taps, d.c_out, p.kc, p.tile_n))
                 return EOQ_ERR_UNSUPPORTED;
             const int tiles = p.num_m_tiles * p.num_n_tiles;
-            e = launch_igemm(p, map_a, map_b, tiles < h->sm_count ? tiles : h->sm_count, s);
+            count_launches(h, 1);
+            {
+                ProfScope prof(h, EOQ_PROF_IGEMM_DGRAD, s);
+                e = launch_igemm(p, map_a, map_b, tiles < h->sm_count ? tiles : h->sm_count, s);
+            }
             if (e != cudaSuccess) return record(h, e);
         }
     // Q_e over the whole tensor: the maximum is complete only now
     e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
                       h->sm_count, s);
+    count_launches(h, 1);
     return record(h, e);
 }
 
@@ -520,13 +611,20 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     p.dev = h->dev;
 
     cudaError_t e = cudaMemsetAsync(acc, 0, g.w_elems * sizeof(long long), s);
-    if (e == cudaSuccess && b1_c != 0) e = launch_b1_error_sums(e3, tap_sums, d, g.ho, g.wo, s);
+    if (e == cudaSuccess && b1_c != 0) {
+        e = launch_b1_error_sums(e3, tap_sums, d, g.ho, g.wo, s);
+        count_launches(h, 1);
+    }
     if (e != cudaSuccess) return record(h, e);
     CUtensorMap map_x, map_e;
     if (!make_im2col_map(&map_x, x, d.n, d.h, d.w, d.c_in, -d.pad, -d.pad, g.wo, g.ho, d.stride, p.kc, p.pixels_per_stage) ||
         !make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage))
         return EOQ_ERR_UNSUPPORTED;
-    e = launch_wgrad(p, map_x, map_e, s);
+    count_launches(h, 3);  // the GEMM and the two kernels of Q_g
+    {
+        ProfScope prof(h, EOQ_PROF_WGRAD, s);
+        e = launch_wgrad(p, map_x, map_e, s);
+    }
     if (e != cudaSuccess) return record(h, e);
     // the kernel leaves sums as [oc][tap][ic], which is the layout of g
     e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
@@ -548,6 +646,7 @@ extern "C" int eoq_quantize(eoq_handle_t handle, int mode, const void *src, int 
     if (mode == EOQ_SQ && !dst_exp) return EOQ_ERR_BAD_ARG;
     if (!aligned16(src) || !aligned16(dst)) return EOQ_ERR_ALIGNMENT;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, mode == EOQ_SQ ? 2 : 1);
     if (src_is_float)
         return record(h, launch_quantize_f32(mode, reinterpret_cast<const float *>(src), n, dst, dst_exp, h->dev, h->sm_count, s));
     if (mode != EOQ_SQ || !src_exp) return EOQ_ERR_UNSUPPORTED;
@@ -564,6 +663,7 @@ extern "C" int eoq_err_prescale(eoq_handle_t handle, const int8_t *e0, const int
     if (!aligned16(e0) || !aligned16(e3) || !aligned16(x2) || (reinterpret_cast<uintptr_t>(relu_mask) & 1)) return EOQ_ERR_ALIGNMENT;
     if (gamma_c < -32768 || gamma_c > 32767) return EOQ_ERR_RANGE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 2);
     return record(h, launch_err_prescale(e0, e0_exp, relu_mask, x2, n_el, gamma_c, e3, e3_exp,
                                          reinterpret_cast<long long *>(sum_e1), reinterpret_cast<long long *>(sum_e1x2),
                                          h->dev, h->sm_count, s));
@@ -587,6 +687,7 @@ extern "C" int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const 
         t[i].n = n[i];
     }
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 2 * ((num + 63) / 64));
     return record(h, launch_update(t, num, lr_mant, lr_exp, round_mode == EOQ_ROUND_STOCHASTIC, seed, step, h->dev, h->sm_count, s));
 }
 
@@ -595,5 +696,17 @@ extern "C" int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
     if (!h || !src || !dst || n <= 0 || c <= 0 || hh <= 0 || ww <= 0 || n > 65535) return EOQ_ERR_BAD_ARG;
+    count_launches(h, 1);
     return record(h, launch_layout_convert(src, dst, n, c, hh, ww, to_nhwc, reinterpret_cast<cudaStream_t>(stream)));
+}
+
+extern "C" int eoq_quantize_image(eoq_handle_t handle, const float *src, size_t pixels, int c_src, int c_dst, int8_t *dst,
+                                  int32_t *dst_exp, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !src || !dst || !dst_exp || pixels == 0 || c_src <= 0 || c_dst < c_src) return EOQ_ERR_BAD_ARG;
+    if (c_dst % 16 || c_dst > 64 || !aligned16(src) || !aligned16(dst)) return EOQ_ERR_ALIGNMENT;
+    count_launches(h, 2);
+    return record(h, launch_quantize_image(src, pixels, c_src, c_dst, dst, dst_exp, h->dev, h->sm_count,
+                                           reinterpret_cast<cudaStream_t>(stream)));
 }

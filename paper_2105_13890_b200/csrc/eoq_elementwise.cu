@@ -125,6 +125,40 @@ __global__ void quantize_f32_kernel(int mode, const float *__restrict__ src, siz
     }
 }
 
+// SQ of an fp32 image under the already reduced maximum, c_src channels in, c_dst (zero-padded) channels out.
+__global__ void quantize_image_kernel(const float *__restrict__ src, size_t pixels, int c_src, int c_dst, int8_t *dst,
+                                      int32_t *dst_exp, DeviceState *dev)
+{
+    const uint32_t mbits = dev->absmax_u32;
+    int up = 7;
+    const bool usable = mbits != 0 && mbits < 0x7f800000u;
+    if (usable) up = 7 - round_log2_f32bits(mbits);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        *dst_exp = usable ? -up : -7;
+        if (mbits == 0) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+    }
+    const int groups = c_dst / 16;
+    const size_t items = pixels * groups;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t pix = i / groups;
+        const int g = (int)(i % groups);
+        int c[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const int ch = g * 16 + k;
+            int v = 0;
+            if (ch < c_src) {
+                const float y = scalbnf(__ldg(src + pix * c_src + ch), up);
+                v = (fabsf(y) < 1.0e9f) ? clampi(__float2int_rn(y), -127, 127) : (y > 0.f ? 127 : (y < 0.f ? -127 : 0));
+            }
+            c[k] = v;
+        }
+        reinterpret_cast<int4 *>(dst)[i] =
+            make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
+                      (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+    }
+}
+
 // ------------------------------------------------------------------ int32 -> SQ (phase 2 of Q_e after dgrad)
 
 __global__ void absmax_i32_kernel(const int32_t *__restrict__ src, size_t n, DeviceState *dev)
@@ -530,6 +564,18 @@ cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst,
         absmax_f32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
     }
     quantize_f32_kernel<<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(mode, src, n, dst, dst_exp, dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_image(const float *src, size_t pixels, int c_src, int c_dst, int8_t *dst, int32_t *dst_exp,
+                                  DeviceState *dev, int sm_count, cudaStream_t s)
+{
+    cudaError_t e = launch_reset_cells(dev, s);
+    if (e != cudaSuccess) return e;
+    const size_t n = pixels * c_src;
+    absmax_f32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
+    quantize_image_kernel<<<grid_for(pixels * (c_dst / 16), sm_count), kThreads, 0, s>>>(src, pixels, c_src, c_dst, dst,
+                                                                                         dst_exp, dev);
     return cudaGetLastError();
 }
 

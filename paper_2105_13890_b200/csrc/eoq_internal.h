@@ -22,12 +22,25 @@ struct DeviceState {
     unsigned tensor_absmax[256];  // per-tensor maxima of the multi-tensor update
 };
 
+struct ProfRecord {
+    int kind;
+    cudaEvent_t begin, end;
+};
+
 struct Handle {
     int device;
     int sm_count;
     int last_cuda_error;
     DeviceState *dev;
+    unsigned long long launches;  // kernels launched through this handle
+    bool profiling;
+    int num_records;
+    ProfRecord *records;          // kMaxProfRecords entries, allocated on first eoq_profile_start
 };
+constexpr int kMaxProfRecords = 8192;
+
+// Counts `n` kernel launches on the handle.
+inline void count_launches(Handle *h, int n) { h->launches += (unsigned long long)n; }
 
 // ---------------------------------------------------------------------------------------------
 // Implicit-GEMM kernel used by the forward pass and by error back-propagation.
@@ -108,6 +121,8 @@ cudaError_t launch_wgrad(const WgradParams &p, const CUtensorMap &map_x, const C
 // Elementwise / reduction kernels
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_reset_cells(DeviceState *dev, cudaStream_t s);
+cudaError_t launch_quantize_image(const float *src, size_t pixels, int c_src, int c_dst, int8_t *dst, int32_t *dst_exp,
+                                  DeviceState *dev, int sm_count, cudaStream_t s);
 cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst, int32_t *dst_exp, DeviceState *dev,
                                 int sm_count, cudaStream_t s);
 cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,

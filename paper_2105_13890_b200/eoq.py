@@ -23,9 +23,10 @@ EOQ_PASS_FWD, EOQ_PASS_DGRAD, EOQ_PASS_WGRAD = 0, 1, 2
 
 EXPORTS = [
     "eoq_create", "eoq_destroy", "eoq_workspace_size", "eoq_conv_fwd", "eoq_conv_dgrad", "eoq_conv_wgrad",
-    "eoq_quantize", "eoq_err_prescale", "eoq_update", "eoq_layout_convert", "eoq_last_status",
-    "eoq_last_cuda_error", "eoq_status_string",
+    "eoq_quantize", "eoq_quantize_image", "eoq_err_prescale", "eoq_update", "eoq_layout_convert", "eoq_last_status",
+    "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count",
 ]
+EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
 
 
 class EoqError(RuntimeError):
@@ -76,11 +77,16 @@ def lib() -> C.CDLL:
         L.eoq_layout_convert.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp]
         L.eoq_last_status.argtypes = [vp, vp, C.POINTER(C.c_uint)]
         L.eoq_last_cuda_error.argtypes = [vp]
+        L.eoq_quantize_image.argtypes = [vp, vp, sz, C.c_int, C.c_int, vp, vp, vp]
+        L.eoq_profile_start.argtypes = [vp]
+        L.eoq_profile_stop.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_double)]
+        L.eoq_launch_count.argtypes = [vp]
         L.eoq_status_string.argtypes = [C.c_int]
         L.eoq_status_string.restype = C.c_char_p
         for name in EXPORTS:
-            if name != "eoq_status_string":
+            if name not in ("eoq_status_string", "eoq_launch_count"):
                 getattr(L, name).restype = C.c_int
+        L.eoq_launch_count.restype = C.c_ulonglong
         _lib = L
     return _lib
 
@@ -207,3 +213,27 @@ def eoq_last_status(handle, stream=None) -> int:
 
 def eoq_last_cuda_error(handle) -> int:
     return lib().eoq_last_cuda_error(handle)
+
+
+def eoq_quantize_image(handle, src, pixels, c_src, c_dst, dst, dst_exp, stream=None, check: bool = True) -> int:
+    st = lib().eoq_quantize_image(handle, _ptr(src), int(pixels), int(c_src), int(c_dst), _ptr(dst), _ptr(dst_exp),
+                                  _stream(stream))
+    if check:
+        _check(st, "eoq_quantize_image")
+    return st
+
+
+def eoq_profile_start(handle) -> None:
+    _check(lib().eoq_profile_start(handle), "eoq_profile_start")
+
+
+def eoq_profile_stop(handle):
+    """-> ([launches per kind], [milliseconds per kind]) for kinds EOQ_PROF_IGEMM_FWD, _IGEMM_DGRAD, _WGRAD."""
+    n = (C.c_int * 3)()
+    ms = (C.c_double * 3)()
+    _check(lib().eoq_profile_stop(handle, n, ms), "eoq_profile_stop")
+    return list(n), list(ms)
+
+
+def eoq_launch_count(handle) -> int:
+    return int(lib().eoq_launch_count(handle))

@@ -1,0 +1,137 @@
+"""One training step's worth of hot-path calls over a workload (buffer plumbing only; all arithmetic is in libeoq).
+
+For every quantized convolution layer of the network the step runs, through the C ABI:
+  forward      eoq_conv_fwd     x0 -> x5 (+ x2 when gamma is trainable, + ReLU mask)
+  error head   eoq_err_prescale e0, mask -> e3 (+ the sums behind g_b2 and g_gamma)
+  dgrad        eoq_conv_dgrad   e3 -> e4          (not for the first layer)
+  wgrad        eoq_conv_wgrad   e3, x0 -> g_w
+and then one eoq_update over all weight tensors.  The network input is quantized by eoq_quantize_image at
+the start of every step.  Layers are fed seeded synthetic tensors of the right shape and distribution
+(post-ReLU codes as inputs, rounded-normal codes as incoming errors); pooling, the float classifier and the
+residual error joins between layers are not part of this path.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import eoq, synth
+from .workloads import Layer, Workload, init_weight_f32
+
+
+@dataclass
+class Scalars:
+    """Integer codes (p = -7) of the layer scalars used for every layer of a step."""
+    b1_c: int = -2
+    gamma_c: int = 118
+    b2_c: int = 3
+
+
+class LayerBuffers:
+    def __init__(self, layer: Layer, dev):
+        self.layer = layer
+        self.desc = eoq.conv_desc(layer.n, layer.h, layer.w, layer.c_in, layer.c_out, layer.k, layer.k, layer.stride, layer.pad)
+        i8, dev_ = torch.int8, dev
+        out_shape = (layer.n, layer.ho, layer.wo, layer.c_out)
+        in_shape = (layer.n, layer.h, layer.w, layer.c_in)
+        self.x0 = torch.empty(in_shape, dtype=i8, device=dev_)
+        self.w = torch.empty((layer.c_out, layer.k, layer.k, layer.c_in), dtype=i8, device=dev_)
+        self.x5 = torch.empty(out_shape, dtype=i8, device=dev_)
+        self.x2 = torch.empty(out_shape, dtype=torch.int16, device=dev_) if layer.gamma_trainable else None
+        n_out = int(np.prod(out_shape))
+        self.mask = torch.empty((n_out + 7) // 8, dtype=torch.uint8, device=dev_) if layer.relu else None
+        self.shortcut = torch.empty(out_shape, dtype=i8, device=dev_) if layer.shortcut else None
+        self.e0 = torch.empty(out_shape, dtype=i8, device=dev_)
+        self.e0_exp = torch.full((1,), -12, dtype=torch.int32, device=dev_)
+        self.e3 = torch.empty(out_shape, dtype=i8, device=dev_)
+        self.e3_exp = torch.zeros(1, dtype=torch.int32, device=dev_)
+        self.e4 = torch.empty(in_shape, dtype=i8, device=dev_) if layer.has_dgrad else None
+        self.e4_exp = torch.zeros(1, dtype=torch.int32, device=dev_)
+        self.sum_e4 = torch.zeros(1, dtype=torch.int64, device=dev_)
+        self.sum_e1 = torch.zeros(1, dtype=torch.int64, device=dev_)
+        self.sum_e1x2 = torch.zeros(1, dtype=torch.int64, device=dev_)
+        self.g = torch.empty_like(self.w)
+        self.g_exp = torch.zeros(1, dtype=torch.int32, device=dev_)
+        self.n_out = n_out
+
+
+class TrainStep:
+    """Allocates device buffers for a workload, fills them with seeded synthetic data, and runs steps."""
+
+    def __init__(self, workload: Workload, handle: int, device: str = "cuda:0", seed: int = synth.BASE_SEED,
+                 scalars: Optional[Scalars] = None, lr_mant: int = 1, lr_exp: int = -6, image_channels: int = 3):
+        self.wl, self.h, self.dev = workload, handle, torch.device(device)
+        self.sc = scalars or Scalars()
+        self.lr_mant, self.lr_exp = lr_mant, lr_exp
+        self.step_no = 0
+        self.layers: List[LayerBuffers] = [LayerBuffers(l, self.dev) for l in workload.layers]
+        ws = 256
+        for lb in self.layers:
+            for p in (eoq.EOQ_PASS_FWD, eoq.EOQ_PASS_DGRAD, eoq.EOQ_PASS_WGRAD):
+                ws = max(ws, eoq.eoq_workspace_size(lb.desc, p))
+        self.workspace = torch.empty(ws, dtype=torch.uint8, device=self.dev)
+        first = workload.layers[0]
+        self.image_channels = image_channels
+        self.image_pixels = first.n * first.h * first.w
+        self.image = torch.empty((first.n, first.h, first.w, image_channels), dtype=torch.float32, device=self.dev)
+        self.image_exp = torch.zeros(1, dtype=torch.int32, device=self.dev)
+        self._fill(seed)
+
+    # ------------------------------------------------------------------ synthetic data (host side, numpy)
+    def host_image(self, seed: int) -> np.ndarray:
+        f = self.wl.layers[0]
+        return synth.normal_f32((f.n, f.h, f.w, self.image_channels), seed, 0)
+
+    def _fill(self, seed: int) -> None:
+        self.image.copy_(torch.from_numpy(self.host_image(seed)))
+        pools = {}
+
+        def pooled(kind, shape, stream):
+            key = (kind, tuple(shape))
+            if key not in pools:
+                gen = {"relu": synth.relu_codes, "err": synth.normal_codes, "uni": synth.int8_uniform}[kind]
+                pools[key] = torch.from_numpy(gen(shape, seed, stream))
+            return pools[key]
+
+        for i, lb in enumerate(self.layers):
+            l = lb.layer
+            if i > 0:
+                lb.x0.copy_(pooled("relu", lb.x0.shape, 1))
+            lb.e0.copy_(pooled("err", lb.e0.shape, 2))
+            if lb.shortcut is not None:
+                lb.shortcut.copy_(pooled("relu", lb.shortcut.shape, 3))
+            wf = init_weight_f32(l, self.wl, synth.normal_f64(tuple(lb.w.shape), seed, 100 + i))
+            wf_d = torch.from_numpy(wf).to(self.dev)
+            eoq.eoq_quantize(self.h, eoq.EOQ_CQ, wf_d, True, None, wf_d.numel(), lb.w)  # Q_w, once at initialisation
+        torch.cuda.synchronize(self.dev)
+
+    # ------------------------------------------------------------------ one step
+    def run(self) -> None:
+        h, sc, ws = self.h, self.sc, self.workspace
+        first = self.layers[0]
+        eoq.eoq_quantize_image(h, self.image, self.image_pixels, self.image_channels, first.layer.c_in, first.x0,
+                               self.image_exp)
+        for i, lb in enumerate(self.layers):
+            l = lb.layer
+            gamma = sc.gamma_c if l.gamma_trainable else 128
+            eoq.eoq_conv_fwd(h, lb.desc, lb.x0, self.image_exp if i == 0 else None, 0 if i == 0 else sc.b1_c, lb.w,
+                             gamma, sc.b2_c if l.relu else 0, lb.shortcut, l.relu, lb.x5, lb.x2, lb.mask, None, ws)
+        for i in range(len(self.layers) - 1, -1, -1):
+            lb = self.layers[i]
+            l = lb.layer
+            gamma = sc.gamma_c if l.gamma_trainable else 128
+            eoq.eoq_err_prescale(h, lb.e0, lb.e0_exp, lb.mask, lb.x2, lb.n_out, gamma, lb.e3, lb.e3_exp, lb.sum_e1,
+                                 lb.sum_e1x2 if lb.x2 is not None else None)
+            if l.has_dgrad:
+                eoq.eoq_conv_dgrad(h, lb.desc, lb.e3, lb.e3_exp, lb.w, lb.e4, lb.e4_exp, lb.sum_e4, None, ws)
+            eoq.eoq_conv_wgrad(h, lb.desc, lb.e3, lb.e3_exp, lb.x0, 0 if i == 0 else sc.b1_c, lb.g, lb.g_exp, None, ws)
+        eoq.eoq_update(h, [lb.w for lb in self.layers], [lb.g for lb in self.layers], [lb.g_exp for lb in self.layers],
+                       self.lr_mant, self.lr_exp, eoq.EOQ_ROUND_STOCHASTIC, seed=synth.BASE_SEED, step=self.step_no)
+        self.step_no += 1
+
+    def result_tensors(self):
+        """Small per-step results a caller would read back: every gradient exponent and the last activation."""
+        return [lb.g_exp for lb in self.layers] + [self.layers[-1].x5]
