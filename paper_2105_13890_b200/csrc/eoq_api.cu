@@ -355,8 +355,9 @@ extern "C" int eoq_workspace_size(const eoq_conv_desc_t *desc, int pass, size_t 
         case EOQ_PASS_DGRAD:  // transposed weights + int32 sums
             *bytes = round256(g.w_elems) + round256(g.in_elems * sizeof(int32_t));
             return EOQ_OK;
-        case EOQ_PASS_WGRAD:  // int64 sums + per-tap error sums
-            *bytes = round256(g.w_elems * sizeof(long long)) + round256((size_t)desc->c_out * g.taps * sizeof(long long));
+        case EOQ_PASS_WGRAD:  // int64 sums + per-tap error sums + per-class error sums
+            *bytes = round256(g.w_elems * sizeof(long long)) + round256((size_t)desc->c_out * g.taps * sizeof(long long)) +
+                     round256(b1_error_scratch_bytes(*desc, bc));
             return EOQ_OK;
         default: return EOQ_ERR_BAD_ARG;
     }
@@ -427,6 +428,7 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     p.dev = h->dev;
     if (b1_c != 0) {
         const BorderClasses bc = border_classes(d, g);
+        if (bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
         p.b1_table = reinterpret_cast<const int32_t *>(workspace);
         p.b1_nlo_h = bc.nlo_h; p.b1_nhi_h = bc.nhi_h; p.b1_nrc = bc.nrc;
         p.b1_nlo_w = bc.nlo_w; p.b1_nhi_w = bc.nhi_w; p.b1_ncc = bc.ncc;
@@ -612,8 +614,12 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
 
     cudaError_t e = cudaMemsetAsync(acc, 0, g.w_elems * sizeof(long long), s);
     if (e == cudaSuccess && b1_c != 0) {
-        e = launch_b1_error_sums(e3, tap_sums, d, g.ho, g.wo, s);
-        count_launches(h, 1);
+        const BorderClasses bc = border_classes(d, g);
+        if (bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
+        long long *class_sums = reinterpret_cast<long long *>(reinterpret_cast<char *>(tap_sums) +
+                                                              round256((size_t)d.c_out * g.taps * sizeof(long long)));
+        e = launch_b1_error_sums(e3, tap_sums, class_sums, d, g.ho, g.wo, bc, h->sm_count, s);
+        count_launches(h, 2);
     }
     if (e != cudaSuccess) return record(h, e);
     CUtensorMap map_x, map_e;

@@ -60,6 +60,34 @@ __device__ __forceinline__ int32_t sq_code64(long long a, int t)
     return (int32_t)(v < -127 ? -127 : (v > 127 ? 127 : v));
 }
 
+// ------------------------------------------------------------------ border classes of the b1 term
+// x1 = x0 + b1 has a zero halo, so conv(x1) = conv(x0) + b1 * (sum of the weights of the taps that fall
+// inside the image).  Which taps are inside depends only on how far the output row (column) is from the
+// image border: rows whose window sticks out at the top (y < nlo) or at the bottom (y >= extent - nhi) get a
+// class each, all interior rows share class nlo.  When the image is so small that no interior row exists
+// (ncls == extent) every row is its own class.
+
+__device__ __forceinline__ int border_class(int y, int extent, int nlo, int nhi, int ncls)
+{
+    if (ncls == extent) return y;
+    if (y < nlo) return y;
+    if (y >= extent - nhi) return nlo + 1 + (y - (extent - nhi));
+    return nlo;
+}
+
+// Is filter tap k inside the image for the rows of class `cls`?
+__device__ __forceinline__ bool tap_valid(int cls, int k, int extent_out, int extent_in, int nlo, int nhi, int ncls,
+                                          int stride, int pad)
+{
+    int y;
+    if (ncls == extent_out) y = cls;
+    else if (cls < nlo) y = cls;
+    else if (cls == nlo) y = nlo;
+    else y = extent_out - nhi + (cls - nlo - 1);
+    const int src = y * stride - pad + k;
+    return src >= 0 && src < extent_in;
+}
+
 // ------------------------------------------------------------------ warp reductions
 
 __device__ __forceinline__ uint32_t warp_max_u32(uint32_t v)

@@ -483,65 +483,104 @@ __global__ void weight_transpose_kernel(const int8_t *__restrict__ w, int8_t *__
 
 // ------------------------------------------------------------------ b1 support
 
-// Is filter tap k inside the image for the rows of class `cls`?
-__device__ __forceinline__ bool tap_valid(int cls, int k, int extent_out, int extent_in, int nlo, int nhi, int ncls,
-                                          int stride, int pad)
-{
-    int y;
-    if (ncls == extent_out) y = cls;
-    else if (cls < nlo) y = cls;
-    else if (cls == nlo) y = nlo;
-    else y = extent_out - nhi + (cls - nlo - 1);
-    const int src = y * stride - pad + k;
-    return src >= 0 && src < extent_in;
-}
-
 // table[class][oc] = sum over the taps valid for the class, and over ic, of w[oc][tap][ic]  (the forward
 // pass adds b1 times this: conv(x0 + b1) = conv(x0) + b1 * conv(indicator of the image)).
+// One block per output channel: warps reduce the taps' channel sums, then threads combine them per class.
 __global__ void b1_weight_table_kernel(const int8_t *__restrict__ w, int32_t *table, eoq_conv_desc_t d, int ho, int wo,
                                        BorderClasses bc)
 {
-    const int oc = blockIdx.x * blockDim.x + threadIdx.x;
-    const int cls = blockIdx.y;
-    if (oc >= d.c_out) return;
-    const int rc = cls / bc.ncc, cc = cls % bc.ncc;
-    int32_t sum = 0;
-    for (int kh = 0; kh < d.kh; ++kh) {
-        if (!tap_valid(rc, kh, ho, d.h, bc.nlo_h, bc.nhi_h, bc.nrc, d.stride, d.pad)) continue;
-        for (int kw = 0; kw < d.kw; ++kw) {
-            if (!tap_valid(cc, kw, wo, d.w, bc.nlo_w, bc.nhi_w, bc.ncc, d.stride, d.pad)) continue;
-            const int8_t *p = w + (((size_t)oc * d.kh + kh) * d.kw + kw) * d.c_in;
-            for (int ic = 0; ic < d.c_in; ++ic) sum += p[ic];
+    __shared__ int32_t tap_sum[kMaxTaps];
+    const int oc = blockIdx.x;
+    const int taps = d.kh * d.kw;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    for (int t = warp; t < taps; t += nwarps) {
+        const int4 *p = reinterpret_cast<const int4 *>(w + ((size_t)oc * taps + t) * d.c_in);
+        int sum = 0;
+        for (int i = lane; i < d.c_in / 16; i += 32) {
+            const int4 v = __ldg(p + i);
+            sum = __dp4a(v.x, 0x01010101, sum);
+            sum = __dp4a(v.y, 0x01010101, sum);
+            sum = __dp4a(v.z, 0x01010101, sum);
+            sum = __dp4a(v.w, 0x01010101, sum);
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == 0) tap_sum[t] = sum;
     }
-    table[(size_t)cls * d.c_out + oc] = sum;
+    __syncthreads();
+    for (int cls = threadIdx.x; cls < bc.nrc * bc.ncc; cls += blockDim.x) {
+        const int rc = cls / bc.ncc, cc = cls % bc.ncc;
+        int32_t sum = 0;
+        for (int kh = 0; kh < d.kh; ++kh) {
+            if (!tap_valid(rc, kh, ho, d.h, bc.nlo_h, bc.nhi_h, bc.nrc, d.stride, d.pad)) continue;
+            for (int kw = 0; kw < d.kw; ++kw)
+                if (tap_valid(cc, kw, wo, d.w, bc.nlo_w, bc.nhi_w, bc.ncc, d.stride, d.pad)) sum += tap_sum[kh * d.kw + kw];
+        }
+        table[(size_t)cls * d.c_out + oc] = sum;
+    }
 }
 
-// tap_sums[oc][tap] = sum of e3[n,y,x,oc] over the pixels whose tap falls inside the image (the weight
-// gradient adds b1 times this to every input channel).  One block per (tap, channel group).
-__global__ void b1_error_sums_kernel(const int8_t *__restrict__ e3, long long *tap_sums, eoq_conv_desc_t d, int ho, int wo)
+// class_sums[class][oc] = sum of e3[n,y,x,oc] over the pixels of a border class.  A block owns a range of
+// pixels and a slab of 128 channels; each lane keeps 4 channels.  Interior pixels (one class, almost all of a
+// large image) accumulate in registers, border pixels in shared memory.
+constexpr int kClassSlab = 128;
+__global__ void b1_class_sums_kernel(const int8_t *__restrict__ e3, long long *class_sums, int c_out, int ho, int wo,
+                                     size_t pixels, int pixels_per_block, BorderClasses bc)
 {
-    const int tap = blockIdx.y;
-    const int kh = tap / d.kw, kw = tap % d.kw;
-    const int oc = blockIdx.x * 32 + (threadIdx.x & 31);
-    const int lanes = blockDim.x >> 5, slot = threadIdx.x >> 5;
-    long long sum = 0;
-    if (oc < d.c_out) {
-        const size_t pixels = (size_t)d.n * ho * wo;
-        for (size_t p = (size_t)blockIdx.z * lanes + slot; p < pixels; p += (size_t)gridDim.z * lanes) {
-            const int x = (int)(p % wo), y = (int)((p / wo) % ho);
-            const int sy = y * d.stride - d.pad + kh, sx = x * d.stride - d.pad + kw;
-            if (sy >= 0 && sy < d.h && sx >= 0 && sx < d.w) sum += e3[p * d.c_out + oc];
+    extern __shared__ int32_t cls_acc[];  // [classes][kClassSlab]
+    const int classes = bc.nrc * bc.ncc;
+    for (int i = threadIdx.x; i < classes * kClassSlab; i += blockDim.x) cls_acc[i] = 0;
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int ch = blockIdx.y * kClassSlab + lane * 4;
+    const bool live = ch < c_out;
+    const int interior = (bc.nrc != ho && bc.ncc != wo) ? bc.nlo_h * bc.ncc + bc.nlo_w : -1;
+    int a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+    const size_t begin = (size_t)blockIdx.x * pixels_per_block;
+    const size_t end = min(pixels, begin + (size_t)pixels_per_block);
+    for (size_t p = begin + warp; p < end; p += nwarps) {
+        const int x = (int)(p % wo), y = (int)((p / wo) % ho);
+        const int cls = border_class(y, ho, bc.nlo_h, bc.nhi_h, bc.nrc) * bc.ncc + border_class(x, wo, bc.nlo_w, bc.nhi_w, bc.ncc);
+        if (!live) continue;
+        const int v = __ldg(reinterpret_cast<const int *>(e3 + p * c_out + ch));
+        const int b0 = (int)(int8_t)(v & 0xff), b1 = (int)(int8_t)((v >> 8) & 0xff), b2 = (int)(int8_t)((v >> 16) & 0xff), b3 = v >> 24;
+        if (cls == interior) {
+            a0 += b0; a1 += b1; a2 += b2; a3 += b3;
+        } else {
+            int32_t *dst = cls_acc + cls * kClassSlab + lane * 4;
+            atomicAdd(dst + 0, b0); atomicAdd(dst + 1, b1); atomicAdd(dst + 2, b2); atomicAdd(dst + 3, b3);
         }
     }
-    __shared__ long long part[32][33];
-    part[slot][threadIdx.x & 31] = sum;
-    __syncthreads();
-    if (slot == 0 && oc < d.c_out) {
-        long long s = 0;
-        for (int k = 0; k < lanes; ++k) s += part[k][threadIdx.x & 31];
-        if (s) atomicAdd(reinterpret_cast<unsigned long long *>(tap_sums + (size_t)oc * (d.kh * d.kw) + tap), (unsigned long long)s);
+    if (live && interior >= 0) {
+        int32_t *dst = cls_acc + interior * kClassSlab + lane * 4;
+        atomicAdd(dst + 0, a0); atomicAdd(dst + 1, a1); atomicAdd(dst + 2, a2); atomicAdd(dst + 3, a3);
     }
+    __syncthreads();
+    for (int i = threadIdx.x; i < classes * kClassSlab; i += blockDim.x) {
+        const int c = blockIdx.y * kClassSlab + (i % kClassSlab);
+        const int32_t v = cls_acc[i];
+        if (v && c < c_out)
+            atomicAdd(reinterpret_cast<unsigned long long *>(class_sums + (size_t)(i / kClassSlab) * c_out + c), (unsigned long long)(long long)v);
+    }
+}
+
+// tap_sums[oc][tap] = sum of the class sums of the classes for which the tap falls inside the image
+// (the weight gradient adds b1 times this to every input channel).
+__global__ void b1_tap_sums_kernel(const long long *__restrict__ class_sums, long long *tap_sums, eoq_conv_desc_t d, int ho,
+                                   int wo, BorderClasses bc)
+{
+    const int taps = d.kh * d.kw;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= d.c_out * taps) return;
+    const int oc = i / taps, tap = i % taps, kh = tap / d.kw, kw = tap % d.kw;
+    long long sum = 0;
+    for (int rc = 0; rc < bc.nrc; ++rc) {
+        if (!tap_valid(rc, kh, ho, d.h, bc.nlo_h, bc.nhi_h, bc.nrc, d.stride, d.pad)) continue;
+        for (int cc = 0; cc < bc.ncc; ++cc)
+            if (tap_valid(cc, kw, wo, d.w, bc.nlo_w, bc.nhi_w, bc.ncc, d.stride, d.pad))
+                sum += class_sums[(size_t)(rc * bc.ncc + cc) * d.c_out + oc];
+    }
+    tap_sums[i] = sum;
 }
 
 }  // namespace
@@ -681,21 +720,33 @@ cudaError_t launch_b1_weight_table(const int8_t *w, int32_t *table, const eoq_co
                                    cudaStream_t s)
 {
     const int ho = (d.h + 2 * d.pad - d.kh) / d.stride + 1, wo = (d.w + 2 * d.pad - d.kw) / d.stride + 1;
-    dim3 grid((d.c_out + 127) / 128, bc.nrc * bc.ncc);
-    b1_weight_table_kernel<<<grid, 128, 0, s>>>(w, table, d, ho, wo, bc);
+    b1_weight_table_kernel<<<d.c_out, 128, 0, s>>>(w, table, d, ho, wo, bc);
     return cudaGetLastError();
 }
 
-cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, const eoq_conv_desc_t &d, int ho, int wo,
-                                 cudaStream_t s)
+size_t b1_error_scratch_bytes(const eoq_conv_desc_t &d, const BorderClasses &bc)
 {
-    cudaError_t e = cudaMemsetAsync(tap_sums, 0, sizeof(long long) * d.c_out * d.kh * d.kw, s);
+    return sizeof(long long) * (size_t)bc.nrc * bc.ncc * d.c_out;
+}
+
+cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, long long *class_sums, const eoq_conv_desc_t &d,
+                                 int ho, int wo, const BorderClasses &bc, int sm_count, cudaStream_t s)
+{
+    const int classes = bc.nrc * bc.ncc;
+    cudaError_t e = cudaMemsetAsync(class_sums, 0, b1_error_scratch_bytes(d, bc), s);
     if (e != cudaSuccess) return e;
     const size_t pixels = (size_t)d.n * ho * wo;
-    int zs = (int)((pixels + 4095) / 4096);
-    zs = zs < 1 ? 1 : (zs > 64 ? 64 : zs);
-    dim3 grid((d.c_out + 31) / 32, d.kh * d.kw, zs);
-    b1_error_sums_kernel<<<grid, 1024, 0, s>>>(e3, tap_sums, d, ho, wo);
+    const int slabs = (d.c_out + kClassSlab - 1) / kClassSlab;
+    int blocks = (4 * sm_count + slabs - 1) / slabs;
+    size_t ppb = (pixels + blocks - 1) / blocks;
+    if (ppb < 64) ppb = 64;
+    if (ppb > (1u << 23)) ppb = 1u << 23;  // keeps the int32 class sums exact
+    blocks = (int)((pixels + ppb - 1) / ppb);
+    dim3 grid(blocks, slabs);
+    b1_class_sums_kernel<<<grid, 256, sizeof(int32_t) * classes * kClassSlab, s>>>(e3, class_sums, d.c_out, ho, wo, pixels,
+                                                                                 (int)ppb, bc);
+    const int n = d.c_out * d.kh * d.kw;
+    b1_tap_sums_kernel<<<(n + 255) / 256, 256, 0, s>>>(class_sums, tap_sums, d, ho, wo, bc);
     return cudaGetLastError();
 }
 

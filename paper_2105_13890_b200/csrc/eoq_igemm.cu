@@ -35,16 +35,6 @@ __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d)
     return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) | ((uint32_t)(d & 0xff) << 24);
 }
 
-// Row class of an output coordinate for the b1 border table: rows whose filter window leaves the image
-// at the top (y < nlo) or at the bottom (y >= extent - nhi) each get a class; the interior shares one.
-__device__ __forceinline__ int border_class(int y, int extent, int nlo, int nhi, int ncls)
-{
-    if (ncls == extent) return y;
-    if (y < nlo) return y;
-    if (y >= extent - nhi) return nlo + 1 + (y - (extent - nhi));
-    return nlo;
-}
-
 // Forward chain on 16 consecutive output channels of one pixel (Sec. 3.2.1: x2 = Q_a1(conv), x3 = gamma x2,
 // x4 = x3 + b2 [+ shortcut], x5 = Q_a2(relu(x4)); mask = [x4 > 0]).
 __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t *acc, size_t off, int col, int cls,

@@ -151,7 +151,9 @@ struct BorderClasses {
 };
 cudaError_t launch_b1_weight_table(const int8_t *w, int32_t *table, const eoq_conv_desc_t &d, const BorderClasses &bc,
                                    cudaStream_t s);
-cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, const eoq_conv_desc_t &d, int ho, int wo,
-                                 cudaStream_t s);
+size_t b1_error_scratch_bytes(const eoq_conv_desc_t &d, const BorderClasses &bc);
+cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, long long *class_sums, const eoq_conv_desc_t &d,
+                                 int ho, int wo, const BorderClasses &bc, int sm_count, cudaStream_t s);
+constexpr int kMaxBorderClasses = 64;  // classes (rows x columns) the b1 kernels keep in shared memory
 
 }  // namespace eoq
