@@ -114,6 +114,31 @@ EOQ_API int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
                    void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * eoq_conv_dgrad without any allocation (the paper has no counterpart; this is a deployment variant).
+ * Some callers may not allocate device memory at all: code running inside a memory pool that owns the whole
+ * device, a plugin loaded into a host application that forbids cudaMalloc after start-up, or a real-time loop
+ * where an allocation's implicit synchronisation is not acceptable.  Such callers cannot use eoq_create (it
+ * allocates the handle's device state) nor supply a workspace.  This entry point needs neither: every byte of
+ * scratch -- reduction cells, transposed weights, int32 sums -- sits in one static device array of
+ * EOQ_STATIC_SCRATCH_BYTES (+4 KiB of cells) that is part of the library image, so each GPU that loads the
+ * library carries it until the process exits.  It calls no cudaMalloc, cudaFree or allocating library routine.
+ *
+ * Arguments and results are those of eoq_conv_dgrad (same kernels, bit-identical outputs); there is no handle,
+ * no workspace and no acc_dump.  status_out (device, optional) receives the EOQ_DEV_* bits of this call.
+ * Limits and rules:
+ *   - geometries whose eoq_workspace_size(desc, EOQ_PASS_DGRAD) exceeds EOQ_STATIC_SCRATCH_BYTES are rejected
+ *     with EOQ_ERR_WORKSPACE and nothing is launched;
+ *   - the first call on a device resolves the array's device address and reads device attributes (no
+ *     allocation); make that first call outside any stream capture, with the device current;
+ *   - all calls on a device share the one array, which keeps the previous call's contents: the cells that must
+ *     start at zero are cleared on the stream at the start of each call, and two calls that overlap on the GPU
+ *     (different streams, no ordering between them) race on it -- order them.
+ */
+#define EOQ_STATIC_SCRATCH_BYTES (16u << 20)
+EOQ_API int eoq_conv_dgrad_static(const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp, const int8_t *w,
+                          int8_t *e4, int32_t *e4_exp, int64_t *sum_e4, uint32_t *status_out, void *stream);
+
+/*
  * Weight gradient (Sec. 3.2.1, third equation block): g_w = Q_g(e3 * x1), the correlation of the
  * error with x1 = x0 + Q_b(b1) (zero halo), summed exactly over batch and space, followed by SQ.
  * device in : e3 and *e3_exp as above; x = x0 [n,h,w,c_in] int8.   host in: b1_c.

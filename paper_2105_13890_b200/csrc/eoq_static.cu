@@ -1,0 +1,76 @@
+// eoq_conv_dgrad_static: error back-propagation for callers that cannot allocate device memory.
+// All scratch (the reduction cells, the transposed weights, the int32 sums) lives in one file-scope device
+// array that every GPU loading the library carries until the process exits.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "eoq_internal.h"
+
+using namespace eoq;
+
+namespace {
+
+constexpr size_t kStaticHeaderBytes = 4096;  // reduction cells and status word (a DeviceState)
+constexpr size_t kStaticScratchBytes = (size_t)EOQ_STATIC_SCRATCH_BYTES;
+static_assert(sizeof(DeviceState) <= kStaticHeaderBytes, "header too small");
+
+// In host code this name is only a handle for the runtime: its device address comes from
+// cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticHeaderBytes + kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+struct PerDevice {
+    bool ready;
+    unsigned char *scratch;  // device address of g_static_scratch on this device
+    int sm_count;
+};
+PerDevice g_per_device[kMaxDevices];
+
+}  // namespace
+
+extern "C" int eoq_conv_dgrad_static(const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                                     const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4,
+                                     uint32_t *status_out, void *stream)
+{
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return EOQ_ERR_CUDA;
+    PerDevice &pd = g_per_device[device];
+    if (!pd.ready) {
+        // first call on this device: resolve the array's device address and the SM count (no allocation)
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return EOQ_ERR_CUDA;
+        int sms = 0, major = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return EOQ_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) return EOQ_ERR_CUDA;
+        if (major != 10) return EOQ_ERR_UNSUPPORTED;
+        pd.scratch = static_cast<unsigned char *>(ptr);
+        pd.sm_count = sms;
+        pd.ready = true;
+    }
+    size_t need = 0;
+    int st = eoq_workspace_size(desc, EOQ_PASS_DGRAD, &need);
+    if (st != EOQ_OK) return st;
+    if (need > kStaticScratchBytes) return EOQ_ERR_WORKSPACE;  // geometry needs more scratch than the array holds
+
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    // the array keeps what the previous call left: the status word and the cells must start at zero
+    if (cudaMemsetAsync(pd.scratch, 0, sizeof(DeviceState), s) != cudaSuccess) return EOQ_ERR_CUDA;
+
+    Handle h;  // host-side bookkeeping only; its device state is the head of the static array
+    h.device = device;
+    h.sm_count = pd.sm_count;
+    h.last_cuda_error = 0;
+    h.dev = reinterpret_cast<DeviceState *>(pd.scratch);
+    h.launches = 0;
+    h.profiling = false;
+    h.num_records = 0;
+    h.records = nullptr;
+    st = eoq_conv_dgrad(reinterpret_cast<eoq_handle_t>(&h), desc, e3, e3_exp, w, e4, e4_exp, sum_e4, nullptr,
+                        pd.scratch + kStaticHeaderBytes, kStaticScratchBytes, stream);
+    if (st != EOQ_OK) return st;
+    if (status_out &&
+        cudaMemcpyAsync(status_out, pd.scratch + offsetof(DeviceState, status), sizeof(uint32_t),
+                        cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return EOQ_ERR_CUDA;
+    return EOQ_OK;
+}

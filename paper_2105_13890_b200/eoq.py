@@ -25,7 +25,9 @@ EXPORTS = [
     "eoq_create", "eoq_destroy", "eoq_workspace_size", "eoq_conv_fwd", "eoq_conv_dgrad", "eoq_conv_wgrad",
     "eoq_quantize", "eoq_quantize_image", "eoq_err_prescale", "eoq_update", "eoq_layout_convert", "eoq_last_status",
     "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count",
+    "eoq_conv_dgrad_static",
 ]
+EOQ_STATIC_SCRATCH_BYTES = 16 << 20
 EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
 
 
@@ -77,6 +79,7 @@ def lib() -> C.CDLL:
         L.eoq_layout_convert.argtypes = [vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp]
         L.eoq_last_status.argtypes = [vp, vp, C.POINTER(C.c_uint)]
         L.eoq_last_cuda_error.argtypes = [vp]
+        L.eoq_conv_dgrad_static.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.eoq_quantize_image.argtypes = [vp, vp, sz, C.c_int, C.c_int, vp, vp, vp]
         L.eoq_profile_start.argtypes = [vp]
         L.eoq_profile_stop.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_double)]
@@ -237,3 +240,13 @@ def eoq_profile_stop(handle):
 
 def eoq_launch_count(handle) -> int:
     return int(lib().eoq_launch_count(handle))
+
+
+def eoq_conv_dgrad_static(desc, e3, e3_exp, w, e4, e4_exp, sum_e4=None, status_out=None, stream=None,
+                          check: bool = True) -> int:
+    """eoq_conv_dgrad for callers that may not allocate: no handle, no workspace (scratch is a static device array)."""
+    st = lib().eoq_conv_dgrad_static(C.byref(desc), _ptr(e3), _ptr(e3_exp), _ptr(w), _ptr(e4), _ptr(e4_exp),
+                                     _ptr(sum_e4), _ptr(status_out), _stream(stream))
+    if check:
+        _check(st, "eoq_conv_dgrad_static")
+    return st
