@@ -46,7 +46,7 @@ class ClockSampler:
         self.proc, self.lines = None, []
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(index)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "20", "-i", str(index)], stdout=subprocess.PIPE, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -175,24 +175,16 @@ def run_reference(args):
 
 def run_gpu(args):
     import torch
-    import torch.distributed as dist
 
-    from paper_2105_13890_b200 import eoq, workloads
+    from paper_2105_13890_b200 import eoq, ranks, workloads
     from paper_2105_13890_b200.step import Scalars, TrainStep
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = ranks.world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+    ranks.init("nccl", torch.device("cuda", local))
+    barrier = ranks.barrier
 
     wl = workloads.get(args.workload, args.batch)
     handle = eoq.eoq_create(local)
@@ -244,21 +236,24 @@ def run_gpu(args):
     for _ in range(args.steps):
         step.run()
     prof_n, prof_ms = eoq.eoq_profile_stop(handle)
-    clocks = ClockSampler.summarize(sampler.window(t_wall0, t_wall1)) if sampler else None
+    t_wall2 = time.time()
+    # clocks while the GPU was under this load: the timed steps first, the whole loaded span if that is too short
+    clocks = None
     if sampler:
+        lines = sampler.window(t_wall0, t_wall1)
+        if len(lines) < 5:
+            lines = sampler.window(t_wall0, t_wall2)
+        clocks = ClockSampler.summarize(lines)
         sampler.stop()
 
-    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=f"cuda:{local}")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_e2e = t.tolist()
+    ms, ms_e2e = ranks.max_over_ranks([ms, ms_e2e], device=f"cuda:{local}")
 
     if rank == 0:
         pk = peaks()
         ops_step = wl.total_ops
         sec = ms / 1e3 / args.steps
-        tops = world * ops_step / sec / 1e12
-        tops_e2e = world * ops_step / (ms_e2e / 1e3 / args.steps) / 1e12
+        tops = ranks.whole_job_rate(ops_step, args.steps, ms, world) / 1e12
+        tops_e2e = ranks.whole_job_rate(ops_step, args.steps, ms_e2e, world) / 1e12
         int8_peak = pk["bf16_sustained"] * INT8_OVER_BF16
         fwd_ops = sum(2 * l.macs for l in wl.layers) * args.steps
         dgrad_ops = sum(2 * l.macs for l in wl.layers if l.has_dgrad) * args.steps
@@ -303,14 +298,13 @@ def run_gpu(args):
                                     "sample": f"{small.name}: every layer of the workload at batch {args.ref_batch}, one step"}
         print(json.dumps(line), flush=True)
     eoq.eoq_destroy(handle)
-    if world > 1:
-        dist.destroy_process_group()
+    ranks.finish()
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="eoq", choices=["eoq", "reference"])
     ap.add_argument("--workload", default="resnet18")
