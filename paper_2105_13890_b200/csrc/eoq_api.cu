@@ -167,9 +167,10 @@ void plan_igemm(IgemmParams &p, int src_channels, int ntaps, int sm_count)
     p.subs_per_stage = 128 / p.kc;
     if (p.subs_per_stage > p.num_sub) p.subs_per_stage = p.num_sub;
     p.num_m_tiles = (p.M + kTileM - 1) / kTileM;
-    // widest column tile that still gives every SM a tile; narrow ones only when the grid would starve
+    // An MMA costs at least ~57 cycles whatever its width and reaches the tensor peak only from 128 columns
+    // up, so tiles stay 128 wide even when that leaves some SMs without one; 256 when there are tiles to spare.
     int tn = p.N < 256 ? p.N : 256;
-    while (tn > 64 && tn % 32 == 0 && (long long)p.num_m_tiles * ((p.N + tn - 1) / tn) < sm_count) tn /= 2;
+    if (tn == 256 && (long long)p.num_m_tiles * ((p.N + 255) / 256) < 2LL * sm_count) tn = 128;
     p.tile_n = tn;
     p.num_n_tiles = (p.N + tn - 1) / tn;
     const size_t stage = (size_t)p.subs_per_stage * (kTileM + tn) * p.kc;
@@ -392,7 +393,7 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
         return EOQ_ERR_RANGE;
     const eoq_conv_desc_t &d = *desc;
     // the accumulator with its b1 term must fit int32: taps * c_in * (127 + |b1|) * 127 < 2^31
-    if ((double)g.taps * d.c_in * (127.0 + (b1_c < 0 ? -b1_c : b1_c)) * 127.0 >= 2147483647.0) return EOQ_ERR_RANGE;
+    if ((double)g.taps * d.c_in * (127.0 + (b1_c < 0 ? -b1_c : b1_c)) * 127.0 >= 2147483647.0 - 16777216.0) return EOQ_ERR_RANGE;
     if (b1_c != 0 && (st = check_workspace(desc, EOQ_PASS_FWD, workspace, workspace_bytes)) != EOQ_OK) return st;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
 

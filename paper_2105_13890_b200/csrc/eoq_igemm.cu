@@ -2,7 +2,7 @@
 // (arXiv 2105.13890, Sec. 3.2.1).  One persistent CTA per SM walks 128-row output tiles:
 //   warp 0   : TMA producer (im2col loads of the activation/error operand, tiled loads of the weights)
 //   warp 1   : owns tensor memory, issues tcgen05.mma kind::i8 (int8 x int8 -> int32 in TMEM)
-//   warps 2-5: epilogue; read the accumulators with tcgen05.ld and apply the layer's quantizers in registers
+//   warps 2-9: epilogue; read the accumulators with tcgen05.ld and apply the layer's quantizers in registers
 // Two accumulator buffers in TMEM let the epilogue of tile i overlap the main loop of tile i+1.
 // Every wait is bounded: when one runs out the CTA raises EOQ_DEV_TIMEOUT, drains and returns.
 #include "eoq_device.cuh"
@@ -35,8 +35,13 @@ __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d)
     return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) | ((uint32_t)(d & 0xff) << 24);
 }
 
+// R(a / 2^7) with ties to even in four integer operations: adding 63 plus the parity of the quotient carries
+// into bit 7 exactly when the remainder exceeds one half, or equals it with an odd quotient.
+__device__ __forceinline__ int32_t rne7(int32_t a) { return (a + 63 + ((a >> 7) & 1)) >> 7; }
+
 // Forward chain on 16 consecutive output channels of one pixel (Sec. 3.2.1: x2 = Q_a1(conv), x3 = gamma x2,
-// x4 = x3 + b2 [+ shortcut], x5 = Q_a2(relu(x4)); mask = [x4 > 0]).
+// x4 = x3 + b2 [+ shortcut], x5 = Q_a2(relu(x4)); mask = [x4 > 0]).  kShift7: the input sits at exponent -7.
+template <bool kShift7>
 __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t *acc, size_t off, int col, int cls,
                                            int shift)
 {
@@ -47,65 +52,65 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t 
         const int4 *t = reinterpret_cast<const int4 *>(p.b1_table + (size_t)cls * p.N + col);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            int4 v = __ldg(t + i);
+            const int4 v = __ldg(t + i);
             a[4 * i + 0] += p.b1_c * v.x;
             a[4 * i + 1] += p.b1_c * v.y;
             a[4 * i + 2] += p.b1_c * v.z;
             a[4 * i + 3] += p.b1_c * v.w;
         }
     }
-    int sc[16];
-    if (p.shortcut) {
-        int4 v = __ldg(reinterpret_cast<const int4 *>(p.shortcut + off));
-        const int8_t *b = reinterpret_cast<const int8_t *>(&v);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) sc[i] = b[i];
-    } else {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) sc[i] = 0;
-    }
-    int32_t x2v[16], x5v[16];
-    uint32_t mbits = 0;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        int32_t v2;
-        if (shift >= 0) {
-            v2 = clampi(rne_shr32(a[i], shift), -32768, 32767);
-        } else {
-            long long w = (long long)a[i] << (-shift);
-            v2 = (int32_t)(w < -32768 ? -32768 : (w > 32767 ? 32767 : w));
-        }
-        int32_t v4 = p.gamma_c * v2 + (p.b2_c << 7) + (sc[i] << 7);
-        mbits |= (v4 > 0 ? 1u : 0u) << i;
-        int32_t r = (p.relu && v4 < 0) ? 0 : v4;
-        x2v[i] = v2;
-        x5v[i] = clampi(rne_shr32(r, 7), -127, 127);
-    }
-    int4 o;
-    o.x = (int)pack4(x5v[0], x5v[1], x5v[2], x5v[3]);
-    o.y = (int)pack4(x5v[4], x5v[5], x5v[6], x5v[7]);
-    o.z = (int)pack4(x5v[8], x5v[9], x5v[10], x5v[11]);
-    o.w = (int)pack4(x5v[12], x5v[13], x5v[14], x5v[15]);
-    *reinterpret_cast<int4 *>(p.x5 + off) = o;
-    if (p.relu_mask) *reinterpret_cast<uint16_t *>(p.relu_mask + (off >> 3)) = (uint16_t)mbits;
-    if (p.x2) {
-        int4 lo, hi;
-        lo.x = (x2v[0] & 0xffff) | (x2v[1] << 16);
-        lo.y = (x2v[2] & 0xffff) | (x2v[3] << 16);
-        lo.z = (x2v[4] & 0xffff) | (x2v[5] << 16);
-        lo.w = (x2v[6] & 0xffff) | (x2v[7] << 16);
-        hi.x = (x2v[8] & 0xffff) | (x2v[9] << 16);
-        hi.y = (x2v[10] & 0xffff) | (x2v[11] << 16);
-        hi.z = (x2v[12] & 0xffff) | (x2v[13] << 16);
-        hi.w = (x2v[14] & 0xffff) | (x2v[15] << 16);
-        int4 *d = reinterpret_cast<int4 *>(p.x2 + off);
-        d[0] = lo;
-        d[1] = hi;
-    }
     if (p.acc_out) {
         int4 *d = reinterpret_cast<int4 *>(p.acc_out + off);
 #pragma unroll
         for (int i = 0; i < 4; ++i) d[i] = make_int4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+    }
+    int32_t add[16];  // (b2 + shortcut) * 2^7, the part of x4 that does not depend on the accumulator
+    const int32_t b2s = p.b2_c << 7;
+    if (p.shortcut) {
+        const int4 v = __ldg(reinterpret_cast<const int4 *>(p.shortcut + off));
+        const int8_t *b = reinterpret_cast<const int8_t *>(&v);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) add[i] = b2s + ((int32_t)b[i] << 7);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) add[i] = b2s;
+    }
+    uint32_t mbits = 0;
+    const int32_t lo = p.relu ? 0 : -127 * 128 - 64;  // below this Q_a2 saturates at -127 anyway
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        int32_t v2;
+        if (kShift7) {
+            v2 = rne7(a[i]);
+        } else if (shift >= 0) {
+            v2 = rne_shr32(a[i], shift);
+        } else {
+            const long long w = (long long)a[i] << (-shift);
+            v2 = (int32_t)(w < -32768 ? -32768 : (w > 32767 ? 32767 : w));
+        }
+        v2 = clampi(v2, -32768, 32767);
+        a[i] = v2;
+        const int32_t v4 = p.gamma_c * v2 + add[i];
+        mbits |= (v4 > 0 ? 1u : 0u) << i;
+        add[i] = min(rne7(max(v4, lo)), 127);
+    }
+    if (!p.relu) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) add[i] = max(add[i], -127);
+    }
+    int4 o;
+    o.x = (int)pack4(add[0], add[1], add[2], add[3]);
+    o.y = (int)pack4(add[4], add[5], add[6], add[7]);
+    o.z = (int)pack4(add[8], add[9], add[10], add[11]);
+    o.w = (int)pack4(add[12], add[13], add[14], add[15]);
+    *reinterpret_cast<int4 *>(p.x5 + off) = o;
+    if (p.relu_mask) *reinterpret_cast<uint16_t *>(p.relu_mask + (off >> 3)) = (uint16_t)mbits;
+    if (p.x2) {
+        int4 *d = reinterpret_cast<int4 *>(p.x2 + off);
+        d[0] = make_int4((a[0] & 0xffff) | (a[1] << 16), (a[2] & 0xffff) | (a[3] << 16), (a[4] & 0xffff) | (a[5] << 16),
+                         (a[6] & 0xffff) | (a[7] << 16));
+        d[1] = make_int4((a[8] & 0xffff) | (a[9] << 16), (a[10] & 0xffff) | (a[11] << 16),
+                         (a[12] & 0xffff) | (a[13] << 16), (a[14] & 0xffff) | (a[15] << 16));
     }
 }
 
@@ -158,7 +163,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(tfull_bar(a), 1);
-            ptx::mbar_init(tempty_bar(a), 4);
+            ptx::mbar_init(tempty_bar(a), kEpilogueWarps);
         }
         ptx::mbar_init(drain_bar, 1);
         abort_s = 0;
@@ -275,8 +280,14 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         }
     } else {
         // ---------------------------------------------------------------------- epilogue
+        // Eight warps, two per scheduler: a warp may read the TMEM lanes of quadrant (warp % 4); the two warps
+        // of a quadrant split the tile's columns.
         const int quad = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int row = quad * 32 + lane;
+        const int groups = p.tile_n / 16;                 // 16-column groups of the tile
+        const int g_begin = half ? (groups + 1) / 2 : 0;  // the first half takes the odd group
+        const int g_end = half ? groups : (groups + 1) / 2;
         int shift = 7;
         if (p.epilogue == kEpiForward && p.x_exp) {
             shift = -__ldg(p.x_exp);
@@ -305,21 +316,18 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                           border_class(x, p.wq, p.b1_nlo_w, p.b1_nhi_w, p.b1_ncc);
             }
             const uint32_t t_row = tmem_base + acc * acc_stride + ((uint32_t)(quad * 32) << 16);
-            for (int c0 = 0; c0 < p.tile_n; c0 += 32) {
+            for (int g = g_begin; g < g_end; ++g) {
                 uint32_t r[32];
-                const int ncol = min(32, p.tile_n - c0);
-                if (ncol == 32) ptx::tmem_ld_32x32(t_row + c0, r);
-                else ptx::tmem_ld_32x16(t_row + c0, r);
+                ptx::tmem_ld_32x16(t_row + g * 16, r);
                 ptx::tmem_ld_wait();
-                if (valid) {
-#pragma unroll
-                    for (int g = 0; g < 2; ++g) {
-                        const int col = nt * p.tile_n + c0 + g * 16;
-                        if (g * 16 < ncol && col < p.N) {
-                            const size_t off = pix * p.N + col;
-                            if (p.epilogue == kEpiForward) forward_16(p, r + g * 16, off, col, cls, shift);
-                            else mx = max(mx, dgrad_16(p, r + g * 16, off));
-                        }
+                const int col = nt * p.tile_n + g * 16;
+                if (valid && col < p.N) {
+                    const size_t off = pix * p.N + col;
+                    if (p.epilogue == kEpiForward) {
+                        if (shift == 7) forward_16<true>(p, r, off, col, cls, shift);
+                        else forward_16<false>(p, r, off, col, cls, shift);
+                    } else {
+                        mx = max(mx, dgrad_16(p, r, off));
                     }
                 }
             }

@@ -10,7 +10,9 @@ namespace eoq {
 
 constexpr int kMaxTaps = 64;        // kh * kw of any supported filter
 constexpr int kTileM = 128;         // GEMM rows per CTA tile (TMEM lanes)
-constexpr int kGemmThreads = 192;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr int kEpilogueWarps = 8;   // implicit GEMM: two epilogue warps per scheduler
+constexpr int kGemmThreads = 64 + 32 * kEpilogueWarps;  // warp 0: TMA, warp 1: MMA + TMEM owner, then the epilogue
+constexpr int kWgradThreads = 192;  // weight gradient: warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 constexpr uint32_t kSpinLimit = 1u << 22;  // polls before a wait gives up (normal waits end within microseconds)
 
 // Device state a handle owns.

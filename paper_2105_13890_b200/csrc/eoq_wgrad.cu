@@ -39,7 +39,7 @@ __device__ __forceinline__ uint64_t mn_major_desc(uint32_t addr, int row_bytes, 
     return make_smem_desc(addr, sub_bytes, 8u * row_bytes, layout_type_for(row_bytes));
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kWgradThreads, 1)
 wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUtensorMap map_x,
              const __grid_constant__ CUtensorMap map_e)
 {
@@ -207,7 +207,7 @@ cudaError_t launch_wgrad(const WgradParams &p, const CUtensorMap &map_x, const C
     cudaError_t e = cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024);
     if (e != cudaSuccess) return e;
     const int grid = p.num_m_tiles * p.num_n_tiles * p.num_k_splits;
-    wgrad_kernel<<<grid, kGemmThreads, wgrad_smem_bytes(p), stream>>>(p, map_x, map_e);
+    wgrad_kernel<<<grid, kWgradThreads, wgrad_smem_bytes(p), stream>>>(p, map_x, map_e);
     return cudaGetLastError();
 }
 
