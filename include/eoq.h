@@ -69,9 +69,15 @@ typedef enum { EOQ_ROUND_RNE = 0, EOQ_ROUND_STOCHASTIC = 1 } eoq_round_t;
 typedef enum { EOQ_PASS_FWD = 0, EOQ_PASS_DGRAD = 1, EOQ_PASS_WGRAD = 2 } eoq_pass_t;
 
 /* Geometry of one convolution: input [n,h,w,c_in], filter kh x kw, square stride and padding.
- * Output spatial size is (h + 2 pad - kh) / stride + 1 by (w + 2 pad - kw) / stride + 1. */
+ * Output spatial size is (h + 2 pad - kh) / stride + 1 by (w + 2 pad - kw) / stride + 1.
+ * x_wmargin (normally 0): the INPUT tensor x is stored with that many zero pixels before and after every image
+ * row, i.e. as [n][h][w + 2 x_wmargin][c_in] with the image in the middle (eoq_quantize_image writes this form).
+ * The margins are part of the zero padding, not of the image.  With c_in = 16, a filter 5 to 8 taps wide and a
+ * margin of at least max(pad, (wo-1) stride - pad + 8 - w) pixels (4 for the 7x7 stride-2 first layer of the
+ * ImageNet ResNets) a whole filter row is fetched as one 128-byte run, which is several times faster than one
+ * 16-byte fetch per tap.  Outputs and the error tensors never carry margins. */
 typedef struct {
-    int n, h, w, c_in, c_out, kh, kw, stride, pad;
+    int n, h, w, c_in, c_out, kh, kw, stride, pad, x_wmargin;
 } eoq_conv_desc_t;
 
 /* Creates a handle on CUDA device `device` (makes it current).  Synchronises. */
@@ -184,14 +190,13 @@ EOQ_API int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const int
                uint64_t seed, uint64_t step, void *stream);
 
 /*
- * Q_e-style input quantizer for the network input (Sec. 5.1 quantizes every layer but the last): SQ(., 8)
- * of an fp32 NHWC image with c_src channels per pixel, written as int8 with c_dst >= c_src channels per
- * pixel (the extra channels are zero), so that the first convolution sees a multiple of 16 channels.
- * device in : src [pixels][c_src] fp32.   device out: dst [pixels][c_dst] int8 (c_dst a multiple of 16, <= 64),
- *             *dst_exp.  The maximum runs over the whole tensor.
+ * Input quantizer for the network input (Sec. 5.1 quantizes every layer but the last): SQ(., 8) of an fp32
+ * NHWC image batch [n][h][w][c_src], written as int8 [n][h][w + 2 wmargin][c_dst] with c_dst >= c_src: the extra
+ * channels and the wmargin pixels at both ends of every row are zero (see eoq_conv_desc_t::x_wmargin).
+ * c_dst is a multiple of 16 and at most 64.  The maximum runs over the whole batch.  *dst_exp is written.
  */
-EOQ_API int eoq_quantize_image(eoq_handle_t handle, const float *src, size_t pixels, int c_src, int c_dst, int8_t *dst,
-                       int32_t *dst_exp, void *stream);
+EOQ_API int eoq_quantize_image(eoq_handle_t handle, const float *src, int n, int h, int w, int c_src, int c_dst,
+                       int wmargin, int8_t *dst, int32_t *dst_exp, void *stream);
 
 /* int8 layout change between NCHW and NHWC ([n,c,h,w] <-> [n,h,w,c]); to_nhwc = 1 reads NCHW. */
 EOQ_API int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t *dst, int n, int c, int h, int w,

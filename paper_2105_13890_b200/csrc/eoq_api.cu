@@ -58,6 +58,24 @@ int chunk_bytes(int c)
 
 // im2col view of an NHWC int8 tensor [n][h][w][c]: `pixels` consecutive positions of the walk that starts at
 // (lower_w, lower_h) and advances by `stride`, `box_c` channels each.  count_w/h = positions per row/column.
+// View for the filter-row path: the pixel of the walk is a 128-byte window of 8 adjacent 16-channel pixels that
+// starts at memory column (first_col + k * stride) of a row w_mem pixels long, so consecutive windows overlap
+// (the W stride of the view is smaller than its inner extent).  Rows are walked with zero fill above and below.
+bool make_row_window_map(CUtensorMap *map, const void *ptr, int n, int h, int w_mem, int first_col, int count_w,
+                         int count_h, int stride, int pad_h, int pixels)
+{
+    cuuint64_t dims[4] = {128, (cuuint64_t)count_w, (cuuint64_t)h, (cuuint64_t)n};
+    cuuint64_t strides[3] = {(cuuint64_t)stride * 16, (cuuint64_t)w_mem * 16, (cuuint64_t)w_mem * 16 * h};
+    int lower[2] = {0, -pad_h};
+    int upper[2] = {0, (count_h - 1) * stride + 1 - pad_h - h};
+    if (upper[1] < -128 || upper[1] > 127 || pad_h > 128) return false;
+    cuuint32_t estr[4] = {1, 1, (cuuint32_t)stride, 1};
+    const char *base = static_cast<const char *>(ptr) + (long long)first_col * 16;
+    return g_encode_im2col(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<char *>(base), dims, strides, lower, upper,
+                           128, (cuuint32_t)pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_im2col_map(CUtensorMap *map, const void *ptr, int n, int h, int w, int c, int lower_w, int lower_h,
                      int count_w, int count_h, int stride, int box_c, int pixels)
 {
@@ -117,6 +135,7 @@ int check_desc(const eoq_conv_desc_t *d, Geometry *g)
         return EOQ_ERR_BAD_ARG;
     if (d->h + 2 * d->pad < d->kh || d->w + 2 * d->pad < d->kw) return EOQ_ERR_BAD_ARG;
     if (d->c_in % 16 || d->c_out % 16) return EOQ_ERR_ALIGNMENT;
+    if (d->x_wmargin < 0 || d->x_wmargin > 64) return EOQ_ERR_BAD_ARG;
     if (d->kh * d->kw > kMaxTaps || d->kh > 16 || d->kw > 16 || d->stride > 8 || d->pad > 64) return EOQ_ERR_UNSUPPORTED;
     g->ho = (d->h + 2 * d->pad - d->kh) / d->stride + 1;
     g->wo = (d->w + 2 * d->pad - d->kw) / d->stride + 1;
@@ -154,6 +173,16 @@ int record(Handle *h, cudaError_t e)
     if (e == cudaSuccess) return EOQ_OK;
     h->last_cuda_error = (int)e;
     return EOQ_ERR_CUDA;
+}
+
+// 16-channel inputs under filters 5 to 8 taps wide (the 7x7 first layer) stored with wide enough zero margins take
+// the filter-row path: a filter row is 8 adjacent 16-byte pixels, one 128-byte K sub-tile, instead of one
+// 16-byte TMA row per tap.
+inline bool use_row_window(const eoq_conv_desc_t &d, int wo)
+{
+    if (d.c_in != 16 || d.kw < 5 || d.kw > 8) return false;
+    const int need_right = (wo - 1) * d.stride - d.pad + 8 - d.w;
+    return d.x_wmargin >= d.pad && d.x_wmargin >= need_right;
 }
 
 // Shared tiling choices of the implicit GEMM: K sub-tiles, pipeline depth, column tile.
@@ -350,8 +379,9 @@ extern "C" int eoq_workspace_size(const eoq_conv_desc_t *desc, int pass, size_t 
     if (st != EOQ_OK) return st;
     const BorderClasses bc = border_classes(*desc, g);
     switch (pass) {
-        case EOQ_PASS_FWD:  // b1 table
-            *bytes = round256((size_t)bc.nrc * bc.ncc * desc->c_out * sizeof(int32_t));
+        case EOQ_PASS_FWD:  // b1 table, then the row-padded weights of the filter-row path
+            *bytes = round256((size_t)bc.nrc * bc.ncc * desc->c_out * sizeof(int32_t)) +
+                     (use_row_window(*desc, g.wo) ? round256((size_t)desc->c_out * desc->kh * 128) : 0);
             return EOQ_OK;
         case EOQ_PASS_DGRAD:  // transposed weights + int32 sums
             *bytes = round256(g.w_elems) + round256(g.in_elems * sizeof(int32_t));
@@ -394,8 +424,10 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     const eoq_conv_desc_t &d = *desc;
     // the accumulator with its b1 term must fit int32: taps * c_in * (127 + |b1|) * 127 < 2^31
     if ((double)g.taps * d.c_in * (127.0 + (b1_c < 0 ? -b1_c : b1_c)) * 127.0 >= 2147483647.0 - 16777216.0) return EOQ_ERR_RANGE;
-    if (b1_c != 0 && (st = check_workspace(desc, EOQ_PASS_FWD, workspace, workspace_bytes)) != EOQ_OK) return st;
+    const bool row_window = use_row_window(d, g.wo);
+    if ((b1_c != 0 || row_window) && (st = check_workspace(desc, EOQ_PASS_FWD, workspace, workspace_bytes)) != EOQ_OK) return st;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int w_mem = d.w + 2 * d.x_wmargin;
 
     IgemmParams p;
     memset(&p, 0, sizeof(p));
@@ -403,14 +435,33 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     p.N = d.c_out;
     p.hq = g.ho;
     p.wq = g.wo;
-    plan_igemm(p, d.c_in, g.taps, h->sm_count);
     p.src_stride = d.stride;
     p.base_h = -d.pad;
-    p.base_w = -d.pad;
-    for (int t = 0; t < g.taps; ++t) {
-        p.tap_dh[t] = (unsigned char)(t / d.kw);
-        p.tap_dw[t] = (unsigned char)(t % d.kw);
-        p.tap_b[t] = (unsigned char)t;
+    int8_t *w_rows = nullptr;
+    if (row_window) {
+        // K sub-tile = one filter row (8 pixels x 16 channels); the map's W axis already steps by the stride
+        plan_igemm(p, 128, d.kh, h->sm_count);
+        p.src_stride_w = 1;
+        p.base_w = 0;
+        for (int t = 0; t < d.kh; ++t) {
+            p.tap_dh[t] = (unsigned char)t;
+            p.tap_dw[t] = 0;
+            p.tap_b[t] = (unsigned char)t;
+        }
+        const BorderClasses bc0 = border_classes(d, g);
+        w_rows = reinterpret_cast<int8_t *>(workspace) + round256((size_t)bc0.nrc * bc0.ncc * d.c_out * sizeof(int32_t));
+        cudaError_t e = launch_weight_pad_rows(w, w_rows, d.c_out, d.kh, d.kw, s);
+        if (e != cudaSuccess) return record(h, e);
+        count_launches(h, 1);
+    } else {
+        plan_igemm(p, d.c_in, g.taps, h->sm_count);
+        p.src_stride_w = d.stride;
+        p.base_w = d.x_wmargin - d.pad;
+        for (int t = 0; t < g.taps; ++t) {
+            p.tap_dh[t] = (unsigned char)(t / d.kw);
+            p.tap_dw[t] = (unsigned char)(t % d.kw);
+            p.tap_b[t] = (unsigned char)t;
+        }
     }
     p.out_h = g.ho;
     p.out_w = g.wo;
@@ -438,9 +489,15 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
         count_launches(h, 1);
     }
     CUtensorMap map_a, map_b;
-    if (!make_im2col_map(&map_a, x, d.n, d.h, d.w, d.c_in, -d.pad, -d.pad, g.wo, g.ho, d.stride, p.kc, kTileM) ||
-        !make_weight_map(&map_b, w, d.c_out, g.taps, d.c_in, p.kc, p.tile_n))
+    if (row_window) {
+        if (!make_row_window_map(&map_a, x, d.n, d.h, w_mem, d.x_wmargin - d.pad, g.wo, g.ho, d.stride, d.pad, kTileM) ||
+            !make_weight_map(&map_b, w_rows, d.c_out, d.kh, 128, 128, p.tile_n))
+            return EOQ_ERR_UNSUPPORTED;
+    } else if (!make_im2col_map(&map_a, x, d.n, d.h, w_mem, d.c_in, d.x_wmargin - d.pad, -d.pad, g.wo, g.ho, d.stride, p.kc,
+                                kTileM) ||
+               !make_weight_map(&map_b, w, d.c_out, g.taps, d.c_in, p.kc, p.tile_n)) {
         return EOQ_ERR_UNSUPPORTED;
+    }
     const int tiles = p.num_m_tiles * p.num_n_tiles;
     count_launches(h, 1);
     ProfScope prof(h, EOQ_PROF_IGEMM_FWD, s);
@@ -512,6 +569,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             p.wq = wq;
             plan_igemm(p, d.c_out, nh * nw, h->sm_count);
             p.src_stride = 1;
+            p.src_stride_w = 1;
             p.base_h = min_h;
             p.base_w = min_w;
             for (int a = 0; a < nh; ++a)
@@ -577,12 +635,18 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     p.c_in = d.c_in;
     p.c_out = d.c_out;
     p.ntaps = g.taps;
-    p.kc = chunk_bytes(d.c_in);
+    const bool row_window = use_row_window(d, g.wo);
+    const int w_mem = d.w + 2 * d.x_wmargin;
+    p.kc = row_window ? 128 : chunk_bytes(d.c_in);
     p.nc = chunk_bytes(d.c_out);
-    p.chunks_per_tap = d.c_in / p.kc;
+    p.chunks_per_tap = row_window ? 1 : d.c_in / p.kc;
     p.rows_total = g.taps * d.c_in;
     p.subs_per_mtile = kTileM / p.kc;
-    p.num_m_tiles = (p.rows_total + kTileM - 1) / kTileM;
+    p.num_m_tiles = row_window ? d.kh : (p.rows_total + kTileM - 1) / kTileM;  // filter-row path: one M tile per filter row
+    if (row_window) {
+        p.ntaps = d.kh;
+        p.row_window_kw = d.kw;
+    }
     p.tile_n = d.c_out < 256 ? d.c_out : 256;
     if (p.tile_n % p.nc) p.tile_n = (p.tile_n / p.nc) * p.nc;
     p.num_n_tiles = (d.c_out + p.tile_n - 1) / p.tile_n;
@@ -605,10 +669,20 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     p.num_stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
     p.src_stride = d.stride;
     p.base_h = -d.pad;
-    p.base_w = -d.pad;
-    for (int t = 0; t < g.taps; ++t) {
-        p.tap_dh[t] = (unsigned char)(t / d.kw);
-        p.tap_dw[t] = (unsigned char)(t % d.kw);
+    if (row_window) {
+        p.src_stride_w = 1;
+        p.base_w = 0;
+        for (int t = 0; t < d.kh; ++t) {
+            p.tap_dh[t] = (unsigned char)t;
+            p.tap_dw[t] = 0;
+        }
+    } else {
+        p.src_stride_w = d.stride;
+        p.base_w = d.x_wmargin - d.pad;
+        for (int t = 0; t < g.taps; ++t) {
+            p.tap_dh[t] = (unsigned char)(t / d.kw);
+            p.tap_dw[t] = (unsigned char)(t % d.kw);
+        }
     }
     p.acc = acc;
     p.dev = h->dev;
@@ -624,8 +698,11 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     }
     if (e != cudaSuccess) return record(h, e);
     CUtensorMap map_x, map_e;
-    if (!make_im2col_map(&map_x, x, d.n, d.h, d.w, d.c_in, -d.pad, -d.pad, g.wo, g.ho, d.stride, p.kc, p.pixels_per_stage) ||
-        !make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage))
+    if (!make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage)) return EOQ_ERR_UNSUPPORTED;
+    if (row_window ? !make_row_window_map(&map_x, x, d.n, d.h, w_mem, d.x_wmargin - d.pad, g.wo, g.ho, d.stride, d.pad,
+                                          p.pixels_per_stage)
+                   : !make_im2col_map(&map_x, x, d.n, d.h, w_mem, d.c_in, d.x_wmargin - d.pad, -d.pad, g.wo, g.ho, d.stride,
+                                      p.kc, p.pixels_per_stage))
         return EOQ_ERR_UNSUPPORTED;
     count_launches(h, 3);  // the GEMM and the two kernels of Q_g
     {
@@ -707,13 +784,15 @@ extern "C" int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t
     return record(h, launch_layout_convert(src, dst, n, c, hh, ww, to_nhwc, reinterpret_cast<cudaStream_t>(stream)));
 }
 
-extern "C" int eoq_quantize_image(eoq_handle_t handle, const float *src, size_t pixels, int c_src, int c_dst, int8_t *dst,
-                                  int32_t *dst_exp, void *stream)
+extern "C" int eoq_quantize_image(eoq_handle_t handle, const float *src, int n, int hh, int ww, int c_src, int c_dst,
+                                  int wmargin, int8_t *dst, int32_t *dst_exp, void *stream)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
-    if (!h || !src || !dst || !dst_exp || pixels == 0 || c_src <= 0 || c_dst < c_src) return EOQ_ERR_BAD_ARG;
+    if (!h || !src || !dst || !dst_exp || n <= 0 || hh <= 0 || ww <= 0 || c_src <= 0 || c_dst < c_src || wmargin < 0 ||
+        wmargin > 64)
+        return EOQ_ERR_BAD_ARG;
     if (c_dst % 16 || c_dst > 64 || !aligned16(src) || !aligned16(dst)) return EOQ_ERR_ALIGNMENT;
     count_launches(h, 2);
-    return record(h, launch_quantize_image(src, pixels, c_src, c_dst, dst, dst_exp, h->dev, h->sm_count,
+    return record(h, launch_quantize_image(src, n, hh, ww, c_src, c_dst, wmargin, dst, dst_exp, h->dev, h->sm_count,
                                            reinterpret_cast<cudaStream_t>(stream)));
 }

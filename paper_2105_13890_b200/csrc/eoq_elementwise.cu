@@ -125,9 +125,10 @@ __global__ void quantize_f32_kernel(int mode, const float *__restrict__ src, siz
     }
 }
 
-// SQ of an fp32 image under the already reduced maximum, c_src channels in, c_dst (zero-padded) channels out.
-__global__ void quantize_image_kernel(const float *__restrict__ src, size_t pixels, int c_src, int c_dst, int8_t *dst,
-                                      int32_t *dst_exp, DeviceState *dev)
+// SQ of an fp32 image under the already reduced maximum: c_src channels in, c_dst (zero-padded) channels out,
+// rows widened by `wmargin` zero pixels at both ends.
+__global__ void quantize_image_kernel(const float *__restrict__ src, int rows, int w, int c_src, int c_dst, int wmargin,
+                                      int8_t *dst, int32_t *dst_exp, DeviceState *dev)
 {
     const uint32_t mbits = dev->absmax_u32;
     int up = 7;
@@ -138,17 +139,20 @@ __global__ void quantize_image_kernel(const float *__restrict__ src, size_t pixe
         if (mbits == 0) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
     }
     const int groups = c_dst / 16;
-    const size_t items = pixels * groups;
+    const int w_mem = w + 2 * wmargin;
+    const size_t items = (size_t)rows * w_mem * groups;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
-        const size_t pix = i / groups;
         const int g = (int)(i % groups);
+        const size_t mp = i / groups;            // pixel index in the widened layout
+        const int xm = (int)(mp % w_mem) - wmargin;
+        const size_t row = mp / w_mem;
         int c[16];
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             const int ch = g * 16 + k;
             int v = 0;
-            if (ch < c_src) {
-                const float y = scalbnf(__ldg(src + pix * c_src + ch), up);
+            if (ch < c_src && xm >= 0 && xm < w) {
+                const float y = scalbnf(__ldg(src + (row * w + xm) * c_src + ch), up);
                 v = (fabsf(y) < 1.0e9f) ? clampi(__float2int_rn(y), -127, 127) : (y > 0.f ? 127 : (y < 0.f ? -127 : 0));
             }
             c[k] = v;
@@ -157,6 +161,17 @@ __global__ void quantize_image_kernel(const float *__restrict__ src, size_t pixe
             make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
                       (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
     }
+}
+
+// w[oc][kh][kw][16] -> wp[oc][kh][8][16] with zeros in the unused taps
+__global__ void weight_pad_rows_kernel(const int8_t *__restrict__ w, int8_t *__restrict__ wp, int rows, int kw)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;  // one 16-byte pixel of the padded layout
+    if (i >= rows * 8) return;
+    const int r = i >> 3, t = i & 7;
+    int4 v = make_int4(0, 0, 0, 0);
+    if (t < kw) v = __ldg(reinterpret_cast<const int4 *>(w) + (size_t)r * kw + t);
+    reinterpret_cast<int4 *>(wp)[i] = v;
 }
 
 // ------------------------------------------------------------------ int32 -> SQ (phase 2 of Q_e after dgrad)
@@ -606,15 +621,22 @@ cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst,
     return cudaGetLastError();
 }
 
-cudaError_t launch_quantize_image(const float *src, size_t pixels, int c_src, int c_dst, int8_t *dst, int32_t *dst_exp,
-                                  DeviceState *dev, int sm_count, cudaStream_t s)
+cudaError_t launch_quantize_image(const float *src, int n, int h, int w, int c_src, int c_dst, int wmargin, int8_t *dst,
+                                  int32_t *dst_exp, DeviceState *dev, int sm_count, cudaStream_t s)
 {
     cudaError_t e = launch_reset_cells(dev, s);
     if (e != cudaSuccess) return e;
-    const size_t n = pixels * c_src;
-    absmax_f32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
-    quantize_image_kernel<<<grid_for(pixels * (c_dst / 16), sm_count), kThreads, 0, s>>>(src, pixels, c_src, c_dst, dst,
-                                                                                         dst_exp, dev);
+    const size_t count = (size_t)n * h * w * c_src;
+    absmax_f32_kernel<<<grid_for(count / 4 + 1, sm_count), kThreads, 0, s>>>(src, count, dev);
+    const size_t items = (size_t)n * h * (w + 2 * wmargin) * (c_dst / 16);
+    quantize_image_kernel<<<grid_for(items, sm_count), kThreads, 0, s>>>(src, n * h, w, c_src, c_dst, wmargin, dst, dst_exp, dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_weight_pad_rows(const int8_t *w, int8_t *wp, int c_out, int kh, int kw, cudaStream_t s)
+{
+    const int rows = c_out * kh;
+    weight_pad_rows_kernel<<<(rows * 8 + 255) / 256, 256, 0, s>>>(w, wp, rows, kw);
     return cudaGetLastError();
 }
 

@@ -196,7 +196,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                 const int mt = tile / p.num_n_tiles, nt = tile % p.num_n_tiles;
                 const int m0 = mt * kTileM;
                 const int img = m0 / pix_per_img, rem = m0 % pix_per_img;
-                const int cw = (rem % p.wq) * p.src_stride + p.base_w;
+                const int cw = (rem % p.wq) * p.src_stride_w + p.base_w;
                 const int ch = (rem / p.wq) * p.src_stride + p.base_h;
                 for (int kit = 0; kit < k_iters; ++kit) {
                     if (!(ok = wait_bar(empty_bar(stage), phase ^ 1u, ctx))) break;

@@ -66,7 +66,8 @@ struct IgemmParams {
     int real_sub;       // sub-tiles that carry data
     int subs_per_stage;
     int num_stages;
-    int src_stride;     // TMA traversal stride in source pixels
+    int src_stride;     // TMA traversal stride in source pixels (rows)
+    int src_stride_w;   // same along a row (1 when the map's W axis already steps by the convolution stride)
     int base_h, base_w; // source coordinate of tap offset (0,0) for pixel (0,0)
     unsigned char tap_dh[kMaxTaps], tap_dw[kMaxTaps];  // im2col offsets of each tap
     unsigned char tap_b[kMaxTaps];                     // tap coordinate of each tap in the B tensor
@@ -110,7 +111,8 @@ struct WgradParams {
     int pixels_per_stage;   // 64
     int stages_per_split;   // pipeline iterations each CTA runs
     int num_stages;
-    int src_stride, base_h, base_w;
+    int src_stride, src_stride_w, base_h, base_w;
+    int row_window_kw;   // 0, or the filter width when an M tile is one filter row of 8 x 16 bytes (7 real taps of 8)
     unsigned char tap_dh[kMaxTaps], tap_dw[kMaxTaps];
     long long *acc;      // [c_out][taps][c_in] int64, zeroed before launch
     DeviceState *dev;
@@ -123,8 +125,10 @@ cudaError_t launch_wgrad(const WgradParams &p, const CUtensorMap &map_x, const C
 // Elementwise / reduction kernels
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_reset_cells(DeviceState *dev, cudaStream_t s);
-cudaError_t launch_quantize_image(const float *src, size_t pixels, int c_src, int c_dst, int8_t *dst, int32_t *dst_exp,
-                                  DeviceState *dev, int sm_count, cudaStream_t s);
+cudaError_t launch_quantize_image(const float *src, int n, int h, int w, int c_src, int c_dst, int wmargin, int8_t *dst,
+                                  int32_t *dst_exp, DeviceState *dev, int sm_count, cudaStream_t s);
+// w[oc][kh][kw][16] -> wp[oc][kh][8][16], zero in the taps kw..7 (weights of the filter-row path)
+cudaError_t launch_weight_pad_rows(const int8_t *w, int8_t *wp, int c_out, int kh, int kw, cudaStream_t s);
 cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst, int32_t *dst_exp, DeviceState *dev,
                                 int sm_count, cudaStream_t s);
 cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,

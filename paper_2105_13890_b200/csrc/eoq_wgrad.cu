@@ -108,7 +108,7 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
                 if (!(ok = wait_bar(empty_bar(stage), phase ^ 1u, ctx))) break;
                 const int q0 = q_begin + it * px;
                 const int img = q0 / pix_per_img, rem = q0 % pix_per_img;
-                const int cw = (rem % p.wo) * p.src_stride + p.base_w;
+                const int cw = (rem % p.wo) * p.src_stride_w + p.base_w;
                 const int ch = (rem / p.wo) * p.src_stride + p.base_h;
                 const uint32_t a_dst = smem_base + stage * stage_bytes;
                 const uint32_t b_dst = a_dst + p.subs_per_mtile * a_sub;
@@ -159,11 +159,17 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
         }
     } else {
         const int quad = warp & 3;
-        const int row = mt * kTileM + quad * 32 + lane;  // (tap, ic) flattened: tap * c_in + ic
+        int row = mt * kTileM + quad * 32 + lane;  // (tap, ic) flattened: tap * c_in + ic
+        bool valid = row < p.rows_total;
+        if (p.row_window_kw) {
+            // the tile's rows are (tap 0..7, channel 0..15) of filter row mt: drop the padding taps
+            const int t = (quad * 32 + lane) >> 4;
+            valid = t < p.row_window_kw;
+            row = (mt * p.row_window_kw + t) * 16 + (lane & 15);
+        }
         bool ok = __all_sync(0xffffffffu, wait_bar(done_bar, 0, ctx));
         if (ok && my_stages > 0) {
             ptx::tc_fence_after();
-            const bool valid = row < p.rows_total;
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
             for (int c0 = 0; c0 < p.tile_n; c0 += 32) {
                 uint32_t r[32];

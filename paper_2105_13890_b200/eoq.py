@@ -38,7 +38,7 @@ class EoqError(RuntimeError):
 
 
 class eoq_conv_desc_t(C.Structure):
-    _fields_ = [(k, C.c_int) for k in ("n", "h", "w", "c_in", "c_out", "kh", "kw", "stride", "pad")]
+    _fields_ = [(k, C.c_int) for k in ("n", "h", "w", "c_in", "c_out", "kh", "kw", "stride", "pad", "x_wmargin")]
 
     @property
     def ho(self) -> int:
@@ -49,8 +49,8 @@ class eoq_conv_desc_t(C.Structure):
         return (self.w + 2 * self.pad - self.kw) // self.stride + 1
 
 
-def conv_desc(n, h, w, c_in, c_out, kh, kw, stride=1, pad=0) -> eoq_conv_desc_t:
-    return eoq_conv_desc_t(n, h, w, c_in, c_out, kh, kw, stride, pad)
+def conv_desc(n, h, w, c_in, c_out, kh, kw, stride=1, pad=0, x_wmargin=0) -> eoq_conv_desc_t:
+    return eoq_conv_desc_t(n, h, w, c_in, c_out, kh, kw, stride, pad, x_wmargin)
 
 
 _lib = None
@@ -80,7 +80,7 @@ def lib() -> C.CDLL:
         L.eoq_last_status.argtypes = [vp, vp, C.POINTER(C.c_uint)]
         L.eoq_last_cuda_error.argtypes = [vp]
         L.eoq_conv_dgrad_static.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp]
-        L.eoq_quantize_image.argtypes = [vp, vp, sz, C.c_int, C.c_int, vp, vp, vp]
+        L.eoq_quantize_image.argtypes = [vp, vp] + [C.c_int] * 6 + [vp, vp, vp]
         L.eoq_profile_start.argtypes = [vp]
         L.eoq_profile_stop.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_double)]
         L.eoq_launch_count.argtypes = [vp]
@@ -218,9 +218,9 @@ def eoq_last_cuda_error(handle) -> int:
     return lib().eoq_last_cuda_error(handle)
 
 
-def eoq_quantize_image(handle, src, pixels, c_src, c_dst, dst, dst_exp, stream=None, check: bool = True) -> int:
-    st = lib().eoq_quantize_image(handle, _ptr(src), int(pixels), int(c_src), int(c_dst), _ptr(dst), _ptr(dst_exp),
-                                  _stream(stream))
+def eoq_quantize_image(handle, src, n, h, w, c_src, c_dst, wmargin, dst, dst_exp, stream=None, check: bool = True) -> int:
+    st = lib().eoq_quantize_image(handle, _ptr(src), int(n), int(h), int(w), int(c_src), int(c_dst), int(wmargin),
+                                  _ptr(dst), _ptr(dst_exp), _stream(stream))
     if check:
         _check(st, "eoq_quantize_image")
     return st

@@ -31,13 +31,15 @@ class Scalars:
 
 
 class LayerBuffers:
-    def __init__(self, layer: Layer, dev):
+    def __init__(self, layer: Layer, dev, wmargin: int = 0):
         self.layer = layer
-        self.desc = eoq.conv_desc(layer.n, layer.h, layer.w, layer.c_in, layer.c_out, layer.k, layer.k, layer.stride, layer.pad)
+        self.wmargin = wmargin
+        self.desc = eoq.conv_desc(layer.n, layer.h, layer.w, layer.c_in, layer.c_out, layer.k, layer.k, layer.stride, layer.pad,
+                                  wmargin)
         i8, dev_ = torch.int8, dev
         out_shape = (layer.n, layer.ho, layer.wo, layer.c_out)
         in_shape = (layer.n, layer.h, layer.w, layer.c_in)
-        self.x0 = torch.empty(in_shape, dtype=i8, device=dev_)
+        self.x0 = torch.zeros((layer.n, layer.h, layer.w + 2 * wmargin, layer.c_in), dtype=i8, device=dev_)
         self.w = torch.empty((layer.c_out, layer.k, layer.k, layer.c_in), dtype=i8, device=dev_)
         self.x5 = torch.empty(out_shape, dtype=i8, device=dev_)
         self.x2 = torch.empty(out_shape, dtype=torch.int16, device=dev_) if layer.gamma_trainable else None
@@ -67,7 +69,11 @@ class TrainStep:
         self.sc = scalars or Scalars()
         self.lr_mant, self.lr_exp = lr_mant, lr_exp
         self.step_no = 0
-        self.layers: List[LayerBuffers] = [LayerBuffers(l, self.dev) for l in workload.layers]
+        # the network input is stored with zero row margins so that a wide first-layer filter can fetch whole
+        # filter rows (eoq_conv_desc_t::x_wmargin); every other layer input is dense
+        first_margin = 4 if workload.layers[0].k >= 5 else 0
+        self.layers: List[LayerBuffers] = [LayerBuffers(l, self.dev, first_margin if i == 0 else 0)
+                                           for i, l in enumerate(workload.layers)]
         ws = 256
         for lb in self.layers:
             for p in (eoq.EOQ_PASS_FWD, eoq.EOQ_PASS_DGRAD, eoq.EOQ_PASS_WGRAD):
@@ -112,7 +118,8 @@ class TrainStep:
     def run(self) -> None:
         h, sc, ws = self.h, self.sc, self.workspace
         first = self.layers[0]
-        eoq.eoq_quantize_image(h, self.image, self.image_pixels, self.image_channels, first.layer.c_in, first.x0,
+        fl = first.layer
+        eoq.eoq_quantize_image(h, self.image, fl.n, fl.h, fl.w, self.image_channels, fl.c_in, first.wmargin, first.x0,
                                self.image_exp)
         for i, lb in enumerate(self.layers):
             l = lb.layer

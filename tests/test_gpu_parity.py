@@ -60,6 +60,57 @@ def test_conv_fwd(d, scal):
     assert np.array_equal(G.unpack_mask(mask, shape), ref["mask"])
 
 
+MARGIN_CASES = [
+    (ConvDesc(2, 20, 20, 16, 64, 7, 7, 2, 3), 4),     # filter-row path of the 7x7 stride-2 first layer
+    (ConvDesc(3, 17, 23, 16, 32, 7, 7, 2, 3), 5),     # odd extents, wider margin
+    (ConvDesc(2, 12, 12, 16, 16, 5, 5, 1, 2), 4),     # 5 taps wide, stride 1
+    (ConvDesc(2, 20, 20, 16, 64, 7, 7, 2, 3), 2),     # margin too small for the filter-row path: per-tap path
+    (ConvDesc(2, 9, 9, 32, 48, 3, 3, 1, 1), 3),       # margins on an ordinary layer
+]
+
+
+def with_margin(x0, m):
+    return np.pad(x0, ((0, 0), (0, 0), (m, m), (0, 0)))
+
+
+@pytest.mark.parametrize("d,m", MARGIN_CASES, ids=[f"k{d.kh}s{d.stride}_c{d.c_in}_m{m}_{d.h}x{d.w}" for d, m in MARGIN_CASES])
+def test_input_with_row_margins(d, m):
+    """Forward and weight gradient on an input stored with zero row margins (x_wmargin)."""
+    x0, w, _, e3 = layer_data(d, 900 + m + d.h)
+    gd = eoq.conv_desc(d.n, d.h, d.w, d.c_in, d.c_out, d.kh, d.kw, d.stride, d.pad, m)
+    xm = G.dev(with_margin(x0, m))
+    for b1 in (0, -4):
+        ref = oracle.layer_forward(d, x0, b1, w, 100, 2)
+        shape = ref["x5"].shape
+        x5, acc = G.zeros(shape, torch.int8), G.zeros(shape, torch.int32)
+        eoq.eoq_conv_fwd(G.handle(), gd, xm, None, b1, G.dev(w), 100, 2, None, True, x5, None, None, acc,
+                         G.workspace(gd, eoq.EOQ_PASS_FWD))
+        assert G.status_clear() == 0
+        assert np.array_equal(G.host(acc).astype(np.int64), ref["acc"]) and np.array_equal(G.host(x5), ref["x5"])
+        Gacc = oracle.conv_wgrad_acc(d, e3, x0, b1)
+        g, pg, _ = oracle.sq_int(Gacc, -16)
+        g_d, gacc, g_exp = G.zeros(Gacc.shape, torch.int8), G.zeros(Gacc.shape, torch.int64), G.zeros(1, torch.int32)
+        eoq.eoq_conv_wgrad(G.handle(), gd, G.dev(e3), G.dev(np.array([-9], dtype=np.int32)), xm, b1, g_d, g_exp, gacc,
+                           G.workspace(gd, eoq.EOQ_PASS_WGRAD))
+        assert G.status_clear() == 0
+        assert np.array_equal(G.host(gacc), Gacc) and g_exp.item() == pg
+        assert np.array_equal(G.host(g_d).astype(np.int32), g)
+
+
+@pytest.mark.parametrize("m", [0, 4])
+def test_quantize_image_pads_channels_and_rows(m):
+    n, h, w = 3, 10, 13
+    img = synth.normal_f32((n, h, w, 3), 950, m)
+    padded = np.zeros((n, h, w, 16), dtype=np.float32)
+    padded[..., :3] = img
+    c, p, _ = oracle.quantize_f32(oracle.MODE_SQ, padded)
+    out = torch.full((n, h, w + 2 * m, 16), 55, dtype=torch.int8, device="cuda:0")
+    ex = G.zeros(1, torch.int32)
+    eoq.eoq_quantize_image(G.handle(), G.dev(img), n, h, w, 3, 16, m, out, ex)
+    assert G.status_clear() == 0 and ex.item() == p
+    assert np.array_equal(G.host(out).astype(np.int32), with_margin(c, m))
+
+
 def test_conv_fwd_without_optional_outputs_and_with_input_exponent():
     d = ConvDesc(2, 12, 12, 16, 32, 3, 3, 1, 1)
     x0, w, _, _ = layer_data(d, 7)
