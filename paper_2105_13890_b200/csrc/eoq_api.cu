@@ -93,6 +93,19 @@ bool make_im2col_map(CUtensorMap *map, const void *ptr, int n, int h, int w, int
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tiled view of an NHWC int8 tensor with a (box_c, box_w, box_h, 1) box: one patch of pixels, halo included.
+bool make_patch_map(CUtensorMap *map, const void *ptr, int n, int h, int w, int c, int box_c, int box_w, int box_h)
+{
+    if (box_w > 256 || box_h > 256) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
+    cuuint64_t strides[3] = {(cuuint64_t)c, (cuuint64_t)c * w, (cuuint64_t)c * w * h};
+    cuuint32_t box[4] = {(cuuint32_t)box_c, (cuuint32_t)box_w, (cuuint32_t)box_h, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(box_c), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Tiled view of a [rows][taps][c] int8 tensor with a (box_c, 1, box_rows) box.
 bool make_weight_map(CUtensorMap *map, const void *ptr, int rows, int taps, int c, int box_c, int box_rows)
 {
@@ -205,6 +218,61 @@ void plan_igemm(IgemmParams &p, int src_channels, int ntaps, int sm_count)
     const size_t stage = (size_t)p.subs_per_stage * (kTileM + tn) * p.kc;
     int stages = (int)((200 * 1024) / stage);
     p.num_stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
+}
+
+// Plan of the patch variant for a stride-1 k x k correlation over a source [n][hs][ws][c_src] producing a
+// [n][hq][wq] grid with n_cols columns.  Returns false when the geometry does not suit it (then the per-tap
+// path is used): strided or 1x1 filters, fewer than 32 channels, rows too wide for a tile, or tiles that would
+// be mostly padding.
+bool plan_patch(IgemmParams &p, PatchPlan &pl, int n_img, int c_src, int hq, int wq, int k, int pad_src, int n_cols,
+                int sm_count)
+{
+    if (k < 2 || c_src % 32 || pad_src < 0 || pad_src > k - 1) return false;
+    const int pw = wq + k - 1;
+    if (pw > kTileM) return false;
+    int r = kTileM / pw;
+    if (r > hq) r = hq;
+    const int tiles_per_img = (hq + r - 1) / r;
+    if ((double)hq * wq < 0.6 * (double)tiles_per_img * kTileM) return false;
+    pl.n_img = n_img;
+    pl.kdim = k;
+    pl.pad = pad_src;
+    pl.pw = pw;
+    pl.r_rows = r;
+    pl.tiles_per_img = tiles_per_img;
+    p.kc = chunk_bytes(c_src);
+    pl.chunks = c_src / p.kc;
+    p.chunks_per_tap = pl.chunks;
+    p.ntaps = k * k;
+    const int patch_rows = r + k - 1;
+    pl.a_box_bytes = p.kc * pw * patch_rows;
+    const int rows_read = (k - 1) * (pw + 1) + kTileM;  // the last tap's tile ends here
+    const int rows = pw * patch_rows > rows_read ? pw * patch_rows : rows_read;
+    pl.a_bytes = (int)((((size_t)rows * p.kc) + 1023) & ~(size_t)1023);
+    p.M = n_img * hq * wq;
+    p.N = n_cols;
+    p.hq = hq;
+    p.wq = wq;
+    p.num_m_tiles = n_img * tiles_per_img;
+    int tn = n_cols < 256 ? n_cols : 256;
+    if (tn == 256 && (long long)p.num_m_tiles * ((n_cols + 255) / 256) < 2LL * sm_count) tn = 128;
+    p.tile_n = tn;
+    p.num_n_tiles = (n_cols + tn - 1) / tn;
+    const size_t budget = 200 * 1024;
+    const size_t b_sub = (size_t)tn * p.kc;
+    const size_t b_all = b_sub * pl.chunks * p.ntaps;
+    pl.b_resident = (p.num_n_tiles == 1 && b_all + 2 * (size_t)pl.a_bytes <= budget && b_all < (1u << 20)) ? 1 : 0;
+    if (pl.b_resident) {
+        size_t na = (budget - b_all) / pl.a_bytes;
+        pl.num_a = na > 4 ? 4 : (int)na;
+        pl.num_b = 1;
+    } else {
+        pl.num_a = pl.chunks > 1 ? 3 : 2;
+        if ((size_t)pl.num_a * pl.a_bytes + 2 * b_sub > budget) return false;
+        size_t nb = (budget - (size_t)pl.num_a * pl.a_bytes) / b_sub;
+        pl.num_b = nb > 8 ? 8 : (int)nb;
+    }
+    return pl.num_a >= 2 || (pl.b_resident && pl.num_a >= 1);
 }
 
 }  // namespace
@@ -431,6 +499,10 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
 
     IgemmParams p;
     memset(&p, 0, sizeof(p));
+    PatchPlan pl;
+    memset(&pl, 0, sizeof(pl));
+    const bool patch = d.stride == 1 && d.kh == d.kw && d.x_wmargin == 0 && !x_exp &&
+                       plan_patch(p, pl, d.n, d.c_in, g.ho, g.wo, d.kh, d.pad, d.c_out, h->sm_count);
     p.M = d.n * g.ho * g.wo;
     p.N = d.c_out;
     p.hq = g.ho;
@@ -438,7 +510,9 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     p.src_stride = d.stride;
     p.base_h = -d.pad;
     int8_t *w_rows = nullptr;
-    if (row_window) {
+    if (patch) {
+        for (int t = 0; t < g.taps; ++t) p.tap_b[t] = (unsigned char)t;
+    } else if (row_window) {
         // K sub-tile = one filter row (8 pixels x 16 channels); the map's W axis already steps by the stride
         plan_igemm(p, 128, d.kh, h->sm_count);
         p.src_stride_w = 1;
@@ -489,6 +563,15 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
         count_launches(h, 1);
     }
     CUtensorMap map_a, map_b;
+    if (patch) {
+        if (!make_patch_map(&map_a, x, d.n, d.h, d.w, d.c_in, p.kc, pl.pw, pl.r_rows + d.kh - 1) ||
+            !make_weight_map(&map_b, w, d.c_out, g.taps, d.c_in, p.kc, p.tile_n))
+            return EOQ_ERR_UNSUPPORTED;
+        const int ptiles = p.num_m_tiles * p.num_n_tiles;
+        count_launches(h, 1);
+        ProfScope prof(h, EOQ_PROF_IGEMM_FWD, s);
+        return record(h, launch_igemm_patch(p, pl, map_a, map_b, ptiles < h->sm_count ? ptiles : h->sm_count, s));
+    }
     if (row_window) {
         if (!make_row_window_map(&map_a, x, d.n, d.h, w_mem, d.x_wmargin - d.pad, g.wo, g.ho, d.stride, d.pad, kTileM) ||
             !make_weight_map(&map_b, w_rows, d.c_out, d.kh, 128, 128, p.tile_n))
@@ -529,6 +612,38 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
 
     // One GEMM per residue class (y mod stride, x mod stride) of the input pixels: within a class the taps
     // kh with (y + pad - kh) divisible by the stride form a unit-stride correlation over e3.
+    if (d.stride == 1 && d.kh == d.kw && d.kh - 1 - d.pad >= 0) {
+        // stride 1: one correlation of e3 with the flipped filter, padding k - 1 - pad
+        IgemmParams p;
+        memset(&p, 0, sizeof(p));
+        PatchPlan pl;
+        memset(&pl, 0, sizeof(pl));
+        if (plan_patch(p, pl, d.n, d.c_out, d.h, d.w, d.kh, d.kh - 1 - d.pad, d.c_in, h->sm_count)) {
+            for (int a = 0; a < d.kh; ++a)
+                for (int b = 0; b < d.kw; ++b) p.tap_b[a * d.kw + b] = (unsigned char)((d.kh - 1 - a) * d.kw + (d.kw - 1 - b));
+            p.out_h = d.h;
+            p.out_w = d.w;
+            p.out_step = 1;
+            p.epilogue = kEpiDgrad;
+            p.acc_out = sums;
+            p.dev = h->dev;
+            CUtensorMap map_a, map_b;
+            if (!make_patch_map(&map_a, e3, d.n, g.ho, g.wo, d.c_out, p.kc, pl.pw, pl.r_rows + d.kh - 1) ||
+                !make_weight_map(&map_b, wt, d.c_in, g.taps, d.c_out, p.kc, p.tile_n))
+                return EOQ_ERR_UNSUPPORTED;
+            const int ptiles = p.num_m_tiles * p.num_n_tiles;
+            count_launches(h, 1);
+            {
+                ProfScope prof(h, EOQ_PROF_IGEMM_DGRAD, s);
+                e = launch_igemm_patch(p, pl, map_a, map_b, ptiles < h->sm_count ? ptiles : h->sm_count, s);
+            }
+            if (e != cudaSuccess) return record(h, e);
+            e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
+                              h->sm_count, s);
+            count_launches(h, 1);
+            return record(h, e);
+        }
+    }
     // a class no tap reaches (e.g. the odd pixels of a strided 1x1 filter) keeps zero sums: clear first
     bool any_empty = false;
     for (int r = 0; r < d.stride; ++r) {

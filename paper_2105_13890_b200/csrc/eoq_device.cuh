@@ -158,6 +158,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *map, uint3
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void *map, uint32_t bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
 // im2col-mode TMA load on a rank-4 (C, W, H, N) tensor: coordinates of the first pixel plus the
 // filter-tap offsets (w, h).
 __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const void *map, uint32_t bar, int c, int w, int h,
@@ -193,6 +200,9 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // D[tmem] (+)= A[smem desc] * B[smem desc], int8 x int8 -> int32.
+// (No memory clobber: the issuing thread's scalar work between two MMAs is what limits narrow tiles, so the
+// compiler must be free to keep loop state in registers.  Ordering against barrier waits and commits comes from
+// those being volatile asm statements with memory clobbers.)
 __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate)
 {
@@ -200,9 +210,9 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate));
 }
+
 // The mbarrier receives one arrival when every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
@@ -246,6 +256,59 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_b
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout_type << 61);
 }
 
+// The same descriptor split in two 32-bit halves, so that an issue loop only adds byte offsets (in 16-byte
+// units) to the low half: low = start address >> 4 | (leading offset >> 4) << 16, high = (stride offset >> 4) |
+// version bit | swizzle mode.  Building the whole descriptor per MMA costs more cycles than a narrow MMA takes.
+__device__ __forceinline__ uint32_t smem_desc_hi(uint32_t sbo_bytes, uint32_t layout_type)
+{
+    return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (layout_type << 29);
+}
+__device__ __forceinline__ uint64_t smem_desc_join(uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; }
+
+// The thread that feeds the tensor core is a single in-order instruction stream: about 25 scalar instructions
+// per MMA cost ~130 cycles, while a 128 x 64 x 32 MMA takes 52.  The issue helpers below are therefore fully
+// unrolled with compile-time MMA indices, so that an MMA costs a handful of integer adds.
+//
+// Successive MMAs of a tile alternate between two partial accumulators d0 / d1 when the tile has them (an MMA
+// that accumulates into the columns its predecessor is still writing waits ~97 cycles; two interleaved chains
+// run at 52 cycles for 64 columns, 69 for 128).  `fresh` is 1 for the first MMAs of a tile, which overwrite.
+
+// kSteps 32-byte K steps of one (A sub-tile, B sub-tile) pair; `parity` = index of the first MMA modulo 2.
+template <int kSteps>
+__device__ __forceinline__ void mma_k_steps(uint32_t d0, uint32_t d1, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
+                                            uint32_t idesc, uint32_t parity, uint32_t fresh0, uint32_t fresh1)
+{
+#pragma unroll
+    for (int kk = 0; kk < kSteps; ++kk) {
+        const bool odd = ((kk & 1) != 0) != (parity != 0);
+        // the first MMA into each accumulator overwrites it
+        uint32_t acc = 1u;
+        if (kk < 2) acc = (odd ? fresh1 : fresh0) ? 0u : 1u;
+        ptx::mma_i8(odd ? d1 : d0, smem_desc_join(a_lo + 2 * kk, hi), smem_desc_join(b_lo + 2 * kk, hi), idesc, acc);
+    }
+}
+
+// All kDim x kDim taps of one channel chunk against resident weights: tap (a, b) reads the patch tile
+// (a * row16 + b * kc16) further (16-byte units); its weights are the next sub-tile.
+template <int kDim, int kSteps>
+__device__ __forceinline__ void mma_patch_chunk(uint32_t d0, uint32_t d1, uint32_t a_lo, uint32_t b_lo, uint32_t row16,
+                                                uint32_t kc16, uint32_t b_sub16, uint32_t hi, uint32_t idesc,
+                                                bool first_chunk, bool two_acc)
+{
+#pragma unroll
+    for (int a = 0; a < kDim; ++a)
+#pragma unroll
+        for (int b = 0; b < kDim; ++b)
+#pragma unroll
+            for (int kk = 0; kk < kSteps; ++kk) {
+                const int idx = (a * kDim + b) * kSteps + kk;
+                uint32_t acc = 1u;
+                if (idx == 0) acc = first_chunk ? 0u : 1u;
+                if (idx == 1) acc = (first_chunk && two_acc) ? 0u : 1u;
+                ptx::mma_i8((idx & 1) ? d1 : d0, smem_desc_join(a_lo + a * row16 + b * kc16 + 2 * kk, hi),
+                            smem_desc_join(b_lo + (a * kDim + b) * b_sub16 + 2 * kk, hi), idesc, acc);
+            }
+}
 // Swizzle field of the descriptor for a sub-tile whose rows are `row_bytes` wide.
 __device__ __forceinline__ uint32_t layout_type_for(int row_bytes)
 {

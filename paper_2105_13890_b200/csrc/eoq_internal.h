@@ -89,6 +89,28 @@ struct IgemmParams {
     DeviceState *dev;
 };
 
+// Patch variant of the implicit GEMM for stride-1 filters (eoq_igemm_patch.cu): an M tile is `r_rows` output rows
+// of one image in the raster of a patch that is (kdim - 1) pixels wider than the output row; the patch of source
+// pixels is loaded once and every filter tap reads it through a descriptor started (a * pw + b) rows further.
+struct PatchPlan {
+    int n_img;
+    int kdim;           // square filter size
+    int pad;            // tap (a, b) reads source pixel (y + a - pad, x + b - pad)
+    int pw;             // patch width = wq + kdim - 1
+    int r_rows;         // output rows per tile
+    int tiles_per_img;
+    int chunks;         // source channels / kc
+    int a_bytes;        // bytes of one patch buffer (multiple of 1024)
+    int a_box_bytes;    // bytes one patch load delivers
+    int num_a, num_b;   // ring depths (patches, weight sub-tiles)
+    int b_resident;     // all weight sub-tiles of the layer stay in shared memory
+};
+constexpr int kPatchThreads = 384;  // warps: 0 patch loads, 1 MMA + TMEM, 2 weight loads, 3 idle, 4..11 epilogue
+
+size_t igemm_patch_smem_bytes(const IgemmParams &p, const PatchPlan &pl);
+cudaError_t launch_igemm_patch(const IgemmParams &p, const PatchPlan &pl, const CUtensorMap &map_a,
+                               const CUtensorMap &map_b, int grid, cudaStream_t stream);
+
 size_t igemm_smem_bytes(const IgemmParams &p);
 cudaError_t launch_igemm(const IgemmParams &p, const CUtensorMap &map_a, const CUtensorMap &map_b, int grid,
                          cudaStream_t stream);

@@ -135,19 +135,24 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, true, true);
+            // descriptor halves that do not change; the loop adds row offsets to the low halves
+            const uint64_t a_proto = mn_major_desc(0, p.kc, a_sub), b_proto = mn_major_desc(0, p.nc, b_sub);
+            const uint32_t a_hi = (uint32_t)(a_proto >> 32), b_hi = (uint32_t)(b_proto >> 32);
+            const uint32_t a_lead = (uint32_t)a_proto, b_lead = (uint32_t)b_proto;  // leading-offset field, address 0
+            const uint32_t a_step16 = (32u * p.kc) >> 4, b_step16 = (32u * p.nc) >> 4;  // 32 pixels further down
             int stage = 0;
             uint32_t phase = 0, accumulate = 0;
             bool ok = true;
             for (int it = 0; it < my_stages; ++it) {
                 if (!(ok = wait_bar(full_bar(stage), phase, ctx))) break;
                 ptx::tc_fence_after();
-                const uint32_t a_base = smem_base + stage * stage_bytes;
-                const uint32_t b_base = a_base + p.subs_per_mtile * a_sub;
+                uint32_t a_lo = ((smem_base + stage * stage_bytes) >> 4) | a_lead;
+                uint32_t b_lo = (((smem_base + stage * stage_bytes) >> 4) + ((p.subs_per_mtile * a_sub) >> 4)) | b_lead;
                 for (int k = 0; k < px; k += 32) {
-                    // 32 pixels further down: 32 rows of the sub-tile
-                    ptx::mma_i8(tmem_base, mn_major_desc(a_base + k * p.kc, p.kc, a_sub),
-                                mn_major_desc(b_base + k * p.nc, p.nc, b_sub), idesc, accumulate);
+                    ptx::mma_i8(tmem_base, smem_desc_join(a_lo, a_hi), smem_desc_join(b_lo, b_hi), idesc, accumulate);
                     accumulate = 1;
+                    a_lo += a_step16;
+                    b_lo += b_step16;
                 }
                 ptx::mma_commit(empty_bar(stage));
                 if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }
