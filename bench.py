@@ -286,6 +286,7 @@ def run_gpu(args):
                 "igemm_dgrad": {"launches": prof_n[1], "ms": prof_ms[1], "tops": dgrad_ops / (prof_ms[1] / 1e3) / 1e12 if prof_ms[1] else None},
                 "wgrad": {"launches": prof_n[2], "ms": prof_ms[2], "tops": fwd_ops / (prof_ms[2] / 1e3) / 1e12 if prof_ms[2] else None},
             },
+            "ms_per_step_by_kind": {name: prof_ms[i] / args.steps for i, name in enumerate(eoq.EOQ_PROF_NAMES)},
         }
         if world == 1 and not args.no_cpu_baseline:
             import oracle

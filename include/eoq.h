@@ -206,16 +206,22 @@ EOQ_API int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t *d
 EOQ_API int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits);
 
 /*
- * Instrumentation (off by default).  Between eoq_profile_start and eoq_profile_stop every launch of the two
- * tensor-core kernels is bracketed by CUDA events on its stream.  eoq_profile_stop synchronises the device,
- * and reports per kind (EOQ_PROF_*) the number of launches and their summed duration in milliseconds; it
- * keeps at most 8192 launches.  eoq_launch_count returns how many kernels this handle has launched so far.
+ * Instrumentation (off by default).  Between eoq_profile_start and eoq_profile_stop the kernels of each call are
+ * bracketed by CUDA events on their stream, grouped in EOQ_PROF_KINDS kinds.  eoq_profile_stop synchronises the
+ * device and reports per kind the number of bracketed groups and their summed duration in milliseconds; it keeps
+ * at most 8192 groups.  eoq_launch_count returns how many kernels this handle has launched so far.
  */
-#define EOQ_PROF_IGEMM_FWD 0
-#define EOQ_PROF_IGEMM_DGRAD 1
-#define EOQ_PROF_WGRAD 2
+#define EOQ_PROF_IGEMM_FWD 0     /* the forward implicit-GEMM kernel, one launch per group */
+#define EOQ_PROF_IGEMM_DGRAD 1   /* the dgrad implicit-GEMM kernel, one launch per group */
+#define EOQ_PROF_WGRAD 2         /* the weight-gradient GEMM kernel */
+#define EOQ_PROF_ERR_HEAD 3      /* eoq_err_prescale (two kernels) */
+#define EOQ_PROF_DGRAD_AUX 4     /* weight transpose, Q_e phase 2 */
+#define EOQ_PROF_WGRAD_AUX 5     /* b1 error sums, Q_g */
+#define EOQ_PROF_FWD_AUX 6       /* b1 weight table, weight row padding */
+#define EOQ_PROF_OTHER 7         /* quantizers, update, layout change */
+#define EOQ_PROF_KINDS 8
 EOQ_API int eoq_profile_start(eoq_handle_t handle);
-EOQ_API int eoq_profile_stop(eoq_handle_t handle, int launches[3], double milliseconds[3]);
+EOQ_API int eoq_profile_stop(eoq_handle_t handle, int launches[EOQ_PROF_KINDS], double milliseconds[EOQ_PROF_KINDS]);
 EOQ_API unsigned long long eoq_launch_count(eoq_handle_t handle);
 
 /* The last cudaError_t a call on this handle recorded (0 if none). */

@@ -275,6 +275,63 @@ bool plan_patch(IgemmParams &p, PatchPlan &pl, int n_img, int c_src, int hq, int
     return pl.num_a >= 2 || (pl.b_resident && pl.num_a >= 1);
 }
 
+// Plan of the patch variant of the weight gradient; false when the geometry does not suit it.
+bool plan_wgrad_patch(WgradPatchPlan &pl, const eoq_conv_desc_t &d, int ho, int wo)
+{
+    if (d.stride != 1 || d.kh != d.kw || d.kh < 2 || d.x_wmargin != 0 || d.c_in % 32 || d.c_out % 32) return false;
+    if (d.pad > d.kh - 1) return false;
+    memset(&pl, 0, sizeof(pl));
+    pl.n_img = d.n; pl.ho = ho; pl.wo = wo; pl.c_in = d.c_in; pl.c_out = d.c_out;
+    pl.kdim = d.kh; pl.pad = d.pad;
+    pl.pw = wo + d.kh - 1;
+    if (pl.pw > 256) return false;
+    pl.kc = chunk_bytes(d.c_in);
+    pl.chunks = d.c_in / pl.kc;
+    pl.apa = 128 / pl.kc;
+    pl.accs_per_row = (d.kh + pl.apa - 1) / pl.apa;
+    pl.tile_n = chunk_bytes(d.c_out);
+    pl.n_tiles = d.c_out / pl.tile_n;
+    int rpg = 512 / (pl.tile_n * pl.accs_per_row);
+    if (rpg * pl.accs_per_row > 8) rpg = 8 / pl.accs_per_row;
+    if (rpg > d.kh) rpg = d.kh;
+    if (rpg < 1) return false;
+    pl.rows_per_group = rpg;
+    pl.row_groups = (d.kh + rpg - 1) / rpg;
+    pl.num_groups = pl.n_tiles * pl.chunks * pl.row_groups;
+    pl.rows_total = d.kh * d.kw * d.c_in;
+    // rows per pixel block: as many as keep one stage near 64 KB (three stages in flight)
+    int r = ho < 32 ? ho : 32;
+    for (; r >= 1; --r) {
+        const int kp = (r * pl.pw + 31) / 32 * 32;
+        int x_rows = (r + d.kh - 1) * pl.pw;
+        const int x_read = (d.kh - 1) * (pl.pw + 1) + pl.apa + kp;
+        if (x_read > x_rows) x_rows = x_read;
+        pl.x_bytes = (x_rows * pl.kc + 1023) / 1024 * 1024;
+        pl.e_bytes = (kp * pl.tile_n + 1023) / 1024 * 1024;
+        pl.kp = kp;
+        if (pl.x_bytes + pl.e_bytes <= 66 * 1024) break;
+    }
+    if (r < 1) return false;
+    pl.r_rows = r;
+    pl.blocks_per_img = (ho + r - 1) / r;
+    pl.x_box_bytes = pl.kc * pl.pw * (r + d.kh - 1);
+    pl.e_box_bytes = pl.tile_n * pl.pw * r;
+    int stages = (200 * 1024) / (pl.x_bytes + pl.e_bytes);
+    pl.num_stages = stages > 4 ? 4 : stages;
+    if (pl.num_stages < 2) return false;
+    const int total_blocks = d.n * pl.blocks_per_img;
+    int splits = (kWgradTargetCtas + pl.num_groups - 1) / pl.num_groups;
+    if (splits > total_blocks) splits = total_blocks;
+    if (splits < 1) splits = 1;
+    int per = (total_blocks + splits - 1) / splits;
+    const int max_per = 130000 / pl.kp;  // keeps a CTA's int32 partial sums exact: rows * 127 * 128 < 2^31
+    if (max_per < 1) return false;
+    if (per > max_per) per = max_per;
+    pl.blocks_per_split = per;
+    pl.num_splits = (total_blocks + per - 1) / per;
+    return true;
+}
+
 }  // namespace
 
 // ================================================================================= handle
@@ -350,13 +407,13 @@ extern "C" int eoq_profile_start(eoq_handle_t handle)
     return EOQ_OK;
 }
 
-extern "C" int eoq_profile_stop(eoq_handle_t handle, int launches[3], double milliseconds[3])
+extern "C" int eoq_profile_stop(eoq_handle_t handle, int launches[EOQ_PROF_KINDS], double milliseconds[EOQ_PROF_KINDS])
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
     if (!h || !launches || !milliseconds) return EOQ_ERR_BAD_ARG;
     h->profiling = false;
     cudaError_t e = cudaDeviceSynchronize();
-    for (int k = 0; k < 3; ++k) {
+    for (int k = 0; k < EOQ_PROF_KINDS; ++k) {
         launches[k] = 0;
         milliseconds[k] = 0.0;
     }
@@ -454,10 +511,13 @@ extern "C" int eoq_workspace_size(const eoq_conv_desc_t *desc, int pass, size_t 
         case EOQ_PASS_DGRAD:  // transposed weights + int32 sums
             *bytes = round256(g.w_elems) + round256(g.in_elems * sizeof(int32_t));
             return EOQ_OK;
-        case EOQ_PASS_WGRAD:  // int64 sums + per-tap error sums + per-class error sums
+        case EOQ_PASS_WGRAD: {  // int64 sums + per-tap error sums + per-class error sums + split-K slices
+            WgradPatchPlan wp;
+            const size_t slices = plan_wgrad_patch(wp, *desc, g.ho, g.wo) ? (size_t)wp.num_splits * g.w_elems * sizeof(int32_t) : 0;
             *bytes = round256(g.w_elems * sizeof(long long)) + round256((size_t)desc->c_out * g.taps * sizeof(long long)) +
-                     round256(b1_error_scratch_bytes(*desc, bc));
+                     round256(b1_error_scratch_bytes(*desc, bc)) + round256(slices);
             return EOQ_OK;
+        }
         default: return EOQ_ERR_BAD_ARG;
     }
 }
@@ -524,6 +584,7 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
         }
         const BorderClasses bc0 = border_classes(d, g);
         w_rows = reinterpret_cast<int8_t *>(workspace) + round256((size_t)bc0.nrc * bc0.ncc * d.c_out * sizeof(int32_t));
+        ProfScope prof(h, EOQ_PROF_FWD_AUX, s);
         cudaError_t e = launch_weight_pad_rows(w, w_rows, d.c_out, d.kh, d.kw, s);
         if (e != cudaSuccess) return record(h, e);
         count_launches(h, 1);
@@ -558,6 +619,7 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
         p.b1_table = reinterpret_cast<const int32_t *>(workspace);
         p.b1_nlo_h = bc.nlo_h; p.b1_nhi_h = bc.nhi_h; p.b1_nrc = bc.nrc;
         p.b1_nlo_w = bc.nlo_w; p.b1_nhi_w = bc.nhi_w; p.b1_ncc = bc.ncc;
+        ProfScope prof(h, EOQ_PROF_FWD_AUX, s);
         cudaError_t e = launch_b1_weight_table(w, reinterpret_cast<int32_t *>(workspace), d, bc, s);
         if (e != cudaSuccess) return record(h, e);
         count_launches(h, 1);
@@ -605,8 +667,12 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
 
     int8_t *wt = reinterpret_cast<int8_t *>(workspace);
     int32_t *sums = acc_dump ? acc_dump : reinterpret_cast<int32_t *>(reinterpret_cast<char *>(workspace) + round256(g.w_elems));
-    cudaError_t e = launch_reset_cells(h->dev, s);
-    if (e == cudaSuccess) e = launch_weight_transpose(w, wt, d.c_out, g.taps, d.c_in, s);
+    cudaError_t e;
+    {
+        ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
+        e = launch_reset_cells(h->dev, s);
+        if (e == cudaSuccess) e = launch_weight_transpose(w, wt, d.c_out, g.taps, d.c_in, s);
+    }
     if (e != cudaSuccess) return record(h, e);
     count_launches(h, 1);
 
@@ -638,8 +704,11 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                 e = launch_igemm_patch(p, pl, map_a, map_b, ptiles < h->sm_count ? ptiles : h->sm_count, s);
             }
             if (e != cudaSuccess) return record(h, e);
-            e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
-                              h->sm_count, s);
+            {
+                ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
+                e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true,
+                                  h->dev, h->sm_count, s);
+            }
             count_launches(h, 1);
             return record(h, e);
         }
@@ -716,8 +785,11 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             if (e != cudaSuccess) return record(h, e);
         }
     // Q_e over the whole tensor: the maximum is complete only now
-    e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
-                      h->sm_count, s);
+    {
+        ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
+        e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
+                          h->sm_count, s);
+    }
     count_launches(h, 1);
     return record(h, e);
 }
@@ -741,6 +813,38 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
 
     long long *acc = reinterpret_cast<long long *>(workspace);
     long long *tap_sums = reinterpret_cast<long long *>(reinterpret_cast<char *>(workspace) + round256(g.w_elems * sizeof(long long)));
+
+    WgradPatchPlan wp;
+    if (plan_wgrad_patch(wp, d, g.ho, g.wo)) {
+        const BorderClasses bc = border_classes(d, g);
+        if (b1_c != 0 && bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
+        long long *class_sums = reinterpret_cast<long long *>(reinterpret_cast<char *>(tap_sums) +
+                                                              round256((size_t)d.c_out * g.taps * sizeof(long long)));
+        wp.partials = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(class_sums) + round256(b1_error_scratch_bytes(d, bc)));
+        wp.dev = h->dev;
+        cudaError_t e = cudaSuccess;
+        if (b1_c != 0) {
+            ProfScope prof(h, EOQ_PROF_WGRAD_AUX, s);
+            e = launch_b1_error_sums(e3, tap_sums, class_sums, d, g.ho, g.wo, bc, h->sm_count, s);
+            count_launches(h, 2);
+        }
+        if (e != cudaSuccess) return record(h, e);
+        CUtensorMap map_x, map_e;
+        if (!make_patch_map(&map_x, x, d.n, d.h, d.w, d.c_in, wp.kc, wp.pw, wp.r_rows + d.kh - 1) ||
+            !make_patch_map(&map_e, e3, d.n, g.ho, g.wo, d.c_out, wp.tile_n, wp.pw, wp.r_rows))
+            return EOQ_ERR_UNSUPPORTED;
+        count_launches(h, 3);
+        {
+            ProfScope prof(h, EOQ_PROF_WGRAD, s);
+            e = launch_wgrad_patch(wp, map_x, map_e, s);
+        }
+        if (e != cudaSuccess) return record(h, e);
+        ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
+        e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
+                          b1_c != 0 ? tap_sums : nullptr, b1_c, g.taps, d.c_in, wp.partials, wp.num_splits, h->dev,
+                          h->sm_count, s);
+        return record(h, e);
+    }
 
     WgradParams p;
     memset(&p, 0, sizeof(p));
@@ -802,6 +906,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     p.acc = acc;
     p.dev = h->dev;
 
+    ProfScope *aux = new (std::nothrow) ProfScope(h, EOQ_PROF_WGRAD_AUX, s);
     cudaError_t e = cudaMemsetAsync(acc, 0, g.w_elems * sizeof(long long), s);
     if (e == cudaSuccess && b1_c != 0) {
         const BorderClasses bc = border_classes(d, g);
@@ -811,6 +916,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         e = launch_b1_error_sums(e3, tap_sums, class_sums, d, g.ho, g.wo, bc, h->sm_count, s);
         count_launches(h, 2);
     }
+    delete aux;
     if (e != cudaSuccess) return record(h, e);
     CUtensorMap map_x, map_e;
     if (!make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage)) return EOQ_ERR_UNSUPPORTED;
@@ -826,8 +932,9 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     }
     if (e != cudaSuccess) return record(h, e);
     // the kernel leaves sums as [oc][tap][ic], which is the layout of g
+    ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
     e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
-                      b1_c != 0 ? tap_sums : nullptr, b1_c, g.taps, d.c_in, h->dev, h->sm_count, s);
+                      b1_c != 0 ? tap_sums : nullptr, b1_c, g.taps, d.c_in, nullptr, 0, h->dev, h->sm_count, s);
     return record(h, e);
 }
 
@@ -846,6 +953,7 @@ extern "C" int eoq_quantize(eoq_handle_t handle, int mode, const void *src, int 
     if (!aligned16(src) || !aligned16(dst)) return EOQ_ERR_ALIGNMENT;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     count_launches(h, mode == EOQ_SQ ? 2 : 1);
+    ProfScope prof(h, EOQ_PROF_OTHER, s);
     if (src_is_float)
         return record(h, launch_quantize_f32(mode, reinterpret_cast<const float *>(src), n, dst, dst_exp, h->dev, h->sm_count, s));
     if (mode != EOQ_SQ || !src_exp) return EOQ_ERR_UNSUPPORTED;
@@ -863,6 +971,7 @@ extern "C" int eoq_err_prescale(eoq_handle_t handle, const int8_t *e0, const int
     if (gamma_c < -32768 || gamma_c > 32767) return EOQ_ERR_RANGE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     count_launches(h, 2);
+    ProfScope prof(h, EOQ_PROF_ERR_HEAD, s);
     return record(h, launch_err_prescale(e0, e0_exp, relu_mask, x2, n_el, gamma_c, e3, e3_exp,
                                          reinterpret_cast<long long *>(sum_e1), reinterpret_cast<long long *>(sum_e1x2),
                                          h->dev, h->sm_count, s));
@@ -887,6 +996,7 @@ extern "C" int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const 
     }
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     count_launches(h, 2 * ((num + 63) / 64));
+    ProfScope prof(h, EOQ_PROF_OTHER, s);
     return record(h, launch_update(t, num, lr_mant, lr_exp, round_mode == EOQ_ROUND_STOCHASTIC, seed, step, h->dev, h->sm_count, s));
 }
 
@@ -908,6 +1018,7 @@ extern "C" int eoq_quantize_image(eoq_handle_t handle, const float *src, int n, 
         return EOQ_ERR_BAD_ARG;
     if (c_dst % 16 || c_dst > 64 || !aligned16(src) || !aligned16(dst)) return EOQ_ERR_ALIGNMENT;
     count_launches(h, 2);
+    ProfScope prof(h, EOQ_PROF_OTHER, reinterpret_cast<cudaStream_t>(stream));
     return record(h, launch_quantize_image(src, n, hh, ww, c_src, c_dst, wmargin, dst, dst_exp, h->dev, h->sm_count,
                                            reinterpret_cast<cudaStream_t>(stream)));
 }

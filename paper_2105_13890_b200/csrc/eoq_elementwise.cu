@@ -238,15 +238,21 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
 // Adds the b1 term of x1 = x0 + b1 (b1 times the sum of the error over the pixels whose tap falls inside
 // the image), optionally copies the exact sums out, and reduces max |.|.
 __global__ void wgrad_fix_absmax_kernel(long long *acc, size_t n, const long long *tap_sums, int32_t b1_c, int taps,
-                                        int c_in, long long *copy_out, DeviceState *dev)
+                                        int c_in, const int32_t *__restrict__ parts, int num_parts, long long *copy_out,
+                                        DeviceState *dev)
 {
     unsigned long long mx = 0;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        long long v = acc[i];
-        if (tap_sums) {
-            v += (long long)b1_c * tap_sums[i / c_in];  // index of (oc, tap)
-            acc[i] = v;
+        long long v;
+        if (parts) {
+            // the split-K slices of the patch kernel: exact in 64 bits whatever the reduction length
+            v = 0;
+            for (int s = 0; s < num_parts; ++s) v += (long long)__ldg(parts + (size_t)s * n + i);
+        } else {
+            v = acc[i];
         }
+        if (tap_sums) v += (long long)b1_c * tap_sums[i / c_in];  // index of (oc, tap)
+        if (parts || tap_sums) acc[i] = v;
         if (copy_out) copy_out[i] = v;
         const unsigned long long a = (unsigned long long)(v < 0 ? -v : v);
         mx = a > mx ? a : mx;
@@ -659,12 +665,12 @@ cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bi
 
 cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int taps,
-                          int c_in, DeviceState *dev, int sm_count, cudaStream_t s)
+                          int c_in, const int32_t *parts, int num_parts, DeviceState *dev, int sm_count, cudaStream_t s)
 {
     cudaError_t e = launch_reset_cells(dev, s);
     if (e != cudaSuccess) return e;
     wgrad_fix_absmax_kernel<<<grid_for(n, sm_count), kThreads, 0, s>>>(const_cast<long long *>(src), n, tap_sums, b1_c,
-                                                                       taps, c_in, copy_out, dev);
+                                                                       taps, c_in, parts, num_parts, copy_out, dev);
     sq_i64_kernel<<<grid_for(n, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, dev);
     return cudaGetLastError();
 }

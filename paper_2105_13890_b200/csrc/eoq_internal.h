@@ -140,6 +140,41 @@ struct WgradParams {
     DeviceState *dev;
 };
 
+// Patch variant of the weight gradient for stride-1 filters (eoq_wgrad_patch.cu).  A pixel block is `r_rows`
+// output rows of one image; the error patch [r_rows x pw pixels] (zero in the pw - wo extra columns) and the
+// activation patch [(r_rows + k - 1) x pw] are loaded once, and the activation operand of tap (a, b) is the same
+// patch read (a * pw + b) rows further.  One CTA = one group (output-channel tile, input-channel chunk, a set of
+// filter rows) x one range of pixel blocks; it leaves int32 partial sums in its own slice (no atomics).
+struct WgradPatchPlan {
+    int n_img, ho, wo;
+    int c_in, c_out;
+    int kdim, pad;
+    int pw;              // patch width = wo + kdim - 1
+    int r_rows;          // output rows per pixel block
+    int blocks_per_img;
+    int kp;              // reduction rows per block, r_rows * pw rounded up to 32
+    int kc, chunks;      // activation channel bytes per chunk (32/64/128), chunks
+    int apa;             // taps per accumulator: 128 / kc adjacent taps of one filter row share an MMA
+    int accs_per_row;    // accumulators per filter row
+    int rows_per_group, row_groups;  // filter rows one CTA handles, groups of them
+    int tile_n, n_tiles; // output-channel columns per CTA (32/64/128)
+    int num_groups;      // n_tiles * chunks * row_groups
+    int num_splits;      // pixel-block ranges
+    int blocks_per_split;
+    int x_bytes, e_bytes;  // bytes of one stage's activation / error buffer (multiples of 1024)
+    int x_box_bytes, e_box_bytes;
+    int num_stages;
+    int rows_total;      // taps * c_in
+    int32_t *partials;   // [num_splits][c_out][taps][c_in]
+    DeviceState *dev;
+};
+constexpr int kWgradPatchThreads = 192;  // warp 0 loads, warp 1 MMA + TMEM, warps 2..5 epilogue
+constexpr int kWgradTargetCtas = 148;    // CTAs the split count aims at (one per SM of a 148-SM part; shared memory allows one)
+
+size_t wgrad_patch_smem_bytes(const WgradPatchPlan &pl);
+cudaError_t launch_wgrad_patch(const WgradPatchPlan &pl, const CUtensorMap &map_x, const CUtensorMap &map_e,
+                               cudaStream_t stream);
+
 size_t wgrad_smem_bytes(const WgradParams &p);
 cudaError_t launch_wgrad(const WgradParams &p, const CUtensorMap &map_x, const CUtensorMap &map_e, cudaStream_t stream);
 
@@ -156,9 +191,11 @@ cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst,
 cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *sum_codes, bool max_already_reduced, DeviceState *dev,
                           int sm_count, cudaStream_t s);
+// Q_g of the exact sums.  `src` holds int64 sums; when `parts` is given the sums are first formed from
+// `num_parts` int32 slices of n elements each (and written to src).
 cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int taps,
-                          int c_in, DeviceState *dev, int sm_count, cudaStream_t s);
+                          int c_in, const int32_t *parts, int num_parts, DeviceState *dev, int sm_count, cudaStream_t s);
 cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const uint8_t *mask, const int16_t *x2,
                                 size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
                                 long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s);

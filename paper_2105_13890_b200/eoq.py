@@ -29,6 +29,8 @@ EXPORTS = [
 ]
 EOQ_STATIC_SCRATCH_BYTES = 16 << 20
 EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
+EOQ_PROF_KINDS = 8
+EOQ_PROF_NAMES = ["igemm_fwd", "igemm_dgrad", "wgrad_gemm", "err_head", "dgrad_aux", "wgrad_aux", "fwd_aux", "other"]
 
 
 class EoqError(RuntimeError):
@@ -231,9 +233,9 @@ def eoq_profile_start(handle) -> None:
 
 
 def eoq_profile_stop(handle):
-    """-> ([launches per kind], [milliseconds per kind]) for kinds EOQ_PROF_IGEMM_FWD, _IGEMM_DGRAD, _WGRAD."""
-    n = (C.c_int * 3)()
-    ms = (C.c_double * 3)()
+    """-> ([groups per kind], [milliseconds per kind]) for the EOQ_PROF_KINDS kinds (names in EOQ_PROF_NAMES)."""
+    n = (C.c_int * EOQ_PROF_KINDS)()
+    ms = (C.c_double * EOQ_PROF_KINDS)()
     _check(lib().eoq_profile_stop(handle, n, ms), "eoq_profile_stop")
     return list(n), list(ms)
 
