@@ -191,27 +191,36 @@ def run_gpu(args):
     step = TrainStep(wl, handle, f"cuda:{local}", scalars=Scalars())
     stream = torch.cuda.current_stream()
 
+    # One step = one replay of a CUDA graph of the whole path (the weight-gradient chain of each layer on a side
+    # stream next to its dgrad chain); --eager launches call by call on one stream instead.
+    if args.eager:
+        do_step = step.run
+    else:
+        step.capture(overlap=True)
+        do_step = step.replay
     for _ in range(args.warmup):
-        step.run()
+        do_step()
     barrier()
-    status = eoq.eoq_last_status(handle)
+    status = step.status()
 
     sampler = ClockSampler(local) if rank == 0 else None
     time.sleep(0.3)
     # ---- timed region: K steps, inputs resident
-    l0 = eoq.eoq_launch_count(handle)
+    l0 = eoq.eoq_launch_count(handle) + eoq.eoq_launch_count(step.h_side)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t_wall0 = time.time()
     ev0.record(stream)
     for _ in range(args.steps):
-        step.run()
+        do_step()
     ev1.record(stream)
     barrier()
     t_wall1 = time.time()
     ms = ev0.elapsed_time(ev1)
-    launches = eoq.eoq_launch_count(handle) - l0
-    status |= eoq.eoq_last_status(handle)
+    launches = eoq.eoq_launch_count(handle) + eoq.eoq_launch_count(step.h_side) - l0
+    if not args.eager:
+        launches = step.launches_per_step * args.steps  # graph replays do not pass through the host-side counter
+    status |= step.status()
 
     # ---- end to end: host image in (pinned), results out, every step
     host_img = torch.from_numpy(step.host_image(12345)).pin_memory()
@@ -224,7 +233,7 @@ def run_gpu(args):
     e0.record(stream)
     for _ in range(args.steps):
         step.image.copy_(host_img, non_blocking=True)
-        step.run()
+        do_step()
         for src, dst in zip(results, host_out):
             dst.copy_(src, non_blocking=True)
     e1.record(stream)
@@ -268,7 +277,8 @@ def run_gpu(args):
             "pct_of_int8_peak": 100.0 * tops / world / int8_peak,
             "config": {"workload": wl.name, "layers": len(wl.layers), "global_batch": world * wl.batch,
                        "gop_per_step": ops_step / 1e9, "l2": "working set larger than L2; no flush between steps",
-                       "scalars": "b1=-2 gamma=118 b2=3 codes", "parallelism": f"replicas x{world}"},
+                       "scalars": "b1=-2 gamma=118 b2=3 codes", "parallelism": f"replicas x{world}",
+                       "launch": "eager, one stream" if args.eager else "CUDA graph replay, wgrad chain on a side stream"},
             "clocks": clocks,
             "e2e": {"value": tops_e2e, "unit": "TOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": ms_e2e / args.steps},
@@ -313,6 +323,7 @@ def main():
     ap.add_argument("--ref-batch", type=int, default=4, help="batch of the CPU-oracle sample timed beside the GPU run")
     ap.add_argument("--ref-arm-batch", type=int, default=1, help="batch of each step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--eager", action="store_true", help="launch call by call on one stream instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

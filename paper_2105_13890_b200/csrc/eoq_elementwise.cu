@@ -235,6 +235,33 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
 
 // ------------------------------------------------------------------ int64 -> SQ (Q_g after the weight gradient)
 
+// Sums the int32 split-K slices of the patch kernel into int64 (exact whatever the reduction length).
+// Block = (256 / groups) elements x `groups` slice groups: every thread adds its share of the slices with
+// independent, coalesced loads; the groups meet in shared memory.  Few slices -> one group, many -> eight.
+__global__ void wgrad_sum_slices_kernel(const int32_t *__restrict__ parts, int num_parts, size_t n, long long *acc)
+{
+    __shared__ long long part[256];
+    const int bx = blockDim.x, groups = blockDim.y;
+    for (size_t base = (size_t)blockIdx.x * bx; base < n; base += (size_t)gridDim.x * bx) {
+        const size_t i = base + threadIdx.x;
+        long long v = 0;
+        if (i < n)
+            for (int s = threadIdx.y; s < num_parts; s += groups) v += (long long)__ldg(parts + (size_t)s * n + i);
+        if (groups == 1) {
+            if (i < n) acc[i] = v;
+            continue;
+        }
+        part[threadIdx.y * bx + threadIdx.x] = v;
+        __syncthreads();
+        if (threadIdx.y == 0 && i < n) {
+            long long t = 0;
+            for (int k = 0; k < groups; ++k) t += part[k * bx + threadIdx.x];
+            acc[i] = t;
+        }
+        __syncthreads();
+    }
+}
+
 // Adds the b1 term of x1 = x0 + b1 (b1 times the sum of the error over the pixels whose tap falls inside
 // the image), optionally copies the exact sums out, and reduces max |.|.
 __global__ void wgrad_fix_absmax_kernel(long long *acc, size_t n, const long long *tap_sums, int32_t b1_c, int taps,
@@ -542,8 +569,9 @@ __global__ void b1_weight_table_kernel(const int8_t *__restrict__ w, int32_t *ta
 }
 
 // class_sums[class][oc] = sum of e3[n,y,x,oc] over the pixels of a border class.  A block owns a range of
-// pixels and a slab of 128 channels; each lane keeps 4 channels.  Interior pixels (one class, almost all of a
-// large image) accumulate in registers, border pixels in shared memory.
+// pixels and a slab of channels; a lane keeps 16 channels (one 128-bit load per pixel), so a warp covers
+// 32 / (slab / 16) pixels per step.  Interior pixels (one class, almost all of a large image) accumulate in
+// registers, border pixels in shared memory.
 constexpr int kClassSlab = 128;
 __global__ void b1_class_sums_kernel(const int8_t *__restrict__ e3, long long *class_sums, int c_out, int ho, int wo,
                                      size_t pixels, int pixels_per_block, BorderClasses bc)
@@ -552,29 +580,39 @@ __global__ void b1_class_sums_kernel(const int8_t *__restrict__ e3, long long *c
     const int classes = bc.nrc * bc.ncc;
     for (int i = threadIdx.x; i < classes * kClassSlab; i += blockDim.x) cls_acc[i] = 0;
     __syncthreads();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    const int ch = blockIdx.y * kClassSlab + lane * 4;
-    const bool live = ch < c_out;
+    const int slab_ch = min(kClassSlab, c_out - (int)blockIdx.y * kClassSlab);  // channels of this slab (multiple of 16)
+    const int lanes_per_pix = slab_ch / 16;
+    const int pix_per_step = blockDim.x / lanes_per_pix;
+    const int sub = threadIdx.x % lanes_per_pix, slot = threadIdx.x / lanes_per_pix;
+    const int ch = blockIdx.y * kClassSlab + sub * 16;
     const int interior = (bc.nrc != ho && bc.ncc != wo) ? bc.nlo_h * bc.ncc + bc.nlo_w : -1;
-    int a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+    int acc[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) acc[k] = 0;
     const size_t begin = (size_t)blockIdx.x * pixels_per_block;
     const size_t end = min(pixels, begin + (size_t)pixels_per_block);
-    for (size_t p = begin + warp; p < end; p += nwarps) {
-        const int x = (int)(p % wo), y = (int)((p / wo) % ho);
-        const int cls = border_class(y, ho, bc.nlo_h, bc.nhi_h, bc.nrc) * bc.ncc + border_class(x, wo, bc.nlo_w, bc.nhi_w, bc.ncc);
-        if (!live) continue;
-        const int v = __ldg(reinterpret_cast<const int *>(e3 + p * c_out + ch));
-        const int b0 = (int)(int8_t)(v & 0xff), b1 = (int)(int8_t)((v >> 8) & 0xff), b2 = (int)(int8_t)((v >> 16) & 0xff), b3 = v >> 24;
-        if (cls == interior) {
-            a0 += b0; a1 += b1; a2 += b2; a3 += b3;
-        } else {
-            int32_t *dst = cls_acc + cls * kClassSlab + lane * 4;
-            atomicAdd(dst + 0, b0); atomicAdd(dst + 1, b1); atomicAdd(dst + 2, b2); atomicAdd(dst + 3, b3);
+    if (slot < pix_per_step) {
+        for (size_t p = begin + slot; p < end; p += pix_per_step) {
+            const int x = (int)(p % wo), y = (int)((p / wo) % ho);
+            const int cls = border_class(y, ho, bc.nlo_h, bc.nhi_h, bc.nrc) * bc.ncc + border_class(x, wo, bc.nlo_w, bc.nhi_w, bc.ncc);
+            const int4 v = __ldg(reinterpret_cast<const int4 *>(e3 + p * c_out + ch));
+            const int8_t *b = reinterpret_cast<const int8_t *>(&v);
+            if (cls == interior) {
+#pragma unroll
+                for (int k = 0; k < 16; ++k) acc[k] += b[k];
+            } else {
+                int32_t *dst = cls_acc + cls * kClassSlab + sub * 16;
+#pragma unroll
+                for (int k = 0; k < 16; ++k)
+                    if (b[k]) atomicAdd(dst + k, (int)b[k]);
+            }
         }
-    }
-    if (live && interior >= 0) {
-        int32_t *dst = cls_acc + interior * kClassSlab + lane * 4;
-        atomicAdd(dst + 0, a0); atomicAdd(dst + 1, a1); atomicAdd(dst + 2, a2); atomicAdd(dst + 3, a3);
+        if (interior >= 0) {
+            int32_t *dst = cls_acc + interior * kClassSlab + sub * 16;
+#pragma unroll
+            for (int k = 0; k < 16; ++k)
+                if (acc[k]) atomicAdd(dst + k, acc[k]);
+        }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < classes * kClassSlab; i += blockDim.x) {
@@ -669,6 +707,14 @@ cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_
 {
     cudaError_t e = launch_reset_cells(dev, s);
     if (e != cudaSuccess) return e;
+    if (parts) {
+        const int groups = num_parts >= 32 ? 8 : (num_parts >= 8 ? 4 : 1);
+        const int bx = 256 / groups;
+        size_t blocks = (n + bx - 1) / bx;
+        if (blocks > (size_t)sm_count * 16) blocks = (size_t)sm_count * 16;
+        wgrad_sum_slices_kernel<<<(unsigned)blocks, dim3(bx, groups), 0, s>>>(parts, num_parts, n, const_cast<long long *>(src));
+        parts = nullptr;
+    }
     wgrad_fix_absmax_kernel<<<grid_for(n, sm_count), kThreads, 0, s>>>(const_cast<long long *>(src), n, tap_sums, b1_c,
                                                                        taps, c_in, parts, num_parts, copy_out, dev);
     sq_i64_kernel<<<grid_for(n, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, dev);

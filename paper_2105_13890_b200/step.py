@@ -79,6 +79,12 @@ class TrainStep:
             for p in (eoq.EOQ_PASS_FWD, eoq.EOQ_PASS_DGRAD, eoq.EOQ_PASS_WGRAD):
                 ws = max(ws, eoq.eoq_workspace_size(lb.desc, p))
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=self.dev)
+        # second handle + workspace: the weight-gradient chain of a layer can then run on a side stream next to
+        # the layer's dgrad chain (a handle's reduction cells and a workspace serve one call at a time)
+        self.h_side = eoq.eoq_create(self.dev.index if self.dev.index is not None else 0)
+        self.workspace_side = torch.empty(ws, dtype=torch.uint8, device=self.dev)
+        self.side = torch.cuda.Stream(device=self.dev)
+        self.graph = None
         first = workload.layers[0]
         self.image_channels = image_channels
         self.image_pixels = first.n * first.h * first.w
@@ -115,8 +121,11 @@ class TrainStep:
         torch.cuda.synchronize(self.dev)
 
     # ------------------------------------------------------------------ one step
-    def run(self) -> None:
+    def run(self, overlap: bool = False) -> None:
+        """One step on the current stream.  overlap=True forks every layer's weight-gradient chain to a side
+        stream (it only needs the layer's e3 and x0) and joins before the update."""
         h, sc, ws = self.h, self.sc, self.workspace
+        main = torch.cuda.current_stream(self.dev)
         first = self.layers[0]
         fl = first.layer
         eoq.eoq_quantize_image(h, self.image, fl.n, fl.h, fl.w, self.image_channels, fl.c_in, first.wmargin, first.x0,
@@ -132,12 +141,42 @@ class TrainStep:
             gamma = sc.gamma_c if l.gamma_trainable else 128
             eoq.eoq_err_prescale(h, lb.e0, lb.e0_exp, lb.mask, lb.x2, lb.n_out, gamma, lb.e3, lb.e3_exp, lb.sum_e1,
                                  lb.sum_e1x2 if lb.x2 is not None else None)
+            if overlap:
+                self.side.wait_stream(main)
+                with torch.cuda.stream(self.side):
+                    eoq.eoq_conv_wgrad(self.h_side, lb.desc, lb.e3, lb.e3_exp, lb.x0, 0 if i == 0 else sc.b1_c, lb.g,
+                                       lb.g_exp, None, self.workspace_side)
             if l.has_dgrad:
                 eoq.eoq_conv_dgrad(h, lb.desc, lb.e3, lb.e3_exp, lb.w, lb.e4, lb.e4_exp, lb.sum_e4, None, ws)
-            eoq.eoq_conv_wgrad(h, lb.desc, lb.e3, lb.e3_exp, lb.x0, 0 if i == 0 else sc.b1_c, lb.g, lb.g_exp, None, ws)
+            if not overlap:
+                eoq.eoq_conv_wgrad(h, lb.desc, lb.e3, lb.e3_exp, lb.x0, 0 if i == 0 else sc.b1_c, lb.g, lb.g_exp, None, ws)
+        if overlap:
+            main.wait_stream(self.side)
         eoq.eoq_update(h, [lb.w for lb in self.layers], [lb.g for lb in self.layers], [lb.g_exp for lb in self.layers],
                        self.lr_mant, self.lr_exp, eoq.EOQ_ROUND_STOCHASTIC, seed=synth.BASE_SEED, step=self.step_no)
         self.step_no += 1
+
+    def capture(self, overlap: bool = True) -> None:
+        """Records one step into a CUDA graph (after an eager warm-up step on the capture stream).  Everything a
+        call depends on is baked in at capture, including the update's step counter: replays repeat the same
+        stochastic-rounding draws."""
+        cap = torch.cuda.Stream(device=self.dev)
+        cap.wait_stream(torch.cuda.current_stream(self.dev))
+        with torch.cuda.stream(cap):
+            self.run(overlap)
+        torch.cuda.synchronize(self.dev)
+        before = eoq.eoq_launch_count(self.h) + eoq.eoq_launch_count(self.h_side)
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph, stream=cap):
+            self.run(overlap)
+        torch.cuda.synchronize(self.dev)
+        self.launches_per_step = eoq.eoq_launch_count(self.h) + eoq.eoq_launch_count(self.h_side) - before
+
+    def replay(self) -> None:
+        self.graph.replay()
+
+    def status(self) -> int:
+        return eoq.eoq_last_status(self.h) | eoq.eoq_last_status(self.h_side)
 
     def result_tensors(self):
         """Small per-step results a caller would read back: every gradient exponent and the last activation."""
