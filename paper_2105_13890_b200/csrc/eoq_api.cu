@@ -870,10 +870,20 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     if (p.tile_n % p.nc) p.tile_n = (p.tile_n / p.nc) * p.nc;
     p.num_n_tiles = (d.c_out + p.tile_n - 1) / p.tile_n;
     p.pixels_per_stage = 64;
+    // M tiles accumulated side by side by one CTA share the stage's error tile (fewer TMA rows per MMA): as many
+    // as tensor memory (512 columns) and three pipeline stages of shared memory allow
+    {
+        int mpc = 512 / p.tile_n;
+        const size_t a_mtile = (size_t)p.subs_per_mtile * p.pixels_per_stage * p.kc, b_tile = (size_t)p.tile_n * p.pixels_per_stage;
+        while (mpc > 1 && 3 * (mpc * a_mtile + b_tile) > 200 * 1024) --mpc;
+        if (mpc > p.num_m_tiles) mpc = p.num_m_tiles;
+        p.mtiles_per_cta = mpc < 1 ? 1 : mpc;
+        p.num_m_groups = (p.num_m_tiles + p.mtiles_per_cta - 1) / p.mtiles_per_cta;
+    }
     const int total_stages = (p.P + p.pixels_per_stage - 1) / p.pixels_per_stage;
     // a 64-pixel stage adds at most 64 * 127 * 255 to an int32 partial sum: cap the stages one CTA runs
     const int max_stages_exact = 1024;
-    const int tiles = p.num_m_tiles * p.num_n_tiles;
+    const int tiles = p.num_m_groups * p.num_n_tiles;
     int splits = (2 * h->sm_count + tiles - 1) / tiles;
     const int max_splits = (total_stages + 7) / 8;  // at least 8 stages of work per CTA
     if (splits > max_splits) splits = max_splits;
@@ -883,7 +893,8 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     splits = (total_stages + per - 1) / per;
     p.stages_per_split = per;
     p.num_k_splits = splits;
-    const size_t stage_bytes = (size_t)p.subs_per_mtile * p.pixels_per_stage * p.kc + (size_t)p.tile_n * p.pixels_per_stage;
+    const size_t stage_bytes = (size_t)p.mtiles_per_cta * p.subs_per_mtile * p.pixels_per_stage * p.kc +
+                               (size_t)p.tile_n * p.pixels_per_stage;
     int stages = (int)((200 * 1024) / stage_bytes);
     p.num_stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
     p.src_stride = d.stride;

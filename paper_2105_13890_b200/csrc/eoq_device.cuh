@@ -104,6 +104,43 @@ __device__ __forceinline__ long long warp_sum_i64(long long v)
     return v;
 }
 
+// Block-wide reductions (every thread of the block must call; the result is valid in thread 0).  Thousands of
+// warps hitting one global cell with an atomic serialise at the L2, so each block sends one.
+__device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v)
+{
+    __shared__ unsigned long long red_max[32];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, v, o);
+        v = other > v ? other : v;
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
+    if (lane == 0) red_max[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        v = lane < nw ? red_max[lane] : 0ull;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, v, o);
+            v = other > v ? other : v;
+        }
+    }
+    __syncthreads();
+    return v;
+}
+
+__device__ __forceinline__ long long block_sum_i64(long long v)
+{
+    __shared__ long long red_sum[32];
+    v = warp_sum_i64(v);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = (blockDim.x + 31) >> 5;
+    if (lane == 0) red_sum[warp] = v;
+    __syncthreads();
+    if (warp == 0) v = warp_sum_i64(lane < nw ? red_sum[lane] : 0ll);
+    __syncthreads();
+    return v;
+}
+
 // ------------------------------------------------------------------ PTX: shared-memory barriers and TMA
 
 namespace ptx {

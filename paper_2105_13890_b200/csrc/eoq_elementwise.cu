@@ -58,9 +58,9 @@ __global__ void absmax_f32_kernel(const float *__restrict__ src, size_t n, Devic
         bad |= a >= 0x7f800000u;
         mx = max(mx, a);
     }
-    mx = warp_max_u32(mx);
-    bad = __any_sync(0xffffffffu, bad);
-    if ((threadIdx.x & 31) == 0) {
+    mx = (uint32_t)block_max_u64(mx);
+    bad = __syncthreads_or(bad);
+    if (threadIdx.x == 0) {
         if (mx) atomicMax(&dev->absmax_u32, mx);
         if (bad) atomicOr(&dev->status, EOQ_DEV_NONFINITE);
     }
@@ -187,8 +187,8 @@ __global__ void absmax_i32_kernel(const int32_t *__restrict__ src, size_t n, Dev
     }
     for (size_t i = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         mx = max(mx, (uint32_t)abs(src[i]));
-    mx = warp_max_u32(mx);
-    if ((threadIdx.x & 31) == 0 && mx) atomicMax(&dev->absmax_u32, mx);
+    mx = (uint32_t)block_max_u64(mx);
+    if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u32, mx);
 }
 
 __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *src_exp, int exp_bias, size_t n,
@@ -228,8 +228,8 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
         dst[i] = (int8_t)c;
     }
     if (sum_codes) {
-        sum = warp_sum_i64(sum);
-        if ((threadIdx.x & 31) == 0 && sum) atomicAdd(reinterpret_cast<unsigned long long *>(sum_codes), (unsigned long long)sum);
+        sum = block_sum_i64(sum);
+        if (threadIdx.x == 0 && sum) atomicAdd(reinterpret_cast<unsigned long long *>(sum_codes), (unsigned long long)sum);
     }
 }
 
@@ -284,12 +284,8 @@ __global__ void wgrad_fix_absmax_kernel(long long *acc, size_t n, const long lon
         const unsigned long long a = (unsigned long long)(v < 0 ? -v : v);
         mx = a > mx ? a : mx;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        unsigned long long other = __shfl_xor_sync(0xffffffffu, mx, o);
-        mx = other > mx ? other : mx;
-    }
-    if ((threadIdx.x & 31) == 0 && mx) atomicMax(&dev->absmax_u64, mx);
+    mx = block_max_u64(mx);
+    if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u64, mx);
     (void)taps;
 }
 
@@ -317,38 +313,61 @@ __device__ __forceinline__ void unpack16(const int4 &v, int (&o)[16])
 }
 
 // Pass 1: max |e1| and the sums behind g_b2 and g_gamma, with e1 = e0 * [x4 > 0].
+// Expands 4 mask bits into 4 byte masks (0x00 / 0xff).
+__device__ __forceinline__ uint32_t bits_to_bytes(uint32_t nibble)
+{
+    return (((nibble & 0xfu) * 0x00204081u) & 0x01010101u) * 0xffu;
+}
+
 __global__ void prescale_reduce_kernel(const int8_t *__restrict__ e0, const uint8_t *__restrict__ mask,
                                        const int16_t *__restrict__ x2, size_t n16, DeviceState *dev)
 {
-    uint32_t mx = 0;
+    uint32_t mx4 = 0;  // four running byte maxima of |e1|
     long long s1 = 0, s2 = 0;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
-        int e[16];
-        unpack16(__ldg(reinterpret_cast<const int4 *>(e0) + i), e);
-        const uint32_t m = mask ? (uint32_t) __ldg(reinterpret_cast<const uint16_t *>(mask) + i) : 0xffffu;
-        int a1 = 0, a2 = 0;
-        int xv[16];
-        if (x2) {
-            const int4 lo = __ldg(reinterpret_cast<const int4 *>(x2) + 2 * i);
-            const int4 hi = __ldg(reinterpret_cast<const int4 *>(x2) + 2 * i + 1);
-            const int16_t *pl = reinterpret_cast<const int16_t *>(&lo), *ph = reinterpret_cast<const int16_t *>(&hi);
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    // four independent 16-element groups per iteration keep enough loads in flight to cover DRAM latency
+    for (size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < n16; i0 += 4 * stride) {
+        int4 ev[4];
+        uint32_t mv[4];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) { xv[k] = pl[k]; xv[8 + k] = ph[k]; }
+        for (int u = 0; u < 4; ++u) {
+            const size_t i = i0 + u * stride;
+            const bool in = i < n16;
+            ev[u] = in ? __ldg(reinterpret_cast<const int4 *>(e0) + i) : make_int4(0, 0, 0, 0);
+            mv[u] = (in && mask) ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(mask) + i) : 0xffffu;
         }
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-            const int e1 = ((m >> k) & 1u) ? e[k] : 0;
-            mx = max(mx, (uint32_t)abs(e1));
-            a1 += e1;
-            if (x2) a2 += e1 * xv[k];  // |e1 * x2| < 2^22, 16 terms
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t w[4] = {(uint32_t)ev[u].x, (uint32_t)ev[u].y, (uint32_t)ev[u].z, (uint32_t)ev[u].w};
+            int a1 = 0;
+            uint32_t e1w[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                e1w[q] = w[q] & bits_to_bytes(mv[u] >> (4 * q));  // e1 = e0 * [x4 > 0], four codes per word
+                mx4 = __vmaxu4(mx4, __vabsss4(e1w[q]));
+                a1 = __dp4a((int)e1w[q], 0x01010101, a1);
+            }
+            s1 += a1;
+            if (x2) {
+                const size_t i = i0 + u * stride;
+                if (i < n16) {
+                    const int4 lo = __ldg(reinterpret_cast<const int4 *>(x2) + 2 * i);
+                    const int4 hi = __ldg(reinterpret_cast<const int4 *>(x2) + 2 * i + 1);
+                    const int16_t *pl = reinterpret_cast<const int16_t *>(&lo), *ph = reinterpret_cast<const int16_t *>(&hi);
+                    const int8_t *eb = reinterpret_cast<const int8_t *>(e1w);
+                    int a2 = 0;  // |e1 * x2| < 2^22, 16 terms
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) a2 += (int)eb[k] * pl[k] + (int)eb[8 + k] * ph[k];
+                    s2 += a2;
+                }
+            }
         }
-        s1 += a1;
-        s2 += a2;
     }
-    mx = warp_max_u32(mx);
-    s1 = warp_sum_i64(s1);
-    s2 = warp_sum_i64(s2);
-    if ((threadIdx.x & 31) == 0) {
+    uint32_t mx = max(max(mx4 & 0xffu, (mx4 >> 8) & 0xffu), max((mx4 >> 16) & 0xffu, mx4 >> 24));
+    mx = (uint32_t)block_max_u64(mx);
+    s1 = block_sum_i64(s1);
+    s2 = block_sum_i64(s2);
+    if (threadIdx.x == 0) {
         if (mx) atomicMax(&dev->absmax_u32, mx);
         if (s1) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum0), (unsigned long long)s1);
         if (s2) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum1), (unsigned long long)s2);
@@ -369,15 +388,29 @@ __global__ void prescale_apply_kernel(const int8_t *__restrict__ e0, const int32
         if (sum_e1) *sum_e1 = dev->sum0;
         if (sum_e1x2) *sum_e1x2 = dev->sum1;
     }
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
-        int e[16], c[16];
-        unpack16(__ldg(reinterpret_cast<const int4 *>(e0) + i), e);
-        const uint32_t m = mask ? (uint32_t) __ldg(reinterpret_cast<const uint16_t *>(mask) + i) : 0xffffu;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < n16; i0 += 4 * stride) {
+        int4 ev[4];
+        uint32_t mv[4];
 #pragma unroll
-        for (int k = 0; k < 16; ++k) c[k] = ((m >> k) & 1u) ? sq_code32(gamma_c * e[k], t) : 0;
-        reinterpret_cast<int4 *>(e3)[i] =
-            make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
-                      (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+        for (int u = 0; u < 4; ++u) {
+            const size_t i = i0 + u * stride;
+            const bool in = i < n16;
+            ev[u] = in ? __ldg(reinterpret_cast<const int4 *>(e0) + i) : make_int4(0, 0, 0, 0);
+            mv[u] = (in && mask) ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(mask) + i) : 0xffffu;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const size_t i = i0 + u * stride;
+            if (i >= n16) continue;
+            int e[16], c[16];
+            unpack16(ev[u], e);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) c[k] = ((mv[u] >> k) & 1u) ? sq_code32(gamma_c * e[k], t) : 0;
+            reinterpret_cast<int4 *>(e3)[i] =
+                make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
+                          (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+        }
     }
 }
 
@@ -423,8 +456,8 @@ __global__ void update_absmax_kernel(const __grid_constant__ UpdateBatch b, Devi
         const size_t tail = vec ? begin + ((end - begin) / 16) * 16 : begin;
         for (size_t j = tail + threadIdx.x; j < end; j += blockDim.x) mx = max(mx, (uint32_t)abs((int)T.g[j]));
     }
-    mx = warp_max_u32(mx);
-    if ((threadIdx.x & 31) == 0 && mx) atomicMax(&dev->tensor_absmax[b.tensor_base + k], mx);
+    mx = (uint32_t)block_max_u64(mx);
+    if (threadIdx.x == 0 && mx) atomicMax(&dev->tensor_absmax[b.tensor_base + k], mx);
 }
 
 // SplitMix64 output function (Steele, Lea, Flood 2014) as a counter hash.

@@ -161,14 +161,14 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         }
     } else {
         // ---------------------------------------------------------------------- epilogue
-        // Eight warps, two per scheduler: a warp may read the TMEM lanes of quadrant (warp % 4); the two warps
+        // Four warps per scheduler: a warp may read the TMEM lanes of quadrant (warp % 4); the warps
         // of a quadrant split the tile's columns.
         const int quad = warp & 3;
-        const int half = (warp - 2) >> 2;
+        const int part = (warp - 2) >> 2;  // the kEpilogueWarps / 4 warps of a lane quadrant split the columns
         const int row = quad * 32 + lane;
         const int groups = p.tile_n / 16;                 // 16-column groups of the tile
-        const int g_begin = half ? (groups + 1) / 2 : 0;  // the first half takes the odd group
-        const int g_end = half ? groups : (groups + 1) / 2;
+        constexpr int kParts = kEpilogueWarps / 4;
+        const int g_begin = (groups * part) / kParts, g_end = (groups * (part + 1)) / kParts;
         int shift = 7;
         if (p.epilogue == kEpiForward && p.x_exp) {
             shift = -__ldg(p.x_exp);

@@ -226,11 +226,11 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
     } else if (warp >= 4) {
         // ---------------------------------------------------------------------- epilogue
         const int quad = warp & 3;
-        const int half = (warp - 4) >> 2;
+        const int part = (warp - 4) >> 2;  // the kEpilogueWarps / 4 warps of a lane quadrant split the columns
         const int row = quad * 32 + lane;
         const int groups = p.tile_n / 16;
-        const int g_begin = half ? (groups + 1) / 2 : 0;
-        const int g_end = half ? groups : (groups + 1) / 2;
+        constexpr int kParts = kEpilogueWarps / 4;
+        const int g_begin = (groups * part) / kParts, g_end = (groups * (part + 1)) / kParts;
         const int yl = row / pl.pw, xx = row % pl.pw;  // position of this thread's row in the patch raster
         int acc = 0;
         uint32_t acc_phase = 0, mx = 0;

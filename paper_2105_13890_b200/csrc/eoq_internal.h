@@ -10,7 +10,7 @@ namespace eoq {
 
 constexpr int kMaxTaps = 64;        // kh * kw of any supported filter
 constexpr int kTileM = 128;         // GEMM rows per CTA tile (TMEM lanes)
-constexpr int kEpilogueWarps = 8;   // implicit GEMM: two epilogue warps per scheduler
+constexpr int kEpilogueWarps = 16;  // implicit GEMM: four epilogue warps per scheduler hide the latency of the integer chain
 constexpr int kGemmThreads = 64 + 32 * kEpilogueWarps;  // warp 0: TMA, warp 1: MMA + TMEM owner, then the epilogue
 constexpr int kWgradThreads = 192;  // weight gradient: warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 constexpr uint32_t kSpinLimit = 1u << 22;  // polls before a wait gives up (normal waits end within microseconds)
@@ -105,7 +105,7 @@ struct PatchPlan {
     int num_a, num_b;   // ring depths (patches, weight sub-tiles)
     int b_resident;     // all weight sub-tiles of the layer stay in shared memory
 };
-constexpr int kPatchThreads = 384;  // warps: 0 patch loads, 1 MMA + TMEM, 2 weight loads, 3 idle, 4..11 epilogue
+constexpr int kPatchThreads = 128 + 32 * kEpilogueWarps;  // warps: 0 patch loads, 1 MMA + TMEM, 2 weight loads, 3 idle, then the epilogue
 
 size_t igemm_patch_smem_bytes(const IgemmParams &p, const PatchPlan &pl);
 cudaError_t launch_igemm_patch(const IgemmParams &p, const PatchPlan &pl, const CUtensorMap &map_a,
@@ -130,6 +130,8 @@ struct WgradParams {
     int subs_per_mtile;  // 128 / kc
     int tile_n;          // c_out columns per CTA (multiple of 16, <= 256)
     int num_m_tiles, num_n_tiles, num_k_splits;
+    int mtiles_per_cta;  // M tiles one CTA accumulates side by side in TMEM (they share the error tile of a stage)
+    int num_m_groups;    // ceil(num_m_tiles / mtiles_per_cta)
     int pixels_per_stage;   // 64
     int stages_per_split;   // pipeline iterations each CTA runs
     int num_stages;

@@ -53,14 +53,15 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
     const int px = p.pixels_per_stage;
     const uint32_t a_sub = (uint32_t)px * p.kc, b_sub = (uint32_t)px * p.nc;
     const int b_subs = p.tile_n / p.nc;
-    const uint32_t stage_bytes = (uint32_t)p.subs_per_mtile * a_sub + (uint32_t)b_subs * b_sub;
+    const uint32_t a_mtile = (uint32_t)p.subs_per_mtile * a_sub;  // bytes of one M tile's activation sub-tiles
+    const uint32_t stage_bytes = (uint32_t)p.mtiles_per_cta * a_mtile + (uint32_t)b_subs * b_sub;
     const uint32_t bar0 = ptx::smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
     const uint32_t done_bar = bar0 + 8u * (2 * kMaxStages);
 
     uint32_t tmem_cols = 32;
-    while (tmem_cols < (uint32_t)p.tile_n) tmem_cols <<= 1;
+    while (tmem_cols < (uint32_t)(p.mtiles_per_cta * p.tile_n)) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.num_stages; ++s) {
@@ -84,12 +85,13 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
     const RoleCtx ctx{&abort_s, p.dev};
 
     // work unit of this CTA
-    const int tiles = p.num_m_tiles * p.num_n_tiles;
+    const int tiles = p.num_m_groups * p.num_n_tiles;
     const int ks = blockIdx.x / tiles, tile = blockIdx.x % tiles;
-    const int mt = tile / p.num_n_tiles, nt = tile % p.num_n_tiles;
-    const int first_sub = mt * p.subs_per_mtile;
+    const int mt0 = (tile / p.num_n_tiles) * p.mtiles_per_cta, nt = tile % p.num_n_tiles;
+    const int my_mtiles = min(p.mtiles_per_cta, p.num_m_tiles - mt0);  // M tiles this CTA accumulates
     const int total_subs = p.ntaps * p.chunks_per_tap;
-    const int subs = min(p.subs_per_mtile, total_subs - first_sub);  // sub-tiles of this M tile that exist
+    int subs_total = 0;  // activation sub-tiles this CTA loads per stage
+    for (int jm = 0; jm < my_mtiles; ++jm) subs_total += min(p.subs_per_mtile, total_subs - (mt0 + jm) * p.subs_per_mtile);
     const int q_begin = ks * p.stages_per_split * px;
     int my_stages = p.stages_per_split;
     {
@@ -111,13 +113,17 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
                 const int cw = (rem % p.wo) * p.src_stride_w + p.base_w;
                 const int ch = (rem / p.wo) * p.src_stride + p.base_h;
                 const uint32_t a_dst = smem_base + stage * stage_bytes;
-                const uint32_t b_dst = a_dst + p.subs_per_mtile * a_sub;
-                ptx::mbar_expect_tx(full_bar(stage), subs * a_sub + b_subs * b_sub);
-                for (int j = 0; j < subs; ++j) {
-                    const int s = first_sub + j;
-                    const int tap = s / p.chunks_per_tap, chunk = s % p.chunks_per_tap;
-                    ptx::tma_load_im2col_4d(a_dst + j * a_sub, &map_x, full_bar(stage), chunk * p.kc, cw, ch, img,
-                                            (uint16_t)p.tap_dw[tap], (uint16_t)p.tap_dh[tap]);
+                const uint32_t b_dst = a_dst + p.mtiles_per_cta * a_mtile;
+                ptx::mbar_expect_tx(full_bar(stage), subs_total * a_sub + b_subs * b_sub);
+                for (int jm = 0; jm < my_mtiles; ++jm) {
+                    const int first_sub = (mt0 + jm) * p.subs_per_mtile;
+                    const int subs = min(p.subs_per_mtile, total_subs - first_sub);  // sub-tiles of this M tile that exist
+                    for (int j = 0; j < subs; ++j) {
+                        const int s = first_sub + j;
+                        const int tap = s / p.chunks_per_tap, chunk = s % p.chunks_per_tap;
+                        ptx::tma_load_im2col_4d(a_dst + jm * a_mtile + j * a_sub, &map_x, full_bar(stage), chunk * p.kc, cw, ch,
+                                                img, (uint16_t)p.tap_dw[tap], (uint16_t)p.tap_dh[tap]);
+                    }
                 }
                 for (int j = 0; j < b_subs; ++j)
                     ptx::tma_load_2d(b_dst + j * b_sub, &map_e, full_bar(stage), nt * p.tile_n + j * p.nc, q0);
@@ -140,6 +146,7 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
             const uint32_t a_hi = (uint32_t)(a_proto >> 32), b_hi = (uint32_t)(b_proto >> 32);
             const uint32_t a_lead = (uint32_t)a_proto, b_lead = (uint32_t)b_proto;  // leading-offset field, address 0
             const uint32_t a_step16 = (32u * p.kc) >> 4, b_step16 = (32u * p.nc) >> 4;  // 32 pixels further down
+            const uint32_t a_mtile16 = a_mtile >> 4;
             int stage = 0;
             uint32_t phase = 0, accumulate = 0;
             bool ok = true;
@@ -147,9 +154,12 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
                 if (!(ok = wait_bar(full_bar(stage), phase, ctx))) break;
                 ptx::tc_fence_after();
                 uint32_t a_lo = ((smem_base + stage * stage_bytes) >> 4) | a_lead;
-                uint32_t b_lo = (((smem_base + stage * stage_bytes) >> 4) + ((p.subs_per_mtile * a_sub) >> 4)) | b_lead;
+                uint32_t b_lo = (((smem_base + stage * stage_bytes) >> 4) + ((p.mtiles_per_cta * a_mtile) >> 4)) | b_lead;
                 for (int k = 0; k < px; k += 32) {
-                    ptx::mma_i8(tmem_base, smem_desc_join(a_lo, a_hi), smem_desc_join(b_lo, b_hi), idesc, accumulate);
+                    // the M tiles of the group meet the same error tile; each has its own accumulator columns
+                    uint32_t a_j = a_lo, d_j = tmem_base;
+                    for (int jm = 0; jm < my_mtiles; ++jm, a_j += a_mtile16, d_j += p.tile_n)
+                        ptx::mma_i8(d_j, smem_desc_join(a_j, a_hi), smem_desc_join(b_lo, b_hi), idesc, accumulate);
                     accumulate = 1;
                     a_lo += a_step16;
                     b_lo += b_step16;
@@ -164,18 +174,19 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
         }
     } else {
         const int quad = warp & 3;
-        int row = mt * kTileM + quad * 32 + lane;  // (tap, ic) flattened: tap * c_in + ic
-        bool valid = row < p.rows_total;
-        if (p.row_window_kw) {
-            // the tile's rows are (tap 0..7, channel 0..15) of filter row mt: drop the padding taps
-            const int t = (quad * 32 + lane) >> 4;
-            valid = t < p.row_window_kw;
-            row = (mt * p.row_window_kw + t) * 16 + (lane & 15);
-        }
         bool ok = __all_sync(0xffffffffu, wait_bar(done_bar, 0, ctx));
-        if (ok && my_stages > 0) {
-            ptx::tc_fence_after();
-            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
+        if (ok && my_stages > 0) ptx::tc_fence_after();
+        for (int jm = 0; jm < my_mtiles && ok && my_stages > 0; ++jm) {
+            const int mt = mt0 + jm;
+            int row = mt * kTileM + quad * 32 + lane;  // (tap, ic) flattened: tap * c_in + ic
+            bool valid = row < p.rows_total;
+            if (p.row_window_kw) {
+                // the tile's rows are (tap 0..7, channel 0..15) of filter row mt: drop the padding taps
+                const int t = (quad * 32 + lane) >> 4;
+                valid = t < p.row_window_kw;
+                row = (mt * p.row_window_kw + t) * 16 + (lane & 15);
+            }
+            const uint32_t t_row = tmem_base + jm * p.tile_n + ((uint32_t)(quad * 32) << 16);
             for (int c0 = 0; c0 < p.tile_n; c0 += 32) {
                 uint32_t r[32];
                 const int ncol = min(32, p.tile_n - c0);
@@ -209,7 +220,8 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
 
 size_t wgrad_smem_bytes(const WgradParams &p)
 {
-    const size_t stage = (size_t)p.subs_per_mtile * p.pixels_per_stage * p.kc + (size_t)p.tile_n * p.pixels_per_stage;
+    const size_t stage = (size_t)p.mtiles_per_cta * p.subs_per_mtile * p.pixels_per_stage * p.kc +
+                         (size_t)p.tile_n * p.pixels_per_stage;
     return stage * p.num_stages + 1024;
 }
 
@@ -217,7 +229,7 @@ cudaError_t launch_wgrad(const WgradParams &p, const CUtensorMap &map_x, const C
 {
     cudaError_t e = cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024);
     if (e != cudaSuccess) return e;
-    const int grid = p.num_m_tiles * p.num_n_tiles * p.num_k_splits;
+    const int grid = p.num_m_groups * p.num_n_tiles * p.num_k_splits;
     wgrad_kernel<<<grid, kWgradThreads, wgrad_smem_bytes(p), stream>>>(p, map_x, map_e);
     return cudaGetLastError();
 }
