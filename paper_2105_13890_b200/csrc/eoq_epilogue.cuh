@@ -36,8 +36,32 @@ __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d)
 // into bit 7 exactly when the remainder exceeds one half, or equals it with an odd quotient.
 __device__ __forceinline__ int32_t rne7(int32_t a) { return (a + 63 + ((a >> 7) & 1)) >> 7; }
 
+// The same rounding on the floating-point pipe, which the integer-heavy epilogue leaves idle.  For an integer t
+// with kMagicBits + t inside [2^23, 2^24) the word kMagicBits + t read as a float is 1.5 * 2^23 + t exactly;
+// one fused multiply-add forms 1.5 * 2^23 + t / 2^7, whose single rounding (nearest, ties to even, unit spacing
+// in that binade) is R(t / 2^7).  Returns kMagicBits + R(t / 2^7): the low 16 bits are the two's-complement code.
+constexpr uint32_t kMagicBits = 0x4B400000u;                     // 1.5 * 2^23 as a float
+constexpr float kMagicRest = 12582912.0f - 12582912.0f / 128.0f;  // exact: 12484608
+__device__ __forceinline__ uint32_t rne7_magic(uint32_t biased)
+{
+    return __float_as_uint(__fmaf_rn(__uint_as_float(biased), 0.0078125f, kMagicRest));
+}
+
+// byte k of w, sign-extended
+template <int k>
+__device__ __forceinline__ int32_t sbyte(uint32_t w)
+{
+    // prmt selector digit 8 + k replicates the sign bit of byte k (the __byte_perm intrinsic drops that bit)
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(r) : "r"(w), "n"(((8 + k) << 12) | ((8 + k) << 8) | ((8 + k) << 4) | k));
+    return (int32_t)r;
+}
+
 // Forward chain on 16 consecutive output channels of one pixel (Sec. 3.2.1: x2 = Q_a1(conv), x3 = gamma x2,
 // x4 = x3 + b2 [+ shortcut], x5 = Q_a2(relu(x4)); mask = [x4 > 0]).  kShift7: the input sits at exponent -7.
+// The integer pipe bounds this code, so clamps are moved in front of the roundings (both are monotonic, the
+// clamp limits are chosen so that the rounded result is unchanged), roundings run as one FMA each, and the
+// constant offsets of that trick are folded into the multiply-add that forms x4.
 template <bool kShift7>
 __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t *acc, size_t off, int col, int cls,
                                            int shift)
@@ -61,53 +85,76 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t 
 #pragma unroll
         for (int i = 0; i < 4; ++i) d[i] = make_int4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
     }
-    int32_t add[16];  // (b2 + shortcut) * 2^7, the part of x4 that does not depend on the accumulator
-    const int32_t b2s = p.b2_c << 7;
+    // q = x2 code + q_bias, the code saturated to 16 bits
+    uint32_t q[16];
+    uint32_t q_bias;
+    if (kShift7) {
+        // R(a / 2^7) lies in [-32768, 32767] exactly when a lies in [-32768 * 128 - 64, 32767 * 128 + 63], and
+        // clamping a to [-32768 * 128, 32767 * 128 + 63] first gives the same code.  |a| < 2^31 - 2^24 (checked
+        // on the host), so neither addition below wraps.
+        q_bias = kMagicBits;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t up = (uint32_t)__viaddmax_s32(a[i], 4194304, 0);  // max(a, -2^22) + 2^22
+            q[i] = rne7_magic(__viaddmin_u32(up, kMagicBits - 4194304u, kMagicBits + 4194239u));
+        }
+    } else {
+        q_bias = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            int32_t v2;
+            if (shift >= 0) {
+                v2 = rne_shr32(a[i], shift);
+            } else {
+                const long long w = (long long)a[i] << (-shift);
+                v2 = (int32_t)(w < -32768 ? -32768 : (w > 32767 ? 32767 : w));
+            }
+            q[i] = (uint32_t)clampi(v2, -32768, 32767);
+        }
+    }
+    // x4 = gamma * x2 + (b2 + shortcut) * 2^7 = gamma * q + add, the bias of q folded into add (mod 2^32)
+    const uint32_t g = (uint32_t)p.gamma_c;
+    const uint32_t base = ((uint32_t)p.b2_c << 7) - g * q_bias;
+    uint32_t add[16];
     if (p.shortcut) {
         const int4 v = __ldg(reinterpret_cast<const int4 *>(p.shortcut + off));
-        const int8_t *b = reinterpret_cast<const int8_t *>(&v);
+        const uint32_t w[4] = {(uint32_t)v.x, (uint32_t)v.y, (uint32_t)v.z, (uint32_t)v.w};
 #pragma unroll
-        for (int i = 0; i < 16; ++i) add[i] = b2s + ((int32_t)b[i] << 7);
+        for (int i = 0; i < 4; ++i) {
+            add[4 * i + 0] = base + (uint32_t)sbyte<0>(w[i]) * 128u;
+            add[4 * i + 1] = base + (uint32_t)sbyte<1>(w[i]) * 128u;
+            add[4 * i + 2] = base + (uint32_t)sbyte<2>(w[i]) * 128u;
+            add[4 * i + 3] = base + (uint32_t)sbyte<3>(w[i]) * 128u;
+        }
     } else {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) add[i] = b2s;
+        for (int i = 0; i < 16; ++i) add[i] = base;
     }
+    // Q_a2: R(x4 / 2^7) saturated to +-127 (and to 0 from below after a ReLU).  16319 / 128 = 127.49.. rounds to
+    // 127 and everything above saturates to 127 too, so x4 is clamped to +-16319 before the rounding.
     uint32_t mbits = 0;
-    const int32_t lo = p.relu ? 0 : -127 * 128 - 64;  // below this Q_a2 saturates at -127 anyway
+    uint32_t r[16];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        int32_t v2;
-        if (kShift7) {
-            v2 = rne7(a[i]);
-        } else if (shift >= 0) {
-            v2 = rne_shr32(a[i], shift);
-        } else {
-            const long long w = (long long)a[i] << (-shift);
-            v2 = (int32_t)(w < -32768 ? -32768 : (w > 32767 ? 32767 : w));
-        }
-        v2 = clampi(v2, -32768, 32767);
-        a[i] = v2;
-        const int32_t v4 = p.gamma_c * v2 + add[i];
-        mbits |= (v4 > 0 ? 1u : 0u) << i;
-        add[i] = min(rne7(max(v4, lo)), 127);
-    }
-    if (!p.relu) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) add[i] = max(add[i], -127);
+    for (int i = 15; i >= 0; --i) {
+        const int32_t v4 = (int32_t)(g * q[i] + add[i]);
+        const int32_t n4 = (int32_t)((0u - g) * q[i] - add[i]);   // -x4: its sign bit is [x4 > 0]
+        mbits = __funnelshift_l((uint32_t)n4, mbits, 1);
+        if (p.relu) r[i] = rne7_magic((uint32_t)__vimin_s32_relu(v4, 16319) | kMagicBits);
+        else r[i] = rne7_magic((uint32_t)clampi(v4, -16319, 16319) + kMagicBits);
     }
     int4 o;
-    o.x = (int)pack4(add[0], add[1], add[2], add[3]);
-    o.y = (int)pack4(add[4], add[5], add[6], add[7]);
-    o.z = (int)pack4(add[8], add[9], add[10], add[11]);
-    o.w = (int)pack4(add[12], add[13], add[14], add[15]);
+    o.x = (int)__byte_perm(__byte_perm(r[0], r[1], 0x0040), __byte_perm(r[2], r[3], 0x0040), 0x5410);
+    o.y = (int)__byte_perm(__byte_perm(r[4], r[5], 0x0040), __byte_perm(r[6], r[7], 0x0040), 0x5410);
+    o.z = (int)__byte_perm(__byte_perm(r[8], r[9], 0x0040), __byte_perm(r[10], r[11], 0x0040), 0x5410);
+    o.w = (int)__byte_perm(__byte_perm(r[12], r[13], 0x0040), __byte_perm(r[14], r[15], 0x0040), 0x5410);
     *reinterpret_cast<int4 *>(p.x5 + off) = o;
     if (p.relu_mask) *reinterpret_cast<uint16_t *>(p.relu_mask + (off >> 3)) = (uint16_t)mbits;
     if (p.x2) {
         int4 *d = reinterpret_cast<int4 *>(p.x2 + off);
-        d[0] = make_int4((a[0] & 0xffff) | (a[1] << 16), (a[2] & 0xffff) | (a[3] << 16), (a[4] & 0xffff) | (a[5] << 16),
-                         (a[6] & 0xffff) | (a[7] << 16));
-        d[1] = make_int4((a[8] & 0xffff) | (a[9] << 16), (a[10] & 0xffff) | (a[11] << 16),
-                         (a[12] & 0xffff) | (a[13] << 16), (a[14] & 0xffff) | (a[15] << 16));
+        d[0] = make_int4((int)__byte_perm(q[0], q[1], 0x5410), (int)__byte_perm(q[2], q[3], 0x5410),
+                         (int)__byte_perm(q[4], q[5], 0x5410), (int)__byte_perm(q[6], q[7], 0x5410));
+        d[1] = make_int4((int)__byte_perm(q[8], q[9], 0x5410), (int)__byte_perm(q[10], q[11], 0x5410),
+                         (int)__byte_perm(q[12], q[13], 0x5410), (int)__byte_perm(q[14], q[15], 0x5410));
     }
 }
 

@@ -154,8 +154,19 @@ def single_layer() -> Workload:
     return Workload("single_conv3x3_n8_c16_32x32", 8, [Layer("conv", 8, 32, 32, 16, 16, 3, 1, 1, 16, in_branch=False)], L=1, m=2)
 
 
+def layer64(batch: int = 512) -> Workload:
+    """Two 3x3 stride-1 layers of the ResNet-18 first stage (64 -> 64 channels, 56x56): the profiling case.
+
+    At batch 512 each activation tensor is 103 MB, so a layer's tensors do not fit in a B200's L2.  The first
+    layer takes the quantized image (device-side input exponent), the second is an ordinary inner layer.
+    """
+    layers = [Layer("conv.a", batch, 56, 56, 64, 64, 3, 1, 1, 64, in_branch=False, has_dgrad=False),
+              Layer("conv.b", batch, 56, 56, 64, 64, 3, 1, 1, 64, in_branch=False)]
+    return Workload(f"conv3x3_c64_56x56_b{batch}_x2", batch, layers, L=1, m=2)
+
+
 def get(name: str, batch: int | None = None) -> Workload:
-    table = {"single": single_layer, "resnet20": resnet20, "resnet18": resnet18, "resnet50": resnet50}
+    table = {"single": single_layer, "layer64": layer64, "resnet20": resnet20, "resnet18": resnet18, "resnet50": resnet50}
     fn = table[name]
     if name == "single" or batch is None:
         return fn()

@@ -60,6 +60,49 @@ def test_conv_fwd(d, scal):
     assert np.array_equal(G.unpack_mask(mask, shape), ref["mask"])
 
 
+EXTREME_CASES = [
+    (ConvDesc(2, 6, 6, 512, 32, 3, 3, 1, 1), (-127, 127, 64, -64, 0, 1), (-127, 127, 1, 2, 0, -1)),   # x2 saturates both ways
+    (ConvDesc(2, 9, 9, 16, 32, 1, 1, 1, 0), (0, 64, -64, 127), (0, 64, -64, 1)),                        # ties of both roundings
+    (ConvDesc(2, 9, 9, 16, 32, 3, 3, 1, 1), (0, 64, -64), (0, 64, -64, 32)),
+    (ConvDesc(1, 8, 8, 64, 64, 3, 3, 2, 1), (0, 64, -64, 1, -1), (0, 64, -64, 127, -127)),
+]
+
+
+@pytest.mark.parametrize("case", EXTREME_CASES, ids=["saturate", "ties_1x1", "ties_3x3", "ties_s2"])
+@pytest.mark.parametrize("scal", [(0, 1, 0, False, True), (0, 1, 0, True, False), (5, 32767, -300, True, True),
+                                  (-5, -32768, 300, True, False), (0, 127, 1, False, False), (0, -1, 0, False, True)],
+                         ids=["g1", "g1_sc_norelu", "gmax", "gmin_norelu", "g127_norelu", "gneg1"])
+def test_conv_fwd_ties_and_saturation(case, scal):
+    """Operands drawn from a few extreme values: accumulators sit on rounding ties and beyond the 16-bit range
+    of x2, and x4 reaches both ends of its range, so every clamp and tie of the forward chain is exercised."""
+    d, xvals, wvals = case
+    b1, gamma, b2, use_sc, relu = scal
+    rng = np.random.Generator(np.random.Philox(key=[d.c_in, d.kh]))
+    x0 = rng.choice(np.array(xvals, dtype=np.int8), size=(d.n, d.h, d.w, d.c_in))
+    w = rng.choice(np.array(wvals, dtype=np.int8), size=(d.c_out, d.kh, d.kw, d.c_in))
+    if case is EXTREME_CASES[0]:  # coherent signs: half of the output channels sum far up, a quarter far down
+        x0 = np.abs(x0)
+        w[0::2] = np.abs(w[0::2])
+        w[1::4] = -np.abs(w[1::4])
+    sc = rng.choice(np.array([-127, -1, 0, 1, 127], dtype=np.int8), size=(d.n, d.ho, d.wo, d.c_out))
+    ref = oracle.layer_forward(d, x0, b1, w, gamma, b2, sc if use_sc else None, relu)
+    gd = G.gdesc(d)
+    shape = ref["x5"].shape
+    x5, x2, acc = G.zeros(shape, torch.int8), G.zeros(shape, torch.int16), G.zeros(shape, torch.int32)
+    mask = G.zeros((ref["x5"].size + 7) // 8, torch.uint8)
+    eoq.eoq_conv_fwd(G.handle(), gd, G.dev(x0), None, b1, G.dev(w), gamma, b2, G.dev(sc) if use_sc else None, relu,
+                     x5, x2, mask, acc, G.workspace(gd, eoq.EOQ_PASS_FWD))
+    assert G.status_clear() == 0
+    assert np.array_equal(G.host(acc).astype(np.int64), ref["acc"])
+    assert np.array_equal(G.host(x2).astype(np.int32), ref["x2"])
+    assert np.array_equal(G.host(x5), ref["x5"])
+    assert np.array_equal(G.unpack_mask(mask, shape), ref["mask"])
+    if case is EXTREME_CASES[0]:
+        assert ref["x2"].max() == 32767 and ref["x2"].min() == -32768
+    if case is EXTREME_CASES[1] and b1 == 0:
+        assert np.any(np.abs(ref["acc"]) % 128 == 64)
+
+
 MARGIN_CASES = [
     (ConvDesc(2, 20, 20, 16, 64, 7, 7, 2, 3), 4),     # filter-row path of the 7x7 stride-2 first layer
     (ConvDesc(3, 17, 23, 16, 32, 7, 7, 2, 3), 5),     # odd extents, wider margin
