@@ -206,7 +206,7 @@ def run_gpu(args):
     sampler = ClockSampler(local) if rank == 0 else None
     time.sleep(0.3)
     # ---- timed region: K steps, inputs resident
-    l0 = eoq.eoq_launch_count(handle) + eoq.eoq_launch_count(step.h_side)
+    l0 = step.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t_wall0 = time.time()
@@ -217,7 +217,7 @@ def run_gpu(args):
     barrier()
     t_wall1 = time.time()
     ms = ev0.elapsed_time(ev1)
-    launches = eoq.eoq_launch_count(handle) + eoq.eoq_launch_count(step.h_side) - l0
+    launches = step.launch_count() - l0
     if not args.eager:
         launches = step.launches_per_step * args.steps  # graph replays do not pass through the host-side counter
     status |= step.status()

@@ -64,7 +64,8 @@ class TrainStep:
     """Allocates device buffers for a workload, fills them with seeded synthetic data, and runs steps."""
 
     def __init__(self, workload: Workload, handle: int, device: str = "cuda:0", seed: int = synth.BASE_SEED,
-                 scalars: Optional[Scalars] = None, lr_mant: int = 1, lr_exp: int = -6, image_channels: int = 3):
+                 scalars: Optional[Scalars] = None, lr_mant: int = 1, lr_exp: int = -6, image_channels: int = 3,
+                 side_streams: int = 1):
         self.wl, self.h, self.dev = workload, handle, torch.device(device)
         self.sc = scalars or Scalars()
         self.lr_mant, self.lr_exp = lr_mant, lr_exp
@@ -79,11 +80,13 @@ class TrainStep:
             for p in (eoq.EOQ_PASS_FWD, eoq.EOQ_PASS_DGRAD, eoq.EOQ_PASS_WGRAD):
                 ws = max(ws, eoq.eoq_workspace_size(lb.desc, p))
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=self.dev)
-        # second handle + workspace: the weight-gradient chain of a layer can then run on a side stream next to
-        # the layer's dgrad chain (a handle's reduction cells and a workspace serve one call at a time)
-        self.h_side = eoq.eoq_create(self.dev.index if self.dev.index is not None else 0)
-        self.workspace_side = torch.empty(ws, dtype=torch.uint8, device=self.dev)
-        self.side = torch.cuda.Stream(device=self.dev)
+        # further handles + workspaces: the weight-gradient chain of a layer can then run on a side stream next
+        # to the layer's dgrad chain (a handle's reduction cells and a workspace serve one call at a time); the
+        # chains of different layers are independent of each other, so they rotate over the side streams
+        dev_index = self.dev.index if self.dev.index is not None else 0
+        self.h_sides = [eoq.eoq_create(dev_index) for _ in range(side_streams)]
+        self.workspace_sides = [torch.empty(ws, dtype=torch.uint8, device=self.dev) for _ in range(side_streams)]
+        self.sides = [torch.cuda.Stream(device=self.dev) for _ in range(side_streams)]
         self.graph = None
         first = workload.layers[0]
         self.image_channels = image_channels
@@ -142,16 +145,18 @@ class TrainStep:
             eoq.eoq_err_prescale(h, lb.e0, lb.e0_exp, lb.mask, lb.x2, lb.n_out, gamma, lb.e3, lb.e3_exp, lb.sum_e1,
                                  lb.sum_e1x2 if lb.x2 is not None else None)
             if overlap:
-                self.side.wait_stream(main)
-                with torch.cuda.stream(self.side):
-                    eoq.eoq_conv_wgrad(self.h_side, lb.desc, lb.e3, lb.e3_exp, lb.x0, 0 if i == 0 else sc.b1_c, lb.g,
-                                       lb.g_exp, None, self.workspace_side)
+                k = i % len(self.sides)
+                self.sides[k].wait_stream(main)
+                with torch.cuda.stream(self.sides[k]):
+                    eoq.eoq_conv_wgrad(self.h_sides[k], lb.desc, lb.e3, lb.e3_exp, lb.x0, 0 if i == 0 else sc.b1_c, lb.g,
+                                       lb.g_exp, None, self.workspace_sides[k])
             if l.has_dgrad:
                 eoq.eoq_conv_dgrad(h, lb.desc, lb.e3, lb.e3_exp, lb.w, lb.e4, lb.e4_exp, lb.sum_e4, None, ws)
             if not overlap:
                 eoq.eoq_conv_wgrad(h, lb.desc, lb.e3, lb.e3_exp, lb.x0, 0 if i == 0 else sc.b1_c, lb.g, lb.g_exp, None, ws)
         if overlap:
-            main.wait_stream(self.side)
+            for side in self.sides:
+                main.wait_stream(side)
         eoq.eoq_update(h, [lb.w for lb in self.layers], [lb.g for lb in self.layers], [lb.g_exp for lb in self.layers],
                        self.lr_mant, self.lr_exp, eoq.EOQ_ROUND_STOCHASTIC, seed=synth.BASE_SEED, step=self.step_no)
         self.step_no += 1
@@ -165,18 +170,24 @@ class TrainStep:
         with torch.cuda.stream(cap):
             self.run(overlap)
         torch.cuda.synchronize(self.dev)
-        before = eoq.eoq_launch_count(self.h) + eoq.eoq_launch_count(self.h_side)
+        before = self.launch_count()
         self.graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(self.graph, stream=cap):
             self.run(overlap)
         torch.cuda.synchronize(self.dev)
-        self.launches_per_step = eoq.eoq_launch_count(self.h) + eoq.eoq_launch_count(self.h_side) - before
+        self.launches_per_step = self.launch_count() - before
 
     def replay(self) -> None:
         self.graph.replay()
 
+    def launch_count(self) -> int:
+        return sum(eoq.eoq_launch_count(h) for h in [self.h] + self.h_sides)
+
     def status(self) -> int:
-        return eoq.eoq_last_status(self.h) | eoq.eoq_last_status(self.h_side)
+        st = 0
+        for h in [self.h] + self.h_sides:
+            st |= eoq.eoq_last_status(h)
+        return st
 
     def result_tensors(self):
         """Small per-step results a caller would read back: every gradient exponent and the last activation."""
