@@ -511,11 +511,11 @@ extern "C" int eoq_workspace_size(const eoq_conv_desc_t *desc, int pass, size_t 
         case EOQ_PASS_DGRAD:  // transposed weights + int32 sums
             *bytes = round256(g.w_elems) + round256(g.in_elems * sizeof(int32_t));
             return EOQ_OK;
-        case EOQ_PASS_WGRAD: {  // int64 sums + per-tap error sums + per-class error sums + split-K slices
+        case EOQ_PASS_WGRAD: {  // per-tap error sums, reduction cell, int64 sums, split-K slices
             WgradPatchPlan wp;
             const size_t slices = plan_wgrad_patch(wp, *desc, g.ho, g.wo) ? (size_t)wp.num_splits * g.w_elems * sizeof(int32_t) : 0;
-            *bytes = round256(g.w_elems * sizeof(long long)) + round256((size_t)desc->c_out * g.taps * sizeof(long long)) +
-                     round256(b1_error_scratch_bytes(*desc, bc)) + round256(slices);
+            *bytes = round256((size_t)desc->c_out * g.taps * sizeof(long long)) + 256 + round256(g.w_elems * sizeof(long long)) +
+                     round256(slices);
             return EOQ_OK;
         }
         default: return EOQ_ERR_BAD_ARG;
@@ -811,22 +811,29 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     const eoq_conv_desc_t &d = *desc;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
 
-    long long *acc = reinterpret_cast<long long *>(workspace);
-    long long *tap_sums = reinterpret_cast<long long *>(reinterpret_cast<char *>(workspace) + round256(g.w_elems * sizeof(long long)));
+    // workspace: [tap sums][reduction cell][int64 sums][split-K slices]; everything a call accumulates into sits
+    // at the front, so one memset clears it
+    const BorderClasses bc = border_classes(d, g);
+    if (b1_c != 0 && bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
+    char *ws = reinterpret_cast<char *>(workspace);
+    long long *tap_sums = reinterpret_cast<long long *>(ws);
+    const size_t tap_bytes = round256((size_t)d.c_out * g.taps * sizeof(long long));
+    WgradCells *cells = reinterpret_cast<WgradCells *>(ws + tap_bytes);
+    long long *acc = reinterpret_cast<long long *>(ws + tap_bytes + 256);
+    const size_t acc_bytes = round256(g.w_elems * sizeof(long long));
 
     WgradPatchPlan wp;
     if (plan_wgrad_patch(wp, d, g.ho, g.wo)) {
-        const BorderClasses bc = border_classes(d, g);
-        if (b1_c != 0 && bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
-        long long *class_sums = reinterpret_cast<long long *>(reinterpret_cast<char *>(tap_sums) +
-                                                              round256((size_t)d.c_out * g.taps * sizeof(long long)));
-        wp.partials = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(class_sums) + round256(b1_error_scratch_bytes(d, bc)));
+        wp.partials = reinterpret_cast<int32_t *>(ws + tap_bytes + 256 + acc_bytes);
         wp.dev = h->dev;
-        cudaError_t e = cudaSuccess;
-        if (b1_c != 0) {
+        cudaError_t e;
+        {
             ProfScope prof(h, EOQ_PROF_WGRAD_AUX, s);
-            e = launch_b1_error_sums(e3, tap_sums, class_sums, d, g.ho, g.wo, bc, h->sm_count, s);
-            count_launches(h, 2);
+            e = b1_c != 0 ? cudaMemsetAsync(ws, 0, tap_bytes + 256, s) : cudaMemsetAsync(cells, 0, 256, s);
+            if (e == cudaSuccess && b1_c != 0) {
+                e = launch_b1_error_sums(e3, tap_sums, d, g.ho, g.wo, bc, h->sm_count, s);
+                count_launches(h, 1);
+            }
         }
         if (e != cudaSuccess) return record(h, e);
         CUtensorMap map_x, map_e;
@@ -841,7 +848,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         if (e != cudaSuccess) return record(h, e);
         ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
         e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
-                          b1_c != 0 ? tap_sums : nullptr, b1_c, g.taps, d.c_in, wp.partials, wp.num_splits, h->dev,
+                          b1_c != 0 ? tap_sums : nullptr, b1_c, d.c_in, wp.partials, wp.num_splits, cells, h->dev,
                           h->sm_count, s);
         return record(h, e);
     }
@@ -917,17 +924,16 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     p.acc = acc;
     p.dev = h->dev;
 
-    ProfScope *aux = new (std::nothrow) ProfScope(h, EOQ_PROF_WGRAD_AUX, s);
-    cudaError_t e = cudaMemsetAsync(acc, 0, g.w_elems * sizeof(long long), s);
-    if (e == cudaSuccess && b1_c != 0) {
-        const BorderClasses bc = border_classes(d, g);
-        if (bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
-        long long *class_sums = reinterpret_cast<long long *>(reinterpret_cast<char *>(tap_sums) +
-                                                              round256((size_t)d.c_out * g.taps * sizeof(long long)));
-        e = launch_b1_error_sums(e3, tap_sums, class_sums, d, g.ho, g.wo, bc, h->sm_count, s);
-        count_launches(h, 2);
+    cudaError_t e;
+    {
+        ProfScope aux(h, EOQ_PROF_WGRAD_AUX, s);
+        // the GEMM adds into the int64 sums with atomics: they are cleared together with the cells and class sums
+        e = cudaMemsetAsync(ws, 0, tap_bytes + 256 + acc_bytes, s);
+        if (e == cudaSuccess && b1_c != 0) {
+            e = launch_b1_error_sums(e3, tap_sums, d, g.ho, g.wo, bc, h->sm_count, s);
+            count_launches(h, 1);
+        }
     }
-    delete aux;
     if (e != cudaSuccess) return record(h, e);
     CUtensorMap map_x, map_e;
     if (!make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage)) return EOQ_ERR_UNSUPPORTED;
@@ -936,7 +942,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                    : !make_im2col_map(&map_x, x, d.n, d.h, w_mem, d.c_in, d.x_wmargin - d.pad, -d.pad, g.wo, g.ho, d.stride,
                                       p.kc, p.pixels_per_stage))
         return EOQ_ERR_UNSUPPORTED;
-    count_launches(h, 3);  // the GEMM and the two kernels of Q_g
+    count_launches(h, 3);  // the GEMM, the finalize kernel and Q_g
     {
         ProfScope prof(h, EOQ_PROF_WGRAD, s);
         e = launch_wgrad(p, map_x, map_e, s);
@@ -945,7 +951,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     // the kernel leaves sums as [oc][tap][ic], which is the layout of g
     ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
     e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
-                      b1_c != 0 ? tap_sums : nullptr, b1_c, g.taps, d.c_in, nullptr, 0, h->dev, h->sm_count, s);
+                      b1_c != 0 ? tap_sums : nullptr, b1_c, d.c_in, nullptr, 0, cells, h->dev, h->sm_count, s);
     return record(h, e);
 }
 

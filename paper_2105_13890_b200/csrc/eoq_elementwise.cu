@@ -235,64 +235,53 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
 
 // ------------------------------------------------------------------ int64 -> SQ (Q_g after the weight gradient)
 
-// Sums the int32 split-K slices of the patch kernel into int64 (exact whatever the reduction length).
-// Block = (256 / groups) elements x `groups` slice groups: every thread adds its share of the slices with
-// independent, coalesced loads; the groups meet in shared memory.  Few slices -> one group, many -> eight.
-__global__ void wgrad_sum_slices_kernel(const int32_t *__restrict__ parts, int num_parts, size_t n, long long *acc)
+// Last step before Q_g: sums the int32 split-K slices of the patch kernel into int64 (exact whatever the reduction
+// length), or takes the int64 sums the other kernel left in `acc`; adds the b1 term of x1 = x0 + b1 (b1 times the
+// sum of the error over the pixels whose tap falls inside the image); optionally copies the exact sums out; and
+// reduces max |.|.  A block of 256 threads is (256 / groups) elements x `groups` slice groups: every thread adds
+// its share of the slices with independent, coalesced loads and the groups meet in shared memory.
+__global__ void wgrad_finalize_kernel(const int32_t *__restrict__ parts, int num_parts, int groups, size_t n, long long *acc,
+                                      const long long *__restrict__ tap_sums, int32_t b1_c, int c_in, long long *copy_out,
+                                      WgradCells *cells)
 {
     __shared__ long long part[256];
-    const int bx = blockDim.x, groups = blockDim.y;
-    for (size_t base = (size_t)blockIdx.x * bx; base < n; base += (size_t)gridDim.x * bx) {
-        const size_t i = base + threadIdx.x;
-        long long v = 0;
-        if (i < n)
-            for (int s = threadIdx.y; s < num_parts; s += groups) v += (long long)__ldg(parts + (size_t)s * n + i);
-        if (groups == 1) {
-            if (i < n) acc[i] = v;
-            continue;
-        }
-        part[threadIdx.y * bx + threadIdx.x] = v;
-        __syncthreads();
-        if (threadIdx.y == 0 && i < n) {
-            long long t = 0;
-            for (int k = 0; k < groups; ++k) t += part[k * bx + threadIdx.x];
-            acc[i] = t;
-        }
-        __syncthreads();
-    }
-}
-
-// Adds the b1 term of x1 = x0 + b1 (b1 times the sum of the error over the pixels whose tap falls inside
-// the image), optionally copies the exact sums out, and reduces max |.|.
-__global__ void wgrad_fix_absmax_kernel(long long *acc, size_t n, const long long *tap_sums, int32_t b1_c, int taps,
-                                        int c_in, const int32_t *__restrict__ parts, int num_parts, long long *copy_out,
-                                        DeviceState *dev)
-{
+    const int bx = 256 / groups, tx = threadIdx.x % bx, ty = threadIdx.x / bx;
     unsigned long long mx = 0;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        long long v;
+    for (size_t base = (size_t)blockIdx.x * bx; base < n; base += (size_t)gridDim.x * bx) {
+        const size_t i = base + tx;
+        long long v = 0;
         if (parts) {
-            // the split-K slices of the patch kernel: exact in 64 bits whatever the reduction length
-            v = 0;
-            for (int s = 0; s < num_parts; ++s) v += (long long)__ldg(parts + (size_t)s * n + i);
-        } else {
+            if (i < n)
+                for (int s = ty; s < num_parts; s += groups) v += (long long)__ldg(parts + (size_t)s * n + i);
+            if (groups > 1) {
+                part[threadIdx.x] = v;
+                __syncthreads();
+                if (ty == 0) {
+                    v = 0;
+                    for (int k = 0; k < groups; ++k) v += part[k * bx + tx];
+                }
+                __syncthreads();
+            }
+        } else if (i < n) {
             v = acc[i];
         }
-        if (tap_sums) v += (long long)b1_c * tap_sums[i / c_in];  // index of (oc, tap)
-        if (parts || tap_sums) acc[i] = v;
-        if (copy_out) copy_out[i] = v;
-        const unsigned long long a = (unsigned long long)(v < 0 ? -v : v);
-        mx = a > mx ? a : mx;
+        if (ty == 0 && i < n) {
+            if (tap_sums)  // index of (oc, tap); a 32-bit division whenever the tensor allows it
+                v += (long long)b1_c * tap_sums[n <= 0xffffffffull ? (size_t)((uint32_t)i / (uint32_t)c_in) : i / (size_t)c_in];
+            if (parts || tap_sums) acc[i] = v;
+            if (copy_out) copy_out[i] = v;
+            const unsigned long long a = (unsigned long long)(v < 0 ? -v : v);
+            mx = a > mx ? a : mx;
+        }
     }
     mx = block_max_u64(mx);
-    if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u64, mx);
-    (void)taps;
+    if (threadIdx.x == 0 && mx) atomicMax(&cells->absmax, mx);
 }
 
 __global__ void sq_i64_kernel(const long long *__restrict__ src, const int32_t *src_exp, int exp_bias, size_t n,
-                              int8_t *dst, int32_t *dst_exp, DeviceState *dev)
+                              int8_t *dst, int32_t *dst_exp, const WgradCells *cells, DeviceState *dev)
 {
-    const unsigned long long M = dev->absmax_u64;
+    const unsigned long long M = cells->absmax;
     const int t = M ? round_log2_u64(M) : 7;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         const int p_in = (src_exp ? *src_exp : 0) + exp_bias;
@@ -601,13 +590,15 @@ __global__ void b1_weight_table_kernel(const int8_t *__restrict__ w, int32_t *ta
     }
 }
 
-// class_sums[class][oc] = sum of e3[n,y,x,oc] over the pixels of a border class.  A block owns a range of
+// tap_sums[oc][tap] += sum of e3[n,y,x,oc] over the pixels for which the tap falls inside the image (the weight
+// gradient adds b1 times this to every input channel).  Pixels are summed per border class first (the taps inside
+// the image are the same for all pixels of a class).  A block owns a range of
 // pixels and a slab of channels; a lane keeps 16 channels (one 128-bit load per pixel), so a warp covers
 // 32 / (slab / 16) pixels per step.  Interior pixels (one class, almost all of a large image) accumulate in
 // registers, border pixels in shared memory.
 constexpr int kClassSlab = 128;
-__global__ void b1_class_sums_kernel(const int8_t *__restrict__ e3, long long *class_sums, int c_out, int ho, int wo,
-                                     size_t pixels, int pixels_per_block, BorderClasses bc)
+__global__ void b1_tap_sums_kernel(const int8_t *__restrict__ e3, long long *tap_sums, int c_out, int ho, int wo,
+                                   size_t pixels, int pixels_per_block, BorderClasses bc, eoq_conv_desc_t d)
 {
     extern __shared__ int32_t cls_acc[];  // [classes][kClassSlab]
     const int classes = bc.nrc * bc.ncc;
@@ -648,31 +639,35 @@ __global__ void b1_class_sums_kernel(const int8_t *__restrict__ e3, long long *c
         }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < classes * kClassSlab; i += blockDim.x) {
-        const int c = blockIdx.y * kClassSlab + (i % kClassSlab);
-        const int32_t v = cls_acc[i];
-        if (v && c < c_out)
-            atomicAdd(reinterpret_cast<unsigned long long *>(class_sums + (size_t)(i / kClassSlab) * c_out + c), (unsigned long long)(long long)v);
-    }
-}
-
-// tap_sums[oc][tap] = sum of the class sums of the classes for which the tap falls inside the image
-// (the weight gradient adds b1 times this to every input channel).
-__global__ void b1_tap_sums_kernel(const long long *__restrict__ class_sums, long long *tap_sums, eoq_conv_desc_t d, int ho,
-                                   int wo, BorderClasses bc)
-{
+    // a tap's sum is the sum over the classes for which the tap falls inside the image: formed here from the
+    // block's class sums, one 64-bit atomic per (channel, tap) and block
     const int taps = d.kh * d.kw;
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= d.c_out * taps) return;
-    const int oc = i / taps, tap = i % taps, kh = tap / d.kw, kw = tap % d.kw;
-    long long sum = 0;
-    for (int rc = 0; rc < bc.nrc; ++rc) {
-        if (!tap_valid(rc, kh, ho, d.h, bc.nlo_h, bc.nhi_h, bc.nrc, d.stride, d.pad)) continue;
+    __shared__ unsigned long long rows_in[32], cols_in[32];  // per filter row / column: the classes it is inside for
+    if (threadIdx.x < d.kh) {
+        unsigned long long m = 0;
+        for (int rc = 0; rc < bc.nrc; ++rc)
+            if (tap_valid(rc, threadIdx.x, ho, d.h, bc.nlo_h, bc.nhi_h, bc.nrc, d.stride, d.pad)) m |= 1ull << rc;
+        rows_in[threadIdx.x] = m;
+    } else if (threadIdx.x >= 32 && threadIdx.x < 32 + d.kw) {
+        unsigned long long m = 0;
         for (int cc = 0; cc < bc.ncc; ++cc)
-            if (tap_valid(cc, kw, wo, d.w, bc.nlo_w, bc.nhi_w, bc.ncc, d.stride, d.pad))
-                sum += class_sums[(size_t)(rc * bc.ncc + cc) * d.c_out + oc];
+            if (tap_valid(cc, threadIdx.x - 32, wo, d.w, bc.nlo_w, bc.nhi_w, bc.ncc, d.stride, d.pad)) m |= 1ull << cc;
+        cols_in[threadIdx.x - 32] = m;
     }
-    tap_sums[i] = sum;
+    __syncthreads();
+    // consecutive threads take consecutive taps of a channel: neighbouring cells of tap_sums[oc][tap]
+    for (int i = threadIdx.x; i < taps * slab_ch; i += blockDim.x) {
+        const int c = i / taps, tap = i % taps;
+        const unsigned long long cols = cols_in[tap % d.kw];
+        long long sum = 0;
+        for (unsigned long long rm = rows_in[tap / d.kw]; rm; rm &= rm - 1) {
+            const int32_t *row = cls_acc + (__ffsll((long long)rm) - 1) * bc.ncc * kClassSlab + c;
+            for (unsigned long long cm = cols; cm; cm &= cm - 1) sum += row[(__ffsll((long long)cm) - 1) * kClassSlab];
+        }
+        if (sum)
+            atomicAdd(reinterpret_cast<unsigned long long *>(tap_sums + (size_t)(blockIdx.y * kClassSlab + c) * taps + tap),
+                      (unsigned long long)sum);
+    }
 }
 
 }  // namespace
@@ -735,22 +730,18 @@ cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bi
 }
 
 cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
-                          int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int taps,
-                          int c_in, const int32_t *parts, int num_parts, DeviceState *dev, int sm_count, cudaStream_t s)
+                          int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int c_in,
+                          const int32_t *parts, int num_parts, WgradCells *cells, DeviceState *dev, int sm_count,
+                          cudaStream_t s)
 {
-    cudaError_t e = launch_reset_cells(dev, s);
-    if (e != cudaSuccess) return e;
-    if (parts) {
-        const int groups = num_parts >= 32 ? 8 : (num_parts >= 8 ? 4 : 1);
-        const int bx = 256 / groups;
-        size_t blocks = (n + bx - 1) / bx;
-        if (blocks > (size_t)sm_count * 16) blocks = (size_t)sm_count * 16;
-        wgrad_sum_slices_kernel<<<(unsigned)blocks, dim3(bx, groups), 0, s>>>(parts, num_parts, n, const_cast<long long *>(src));
-        parts = nullptr;
-    }
-    wgrad_fix_absmax_kernel<<<grid_for(n, sm_count), kThreads, 0, s>>>(const_cast<long long *>(src), n, tap_sums, b1_c,
-                                                                       taps, c_in, parts, num_parts, copy_out, dev);
-    sq_i64_kernel<<<grid_for(n, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, dev);
+    // the cells were zeroed by the caller's one memset at the head of the weight-gradient call
+    const int groups = !parts ? 1 : (num_parts >= 32 ? 8 : (num_parts >= 8 ? 4 : 1));
+    const int bx = 256 / groups;
+    size_t blocks = (n + bx - 1) / bx;
+    if (blocks > (size_t)sm_count * 16) blocks = (size_t)sm_count * 16;
+    wgrad_finalize_kernel<<<(unsigned)blocks, 256, 0, s>>>(parts, num_parts, groups, n, const_cast<long long *>(src), tap_sums,
+                                                           b1_c, c_in, copy_out, cells);
+    sq_i64_kernel<<<grid_for(n, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, cells, dev);
     return cudaGetLastError();
 }
 
@@ -831,17 +822,11 @@ cudaError_t launch_b1_weight_table(const int8_t *w, int32_t *table, const eoq_co
     return cudaGetLastError();
 }
 
-size_t b1_error_scratch_bytes(const eoq_conv_desc_t &d, const BorderClasses &bc)
+cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, const eoq_conv_desc_t &d, int ho, int wo,
+                                 const BorderClasses &bc, int sm_count, cudaStream_t s)
 {
-    return sizeof(long long) * (size_t)bc.nrc * bc.ncc * d.c_out;
-}
-
-cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, long long *class_sums, const eoq_conv_desc_t &d,
-                                 int ho, int wo, const BorderClasses &bc, int sm_count, cudaStream_t s)
-{
+    // tap_sums was zeroed by the caller
     const int classes = bc.nrc * bc.ncc;
-    cudaError_t e = cudaMemsetAsync(class_sums, 0, b1_error_scratch_bytes(d, bc), s);
-    if (e != cudaSuccess) return e;
     const size_t pixels = (size_t)d.n * ho * wo;
     const int slabs = (d.c_out + kClassSlab - 1) / kClassSlab;
     int blocks = (4 * sm_count + slabs - 1) / slabs;
@@ -850,10 +835,8 @@ cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, long lon
     if (ppb > (1u << 23)) ppb = 1u << 23;  // keeps the int32 class sums exact
     blocks = (int)((pixels + ppb - 1) / ppb);
     dim3 grid(blocks, slabs);
-    b1_class_sums_kernel<<<grid, 256, sizeof(int32_t) * classes * kClassSlab, s>>>(e3, class_sums, d.c_out, ho, wo, pixels,
-                                                                                 (int)ppb, bc);
-    const int n = d.c_out * d.kh * d.kw;
-    b1_tap_sums_kernel<<<(n + 255) / 256, 256, 0, s>>>(class_sums, tap_sums, d, ho, wo, bc);
+    b1_tap_sums_kernel<<<grid, 256, sizeof(int32_t) * classes * kClassSlab, s>>>(e3, tap_sums, d.c_out, ho, wo, pixels, (int)ppb,
+                                                                               bc, d);
     return cudaGetLastError();
 }
 

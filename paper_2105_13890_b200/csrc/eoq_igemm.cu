@@ -1,8 +1,10 @@
 // Implicit-GEMM convolution kernel for sm_100a: forward pass and error back-propagation of the EOQ layer
 // (arXiv 2105.13890, Sec. 3.2.1).  One persistent CTA per SM walks 128-row output tiles:
-//   warp 0   : TMA producer (im2col loads of the activation/error operand, tiled loads of the weights)
-//   warp 1   : owns tensor memory, issues tcgen05.mma kind::i8 (int8 x int8 -> int32 in TMEM)
-//   warps 2-9: epilogue; read the accumulators with tcgen05.ld and apply the layer's quantizers in registers
+//   warps 0, 2, 3: TMA producers (im2col loads of the activation/error operand, tiled loads of the weights); a
+//              thread gets a TMA instruction out only every few hundred cycles, but threads of different warps
+//              issue side by side, so the pipeline stages rotate over three producers
+//   warp 1       : owns tensor memory, issues tcgen05.mma kind::i8 (int8 x int8 -> int32 in TMEM)
+//   warps 4-19   : epilogue; read the accumulators with tcgen05.ld and apply the layer's quantizers in registers
 // Two accumulator buffers in TMEM let the epilogue of tile i overlap the main loop of tile i+1.
 // Every wait is bounded: when one runs out the CTA raises EOQ_DEV_TIMEOUT, drains and returns.
 #include "eoq_device.cuh"
@@ -14,6 +16,7 @@ namespace eoq {
 namespace {
 
 constexpr int kMaxStages = 8;
+constexpr int kProducers = 3;
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
 igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUtensorMap map_a,
@@ -37,7 +40,11 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
 
     uint32_t acc_stride = 32;
     while (acc_stride < (uint32_t)p.tile_n) acc_stride <<= 1;
-    const uint32_t tmem_cols = 2 * acc_stride;
+    // Tiles up to 128 columns keep two partial accumulators that successive MMAs alternate between (summed
+    // exactly in the epilogue), which removes the wait of an MMA on its predecessor's write-back.
+    const uint32_t nacc = (p.tile_n <= 128 && p.kc >= 32 && p.num_sub * (p.kc / 32) >= 2) ? 2u : 1u;
+    const uint32_t buf_stride = nacc * acc_stride;
+    const uint32_t tmem_cols = 2 * buf_stride;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.num_stages; ++s) {
@@ -68,11 +75,14 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
     const int k_iters = (p.num_sub + p.subs_per_stage - 1) / p.subs_per_stage;
     const int pix_per_img = p.hq * p.wq;
 
-    if (warp == 0) {
+    if (warp == 0 || warp == 2 || warp == 3) {
         if (lane == 0) {
-            // ------------------------------------------------------------------ TMA producer
-            int stage = 0;
-            uint32_t phase = 0;
+            // ------------------------------------------------------------------ TMA producers
+            // producer q fills the pipeline slots q, q + 3, q + 6, ... of the CTA's sequence of (tile, k iteration)
+            const int q = warp == 0 ? 0 : warp - 1;
+            int stage = q % p.num_stages;
+            uint32_t phase = (uint32_t)(q / p.num_stages) & 1u;
+            int turn = q;  // slots until this producer's next one
             uint32_t inflight = 0, inflight_parity = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
@@ -82,7 +92,9 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                 const int cw = (rem % p.wq) * p.src_stride_w + p.base_w;
                 const int ch = (rem / p.wq) * p.src_stride + p.base_h;
                 for (int kit = 0; kit < k_iters; ++kit) {
-                    if (!(ok = wait_bar(empty_bar(stage), phase ^ 1u, ctx))) break;
+                    if (turn-- != 0) continue;
+                    turn = kProducers - 1;
+                    if (!(ok = wait_bar<32>(empty_bar(stage), phase ^ 1u, ctx))) break;
                     const int s0 = kit * p.subs_per_stage;
                     const int subs = min(p.subs_per_stage, p.num_sub - s0);
                     const uint32_t a_dst = smem_base + stage * stage_bytes;
@@ -100,7 +112,8 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                     }
                     inflight |= 1u << stage;
                     inflight_parity = (inflight_parity & ~(1u << stage)) | (phase << stage);
-                    if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }
+                    stage += kProducers;
+                    while (stage >= p.num_stages) { stage -= p.num_stages; phase ^= 1u; }
                 }
             }
             if (!ok) {
@@ -130,22 +143,36 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 if (!(ok = wait_bar(tempty_bar(acc), acc_phase ^ 1u, ctx))) break;
                 ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * acc_stride;
+                const uint32_t d_tmem = tmem_base + acc * buf_stride, d_other = nacc == 2 ? d_tmem + acc_stride : d_tmem;
                 uint32_t accumulate = 0;
+                uint32_t fresh0 = 1u, fresh1 = nacc == 2 ? 1u : 0u;
                 for (int kit = 0; kit < k_iters; ++kit) {
                     if (!(ok = wait_bar(full_bar(stage), phase, ctx))) break;
                     ptx::tc_fence_after();
                     const int subs = min(p.subs_per_stage, p.num_sub - kit * p.subs_per_stage);
                     uint32_t a_lo = ((smem_base + stage * stage_bytes) >> 4) | a_lead;
                     uint32_t b_lo = (((smem_base + stage * stage_bytes) >> 4) + p.subs_per_stage * a_sub16) | b_lead;
-                    for (int j = 0; j < subs; j += sub_step) {
-                        for (int kk = 0; kk < k_steps; ++kk) {
-                            ptx::mma_i8(d_tmem, smem_desc_join(a_lo + 2 * kk, hi), smem_desc_join(b_lo + 2 * kk, hi), idesc,
-                                        accumulate);
-                            accumulate = 1;
+                    if (wide && k_steps >= 2) {
+                        // 2 or 4 MMAs per sub-tile, alternating between the two partial accumulators
+                        for (int j = 0; j < subs; ++j) {
+                            if (k_steps == 4) mma_k_steps<4>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1);
+                            else mma_k_steps<2>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1);
+                            fresh0 = 0;
+                            fresh1 = 0;
+                            a_lo += a_sub16;
+                            b_lo += b_sub16;
                         }
-                        a_lo += sub_step * a_sub16;
-                        b_lo += sub_step * b_sub16;
+                    } else {
+                        for (int j = 0; j < subs; j += sub_step) {
+                            // one MMA per step; with two accumulators successive steps alternate
+                            const bool odd = nacc == 2 && (accumulate & 2u);
+                            ptx::mma_i8(odd ? d_other : d_tmem, smem_desc_join(a_lo, hi), smem_desc_join(b_lo, hi), idesc,
+                                        odd ? (fresh1 ? 0u : 1u) : (fresh0 ? 0u : 1u));
+                            if (odd) fresh1 = 0; else fresh0 = 0;
+                            if (nacc == 2) accumulate ^= 2u;
+                            a_lo += sub_step * a_sub16;
+                            b_lo += sub_step * b_sub16;
+                        }
                     }
                     ptx::mma_commit(empty_bar(stage));
                     if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }
@@ -164,7 +191,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         // Four warps per scheduler: a warp may read the TMEM lanes of quadrant (warp % 4); the warps
         // of a quadrant split the tile's columns.
         const int quad = warp & 3;
-        const int part = (warp - 2) >> 2;  // the kEpilogueWarps / 4 warps of a lane quadrant split the columns
+        const int part = (warp - 4) >> 2;  // the kEpilogueWarps / 4 warps of a lane quadrant split the columns
         const int row = quad * 32 + lane;
         const int groups = p.tile_n / 16;                 // 16-column groups of the tile
         constexpr int kParts = kEpilogueWarps / 4;
@@ -196,11 +223,19 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                     cls = border_class(y, p.hq, p.b1_nlo_h, p.b1_nhi_h, p.b1_nrc) * p.b1_ncc +
                           border_class(x, p.wq, p.b1_nlo_w, p.b1_nhi_w, p.b1_ncc);
             }
-            const uint32_t t_row = tmem_base + acc * acc_stride + ((uint32_t)(quad * 32) << 16);
+            const uint32_t t_row = tmem_base + acc * buf_stride + ((uint32_t)(quad * 32) << 16);
             for (int g = g_begin; g < g_end; ++g) {
                 uint32_t r[32];
                 ptx::tmem_ld_32x16(t_row + g * 16, r);
-                ptx::tmem_ld_wait();
+                if (nacc == 2) {
+                    uint32_t r2[32];
+                    ptx::tmem_ld_32x16(t_row + acc_stride + g * 16, r2);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) r[i] += r2[i];  // the two partial accumulators of the tile
+                } else {
+                    ptx::tmem_ld_wait();
+                }
                 const int col = nt * p.tile_n + g * 16;
                 if (valid && col < p.N) {
                     const size_t off = pix * p.N + col;

@@ -11,8 +11,8 @@ namespace eoq {
 constexpr int kMaxTaps = 64;        // kh * kw of any supported filter
 constexpr int kTileM = 128;         // GEMM rows per CTA tile (TMEM lanes)
 constexpr int kEpilogueWarps = 16;  // implicit GEMM: four epilogue warps per scheduler hide the latency of the integer chain
-constexpr int kGemmThreads = 64 + 32 * kEpilogueWarps;  // warp 0: TMA, warp 1: MMA + TMEM owner, then the epilogue
-constexpr int kWgradThreads = 192;  // weight gradient: warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int kGemmThreads = 128 + 32 * kEpilogueWarps;  // warps 0, 2, 3: TMA, warp 1: MMA + TMEM owner, then the epilogue
+constexpr int kWgradThreads = 256;  // weight gradient: warps 0, 2, 3 TMA, warp 1 MMA, warps 4..7 epilogue
 constexpr uint32_t kSpinLimit = 1u << 22;  // polls before a wait gives up (normal waits end within microseconds)
 
 // Device state a handle owns.
@@ -195,9 +195,16 @@ cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bi
                           int sm_count, cudaStream_t s);
 // Q_g of the exact sums.  `src` holds int64 sums; when `parts` is given the sums are first formed from
 // `num_parts` int32 slices of n elements each (and written to src).
+// Reduction cell of one weight-gradient call; it lives in the call's workspace next to the tap sums so that one
+// memset at the head of the call clears everything the call accumulates into.
+struct WgradCells {
+    unsigned long long absmax;  // max |sum| over the weight tensor
+    unsigned long long pad;
+};
 cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
-                          int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int taps,
-                          int c_in, const int32_t *parts, int num_parts, DeviceState *dev, int sm_count, cudaStream_t s);
+                          int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int c_in,
+                          const int32_t *parts, int num_parts, WgradCells *cells, DeviceState *dev, int sm_count,
+                          cudaStream_t s);
 cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const uint8_t *mask, const int16_t *x2,
                                 size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
                                 long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s);
@@ -218,9 +225,8 @@ struct BorderClasses {
 };
 cudaError_t launch_b1_weight_table(const int8_t *w, int32_t *table, const eoq_conv_desc_t &d, const BorderClasses &bc,
                                    cudaStream_t s);
-size_t b1_error_scratch_bytes(const eoq_conv_desc_t &d, const BorderClasses &bc);
-cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, long long *class_sums, const eoq_conv_desc_t &d,
-                                 int ho, int wo, const BorderClasses &bc, int sm_count, cudaStream_t s);
+cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, const eoq_conv_desc_t &d, int ho, int wo,
+                                 const BorderClasses &bc, int sm_count, cudaStream_t s);
 constexpr int kMaxBorderClasses = 64;  // classes (rows x columns) the b1 kernels keep in shared memory
 
 }  // namespace eoq

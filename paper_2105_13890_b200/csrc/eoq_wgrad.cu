@@ -4,7 +4,9 @@
 // tcgen05.mma as MN-major tiles: a TMA im2col load brings [pixels][channels] of the activation for one
 // filter tap, a tiled TMA load brings [pixels][channels] of the error.  The pixel range is split across
 // CTAs (split-K); int32 partial sums leave TMEM and are combined exactly with 64-bit atomics.
-// Roles: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-5 epilogue.  All waits are bounded.
+// Roles: warps 0, 2, 3 TMA producers (a thread gets a TMA instruction out only every few hundred cycles, threads
+// of different warps issue side by side: the loads of every stage are dealt out over three producers), warp 1
+// MMA issuer and TMEM owner, warps 4-7 epilogue.  All waits are bounded.
 #include "eoq_device.cuh"
 #include "eoq_internal.h"
 
@@ -13,6 +15,7 @@ namespace eoq {
 namespace {
 
 constexpr int kMaxStages = 8;
+constexpr int kProducers = 3;
 
 struct RoleCtx {
     volatile uint32_t *abort_flag;
@@ -65,7 +68,7 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.num_stages; ++s) {
-            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(full_bar(s), kProducers);  // every producer announces its share of the stage's bytes
             ptx::mbar_init(empty_bar(s), 1);
         }
         ptx::mbar_init(done_bar, 1);
@@ -100,8 +103,14 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
         if (my_stages < 0) my_stages = 0;
     }
 
-    if (warp == 0) {
+    if (warp == 0 || warp == 2 || warp == 3) {
         if (lane == 0) {
+            // producer q issues the loads number q, q + 3, q + 6, ... of every stage (activation sub-tiles first,
+            // then the error sub-tiles)
+            const int q = warp == 0 ? 0 : warp - 1;
+            const int n_ops = subs_total + b_subs;
+            uint32_t my_bytes = 0;
+            for (int o = q; o < n_ops; o += kProducers) my_bytes += o < subs_total ? a_sub : b_sub;
             int stage = 0;
             uint32_t phase = 0, inflight = 0, inflight_parity = 0;
             bool ok = true;
@@ -114,19 +123,22 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
                 const int ch = (rem / p.wo) * p.src_stride + p.base_h;
                 const uint32_t a_dst = smem_base + stage * stage_bytes;
                 const uint32_t b_dst = a_dst + p.mtiles_per_cta * a_mtile;
-                ptx::mbar_expect_tx(full_bar(stage), subs_total * a_sub + b_subs * b_sub);
+                ptx::mbar_expect_tx(full_bar(stage), my_bytes);
+                int o = 0;
                 for (int jm = 0; jm < my_mtiles; ++jm) {
                     const int first_sub = (mt0 + jm) * p.subs_per_mtile;
                     const int subs = min(p.subs_per_mtile, total_subs - first_sub);  // sub-tiles of this M tile that exist
-                    for (int j = 0; j < subs; ++j) {
+                    for (int j = 0; j < subs; ++j, ++o) {
+                        if (o % kProducers != q) continue;
                         const int s = first_sub + j;
                         const int tap = s / p.chunks_per_tap, chunk = s % p.chunks_per_tap;
                         ptx::tma_load_im2col_4d(a_dst + jm * a_mtile + j * a_sub, &map_x, full_bar(stage), chunk * p.kc, cw, ch,
                                                 img, (uint16_t)p.tap_dw[tap], (uint16_t)p.tap_dh[tap]);
                     }
                 }
-                for (int j = 0; j < b_subs; ++j)
-                    ptx::tma_load_2d(b_dst + j * b_sub, &map_e, full_bar(stage), nt * p.tile_n + j * p.nc, q0);
+                for (int j = 0; j < b_subs; ++j, ++o)
+                    if (o % kProducers == q)
+                        ptx::tma_load_2d(b_dst + j * b_sub, &map_e, full_bar(stage), nt * p.tile_n + j * p.nc, q0);
                 inflight |= 1u << stage;
                 inflight_parity = (inflight_parity & ~(1u << stage)) | (phase << stage);
                 if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }

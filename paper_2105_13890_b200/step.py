@@ -165,7 +165,9 @@ class TrainStep:
         """Records one step into a CUDA graph (after an eager warm-up step on the capture stream).  Everything a
         call depends on is baked in at capture, including the update's step counter: replays repeat the same
         stochastic-rounding draws."""
-        cap = torch.cuda.Stream(device=self.dev)
+        # the capture stream carries the chain every layer waits on (error head -> dgrad -> next error head): it gets
+        # the higher priority, so that its kernels are placed before the side streams' weight-gradient work
+        cap = torch.cuda.Stream(device=self.dev, priority=-1)
         cap.wait_stream(torch.cuda.current_stream(self.dev))
         with torch.cuda.stream(cap):
             self.run(overlap)
