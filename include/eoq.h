@@ -15,7 +15,8 @@
  *     host round trip separates producer and consumer.
  *   - All bit widths are 8 (Sec. 5.1).  R(.) rounds to nearest, ties to even.
  *   - Layouts: activations and errors NHWC int8; weights [c_out][kh][kw][c_in]
- *     int8.  c_in and c_out must be multiples of 16 (pad with zero channels).
+ *     int8.  c_in and c_out must be multiples of 16 (pad with zero channels); c_in may
+ *     also be 8 for a first layer that takes the filter-row path (eoq_conv_desc_t).
  *   - Pointers named in a "device" list are device pointers the caller owns; the
  *     library never allocates or frees tensor memory.  Tensor pointers must be
  *     16-byte aligned.  Scratch memory is the caller's `workspace` (device, 256-byte
@@ -51,7 +52,7 @@ typedef struct eoq_handle_s *eoq_handle_t;
 typedef enum {
     EOQ_OK = 0,
     EOQ_ERR_BAD_ARG = 1,     /* null pointer, non-positive size, inconsistent geometry */
-    EOQ_ERR_ALIGNMENT = 2,   /* pointer not 16-byte aligned, channel count not a multiple of 16 */
+    EOQ_ERR_ALIGNMENT = 2,   /* pointer not 16-byte aligned, channel count not a multiple of 16 (or c_in = 8) */
     EOQ_ERR_UNSUPPORTED = 3, /* geometry outside what the kernels cover */
     EOQ_ERR_WORKSPACE = 4,   /* workspace missing, misaligned or too small */
     EOQ_ERR_RANGE = 5,       /* a scalar code outside its range */
@@ -72,10 +73,13 @@ typedef enum { EOQ_PASS_FWD = 0, EOQ_PASS_DGRAD = 1, EOQ_PASS_WGRAD = 2 } eoq_pa
  * Output spatial size is (h + 2 pad - kh) / stride + 1 by (w + 2 pad - kw) / stride + 1.
  * x_wmargin (normally 0): the INPUT tensor x is stored with that many zero pixels before and after every image
  * row, i.e. as [n][h][w + 2 x_wmargin][c_in] with the image in the middle (eoq_quantize_image writes this form).
- * The margins are part of the zero padding, not of the image.  With c_in = 16, a filter 5 to 8 taps wide and a
- * margin of at least max(pad, (wo-1) stride - pad + 8 - w) pixels (4 for the 7x7 stride-2 first layer of the
- * ImageNet ResNets) a whole filter row is fetched as one 128-byte run, which is several times faster than one
- * 16-byte fetch per tap.  Outputs and the error tensors never carry margins. */
+ * The margins are part of the zero padding, not of the image.  With c_in = 16 or 8, a filter 5 to 8 taps wide and
+ * a margin of at least max(pad, (wo-1) stride - pad + 8 - w) pixels (4 for the 7x7 stride-2 first layer of the
+ * ImageNet ResNets) a whole filter row is fetched as one 128- or 64-byte run (the filter-row path), which is
+ * several times faster than one 16-byte fetch per tap.  c_in = 8 (an RGB image padded to 8 channels) halves the
+ * padded reduction length again; it exists only on this path and needs an even stride, an even w and an even
+ * x_wmargin - pad (5 for that first layer), else forward and wgrad return EOQ_ERR_UNSUPPORTED; dgrad does not
+ * take c_in = 8 (the network input receives no error).  Outputs and the error tensors never carry margins. */
 typedef struct {
     int n, h, w, c_in, c_out, kh, kw, stride, pad, x_wmargin;
 } eoq_conv_desc_t;
@@ -193,7 +197,7 @@ EOQ_API int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const int
  * Input quantizer for the network input (Sec. 5.1 quantizes every layer but the last): SQ(., 8) of an fp32
  * NHWC image batch [n][h][w][c_src], written as int8 [n][h][w + 2 wmargin][c_dst] with c_dst >= c_src: the extra
  * channels and the wmargin pixels at both ends of every row are zero (see eoq_conv_desc_t::x_wmargin).
- * c_dst is a multiple of 16 and at most 64.  The maximum runs over the whole batch.  *dst_exp is written.
+ * c_dst is 8 or a multiple of 16 and at most 64.  The maximum runs over the whole batch.  *dst_exp is written.
  */
 EOQ_API int eoq_quantize_image(eoq_handle_t handle, const float *src, int n, int h, int w, int c_src, int c_dst,
                        int wmargin, int8_t *dst, int32_t *dst_exp, void *stream);

@@ -61,19 +61,21 @@ int chunk_bytes(int c)
 // View for the filter-row path: the pixel of the walk is a 128-byte window of 8 adjacent 16-channel pixels that
 // starts at memory column (first_col + k * stride) of a row w_mem pixels long, so consecutive windows overlap
 // (the W stride of the view is smaller than its inner extent).  Rows are walked with zero fill above and below.
-bool make_row_window_map(CUtensorMap *map, const void *ptr, int n, int h, int w_mem, int first_col, int count_w,
+bool make_row_window_map(CUtensorMap *map, const void *ptr, int n, int h, int w_mem, int c, int first_col, int count_w,
                          int count_h, int stride, int pad_h, int pixels)
 {
-    cuuint64_t dims[4] = {128, (cuuint64_t)count_w, (cuuint64_t)h, (cuuint64_t)n};
-    cuuint64_t strides[3] = {(cuuint64_t)stride * 16, (cuuint64_t)w_mem * 16, (cuuint64_t)w_mem * 16 * h};
+    const cuuint64_t window = 8u * c;  // bytes of 8 adjacent pixels
+    cuuint64_t dims[4] = {window, (cuuint64_t)count_w, (cuuint64_t)h, (cuuint64_t)n};
+    cuuint64_t strides[3] = {(cuuint64_t)stride * c, (cuuint64_t)w_mem * c, (cuuint64_t)w_mem * c * h};
     int lower[2] = {0, -pad_h};
     int upper[2] = {0, (count_h - 1) * stride + 1 - pad_h - h};
     if (upper[1] < -128 || upper[1] > 127 || pad_h > 128) return false;
     cuuint32_t estr[4] = {1, 1, (cuuint32_t)stride, 1};
-    const char *base = static_cast<const char *>(ptr) + (long long)first_col * 16;
+    const char *base = static_cast<const char *>(ptr) + (long long)first_col * c;
     return g_encode_im2col(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<char *>(base), dims, strides, lower, upper,
-                           128, (cuuint32_t)pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+                           (cuuint32_t)window, (cuuint32_t)pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           swizzle_for((int)window), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 bool make_im2col_map(CUtensorMap *map, const void *ptr, int n, int h, int w, int c, int lower_w, int lower_h,
@@ -147,7 +149,7 @@ int check_desc(const eoq_conv_desc_t *d, Geometry *g)
         d->stride <= 0 || d->pad < 0)
         return EOQ_ERR_BAD_ARG;
     if (d->h + 2 * d->pad < d->kh || d->w + 2 * d->pad < d->kw) return EOQ_ERR_BAD_ARG;
-    if (d->c_in % 16 || d->c_out % 16) return EOQ_ERR_ALIGNMENT;
+    if ((d->c_in % 16 && d->c_in != 8) || d->c_out % 16) return EOQ_ERR_ALIGNMENT;  // 8: the filter-row path only
     if (d->x_wmargin < 0 || d->x_wmargin > 64) return EOQ_ERR_BAD_ARG;
     if (d->kh * d->kw > kMaxTaps || d->kh > 16 || d->kw > 16 || d->stride > 8 || d->pad > 64) return EOQ_ERR_UNSUPPORTED;
     g->ho = (d->h + 2 * d->pad - d->kh) / d->stride + 1;
@@ -188,12 +190,15 @@ int record(Handle *h, cudaError_t e)
     return EOQ_ERR_CUDA;
 }
 
-// 16-channel inputs under filters 5 to 8 taps wide (the 7x7 first layer) stored with wide enough zero margins take
-// the filter-row path: a filter row is 8 adjacent 16-byte pixels, one 128-byte K sub-tile, instead of one
-// 16-byte TMA row per tap.
+// 16- or 8-channel inputs under filters 5 to 8 taps wide (the 7x7 first layer) stored with wide enough zero margins
+// take the filter-row path: a filter row is 8 adjacent pixels, one 128- or 64-byte K sub-tile, instead of one TMA
+// row per tap.  The window of an output pixel starts (stride * c_in) bytes after its neighbour's and the first one
+// (x_wmargin - pad) pixels into the row: both must be multiples of 16 bytes, which 8 channels meet for even strides
+// and an even distance between margin and padding.
 inline bool use_row_window(const eoq_conv_desc_t &d, int wo)
 {
-    if (d.c_in != 16 || d.kw < 5 || d.kw > 8) return false;
+    if ((d.c_in != 16 && d.c_in != 8) || d.kw < 5 || d.kw > 8) return false;
+    if (d.c_in == 8 && ((d.stride & 1) || ((d.x_wmargin - d.pad) & 1) || (d.w & 1))) return false;
     const int need_right = (wo - 1) * d.stride - d.pad + 8 - d.w;
     return d.x_wmargin >= d.pad && d.x_wmargin >= need_right;
 }
@@ -506,7 +511,7 @@ extern "C" int eoq_workspace_size(const eoq_conv_desc_t *desc, int pass, size_t 
     switch (pass) {
         case EOQ_PASS_FWD:  // b1 table, then the row-padded weights of the filter-row path
             *bytes = round256((size_t)bc.nrc * bc.ncc * desc->c_out * sizeof(int32_t)) +
-                     (use_row_window(*desc, g.wo) ? round256((size_t)desc->c_out * desc->kh * 128) : 0);
+                     (use_row_window(*desc, g.wo) ? round256((size_t)desc->c_out * desc->kh * 8 * desc->c_in) : 0);
             return EOQ_OK;
         case EOQ_PASS_DGRAD:  // transposed weights + int32 sums
             *bytes = round256(g.w_elems) + round256(g.in_elems * sizeof(int32_t));
@@ -553,6 +558,7 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     // the accumulator with its b1 term must fit int32: taps * c_in * (127 + |b1|) * 127 < 2^31
     if ((double)g.taps * d.c_in * (127.0 + (b1_c < 0 ? -b1_c : b1_c)) * 127.0 >= 2147483647.0 - 16777216.0) return EOQ_ERR_RANGE;
     const bool row_window = use_row_window(d, g.wo);
+    if (d.c_in == 8 && !row_window) return EOQ_ERR_UNSUPPORTED;
     if ((b1_c != 0 || row_window) && (st = check_workspace(desc, EOQ_PASS_FWD, workspace, workspace_bytes)) != EOQ_OK) return st;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const int w_mem = d.w + 2 * d.x_wmargin;
@@ -573,8 +579,8 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     if (patch) {
         for (int t = 0; t < g.taps; ++t) p.tap_b[t] = (unsigned char)t;
     } else if (row_window) {
-        // K sub-tile = one filter row (8 pixels x 16 channels); the map's W axis already steps by the stride
-        plan_igemm(p, 128, d.kh, h->sm_count);
+        // K sub-tile = one filter row (8 pixels x c_in channels); the map's W axis already steps by the stride
+        plan_igemm(p, 8 * d.c_in, d.kh, h->sm_count);
         p.src_stride_w = 1;
         p.base_w = 0;
         for (int t = 0; t < d.kh; ++t) {
@@ -585,7 +591,7 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
         const BorderClasses bc0 = border_classes(d, g);
         w_rows = reinterpret_cast<int8_t *>(workspace) + round256((size_t)bc0.nrc * bc0.ncc * d.c_out * sizeof(int32_t));
         ProfScope prof(h, EOQ_PROF_FWD_AUX, s);
-        cudaError_t e = launch_weight_pad_rows(w, w_rows, d.c_out, d.kh, d.kw, s);
+        cudaError_t e = launch_weight_pad_rows(w, w_rows, d.c_out, d.kh, d.kw, d.c_in, s);
         if (e != cudaSuccess) return record(h, e);
         count_launches(h, 1);
     } else {
@@ -635,8 +641,8 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
         return record(h, launch_igemm_patch(p, pl, map_a, map_b, ptiles < h->sm_count ? ptiles : h->sm_count, s));
     }
     if (row_window) {
-        if (!make_row_window_map(&map_a, x, d.n, d.h, w_mem, d.x_wmargin - d.pad, g.wo, g.ho, d.stride, d.pad, kTileM) ||
-            !make_weight_map(&map_b, w_rows, d.c_out, d.kh, 128, 128, p.tile_n))
+        if (!make_row_window_map(&map_a, x, d.n, d.h, w_mem, d.c_in, d.x_wmargin - d.pad, g.wo, g.ho, d.stride, d.pad, kTileM) ||
+            !make_weight_map(&map_b, w_rows, d.c_out, d.kh, 8 * d.c_in, 8 * d.c_in, p.tile_n))
             return EOQ_ERR_UNSUPPORTED;
     } else if (!make_im2col_map(&map_a, x, d.n, d.h, w_mem, d.c_in, d.x_wmargin - d.pad, -d.pad, g.wo, g.ho, d.stride, p.kc,
                                 kTileM) ||
@@ -661,6 +667,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     int st = check_desc(desc, &g);
     if (st != EOQ_OK) return st;
     if (!aligned16(e3) || !aligned16(w) || !aligned16(e4) || !aligned16(acc_dump)) return EOQ_ERR_ALIGNMENT;
+    if (desc->c_in % 16) return EOQ_ERR_UNSUPPORTED;  // 8 channels exist for the network input, which takes no error
     if ((st = check_workspace(desc, EOQ_PASS_DGRAD, workspace, workspace_bytes)) != EOQ_OK) return st;
     const eoq_conv_desc_t &d = *desc;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
@@ -862,13 +869,15 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     p.c_out = d.c_out;
     p.ntaps = g.taps;
     const bool row_window = use_row_window(d, g.wo);
+    if (d.c_in == 8 && !row_window) return EOQ_ERR_UNSUPPORTED;
     const int w_mem = d.w + 2 * d.x_wmargin;
-    p.kc = row_window ? 128 : chunk_bytes(d.c_in);
+    p.kc = row_window ? 8 * d.c_in : chunk_bytes(d.c_in);
     p.nc = chunk_bytes(d.c_out);
     p.chunks_per_tap = row_window ? 1 : d.c_in / p.kc;
     p.rows_total = g.taps * d.c_in;
     p.subs_per_mtile = kTileM / p.kc;
-    p.num_m_tiles = row_window ? d.kh : (p.rows_total + kTileM - 1) / kTileM;  // filter-row path: one M tile per filter row
+    // filter-row path: a filter row is 8 taps x c_in rows, 128 / (8 c_in) filter rows per M tile
+    p.num_m_tiles = row_window ? (d.kh * p.kc + kTileM - 1) / kTileM : (p.rows_total + kTileM - 1) / kTileM;
     if (row_window) {
         p.ntaps = d.kh;
         p.row_window_kw = d.kw;
@@ -937,7 +946,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     if (e != cudaSuccess) return record(h, e);
     CUtensorMap map_x, map_e;
     if (!make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage)) return EOQ_ERR_UNSUPPORTED;
-    if (row_window ? !make_row_window_map(&map_x, x, d.n, d.h, w_mem, d.x_wmargin - d.pad, g.wo, g.ho, d.stride, d.pad,
+    if (row_window ? !make_row_window_map(&map_x, x, d.n, d.h, w_mem, d.c_in, d.x_wmargin - d.pad, g.wo, g.ho, d.stride, d.pad,
                                           p.pixels_per_stage)
                    : !make_im2col_map(&map_x, x, d.n, d.h, w_mem, d.c_in, d.x_wmargin - d.pad, -d.pad, g.wo, g.ho, d.stride,
                                       p.kc, p.pixels_per_stage))
@@ -1033,7 +1042,7 @@ extern "C" int eoq_quantize_image(eoq_handle_t handle, const float *src, int n, 
     if (!h || !src || !dst || !dst_exp || n <= 0 || hh <= 0 || ww <= 0 || c_src <= 0 || c_dst < c_src || wmargin < 0 ||
         wmargin > 64)
         return EOQ_ERR_BAD_ARG;
-    if (c_dst % 16 || c_dst > 64 || !aligned16(src) || !aligned16(dst)) return EOQ_ERR_ALIGNMENT;
+    if ((c_dst % 16 && c_dst != 8) || c_dst > 64 || !aligned16(src) || !aligned16(dst)) return EOQ_ERR_ALIGNMENT;
     count_launches(h, 2);
     ProfScope prof(h, EOQ_PROF_OTHER, reinterpret_cast<cudaStream_t>(stream));
     return record(h, launch_quantize_image(src, n, hh, ww, c_src, c_dst, wmargin, dst, dst_exp, h->dev, h->sm_count,

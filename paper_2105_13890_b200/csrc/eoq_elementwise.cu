@@ -126,7 +126,8 @@ __global__ void quantize_f32_kernel(int mode, const float *__restrict__ src, siz
 }
 
 // SQ of an fp32 image under the already reduced maximum: c_src channels in, c_dst (zero-padded) channels out,
-// rows widened by `wmargin` zero pixels at both ends.
+// rows widened by `wmargin` zero pixels at both ends.  A thread writes kG = 16 or 8 channels of a pixel.
+template <int kG>
 __global__ void quantize_image_kernel(const float *__restrict__ src, int rows, int w, int c_src, int c_dst, int wmargin,
                                       int8_t *dst, int32_t *dst_exp, DeviceState *dev)
 {
@@ -138,7 +139,7 @@ __global__ void quantize_image_kernel(const float *__restrict__ src, int rows, i
         *dst_exp = usable ? -up : -7;
         if (mbits == 0) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
     }
-    const int groups = c_dst / 16;
+    const int groups = c_dst / kG;
     const int w_mem = w + 2 * wmargin;
     const size_t items = (size_t)rows * w_mem * groups;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
@@ -146,10 +147,10 @@ __global__ void quantize_image_kernel(const float *__restrict__ src, int rows, i
         const size_t mp = i / groups;            // pixel index in the widened layout
         const int xm = (int)(mp % w_mem) - wmargin;
         const size_t row = mp / w_mem;
-        int c[16];
+        int c[kG];
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-            const int ch = g * 16 + k;
+        for (int k = 0; k < kG; ++k) {
+            const int ch = g * kG + k;
             int v = 0;
             if (ch < c_src && xm >= 0 && xm < w) {
                 const float y = scalbnf(__ldg(src + (row * w + xm) * c_src + ch), up);
@@ -157,21 +158,25 @@ __global__ void quantize_image_kernel(const float *__restrict__ src, int rows, i
             }
             c[k] = v;
         }
-        reinterpret_cast<int4 *>(dst)[i] =
-            make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
-                      (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+        if (kG == 16)
+            reinterpret_cast<int4 *>(dst)[i] =
+                make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
+                          (int)pack4(c[8 % kG], c[9 % kG], c[10 % kG], c[11 % kG]), (int)pack4(c[12 % kG], c[13 % kG], c[14 % kG], c[15 % kG]));
+        else
+            reinterpret_cast<int2 *>(dst)[i] = make_int2((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]));
     }
 }
 
-// w[oc][kh][kw][16] -> wp[oc][kh][8][16] with zeros in the unused taps
+// w[oc][kh][kw][c] -> wp[oc][kh][8][c] with zeros in the unused taps; c = 16 (Pixel = int4) or 8 (int2)
+template <typename Pixel>
 __global__ void weight_pad_rows_kernel(const int8_t *__restrict__ w, int8_t *__restrict__ wp, int rows, int kw)
 {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;  // one 16-byte pixel of the padded layout
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;  // one pixel of the padded layout
     if (i >= rows * 8) return;
     const int r = i >> 3, t = i & 7;
-    int4 v = make_int4(0, 0, 0, 0);
-    if (t < kw) v = __ldg(reinterpret_cast<const int4 *>(w) + (size_t)r * kw + t);
-    reinterpret_cast<int4 *>(wp)[i] = v;
+    Pixel v = Pixel();
+    if (t < kw) v = __ldg(reinterpret_cast<const Pixel *>(w) + (size_t)r * kw + t);
+    reinterpret_cast<Pixel *>(wp)[i] = v;
 }
 
 // ------------------------------------------------------------------ int32 -> SQ (phase 2 of Q_e after dgrad)
@@ -573,6 +578,11 @@ __global__ void b1_weight_table_kernel(const int8_t *__restrict__ w, int32_t *ta
             sum = __dp4a(v.z, 0x01010101, sum);
             sum = __dp4a(v.w, 0x01010101, sum);
         }
+        if (d.c_in == 8 && lane == 0) {  // the 8-channel first layer: one 8-byte pixel per tap
+            const int2 v = __ldg(reinterpret_cast<const int2 *>(p));
+            sum = __dp4a(v.x, 0x01010101, sum);
+            sum = __dp4a(v.y, 0x01010101, sum);
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
         if (lane == 0) tap_sum[t] = sum;
@@ -700,15 +710,21 @@ cudaError_t launch_quantize_image(const float *src, int n, int h, int w, int c_s
     if (e != cudaSuccess) return e;
     const size_t count = (size_t)n * h * w * c_src;
     absmax_f32_kernel<<<grid_for(count / 4 + 1, sm_count), kThreads, 0, s>>>(src, count, dev);
-    const size_t items = (size_t)n * h * (w + 2 * wmargin) * (c_dst / 16);
-    quantize_image_kernel<<<grid_for(items, sm_count), kThreads, 0, s>>>(src, n * h, w, c_src, c_dst, wmargin, dst, dst_exp, dev);
+    if (c_dst % 16 == 0) {
+        const size_t items = (size_t)n * h * (w + 2 * wmargin) * (c_dst / 16);
+        quantize_image_kernel<16><<<grid_for(items, sm_count), kThreads, 0, s>>>(src, n * h, w, c_src, c_dst, wmargin, dst, dst_exp, dev);
+    } else {
+        const size_t items = (size_t)n * h * (w + 2 * wmargin) * (c_dst / 8);
+        quantize_image_kernel<8><<<grid_for(items, sm_count), kThreads, 0, s>>>(src, n * h, w, c_src, c_dst, wmargin, dst, dst_exp, dev);
+    }
     return cudaGetLastError();
 }
 
-cudaError_t launch_weight_pad_rows(const int8_t *w, int8_t *wp, int c_out, int kh, int kw, cudaStream_t s)
+cudaError_t launch_weight_pad_rows(const int8_t *w, int8_t *wp, int c_out, int kh, int kw, int c_in, cudaStream_t s)
 {
     const int rows = c_out * kh;
-    weight_pad_rows_kernel<<<(rows * 8 + 255) / 256, 256, 0, s>>>(w, wp, rows, kw);
+    if (c_in == 16) weight_pad_rows_kernel<int4><<<(rows * 8 + 255) / 256, 256, 0, s>>>(w, wp, rows, kw);
+    else weight_pad_rows_kernel<int2><<<(rows * 8 + 255) / 256, 256, 0, s>>>(w, wp, rows, kw);
     return cudaGetLastError();
 }
 

@@ -187,7 +187,7 @@ cudaError_t launch_reset_cells(DeviceState *dev, cudaStream_t s);
 cudaError_t launch_quantize_image(const float *src, int n, int h, int w, int c_src, int c_dst, int wmargin, int8_t *dst,
                                   int32_t *dst_exp, DeviceState *dev, int sm_count, cudaStream_t s);
 // w[oc][kh][kw][16] -> wp[oc][kh][8][16], zero in the taps kw..7 (weights of the filter-row path)
-cudaError_t launch_weight_pad_rows(const int8_t *w, int8_t *wp, int c_out, int kh, int kw, cudaStream_t s);
+cudaError_t launch_weight_pad_rows(const int8_t *w, int8_t *wp, int c_out, int kh, int kw, int c_in, cudaStream_t s);
 cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst, int32_t *dst_exp, DeviceState *dev,
                                 int sm_count, cudaStream_t s);
 cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,

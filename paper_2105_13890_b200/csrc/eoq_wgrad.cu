@@ -193,10 +193,11 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
             int row = mt * kTileM + quad * 32 + lane;  // (tap, ic) flattened: tap * c_in + ic
             bool valid = row < p.rows_total;
             if (p.row_window_kw) {
-                // the tile's rows are (tap 0..7, channel 0..15) of filter row mt: drop the padding taps
-                const int t = (quad * 32 + lane) >> 4;
-                valid = t < p.row_window_kw;
-                row = (mt * p.row_window_kw + t) * 16 + (lane & 15);
+                // filter-row path: the rows are (filter row, tap 0..7, channel): drop the padding taps
+                const int per_frow = 8 * p.c_in, fr = row / per_frow, within = row % per_frow;
+                const int t = within / p.c_in;
+                valid = fr < p.ntaps && t < p.row_window_kw;
+                row = (fr * p.row_window_kw + t) * p.c_in + within % p.c_in;
             }
             const uint32_t t_row = tmem_base + jm * p.tile_n + ((uint32_t)(quad * 32) << 16);
             for (int c0 = 0; c0 < p.tile_n; c0 += 32) {

@@ -72,7 +72,8 @@ class TrainStep:
         self.step_no = 0
         # the network input is stored with zero row margins so that a wide first-layer filter can fetch whole
         # filter rows (eoq_conv_desc_t::x_wmargin); every other layer input is dense
-        first_margin = 4 if workload.layers[0].k >= 5 else 0
+        # 5 = padding 3 plus an even distance, which the 8-channel layout needs for 16-byte aligned windows
+        first_margin = 5 if workload.layers[0].k >= 5 else 0
         self.layers: List[LayerBuffers] = [LayerBuffers(l, self.dev, first_margin if i == 0 else 0)
                                            for i, l in enumerate(workload.layers)]
         ws = 256

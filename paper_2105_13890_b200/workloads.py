@@ -5,7 +5,8 @@ carries the geometry the C ABI needs plus what the Fixup layer unit around the c
 3.2.1): whether a ReLU follows, whether a shortcut joins before it, whether gamma is trainable (then x2 is
 kept for g_gamma), whether the layer sits in a residual branch (then its Kaiming weights are scaled by
 L^(-1/(2m-2))), and whether an error has to be propagated to its input (not for the first layer).
-Channel counts are padded to multiples of 16 for the kernels; `c_in_true` keeps the real count for op counting.
+Channel counts are padded to multiples of 16 for the kernels (8 for the RGB input of a 7x7 first layer);
+`c_in_true` keeps the real count for op counting.
 """
 from __future__ import annotations
 
@@ -105,9 +106,14 @@ def _basic_stage(layers, name, n, h, c_in, c_out, blocks, stride):
     return h
 
 
+# The RGB input of a 7x7 stride-2 first layer is stored with 8 channels (3 real): the library's filter-row path
+# takes 8- or 16-channel inputs and a filter row of 8 pixels is then a 64-byte K slice instead of 128.
+STEM_CHANNELS = 8
+
+
 def resnet18(batch: int = 64, image: int = 224) -> Workload:
     layers: List[Layer] = []
-    layers.append(Layer("stem", batch, image, image, _pad16(3), 64, 7, 2, 3, 3, in_branch=False, has_dgrad=False))
+    layers.append(Layer("stem", batch, image, image, STEM_CHANNELS, 64, 7, 2, 3, 3, in_branch=False, has_dgrad=False))
     h = (image + 6 - 7) // 2 + 1
     h = (h + 2 - 3) // 2 + 1  # 3x3 stride-2 max-pool
     c = 64
@@ -129,7 +135,7 @@ def resnet20(batch: int = 128, image: int = 32) -> Workload:
 
 def resnet50(batch: int = 32, image: int = 224) -> Workload:
     layers: List[Layer] = []
-    layers.append(Layer("stem", batch, image, image, _pad16(3), 64, 7, 2, 3, 3, in_branch=False, has_dgrad=False))
+    layers.append(Layer("stem", batch, image, image, STEM_CHANNELS, 64, 7, 2, 3, 3, in_branch=False, has_dgrad=False))
     h = (image + 6 - 7) // 2 + 1
     h = (h + 2 - 3) // 2 + 1
     c = 64

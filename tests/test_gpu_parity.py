@@ -109,6 +109,9 @@ MARGIN_CASES = [
     (ConvDesc(2, 12, 12, 16, 16, 5, 5, 1, 2), 4),     # 5 taps wide, stride 1
     (ConvDesc(2, 20, 20, 16, 64, 7, 7, 2, 3), 2),     # margin too small for the filter-row path: per-tap path
     (ConvDesc(2, 9, 9, 32, 48, 3, 3, 1, 1), 3),       # margins on an ordinary layer
+    (ConvDesc(2, 20, 20, 8, 64, 7, 7, 2, 3), 5),      # 8-channel input: a filter row is a 64-byte K slice
+    (ConvDesc(3, 18, 22, 8, 32, 7, 7, 2, 3), 7),      # 8 channels, unequal extents, wider margin
+    (ConvDesc(2, 16, 16, 8, 16, 5, 5, 2, 2), 4),      # 8 channels, 5 taps, pad 2
 ]
 
 
@@ -140,16 +143,16 @@ def test_input_with_row_margins(d, m):
         assert np.array_equal(G.host(g_d).astype(np.int32), g)
 
 
-@pytest.mark.parametrize("m", [0, 4])
-def test_quantize_image_pads_channels_and_rows(m):
+@pytest.mark.parametrize("m,c_dst", [(0, 16), (4, 16), (5, 8), (0, 8)])
+def test_quantize_image_pads_channels_and_rows(m, c_dst):
     n, h, w = 3, 10, 13
     img = synth.normal_f32((n, h, w, 3), 950, m)
-    padded = np.zeros((n, h, w, 16), dtype=np.float32)
+    padded = np.zeros((n, h, w, c_dst), dtype=np.float32)
     padded[..., :3] = img
     c, p, _ = oracle.quantize_f32(oracle.MODE_SQ, padded)
-    out = torch.full((n, h, w + 2 * m, 16), 55, dtype=torch.int8, device="cuda:0")
+    out = torch.full((n, h, w + 2 * m, c_dst), 55, dtype=torch.int8, device="cuda:0")
     ex = G.zeros(1, torch.int32)
-    eoq.eoq_quantize_image(G.handle(), G.dev(img), n, h, w, 3, 16, m, out, ex)
+    eoq.eoq_quantize_image(G.handle(), G.dev(img), n, h, w, 3, c_dst, m, out, ex)
     assert G.status_clear() == 0 and ex.item() == p
     assert np.array_equal(G.host(out).astype(np.int32), with_margin(c, m))
 
@@ -330,4 +333,9 @@ def test_argument_errors_launch_nothing():
     ex = G.zeros(1, torch.int32)
     assert eoq.eoq_conv_dgrad(h, d, y, ex, w, x, ex, check=False) == eoq.EOQ_ERR_WORKSPACE
     assert eoq.eoq_conv_fwd(h, eoq.conv_desc(1, 8, 8, 16, 16, 9, 9, 1, 4), x, None, 0, w, 128, 0, None, True, y, check=False) == eoq.EOQ_ERR_UNSUPPORTED
+    # 8 input channels exist only on the filter-row path: ordinary layers, odd margin distances and dgrad refuse them
+    ws = G.zeros(1 << 20, torch.uint8)
+    assert eoq.eoq_conv_fwd(h, eoq.conv_desc(1, 8, 8, 8, 16, 3, 3, 1, 1), x, None, 0, w, 128, 0, None, True, y, None, None, None, ws, check=False) == eoq.EOQ_ERR_UNSUPPORTED
+    assert eoq.eoq_conv_fwd(h, eoq.conv_desc(1, 8, 8, 8, 16, 7, 7, 2, 3, 4), x, None, 0, w, 128, 0, None, True, y, None, None, None, ws, check=False) == eoq.EOQ_ERR_UNSUPPORTED
+    assert eoq.eoq_conv_dgrad(h, eoq.conv_desc(1, 8, 8, 8, 16, 7, 7, 2, 3, 5), y, ex, w, x, ex, None, None, ws, check=False) == eoq.EOQ_ERR_UNSUPPORTED
     assert G.status_clear() == 0
