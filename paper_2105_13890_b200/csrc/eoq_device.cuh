@@ -236,24 +236,50 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem desc] * B[smem desc], int8 x int8 -> int32.
-// (No memory clobber: the issuing thread's scalar work between two MMAs is what limits narrow tiles, so the
+// The warp that feeds the tensor core runs its whole loop with all 32 lanes (so that every address and
+// descriptor it computes is the same in all lanes and can live in the uniform datapath, which is where the MMA
+// instruction takes its operands from) and only the instructions that must come from a single thread are
+// predicated on one elected lane.  Issued from inside a one-lane branch instead, every operand has to be moved
+// from a vector to a uniform register per MMA, which costs more cycles than a narrow MMA takes.
+
+// 1 in exactly one lane of the (fully active) warp, 0 in the others.
+__device__ __forceinline__ uint32_t elect_one()
+{
+    uint32_t leader;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(leader));
+    return leader;
+}
+
+// Index of the calling warp in its block, in a form the compiler knows to be the same in all lanes.
+__device__ __forceinline__ int warp_index_uniform() { return __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0); }
+
+// D[tmem] (+)= A[smem desc] * B[smem desc], int8 x int8 -> int32, issued by the lane whose `leader` is non-zero.
+// (No memory clobber: the issuing warp's scalar work between two MMAs is what limits narrow tiles, so the
 // compiler must be free to keep loop state in registers.  Ordering against barrier waits and commits comes from
 // those being volatile asm statements with memory clobbers.)
 __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate)
+                                       uint32_t accumulate, uint32_t leader)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate));
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader));
 }
 
-// The mbarrier receives one arrival when every MMA issued so far by this thread has completed.
-__device__ __forceinline__ void mma_commit(uint32_t bar)
+// The mbarrier receives one arrival when every MMA issued so far by the leader lane has completed.
+__device__ __forceinline__ void mma_commit(uint32_t bar, uint32_t leader)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(bar), "r"(leader) : "memory");
 }
 
 // 32 lanes x 32 columns of 32-bit accumulators: thread t of the warp receives lane (base lane + t).
@@ -284,6 +310,9 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 
 }  // namespace ptx
 
+using ptx::elect_one;
+using ptx::warp_index_uniform;
+
 // 64-bit shared-memory matrix descriptor of tcgen05.mma (start address, leading and stride byte offsets
 // in 16-byte units, descriptor version 1 at bit 46, swizzle mode at bits 61..63).
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes,
@@ -302,7 +331,7 @@ __device__ __forceinline__ uint32_t smem_desc_hi(uint32_t sbo_bytes, uint32_t la
 }
 __device__ __forceinline__ uint64_t smem_desc_join(uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; }
 
-// The thread that feeds the tensor core is a single in-order instruction stream: about 25 scalar instructions
+// The warp that feeds the tensor core is a single in-order instruction stream: about 25 scalar instructions
 // per MMA cost ~130 cycles, while a 128 x 64 x 32 MMA takes 52.  The issue helpers below are therefore fully
 // unrolled with compile-time MMA indices, so that an MMA costs a handful of integer adds.
 //
@@ -313,7 +342,8 @@ __device__ __forceinline__ uint64_t smem_desc_join(uint32_t lo, uint32_t hi) { r
 // kSteps 32-byte K steps of one (A sub-tile, B sub-tile) pair; `parity` = index of the first MMA modulo 2.
 template <int kSteps>
 __device__ __forceinline__ void mma_k_steps(uint32_t d0, uint32_t d1, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
-                                            uint32_t idesc, uint32_t parity, uint32_t fresh0, uint32_t fresh1)
+                                            uint32_t idesc, uint32_t parity, uint32_t fresh0, uint32_t fresh1,
+                                            uint32_t leader)
 {
 #pragma unroll
     for (int kk = 0; kk < kSteps; ++kk) {
@@ -321,7 +351,7 @@ __device__ __forceinline__ void mma_k_steps(uint32_t d0, uint32_t d1, uint32_t a
         // the first MMA into each accumulator overwrites it
         uint32_t acc = 1u;
         if (kk < 2) acc = (odd ? fresh1 : fresh0) ? 0u : 1u;
-        ptx::mma_i8(odd ? d1 : d0, smem_desc_join(a_lo + 2 * kk, hi), smem_desc_join(b_lo + 2 * kk, hi), idesc, acc);
+        ptx::mma_i8(odd ? d1 : d0, smem_desc_join(a_lo + 2 * kk, hi), smem_desc_join(b_lo + 2 * kk, hi), idesc, acc, leader);
     }
 }
 
@@ -330,7 +360,7 @@ __device__ __forceinline__ void mma_k_steps(uint32_t d0, uint32_t d1, uint32_t a
 template <int kDim, int kSteps>
 __device__ __forceinline__ void mma_patch_chunk(uint32_t d0, uint32_t d1, uint32_t a_lo, uint32_t b_lo, uint32_t row16,
                                                 uint32_t kc16, uint32_t b_sub16, uint32_t hi, uint32_t idesc,
-                                                bool first_chunk, bool two_acc)
+                                                bool first_chunk, bool two_acc, uint32_t leader)
 {
 #pragma unroll
     for (int a = 0; a < kDim; ++a)
@@ -343,7 +373,7 @@ __device__ __forceinline__ void mma_patch_chunk(uint32_t d0, uint32_t d1, uint32
                 if (idx == 0) acc = first_chunk ? 0u : 1u;
                 if (idx == 1) acc = (first_chunk && two_acc) ? 0u : 1u;
                 ptx::mma_i8((idx & 1) ? d1 : d0, smem_desc_join(a_lo + a * row16 + b * kc16 + 2 * kk, hi),
-                            smem_desc_join(b_lo + (a * kDim + b) * b_sub16 + 2 * kk, hi), idesc, acc);
+                            smem_desc_join(b_lo + (a * kDim + b) * b_sub16 + 2 * kk, hi), idesc, acc, leader);
             }
 }
 // Swizzle field of the descriptor for a sub-tile whose rows are `row_bytes` wide.

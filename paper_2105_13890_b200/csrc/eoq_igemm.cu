@@ -27,7 +27,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile uint32_t abort_s;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_sub = (uint32_t)kTileM * p.kc, b_sub = (uint32_t)p.tile_n * p.kc;
     const uint32_t stage_bytes = (uint32_t)p.subs_per_stage * (a_sub + b_sub);
@@ -125,66 +125,67 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ------------------------------------------------------------------ MMA issuer
-            const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, false, false);
-            // Descriptors are assembled from precomputed halves; the loop only adds offsets in 16-byte units.
-            // kc >= 32: swizzled K-major sub-tiles, rows kc bytes wide, 8-row groups 8*kc apart; a 32-byte K step
-            // moves the start address inside the swizzle span.  kc == 16: no swizzle, one MMA spans two sub-tiles
-            // (two taps): the second half of K sits one sub-tile further (leading offset), 8-row groups 128 B apart.
-            const bool wide = p.kc >= 32;
-            const uint32_t hi = wide ? smem_desc_hi(8u * p.kc, layout_type_for(p.kc)) : smem_desc_hi(128, 0);
-            const uint32_t a_sub16 = a_sub >> 4, b_sub16 = b_sub >> 4;
-            const uint32_t a_lead = wide ? 0u : (a_sub16 << 16), b_lead = wide ? 0u : (b_sub16 << 16);
-            const int sub_step = wide ? 1 : 2, k_steps = wide ? p.kc / 32 : 1;
-            int stage = 0, acc = 0;
-            uint32_t phase = 0, acc_phase = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                if (!(ok = wait_bar(tempty_bar(acc), acc_phase ^ 1u, ctx))) break;
+        // the whole warp runs the issue loop; one elected lane issues the MMAs and commits (see elect_one)
+        const uint32_t leader = elect_one();
+        const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_s, 0);
+        // ------------------------------------------------------------------ MMA issuer
+        const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, false, false);
+        // Descriptors are assembled from precomputed halves; the loop only adds offsets in 16-byte units.
+        // kc >= 32: swizzled K-major sub-tiles, rows kc bytes wide, 8-row groups 8*kc apart; a 32-byte K step
+        // moves the start address inside the swizzle span.  kc == 16: no swizzle, one MMA spans two sub-tiles
+        // (two taps): the second half of K sits one sub-tile further (leading offset), 8-row groups 128 B apart.
+        const bool wide = p.kc >= 32;
+        const uint32_t hi = wide ? smem_desc_hi(8u * p.kc, layout_type_for(p.kc)) : smem_desc_hi(128, 0);
+        const uint32_t a_sub16 = a_sub >> 4, b_sub16 = b_sub >> 4;
+        const uint32_t a_lead = wide ? 0u : (a_sub16 << 16), b_lead = wide ? 0u : (b_sub16 << 16);
+        const int sub_step = wide ? 1 : 2, k_steps = wide ? p.kc / 32 : 1;
+        int stage = 0, acc = 0;
+        uint32_t phase = 0, acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            if (!(ok = __all_sync(0xffffffffu, wait_bar(tempty_bar(acc), acc_phase ^ 1u, ctx)))) break;
+            ptx::tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * buf_stride, d_other = nacc == 2 ? d_tmem + acc_stride : d_tmem;
+            uint32_t accumulate = 0;
+            uint32_t fresh0 = 1u, fresh1 = nacc == 2 ? 1u : 0u;
+            for (int kit = 0; kit < k_iters; ++kit) {
+                if (!(ok = __all_sync(0xffffffffu, wait_bar(full_bar(stage), phase, ctx)))) break;
                 ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * buf_stride, d_other = nacc == 2 ? d_tmem + acc_stride : d_tmem;
-                uint32_t accumulate = 0;
-                uint32_t fresh0 = 1u, fresh1 = nacc == 2 ? 1u : 0u;
-                for (int kit = 0; kit < k_iters; ++kit) {
-                    if (!(ok = wait_bar(full_bar(stage), phase, ctx))) break;
-                    ptx::tc_fence_after();
-                    const int subs = min(p.subs_per_stage, p.num_sub - kit * p.subs_per_stage);
-                    uint32_t a_lo = ((smem_base + stage * stage_bytes) >> 4) | a_lead;
-                    uint32_t b_lo = (((smem_base + stage * stage_bytes) >> 4) + p.subs_per_stage * a_sub16) | b_lead;
-                    if (wide && k_steps >= 2) {
-                        // 2 or 4 MMAs per sub-tile, alternating between the two partial accumulators
-                        for (int j = 0; j < subs; ++j) {
-                            if (k_steps == 4) mma_k_steps<4>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1);
-                            else mma_k_steps<2>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1);
-                            fresh0 = 0;
-                            fresh1 = 0;
-                            a_lo += a_sub16;
-                            b_lo += b_sub16;
-                        }
-                    } else {
-                        for (int j = 0; j < subs; j += sub_step) {
-                            // one MMA per step; with two accumulators successive steps alternate
-                            const bool odd = nacc == 2 && (accumulate & 2u);
-                            ptx::mma_i8(odd ? d_other : d_tmem, smem_desc_join(a_lo, hi), smem_desc_join(b_lo, hi), idesc,
-                                        odd ? (fresh1 ? 0u : 1u) : (fresh0 ? 0u : 1u));
-                            if (odd) fresh1 = 0; else fresh0 = 0;
-                            if (nacc == 2) accumulate ^= 2u;
-                            a_lo += sub_step * a_sub16;
-                            b_lo += sub_step * b_sub16;
-                        }
+                const int subs = min(p.subs_per_stage, p.num_sub - kit * p.subs_per_stage);
+                uint32_t a_lo = ((smem_base + stage * stage_bytes) >> 4) | a_lead;
+                uint32_t b_lo = (((smem_base + stage * stage_bytes) >> 4) + p.subs_per_stage * a_sub16) | b_lead;
+                if (wide && k_steps >= 2) {
+                    // 2 or 4 MMAs per sub-tile, alternating between the two partial accumulators
+                    for (int j = 0; j < subs; ++j) {
+                        if (k_steps == 4) mma_k_steps<4>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1, leader);
+                        else mma_k_steps<2>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1, leader);
+                        fresh0 = 0;
+                        fresh1 = 0;
+                        a_lo += a_sub16;
+                        b_lo += b_sub16;
                     }
-                    ptx::mma_commit(empty_bar(stage));
-                    if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }
+                } else {
+                    for (int j = 0; j < subs; j += sub_step) {
+                        // one MMA per step; with two accumulators successive steps alternate
+                        const bool odd = nacc == 2 && (accumulate & 2u);
+                        ptx::mma_i8(odd ? d_other : d_tmem, smem_desc_join(a_lo, hi), smem_desc_join(b_lo, hi), idesc,
+                                    odd ? (fresh1 ? 0u : 1u) : (fresh0 ? 0u : 1u), leader);
+                        if (odd) fresh1 = 0; else fresh0 = 0;
+                        if (nacc == 2) accumulate ^= 2u;
+                        a_lo += sub_step * a_sub16;
+                        b_lo += sub_step * b_sub16;
+                    }
                 }
-                if (ok) ptx::mma_commit(tfull_bar(acc));
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                ptx::mma_commit(empty_bar(stage), leader);
+                if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }
             }
-            if (!ok) {
-                ptx::mma_commit(drain_bar);
-                for (uint32_t i = 0; i < kSpinLimit; ++i)
-                    if (ptx::mbar_try_wait(drain_bar, 0)) break;
-            }
+            if (ok) ptx::mma_commit(tfull_bar(acc), leader);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (!ok) {
+            ptx::mma_commit(drain_bar, leader);
+            for (uint32_t i = 0; i < kSpinLimit; ++i)
+                if (ptx::mbar_try_wait(drain_bar, 0)) break;
         }
     } else {
         // ---------------------------------------------------------------------- epilogue

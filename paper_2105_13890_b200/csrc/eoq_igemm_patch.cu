@@ -32,7 +32,7 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile uint32_t abort_s;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t b_sub = (uint32_t)p.tile_n * p.kc;
     const uint32_t b_region = smem_base + (uint32_t)pl.num_a * pl.a_bytes;
@@ -143,85 +143,85 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ------------------------------------------------------------------ MMA issuer
-            const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, false, false);
-            const uint32_t hi = smem_desc_hi(8u * p.kc, layout_type_for(p.kc));
-            const uint32_t b_sub16 = b_sub >> 4, b_ring_lo = b_region >> 4;
-            const uint32_t kc16 = (uint32_t)p.kc >> 4, row16 = (uint32_t)(pl.pw * p.kc) >> 4;  // one pixel / one patch row
-            const int k_steps = p.kc / 32, kdim = pl.kdim, chunks = pl.chunks, num_a = pl.num_a, num_b = pl.num_b;
-            const bool resident = pl.b_resident != 0;
-            int ia = 0, ib = 0, acc = 0;
-            uint32_t pha = 0, phb = 0, acc_phase = 0;
-            bool ok = true;
-            if (resident) ok = wait_bar(b_full(0), 0, ctx);
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                if (!(ok = wait_bar(tempty_bar(acc), acc_phase ^ 1u, ctx))) break;
+        // ---------------------------------------------------------------------- MMA issuer (whole warp, see elect_one)
+        const uint32_t leader = elect_one();
+        const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_s, 0);
+        const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, false, false);
+        const uint32_t hi = smem_desc_hi(8u * p.kc, layout_type_for(p.kc));
+        const uint32_t b_sub16 = b_sub >> 4, b_ring_lo = b_region >> 4;
+        const uint32_t kc16 = (uint32_t)p.kc >> 4, row16 = (uint32_t)(pl.pw * p.kc) >> 4;  // one pixel / one patch row
+        const int k_steps = p.kc / 32, kdim = pl.kdim, chunks = pl.chunks, num_a = pl.num_a, num_b = pl.num_b;
+        const bool resident = pl.b_resident != 0;
+        int ia = 0, ib = 0, acc = 0;
+        uint32_t pha = 0, phb = 0, acc_phase = 0;
+        bool ok = true;
+        if (resident) ok = __all_sync(0xffffffffu, wait_bar(b_full(0), 0, ctx));
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            if (!(ok = __all_sync(0xffffffffu, wait_bar(tempty_bar(acc), acc_phase ^ 1u, ctx)))) break;
+            ptx::tc_fence_after();
+            uint32_t d0 = tmem_base + acc * buf_stride, d1 = nacc == 2 ? d0 + acc_stride : d0;
+            const bool two_acc = nacc == 2;
+            uint32_t b_res_lo = b_ring_lo;  // resident weights: walks (chunk, tap) sub-tiles in order
+            uint32_t parity = 0;            // index of the next MMA of this tile, modulo 2 (generic path)
+            bool fresh0 = true, fresh1 = two_acc;
+            for (int c = 0; c < chunks && ok; ++c) {
+                if (!(ok = __all_sync(0xffffffffu, wait_bar(a_full(ia), pha, ctx)))) break;
                 ptx::tc_fence_after();
-                uint32_t d0 = tmem_base + acc * buf_stride, d1 = nacc == 2 ? d0 + acc_stride : d0;
-                const bool two_acc = nacc == 2;
-                uint32_t b_res_lo = b_ring_lo;  // resident weights: walks (chunk, tap) sub-tiles in order
-                uint32_t parity = 0;            // index of the next MMA of this tile, modulo 2 (generic path)
-                bool fresh0 = true, fresh1 = two_acc;
-                for (int c = 0; c < chunks && ok; ++c) {
-                    if (!(ok = wait_bar(a_full(ia), pha, ctx))) break;
-                    ptx::tc_fence_after();
-                    uint32_t a_row = (smem_base + ia * pl.a_bytes) >> 4;
-                    if (resident && kdim == 3) {
-                        // common case, fully unrolled: 9 taps x k_steps MMAs
-                        if (k_steps == 4) mma_patch_chunk<3, 4>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc);
-                        else if (k_steps == 2) mma_patch_chunk<3, 2>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc);
-                        else {
-                            mma_patch_chunk<3, 1>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc);
-                            const uint32_t t = d0; d0 = d1; d1 = t;  // 9 MMAs: the next chunk starts on the other accumulator
-                        }
-                        b_res_lo += 9 * b_sub16;
-                    } else {
-                        // tap (a, b) reads the patch tile (a * pw + b) rows further
-                        for (int a = 0; a < kdim && ok; ++a, a_row += row16) {
-                            uint32_t a_tap = a_row;
-                            for (int b = 0; b < kdim; ++b, a_tap += kc16) {
-                                uint32_t b_lo;
-                                if (resident) {
-                                    b_lo = b_res_lo;
-                                    b_res_lo += b_sub16;
-                                } else {
-                                    if (!(ok = wait_bar(b_full(ib), phb, ctx))) break;
-                                    ptx::tc_fence_after();
-                                    b_lo = b_ring_lo + ib * b_sub16;
-                                }
-                                if (k_steps == 4) mma_k_steps<4>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1);
-                                else if (k_steps == 2) mma_k_steps<2>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1);
-                                else mma_k_steps<1>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1);
-                                if (k_steps == 1) {
-                                    // one MMA per tap: it went to accumulator `parity`; for a single accumulator d0 == d1
-                                    if (parity == 0) fresh0 = false; else fresh1 = false;
-                                    parity ^= 1u;
-                                } else {
-                                    fresh0 = false;
-                                    fresh1 = false;
-                                }
-                                if (!resident) {
-                                    ptx::mma_commit(b_empty(ib));
-                                    if (++ib == num_b) { ib = 0; phb ^= 1u; }
-                                }
+                uint32_t a_row = (smem_base + ia * pl.a_bytes) >> 4;
+                if (resident && kdim == 3) {
+                    // common case, fully unrolled: 9 taps x k_steps MMAs
+                    if (k_steps == 4) mma_patch_chunk<3, 4>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc, leader);
+                    else if (k_steps == 2) mma_patch_chunk<3, 2>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc, leader);
+                    else {
+                        mma_patch_chunk<3, 1>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc, leader);
+                        const uint32_t t = d0; d0 = d1; d1 = t;  // 9 MMAs: the next chunk starts on the other accumulator
+                    }
+                    b_res_lo += 9 * b_sub16;
+                } else {
+                    // tap (a, b) reads the patch tile (a * pw + b) rows further
+                    for (int a = 0; a < kdim && ok; ++a, a_row += row16) {
+                        uint32_t a_tap = a_row;
+                        for (int b = 0; b < kdim; ++b, a_tap += kc16) {
+                            uint32_t b_lo;
+                            if (resident) {
+                                b_lo = b_res_lo;
+                                b_res_lo += b_sub16;
+                            } else {
+                                if (!(ok = __all_sync(0xffffffffu, wait_bar(b_full(ib), phb, ctx)))) break;
+                                ptx::tc_fence_after();
+                                b_lo = b_ring_lo + ib * b_sub16;
+                            }
+                            if (k_steps == 4) mma_k_steps<4>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1, leader);
+                            else if (k_steps == 2) mma_k_steps<2>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1, leader);
+                            else mma_k_steps<1>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1, leader);
+                            if (k_steps == 1) {
+                                // one MMA per tap: it went to accumulator `parity`; for a single accumulator d0 == d1
+                                if (parity == 0) fresh0 = false; else fresh1 = false;
+                                parity ^= 1u;
+                            } else {
+                                fresh0 = false;
+                                fresh1 = false;
+                            }
+                            if (!resident) {
+                                ptx::mma_commit(b_empty(ib), leader);
+                                if (++ib == num_b) { ib = 0; phb ^= 1u; }
                             }
                         }
                     }
-                    ptx::mma_commit(a_empty(ia));
-                    if (++ia == num_a) { ia = 0; pha ^= 1u; }
                 }
-                if (ok) ptx::mma_commit(tfull_bar(acc));
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                ptx::mma_commit(a_empty(ia), leader);
+                if (++ia == num_a) { ia = 0; pha ^= 1u; }
             }
-            if (!ok) {
-                ptx::mma_commit(drain_bar);
+            if (ok) ptx::mma_commit(tfull_bar(acc), leader);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (!ok) {
+            ptx::mma_commit(drain_bar, leader);
+            for (uint32_t i = 0; i < kSpinLimit; ++i)
+                if (ptx::mbar_try_wait(drain_bar, 0)) break;
+            if (pl.b_resident)
                 for (uint32_t i = 0; i < kSpinLimit; ++i)
-                    if (ptx::mbar_try_wait(drain_bar, 0)) break;
-                if (pl.b_resident)
-                    for (uint32_t i = 0; i < kSpinLimit; ++i)
-                        if (ptx::mbar_try_wait(b_full(0), 0)) break;
-            }
+                    if (ptx::mbar_try_wait(b_full(0), 0)) break;
         }
     } else if (warp >= 4) {
         // ---------------------------------------------------------------------- epilogue

@@ -51,7 +51,7 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile uint32_t abort_s;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     const int px = p.pixels_per_stage;
     const uint32_t a_sub = (uint32_t)px * p.kc, b_sub = (uint32_t)px * p.nc;
@@ -151,39 +151,40 @@ wgrad_kernel(const __grid_constant__ WgradParams p, const __grid_constant__ CUte
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, true, true);
-            // descriptor halves that do not change; the loop adds row offsets to the low halves
-            const uint64_t a_proto = mn_major_desc(0, p.kc, a_sub), b_proto = mn_major_desc(0, p.nc, b_sub);
-            const uint32_t a_hi = (uint32_t)(a_proto >> 32), b_hi = (uint32_t)(b_proto >> 32);
-            const uint32_t a_lead = (uint32_t)a_proto, b_lead = (uint32_t)b_proto;  // leading-offset field, address 0
-            const uint32_t a_step16 = (32u * p.kc) >> 4, b_step16 = (32u * p.nc) >> 4;  // 32 pixels further down
-            const uint32_t a_mtile16 = a_mtile >> 4;
-            int stage = 0;
-            uint32_t phase = 0, accumulate = 0;
-            bool ok = true;
-            for (int it = 0; it < my_stages; ++it) {
-                if (!(ok = wait_bar(full_bar(stage), phase, ctx))) break;
-                ptx::tc_fence_after();
-                uint32_t a_lo = ((smem_base + stage * stage_bytes) >> 4) | a_lead;
-                uint32_t b_lo = (((smem_base + stage * stage_bytes) >> 4) + ((p.mtiles_per_cta * a_mtile) >> 4)) | b_lead;
-                for (int k = 0; k < px; k += 32) {
-                    // the M tiles of the group meet the same error tile; each has its own accumulator columns
-                    uint32_t a_j = a_lo, d_j = tmem_base;
-                    for (int jm = 0; jm < my_mtiles; ++jm, a_j += a_mtile16, d_j += p.tile_n)
-                        ptx::mma_i8(d_j, smem_desc_join(a_j, a_hi), smem_desc_join(b_lo, b_hi), idesc, accumulate);
-                    accumulate = 1;
-                    a_lo += a_step16;
-                    b_lo += b_step16;
-                }
-                ptx::mma_commit(empty_bar(stage));
-                if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }
+        // the whole warp runs the issue loop; one elected lane issues the MMAs and commits (see elect_one)
+        const uint32_t leader = elect_one();
+        const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_s, 0);
+        const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, true, true);
+        // descriptor halves that do not change; the loop adds row offsets to the low halves
+        const uint64_t a_proto = mn_major_desc(0, p.kc, a_sub), b_proto = mn_major_desc(0, p.nc, b_sub);
+        const uint32_t a_hi = (uint32_t)(a_proto >> 32), b_hi = (uint32_t)(b_proto >> 32);
+        const uint32_t a_lead = (uint32_t)a_proto, b_lead = (uint32_t)b_proto;  // leading-offset field, address 0
+        const uint32_t a_step16 = (32u * p.kc) >> 4, b_step16 = (32u * p.nc) >> 4;  // 32 pixels further down
+        const uint32_t a_mtile16 = a_mtile >> 4;
+        int stage = 0;
+        uint32_t phase = 0, accumulate = 0;
+        bool ok = true;
+        for (int it = 0; it < my_stages; ++it) {
+            if (!(ok = __all_sync(0xffffffffu, wait_bar(full_bar(stage), phase, ctx)))) break;
+            ptx::tc_fence_after();
+            uint32_t a_lo = ((smem_base + stage * stage_bytes) >> 4) | a_lead;
+            uint32_t b_lo = (((smem_base + stage * stage_bytes) >> 4) + ((p.mtiles_per_cta * a_mtile) >> 4)) | b_lead;
+            for (int k = 0; k < px; k += 32) {
+                // the M tiles of the group meet the same error tile; each has its own accumulator columns
+                uint32_t a_j = a_lo, d_j = tmem_base;
+                for (int jm = 0; jm < my_mtiles; ++jm, a_j += a_mtile16, d_j += p.tile_n)
+                    ptx::mma_i8(d_j, smem_desc_join(a_j, a_hi), smem_desc_join(b_lo, b_hi), idesc, accumulate, leader);
+                accumulate = 1;
+                a_lo += a_step16;
+                b_lo += b_step16;
             }
-            ptx::mma_commit(done_bar);
-            if (!ok)
-                for (uint32_t i = 0; i < kSpinLimit; ++i)
-                    if (ptx::mbar_try_wait(done_bar, 0)) break;
+            ptx::mma_commit(empty_bar(stage), leader);
+            if (++stage == p.num_stages) { stage = 0; phase ^= 1u; }
         }
+        ptx::mma_commit(done_bar, leader);
+        if (!ok)
+            for (uint32_t i = 0; i < kSpinLimit; ++i)
+                if (ptx::mbar_try_wait(done_bar, 0)) break;
     } else {
         const int quad = warp & 3;
         bool ok = __all_sync(0xffffffffu, wait_bar(done_bar, 0, ctx));

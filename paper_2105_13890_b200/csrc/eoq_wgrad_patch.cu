@@ -35,7 +35,7 @@ wgrad_patch_kernel(const __grid_constant__ WgradPatchPlan pl, const __grid_const
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile uint32_t abort_s;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t stage_bytes = (uint32_t)(pl.x_bytes + pl.e_bytes);
     const uint32_t bar0 = ptx::smem_u32(bars);
@@ -114,48 +114,49 @@ wgrad_patch_kernel(const __grid_constant__ WgradPatchPlan pl, const __grid_const
                             if (ptx::mbar_try_wait(full_bar(s), (inflight_parity >> s) & 1u)) break;
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_i8(kTileM, pl.tile_n, true, true);
-            // MN-major descriptors: activation atoms (taps) are one pixel (kc bytes) apart; 8-pixel groups 8 rows apart
-            const uint32_t a_hi = smem_desc_hi(8u * pl.kc, layout_type_for(pl.kc));
-            const uint32_t b_hi = smem_desc_hi(8u * pl.tile_n, layout_type_for(pl.tile_n));
-            const uint32_t a_lead = ((uint32_t)pl.kc >> 4) << 16;
-            const uint32_t a_step16 = (32u * pl.kc) >> 4, b_step16 = (32u * pl.tile_n) >> 4;  // 32 pixels further
-            const uint32_t kc16 = (uint32_t)pl.kc >> 4, row16 = (uint32_t)(pl.pw * pl.kc) >> 4;
-            // start offset of each accumulator's first tap inside the activation patch (16-byte units)
-            uint32_t acc_off[kMaxAcc];
+        // the whole warp runs the issue loop; one elected lane issues the MMAs and commits (see elect_one)
+        const uint32_t leader = elect_one();
+        const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_s, 0);
+        const uint32_t idesc = make_idesc_i8(kTileM, pl.tile_n, true, true);
+        // MN-major descriptors: activation atoms (taps) are one pixel (kc bytes) apart; 8-pixel groups 8 rows apart
+        const uint32_t a_hi = smem_desc_hi(8u * pl.kc, layout_type_for(pl.kc));
+        const uint32_t b_hi = smem_desc_hi(8u * pl.tile_n, layout_type_for(pl.tile_n));
+        const uint32_t a_lead = ((uint32_t)pl.kc >> 4) << 16;
+        const uint32_t a_step16 = (32u * pl.kc) >> 4, b_step16 = (32u * pl.tile_n) >> 4;  // 32 pixels further
+        const uint32_t kc16 = (uint32_t)pl.kc >> 4, row16 = (uint32_t)(pl.pw * pl.kc) >> 4;
+        // start offset of each accumulator's first tap inside the activation patch (16-byte units)
+        uint32_t acc_off[kMaxAcc];
 #pragma unroll
-            for (int j = 0; j < kMaxAcc; ++j) {
-                const int a = row0 + j / pl.accs_per_row, b0 = (j % pl.accs_per_row) * pl.apa;
-                acc_off[j] = (uint32_t)a * row16 + (uint32_t)b0 * kc16;
-            }
-            const int k_steps = pl.kp / 32;
-            int stage = 0;
-            uint32_t phase = 0, accumulate = 0;
-            bool ok = true;
-            for (int it = 0; it < my_blocks; ++it) {
-                if (!(ok = wait_bar(full_bar(stage), phase, ctx))) break;
-                ptx::tc_fence_after();
-                uint32_t a_lo = ((smem_base + stage * stage_bytes) >> 4) | a_lead;
-                uint32_t b_lo = (smem_base + stage * stage_bytes + pl.x_bytes) >> 4;
-                for (int k = 0; k < k_steps; ++k) {
-#pragma unroll
-                    for (int j = 0; j < kMaxAcc; ++j)
-                        if (j < num_acc)
-                            ptx::mma_i8(tmem_base + j * pl.tile_n, smem_desc_join(a_lo + acc_off[j], a_hi),
-                                        smem_desc_join(b_lo, b_hi), idesc, accumulate);
-                    accumulate = 1;
-                    a_lo += a_step16;
-                    b_lo += b_step16;
-                }
-                ptx::mma_commit(empty_bar(stage));
-                if (++stage == pl.num_stages) { stage = 0; phase ^= 1u; }
-            }
-            ptx::mma_commit(done_bar);
-            if (!ok)
-                for (uint32_t i = 0; i < kSpinLimit; ++i)
-                    if (ptx::mbar_try_wait(done_bar, 0)) break;
+        for (int j = 0; j < kMaxAcc; ++j) {
+            const int a = row0 + j / pl.accs_per_row, b0 = (j % pl.accs_per_row) * pl.apa;
+            acc_off[j] = (uint32_t)a * row16 + (uint32_t)b0 * kc16;
         }
+        const int k_steps = pl.kp / 32;
+        int stage = 0;
+        uint32_t phase = 0, accumulate = 0;
+        bool ok = true;
+        for (int it = 0; it < my_blocks; ++it) {
+            if (!(ok = __all_sync(0xffffffffu, wait_bar(full_bar(stage), phase, ctx)))) break;
+            ptx::tc_fence_after();
+            uint32_t a_lo = ((smem_base + stage * stage_bytes) >> 4) | a_lead;
+            uint32_t b_lo = (smem_base + stage * stage_bytes + pl.x_bytes) >> 4;
+            for (int k = 0; k < k_steps; ++k) {
+#pragma unroll
+                for (int j = 0; j < kMaxAcc; ++j)
+                    if (j < num_acc)
+                        ptx::mma_i8(tmem_base + j * pl.tile_n, smem_desc_join(a_lo + acc_off[j], a_hi),
+                                    smem_desc_join(b_lo, b_hi), idesc, accumulate, leader);
+                accumulate = 1;
+                a_lo += a_step16;
+                b_lo += b_step16;
+            }
+            ptx::mma_commit(empty_bar(stage), leader);
+            if (++stage == pl.num_stages) { stage = 0; phase ^= 1u; }
+        }
+        ptx::mma_commit(done_bar, leader);
+        if (!ok)
+            for (uint32_t i = 0; i < kSpinLimit; ++i)
+                if (ptx::mbar_try_wait(done_bar, 0)) break;
     } else {
         const int quad = warp & 3;
         const int r = quad * 32 + lane;  // accumulator row: (tap within the accumulator, channel of the chunk)

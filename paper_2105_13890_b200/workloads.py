@@ -111,16 +111,26 @@ def _basic_stage(layers, name, n, h, c_in, c_out, blocks, stride):
 STEM_CHANNELS = 8
 
 
-def resnet18(batch: int = 64, image: int = 224) -> Workload:
+def _imagenet_basic(name: str, blocks, batch: int, image: int) -> Workload:
+    """ImageNet-shaped ResNet of basic blocks: 7x7 stride-2 first layer, 3x3 stride-2 max-pool, four stages."""
     layers: List[Layer] = []
     layers.append(Layer("stem", batch, image, image, STEM_CHANNELS, 64, 7, 2, 3, 3, in_branch=False, has_dgrad=False))
     h = (image + 6 - 7) // 2 + 1
     h = (h + 2 - 3) // 2 + 1  # 3x3 stride-2 max-pool
     c = 64
     for i, (co, s) in enumerate(((64, 1), (128, 2), (256, 2), (512, 2))):
-        h = _basic_stage(layers, f"layer{i + 1}", batch, h, c, co, 2, s)
+        h = _basic_stage(layers, f"layer{i + 1}", batch, h, c, co, blocks[i], s)
         c = co
-    return Workload(f"fixup_resnet18_b{batch}_{image}", batch, layers, L=8, m=2)
+    return Workload(f"fixup_{name}_b{batch}_{image}", batch, layers, L=sum(blocks), m=2)
+
+
+def resnet18(batch: int = 64, image: int = 224) -> Workload:
+    return _imagenet_basic("resnet18", (2, 2, 2, 2), batch, image)
+
+
+def resnet34(batch: int = 64, image: int = 224) -> Workload:
+    """ResNet-34, the second ImageNet network of Sec. 5.1: basic blocks [3, 4, 6, 3], L = 16."""
+    return _imagenet_basic("resnet34", (3, 4, 6, 3), batch, image)
 
 
 def resnet20(batch: int = 128, image: int = 32) -> Workload:
@@ -131,6 +141,18 @@ def resnet20(batch: int = 128, image: int = 32) -> Workload:
         h = _basic_stage(layers, f"stage{i + 1}", batch, h, c, co, 3, s)
         c = co
     return Workload(f"fixup_resnet20_b{batch}_{image}", batch, layers, L=9, m=2)
+
+
+def resnet110(batch: int = 128, image: int = 32) -> Workload:
+    """ResNet-110 on CIFAR-shaped input, the network of the small-batch experiment (Sec. 5.4): three stages of
+    18 basic blocks with 16 / 32 / 64 channels, L = 54."""
+    layers: List[Layer] = []
+    layers.append(Layer("stem", batch, image, image, _pad16(3), 16, 3, 1, 1, 3, in_branch=False, has_dgrad=False))
+    h, c = image, 16
+    for i, (co, s) in enumerate(((16, 1), (32, 2), (64, 2))):
+        h = _basic_stage(layers, f"stage{i + 1}", batch, h, c, co, 18, s)
+        c = co
+    return Workload(f"fixup_resnet110_b{batch}_{image}", batch, layers, L=54, m=2)
 
 
 def resnet50(batch: int = 32, image: int = 224) -> Workload:
@@ -172,7 +194,8 @@ def layer64(batch: int = 512) -> Workload:
 
 
 def get(name: str, batch: int | None = None) -> Workload:
-    table = {"single": single_layer, "layer64": layer64, "resnet20": resnet20, "resnet18": resnet18, "resnet50": resnet50}
+    table = {"single": single_layer, "layer64": layer64, "resnet20": resnet20, "resnet18": resnet18, "resnet34": resnet34,
+             "resnet50": resnet50, "resnet110": resnet110}
     fn = table[name]
     if name == "single" or batch is None:
         return fn()

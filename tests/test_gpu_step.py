@@ -59,3 +59,74 @@ def test_first_layer_of_a_step_matches_the_oracle():
     want, _, _ = oracle.update(w_before.cpu().numpy(), bwd["g_w"], bwd["p_gw"], st.lr_mant, st.lr_exp, stochastic=True,
                                seed=synth.BASE_SEED, step=0, tensor_id=1)
     assert np.array_equal(lb.w.cpu().numpy().astype(np.int32), want)
+
+
+def _host_inputs(st, wl):
+    """The step's inputs regenerated on the host from the seeded streams (what TrainStep uploaded), with the
+    weights quantized by the oracle."""
+    seed = synth.BASE_SEED
+    out = []
+    pools = {}
+
+    def pooled(kind, shape, stream):
+        # TrainStep draws one tensor per (kind, shape) and reuses it for every buffer of that kind and shape
+        if (kind, shape) not in pools:
+            pools[(kind, shape)] = (synth.relu_codes if kind == "relu" else synth.normal_codes)(shape, seed, stream)
+        return pools[(kind, shape)]
+
+    for i, l in enumerate(wl.layers):
+        x0 = None if i == 0 else pooled("relu", (l.n, l.h, l.w, l.c_in), 1)
+        e0 = pooled("err", (l.n, l.ho, l.wo, l.c_out), 2)
+        sc = pooled("relu", (l.n, l.ho, l.wo, l.c_out), 3) if l.shortcut else None
+        wf = workloads.init_weight_f32(l, wl, synth.normal_f64((l.c_out, l.k, l.k, l.c_in), seed, 100 + i))
+        out.append((x0, e0, sc, oracle.q_w(wf)))
+    return out
+
+
+@pytest.mark.parametrize("name,batch", [("resnet20", 2), ("resnet110", 1), ("resnet18", 1), ("resnet34", 1), ("resnet50", 1)])
+def test_every_layer_of_a_step_matches_the_oracle(name, batch):
+    """One whole step of each network at a small batch: every layer's activation, error, weight gradient
+    (codes and exponents), reduction sums and updated weights against the oracle, which is fed the same seeded
+    inputs generated on the host."""
+    wl = workloads.get(name, batch)
+    st = TrainStep(wl, eoq.eoq_create(0), scalars=Scalars())
+    host = _host_inputs(st, wl)
+    for lb, (_, _, _, wq) in zip(st.layers, host):
+        assert np.array_equal(lb.w.cpu().numpy(), wq), lb.layer.name   # Q_w at initialisation
+    st.run()
+    torch.cuda.synchronize()
+    assert st.status() & eoq.EOQ_DEV_TIMEOUT == 0
+    sc = st.sc
+    for i, (lb, (x0, e0, short, wq)) in enumerate(zip(st.layers, host)):
+        l = lb.layer
+        d = ConvDesc(l.n, l.h, l.w, l.c_in, l.c_out, l.k, l.k, l.stride, l.pad)
+        gamma = sc.gamma_c if l.gamma_trainable else 128
+        b1 = 0 if i == 0 else sc.b1_c
+        x_exp = -7
+        if i == 0:
+            # the network input: SQ of the fp32 image padded to the stored channel count
+            img = st.host_image(synth.BASE_SEED)
+            padded = np.zeros(img.shape[:3] + (l.c_in,), dtype=np.float32)
+            padded[..., :img.shape[3]] = img
+            codes, x_exp, _ = oracle.quantize_f32(oracle.MODE_SQ, padded)
+            x0 = codes.astype(np.int8)
+            m = lb.wmargin
+            stored = lb.x0.cpu().numpy()
+            assert np.array_equal(stored[:, :, m:m + l.w, :], x0) and st.image_exp.item() == x_exp
+        fwd = oracle.layer_forward(d, x0, b1, wq, gamma, sc.b2_c if l.relu else 0, short, l.relu, x_exp=x_exp)
+        assert np.array_equal(lb.x5.cpu().numpy(), fwd["x5"]), (l.name, "x5")
+        if lb.x2 is not None:
+            assert np.array_equal(lb.x2.cpu().numpy().astype(np.int32), fwd["x2"]), (l.name, "x2")
+        bwd = oracle.layer_backward(d, e0, -12, fwd["mask"] if l.relu else np.ones_like(fwd["mask"]),
+                                    fwd["x2"] if lb.x2 is not None else None, x0, b1, wq, gamma)
+        assert np.array_equal(lb.e3.cpu().numpy(), bwd["e3"]) and lb.e3_exp.item() == bwd["p3"], (l.name, "e3")
+        assert lb.sum_e1.item() == bwd["sum_e1"], (l.name, "sum_e1")
+        if lb.x2 is not None:
+            assert lb.sum_e1x2.item() == bwd["sum_e1x2"], (l.name, "sum_e1x2")
+        if l.has_dgrad:
+            assert np.array_equal(lb.e4.cpu().numpy(), bwd["e4"]) and lb.e4_exp.item() == bwd["p4"], (l.name, "e4")
+            assert lb.sum_e4.item() == bwd["sum_e4"], (l.name, "sum_e4")
+        assert np.array_equal(lb.g.cpu().numpy(), bwd["g_w"]) and lb.g_exp.item() == bwd["p_gw"], (l.name, "g_w")
+        want, _, _ = oracle.update(wq, bwd["g_w"], bwd["p_gw"], st.lr_mant, st.lr_exp, stochastic=True,
+                                   seed=synth.BASE_SEED, step=0, tensor_id=i)
+        assert np.array_equal(lb.w.cpu().numpy().astype(np.int32), want), (l.name, "w")

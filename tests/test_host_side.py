@@ -56,6 +56,12 @@ def test_workload_op_counts_and_fixup_coefficient():
     assert r20.total_macs == pytest.approx(15.6e9, rel=2e-3) and len(r20.layers) == 21
     assert r50.total_macs == pytest.approx(388.6e9, rel=1e-3) and len(r50.layers) == 53
     assert sum(l.weight_elems for l in r18.layers) == pytest.approx(11.2e6, rel=2e-3)
+    # the paper's other two networks (Sec. 5.1, 5.4): 3.66 and 0.253 GMAC per image forward
+    r34, r110 = workloads.resnet34(), workloads.resnet110()
+    assert len(r34.layers) == 36 and r34.L == 16 and len(r110.layers) == 111 and r110.L == 54
+    assert sum(l.macs for l in r34.layers) / r34.batch == pytest.approx(3.663e9, rel=1e-3)
+    assert sum(l.macs for l in r110.layers) / r110.batch == pytest.approx(0.2531e9, rel=1e-3)
+    assert workloads.get("resnet110", 4).batch == 4 and workloads.get("resnet34", 2).layers[0].k == 7
     for L, m in ((8, 2), (9, 2), (16, 3), (54, 2)):
         assert workloads.fixup_alpha(L, m) == pytest.approx(oracle.fixup_alpha(L, m), rel=1e-15)
     layer = r18.layers[1]
