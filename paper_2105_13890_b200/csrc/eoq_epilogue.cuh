@@ -62,18 +62,40 @@ __device__ __forceinline__ int32_t sbyte(uint32_t w)
 // The integer pipe bounds this code, so clamps are moved in front of the roundings (both are monotonic, the
 // clamp limits are chosen so that the rounded result is unchanged), roundings run as one FMA each, and the
 // constant offsets of that trick are folded into the multiply-add that forms x4.
+// Global operands of the forward chain for 16 channels of one pixel (b1 table row, shortcut codes).  They do not
+// depend on the accumulator, so the epilogue requests them before it waits for the tile's MMAs: their latency
+// is then hidden behind that wait instead of being added to every tile.
+struct ForwardOperands {
+    int4 table[4];
+    int4 shortcut;
+};
+
+__device__ __forceinline__ ForwardOperands forward_operands(const IgemmParams &p, bool active, size_t off, int col, int cls)
+{
+    ForwardOperands o;
+    if (active && p.b1_table) {
+        const int4 *t = reinterpret_cast<const int4 *>(p.b1_table + (size_t)cls * p.N + col);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o.table[i] = __ldg(t + i);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o.table[i] = make_int4(0, 0, 0, 0);
+    }
+    o.shortcut = (active && p.shortcut) ? __ldg(reinterpret_cast<const int4 *>(p.shortcut + off)) : make_int4(0, 0, 0, 0);
+    return o;
+}
+
 template <bool kShift7>
-__device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t *acc, size_t off, int col, int cls,
+__device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t *acc, size_t off, const ForwardOperands &ops,
                                            int shift)
 {
     int32_t a[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) a[i] = (int32_t)acc[i];
     if (p.b1_table) {
-        const int4 *t = reinterpret_cast<const int4 *>(p.b1_table + (size_t)cls * p.N + col);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const int4 v = __ldg(t + i);
+            const int4 v = ops.table[i];
             a[4 * i + 0] += p.b1_c * v.x;
             a[4 * i + 1] += p.b1_c * v.y;
             a[4 * i + 2] += p.b1_c * v.z;
@@ -117,7 +139,7 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t 
     const uint32_t base = ((uint32_t)p.b2_c << 7) - g * q_bias;
     uint32_t add[16];
     if (p.shortcut) {
-        const int4 v = __ldg(reinterpret_cast<const int4 *>(p.shortcut + off));
+        const int4 v = ops.shortcut;
         const uint32_t w[4] = {(uint32_t)v.x, (uint32_t)v.y, (uint32_t)v.z, (uint32_t)v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {

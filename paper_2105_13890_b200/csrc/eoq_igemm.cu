@@ -53,7 +53,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(tfull_bar(a), 1);
-            ptx::mbar_init(tempty_bar(a), kEpilogueWarps);
+            ptx::mbar_init(tempty_bar(a), kEpilogueWarps / 2);
         }
         ptx::mbar_init(drain_bar, 1);
         abort_s = 0;
@@ -189,29 +189,30 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         }
     } else {
         // ---------------------------------------------------------------------- epilogue
-        // Four warps per scheduler: a warp may read the TMEM lanes of quadrant (warp % 4); the warps
-        // of a quadrant split the tile's columns.
+        // A warp may read the TMEM lanes of quadrant (warp % 4).  The four warps of a quadrant form two pairs;
+        // pair `grp` serves every second tile of this CTA (accumulator buffer `grp`), the two warps of a pair
+        // split the tile's columns, so that two tiles are in the epilogue at the same time.  Everything that does
+        // not depend on the sums is formed before the wait for the tile's MMAs.
         const int quad = warp & 3;
-        const int part = (warp - 4) >> 2;  // the kEpilogueWarps / 4 warps of a lane quadrant split the columns
+        const int ew = (warp - 4) >> 2;
+        const int grp = ew & 1, part = ew >> 1;
         const int row = quad * 32 + lane;
         const int groups = p.tile_n / 16;                 // 16-column groups of the tile
-        constexpr int kParts = kEpilogueWarps / 4;
+        constexpr int kParts = kEpilogueWarps / 8;
         const int g_begin = (groups * part) / kParts, g_end = (groups * (part + 1)) / kParts;
+        const bool fwd = p.epilogue == kEpiForward;
         int shift = 7;
-        if (p.epilogue == kEpiForward && p.x_exp) {
+        if (fwd && p.x_exp) {
             shift = -__ldg(p.x_exp);
             if (shift > 31 || shift < -16) {
                 if (lane == 0) atomicOr(&p.dev->status, EOQ_DEV_RANGE);
                 shift = max(-16, min(31, shift));
             }
         }
-        int acc = 0;
         uint32_t acc_phase = 0, mx = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        for (int tile = blockIdx.x + grp * gridDim.x; tile < num_tiles && ok; tile += 2 * gridDim.x) {
             const int mt = tile / p.num_n_tiles, nt = tile % p.num_n_tiles;
-            if (!(ok = __all_sync(0xffffffffu, wait_bar(tfull_bar(acc), acc_phase, ctx)))) break;  // warp-uniform
-            ptx::tc_fence_after();
             const int m = mt * kTileM + row;
             const bool valid = m < p.M;
             size_t pix = 0;
@@ -224,34 +225,39 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                     cls = border_class(y, p.hq, p.b1_nlo_h, p.b1_nhi_h, p.b1_nrc) * p.b1_ncc +
                           border_class(x, p.wq, p.b1_nlo_w, p.b1_nhi_w, p.b1_ncc);
             }
-            const uint32_t t_row = tmem_base + acc * buf_stride + ((uint32_t)(quad * 32) << 16);
-            for (int g = g_begin; g < g_end; ++g) {
+            int col = nt * p.tile_n + g_begin * 16;
+            size_t off = pix * p.N + col;
+            ForwardOperands ops = forward_operands(p, fwd && valid && col < p.N, off, col, cls);
+            if (!(ok = __all_sync(0xffffffffu, wait_bar(tfull_bar(grp), acc_phase, ctx)))) break;  // warp-uniform
+            ptx::tc_fence_after();
+            const uint32_t t_row = tmem_base + grp * buf_stride + ((uint32_t)(quad * 32) << 16);
+            for (int g = g_begin; g < g_end; ++g, col += 16, off += 16) {
                 uint32_t r[32];
                 ptx::tmem_ld_32x16(t_row + g * 16, r);
+                uint32_t r2[32];
+                if (nacc == 2) ptx::tmem_ld_32x16(t_row + acc_stride + g * 16, r2);
+                // the next group's operands travel while this group is computed
+                ForwardOperands next = ops;
+                if (g + 1 < g_end) next = forward_operands(p, fwd && valid && col + 16 < p.N, off + 16, col + 16, cls);
+                ptx::tmem_ld_wait();
                 if (nacc == 2) {
-                    uint32_t r2[32];
-                    ptx::tmem_ld_32x16(t_row + acc_stride + g * 16, r2);
-                    ptx::tmem_ld_wait();
 #pragma unroll
                     for (int i = 0; i < 16; ++i) r[i] += r2[i];  // the two partial accumulators of the tile
-                } else {
-                    ptx::tmem_ld_wait();
                 }
-                const int col = nt * p.tile_n + g * 16;
                 if (valid && col < p.N) {
-                    const size_t off = pix * p.N + col;
-                    if (p.epilogue == kEpiForward) {
-                        if (shift == 7) forward_16<true>(p, r, off, col, cls, shift);
-                        else forward_16<false>(p, r, off, col, cls, shift);
+                    if (fwd) {
+                        if (shift == 7) forward_16<true>(p, r, off, ops, shift);
+                        else forward_16<false>(p, r, off, ops, shift);
                     } else {
                         mx = max(mx, dgrad_16(p, r, off));
                     }
                 }
+                ops = next;
             }
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
-            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            if (lane == 0) ptx::mbar_arrive(tempty_bar(grp));
+            acc_phase ^= 1u;
         }
         if (p.epilogue == kEpiDgrad) {
             mx = warp_max_u32(mx);

@@ -11,8 +11,9 @@
 // dropped.  Weights either stay resident in shared memory for the whole kernel (when the layer's weights fit) or
 // stream through their own ring.
 //
-// Roles: warp 0 patch loads, warp 1 TMEM owner + tcgen05.mma issuer, warp 2 weight loads, warps 4-11 epilogue
-// (two per scheduler, the two warps of a TMEM lane quadrant split the columns).  All waits are bounded.
+// Roles: warp 0 patch loads, warp 1 TMEM owner + tcgen05.mma issuer, warp 2 weight loads, warps 4-19 epilogue
+// (four per TMEM lane quadrant: two pairs that take alternate tiles, the warps of a pair split the columns).
+// All waits are bounded.
 #include "eoq_device.cuh"
 #include "eoq_epilogue.cuh"
 #include "eoq_internal.h"
@@ -64,7 +65,7 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(tfull_bar(a), 1);
-            ptx::mbar_init(tempty_bar(a), kEpilogueWarps);
+            ptx::mbar_init(tempty_bar(a), kEpilogueWarps / 2);
         }
         ptx::mbar_init(drain_bar, 1);
         abort_s = 0;
@@ -225,20 +226,24 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
         }
     } else if (warp >= 4) {
         // ---------------------------------------------------------------------- epilogue
+        // The four warps of a TMEM lane quadrant form two pairs; pair `grp` serves every second tile of this CTA
+        // (the tiles whose sums sit in accumulator buffer `grp`), and the two warps of a pair split the columns.
+        // Two tiles are therefore in the epilogue at the same time: while one pair waits for tensor-memory loads
+        // or stores, the other has arithmetic to issue.  Everything that does not depend on the sums (pixel
+        // index, border class, b1 table row, shortcut codes) is formed before the wait for the tile's MMAs.
         const int quad = warp & 3;
-        const int part = (warp - 4) >> 2;  // the kEpilogueWarps / 4 warps of a lane quadrant split the columns
+        const int ew = (warp - 4) >> 2;
+        const int grp = ew & 1, part = ew >> 1;
         const int row = quad * 32 + lane;
         const int groups = p.tile_n / 16;
-        constexpr int kParts = kEpilogueWarps / 4;
+        constexpr int kParts = kEpilogueWarps / 8;
         const int g_begin = (groups * part) / kParts, g_end = (groups * (part + 1)) / kParts;
         const int yl = row / pl.pw, xx = row % pl.pw;  // position of this thread's row in the patch raster
-        int acc = 0;
+        const bool fwd = p.epilogue == kEpiForward;
         uint32_t acc_phase = 0, mx = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        for (int tile = blockIdx.x + grp * gridDim.x; tile < num_tiles && ok; tile += 2 * gridDim.x) {
             const int mt = tile / p.num_n_tiles, nt = tile % p.num_n_tiles;
-            if (!(ok = __all_sync(0xffffffffu, wait_bar<64>(tfull_bar(acc), acc_phase, ctx)))) break;
-            ptx::tc_fence_after();
             const int img = mt / pl.tiles_per_img, y = (mt % pl.tiles_per_img) * pl.r_rows + yl;
             const bool valid = yl < pl.r_rows && xx < p.wq && y < p.hq;
             size_t pix = 0;
@@ -249,30 +254,35 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                     cls = border_class(y, p.hq, p.b1_nlo_h, p.b1_nhi_h, p.b1_nrc) * p.b1_ncc +
                           border_class(xx, p.wq, p.b1_nlo_w, p.b1_nhi_w, p.b1_ncc);
             }
-            const uint32_t t_row = tmem_base + acc * buf_stride + ((uint32_t)(quad * 32) << 16);
-            for (int g = g_begin; g < g_end; ++g) {
+            int col = nt * p.tile_n + g_begin * 16;
+            size_t off = pix * p.N + col;
+            ForwardOperands ops = forward_operands(p, fwd && valid && col < p.N, off, col, cls);
+            if (!(ok = __all_sync(0xffffffffu, wait_bar<64>(tfull_bar(grp), acc_phase, ctx)))) break;
+            ptx::tc_fence_after();
+            const uint32_t t_row = tmem_base + grp * buf_stride + ((uint32_t)(quad * 32) << 16);
+            for (int g = g_begin; g < g_end; ++g, col += 16, off += 16) {
                 uint32_t r[32];
                 ptx::tmem_ld_32x16(t_row + g * 16, r);
+                uint32_t r2[32];
+                if (nacc == 2) ptx::tmem_ld_32x16(t_row + acc_stride + g * 16, r2);
+                // the next group's operands travel while this group is computed
+                ForwardOperands next = ops;
+                if (g + 1 < g_end) next = forward_operands(p, fwd && valid && col + 16 < p.N, off + 16, col + 16, cls);
+                ptx::tmem_ld_wait();
                 if (nacc == 2) {
-                    uint32_t r2[32];
-                    ptx::tmem_ld_32x16(t_row + acc_stride + g * 16, r2);
-                    ptx::tmem_ld_wait();
 #pragma unroll
                     for (int i = 0; i < 16; ++i) r[i] += r2[i];  // the two partial accumulators of the tile
-                } else {
-                    ptx::tmem_ld_wait();
                 }
-                const int col = nt * p.tile_n + g * 16;
                 if (valid && col < p.N) {
-                    const size_t off = pix * p.N + col;
-                    if (p.epilogue == kEpiForward) forward_16<true>(p, r, off, col, cls, 7);
+                    if (fwd) forward_16<true>(p, r, off, ops, 7);
                     else mx = max(mx, dgrad_16(p, r, off));
                 }
+                ops = next;
             }
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
-            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            if (lane == 0) ptx::mbar_arrive(tempty_bar(grp));
+            acc_phase ^= 1u;
         }
         if (p.epilogue == kEpiDgrad) {
             mx = warp_max_u32(mx);
