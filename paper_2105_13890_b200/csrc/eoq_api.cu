@@ -475,6 +475,12 @@ extern "C" int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits
     cudaError_t e = cudaMemcpyAsync(&v, &h->dev->status, sizeof(unsigned), cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaMemsetAsync(&h->dev->status, 0, sizeof(unsigned), s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e == cudaSuccess && (v & EOQ_DEV_TIMEOUT)) {
+        // a kernel that gave up may not have put the reduction cells back to zero
+        e = launch_reset_cells(h->dev, s);
+        if (e == cudaSuccess) e = cudaMemsetAsync(&h->dev->ticket, 0, sizeof(unsigned), s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    }
     *bits = v;
     return record(h, e);
 }
@@ -677,8 +683,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     cudaError_t e;
     {
         ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
-        e = launch_reset_cells(h->dev, s);
-        if (e == cudaSuccess) e = launch_weight_transpose(w, wt, d.c_out, g.taps, d.c_in, s);
+        e = launch_weight_transpose(w, wt, d.c_out, g.taps, d.c_in, s);
     }
     if (e != cudaSuccess) return record(h, e);
     count_launches(h, 1);

@@ -25,6 +25,26 @@ inline int grid_for(size_t work_items, int sm_count, int per_sm = 8)
     return (int)blocks;
 }
 
+// Every thread of every block calls this after the block's last use of the handle's reduction cells (no early
+// returns before it).  True in thread 0 of the block that arrives last: by then every block has read what it
+// needed and added what it had to add, so that thread may publish the sums and must put the cells back to zero.
+__device__ __forceinline__ bool last_block_done(DeviceState *dev)
+{
+    __shared__ unsigned last_s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned t = atomicAdd(&dev->ticket, 1u);
+        last_s = (t == gridDim.x - 1) ? 1u : 0u;
+        if (last_s) {
+            __threadfence();
+            dev->ticket = 0;
+        }
+    }
+    __syncthreads();
+    return last_s != 0 && threadIdx.x == 0;
+}
+
 // ------------------------------------------------------------------ fp32 -> Q / CQ / SQ
 
 // R(log2 M) for a positive finite float given by its bit pattern.
@@ -123,6 +143,7 @@ __global__ void quantize_f32_kernel(int mode, const float *__restrict__ src, siz
         if (mode == 0) reinterpret_cast<int16_t *>(dst)[i] = (int16_t)c;
         else reinterpret_cast<int8_t *>(dst)[i] = (int8_t)c;
     }
+    if (mode == 2 && last_block_done(dev)) dev->absmax_u32 = 0;
 }
 
 // SQ of an fp32 image under the already reduced maximum: c_src channels in, c_dst (zero-padded) channels out,
@@ -165,6 +186,7 @@ __global__ void quantize_image_kernel(const float *__restrict__ src, int rows, i
         else
             reinterpret_cast<int2 *>(dst)[i] = make_int2((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]));
     }
+    if (last_block_done(dev)) dev->absmax_u32 = 0;
 }
 
 // w[oc][kh][kw][c] -> wp[oc][kh][8][c] with zeros in the unused taps; c = 16 (Pixel = int4) or 8 (int2)
@@ -234,7 +256,11 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
     }
     if (sum_codes) {
         sum = block_sum_i64(sum);
-        if (threadIdx.x == 0 && sum) atomicAdd(reinterpret_cast<unsigned long long *>(sum_codes), (unsigned long long)sum);
+        if (threadIdx.x == 0 && sum) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum0), (unsigned long long)sum);
+    }
+    if (last_block_done(dev)) {
+        if (sum_codes) *sum_codes = (long long)atomicExch(reinterpret_cast<unsigned long long *>(&dev->sum0), 0ull);
+        dev->absmax_u32 = 0;
     }
 }
 
@@ -405,6 +431,11 @@ __global__ void prescale_apply_kernel(const int8_t *__restrict__ e0, const int32
                 make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
                           (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
         }
+    }
+    if (last_block_done(dev)) {
+        dev->absmax_u32 = 0;
+        dev->sum0 = 0;
+        dev->sum1 = 0;
     }
 }
 
@@ -695,8 +726,6 @@ cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst,
                                 int sm_count, cudaStream_t s)
 {
     if (mode == 2) {
-        cudaError_t e = launch_reset_cells(dev, s);
-        if (e != cudaSuccess) return e;
         absmax_f32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
     }
     quantize_f32_kernel<<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(mode, src, n, dst, dst_exp, dev);
@@ -706,8 +735,6 @@ cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst,
 cudaError_t launch_quantize_image(const float *src, int n, int h, int w, int c_src, int c_dst, int wmargin, int8_t *dst,
                                   int32_t *dst_exp, DeviceState *dev, int sm_count, cudaStream_t s)
 {
-    cudaError_t e = launch_reset_cells(dev, s);
-    if (e != cudaSuccess) return e;
     const size_t count = (size_t)n * h * w * c_src;
     absmax_f32_kernel<<<grid_for(count / 4 + 1, sm_count), kThreads, 0, s>>>(src, count, dev);
     if (c_dst % 16 == 0) {
@@ -732,15 +759,7 @@ cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bi
                           int32_t *dst_exp, long long *sum_codes, bool max_already_reduced, DeviceState *dev,
                           int sm_count, cudaStream_t s)
 {
-    if (!max_already_reduced) {
-        cudaError_t e = launch_reset_cells(dev, s);
-        if (e != cudaSuccess) return e;
-        absmax_i32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
-    }
-    if (sum_codes) {
-        cudaError_t e = cudaMemsetAsync(sum_codes, 0, sizeof(long long), s);
-        if (e != cudaSuccess) return e;
-    }
+    if (!max_already_reduced) absmax_i32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
     sq_i32_kernel<<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes, dev);
     return cudaGetLastError();
 }
@@ -765,8 +784,6 @@ cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const u
                                 size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
                                 long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s)
 {
-    cudaError_t e = launch_reset_cells(dev, s);
-    if (e != cudaSuccess) return e;
     const size_t n16 = n_el / 16;
     prescale_reduce_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, mask, x2, n16, dev);
     prescale_apply_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, e0_exp, mask, n16, gamma_c, e3, e3_exp,

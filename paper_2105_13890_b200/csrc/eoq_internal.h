@@ -22,7 +22,12 @@ struct DeviceState {
     unsigned long long absmax_u64;
     long long sum0, sum1;  // reduction cells for integer sums
     unsigned tensor_absmax[256];  // per-tensor maxima of the multi-tensor update
+    unsigned ticket;       // blocks of the kernel that consumes the cells last count themselves here (see last_block_done)
 };
+// Invariant: absmax_u32, absmax_u64, sum0, sum1 and ticket are zero whenever no call is in flight on the handle.
+// The kernel that reads a call's reductions last puts the cells it used back to zero (its last block does), so
+// no call starts with a memset.  A kernel that gave up on a wait (EOQ_DEV_TIMEOUT) may leave them dirty:
+// eoq_last_status clears them again when it reports that bit.
 
 struct ProfRecord {
     int kind;
