@@ -681,12 +681,6 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     int8_t *wt = reinterpret_cast<int8_t *>(workspace);
     int32_t *sums = acc_dump ? acc_dump : reinterpret_cast<int32_t *>(reinterpret_cast<char *>(workspace) + round256(g.w_elems));
     cudaError_t e;
-    {
-        ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
-        e = launch_weight_transpose(w, wt, d.c_out, g.taps, d.c_in, s);
-    }
-    if (e != cudaSuccess) return record(h, e);
-    count_launches(h, 1);
 
     // One GEMM per residue class (y mod stride, x mod stride) of the input pixels: within a class the taps
     // kh with (y + pad - kh) divisible by the stride form a unit-stride correlation over e3.
@@ -705,9 +699,13 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             p.epilogue = kEpiDgrad;
             p.acc_out = sums;
             p.dev = h->dev;
+            // the weights are read where they are, [c_out][tap][c_in]: the reduction (c_out) is their slow axis, so
+            // they reach the MMA as MN-major atoms of b_row input channels
+            p.b_mn = 1;
+            p.b_row = chunk_bytes(p.tile_n);
             CUtensorMap map_a, map_b;
             if (!make_patch_map(&map_a, e3, d.n, g.ho, g.wo, d.c_out, p.kc, pl.pw, pl.r_rows + d.kh - 1) ||
-                !make_weight_map(&map_b, wt, d.c_in, g.taps, d.c_out, p.kc, p.tile_n))
+                !make_weight_map(&map_b, w, d.c_out, g.taps, d.c_in, p.b_row, p.kc))
                 return EOQ_ERR_UNSUPPORTED;
             const int ptiles = p.num_m_tiles * p.num_n_tiles;
             count_launches(h, 1);
@@ -725,6 +723,13 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             return record(h, e);
         }
     }
+    // the per-class GEMMs read the weights K-major: [c_in][tap][c_out]
+    {
+        ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
+        e = launch_weight_transpose(w, wt, d.c_out, g.taps, d.c_in, s);
+    }
+    if (e != cudaSuccess) return record(h, e);
+    count_launches(h, 1);
     // a class no tap reaches (e.g. the odd pixels of a strided 1x1 filter) keeps zero sums: clear first
     bool any_empty = false;
     for (int r = 0; r < d.stride; ++r) {

@@ -340,10 +340,12 @@ __device__ __forceinline__ uint64_t smem_desc_join(uint32_t lo, uint32_t hi) { r
 // run at 52 cycles for 64 columns, 69 for 128).  `fresh` is 1 for the first MMAs of a tile, which overwrite.
 
 // kSteps 32-byte K steps of one (A sub-tile, B sub-tile) pair; `parity` = index of the first MMA modulo 2.
+// The B operand has its own descriptor half `b_hi` and its own K step `b_k16` (16-byte units): 2 for a K-major
+// tile (32 bytes along the row), 2 * row bytes for an MN-major one (32 rows further).
 template <int kSteps>
 __device__ __forceinline__ void mma_k_steps(uint32_t d0, uint32_t d1, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
                                             uint32_t idesc, uint32_t parity, uint32_t fresh0, uint32_t fresh1,
-                                            uint32_t leader)
+                                            uint32_t leader, uint32_t b_hi, uint32_t b_k16)
 {
 #pragma unroll
     for (int kk = 0; kk < kSteps; ++kk) {
@@ -351,7 +353,7 @@ __device__ __forceinline__ void mma_k_steps(uint32_t d0, uint32_t d1, uint32_t a
         // the first MMA into each accumulator overwrites it
         uint32_t acc = 1u;
         if (kk < 2) acc = (odd ? fresh1 : fresh0) ? 0u : 1u;
-        ptx::mma_i8(odd ? d1 : d0, smem_desc_join(a_lo + 2 * kk, hi), smem_desc_join(b_lo + 2 * kk, hi), idesc, acc, leader);
+        ptx::mma_i8(odd ? d1 : d0, smem_desc_join(a_lo + 2 * kk, hi), smem_desc_join(b_lo + kk * b_k16, b_hi), idesc, acc, leader);
     }
 }
 
@@ -360,7 +362,8 @@ __device__ __forceinline__ void mma_k_steps(uint32_t d0, uint32_t d1, uint32_t a
 template <int kDim, int kSteps>
 __device__ __forceinline__ void mma_patch_chunk(uint32_t d0, uint32_t d1, uint32_t a_lo, uint32_t b_lo, uint32_t row16,
                                                 uint32_t kc16, uint32_t b_sub16, uint32_t hi, uint32_t idesc,
-                                                bool first_chunk, bool two_acc, uint32_t leader)
+                                                bool first_chunk, bool two_acc, uint32_t leader, uint32_t b_hi,
+                                                uint32_t b_k16)
 {
 #pragma unroll
     for (int a = 0; a < kDim; ++a)
@@ -373,7 +376,7 @@ __device__ __forceinline__ void mma_patch_chunk(uint32_t d0, uint32_t d1, uint32
                 if (idx == 0) acc = first_chunk ? 0u : 1u;
                 if (idx == 1) acc = (first_chunk && two_acc) ? 0u : 1u;
                 ptx::mma_i8((idx & 1) ? d1 : d0, smem_desc_join(a_lo + a * row16 + b * kc16 + 2 * kk, hi),
-                            smem_desc_join(b_lo + (a * kDim + b) * b_sub16 + 2 * kk, hi), idesc, acc, leader);
+                            smem_desc_join(b_lo + (a * kDim + b) * b_sub16 + kk * b_k16, b_hi), idesc, acc, leader);
             }
 }
 // Swizzle field of the descriptor for a sub-tile whose rows are `row_bytes` wide.

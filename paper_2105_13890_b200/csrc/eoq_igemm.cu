@@ -157,8 +157,8 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                 if (wide && k_steps >= 2) {
                     // 2 or 4 MMAs per sub-tile, alternating between the two partial accumulators
                     for (int j = 0; j < subs; ++j) {
-                        if (k_steps == 4) mma_k_steps<4>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1, leader);
-                        else mma_k_steps<2>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1, leader);
+                        if (k_steps == 4) mma_k_steps<4>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1, leader, hi, 2u);
+                        else mma_k_steps<2>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1, leader, hi, 2u);
                         fresh0 = 0;
                         fresh1 = 0;
                         a_lo += a_sub16;

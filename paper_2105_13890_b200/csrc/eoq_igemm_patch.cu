@@ -114,11 +114,22 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
     } else if (warp == 2) {
         if (lane == 0) {
             // ------------------------------------------------------------------ weight loads
+            // One sub-tile = the weights of one tap for kc reduction channels and tile_n columns.  K-major: one box
+            // [tile_n rows][kc bytes].  MN-major: tile_n / b_row boxes [kc rows][b_row bytes], one per atom.
+            auto load_b = [&](uint32_t dst, uint32_t bar, int chunk, int tap, int n0) {
+                if (!p.b_mn) {
+                    ptx::tma_load_3d(dst, &map_b, bar, chunk * p.kc, tap, n0);
+                } else {
+                    const uint32_t atom = (uint32_t)p.kc * p.b_row;
+                    for (int a = 0, na = p.tile_n / p.b_row; a < na; ++a)
+                        ptx::tma_load_3d(dst + a * atom, &map_b, bar, n0 + a * p.b_row, tap, chunk * p.kc);
+                }
+            };
             if (pl.b_resident) {
                 ptx::mbar_expect_tx(b_full(0), (uint32_t)pl.chunks * taps * b_sub);
                 for (int c = 0; c < pl.chunks; ++c)
                     for (int t = 0; t < taps; ++t)
-                        ptx::tma_load_3d(b_region + (c * taps + t) * b_sub, &map_b, b_full(0), c * p.kc, (int)p.tap_b[t], 0);
+                        load_b(b_region + (c * taps + t) * b_sub, b_full(0), c, (int)p.tap_b[t], 0);
                 // completion is observed by the MMA thread, which every path out of this kernel waits for
             } else {
                 int ib = 0;
@@ -130,7 +141,7 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                         for (int t = 0; t < taps; ++t) {
                             if (!(ok = wait_bar<64>(b_empty(ib), phb ^ 1u, ctx))) break;
                             ptx::mbar_expect_tx(b_full(ib), b_sub);
-                            ptx::tma_load_3d(b_region + ib * b_sub, &map_b, b_full(ib), c * p.kc, (int)p.tap_b[t], nt * p.tile_n);
+                            load_b(b_region + ib * b_sub, b_full(ib), c, (int)p.tap_b[t], nt * p.tile_n);
                             inflight |= 1u << ib;
                             inflight_parity = (inflight_parity & ~(1u << ib)) | (phb << ib);
                             if (++ib == pl.num_b) { ib = 0; phb ^= 1u; }
@@ -147,9 +158,24 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
         // ---------------------------------------------------------------------- MMA issuer (whole warp, see elect_one)
         const uint32_t leader = elect_one();
         const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_s, 0);
-        const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, false, false);
+        const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, false, p.b_mn != 0);
         const uint32_t hi = smem_desc_hi(8u * p.kc, layout_type_for(p.kc));
-        const uint32_t b_sub16 = b_sub >> 4, b_ring_lo = b_region >> 4;
+        // B: K-major like A, or MN-major atoms (swizzled rows: atoms kc * b_row apart along the columns = leading
+        // offset, 8-row groups 8 * b_row apart = stride offset; 16-byte rows carry no swizzle and the two offsets
+        // swap roles); a 32-deep K step is 32 bytes along a K-major row, 32 rows of an MN-major atom
+        uint32_t b_hi = hi, b_k16 = 2u, b_lead = 0u;
+        if (p.b_mn) {
+            const uint32_t atom = (uint32_t)p.kc * p.b_row;
+            if (p.b_row == 16) {
+                b_hi = smem_desc_hi(atom, 0);
+                b_lead = (128u >> 4) << 16;
+            } else {
+                b_hi = smem_desc_hi(8u * p.b_row, layout_type_for(p.b_row));
+                b_lead = ((atom >> 4) & 0x3FFFu) << 16;
+            }
+            b_k16 = (32u * p.b_row) >> 4;
+        }
+        const uint32_t b_sub16 = b_sub >> 4, b_ring_lo = (b_region >> 4) | b_lead;
         const uint32_t kc16 = (uint32_t)p.kc >> 4, row16 = (uint32_t)(pl.pw * p.kc) >> 4;  // one pixel / one patch row
         const int k_steps = p.kc / 32, kdim = pl.kdim, chunks = pl.chunks, num_a = pl.num_a, num_b = pl.num_b;
         const bool resident = pl.b_resident != 0;
@@ -171,10 +197,10 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                 uint32_t a_row = (smem_base + ia * pl.a_bytes) >> 4;
                 if (resident && kdim == 3) {
                     // common case, fully unrolled: 9 taps x k_steps MMAs
-                    if (k_steps == 4) mma_patch_chunk<3, 4>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc, leader);
-                    else if (k_steps == 2) mma_patch_chunk<3, 2>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc, leader);
+                    if (k_steps == 4) mma_patch_chunk<3, 4>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc, leader, b_hi, b_k16);
+                    else if (k_steps == 2) mma_patch_chunk<3, 2>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc, leader, b_hi, b_k16);
                     else {
-                        mma_patch_chunk<3, 1>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc, leader);
+                        mma_patch_chunk<3, 1>(d0, d1, a_row, b_res_lo, row16, kc16, b_sub16, hi, idesc, c == 0, two_acc, leader, b_hi, b_k16);
                         const uint32_t t = d0; d0 = d1; d1 = t;  // 9 MMAs: the next chunk starts on the other accumulator
                     }
                     b_res_lo += 9 * b_sub16;
@@ -192,9 +218,9 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                                 ptx::tc_fence_after();
                                 b_lo = b_ring_lo + ib * b_sub16;
                             }
-                            if (k_steps == 4) mma_k_steps<4>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1, leader);
-                            else if (k_steps == 2) mma_k_steps<2>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1, leader);
-                            else mma_k_steps<1>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1, leader);
+                            if (k_steps == 4) mma_k_steps<4>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1, leader, b_hi, b_k16);
+                            else if (k_steps == 2) mma_k_steps<2>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1, leader, b_hi, b_k16);
+                            else mma_k_steps<1>(d0, d1, a_tap, b_lo, hi, idesc, parity, fresh0, fresh1, leader, b_hi, b_k16);
                             if (k_steps == 1) {
                                 // one MMA per tap: it went to accumulator `parity`; for a single accumulator d0 == d1
                                 if (parity == 0) fresh0 = false; else fresh1 = false;

@@ -92,6 +92,10 @@ struct IgemmParams {
     uint8_t *relu_mask;
     int32_t *acc_out;         // forward: optional dump; dgrad: the int32 scratch (required)
     DeviceState *dev;
+    // B operand read MN-major (patch kernel, error back-propagation): the weights stay [c_out][tap][c_in], a sub-tile
+    // is [kc reduction rows][tile_n columns] made of tile_n / b_row atoms of b_row-byte rows, kc * b_row bytes apart
+    int b_mn;
+    int b_row;
 };
 
 // Patch variant of the implicit GEMM for stride-1 filters (eoq_igemm_patch.cu): an M tile is `r_rows` output rows
