@@ -53,6 +53,15 @@ __device__ __forceinline__ int32_t sq_code32(int32_t a, int t)
     return clampi(v, -127, 127);
 }
 
+// The same code for a shift s = t - 7 >= 1 known to the whole kernel, in four integer operations before the
+// clamp: adding 2^(s-1) - 1 plus the parity of the quotient carries into bit s exactly when the remainder exceeds
+// one half, or equals it with an odd quotient.  `half_m1` = 2^(s-1) - 1.  Needs |a| + 2^(s-1) < 2^31, which holds
+// because 2^(s-1) <= max|a| / 2^7.
+__device__ __forceinline__ int32_t sq_code32_shr(int32_t a, int s, int32_t half_m1)
+{
+    return clampi((a + half_m1 + ((a >> s) & 1)) >> s, -127, 127);
+}
+
 __device__ __forceinline__ int32_t sq_code64(long long a, int t)
 {
     int s = t - 7;

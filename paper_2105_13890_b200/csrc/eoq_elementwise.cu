@@ -231,15 +231,30 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
     long long sum = 0;
     const size_t n16 = n / 16;
     const int4 *s4 = reinterpret_cast<const int4 *>(src);
+    const int sh = t - 7;
+    // the maximum bounds every element, so |a| + 2^(sh-1) cannot wrap as long as M + M / 2^7 < 2^31
+    const bool fast = sh >= 1 && M < 0x7e000000u;
+    const int32_t half_m1 = fast ? (1 << (sh - 1)) - 1 : 0;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
         int c[16];
+        if (fast) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            int4 v = __ldcs(s4 + i * 4 + k);
-            c[4 * k + 0] = sq_code32(v.x, t);
-            c[4 * k + 1] = sq_code32(v.y, t);
-            c[4 * k + 2] = sq_code32(v.z, t);
-            c[4 * k + 3] = sq_code32(v.w, t);
+            for (int k = 0; k < 4; ++k) {
+                int4 v = __ldcs(s4 + i * 4 + k);
+                c[4 * k + 0] = sq_code32_shr(v.x, sh, half_m1);
+                c[4 * k + 1] = sq_code32_shr(v.y, sh, half_m1);
+                c[4 * k + 2] = sq_code32_shr(v.z, sh, half_m1);
+                c[4 * k + 3] = sq_code32_shr(v.w, sh, half_m1);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                int4 v = __ldcs(s4 + i * 4 + k);
+                c[4 * k + 0] = sq_code32(v.x, t);
+                c[4 * k + 1] = sq_code32(v.y, t);
+                c[4 * k + 2] = sq_code32(v.z, t);
+                c[4 * k + 3] = sq_code32(v.w, t);
+            }
         }
         int s = 0;
 #pragma unroll
@@ -408,6 +423,14 @@ __global__ void prescale_apply_kernel(const int8_t *__restrict__ e0, const int32
         if (sum_e1) *sum_e1 = dev->sum0;
         if (sum_e1x2) *sum_e1x2 = dev->sum1;
     }
+    // R(v * 2^(7-t)) for v = gamma * e1 (|v| < 2^22) on the floating-point pipe: kMagic + v read as a float is
+    // 1.5 * 2^23 + v exactly; one fused multiply-add forms 1.5 * 2^23 + v * 2^(7-t) (the products are exact, the sum
+    // is rounded once, to nearest even at unit spacing), so the low bits of the result are the rounded quotient.
+    // For t < 7 the scaling is a left shift and nothing is rounded; either way |result| < 2^22 keeps the binade.
+    constexpr uint32_t kMagic = 0x4B400000u;  // 1.5 * 2^23
+    const float scale = __int_as_float((127 + 7 - t) << 23);  // 2^(7-t), t in [0, 22]
+    const float rest = 12582912.0f - 12582912.0f * scale;  // exact: a multiple of a power of two below 2^31
+    const uint32_t g = (uint32_t)gamma_c;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     for (size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < n16; i0 += 4 * stride) {
         int4 ev[4];
@@ -423,10 +446,19 @@ __global__ void prescale_apply_kernel(const int8_t *__restrict__ e0, const int32
         for (int u = 0; u < 4; ++u) {
             const size_t i = i0 + u * stride;
             if (i >= n16) continue;
-            int e[16], c[16];
-            unpack16(ev[u], e);
+            const uint32_t w[4] = {(uint32_t)ev[u].x, (uint32_t)ev[u].y, (uint32_t)ev[u].z, (uint32_t)ev[u].w};
+            int c[16];
 #pragma unroll
-            for (int k = 0; k < 16; ++k) c[k] = ((mv[u] >> k) & 1u) ? sq_code32(gamma_c * e[k], t) : 0;
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t e1w = w[q] & bits_to_bytes(mv[u] >> (4 * q));  // e1 = e0 * [x4 > 0], four codes
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int32_t e1 = (int32_t)(int8_t)(e1w >> (8 * k));
+                    const uint32_t biased = g * (uint32_t)e1 + kMagic;
+                    const uint32_t r = __float_as_uint(__fmaf_rn(__uint_as_float(biased), scale, rest));
+                    c[4 * q + k] = clampi((int32_t)(r - kMagic), -127, 127);
+                }
+            }
             reinterpret_cast<int4 *>(e3)[i] =
                 make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
                           (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));

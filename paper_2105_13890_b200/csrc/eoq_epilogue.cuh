@@ -85,13 +85,21 @@ __device__ __forceinline__ ForwardOperands forward_operands(const IgemmParams &p
     return o;
 }
 
-template <bool kShift7>
-__device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t *acc, size_t off, const ForwardOperands &ops,
-                                           int shift)
+// `acc1` holds the tile's second partial sums when `two` is set; kRelu = a ReLU follows.
+template <bool kShift7, bool kRelu>
+__device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t (&acc)[32], const uint32_t (&acc1)[32],
+                                           bool two, size_t off, const ForwardOperands &ops, int shift)
 {
     int32_t a[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) a[i] = (int32_t)acc[i];
+    if (two && (!kShift7 || p.acc_out)) {
+        // paths that need the whole sum as a value (the dump, the generic shift) merge the partial sums here;
+        // the common path below merges them inside its first clamp
+#pragma unroll
+        for (int i = 0; i < 16; ++i) a[i] += (int32_t)acc1[i];
+        two = false;
+    }
     if (p.b1_table) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -114,11 +122,13 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t 
         // R(a / 2^7) lies in [-32768, 32767] exactly when a lies in [-32768 * 128 - 64, 32767 * 128 + 63], and
         // clamping a to [-32768 * 128, 32767 * 128 + 63] first gives the same code.  |a| < 2^31 - 2^24 (checked
         // on the host), so neither addition below wraps.
+        // The lower clamp merges the second partial sum (one add-max); the add of kMagicBits that follows is taken
+        // modulo 2^32, where max(A, -2^22) + kMagicBits is the true (positive) sum for every A < 2^31 - 2^24.
         q_bias = kMagicBits;
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-            const uint32_t up = (uint32_t)__viaddmax_s32(a[i], 4194304, 0);  // max(a, -2^22) + 2^22
-            q[i] = rne7_magic(__viaddmin_u32(up, kMagicBits - 4194304u, kMagicBits + 4194239u));
+            const int32_t lo = two ? __viaddmax_s32(a[i], (int32_t)acc1[i], -4194304) : max(a[i], -4194304);
+            q[i] = rne7_magic(__viaddmin_u32((uint32_t)lo, kMagicBits, kMagicBits + 4194239u));
         }
     } else {
         q_bias = 0;
@@ -134,9 +144,11 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t 
             q[i] = (uint32_t)clampi(v2, -32768, 32767);
         }
     }
-    // x4 = gamma * x2 + (b2 + shortcut) * 2^7 = gamma * q + add, the bias of q folded into add (mod 2^32)
+    // x4 - 1 = gamma * x2 + (b2 + shortcut) * 2^7 - 1 = gamma * q + add, the bias of q folded into add (mod 2^32).
+    // Forming x4 - 1 instead of x4 makes its sign bit [x4 <= 0], the complement of the mask bit, so the mask
+    // costs one funnel shift per element; the + 1 rides on the add-min that clamps x4.
     const uint32_t g = (uint32_t)p.gamma_c;
-    const uint32_t base = ((uint32_t)p.b2_c << 7) - g * q_bias;
+    const uint32_t base = ((uint32_t)p.b2_c << 7) - g * q_bias - 1u;
     uint32_t add[16];
     if (p.shortcut) {
         const int4 v = ops.shortcut;
@@ -154,15 +166,14 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t 
     }
     // Q_a2: R(x4 / 2^7) saturated to +-127 (and to 0 from below after a ReLU).  16319 / 128 = 127.49.. rounds to
     // 127 and everything above saturates to 127 too, so x4 is clamped to +-16319 before the rounding.
-    uint32_t mbits = 0;
+    uint32_t nbits = 0;  // bit i = [x4 <= 0] of channel i
     uint32_t r[16];
 #pragma unroll
     for (int i = 15; i >= 0; --i) {
-        const int32_t v4 = (int32_t)(g * q[i] + add[i]);
-        const int32_t n4 = (int32_t)((0u - g) * q[i] - add[i]);   // -x4: its sign bit is [x4 > 0]
-        mbits = __funnelshift_l((uint32_t)n4, mbits, 1);
-        if (p.relu) r[i] = rne7_magic((uint32_t)__vimin_s32_relu(v4, 16319) | kMagicBits);
-        else r[i] = rne7_magic((uint32_t)clampi(v4, -16319, 16319) + kMagicBits);
+        const int32_t w = (int32_t)(g * q[i] + add[i]);  // x4 - 1
+        nbits = __funnelshift_l((uint32_t)w, nbits, 1);
+        if (kRelu) r[i] = rne7_magic((uint32_t)__viaddmin_s32_relu(w, 1, 16319) | kMagicBits);
+        else r[i] = rne7_magic((uint32_t)max(__viaddmin_s32(w, 1, 16319), -16319) + kMagicBits);
     }
     int4 o;
     o.x = (int)__byte_perm(__byte_perm(r[0], r[1], 0x0040), __byte_perm(r[2], r[3], 0x0040), 0x5410);
@@ -170,7 +181,7 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t 
     o.z = (int)__byte_perm(__byte_perm(r[8], r[9], 0x0040), __byte_perm(r[10], r[11], 0x0040), 0x5410);
     o.w = (int)__byte_perm(__byte_perm(r[12], r[13], 0x0040), __byte_perm(r[14], r[15], 0x0040), 0x5410);
     *reinterpret_cast<int4 *>(p.x5 + off) = o;
-    if (p.relu_mask) *reinterpret_cast<uint16_t *>(p.relu_mask + (off >> 3)) = (uint16_t)mbits;
+    if (p.relu_mask) *reinterpret_cast<uint16_t *>(p.relu_mask + (off >> 3)) = (uint16_t)~nbits;
     if (p.x2) {
         int4 *d = reinterpret_cast<int4 *>(p.x2 + off);
         d[0] = make_int4((int)__byte_perm(q[0], q[1], 0x5410), (int)__byte_perm(q[2], q[3], 0x5410),

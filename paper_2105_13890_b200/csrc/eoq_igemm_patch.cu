@@ -295,12 +295,15 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                 ForwardOperands next = ops;
                 if (g + 1 < g_end) next = forward_operands(p, fwd && valid && col + 16 < p.N, off + 16, col + 16, cls);
                 ptx::tmem_ld_wait();
-                if (nacc == 2) {
+                if (nacc == 2 && !fwd) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) r[i] += r2[i];  // the two partial accumulators of the tile
                 }
                 if (valid && col < p.N) {
-                    if (fwd) forward_16<true>(p, r, off, ops, 7);
+                    if (fwd) {
+                        if (p.relu) forward_16<true, true>(p, r, r2, nacc == 2, off, ops, 7);
+                        else forward_16<true, false>(p, r, r2, nacc == 2, off, ops, 7);
+                    }
                     else mx = max(mx, dgrad_16(p, r, off));
                 }
                 ops = next;

@@ -65,7 +65,7 @@ class TrainStep:
 
     def __init__(self, workload: Workload, handle: int, device: str = "cuda:0", seed: int = synth.BASE_SEED,
                  scalars: Optional[Scalars] = None, lr_mant: int = 1, lr_exp: int = -6, image_channels: int = 3,
-                 side_streams: int = 1):
+                 side_streams: int = 2):
         self.wl, self.h, self.dev = workload, handle, torch.device(device)
         self.sc = scalars or Scalars()
         self.lr_mant, self.lr_exp = lr_mant, lr_exp
