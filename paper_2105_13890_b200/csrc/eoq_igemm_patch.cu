@@ -268,9 +268,16 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
         const bool fwd = p.epilogue == kEpiForward;
         uint32_t acc_phase = 0, mx = 0;
         bool ok = true;
-        for (int tile = blockIdx.x + grp * gridDim.x; tile < num_tiles && ok; tile += 2 * gridDim.x) {
-            const int mt = tile / p.num_n_tiles, nt = tile % p.num_n_tiles;
-            const int img = mt / pl.tiles_per_img, y = (mt % pl.tiles_per_img) * pl.r_rows + yl;
+        // (column tile, image, row tile in the image) of the current tile, carried from tile to tile: the step
+        // between two tiles of this pair is constant, so its quotients are formed once instead of four integer
+        // divisions per tile and warp
+        const int tile0 = blockIdx.x + grp * gridDim.x, step = 2 * gridDim.x;
+        int nt = tile0 % p.num_n_tiles, mt0 = tile0 / p.num_n_tiles;
+        int img = mt0 / pl.tiles_per_img, ti = mt0 % pl.tiles_per_img;
+        const int step_nt = step % p.num_n_tiles, step_mt = step / p.num_n_tiles;
+        const int step_img = step_mt / pl.tiles_per_img, step_ti = step_mt % pl.tiles_per_img;
+        for (int tile = tile0; tile < num_tiles && ok; tile += step) {
+            const int y = ti * pl.r_rows + yl;
             const bool valid = yl < pl.r_rows && xx < p.wq && y < p.hq;
             size_t pix = 0;
             int cls = 0;
@@ -312,6 +319,12 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(tempty_bar(grp));
             acc_phase ^= 1u;
+            nt += step_nt;
+            ti += step_ti;
+            if (nt >= p.num_n_tiles) { nt -= p.num_n_tiles; ++ti; }
+            img += step_img;
+            if (ti >= pl.tiles_per_img) { ti -= pl.tiles_per_img; ++img; }
+            if (ti >= pl.tiles_per_img) { ti -= pl.tiles_per_img; ++img; }
         }
         if (p.epilogue == kEpiDgrad) {
             mx = warp_max_u32(mx);

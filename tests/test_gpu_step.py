@@ -130,3 +130,42 @@ def test_every_layer_of_a_step_matches_the_oracle(name, batch):
         want, _, _ = oracle.update(wq, bwd["g_w"], bwd["p_gw"], st.lr_mant, st.lr_exp, stochastic=True,
                                    seed=synth.BASE_SEED, step=0, tensor_id=i)
         assert np.array_equal(lb.w.cpu().numpy().astype(np.int32), want), (l.name, "w")
+
+
+@pytest.mark.parametrize("batch", [1, 2, 4])
+def test_weight_trajectory_over_consecutive_steps(batch):
+    """Small-batch online training: several consecutive steps (each with its own stochastic-rounding draws) must
+    leave, after every step, exactly the int8 weights the oracle reaches when it repeats the same steps."""
+    steps = 4
+    wl = workloads.get("resnet20", batch)
+    st = TrainStep(wl, eoq.eoq_create(0), scalars=Scalars(), lr_mant=3, lr_exp=-4)
+    host = _host_inputs(st, wl)
+    sc = st.sc
+    w_ref = [wq.copy() for (_, _, _, wq) in host]
+    img = st.host_image(synth.BASE_SEED)
+    changed = 0
+    for k in range(steps):
+        st.run()
+        torch.cuda.synchronize()
+        assert st.status() & eoq.EOQ_DEV_TIMEOUT == 0
+        for i, (lb, (x0, e0, short, _)) in enumerate(zip(st.layers, host)):
+            l = lb.layer
+            d = ConvDesc(l.n, l.h, l.w, l.c_in, l.c_out, l.k, l.k, l.stride, l.pad)
+            gamma = sc.gamma_c if l.gamma_trainable else 128
+            b1 = 0 if i == 0 else sc.b1_c
+            x_exp = -7
+            if i == 0:
+                padded = np.zeros(img.shape[:3] + (l.c_in,), dtype=np.float32)
+                padded[..., :img.shape[3]] = img
+                codes, x_exp, _ = oracle.quantize_f32(oracle.MODE_SQ, padded)
+                x0 = codes.astype(np.int8)
+            fwd = oracle.layer_forward(d, x0, b1, w_ref[i], gamma, sc.b2_c if l.relu else 0, short, l.relu, x_exp=x_exp)
+            bwd = oracle.layer_backward(d, e0, -12, fwd["mask"] if l.relu else np.ones_like(fwd["mask"]),
+                                        fwd["x2"] if lb.x2 is not None else None, x0, b1, w_ref[i], gamma)
+            want, _, _ = oracle.update(w_ref[i], bwd["g_w"], bwd["p_gw"], st.lr_mant, st.lr_exp, stochastic=True,
+                                       seed=synth.BASE_SEED, step=k, tensor_id=i)
+            want = want.astype(np.int8)
+            changed += int(np.count_nonzero(want != w_ref[i]))
+            w_ref[i] = want
+            assert np.array_equal(lb.w.cpu().numpy(), want), (k, l.name)
+    assert changed > 0  # the trajectory is not vacuous: updates moved weight codes
