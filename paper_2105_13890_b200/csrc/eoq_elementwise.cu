@@ -164,10 +164,19 @@ __global__ void quantize_image_kernel(const float *__restrict__ src, int rows, i
     const int w_mem = w + 2 * wmargin;
     const size_t items = (size_t)rows * w_mem * groups;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
-        const int g = (int)(i % groups);
-        const size_t mp = i / groups;            // pixel index in the widened layout
-        const int xm = (int)(mp % w_mem) - wmargin;
-        const size_t row = mp / w_mem;
+        int g, xm;
+        size_t row;
+        if (items <= 0xffffffffull) {  // 32-bit index arithmetic: three 64-bit divisions would dominate the item's work
+            const uint32_t mp = (uint32_t)i / (uint32_t)groups, r = mp / (uint32_t)w_mem;
+            g = (int)((uint32_t)i - mp * (uint32_t)groups);
+            xm = (int)(mp - r * (uint32_t)w_mem) - wmargin;
+            row = r;
+        } else {
+            g = (int)(i % groups);
+            const size_t mp = i / groups;            // pixel index in the widened layout
+            xm = (int)(mp % w_mem) - wmargin;
+            row = mp / w_mem;
+        }
         int c[kG];
 #pragma unroll
         for (int k = 0; k < kG; ++k) {
@@ -688,9 +697,18 @@ __global__ void b1_tap_sums_kernel(const int8_t *__restrict__ e3, long long *tap
     for (int k = 0; k < 16; ++k) acc[k] = 0;
     const size_t begin = (size_t)blockIdx.x * pixels_per_block;
     const size_t end = min(pixels, begin + (size_t)pixels_per_block);
+    const bool small = pixels <= 0xffffffffull;
     if (slot < pix_per_step) {
         for (size_t p = begin + slot; p < end; p += pix_per_step) {
-            const int x = (int)(p % wo), y = (int)((p / wo) % ho);
+            int x, y;
+            if (small) {  // 32-bit index arithmetic (a 64-bit division costs more than the rest of the pixel's work)
+                const uint32_t q = (uint32_t)p / (uint32_t)wo;
+                x = (int)((uint32_t)p - q * (uint32_t)wo);
+                y = (int)(q % (uint32_t)ho);
+            } else {
+                x = (int)(p % wo);
+                y = (int)((p / wo) % ho);
+            }
             const int cls = border_class(y, ho, bc.nlo_h, bc.nhi_h, bc.nrc) * bc.ncc + border_class(x, wo, bc.nlo_w, bc.nhi_w, bc.ncc);
             const int4 v = __ldg(reinterpret_cast<const int4 *>(e3 + p * c_out + ch));
             const int8_t *b = reinterpret_cast<const int8_t *>(&v);
@@ -894,7 +912,7 @@ cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, const eo
     const int classes = bc.nrc * bc.ncc;
     const size_t pixels = (size_t)d.n * ho * wo;
     const int slabs = (d.c_out + kClassSlab - 1) / kClassSlab;
-    int blocks = (4 * sm_count + slabs - 1) / slabs;
+    int blocks = (2 * sm_count + slabs - 1) / slabs;  // more blocks only add contention on the per-tap cells
     size_t ppb = (pixels + blocks - 1) / blocks;
     if (ppb < 64) ppb = 64;
     if (ppb > (1u << 23)) ppb = 1u << 23;  // keeps the int32 class sums exact
