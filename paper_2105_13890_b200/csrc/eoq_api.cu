@@ -356,6 +356,8 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
     h->profiling = false;
     h->num_records = 0;
     h->records = nullptr;
+    h->branch = nullptr;
+    h->fork_ev = h->join_ev = nullptr;
     cudaDeviceProp prop;
     cudaError_t e = cudaGetDeviceProperties(&prop, device);
     if (e == cudaSuccess) {
@@ -367,8 +369,14 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
         e = cudaMalloc(reinterpret_cast<void **>(&h->dev), sizeof(DeviceState));
     }
     if (e == cudaSuccess) e = cudaMemset(h->dev, 0, sizeof(DeviceState));
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->branch, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->fork_ev, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->join_ev, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
+        if (h->join_ev) cudaEventDestroy(h->join_ev);
+        if (h->fork_ev) cudaEventDestroy(h->fork_ev);
+        if (h->branch) cudaStreamDestroy(h->branch);
         if (h->dev) cudaFree(h->dev);
         delete h;
         return EOQ_ERR_CUDA;
@@ -383,6 +391,9 @@ extern "C" int eoq_destroy(eoq_handle_t handle)
     if (!h) return EOQ_ERR_BAD_ARG;
     cudaSetDevice(h->device);
     cudaDeviceSynchronize();
+    if (h->join_ev) cudaEventDestroy(h->join_ev);
+    if (h->fork_ev) cudaEventDestroy(h->fork_ev);
+    if (h->branch) cudaStreamDestroy(h->branch);
     if (h->dev) cudaFree(h->dev);
     if (h->records) {
         for (int i = 0; i < h->num_records; ++i) {
@@ -813,6 +824,30 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
 
 // ================================================================================= weight gradient
 
+// The b1 tap sums (one pass over e3) next to the weight-gradient GEMM: issued on the handle's branch stream
+// behind a fork event recorded on `s` (everything queued on `s` so far, the clearing memset included, comes
+// first); the caller waits for join_ev on `s` before the kernel that reads the sums.  Without a branch stream
+// (the allocation-free handle) they are issued on `s` itself.
+static cudaError_t launch_tap_sums_beside(Handle *h, const int8_t *e3, long long *tap_sums, const eoq_conv_desc_t &d,
+                                          int ho, int wo, const BorderClasses &bc, cudaStream_t s, bool *joined)
+{
+    *joined = false;
+    count_launches(h, 1);
+    if (!h->branch) {
+        ProfScope prof(h, EOQ_PROF_WGRAD_AUX, s);
+        return launch_b1_error_sums(e3, tap_sums, d, ho, wo, bc, h->sm_count, s);
+    }
+    cudaError_t e = cudaEventRecord(h->fork_ev, s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->branch, h->fork_ev, 0);
+    if (e == cudaSuccess) {
+        ProfScope prof(h, EOQ_PROF_WGRAD_AUX, h->branch);
+        e = launch_b1_error_sums(e3, tap_sums, d, ho, wo, bc, h->sm_count, h->branch);
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(h->join_ev, h->branch);
+    *joined = e == cudaSuccess;
+    return e;
+}
+
 extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3,
                               const int32_t *e3_exp, const int8_t *x, int32_t b1_c, int8_t *gq, int32_t *g_exp,
                               int64_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
@@ -839,6 +874,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     long long *acc = reinterpret_cast<long long *>(ws + tap_bytes + 256);
     const size_t acc_bytes = round256(g.w_elems * sizeof(long long));
 
+    bool joined = false;  // the tap sums run on the handle's branch stream and must be waited for
     WgradPatchPlan wp;
     if (plan_wgrad_patch(wp, d, g.ho, g.wo)) {
         wp.partials = reinterpret_cast<int32_t *>(ws + tap_bytes + 256 + acc_bytes);
@@ -847,11 +883,8 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         {
             ProfScope prof(h, EOQ_PROF_WGRAD_AUX, s);
             e = b1_c != 0 ? cudaMemsetAsync(ws, 0, tap_bytes + 256, s) : cudaMemsetAsync(cells, 0, 256, s);
-            if (e == cudaSuccess && b1_c != 0) {
-                e = launch_b1_error_sums(e3, tap_sums, d, g.ho, g.wo, bc, h->sm_count, s);
-                count_launches(h, 1);
-            }
         }
+        if (e == cudaSuccess && b1_c != 0) e = launch_tap_sums_beside(h, e3, tap_sums, d, g.ho, g.wo, bc, s, &joined);
         if (e != cudaSuccess) return record(h, e);
         CUtensorMap map_x, map_e;
         if (!make_patch_map(&map_x, x, d.n, d.h, d.w, d.c_in, wp.kc, wp.pw, wp.r_rows + d.kh - 1) ||
@@ -862,6 +895,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             ProfScope prof(h, EOQ_PROF_WGRAD, s);
             e = launch_wgrad_patch(wp, map_x, map_e, s);
         }
+        if (e == cudaSuccess && joined) e = cudaStreamWaitEvent(s, h->join_ev, 0);
         if (e != cudaSuccess) return record(h, e);
         ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
         e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
@@ -948,11 +982,8 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         ProfScope aux(h, EOQ_PROF_WGRAD_AUX, s);
         // the GEMM adds into the int64 sums with atomics: they are cleared together with the cells and class sums
         e = cudaMemsetAsync(ws, 0, tap_bytes + 256 + acc_bytes, s);
-        if (e == cudaSuccess && b1_c != 0) {
-            e = launch_b1_error_sums(e3, tap_sums, d, g.ho, g.wo, bc, h->sm_count, s);
-            count_launches(h, 1);
-        }
     }
+    if (e == cudaSuccess && b1_c != 0) e = launch_tap_sums_beside(h, e3, tap_sums, d, g.ho, g.wo, bc, s, &joined);
     if (e != cudaSuccess) return record(h, e);
     CUtensorMap map_x, map_e;
     if (!make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage)) return EOQ_ERR_UNSUPPORTED;
@@ -966,6 +997,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         ProfScope prof(h, EOQ_PROF_WGRAD, s);
         e = launch_wgrad(p, map_x, map_e, s);
     }
+    if (e == cudaSuccess && joined) e = cudaStreamWaitEvent(s, h->join_ev, 0);
     if (e != cudaSuccess) return record(h, e);
     // the kernel leaves sums as [oc][tap][ic], which is the layout of g
     ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);

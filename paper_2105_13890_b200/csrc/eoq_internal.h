@@ -43,6 +43,11 @@ struct Handle {
     bool profiling;
     int num_records;
     ProfRecord *records;          // kMaxProfRecords entries, allocated on first eoq_profile_start
+    // Branch stream of the weight-gradient call: the b1 tap sums do not depend on the GEMM, so they are issued
+    // on this stream between a fork and a join event and run beside it (null: everything stays on the caller's
+    // stream).  Under stream capture the fork and join become graph edges.
+    cudaStream_t branch;
+    cudaEvent_t fork_ev, join_ev;
 };
 constexpr int kMaxProfRecords = 8192;
 
