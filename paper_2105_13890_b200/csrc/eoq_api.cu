@@ -489,7 +489,7 @@ extern "C" int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits
     if (e == cudaSuccess && (v & EOQ_DEV_TIMEOUT)) {
         // a kernel that gave up may not have put the reduction cells back to zero
         e = launch_reset_cells(h->dev, s);
-        if (e == cudaSuccess) e = cudaMemsetAsync(&h->dev->ticket, 0, sizeof(unsigned), s);
+        if (e == cudaSuccess) e = cudaMemsetAsync(&h->dev->ticket, 0, 2 * sizeof(unsigned), s);  // ticket and arrivals
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     }
     *bits = v;

@@ -480,6 +480,118 @@ __global__ void prescale_apply_kernel(const int8_t *__restrict__ e0, const int32
     }
 }
 
+// Both passes of the error head in one kernel, for tensors small enough that every thread keeps its share of e1
+// (up to kFusedGroups groups of 16 codes) in registers between the passes: e0 and the mask are read once and no
+// second launch is needed.  Between the passes all blocks meet at a grid-wide barrier (a counter in the handle's
+// device state), so the kernel is launched cooperatively: the launch guarantees that all its blocks are resident
+// together.  The wait is bounded like every wait of the library; on timeout the kernel flags it and writes nothing.
+constexpr int kFusedGroups = 6;
+__global__ void __launch_bounds__(kThreads)
+prescale_fused_kernel(const int8_t *__restrict__ e0, const int32_t *e0_exp, const uint8_t *__restrict__ mask,
+                      const int16_t *__restrict__ x2, size_t n16, int32_t gamma_c, int8_t *e3, int32_t *e3_exp,
+                      long long *sum_e1, long long *sum_e1x2, DeviceState *dev)
+{
+    __shared__ unsigned go_s;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t e1w[kFusedGroups][4];
+    uint32_t mx4 = 0;
+    long long s1 = 0, s2 = 0;
+    {
+        int4 ev[kFusedGroups];
+        uint32_t mv[kFusedGroups];
+#pragma unroll
+        for (int u = 0; u < kFusedGroups; ++u) {
+            const size_t i = i0 + u * stride;
+            const bool in = i < n16;
+            ev[u] = in ? __ldg(reinterpret_cast<const int4 *>(e0) + i) : make_int4(0, 0, 0, 0);
+            mv[u] = (in && mask) ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(mask) + i) : 0xffffu;
+        }
+#pragma unroll
+        for (int u = 0; u < kFusedGroups; ++u) {
+            const uint32_t w[4] = {(uint32_t)ev[u].x, (uint32_t)ev[u].y, (uint32_t)ev[u].z, (uint32_t)ev[u].w};
+            int a1 = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                e1w[u][q] = w[q] & bits_to_bytes(mv[u] >> (4 * q));  // e1 = e0 * [x4 > 0], four codes per word
+                mx4 = __vmaxu4(mx4, __vabsss4(e1w[u][q]));
+                a1 = __dp4a((int)e1w[u][q], 0x01010101, a1);
+            }
+            s1 += a1;
+            const size_t i = i0 + u * stride;
+            if (x2 && i < n16) {
+                const int4 lo = __ldg(reinterpret_cast<const int4 *>(x2) + 2 * i);
+                const int4 hi = __ldg(reinterpret_cast<const int4 *>(x2) + 2 * i + 1);
+                const int16_t *pl = reinterpret_cast<const int16_t *>(&lo), *ph = reinterpret_cast<const int16_t *>(&hi);
+                const int8_t *eb = reinterpret_cast<const int8_t *>(e1w[u]);
+                int a2 = 0;  // |e1 * x2| < 2^22, 16 terms
+#pragma unroll
+                for (int k = 0; k < 8; ++k) a2 += (int)eb[k] * pl[k] + (int)eb[8 + k] * ph[k];
+                s2 += a2;
+            }
+        }
+    }
+    uint32_t mx = max(max(mx4 & 0xffu, (mx4 >> 8) & 0xffu), max((mx4 >> 16) & 0xffu, mx4 >> 24));
+    mx = (uint32_t)block_max_u64(mx);
+    s1 = block_sum_i64(s1);
+    s2 = block_sum_i64(s2);
+    if (threadIdx.x == 0) {
+        if (mx) atomicMax(&dev->absmax_u32, mx);
+        if (s1) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum0), (unsigned long long)s1);
+        if (s2) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum1), (unsigned long long)s2);
+        // grid-wide barrier: every block's contribution is in the cells once all have arrived
+        __threadfence();
+        atomicAdd(&dev->arrivals, 1u);
+        unsigned ok = 0;
+        for (uint32_t it = 0; it < kSpinLimit; ++it) {
+            if (*reinterpret_cast<volatile unsigned *>(&dev->arrivals) >= gridDim.x) { ok = 1; break; }
+            __nanosleep(100);
+        }
+        if (!ok) atomicOr(&dev->status, EOQ_DEV_TIMEOUT);
+        __threadfence();
+        go_s = ok;
+    }
+    __syncthreads();
+    if (!go_s) return;
+    const uint32_t M = *reinterpret_cast<volatile unsigned *>(&dev->absmax_u32) * (uint32_t)abs(gamma_c);
+    const int t = M ? round_log2_u32(M) : 7;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const int p_in = *e0_exp - 7;
+        *e3_exp = M ? p_in + t - 7 : p_in;
+        if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+        if (sum_e1) *sum_e1 = *reinterpret_cast<volatile long long *>(&dev->sum0);
+        if (sum_e1x2) *sum_e1x2 = *reinterpret_cast<volatile long long *>(&dev->sum1);
+    }
+    // same rounding as prescale_apply_kernel: R(gamma * e1 * 2^(7-t)) with one FMA
+    constexpr uint32_t kMagic = 0x4B400000u;
+    const float scale = __int_as_float((127 + 7 - t) << 23);
+    const float rest = 12582912.0f - 12582912.0f * scale;
+    const uint32_t g = (uint32_t)gamma_c;
+#pragma unroll
+    for (int u = 0; u < kFusedGroups; ++u) {
+        const size_t i = i0 + u * stride;
+        if (i >= n16) continue;
+        int c[16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int32_t e1 = (int32_t)(int8_t)(e1w[u][q] >> (8 * k));
+                const uint32_t r = __float_as_uint(__fmaf_rn(__uint_as_float(g * (uint32_t)e1 + kMagic), scale, rest));
+                c[4 * q + k] = clampi((int32_t)(r - kMagic), -127, 127);
+            }
+        reinterpret_cast<int4 *>(e3)[i] =
+            make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
+                      (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+    }
+    if (last_block_done(dev)) {
+        dev->absmax_u32 = 0;
+        dev->sum0 = 0;
+        dev->sum1 = 0;
+        dev->arrivals = 0;
+    }
+}
+
 // ------------------------------------------------------------------ 8-bit update
 
 constexpr int kUpdChunk = 64;           // tensors per launch
@@ -835,6 +947,28 @@ cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const u
                                 long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s)
 {
     const size_t n16 = n_el / 16;
+    // one cooperative kernel when every thread can hold its share of the tensor between the two passes
+    static int blocks_per_sm = -1;
+    static bool coop = false;
+    if (blocks_per_sm < 0) {
+        int dev_id = 0, can = 0, bps = 0;
+        if (cudaGetDevice(&dev_id) == cudaSuccess &&
+            cudaDeviceGetAttribute(&can, cudaDevAttrCooperativeLaunch, dev_id) == cudaSuccess && can &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, prescale_fused_kernel, kThreads, 0) == cudaSuccess && bps > 0) {
+            coop = true;
+            blocks_per_sm = bps > 4 ? 4 : bps;  // leaves room on every SM for kernels of other streams
+        } else {
+            blocks_per_sm = 0;
+        }
+    }
+    const size_t max_blocks = (size_t)blocks_per_sm * sm_count;
+    const size_t need_blocks = (n16 + (size_t)kThreads * kFusedGroups - 1) / ((size_t)kThreads * kFusedGroups);
+    if (coop && n16 > 0 && need_blocks <= max_blocks) {
+        void *args[] = {(void *)&e0, (void *)&e0_exp, (void *)&mask, (void *)&x2, (void *)&n16, (void *)&gamma_c,
+                        (void *)&e3, (void *)&e3_exp, (void *)&sum_e1, (void *)&sum_e1x2, (void *)&dev};
+        return cudaLaunchCooperativeKernel((const void *)prescale_fused_kernel, dim3((unsigned)need_blocks), dim3(kThreads),
+                                           args, 0, s);
+    }
     prescale_reduce_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, mask, x2, n16, dev);
     prescale_apply_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, e0_exp, mask, n16, gamma_c, e3, e3_exp,
                                                                        sum_e1, sum_e1x2, dev);

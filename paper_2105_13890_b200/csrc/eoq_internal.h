@@ -23,8 +23,9 @@ struct DeviceState {
     long long sum0, sum1;  // reduction cells for integer sums
     unsigned tensor_absmax[256];  // per-tensor maxima of the multi-tensor update
     unsigned ticket;       // blocks of the kernel that consumes the cells last count themselves here (see last_block_done)
+    unsigned arrivals;     // grid-wide barrier of the one-kernel error head (cooperative launch)
 };
-// Invariant: absmax_u32, absmax_u64, sum0, sum1 and ticket are zero whenever no call is in flight on the handle.
+// Invariant: absmax_u32, absmax_u64, sum0, sum1, ticket and arrivals are zero whenever no call is in flight on the handle.
 // The kernel that reads a call's reductions last puts the cells it used back to zero (its last block does), so
 // no call starts with a memset.  A kernel that gave up on a wait (EOQ_DEV_TIMEOUT) may leave them dirty:
 // eoq_last_status clears them again when it reports that bit.
