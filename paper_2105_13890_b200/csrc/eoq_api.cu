@@ -203,6 +203,16 @@ inline bool use_row_window(const eoq_conv_desc_t &d, int wo)
     return d.x_wmargin >= d.pad && d.x_wmargin >= need_right;
 }
 
+// CTAs of a persistent GEMM over `tiles` tiles.  The kernel lasts as long as its busiest CTA, ceil(tiles / SMs)
+// tiles; spreading the tiles evenly over the fewest CTAs that keep that maximum costs nothing and leaves the other
+// SMs to kernels of other streams (448 tiles on 148 SMs: 112 CTAs of 4 tiles instead of 148 of 3 or 4).
+inline int persistent_grid(int tiles, int sm_count)
+{
+    if (tiles <= sm_count) return tiles < 1 ? 1 : tiles;
+    const int per_cta = (tiles + sm_count - 1) / sm_count;
+    return (tiles + per_cta - 1) / per_cta;
+}
+
 // Shared tiling choices of the implicit GEMM: K sub-tiles, pipeline depth, column tile.
 void plan_igemm(IgemmParams &p, int src_channels, int ntaps, int sm_count)
 {
@@ -655,7 +665,7 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
         const int ptiles = p.num_m_tiles * p.num_n_tiles;
         count_launches(h, 1);
         ProfScope prof(h, EOQ_PROF_IGEMM_FWD, s);
-        return record(h, launch_igemm_patch(p, pl, map_a, map_b, ptiles < h->sm_count ? ptiles : h->sm_count, s));
+        return record(h, launch_igemm_patch(p, pl, map_a, map_b, persistent_grid(ptiles, h->sm_count), s));
     }
     if (row_window) {
         if (!make_row_window_map(&map_a, x, d.n, d.h, w_mem, d.c_in, d.x_wmargin - d.pad, g.wo, g.ho, d.stride, d.pad, kTileM) ||
@@ -669,7 +679,7 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     const int tiles = p.num_m_tiles * p.num_n_tiles;
     count_launches(h, 1);
     ProfScope prof(h, EOQ_PROF_IGEMM_FWD, s);
-    return record(h, launch_igemm(p, map_a, map_b, tiles < h->sm_count ? tiles : h->sm_count, s));
+    return record(h, launch_igemm(p, map_a, map_b, persistent_grid(tiles, h->sm_count), s));
 }
 
 // ================================================================================= error back-propagation
@@ -722,7 +732,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             count_launches(h, 1);
             {
                 ProfScope prof(h, EOQ_PROF_IGEMM_DGRAD, s);
-                e = launch_igemm_patch(p, pl, map_a, map_b, ptiles < h->sm_count ? ptiles : h->sm_count, s);
+                e = launch_igemm_patch(p, pl, map_a, map_b, persistent_grid(ptiles, h->sm_count), s);
             }
             if (e != cudaSuccess) return record(h, e);
             {
@@ -808,7 +818,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             count_launches(h, 1);
             {
                 ProfScope prof(h, EOQ_PROF_IGEMM_DGRAD, s);
-                e = launch_igemm(p, map_a, map_b, tiles < h->sm_count ? tiles : h->sm_count, s);
+                e = launch_igemm(p, map_a, map_b, persistent_grid(tiles, h->sm_count), s);
             }
             if (e != cudaSuccess) return record(h, e);
         }
