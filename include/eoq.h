@@ -228,6 +228,14 @@ EOQ_API int eoq_profile_start(eoq_handle_t handle);
 EOQ_API int eoq_profile_stop(eoq_handle_t handle, int launches[EOQ_PROF_KINDS], double milliseconds[EOQ_PROF_KINDS]);
 EOQ_API unsigned long long eoq_launch_count(eoq_handle_t handle);
 
+/* Caps the CTAs (one per SM) that the GEMM launches of this handle use; 0 = one per SM of the device (the
+ * default).  Every GEMM kernel is persistent: with fewer CTAs a launch walks more tiles per CTA and leaves the
+ * other SMs free, so that GEMMs issued through two handles on two streams run side by side instead of one after
+ * the other (in the training step of Sec. 3.2.1 the error back-propagation of a layer and its weight gradient are
+ * independent once e3 exists).  Results do not depend on the setting.  Host-side state only; applies to the calls
+ * made after it. */
+EOQ_API int eoq_set_gemm_ctas(eoq_handle_t handle, int ctas);
+
 /* The last cudaError_t a call on this handle recorded (0 if none). */
 EOQ_API int eoq_last_cuda_error(eoq_handle_t handle);
 

@@ -291,7 +291,7 @@ bool plan_patch(IgemmParams &p, PatchPlan &pl, int n_img, int c_src, int hq, int
 }
 
 // Plan of the patch variant of the weight gradient; false when the geometry does not suit it.
-bool plan_wgrad_patch(WgradPatchPlan &pl, const eoq_conv_desc_t &d, int ho, int wo)
+bool plan_wgrad_patch(WgradPatchPlan &pl, const eoq_conv_desc_t &d, int ho, int wo, int target_ctas = kWgradTargetCtas)
 {
     if (d.stride != 1 || d.kh != d.kw || d.kh < 2 || d.x_wmargin != 0 || d.c_in % 32 || d.c_out % 32) return false;
     if (d.pad > d.kh - 1) return false;
@@ -335,7 +335,7 @@ bool plan_wgrad_patch(WgradPatchPlan &pl, const eoq_conv_desc_t &d, int ho, int 
     pl.num_stages = stages > 4 ? 4 : stages;
     if (pl.num_stages < 2) return false;
     const int total_blocks = d.n * pl.blocks_per_img;
-    int splits = (kWgradTargetCtas + pl.num_groups - 1) / pl.num_groups;
+    int splits = (target_ctas + pl.num_groups - 1) / pl.num_groups;
     if (splits > total_blocks) splits = total_blocks;
     if (splits < 1) splits = 1;
     int per = (total_blocks + splits - 1) / splits;
@@ -372,6 +372,7 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
     cudaError_t e = cudaGetDeviceProperties(&prop, device);
     if (e == cudaSuccess) {
         h->sm_count = prop.multiProcessorCount;
+        h->gemm_ctas = h->sm_count;
         if (prop.major != 10) {
             delete h;
             return EOQ_ERR_UNSUPPORTED;  // the kernels are sm_100a only
@@ -450,6 +451,14 @@ extern "C" int eoq_profile_stop(eoq_handle_t handle, int launches[EOQ_PROF_KINDS
         milliseconds[h->records[i].kind] += ms;
     }
     return record(h, e);
+}
+
+extern "C" int eoq_set_gemm_ctas(eoq_handle_t handle, int ctas)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || ctas < 0) return EOQ_ERR_BAD_ARG;
+    h->gemm_ctas = (ctas == 0 || ctas > h->sm_count) ? h->sm_count : ctas;
+    return EOQ_OK;
 }
 
 extern "C" unsigned long long eoq_launch_count(eoq_handle_t handle)
@@ -665,7 +674,7 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
         const int ptiles = p.num_m_tiles * p.num_n_tiles;
         count_launches(h, 1);
         ProfScope prof(h, EOQ_PROF_IGEMM_FWD, s);
-        return record(h, launch_igemm_patch(p, pl, map_a, map_b, persistent_grid(ptiles, h->sm_count), s));
+        return record(h, launch_igemm_patch(p, pl, map_a, map_b, persistent_grid(ptiles, h->gemm_ctas), s));
     }
     if (row_window) {
         if (!make_row_window_map(&map_a, x, d.n, d.h, w_mem, d.c_in, d.x_wmargin - d.pad, g.wo, g.ho, d.stride, d.pad, kTileM) ||
@@ -679,7 +688,7 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     const int tiles = p.num_m_tiles * p.num_n_tiles;
     count_launches(h, 1);
     ProfScope prof(h, EOQ_PROF_IGEMM_FWD, s);
-    return record(h, launch_igemm(p, map_a, map_b, persistent_grid(tiles, h->sm_count), s));
+    return record(h, launch_igemm(p, map_a, map_b, persistent_grid(tiles, h->gemm_ctas), s));
 }
 
 // ================================================================================= error back-propagation
@@ -732,7 +741,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             count_launches(h, 1);
             {
                 ProfScope prof(h, EOQ_PROF_IGEMM_DGRAD, s);
-                e = launch_igemm_patch(p, pl, map_a, map_b, persistent_grid(ptiles, h->sm_count), s);
+                e = launch_igemm_patch(p, pl, map_a, map_b, persistent_grid(ptiles, h->gemm_ctas), s);
             }
             if (e != cudaSuccess) return record(h, e);
             {
@@ -818,7 +827,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             count_launches(h, 1);
             {
                 ProfScope prof(h, EOQ_PROF_IGEMM_DGRAD, s);
-                e = launch_igemm(p, map_a, map_b, persistent_grid(tiles, h->sm_count), s);
+                e = launch_igemm(p, map_a, map_b, persistent_grid(tiles, h->gemm_ctas), s);
             }
             if (e != cudaSuccess) return record(h, e);
         }
@@ -886,7 +895,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
 
     bool joined = false;  // the tap sums run on the handle's branch stream and must be waited for
     WgradPatchPlan wp;
-    if (plan_wgrad_patch(wp, d, g.ho, g.wo)) {
+    if (plan_wgrad_patch(wp, d, g.ho, g.wo, h->gemm_ctas < kWgradTargetCtas ? h->gemm_ctas : kWgradTargetCtas)) {
         wp.partials = reinterpret_cast<int32_t *>(ws + tap_bytes + 256 + acc_bytes);
         wp.dev = h->dev;
         cudaError_t e;
@@ -954,7 +963,7 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     // a 64-pixel stage adds at most 64 * 127 * 255 to an int32 partial sum: cap the stages one CTA runs
     const int max_stages_exact = 1024;
     const int tiles = p.num_m_groups * p.num_n_tiles;
-    int splits = (2 * h->sm_count + tiles - 1) / tiles;
+    int splits = (2 * h->gemm_ctas + tiles - 1) / tiles;
     const int max_splits = (total_stages + 7) / 8;  // at least 8 stages of work per CTA
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;

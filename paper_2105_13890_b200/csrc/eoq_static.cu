@@ -66,6 +66,7 @@ extern "C" int eoq_conv_dgrad_static(const eoq_conv_desc_t *desc, const int8_t *
     h.num_records = 0;
     h.records = nullptr;
     h.branch = nullptr;
+    h.gemm_ctas = pd.sm_count;
     h.fork_ev = h.join_ev = nullptr;
     st = eoq_conv_dgrad(reinterpret_cast<eoq_handle_t>(&h), desc, e3, e3_exp, w, e4, e4_exp, sum_e4, nullptr,
                         pd.scratch + kStaticHeaderBytes, kStaticScratchBytes, stream);

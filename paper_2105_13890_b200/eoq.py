@@ -24,7 +24,7 @@ EOQ_PASS_FWD, EOQ_PASS_DGRAD, EOQ_PASS_WGRAD = 0, 1, 2
 EXPORTS = [
     "eoq_create", "eoq_destroy", "eoq_workspace_size", "eoq_conv_fwd", "eoq_conv_dgrad", "eoq_conv_wgrad",
     "eoq_quantize", "eoq_quantize_image", "eoq_err_prescale", "eoq_update", "eoq_layout_convert", "eoq_last_status",
-    "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count",
+    "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count", "eoq_set_gemm_ctas",
     "eoq_conv_dgrad_static",
 ]
 EOQ_STATIC_SCRATCH_BYTES = 16 << 20
@@ -86,6 +86,7 @@ def lib() -> C.CDLL:
         L.eoq_profile_start.argtypes = [vp]
         L.eoq_profile_stop.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_double)]
         L.eoq_launch_count.argtypes = [vp]
+        L.eoq_set_gemm_ctas.argtypes = [vp, C.c_int]
         L.eoq_status_string.argtypes = [C.c_int]
         L.eoq_status_string.restype = C.c_char_p
         for name in EXPORTS:
@@ -238,6 +239,11 @@ def eoq_profile_stop(handle):
     ms = (C.c_double * EOQ_PROF_KINDS)()
     _check(lib().eoq_profile_stop(handle, n, ms), "eoq_profile_stop")
     return list(n), list(ms)
+
+
+def eoq_set_gemm_ctas(handle, ctas: int) -> None:
+    """Caps the CTAs the handle's GEMM launches use (0 = one per SM)."""
+    _check(lib().eoq_set_gemm_ctas(handle, ctas), "eoq_set_gemm_ctas")
 
 
 def eoq_launch_count(handle) -> int:

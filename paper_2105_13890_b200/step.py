@@ -87,6 +87,11 @@ class TrainStep:
         dev_index = self.dev.index if self.dev.index is not None else 0
         self.h_sides = [eoq.eoq_create(dev_index) for _ in range(side_streams)]
         self.workspace_sides = [torch.empty(ws, dtype=torch.uint8, device=self.dev) for _ in range(side_streams)]
+        # the weight-gradient GEMMs of the side streams take half of the SMs each: two of them then run side by side
+        # (and beside the helper kernels of the main chain) instead of one after the other
+        half = torch.cuda.get_device_properties(self.dev).multi_processor_count // 2
+        for hs in self.h_sides:
+            eoq.eoq_set_gemm_ctas(hs, half)
         self.sides = [torch.cuda.Stream(device=self.dev) for _ in range(side_streams)]
         self.graph = None
         first = workload.layers[0]

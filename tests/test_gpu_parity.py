@@ -339,3 +339,35 @@ def test_argument_errors_launch_nothing():
     assert eoq.eoq_conv_fwd(h, eoq.conv_desc(1, 8, 8, 8, 16, 7, 7, 2, 3, 4), x, None, 0, w, 128, 0, None, True, y, None, None, None, ws, check=False) == eoq.EOQ_ERR_UNSUPPORTED
     assert eoq.eoq_conv_dgrad(h, eoq.conv_desc(1, 8, 8, 8, 16, 7, 7, 2, 3, 5), y, ex, w, x, ex, None, None, ws, check=False) == eoq.EOQ_ERR_UNSUPPORTED
     assert G.status_clear() == 0
+
+
+@pytest.mark.parametrize("ctas", [1, 37, 74])
+def test_gemm_cta_cap_does_not_change_results(ctas):
+    """eoq_set_gemm_ctas only changes how many persistent CTAs walk the tiles: every output stays bit-identical
+    to the oracle."""
+    d = ConvDesc(6, 14, 14, 64, 128, 3, 3, 1, 1)
+    x0, w, sc, e3 = layer_data(d, 4100 + ctas)
+    gd = G.gdesc(d)
+    h = eoq.eoq_create(0)
+    eoq.eoq_set_gemm_ctas(h, ctas)
+    ref = oracle.layer_forward(d, x0, -3, w, 90, 5, sc, True)
+    x5 = G.zeros(ref["x5"].shape, torch.int8)
+    eoq.eoq_conv_fwd(h, gd, G.dev(x0), None, -3, G.dev(w), 90, 5, G.dev(sc), True, x5, None, None, None,
+                     G.workspace(gd, eoq.EOQ_PASS_FWD))
+    assert np.array_equal(G.host(x5), ref["x5"])
+    B = oracle.conv_dgrad_acc(d, e3, w)
+    e4_ref, p4, _ = oracle.sq_int(B, -9 - 7)
+    e4, e4_exp = G.zeros(x0.shape, torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_conv_dgrad(h, gd, G.dev(e3), G.dev(np.array([-9], dtype=np.int32)), G.dev(w), e4, e4_exp, None, None,
+                       G.workspace(gd, eoq.EOQ_PASS_DGRAD))
+    assert np.array_equal(G.host(e4).astype(np.int32), e4_ref) and e4_exp.item() == p4
+    Gacc = oracle.conv_wgrad_acc(d, e3, x0, -3)
+    g_ref, pg, _ = oracle.sq_int(Gacc, -9 - 7)
+    g_d, g_exp = G.zeros(Gacc.shape, torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_conv_wgrad(h, gd, G.dev(e3), G.dev(np.array([-9], dtype=np.int32)), G.dev(x0), -3, g_d, g_exp, None,
+                       G.workspace(gd, eoq.EOQ_PASS_WGRAD))
+    assert np.array_equal(G.host(g_d).astype(np.int32), g_ref) and g_exp.item() == pg
+    assert eoq.eoq_last_status(h) == 0
+    with pytest.raises(eoq.EoqError):
+        eoq.eoq_set_gemm_ctas(h, -1)
+    eoq.eoq_destroy(h)
