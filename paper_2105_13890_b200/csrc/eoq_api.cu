@@ -368,6 +368,10 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
     h->records = nullptr;
     h->branch = nullptr;
     h->fork_ev = h->join_ev = nullptr;
+    for (int k = 0; k < kClassBranches; ++k) {
+        h->class_branch[k] = nullptr;
+        h->class_join[k] = nullptr;
+    }
     cudaDeviceProp prop;
     cudaError_t e = cudaGetDeviceProperties(&prop, device);
     if (e == cudaSuccess) {
@@ -383,8 +387,16 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->branch, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->fork_ev, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->join_ev, cudaEventDisableTiming);
+    for (int k = 0; k < kClassBranches && e == cudaSuccess; ++k) {
+        e = cudaStreamCreateWithFlags(&h->class_branch[k], cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->class_join[k], cudaEventDisableTiming);
+    }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
+        for (int k = 0; k < kClassBranches; ++k) {
+            if (h->class_join[k]) cudaEventDestroy(h->class_join[k]);
+            if (h->class_branch[k]) cudaStreamDestroy(h->class_branch[k]);
+        }
         if (h->join_ev) cudaEventDestroy(h->join_ev);
         if (h->fork_ev) cudaEventDestroy(h->fork_ev);
         if (h->branch) cudaStreamDestroy(h->branch);
@@ -402,6 +414,10 @@ extern "C" int eoq_destroy(eoq_handle_t handle)
     if (!h) return EOQ_ERR_BAD_ARG;
     cudaSetDevice(h->device);
     cudaDeviceSynchronize();
+    for (int k = 0; k < kClassBranches; ++k) {
+        if (h->class_join[k]) cudaEventDestroy(h->class_join[k]);
+        if (h->class_branch[k]) cudaStreamDestroy(h->class_branch[k]);
+    }
     if (h->join_ev) cudaEventDestroy(h->join_ev);
     if (h->fork_ev) cudaEventDestroy(h->fork_ev);
     if (h->branch) cudaStreamDestroy(h->branch);
@@ -772,6 +788,34 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         e = cudaMemsetAsync(sums, 0, g.in_elems * sizeof(int32_t), s);
         if (e != cudaSuccess) return record(h, e);
     }
+    // The classes write disjoint pixels, so their GEMMs are independent: with more than one class and branch streams
+    // at hand they are issued side by side (fork on `s`, one stream per class, joins before Q_e), each with a
+    // share of the CTAs in proportion to its taps, instead of one after the other at full width.
+    int total_taps = 0, live_classes = 0;
+    for (int py = 0; py < d.stride && py < d.h; ++py)
+        for (int px = 0; px < d.stride && px < d.w; ++px) {
+            int nh = 0, nw = 0;
+            for (int kh = 0; kh < d.kh; ++kh) nh += (py + d.pad - kh) % d.stride == 0;
+            for (int kw = 0; kw < d.kw; ++kw) nw += (px + d.pad - kw) % d.stride == 0;
+            total_taps += nh * nw;
+            live_classes += nh * nw > 0;
+        }
+    // (worth it only while a class alone cannot keep the device busy for more than a wave of tiles)
+    const long long class_tiles = ((long long)d.n * ((d.h + d.stride - 1) / d.stride) * ((d.w + d.stride - 1) / d.stride) +
+                                   kTileM - 1) / kTileM * ((d.c_in + 255) / 256);
+    const bool side_by_side = live_classes > 1 && h->class_branch[0] != nullptr && class_tiles <= h->gemm_ctas;
+    // timed as one group on `s` (fork to join): the brackets of kernels that run side by side would overlap
+    ProfScope *group = side_by_side ? new (std::nothrow) ProfScope(h, EOQ_PROF_IGEMM_DGRAD, s) : nullptr;
+    struct GroupEnd {
+        ProfScope *&g;
+        ~GroupEnd() { delete g; }
+    } group_end{group};
+    if (side_by_side) {
+        e = cudaEventRecord(h->fork_ev, s);
+        if (e != cudaSuccess) return record(h, e);
+    }
+    int class_no = 0;
+    unsigned joins = 0;
     for (int py = 0; py < d.stride && py < d.h; ++py)
         for (int px = 0; px < d.stride && px < d.w; ++px) {
             IgemmParams p;
@@ -825,12 +869,37 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                 return EOQ_ERR_UNSUPPORTED;
             const int tiles = p.num_m_tiles * p.num_n_tiles;
             count_launches(h, 1);
-            {
-                ProfScope prof(h, EOQ_PROF_IGEMM_DGRAD, s);
-                e = launch_igemm(p, map_a, map_b, persistent_grid(tiles, h->gemm_ctas), s);
+            cudaStream_t cs = s;
+            int ctas = h->gemm_ctas;
+            if (side_by_side) {
+                ctas = (int)((long long)h->gemm_ctas * (nh * nw) / total_taps);
+                if (ctas < 1) ctas = 1;
+                if (class_no > 0) {
+                    const int k = (class_no - 1) % kClassBranches;
+                    cs = h->class_branch[k];
+                    // a stream that already carries a class of this call simply queues the next one behind it
+                    if (!(joins & (1u << k))) e = cudaStreamWaitEvent(cs, h->fork_ev, 0);
+                    if (e != cudaSuccess) return record(h, e);
+                    joins |= 1u << k;
+                }
+            }
+            ++class_no;
+            if (side_by_side) {
+                e = launch_igemm(p, map_a, map_b, persistent_grid(tiles, ctas), cs);
+            } else {
+                ProfScope prof(h, EOQ_PROF_IGEMM_DGRAD, cs);
+                e = launch_igemm(p, map_a, map_b, persistent_grid(tiles, ctas), cs);
             }
             if (e != cudaSuccess) return record(h, e);
         }
+    for (int k = 0; k < kClassBranches; ++k)
+        if (joins & (1u << k)) {
+            e = cudaEventRecord(h->class_join[k], h->class_branch[k]);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(s, h->class_join[k], 0);
+            if (e != cudaSuccess) return record(h, e);
+        }
+    delete group;  // closes the group's bracket on `s`, behind the joins
+    group = nullptr;
     // Q_e over the whole tensor: the maximum is complete only now
     {
         ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);

@@ -30,6 +30,8 @@ struct DeviceState {
 // no call starts with a memset.  A kernel that gave up on a wait (EOQ_DEV_TIMEOUT) may leave them dirty:
 // eoq_last_status clears them again when it reports that bit.
 
+constexpr int kClassBranches = 3;
+
 struct ProfRecord {
     int kind;
     cudaEvent_t begin, end;
@@ -50,6 +52,10 @@ struct Handle {
     int gemm_ctas;                // most CTAs a GEMM launch of this handle may use (eoq_set_gemm_ctas; default: one per SM)
     cudaStream_t branch;
     cudaEvent_t fork_ev, join_ev;
+    // further branch streams: the per-class GEMMs of a strided error back-propagation write disjoint pixels and
+    // run side by side, each with its share of the CTAs
+    cudaStream_t class_branch[kClassBranches];
+    cudaEvent_t class_join[kClassBranches];
 };
 constexpr int kMaxProfRecords = 8192;
 

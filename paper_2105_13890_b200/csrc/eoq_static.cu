@@ -68,6 +68,10 @@ extern "C" int eoq_conv_dgrad_static(const eoq_conv_desc_t *desc, const int8_t *
     h.branch = nullptr;
     h.gemm_ctas = pd.sm_count;
     h.fork_ev = h.join_ev = nullptr;
+    for (int k = 0; k < kClassBranches; ++k) {
+        h.class_branch[k] = nullptr;
+        h.class_join[k] = nullptr;
+    }
     st = eoq_conv_dgrad(reinterpret_cast<eoq_handle_t>(&h), desc, e3, e3_exp, w, e4, e4_exp, sum_e4, nullptr,
                         pd.scratch + kStaticHeaderBytes, kStaticScratchBytes, stream);
     if (st != EOQ_OK) return st;
