@@ -1126,11 +1126,13 @@ extern "C" int eoq_err_prescale(eoq_handle_t handle, const int8_t *e0, const int
     if (!aligned16(e0) || !aligned16(e3) || !aligned16(x2) || (reinterpret_cast<uintptr_t>(relu_mask) & 1)) return EOQ_ERR_ALIGNMENT;
     if (gamma_c < -32768 || gamma_c > 32767) return EOQ_ERR_RANGE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    count_launches(h, 2);
     ProfScope prof(h, EOQ_PROF_ERR_HEAD, s);
-    return record(h, launch_err_prescale(e0, e0_exp, relu_mask, x2, n_el, gamma_c, e3, e3_exp,
-                                         reinterpret_cast<long long *>(sum_e1), reinterpret_cast<long long *>(sum_e1x2),
-                                         h->dev, h->sm_count, s));
+    int kernels = 0;
+    const cudaError_t e = launch_err_prescale(e0, e0_exp, relu_mask, x2, n_el, gamma_c, e3, e3_exp,
+                                              reinterpret_cast<long long *>(sum_e1), reinterpret_cast<long long *>(sum_e1x2),
+                                              h->dev, h->sm_count, s, &kernels);
+    count_launches(h, kernels);
+    return record(h, e);
 }
 
 extern "C" int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const int8_t *const *g,

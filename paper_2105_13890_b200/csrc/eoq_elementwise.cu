@@ -944,9 +944,10 @@ cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_
 
 cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const uint8_t *mask, const int16_t *x2,
                                 size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
-                                long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s)
+                                long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s, int *kernels)
 {
     const size_t n16 = n_el / 16;
+    *kernels = 2;
     // one cooperative kernel when every thread can hold its share of the tensor between the two passes
     static int blocks_per_sm = -1;
     static bool coop = false;
@@ -966,6 +967,7 @@ cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const u
     if (coop && n16 > 0 && need_blocks <= max_blocks) {
         void *args[] = {(void *)&e0, (void *)&e0_exp, (void *)&mask, (void *)&x2, (void *)&n16, (void *)&gamma_c,
                         (void *)&e3, (void *)&e3_exp, (void *)&sum_e1, (void *)&sum_e1x2, (void *)&dev};
+        *kernels = 1;
         return cudaLaunchCooperativeKernel((const void *)prescale_fused_kernel, dim3((unsigned)need_blocks), dim3(kThreads),
                                            args, 0, s);
     }

@@ -229,7 +229,7 @@ cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_
                           cudaStream_t s);
 cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const uint8_t *mask, const int16_t *x2,
                                 size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
-                                long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s);
+                                long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s, int *kernels);
 struct UpdateTensor {
     int8_t *w;
     const int8_t *g;
