@@ -22,10 +22,16 @@
  *     16-byte aligned.  Scratch memory is the caller's `workspace` (device, 256-byte
  *     aligned, at least eoq_workspace_size() bytes; contents are undefined on
  *     entry and on return).  The handle owns only a few hundred bytes of device
- *     state (status word, small reduction cells).
+ *     state (status word, small reduction cells) and a few internal streams and
+ *     events.  A handle serves one call at a time: calls that may overlap on the
+ *     device (different streams) need a handle and a workspace each.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls enqueue work and return without synchronising, except
- *     eoq_create, eoq_destroy and eoq_last_status.
+ *     eoq_create, eoq_destroy and eoq_last_status.  A call may issue independent
+ *     parts of its work on the handle's internal streams, forked from and joined
+ *     back into `stream` with events (under stream capture these become graph
+ *     edges); when the call returns, everything it enqueued is ordered before
+ *     whatever is enqueued on `stream` next.
  *   - Every function returns an eoq_status_t.  Nothing throws, traps or aborts.
  *     Conditions only the device can see (a wait that ran out, a non-finite
  *     input, an all-zero SQ input) are OR-ed into the handle's device status
@@ -219,7 +225,7 @@ EOQ_API int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits);
 #define EOQ_PROF_IGEMM_DGRAD 1   /* the dgrad implicit-GEMM kernel, one launch per group */
 #define EOQ_PROF_WGRAD 2         /* the weight-gradient GEMM kernel */
 #define EOQ_PROF_ERR_HEAD 3      /* eoq_err_prescale (two kernels) */
-#define EOQ_PROF_DGRAD_AUX 4     /* weight transpose, Q_e phase 2 */
+#define EOQ_PROF_DGRAD_AUX 4     /* weight transpose (strided, 1x1 and small-image layers), Q_e phase 2 */
 #define EOQ_PROF_WGRAD_AUX 5     /* b1 error sums, Q_g */
 #define EOQ_PROF_FWD_AUX 6       /* b1 weight table, weight row padding */
 #define EOQ_PROF_OTHER 7         /* quantizers, update, layout change */
