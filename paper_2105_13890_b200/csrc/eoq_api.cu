@@ -769,13 +769,17 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             return record(h, e);
         }
     }
-    // the per-class GEMMs read the weights K-major: [c_in][tap][c_out]
-    {
-        ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
-        e = launch_weight_transpose(w, wt, d.c_out, g.taps, d.c_in, s);
+    // With at least 32 output channels per K chunk the per-class GEMMs read the weights in place as MN-major atoms
+    // (as the patch kernel does); narrower layers read a K-major transposed copy [c_in][tap][c_out].
+    const bool weights_in_place = d.c_out % 32 == 0;
+    if (!weights_in_place) {
+        {
+            ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
+            e = launch_weight_transpose(w, wt, d.c_out, g.taps, d.c_in, s);
+        }
+        if (e != cudaSuccess) return record(h, e);
+        count_launches(h, 1);
     }
-    if (e != cudaSuccess) return record(h, e);
-    count_launches(h, 1);
     // a class no tap reaches (e.g. the odd pixels of a strided 1x1 filter) keeps zero sums: clear first
     bool any_empty = false;
     for (int r = 0; r < d.stride; ++r) {
@@ -864,8 +868,13 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             p.acc_out = sums;
             p.dev = h->dev;
             CUtensorMap map_a, map_b;
+            if (weights_in_place) {
+                p.b_mn = 1;
+                p.b_row = chunk_bytes(p.tile_n);
+            }
             if (!make_im2col_map(&map_a, e3, d.n, g.ho, g.wo, d.c_out, min_w, min_h, wq, hq, 1, p.kc, kTileM) ||
-                !make_weight_map(&map_b, wt, d.c_in, g.taps, d.c_out, p.kc, p.tile_n))
+                !(weights_in_place ? make_weight_map(&map_b, w, d.c_out, g.taps, d.c_in, p.b_row, p.kc)
+                                   : make_weight_map(&map_b, wt, d.c_in, g.taps, d.c_out, p.kc, p.tile_n)))
                 return EOQ_ERR_UNSUPPORTED;
             const int tiles = p.num_m_tiles * p.num_n_tiles;
             count_launches(h, 1);
@@ -890,7 +899,10 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                 ProfScope prof(h, EOQ_PROF_IGEMM_DGRAD, cs);
                 e = launch_igemm(p, map_a, map_b, persistent_grid(tiles, ctas), cs);
             }
-            if (e != cudaSuccess) return record(h, e);
+            if (e != cudaSuccess) {
+                launch_reset_cells(h->dev, s);  // GEMMs already queued have touched the maximum cell
+                return record(h, e);
+            }
         }
     for (int k = 0; k < kClassBranches; ++k)
         if (joins & (1u << k)) {

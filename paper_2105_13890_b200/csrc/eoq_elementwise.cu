@@ -967,9 +967,13 @@ cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const u
     if (coop && n16 > 0 && need_blocks <= max_blocks) {
         void *args[] = {(void *)&e0, (void *)&e0_exp, (void *)&mask, (void *)&x2, (void *)&n16, (void *)&gamma_c,
                         (void *)&e3, (void *)&e3_exp, (void *)&sum_e1, (void *)&sum_e1x2, (void *)&dev};
-        *kernels = 1;
-        return cudaLaunchCooperativeKernel((const void *)prescale_fused_kernel, dim3((unsigned)need_blocks), dim3(kThreads),
-                                           args, 0, s);
+        const cudaError_t e = cudaLaunchCooperativeKernel((const void *)prescale_fused_kernel, dim3((unsigned)need_blocks),
+                                                          dim3(kThreads), args, 0, s);
+        if (e != cudaErrorCooperativeLaunchTooLarge) {
+            *kernels = 1;
+            return e;
+        }
+        (void)cudaGetLastError();  // fewer SMs at hand than at start-up (e.g. a partitioned device): two kernels instead
     }
     prescale_reduce_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, mask, x2, n16, dev);
     prescale_apply_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, e0_exp, mask, n16, gamma_c, e3, e3_exp,

@@ -106,9 +106,17 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                         const int tap = sd / p.chunks_per_tap, chunk = sd % p.chunks_per_tap;
                         ptx::tma_load_im2col_4d(a_dst + j * a_sub, &map_a, full_bar(stage), chunk * p.kc, cw, ch, img,
                                                 (uint16_t)p.tap_dw[tap], (uint16_t)p.tap_dh[tap]);
-                        // tap coordinate p.ntaps lies outside the weight tensor: the padding sub-tile is zero-filled
-                        ptx::tma_load_3d(b_dst + j * b_sub, &map_b, full_bar(stage), chunk * p.kc,
-                                         s < p.real_sub ? (int)p.tap_b[tap] : 0x7fff, nt * p.tile_n);
+                        if (p.b_mn) {
+                            // weights in place, [reduction rows][tap][columns]: tile_n / b_row atoms of [kc rows][b_row bytes]
+                            const uint32_t atom = (uint32_t)p.kc * p.b_row;
+                            for (int a = 0, na = p.tile_n / p.b_row; a < na; ++a)
+                                ptx::tma_load_3d(b_dst + j * b_sub + a * atom, &map_b, full_bar(stage),
+                                                 nt * p.tile_n + a * p.b_row, (int)p.tap_b[tap], chunk * p.kc);
+                        } else {
+                            // tap coordinate p.ntaps lies outside the weight tensor: the padding sub-tile is zero-filled
+                            ptx::tma_load_3d(b_dst + j * b_sub, &map_b, full_bar(stage), chunk * p.kc,
+                                             s < p.real_sub ? (int)p.tap_b[tap] : 0x7fff, nt * p.tile_n);
+                        }
                     }
                     inflight |= 1u << stage;
                     inflight_parity = (inflight_parity & ~(1u << stage)) | (phase << stage);
@@ -129,7 +137,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         const uint32_t leader = elect_one();
         const uint32_t tmem_base = __shfl_sync(0xffffffffu, tmem_base_s, 0);
         // ------------------------------------------------------------------ MMA issuer
-        const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, false, false);
+        const uint32_t idesc = make_idesc_i8(kTileM, p.tile_n, false, p.b_mn != 0);
         // Descriptors are assembled from precomputed halves; the loop only adds offsets in 16-byte units.
         // kc >= 32: swizzled K-major sub-tiles, rows kc bytes wide, 8-row groups 8*kc apart; a 32-byte K step
         // moves the start address inside the swizzle span.  kc == 16: no swizzle, one MMA spans two sub-tiles
@@ -137,7 +145,23 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         const bool wide = p.kc >= 32;
         const uint32_t hi = wide ? smem_desc_hi(8u * p.kc, layout_type_for(p.kc)) : smem_desc_hi(128, 0);
         const uint32_t a_sub16 = a_sub >> 4, b_sub16 = b_sub >> 4;
-        const uint32_t a_lead = wide ? 0u : (a_sub16 << 16), b_lead = wide ? 0u : (b_sub16 << 16);
+        const uint32_t a_lead = wide ? 0u : (a_sub16 << 16);
+        uint32_t b_lead = wide ? 0u : (b_sub16 << 16);
+        // B read MN-major (only with kc >= 32): atoms kc * b_row apart along the columns (leading offset), 8-row
+        // groups 8 * b_row apart (stride offset); 16-byte rows carry no swizzle and the two offsets swap roles; a
+        // 32-deep K step is 32 rows of an atom
+        uint32_t b_hi = hi, b_k16 = 2u;
+        if (p.b_mn) {
+            const uint32_t atom = (uint32_t)p.kc * p.b_row;
+            if (p.b_row == 16) {
+                b_hi = smem_desc_hi(atom, 0);
+                b_lead = (128u >> 4) << 16;
+            } else {
+                b_hi = smem_desc_hi(8u * p.b_row, layout_type_for(p.b_row));
+                b_lead = ((atom >> 4) & 0x3FFFu) << 16;
+            }
+            b_k16 = (32u * p.b_row) >> 4;
+        }
         const int sub_step = wide ? 1 : 2, k_steps = wide ? p.kc / 32 : 1;
         int stage = 0, acc = 0;
         uint32_t phase = 0, acc_phase = 0;
@@ -157,8 +181,8 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                 if (wide && k_steps >= 2) {
                     // 2 or 4 MMAs per sub-tile, alternating between the two partial accumulators
                     for (int j = 0; j < subs; ++j) {
-                        if (k_steps == 4) mma_k_steps<4>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1, leader, hi, 2u);
-                        else mma_k_steps<2>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1, leader, hi, 2u);
+                        if (k_steps == 4) mma_k_steps<4>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1, leader, b_hi, b_k16);
+                        else mma_k_steps<2>(d_tmem, d_other, a_lo, b_lo, hi, idesc, 0, fresh0, fresh1, leader, b_hi, b_k16);
                         fresh0 = 0;
                         fresh1 = 0;
                         a_lo += a_sub16;
@@ -168,7 +192,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                     for (int j = 0; j < subs; j += sub_step) {
                         // one MMA per step; with two accumulators successive steps alternate
                         const bool odd = nacc == 2 && (accumulate & 2u);
-                        ptx::mma_i8(odd ? d_other : d_tmem, smem_desc_join(a_lo, hi), smem_desc_join(b_lo, hi), idesc,
+                        ptx::mma_i8(odd ? d_other : d_tmem, smem_desc_join(a_lo, hi), smem_desc_join(b_lo, b_hi), idesc,
                                     odd ? (fresh1 ? 0u : 1u) : (fresh0 ? 0u : 1u), leader);
                         if (odd) fresh1 = 0; else fresh0 = 0;
                         if (nacc == 2) accumulate ^= 2u;
