@@ -26,7 +26,7 @@ INT8_OVER_BF16 = 2.0  # nominal dense ratio (4.5 / 2.25 PFLOP/s)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the implicit-GEMM kernels (forward + dgrad), averaged
 # over the launches of one step, from the one-pass ncu capture summarised in
 # profiles/dram_traffic_gemm_kernels_fixup_resnet18_b64_224.md; other workloads have no capture
-IGEMM_DRAM_BYTES_PER_LAUNCH = {"fixup_resnet18_b64_224": 7.57e6}
+IGEMM_DRAM_BYTES_PER_LAUNCH = {"fixup_resnet18_b64_224": 7.59e6}
 
 
 def peaks():
