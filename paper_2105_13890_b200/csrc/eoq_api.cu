@@ -788,7 +788,11 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         for (int kw = 0; kw < d.kw; ++kw) hit_w |= (r + d.pad - kw) % d.stride == 0;
         any_empty |= (r < d.h && !hit_h) || (r < d.w && !hit_w);
     }
-    if (any_empty) {
+    // A strided 1x1 filter without padding reaches only the pixels on the stride grid: its one GEMM leaves compact
+    // sums [n][hq][wq][c_in] and Q_e scatters them into the full tensor (zeros elsewhere), so nothing is cleared.
+    const bool compact = d.kh == 1 && d.kw == 1 && d.pad == 0 && d.stride > 1 && !acc_dump &&
+                         (size_t)d.n * d.h * d.w * (d.c_in / 16) <= 0xffffffffull;
+    if (any_empty && !compact) {
         e = cudaMemsetAsync(sums, 0, g.in_elems * sizeof(int32_t), s);
         if (e != cudaSuccess) return record(h, e);
     }
@@ -859,9 +863,9 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                     p.tap_dw[t] = (unsigned char)(dw[b] - min_w);
                     p.tap_b[t] = (unsigned char)(kh_of[a] * d.kw + kw_of[b]);
                 }
-            p.out_h = d.h;
-            p.out_w = d.w;
-            p.out_step = d.stride;
+            p.out_h = compact ? hq : d.h;
+            p.out_w = compact ? wq : d.w;
+            p.out_step = compact ? 1 : d.stride;
             p.out_off_h = py;
             p.out_off_w = px;
             p.epilogue = kEpiDgrad;
@@ -915,8 +919,13 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     // Q_e over the whole tensor: the maximum is complete only now
     {
         ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
-        e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
-                          h->sm_count, s);
+        if (compact)
+            e = launch_sq_i32_scatter(sums, e3_exp, -7, d.n, d.h, d.w, d.c_in, d.stride, (d.h + d.stride - 1) / d.stride,
+                                      (d.w + d.stride - 1) / d.stride, e4, e4_exp, reinterpret_cast<long long *>(sum_e4),
+                                      h->dev, h->sm_count, s);
+        else
+            e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
+                              h->sm_count, s);
     }
     count_launches(h, 1);
     return record(h, e);

@@ -288,6 +288,60 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
     }
 }
 
+// Q_e for a strided 1x1 filter: only the pixels (y, x) with y and x multiples of the stride receive an error, the
+// others are exactly zero.  The GEMM leaves its sums compact, [n][hq][wq][c]; this kernel writes the full tensor
+// [n][h][w][c], codes on the grid and zeros elsewhere, so neither a cleared full-size int32 tensor nor a pass over
+// it is needed.  A thread writes 16 channels of one pixel.
+__global__ void sq_i32_scatter_kernel(const int32_t *__restrict__ src, const int32_t *src_exp, int exp_bias, int n_img, int hh,
+                                      int ww, int c, int stride, int hq, int wq, int8_t *dst, int32_t *dst_exp,
+                                      long long *sum_codes, DeviceState *dev)
+{
+    const uint32_t M = dev->absmax_u32;
+    const int t = M ? round_log2_u32(M) : 7;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const int p_in = (src_exp ? *src_exp : 0) + exp_bias;
+        *dst_exp = M ? p_in + t - 7 : p_in;
+        if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+    }
+    long long sum = 0;
+    const uint32_t groups = (uint32_t)c / 16u;
+    const size_t items = (size_t)n_img * hh * ww * groups;  // fits 32 bits (checked by the launcher)
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
+        const uint32_t pix = (uint32_t)i / groups, g = (uint32_t)i - pix * groups;
+        const uint32_t row = pix / (uint32_t)ww, x = pix - row * (uint32_t)ww;
+        const uint32_t img = row / (uint32_t)hh, y = row - img * (uint32_t)hh;
+        int4 out = make_int4(0, 0, 0, 0);
+        if (y % (uint32_t)stride == 0 && x % (uint32_t)stride == 0) {
+            const size_t q = (((size_t)img * hq + y / (uint32_t)stride) * wq + x / (uint32_t)stride) * c + g * 16u;
+            const int4 *s4 = reinterpret_cast<const int4 *>(src + q);
+            int cdes[16];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int4 v = __ldcs(s4 + k);
+                cdes[4 * k + 0] = sq_code32(v.x, t);
+                cdes[4 * k + 1] = sq_code32(v.y, t);
+                cdes[4 * k + 2] = sq_code32(v.z, t);
+                cdes[4 * k + 3] = sq_code32(v.w, t);
+            }
+            int sc = 0;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) sc += cdes[k];
+            sum += sc;
+            out = make_int4((int)pack4(cdes[0], cdes[1], cdes[2], cdes[3]), (int)pack4(cdes[4], cdes[5], cdes[6], cdes[7]),
+                            (int)pack4(cdes[8], cdes[9], cdes[10], cdes[11]), (int)pack4(cdes[12], cdes[13], cdes[14], cdes[15]));
+        }
+        reinterpret_cast<int4 *>(dst)[i] = out;
+    }
+    if (sum_codes) {
+        sum = block_sum_i64(sum);
+        if (threadIdx.x == 0 && sum) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum0), (unsigned long long)sum);
+    }
+    if (last_block_done(dev)) {
+        if (sum_codes) *sum_codes = (long long)atomicExch(reinterpret_cast<unsigned long long *>(&dev->sum0), 0ull);
+        dev->absmax_u32 = 0;
+    }
+}
+
 // ------------------------------------------------------------------ int64 -> SQ (Q_g after the weight gradient)
 
 // Last step before Q_g: sums the int32 split-K slices of the patch kernel into int64 (exact whatever the reduction
@@ -923,6 +977,16 @@ cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bi
 {
     if (!max_already_reduced) absmax_i32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
     sq_i32_kernel<<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes, dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sq_i32_scatter(const int32_t *src, const int32_t *src_exp, int exp_bias, int n_img, int hh, int ww, int c,
+                                  int stride, int hq, int wq, int8_t *dst, int32_t *dst_exp, long long *sum_codes,
+                                  DeviceState *dev, int sm_count, cudaStream_t s)
+{
+    const size_t items = (size_t)n_img * hh * ww * (c / 16);
+    sq_i32_scatter_kernel<<<grid_for(items, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n_img, hh, ww, c, stride, hq, wq,
+                                                                        dst, dst_exp, sum_codes, dev);
     return cudaGetLastError();
 }
 

@@ -223,6 +223,9 @@ struct WgradCells {
     unsigned long long absmax;  // max |sum| over the weight tensor
     unsigned long long pad;
 };
+cudaError_t launch_sq_i32_scatter(const int32_t *src, const int32_t *src_exp, int exp_bias, int n_img, int hh, int ww, int c,
+                                  int stride, int hq, int wq, int8_t *dst, int32_t *dst_exp, long long *sum_codes,
+                                  DeviceState *dev, int sm_count, cudaStream_t s);
 cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int c_in,
                           const int32_t *parts, int num_parts, WgradCells *cells, DeviceState *dev, int sm_count,

@@ -371,3 +371,23 @@ def test_gemm_cta_cap_does_not_change_results(ctas):
     with pytest.raises(eoq.EoqError):
         eoq.eoq_set_gemm_ctas(h, -1)
     eoq.eoq_destroy(h)
+
+
+@pytest.mark.parametrize("d", [ConvDesc(2, 16, 16, 64, 128, 1, 1, 2, 0), ConvDesc(3, 9, 7, 32, 48, 1, 1, 2, 0),
+                               ConvDesc(2, 10, 10, 64, 64, 1, 1, 3, 0)],
+                         ids=["s2_even", "s2_odd_extents", "s3"])
+def test_strided_1x1_dgrad_without_sum_dump(d):
+    """Without an int32 dump a strided 1x1 filter takes the compact path (sums only on the stride grid, Q_e
+    scatters them): e4 must carry the oracle's codes on the grid and exact zeros elsewhere."""
+    _, w, _, e3 = layer_data(d, 5200 + d.h)
+    B = oracle.conv_dgrad_acc(d, e3, w)
+    ref, p4, _ = oracle.sq_int(B, -10 - 7)
+    gd = G.gdesc(d)
+    e4 = torch.full((d.n, d.h, d.w, d.c_in), 77, dtype=torch.int8, device="cuda:0")
+    e4_exp, s4 = G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+    for _ in range(2):  # twice: the reduction cells must come back clean
+        eoq.eoq_conv_dgrad(G.handle(), gd, G.dev(e3), G.dev(np.array([-10], dtype=np.int32)), G.dev(w), e4, e4_exp, s4, None,
+                           G.workspace(gd, eoq.EOQ_PASS_DGRAD))
+        assert G.status_clear() == 0
+        assert np.array_equal(G.host(e4).astype(np.int32), ref) and e4_exp.item() == p4
+        assert s4.item() == int(ref.astype(np.int64).sum())
