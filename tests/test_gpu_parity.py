@@ -291,6 +291,26 @@ def test_err_prescale(n_el, gamma):
     assert s1_d.item() == s1 and s2_d.item() == s2
 
 
+def test_err_prescale_two_kernel_path():
+    """Tensors too large for the one-kernel error head (more than 6 groups of 16 codes per resident thread) take
+    the reduce + apply pair; the first layer of the ImageNet networks at batch 64 is such a tensor."""
+    n_el = 14_720_000  # 920,000 groups of 16: above the one-kernel capacity of a 148-SM device (909,312 groups)
+    gamma = 118
+    e0 = synth.normal_codes(n_el, 610, 1)
+    mask = synth.bits(n_el, 611, 0)
+    p0 = -12
+    e3, p3, s1, _, _ = oracle.err_prescale(e0, p0, mask, None, gamma)
+    e3_d, e3_exp, s1_d = G.zeros(n_el, torch.int8), G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+    h = G.handle()
+    before = eoq.eoq_launch_count(h)
+    for _ in range(2):  # twice: the reduction cells must come back clean
+        eoq.eoq_err_prescale(h, G.dev(e0), G.dev(np.array([p0], dtype=np.int32)), G.dev(G.pack_mask(mask)), None, n_el,
+                             gamma, e3_d, e3_exp, s1_d, None)
+        assert G.status_clear() == 0
+        assert np.array_equal(G.host(e3_d), e3) and e3_exp.item() == p3 and s1_d.item() == s1
+    assert eoq.eoq_launch_count(h) - before == 4  # two kernels per call
+
+
 @pytest.mark.parametrize("stochastic", [False, True])
 def test_update_multi_tensor(stochastic):
     sizes = [16, 2304, 36864 + 5, 100000, 1, 8192, 8193]
