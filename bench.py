@@ -7,6 +7,11 @@ update of all weights.  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet18|resnet20|resnet50|single] [--batch B]
   python bench.py --impl reference ...     # the CPU oracle on host cores, same metric, bounded sample per step
+  python bench.py --probe mma_i8           # INT8 tensor-pipe denominators: own tcgen05.mma issue-rate probe + a library int8 matmul
+
+With --gpus N > 1 and no launcher environment the script starts N ranks of itself (one per GPU, rendezvous on
+127.0.0.1); under torchrun it is one of the ranks.  Every rank runs the whole per-GPU workload (replicas), rank 0
+prints the line.
 """
 from __future__ import annotations
 
@@ -23,10 +28,10 @@ sys.path.insert(0, ROOT)
 
 METRIC = "int8 conv TOPS per train step (fwd+dgrad+wgrad) and img/s, % of INT8 roofline"
 INT8_OVER_BF16 = 2.0  # nominal dense ratio (4.5 / 2.25 PFLOP/s)
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the implicit-GEMM kernels (forward + dgrad), averaged
-# over the launches of one step, from the one-pass ncu capture summarised in
-# profiles/dram_traffic_gemm_kernels_fixup_resnet18_b64_224.md; other workloads have no capture
-IGEMM_DRAM_BYTES_PER_LAUNCH = {"fixup_resnet18_b64_224": 7.59e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the implicit-GEMM kernels, from an ncu capture of the
+# present kernels (profiles/); None while no capture of the current kernels exists
+IGEMM_DRAM_BYTES_PER_LAUNCH = {}
+NOMINAL_INT8_TOPS = 4500.0  # public dense figure, context only
 
 
 def peaks():
@@ -102,7 +107,6 @@ def oracle_step(wl, seed, scal):
     import oracle
     from oracle import ConvDesc
     from paper_2105_13890_b200 import synth
-    from paper_2105_13890_b200.workloads import init_weight_f32
 
     b1_c, gamma_c, b2_c = scal
     # inputs first (not timed: the GPU arm's inputs are resident before its timed region too)
@@ -114,8 +118,10 @@ def oracle_step(wl, seed, scal):
         x0 = synth.relu_codes((l.n, l.h, l.w, l.c_in), seed, 1) if i else None
         e0 = synth.normal_codes((l.n, l.ho, l.wo, l.c_out), seed, 2)
         sc = synth.relu_codes((l.n, l.ho, l.wo, l.c_out), seed, 3) if l.shortcut else None
-        w = oracle.q_w(init_weight_f32(l, wl, synth.normal_f64((l.c_out, l.k, l.k, l.c_in), seed, 100 + i)))
-        data.append((l, d, x0, e0, sc, w))
+        wf = oracle.fixup_weights_f32(synth.normal_f64((l.c_out, l.k, l.k, l.c_in), seed, 100 + i),
+                                      l.c_in_true * l.k * l.k, wl.L, wl.m, l.in_branch)
+        wf[..., l.c_in_true:] = 0.0
+        data.append((l, d, x0, e0, sc, oracle.q_w(wf)))
     t0 = time.perf_counter()
     img = np.zeros((first.n, first.h, first.w, first.c_in), dtype=np.float32)
     img[..., :3] = image
@@ -140,7 +146,7 @@ def oracle_step(wl, seed, scal):
         g, pg, _ = oracle.sq_int(oracle.conv_wgrad_acc(d, e3, x0, 0 if i == 0 else b1_c), p3 - 7)
         grads.append((i, g.astype(np.int8), pg))
     for i, g, pg in grads:
-        oracle.update(data[i][5], g, pg, 1, -6, stochastic=True, seed=seed, step=0, tensor_id=i)
+        oracle.update(data[i][5], g, pg, 1, -6, stochastic=False)
     return time.perf_counter() - t0
 
 
@@ -177,6 +183,21 @@ def run_reference(args):
 
 # ----------------------------------------------------------------------------------------------- GPU arm
 
+def bandwidth_bytes(wl):
+    """Algorithmic bytes per step of the bandwidth-bound kernel groups (what the method itself must move)."""
+    head = dq = fin = upd = 0
+    for l in wl.layers:
+        n_out = l.n * l.ho * l.wo * l.c_out
+        head += n_out * (1 + 1 + 0.125 + (2 if l.gamma_trainable else 0))   # e0 in, e3 out, mask, x2 for g_gamma
+        if l.has_dgrad:
+            dq += l.n * l.h * l.w * l.c_in * (4 + 1)                        # exact int32 sums in, e4 codes out
+        fin += l.weight_elems * (4 + 1)                                     # exact sums in, g codes out
+        upd += l.weight_elems * 3                                           # g in, w in, w out
+    f = wl.layers[0]
+    inq = f.n * f.h * f.w * (3 * 4 * 2 + f.c_in)                            # fp32 image read twice (max, code), codes out
+    return {"err_head": head, "dgrad_aux": dq, "wgrad_aux": fin, "update": upd, "input_quantizer": inq}
+
+
 def run_gpu(args):
     import torch
 
@@ -192,7 +213,8 @@ def run_gpu(args):
 
     wl = workloads.get(args.workload, args.batch)
     handle = eoq.eoq_create(local)
-    step = TrainStep(wl, handle, f"cuda:{local}", scalars=Scalars())
+    round_mode = eoq.EOQ_ROUND_STOCHASTIC if args.stochastic else eoq.EOQ_ROUND_RNE
+    step = TrainStep(wl, handle, f"cuda:{local}", scalars=Scalars(), round_mode=round_mode)
     stream = torch.cuda.current_stream()
 
     # One step = one replay of a CUDA graph of the whole path (the weight-gradient chain of each layer on a side
@@ -265,7 +287,13 @@ def run_gpu(args):
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
-    # ---- per-kernel timing of the tensor-core kernels (events around each launch, same stream)
+    # ---- the convolution kernels alone, replayed back to back from their own graphs (forward: one GEMM launch per
+    # layer; dgrad: GEMM + Q_e; wgrad: the whole weight-gradient call), CUDA events around a run of replays on the
+    # launching stream.  This is the launch duration the roofline figure uses: event brackets around single launches
+    # add several microseconds of event overhead to kernels that last 10 to 30.
+    conv_ms = step.time_conv_passes(replays=max(3, min(10, args.steps)))
+
+    # ---- per-kind timing (events around each launch, eager, one stream)
     # Each eager step is queued behind a few milliseconds of device-side delay, so that the host has issued the
     # whole step before the device starts it: the events then bracket device time only, not host launch gaps.
     # The library keeps a bounded number of event pairs per profiling session (8192): profile as many steps as fit.
@@ -293,14 +321,21 @@ def run_gpu(args):
         sec = ms / 1e3 / args.steps
         tops = ranks.whole_job_rate(ops_step, args.steps, ms, world) / 1e12
         tops_e2e = ranks.whole_job_rate(ops_step, args.steps, ms_e2e, world) / 1e12
-        # the GEMM launches are timed one by one with events and the clocks stay at their maximum over the step
-        # (see "clocks"), so the burst bf16 figure is the denominator, not the power-capped sustained one
+        # the clocks stay at their maximum over the step (see "clocks"), so the burst bf16 figure is the denominator
         int8_peak = pk["bf16_burst"] * INT8_OVER_BF16
-        fwd_ops = sum(2 * l.macs for l in wl.layers) * prof_steps
-        dgrad_ops = sum(2 * l.macs for l in wl.layers if l.has_dgrad) * prof_steps
-        igemm_ms = prof_ms[0] + prof_ms[1]
-        igemm_n = prof_n[0] + prof_n[1]
-        achieved = (fwd_ops + dgrad_ops) / (igemm_ms / 1e3) / 1e12 if igemm_ms > 0 else None
+        fwd_ops = sum(2 * l.macs for l in wl.layers)
+        dgrad_ops = sum(2 * l.macs for l in wl.layers if l.has_dgrad)
+        n_fwd = len(wl.layers)
+        n_dgrad = sum(1 for l in wl.layers if l.has_dgrad)
+        igemm_ms = conv_ms["fwd"] + conv_ms["dgrad_gemm"]
+        achieved = (fwd_ops + dgrad_ops) / (igemm_ms / 1e3) / 1e12
+        names = eoq.EOQ_PROF_NAMES
+        by_kind = {name: prof_ms[i] / prof_steps for i, name in enumerate(names)}
+        bw = {}
+        for kind, nbytes in bandwidth_bytes(wl).items():
+            t_ms = by_kind.get(kind, 0.0)
+            gbs = nbytes / (t_ms / 1e3) / 1e9 if t_ms > 0 else None
+            bw[kind] = {"algorithmic_bytes": nbytes, "ms": t_ms, "gbs": gbs, "frac_of_hbm": gbs / pk["hbm_gbs"] if gbs else None}
         line = {
             "metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -309,7 +344,9 @@ def run_gpu(args):
             "pct_of_int8_peak": 100.0 * tops / world / int8_peak,
             "config": {"workload": wl.name, "layers": len(wl.layers), "global_batch": world * wl.batch,
                        "gop_per_step": ops_step / 1e9, "l2": "working set larger than L2; no flush between steps",
-                       "scalars": "b1=-2 gamma=118 b2=3 codes", "parallelism": f"replicas x{world}",
+                       "scalars": "b1=-2 gamma=118 b2=3 codes, device-resident",
+                       "update": "stochastic rounding (extension)" if args.stochastic else "round to nearest even (Sec. 3.2.2)",
+                       "parallelism": f"replicas x{world}",
                        "launch": "eager, one stream" if args.eager else "CUDA graph replay, wgrad chains on two side streams"},
             "clocks": clocks,
             "e2e": {"value": tops_e2e, "unit": "TOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -317,32 +354,129 @@ def run_gpu(args):
             "gpu_launches": int(launches),
             "device_status": int(status),
             "roofline": {
-                "kernel": "igemm_kernel (forward + dgrad implicit GEMM, tcgen05 kind::i8)", "bound": "tensor",
-                "achieved": achieved, "peak": int8_peak, "unit": "TOPS",
-                "frac": (achieved / int8_peak) if achieved else None,
+                "kernel": "igemm_kernel + igemm_patch_kernel (forward + dgrad implicit GEMM, tcgen05 kind::i8)",
+                "bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOPS", "frac": achieved / int8_peak,
                 "traffic": IGEMM_DRAM_BYTES_PER_LAUNCH.get(wl.name),
                 "peak_source": f"{pk['source']} burst bf16 {pk['bf16_burst']} TFLOP/s x {INT8_OVER_BF16} (nominal int8:bf16)",
-                "launches": igemm_n, "avg_launch_ms": igemm_ms / igemm_n if igemm_n else None,
+                "launches": n_fwd + n_dgrad, "avg_launch_ms": igemm_ms / (n_fwd + n_dgrad),
+                "timing": "graph replay of the launches back to back, CUDA events around the run",
+                "frac_of_nominal_4500": achieved / NOMINAL_INT8_TOPS,
+                "frac_of_sustained_bf16_x2": achieved / (pk["bf16_sustained"] * INT8_OVER_BF16),
             },
             "kernels": {
-                "igemm_fwd": {"launches": prof_n[0], "ms": prof_ms[0], "tops": fwd_ops / (prof_ms[0] / 1e3) / 1e12 if prof_ms[0] else None},
-                "igemm_dgrad": {"launches": prof_n[1], "ms": prof_ms[1], "tops": dgrad_ops / (prof_ms[1] / 1e3) / 1e12 if prof_ms[1] else None},
-                "wgrad": {"launches": prof_n[2], "ms": prof_ms[2], "tops": fwd_ops / (prof_ms[2] / 1e3) / 1e12 if prof_ms[2] else None},
+                "igemm_fwd": {"launches": n_fwd, "ms": conv_ms["fwd"], "tops": fwd_ops / (conv_ms["fwd"] / 1e3) / 1e12},
+                "igemm_dgrad": {"launches": n_dgrad, "ms": conv_ms["dgrad_gemm"],
+                                "tops": dgrad_ops / (conv_ms["dgrad_gemm"] / 1e3) / 1e12},
+                "dgrad_with_Qe": {"ms": conv_ms["dgrad"], "tops": dgrad_ops / (conv_ms["dgrad"] / 1e3) / 1e12},
+                "wgrad": {"launches": n_fwd, "ms": conv_ms["wgrad_gemm"], "tops": fwd_ops / (conv_ms["wgrad_gemm"] / 1e3) / 1e12},
+                "wgrad_with_Qg": {"ms": conv_ms["wgrad"], "tops": fwd_ops / (conv_ms["wgrad"] / 1e3) / 1e12},
             },
-            "ms_per_step_by_kind": {name: prof_ms[i] / prof_steps for i, name in enumerate(eoq.EOQ_PROF_NAMES)},
+            "bandwidth_kernels": bw,
+            "ms_per_step_by_kind": by_kind,
             "profiled_steps": prof_steps,
         }
+        if args.int8_peaks:
+            # the two measured INT8 figures next to the denominator in use (see --probe)
+            line["int8_peaks"] = json.loads(args.int8_peaks)
+            for k, v in line["int8_peaks"].items():
+                if isinstance(v, (int, float)) and v > 0 and k.endswith("_tops"):
+                    line["roofline"][f"frac_of_{k}"] = achieved / v
         if world == 1 and not args.no_cpu_baseline:
             import oracle
 
             oracle.build()
-            small = workloads.get(args.workload, args.ref_batch)
+            small = workloads.get(args.workload, args.ref_batch if args.ref_batch else wl.batch)
             secs = oracle_step(small, 1, (-2, 118, 3))
             line["cpu_baseline"] = {"value": small.total_ops / secs / 1e12, "unit": "TOPS", "cores": os.cpu_count(),
                                     "kind": "oracle", "seconds": secs,
-                                    "sample": f"{small.name}: every layer of the workload at batch {args.ref_batch}, one step"}
+                                    "sample": f"{small.name}: every layer of the workload at batch {small.batch}, one step"}
         print(json.dumps(line), flush=True)
     eoq.eoq_destroy(handle)
+    ranks.finish()
+
+
+# ----------------------------------------------------------------------------------------------- INT8 peak probe
+
+def run_probe(args):
+    """INT8 tensor-pipe figures to hold the roofline against: the library's own tcgen05.mma kind::i8 issue-rate probe
+    (operands in shared memory, every SM) and, as an independent library figure, an int8 matmul through torch."""
+    import torch
+
+    from paper_2105_13890_b200 import eoq
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --probe needs a CUDA device")
+    h = eoq.eoq_create(0)
+    out = {"probe": "mma_i8", "unit": "TOPS"}
+    sampler = ClockSampler(0)
+    t0 = time.time()
+    for n in (256, 128, 64):
+        burst, cyc = eoq.eoq_probe_mma_i8(h, n, 2048, 10)           # ~1 ms per launch
+        t_end = time.time() + args.probe_seconds
+        sustained = []
+        while time.time() < t_end:
+            sustained.append(eoq.eoq_probe_mma_i8(h, n, 8192, 50)[0])
+        out[f"mma_i8_n{n}_burst_tops"] = burst
+        out[f"mma_i8_n{n}_sustained_tops"] = sum(sustained[len(sustained) // 2:]) / max(1, len(sustained) - len(sustained) // 2)
+        out[f"mma_i8_n{n}_cycles_per_mma"] = cyc
+    assert eoq.eoq_last_status(h) == 0
+    # library int8 matmul, 8192^3 (measurement only; never on the layer's path)
+    try:
+        a = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device="cuda")
+        b = torch.randint(-8, 8, (8192, 8192), dtype=torch.int8, device="cuda").t()
+        for _ in range(3):
+            torch._int_mm(a, b)
+        best = None
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch._int_mm(a, b)
+            e1.record()
+            torch.cuda.synchronize()
+            t = e0.elapsed_time(e1)
+            best = t if best is None or t < best else best
+        out["library_int8_matmul_8192_tops"] = 2 * 8192 ** 3 / (best / 1e3) / 1e12
+    except Exception as ex:  # the library routine is optional: report why it is absent
+        out["library_int8_matmul_8192_tops"] = None
+        out["library_int8_matmul_error"] = str(ex)[:200]
+    out["clocks"] = ClockSampler.summarize(sampler.window(t0, time.time()))
+    sampler.stop()
+    pk = peaks()
+    out["denominator_in_bench_line"] = pk["bf16_burst"] * INT8_OVER_BF16
+    out["nominal_tops"] = NOMINAL_INT8_TOPS
+    eoq.eoq_destroy(h)
+    print(json.dumps(out), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------- launcher
+
+def launch_ranks(args, argv):
+    """--gpus N without a launcher environment: start N ranks of this script (torch.distributed.run, one node,
+    rendezvous on 127.0.0.1) and pass their output through; rank 0 prints the JSON line."""
+    import socket
+
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + argv
+    return subprocess.call(cmd)
+
+
+def run_dry(args):
+    """--dry-run: the rank plumbing alone (rendezvous, barrier, max-over-ranks of a stand-in timing, one JSON line
+    from rank 0) on CPU with gloo; what the multi-rank tests drive."""
+    from paper_2105_13890_b200 import ranks
+
+    world, rank, _ = ranks.world()
+    ranks.init("gloo")
+    ranks.barrier(sync_cuda=False)
+    ms = ranks.max_over_ranks([10.0 + rank], device="cpu")[0]
+    ranks.barrier(sync_cuda=False)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "n_gpus": world, "dry_run": True, "ms_per_step": ms / args.steps,
+                          "value": ranks.whole_job_rate(1e12, args.steps, ms, world) / 1e12, "unit": "TOPS",
+                          "scaling": "weak", "config": {"parallelism": f"replicas x{world}"}}), flush=True)
     ranks.finish()
 
 
@@ -354,14 +488,26 @@ def main():
     ap.add_argument("--impl", default="eoq", choices=["eoq", "reference"])
     ap.add_argument("--workload", default="resnet18")
     ap.add_argument("--batch", type=int, default=None)
-    ap.add_argument("--ref-batch", type=int, default=4, help="batch of the CPU-oracle sample timed beside the GPU run")
+    ap.add_argument("--ref-batch", type=int, default=0,
+                    help="batch of the CPU-oracle step timed beside the GPU run (0 = the workload's own batch)")
     ap.add_argument("--ref-arm-batch", type=int, default=1, help="batch of each step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eager", action="store_true", help="launch call by call on one stream instead of replaying a CUDA graph")
+    ap.add_argument("--stochastic", action="store_true", help="stochastic rounding in the update (an extension; default: nearest even)")
+    ap.add_argument("--probe", default=None, choices=["mma_i8"], help="measure the INT8 tensor-pipe figures and exit")
+    ap.add_argument("--probe-seconds", type=float, default=2.0, help="length of each sustained probe loop")
+    ap.add_argument("--int8-peaks", default=None, help="JSON printed by --probe, to report fractions of those figures too")
+    ap.add_argument("--dry-run", action="store_true", help="rank plumbing only, on CPU with gloo (tests)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(launch_ranks(args, sys.argv[1:]))
+    if args.dry_run:
+        run_dry(args)
+    elif args.probe:
+        run_probe(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

@@ -118,6 +118,35 @@ EOQ_API int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, const
                  size_t workspace_bytes, void *stream);
 
 /*
+ * The same forward chain for a training loop whose scalars live in device memory and whose weights change only in
+ * the update (Sec. 3.2.1, first equation block; Sec. 3.2.3 for what changes them).
+ *   scalars (device, three int32: b1_c, gamma_c, b2_c, codes at p = -7) replace the three host arguments: a step
+ *   recorded once into a CUDA graph then reads the current codes at every replay.  Codes outside 16 bits, or a b1
+ *   that would let the accumulator leave int32, raise EOQ_DEV_RANGE and are clamped.
+ *   w_prep (device, 256-byte aligned, eoq_weight_prep_size() bytes) holds what eoq_weight_prep derived from w: the
+ *   per-border-class weight sums of the b1 term and, on the filter-row path, the row-padded weights.  With w_prep
+ *   no helper kernel runs in front of the convolution.  w_prep = NULL states that the layer has no bias before its
+ *   convolution: scalars[0] must then be 0 (anything else raises EOQ_DEV_RANGE and counts as 0); the filter-row
+ *   path always needs w_prep.
+ * Everything else is as in eoq_conv_fwd; there is no accumulator dump and no workspace.
+ */
+EOQ_API int eoq_conv_fwd_dev(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *x, const int32_t *x_exp,
+                     const int32_t *scalars, const int8_t *w, const void *w_prep, const int8_t *shortcut, int relu,
+                     int8_t *x5, int16_t *x2, uint8_t *relu_mask, void *stream);
+
+/*
+ * What the forward pass needs from the weights besides the codes themselves (x1 = x0 + Q_b(b1) with a zero halo,
+ * Sec. 3.2.1: conv(x1) = conv(x0) + b1 * sum of the weights of the taps inside the image).  It depends on w and the
+ * geometry only, so it is formed once per weight version -- after initialisation and after every eoq_update --
+ * for `num` layers in one launch per 32 layers.
+ * host in   : descs[num]; arrays (host memory) of device pointers w[i] and prep[i] (256-byte aligned,
+ *             eoq_weight_prep_size(&descs[i]) bytes each).
+ */
+EOQ_API int eoq_weight_prep_size(const eoq_conv_desc_t *desc, size_t *bytes);
+EOQ_API int eoq_weight_prep(eoq_handle_t handle, int num, const eoq_conv_desc_t *descs, const int8_t *const *w,
+                    void *const *prep, void *stream);
+
+/*
  * Error back-propagation through the convolution (Sec. 3.2.1, second equation block):
  *   e4 = Q_e(e3 * Q_w(w)), the transposed convolution followed by SQ over the whole tensor.
  * device in : e3 [n,ho,wo,c_out] int8 with exponent *e3_exp; w.
@@ -164,6 +193,12 @@ EOQ_API int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
                    const int8_t *x, int32_t b1_c, int8_t *g, int32_t *g_exp, int64_t *acc_dump,
                    void *workspace, size_t workspace_bytes, void *stream);
 
+/* eoq_conv_wgrad with b1 read from device memory (one int32 code; NULL = the layer has no bias before its
+ * convolution).  No accumulator dump.  See eoq_conv_fwd_dev. */
+EOQ_API int eoq_conv_wgrad_dev(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                       const int8_t *x, const int32_t *b1_c, int8_t *g, int32_t *g_exp, void *workspace,
+                       size_t workspace_bytes, void *stream);
+
 /*
  * The three quantization functions (Sec. 3.2.2) on a flat tensor of n elements.
  *   src_is_float = 1: src is fp32.  Q -> int16 codes R(x * 2^7) (saturated to int16);
@@ -187,6 +222,11 @@ EOQ_API int eoq_err_prescale(eoq_handle_t handle, const int8_t *e0, const int32_
                      const int16_t *x2, size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp,
                      int64_t *sum_e1, int64_t *sum_e1x2, void *stream);
 
+/* eoq_err_prescale with gamma read from device memory (one int32 code, required).  See eoq_conv_fwd_dev. */
+EOQ_API int eoq_err_prescale_dev(eoq_handle_t handle, const int8_t *e0, const int32_t *e0_exp, const uint8_t *relu_mask,
+                         const int16_t *x2, size_t n_el, const int32_t *gamma_c, int8_t *e3, int32_t *e3_exp,
+                         int64_t *sum_e1, int64_t *sum_e1x2, void *stream);
+
 /*
  * The 8-bit update (Sec. 3.2.3, update quantization) on `num` weight tensors in one call:
  *   u = Q_u(lr * g) = SQ(lr * g, 8), lr = lr_mant * 2^lr_exp, lr_mant in [1, 255];
@@ -198,6 +238,12 @@ EOQ_API int eoq_err_prescale(eoq_handle_t handle, const int8_t *e0, const int32_
 EOQ_API int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const int8_t *const *g,
                const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp, int round_mode,
                uint64_t seed, uint64_t step, void *stream);
+
+/* eoq_update with the step counter in device memory (one uint64, 8-byte aligned): the update reads *step and the
+ * call increments it on the device afterwards, so that every replay of a captured step draws fresh rounding bits. */
+EOQ_API int eoq_update_dev(eoq_handle_t handle, int num, int8_t *const *w, const int8_t *const *g,
+                   const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp, int round_mode,
+                   uint64_t seed, uint64_t *step, void *stream);
 
 /*
  * Input quantizer for the network input (Sec. 5.1 quantizes every layer but the last): SQ(., 8) of an fp32
@@ -224,15 +270,23 @@ EOQ_API int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits);
 #define EOQ_PROF_IGEMM_FWD 0     /* the forward implicit-GEMM kernel, one launch per group */
 #define EOQ_PROF_IGEMM_DGRAD 1   /* the dgrad implicit-GEMM kernel, one launch per group */
 #define EOQ_PROF_WGRAD 2         /* the weight-gradient GEMM kernel */
-#define EOQ_PROF_ERR_HEAD 3      /* eoq_err_prescale (two kernels) */
-#define EOQ_PROF_DGRAD_AUX 4     /* weight transpose (strided, 1x1 and small-image layers), Q_e phase 2 */
-#define EOQ_PROF_WGRAD_AUX 5     /* b1 error sums, Q_g */
-#define EOQ_PROF_FWD_AUX 6       /* b1 weight table, weight row padding */
-#define EOQ_PROF_OTHER 7         /* quantizers, update, layout change */
-#define EOQ_PROF_KINDS 8
+#define EOQ_PROF_ERR_HEAD 3      /* eoq_err_prescale (one kernel; two for tensors beyond the one-kernel capacity) */
+#define EOQ_PROF_DGRAD_AUX 4     /* Q_e phase 2; weight transpose (only layers with fewer than 32 output channels) */
+#define EOQ_PROF_WGRAD_AUX 5     /* slice sum + b1 term + Q_g behind the weight-gradient GEMM (and the memset in front of it) */
+#define EOQ_PROF_FWD_AUX 6       /* b1 weight table, weight row padding (eoq_weight_prep, or per call without it) */
+#define EOQ_PROF_OTHER 7         /* eoq_quantize */
+#define EOQ_PROF_UPDATE 8        /* eoq_update */
+#define EOQ_PROF_INPUT_Q 9       /* eoq_quantize_image */
+#define EOQ_PROF_WGRAD_TAPS 10   /* b1 error sums of the weight gradient (on the handle's branch stream) */
+#define EOQ_PROF_KINDS 11
 EOQ_API int eoq_profile_start(eoq_handle_t handle);
 EOQ_API int eoq_profile_stop(eoq_handle_t handle, int launches[EOQ_PROF_KINDS], double milliseconds[EOQ_PROF_KINDS]);
 EOQ_API unsigned long long eoq_launch_count(eoq_handle_t handle);
+/* Timing aid: while on, eoq_conv_dgrad and eoq_conv_wgrad (and their _dev forms) on this handle launch their GEMM
+ * kernel only -- no quantizer behind it, no helper in front -- so the outputs of those calls are NOT produced; used
+ * to time the tensor-core kernels alone, back to back.  Synchronises the device; switching it off puts the handle's
+ * reduction cells back to zero. */
+EOQ_API int eoq_profile_gemm_only(eoq_handle_t handle, int on);
 
 /* Caps the CTAs (one per SM) that the GEMM launches of this handle use; 0 = one per SM of the device (the
  * default).  Every GEMM kernel is persistent: with fewer CTAs a launch walks more tiles per CTA and leaves the
@@ -241,6 +295,29 @@ EOQ_API unsigned long long eoq_launch_count(eoq_handle_t handle);
  * independent once e3 exists).  Results do not depend on the setting.  Host-side state only; applies to the calls
  * made after it. */
 EOQ_API int eoq_set_gemm_ctas(eoq_handle_t handle, int ctas);
+
+/*
+ * Measures what the tensor pipe delivers for the instruction all three convolution passes run on, tcgen05.mma
+ * kind::i8 with a 128 x n_cols x 32 shape (int8 x int8 -> int32, Sec. 3.2.1): one CTA per SM, operands resident in
+ * shared memory, two accumulators in tensor memory, `iters` x 4 MMAs per CTA and launch, `launches` launches timed
+ * with CUDA events on `stream`.  Synchronises.  *tops = operations (2 per multiply-add) per second / 1e12 over the
+ * timed launches, launch gaps included; *cycles_per_mma (optional) = SM clock cycles per MMA inside the longest
+ * issue loop.  n_cols: a multiple of 16 in [16, 256].  A measurement aid for roofline denominators, not part of
+ * the layer.
+ */
+EOQ_API int eoq_probe_mma_i8(eoq_handle_t handle, int n_cols, int iters, int launches, double *tops, double *cycles_per_mma,
+                     void *stream);
+
+/* One line of text saying which kernel and tiling a pass of this geometry takes on this handle (for tests and
+ * reports; the format is not an interface).  buf receives at most buf_bytes bytes, NUL-terminated. */
+EOQ_API int eoq_describe_plan(eoq_handle_t handle, const eoq_conv_desc_t *desc, int pass, char *buf, size_t buf_bytes);
+
+/* Self-test of the bounded device waits: the next eoq_err_prescale / eoq_err_prescale_dev call on this handle that
+ * takes the one-kernel path waits at its grid-wide barrier for one block more than exists, with a limit of 2048
+ * polls (about 0.2 ms).  The wait runs out, the kernel raises EOQ_DEV_TIMEOUT, writes no output and returns;
+ * eoq_last_status then reports the bit and puts the handle's reduction cells back to zero.  Nothing faults or
+ * hangs; one call only, then the handle behaves normally again. */
+EOQ_API int eoq_debug_force_wait_timeout(eoq_handle_t handle);
 
 /* The last cudaError_t a call on this handle recorded (0 if none). */
 EOQ_API int eoq_last_cuda_error(eoq_handle_t handle);

@@ -2,6 +2,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
+#include <stdio.h>
 #include <string.h>
 
 #include <new>
@@ -335,7 +336,7 @@ bool plan_wgrad_patch(WgradPatchPlan &pl, const eoq_conv_desc_t &d, int ho, int 
     pl.num_stages = stages > 4 ? 4 : stages;
     if (pl.num_stages < 2) return false;
     const int total_blocks = d.n * pl.blocks_per_img;
-    int splits = (target_ctas + pl.num_groups - 1) / pl.num_groups;
+    int splits = target_ctas / pl.num_groups;  // rounded down: a few CTAs beyond one wave would double the kernel's time
     if (splits > total_blocks) splits = total_blocks;
     if (splits < 1) splits = 1;
     int per = (total_blocks + splits - 1) / splits;
@@ -364,6 +365,8 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
     h->dev = nullptr;
     h->launches = 0;
     h->profiling = false;
+    h->force_timeout = false;
+    h->gemm_only = false;
     h->num_records = 0;
     h->records = nullptr;
     h->branch = nullptr;
@@ -469,6 +472,20 @@ extern "C" int eoq_profile_stop(eoq_handle_t handle, int launches[EOQ_PROF_KINDS
     return record(h, e);
 }
 
+extern "C" int eoq_profile_gemm_only(eoq_handle_t handle, int on)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h) return EOQ_ERR_BAD_ARG;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess && h->gemm_only && !on) {
+        // the GEMMs that ran without their consumers left maxima in the reduction cells
+        e = launch_reset_cells(h->dev, nullptr);
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    }
+    h->gemm_only = on != 0;
+    return record(h, e);
+}
+
 extern "C" int eoq_set_gemm_ctas(eoq_handle_t handle, int ctas)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
@@ -571,8 +588,8 @@ extern "C" int eoq_workspace_size(const eoq_conv_desc_t *desc, int pass, size_t 
         case EOQ_PASS_WGRAD: {  // per-tap error sums, reduction cell, int64 sums, split-K slices
             WgradPatchPlan wp;
             const size_t slices = plan_wgrad_patch(wp, *desc, g.ho, g.wo) ? (size_t)wp.num_splits * g.w_elems * sizeof(int32_t) : 0;
-            *bytes = round256((size_t)desc->c_out * g.taps * sizeof(long long)) + 256 + round256(g.w_elems * sizeof(long long)) +
-                     round256(slices);
+            *bytes = kTapReplicas * round256((size_t)desc->c_out * g.taps * sizeof(long long)) + 256 +
+                     round256(g.w_elems * sizeof(long long)) + round256(slices);
             return EOQ_OK;
         }
         default: return EOQ_ERR_BAD_ARG;
@@ -591,10 +608,13 @@ static int check_workspace(const eoq_conv_desc_t *desc, int pass, const void *ws
 
 // ================================================================================= forward
 
-extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *x, const int32_t *x_exp,
-                            int32_t b1_c, const int8_t *w, int32_t gamma_c, int32_t b2_c, const int8_t *shortcut,
-                            int relu, int8_t *x5, int16_t *x2, uint8_t *relu_mask, int32_t *acc_dump, void *workspace,
-                            size_t workspace_bytes, void *stream)
+// Forward chain behind eoq_conv_fwd and eoq_conv_fwd_dev.  The scalars are the three host codes, or the device
+// array `scal_dev`.  `prep` holds what eoq_weight_prep derives from the weights; when it is null the call derives it
+// itself into `workspace` (two more kernels on the forward chain).
+static int conv_fwd_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *x, const int32_t *x_exp,
+                         int32_t b1_c, int32_t gamma_c, int32_t b2_c, const int32_t *scal_dev, const int8_t *w,
+                         const void *prep, const int8_t *shortcut, int relu, int8_t *x5, int16_t *x2, uint8_t *relu_mask,
+                         int32_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
     Geometry g;
@@ -611,7 +631,12 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     if ((double)g.taps * d.c_in * (127.0 + (b1_c < 0 ? -b1_c : b1_c)) * 127.0 >= 2147483647.0 - 16777216.0) return EOQ_ERR_RANGE;
     const bool row_window = use_row_window(d, g.wo);
     if (d.c_in == 8 && !row_window) return EOQ_ERR_UNSUPPORTED;
-    if ((b1_c != 0 || row_window) && (st = check_workspace(desc, EOQ_PASS_FWD, workspace, workspace_bytes)) != EOQ_OK) return st;
+    // with device scalars b1 is unknown here: the table is applied whenever prepared weights are at hand
+    const bool use_b1 = scal_dev ? prep != nullptr : b1_c != 0;
+    if (scal_dev && !prep && row_window) return EOQ_ERR_BAD_ARG;
+    if (!prep && (use_b1 || row_window) && (st = check_workspace(desc, EOQ_PASS_FWD, workspace, workspace_bytes)) != EOQ_OK) return st;
+    if (prep && (reinterpret_cast<uintptr_t>(prep) & 255)) return EOQ_ERR_ALIGNMENT;
+    char *prep_base = prep ? static_cast<char *>(const_cast<void *>(prep)) : static_cast<char *>(workspace);
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const int w_mem = d.w + 2 * d.x_wmargin;
 
@@ -641,11 +666,13 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
             p.tap_b[t] = (unsigned char)t;
         }
         const BorderClasses bc0 = border_classes(d, g);
-        w_rows = reinterpret_cast<int8_t *>(workspace) + round256((size_t)bc0.nrc * bc0.ncc * d.c_out * sizeof(int32_t));
-        ProfScope prof(h, EOQ_PROF_FWD_AUX, s);
-        cudaError_t e = launch_weight_pad_rows(w, w_rows, d.c_out, d.kh, d.kw, d.c_in, s);
-        if (e != cudaSuccess) return record(h, e);
-        count_launches(h, 1);
+        w_rows = reinterpret_cast<int8_t *>(prep_base) + round256((size_t)bc0.nrc * bc0.ncc * d.c_out * sizeof(int32_t));
+        if (!prep) {
+            ProfScope prof(h, EOQ_PROF_FWD_AUX, s);
+            cudaError_t e = launch_weight_pad_rows(w, w_rows, d.c_out, d.kh, d.kw, d.c_in, s);
+            if (e != cudaSuccess) return record(h, e);
+            count_launches(h, 1);
+        }
     } else {
         plan_igemm(p, d.c_in, g.taps, h->sm_count);
         p.src_stride_w = d.stride;
@@ -664,6 +691,8 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     p.b1_c = b1_c;
     p.gamma_c = gamma_c;
     p.b2_c = b2_c;
+    p.scal_dev = scal_dev;
+    p.k_total = g.taps * d.c_in;
     p.shortcut = shortcut;
     p.relu = relu ? 1 : 0;
     p.x5 = x5;
@@ -671,16 +700,18 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     p.relu_mask = relu_mask;
     p.acc_out = acc_dump;
     p.dev = h->dev;
-    if (b1_c != 0) {
+    if (use_b1) {
         const BorderClasses bc = border_classes(d, g);
         if (bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
-        p.b1_table = reinterpret_cast<const int32_t *>(workspace);
+        p.b1_table = reinterpret_cast<const int32_t *>(prep_base);
         p.b1_nlo_h = bc.nlo_h; p.b1_nhi_h = bc.nhi_h; p.b1_nrc = bc.nrc;
         p.b1_nlo_w = bc.nlo_w; p.b1_nhi_w = bc.nhi_w; p.b1_ncc = bc.ncc;
-        ProfScope prof(h, EOQ_PROF_FWD_AUX, s);
-        cudaError_t e = launch_b1_weight_table(w, reinterpret_cast<int32_t *>(workspace), d, bc, s);
-        if (e != cudaSuccess) return record(h, e);
-        count_launches(h, 1);
+        if (!prep) {
+            ProfScope prof(h, EOQ_PROF_FWD_AUX, s);
+            cudaError_t e = launch_b1_weight_table(w, reinterpret_cast<int32_t *>(prep_base), d, bc, s);
+            if (e != cudaSuccess) return record(h, e);
+            count_launches(h, 1);
+        }
     }
     CUtensorMap map_a, map_b;
     if (patch) {
@@ -705,6 +736,76 @@ extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, co
     count_launches(h, 1);
     ProfScope prof(h, EOQ_PROF_IGEMM_FWD, s);
     return record(h, launch_igemm(p, map_a, map_b, persistent_grid(tiles, h->gemm_ctas), s));
+}
+
+extern "C" int eoq_conv_fwd(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *x, const int32_t *x_exp,
+                            int32_t b1_c, const int8_t *w, int32_t gamma_c, int32_t b2_c, const int8_t *shortcut,
+                            int relu, int8_t *x5, int16_t *x2, uint8_t *relu_mask, int32_t *acc_dump, void *workspace,
+                            size_t workspace_bytes, void *stream)
+{
+    return conv_fwd_impl(handle, desc, x, x_exp, b1_c, gamma_c, b2_c, nullptr, w, nullptr, shortcut, relu, x5, x2, relu_mask,
+                         acc_dump, workspace, workspace_bytes, stream);
+}
+
+extern "C" int eoq_conv_fwd_dev(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *x, const int32_t *x_exp,
+                                const int32_t *scalars, const int8_t *w, const void *w_prep, const int8_t *shortcut,
+                                int relu, int8_t *x5, int16_t *x2, uint8_t *relu_mask, void *stream)
+{
+    if (!scalars || (reinterpret_cast<uintptr_t>(scalars) & 3)) return EOQ_ERR_BAD_ARG;
+    return conv_fwd_impl(handle, desc, x, x_exp, 0, 128, 0, scalars, w, w_prep, shortcut, relu, x5, x2, relu_mask, nullptr,
+                         nullptr, 0, stream);
+}
+
+extern "C" int eoq_weight_prep_size(const eoq_conv_desc_t *desc, size_t *bytes)
+{
+    return eoq_workspace_size(desc, EOQ_PASS_FWD, bytes);
+}
+
+extern "C" int eoq_weight_prep(eoq_handle_t handle, int num, const eoq_conv_desc_t *descs, const int8_t *const *w,
+                               void *const *prep, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || num <= 0 || !descs || !w || !prep) return EOQ_ERR_BAD_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    // every argument is checked before the first launch
+    for (int i = 0; i < num; ++i) {
+        Geometry g;
+        int st = check_desc(&descs[i], &g);
+        if (st != EOQ_OK) return st;
+        if (!w[i] || !prep[i]) return EOQ_ERR_BAD_ARG;
+        if (!aligned16(w[i]) || (reinterpret_cast<uintptr_t>(prep[i]) & 255)) return EOQ_ERR_ALIGNMENT;
+        const BorderClasses bc = border_classes(descs[i], g);
+        if (bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
+    }
+    for (int base = 0; base < num; base += kPrepChunk) {
+        PrepBatch b;
+        memset(&b, 0, sizeof(b));
+        b.num = num - base < kPrepChunk ? num - base : kPrepChunk;
+        int blocks = 0;
+        for (int k = 0; k < b.num; ++k) {
+            const eoq_conv_desc_t &d = descs[base + k];
+            Geometry g;
+            check_desc(&d, &g);
+            PrepItem &it = b.item[k];
+            it.w = w[base + k];
+            it.table = static_cast<int32_t *>(prep[base + k]);
+            it.d = d;
+            it.ho = g.ho;
+            it.wo = g.wo;
+            it.bc = border_classes(d, g);
+            it.w_rows = use_row_window(d, g.wo)
+                            ? static_cast<int8_t *>(prep[base + k]) + round256((size_t)it.bc.nrc * it.bc.ncc * d.c_out * sizeof(int32_t))
+                            : nullptr;
+            b.first_block[k] = blocks;
+            blocks += d.c_out;
+        }
+        b.first_block[b.num] = blocks;
+        ProfScope prof(h, EOQ_PROF_FWD_AUX, s);
+        cudaError_t e = launch_weight_prep(b, s);
+        if (e != cudaSuccess) return record(h, e);
+        count_launches(h, 1);
+    }
+    return EOQ_OK;
 }
 
 // ================================================================================= error back-propagation
@@ -759,7 +860,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                 ProfScope prof(h, EOQ_PROF_IGEMM_DGRAD, s);
                 e = launch_igemm_patch(p, pl, map_a, map_b, persistent_grid(ptiles, h->gemm_ctas), s);
             }
-            if (e != cudaSuccess) return record(h, e);
+            if (e != cudaSuccess || h->gemm_only) return record(h, e);
             {
                 ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
                 e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true,
@@ -916,6 +1017,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         }
     delete group;  // closes the group's bracket on `s`, behind the joins
     group = nullptr;
+    if (h->gemm_only) return EOQ_OK;
     // Q_e over the whole tensor: the maximum is complete only now
     {
         ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
@@ -937,29 +1039,34 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
 // behind a fork event recorded on `s` (everything queued on `s` so far, the clearing memset included, comes
 // first); the caller waits for join_ev on `s` before the kernel that reads the sums.  Without a branch stream
 // (the allocation-free handle) they are issued on `s` itself.
-static cudaError_t launch_tap_sums_beside(Handle *h, const int8_t *e3, long long *tap_sums, const eoq_conv_desc_t &d,
-                                          int ho, int wo, const BorderClasses &bc, cudaStream_t s, bool *joined)
+static cudaError_t launch_tap_sums_beside(Handle *h, const int8_t *e3, long long *tap_sums, size_t tap_bytes,
+                                          const eoq_conv_desc_t &d, int ho, int wo, const BorderClasses &bc,
+                                          cudaStream_t s, bool *joined)
 {
+    const size_t tap_stride = tap_bytes / kTapReplicas / sizeof(long long);
     *joined = false;
     count_launches(h, 1);
     if (!h->branch) {
-        ProfScope prof(h, EOQ_PROF_WGRAD_AUX, s);
-        return launch_b1_error_sums(e3, tap_sums, d, ho, wo, bc, h->sm_count, s);
+        ProfScope prof(h, EOQ_PROF_WGRAD_TAPS, s);
+        cudaError_t e = cudaMemsetAsync(tap_sums, 0, tap_bytes, s);  // the kernel adds into them
+        return e != cudaSuccess ? e : launch_b1_error_sums(e3, tap_sums, tap_stride, d, ho, wo, bc, h->sm_count, s);
     }
     cudaError_t e = cudaEventRecord(h->fork_ev, s);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(h->branch, h->fork_ev, 0);
     if (e == cudaSuccess) {
-        ProfScope prof(h, EOQ_PROF_WGRAD_AUX, h->branch);
-        e = launch_b1_error_sums(e3, tap_sums, d, ho, wo, bc, h->sm_count, h->branch);
+        ProfScope prof(h, EOQ_PROF_WGRAD_TAPS, h->branch);
+        e = cudaMemsetAsync(tap_sums, 0, tap_bytes, h->branch);
+        if (e == cudaSuccess) e = launch_b1_error_sums(e3, tap_sums, tap_stride, d, ho, wo, bc, h->sm_count, h->branch);
     }
     if (e == cudaSuccess) e = cudaEventRecord(h->join_ev, h->branch);
     *joined = e == cudaSuccess;
     return e;
 }
 
-extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3,
-                              const int32_t *e3_exp, const int8_t *x, int32_t b1_c, int8_t *gq, int32_t *g_exp,
-                              int64_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
+// Weight gradient behind eoq_conv_wgrad and eoq_conv_wgrad_dev: b1 is the host code b1_c, or the code at b1_dev.
+static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                           const int8_t *x, int32_t b1_c, const int32_t *b1_dev, int8_t *gq, int32_t *g_exp,
+                           int64_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
     Geometry g;
@@ -972,14 +1079,14 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     const eoq_conv_desc_t &d = *desc;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
 
-    // workspace: [tap sums][reduction cell][int64 sums][split-K slices]; everything a call accumulates into sits
-    // at the front, so one memset clears it
+    // workspace: [tap sums][256 spare bytes][int64 sums][split-K slices]
     const BorderClasses bc = border_classes(d, g);
-    if (b1_c != 0 && bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
+    const bool use_b1 = b1_dev != nullptr || b1_c != 0;  // a device-resident b1 may be anything: its term is always formed
+    if (use_b1 && bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
     char *ws = reinterpret_cast<char *>(workspace);
     long long *tap_sums = reinterpret_cast<long long *>(ws);
-    const size_t tap_bytes = round256((size_t)d.c_out * g.taps * sizeof(long long));
-    WgradCells *cells = reinterpret_cast<WgradCells *>(ws + tap_bytes);
+    const size_t tap_stride = round256((size_t)d.c_out * g.taps * sizeof(long long)) / sizeof(long long);  // one copy, in elements
+    const size_t tap_bytes = kTapReplicas * tap_stride * sizeof(long long);
     long long *acc = reinterpret_cast<long long *>(ws + tap_bytes + 256);
     const size_t acc_bytes = round256(g.w_elems * sizeof(long long));
 
@@ -989,17 +1096,21 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         wp.partials = reinterpret_cast<int32_t *>(ws + tap_bytes + 256 + acc_bytes);
         wp.dev = h->dev;
         cudaError_t e;
-        {
-            ProfScope prof(h, EOQ_PROF_WGRAD_AUX, s);
-            e = b1_c != 0 ? cudaMemsetAsync(ws, 0, tap_bytes + 256, s) : cudaMemsetAsync(cells, 0, 256, s);
+        if (h->gemm_only) {
+            CUtensorMap mx, me;
+            if (!make_patch_map(&mx, x, d.n, d.h, d.w, d.c_in, wp.kc, wp.pw, wp.r_rows + d.kh - 1) ||
+                !make_patch_map(&me, e3, d.n, g.ho, g.wo, d.c_out, wp.tile_n, wp.pw, wp.r_rows))
+                return EOQ_ERR_UNSUPPORTED;
+            count_launches(h, 1);
+            return record(h, launch_wgrad_patch(wp, mx, me, s));
         }
-        if (e == cudaSuccess && b1_c != 0) e = launch_tap_sums_beside(h, e3, tap_sums, d, g.ho, g.wo, bc, s, &joined);
+        e = use_b1 ? launch_tap_sums_beside(h, e3, tap_sums, tap_bytes, d, g.ho, g.wo, bc, s, &joined) : cudaSuccess;
         if (e != cudaSuccess) return record(h, e);
         CUtensorMap map_x, map_e;
         if (!make_patch_map(&map_x, x, d.n, d.h, d.w, d.c_in, wp.kc, wp.pw, wp.r_rows + d.kh - 1) ||
             !make_patch_map(&map_e, e3, d.n, g.ho, g.wo, d.c_out, wp.tile_n, wp.pw, wp.r_rows))
             return EOQ_ERR_UNSUPPORTED;
-        count_launches(h, 3);
+        count_launches(h, 1);
         {
             ProfScope prof(h, EOQ_PROF_WGRAD, s);
             e = launch_wgrad_patch(wp, map_x, map_e, s);
@@ -1008,8 +1119,8 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         if (e != cudaSuccess) return record(h, e);
         ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
         e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
-                          b1_c != 0 ? tap_sums : nullptr, b1_c, d.c_in, wp.partials, wp.num_splits, cells, h->dev,
-                          h->sm_count, s);
+                          use_b1 ? tap_sums : nullptr, tap_stride, b1_c, b1_dev, d.c_in, wp.partials, wp.num_splits, h->dev, h->sm_count, s);
+        count_launches(h, 2);
         return record(h, e);
     }
 
@@ -1086,13 +1197,12 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     p.acc = acc;
     p.dev = h->dev;
 
-    cudaError_t e;
-    {
+    cudaError_t e = cudaSuccess;
+    if (!h->gemm_only) {
         ProfScope aux(h, EOQ_PROF_WGRAD_AUX, s);
-        // the GEMM adds into the int64 sums with atomics: they are cleared together with the cells and class sums
-        e = cudaMemsetAsync(ws, 0, tap_bytes + 256 + acc_bytes, s);
+        e = cudaMemsetAsync(acc, 0, acc_bytes, s);  // the GEMM adds into the int64 sums with atomics
     }
-    if (e == cudaSuccess && b1_c != 0) e = launch_tap_sums_beside(h, e3, tap_sums, d, g.ho, g.wo, bc, s, &joined);
+    if (e == cudaSuccess && use_b1 && !h->gemm_only) e = launch_tap_sums_beside(h, e3, tap_sums, tap_bytes, d, g.ho, g.wo, bc, s, &joined);
     if (e != cudaSuccess) return record(h, e);
     CUtensorMap map_x, map_e;
     if (!make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage)) return EOQ_ERR_UNSUPPORTED;
@@ -1101,18 +1211,125 @@ extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                    : !make_im2col_map(&map_x, x, d.n, d.h, w_mem, d.c_in, d.x_wmargin - d.pad, -d.pad, g.wo, g.ho, d.stride,
                                       p.kc, p.pixels_per_stage))
         return EOQ_ERR_UNSUPPORTED;
-    count_launches(h, 3);  // the GEMM, the finalize kernel and Q_g
+    count_launches(h, 1);
     {
         ProfScope prof(h, EOQ_PROF_WGRAD, s);
         e = launch_wgrad(p, map_x, map_e, s);
     }
     if (e == cudaSuccess && joined) e = cudaStreamWaitEvent(s, h->join_ev, 0);
-    if (e != cudaSuccess) return record(h, e);
+    if (e != cudaSuccess || h->gemm_only) return record(h, e);
     // the kernel leaves sums as [oc][tap][ic], which is the layout of g
     ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
     e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
-                      b1_c != 0 ? tap_sums : nullptr, b1_c, d.c_in, nullptr, 0, cells, h->dev, h->sm_count, s);
+                      use_b1 ? tap_sums : nullptr, tap_stride, b1_c, b1_dev, d.c_in, nullptr, 0, h->dev, h->sm_count, s);
+    count_launches(h, 2);
     return record(h, e);
+}
+
+extern "C" int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3,
+                              const int32_t *e3_exp, const int8_t *x, int32_t b1_c, int8_t *gq, int32_t *g_exp,
+                              int64_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return conv_wgrad_impl(handle, desc, e3, e3_exp, x, b1_c, nullptr, gq, g_exp, acc_dump, workspace, workspace_bytes, stream);
+}
+
+extern "C" int eoq_conv_wgrad_dev(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3,
+                                  const int32_t *e3_exp, const int8_t *x, const int32_t *b1_c, int8_t *gq, int32_t *g_exp,
+                                  void *workspace, size_t workspace_bytes, void *stream)
+{
+    // b1_c null: the layer has no bias in front of its convolution (the first layer of a network)
+    return conv_wgrad_impl(handle, desc, e3, e3_exp, x, 0, b1_c, gq, g_exp, nullptr, workspace, workspace_bytes, stream);
+}
+
+// ================================================================================= tensor-pipe probe
+
+extern "C" int eoq_probe_mma_i8(eoq_handle_t handle, int n_cols, int iters, int launches, double *tops,
+                                double *cycles_per_mma, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !tops || n_cols < 16 || n_cols > 256 || (n_cols % 16) || iters < 1 || iters > (1 << 20) || launches < 1 ||
+        launches > 100000)
+        return EOQ_ERR_BAD_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaError_t e = cudaEventCreate(&a);
+    if (e == cudaSuccess) e = cudaEventCreate(&b);
+    unsigned long long *cyc = &h->dev->probe_cycles;
+    if (e == cudaSuccess) e = launch_probe_mma_i8(n_cols, iters, h->sm_count, h->dev, cyc, s);  // warm-up
+    if (e == cudaSuccess) e = cudaMemsetAsync(cyc, 0, sizeof(unsigned long long), s);
+    if (e == cudaSuccess) e = cudaEventRecord(a, s);
+    for (int i = 0; i < launches && e == cudaSuccess; ++i) e = launch_probe_mma_i8(n_cols, iters, h->sm_count, h->dev, cyc, s);
+    if (e == cudaSuccess) e = cudaEventRecord(b, s);
+    if (e == cudaSuccess) e = cudaEventSynchronize(b);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
+    unsigned long long cycles = 0;
+    if (e == cudaSuccess) e = cudaMemcpy(&cycles, cyc, sizeof(cycles), cudaMemcpyDeviceToHost);
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (e != cudaSuccess) return record(h, e);
+    count_launches(h, launches + 1);
+    const double ops = 2.0 * kTileM * n_cols * 32.0 * 4.0 * iters * (double)h->sm_count * launches;
+    *tops = ms > 0.f ? ops / (ms * 1e-3) / 1e12 : 0.0;
+    if (cycles_per_mma) *cycles_per_mma = (double)cycles / (4.0 * iters);
+    return EOQ_OK;
+}
+
+// ================================================================================= plan report
+
+extern "C" int eoq_describe_plan(eoq_handle_t handle, const eoq_conv_desc_t *desc, int pass, char *buf, size_t buf_bytes)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    Geometry g;
+    if (!h || !buf || buf_bytes == 0) return EOQ_ERR_BAD_ARG;
+    int st = check_desc(desc, &g);
+    if (st != EOQ_OK) return st;
+    const eoq_conv_desc_t &d = *desc;
+    IgemmParams p;
+    memset(&p, 0, sizeof(p));
+    PatchPlan pl;
+    memset(&pl, 0, sizeof(pl));
+    buf[0] = 0;
+    if (pass == EOQ_PASS_FWD) {
+        if (d.stride == 1 && d.kh == d.kw && d.x_wmargin == 0 &&
+            plan_patch(p, pl, d.n, d.c_in, g.ho, g.wo, d.kh, d.pad, d.c_out, h->sm_count)) {
+            snprintf(buf, buf_bytes, "kernel=igemm_patch tile_n=%d accumulators=%d m_tiles=%d n_tiles=%d weights=%s", p.tile_n,
+                     p.tile_n <= 128 ? 2 : 1, p.num_m_tiles, p.num_n_tiles, pl.b_resident ? "resident" : "streamed");
+            return EOQ_OK;
+        }
+        p.M = d.n * g.ho * g.wo;
+        p.N = d.c_out;
+        const bool rw = use_row_window(d, g.wo);
+        plan_igemm(p, rw ? 8 * d.c_in : d.c_in, rw ? d.kh : g.taps, h->sm_count);
+        snprintf(buf, buf_bytes, "kernel=igemm%s tile_n=%d m_tiles=%d n_tiles=%d kc=%d stages=%d", rw ? "_filter_rows" : "",
+                 p.tile_n, p.num_m_tiles, p.num_n_tiles, p.kc, p.num_stages);
+        return EOQ_OK;
+    }
+    if (pass == EOQ_PASS_DGRAD) {
+        if (d.stride == 1 && d.kh == d.kw && d.kh - 1 - d.pad >= 0 &&
+            plan_patch(p, pl, d.n, d.c_out, d.h, d.w, d.kh, d.kh - 1 - d.pad, d.c_in, h->sm_count)) {
+            snprintf(buf, buf_bytes, "kernel=igemm_patch tile_n=%d accumulators=%d m_tiles=%d n_tiles=%d weights=%s", p.tile_n,
+                     p.tile_n <= 128 ? 2 : 1, p.num_m_tiles, p.num_n_tiles, pl.b_resident ? "resident" : "streamed");
+            return EOQ_OK;
+        }
+        const int hq = (d.h + d.stride - 1) / d.stride, wq = (d.w + d.stride - 1) / d.stride;
+        p.M = d.n * hq * wq;
+        p.N = d.c_in;
+        plan_igemm(p, d.c_out, ((d.kh + d.stride - 1) / d.stride) * ((d.kw + d.stride - 1) / d.stride), h->sm_count);
+        snprintf(buf, buf_bytes, "kernel=igemm classes=%d tile_n=%d m_tiles=%d n_tiles=%d kc=%d", d.stride * d.stride, p.tile_n,
+                 p.num_m_tiles, p.num_n_tiles, p.kc);
+        return EOQ_OK;
+    }
+    if (pass == EOQ_PASS_WGRAD) {
+        WgradPatchPlan wp;
+        if (plan_wgrad_patch(wp, d, g.ho, g.wo, h->gemm_ctas < kWgradTargetCtas ? h->gemm_ctas : kWgradTargetCtas))
+            snprintf(buf, buf_bytes, "kernel=wgrad_patch groups=%d splits=%d tile_n=%d kc=%d", wp.num_groups, wp.num_splits, wp.tile_n,
+                     wp.kc);
+        else
+            snprintf(buf, buf_bytes, "kernel=wgrad%s", use_row_window(d, g.wo) ? "_filter_rows" : "");
+        return EOQ_OK;
+    }
+    return EOQ_ERR_BAD_ARG;
 }
 
 // ================================================================================= elementwise entry points
@@ -1138,9 +1355,9 @@ extern "C" int eoq_quantize(eoq_handle_t handle, int mode, const void *src, int 
                                    dst_exp, nullptr, false, h->dev, h->sm_count, s));
 }
 
-extern "C" int eoq_err_prescale(eoq_handle_t handle, const int8_t *e0, const int32_t *e0_exp, const uint8_t *relu_mask,
-                                const int16_t *x2, size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp,
-                                int64_t *sum_e1, int64_t *sum_e1x2, void *stream)
+static int err_prescale_impl(eoq_handle_t handle, const int8_t *e0, const int32_t *e0_exp, const uint8_t *relu_mask,
+                             const int16_t *x2, size_t n_el, int32_t gamma_c, const int32_t *gamma_dev, int8_t *e3,
+                             int32_t *e3_exp, int64_t *sum_e1, int64_t *sum_e1x2, void *stream)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
     if (!h || !e0 || !e0_exp || !e3 || !e3_exp || n_el == 0 || (n_el % 16)) return EOQ_ERR_BAD_ARG;
@@ -1149,16 +1366,41 @@ extern "C" int eoq_err_prescale(eoq_handle_t handle, const int8_t *e0, const int
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     ProfScope prof(h, EOQ_PROF_ERR_HEAD, s);
     int kernels = 0;
-    const cudaError_t e = launch_err_prescale(e0, e0_exp, relu_mask, x2, n_el, gamma_c, e3, e3_exp,
+    const bool force_timeout = h->force_timeout;
+    h->force_timeout = false;
+    const cudaError_t e = launch_err_prescale(e0, e0_exp, relu_mask, x2, n_el, gamma_c, gamma_dev, e3, e3_exp,
                                               reinterpret_cast<long long *>(sum_e1), reinterpret_cast<long long *>(sum_e1x2),
-                                              h->dev, h->sm_count, s, &kernels);
+                                              h->dev, h->sm_count, s, &kernels, force_timeout);
     count_launches(h, kernels);
     return record(h, e);
 }
 
-extern "C" int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const int8_t *const *g,
-                          const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp,
-                          int round_mode, uint64_t seed, uint64_t step, void *stream)
+extern "C" int eoq_err_prescale(eoq_handle_t handle, const int8_t *e0, const int32_t *e0_exp, const uint8_t *relu_mask,
+                                const int16_t *x2, size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp,
+                                int64_t *sum_e1, int64_t *sum_e1x2, void *stream)
+{
+    return err_prescale_impl(handle, e0, e0_exp, relu_mask, x2, n_el, gamma_c, nullptr, e3, e3_exp, sum_e1, sum_e1x2, stream);
+}
+
+extern "C" int eoq_err_prescale_dev(eoq_handle_t handle, const int8_t *e0, const int32_t *e0_exp, const uint8_t *relu_mask,
+                                    const int16_t *x2, size_t n_el, const int32_t *gamma_c, int8_t *e3, int32_t *e3_exp,
+                                    int64_t *sum_e1, int64_t *sum_e1x2, void *stream)
+{
+    if (!gamma_c) return EOQ_ERR_BAD_ARG;
+    return err_prescale_impl(handle, e0, e0_exp, relu_mask, x2, n_el, 128, gamma_c, e3, e3_exp, sum_e1, sum_e1x2, stream);
+}
+
+extern "C" int eoq_debug_force_wait_timeout(eoq_handle_t handle)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h) return EOQ_ERR_BAD_ARG;
+    h->force_timeout = true;
+    return EOQ_OK;
+}
+
+static int update_impl(eoq_handle_t handle, int num, int8_t *const *w, const int8_t *const *g,
+                       const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp, int round_mode,
+                       uint64_t seed, uint64_t step, uint64_t *step_dev, void *stream)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
     if (!h || num <= 0 || !w || !g || !g_exp || !n) return EOQ_ERR_BAD_ARG;
@@ -1174,9 +1416,25 @@ extern "C" int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const 
         t[i].n = n[i];
     }
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    count_launches(h, 2 * ((num + 63) / 64));
-    ProfScope prof(h, EOQ_PROF_OTHER, s);
-    return record(h, launch_update(t, num, lr_mant, lr_exp, round_mode == EOQ_ROUND_STOCHASTIC, seed, step, h->dev, h->sm_count, s));
+    count_launches(h, 2 * ((num + 63) / 64) + (step_dev ? 1 : 0));
+    ProfScope prof(h, EOQ_PROF_UPDATE, s);
+    return record(h, launch_update(t, num, lr_mant, lr_exp, round_mode == EOQ_ROUND_STOCHASTIC, seed, step,
+                                   reinterpret_cast<unsigned long long *>(step_dev), h->dev, h->sm_count, s));
+}
+
+extern "C" int eoq_update(eoq_handle_t handle, int num, int8_t *const *w, const int8_t *const *g,
+                          const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp,
+                          int round_mode, uint64_t seed, uint64_t step, void *stream)
+{
+    return update_impl(handle, num, w, g, g_exp, n, lr_mant, lr_exp, round_mode, seed, step, nullptr, stream);
+}
+
+extern "C" int eoq_update_dev(eoq_handle_t handle, int num, int8_t *const *w, const int8_t *const *g,
+                              const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp,
+                              int round_mode, uint64_t seed, uint64_t *step, void *stream)
+{
+    if (!step || (reinterpret_cast<uintptr_t>(step) & 7)) return EOQ_ERR_BAD_ARG;
+    return update_impl(handle, num, w, g, g_exp, n, lr_mant, lr_exp, round_mode, seed, 0, step, stream);
 }
 
 extern "C" int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t *dst, int n, int c, int hh, int ww,
@@ -1197,7 +1455,7 @@ extern "C" int eoq_quantize_image(eoq_handle_t handle, const float *src, int n, 
         return EOQ_ERR_BAD_ARG;
     if ((c_dst % 16 && c_dst != 8) || c_dst > 64 || !aligned16(src) || !aligned16(dst)) return EOQ_ERR_ALIGNMENT;
     count_launches(h, 2);
-    ProfScope prof(h, EOQ_PROF_OTHER, reinterpret_cast<cudaStream_t>(stream));
+    ProfScope prof(h, EOQ_PROF_INPUT_Q, reinterpret_cast<cudaStream_t>(stream));
     return record(h, launch_quantize_image(src, n, hh, ww, c_src, c_dst, wmargin, dst, dst_exp, h->dev, h->sm_count,
                                            reinterpret_cast<cudaStream_t>(stream)));
 }

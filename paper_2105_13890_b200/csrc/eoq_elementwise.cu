@@ -350,18 +350,27 @@ __global__ void sq_i32_scatter_kernel(const int32_t *__restrict__ src, const int
 // reduces max |.|.  A block of 256 threads is (256 / groups) elements x `groups` slice groups: every thread adds
 // its share of the slices with independent, coalesced loads and the groups meet in shared memory.
 __global__ void wgrad_finalize_kernel(const int32_t *__restrict__ parts, int num_parts, int groups, size_t n, long long *acc,
-                                      const long long *__restrict__ tap_sums, int32_t b1_c, int c_in, long long *copy_out,
-                                      WgradCells *cells)
+                                      const long long *__restrict__ tap_sums, size_t replica_stride, int32_t b1_c,
+                                      const int32_t *b1_dev, int c_in, long long *copy_out, DeviceState *dev)
 {
     __shared__ long long part[256];
+    if (b1_dev) b1_c = clampi(__ldg(b1_dev), -32768, 32767);
     const int bx = 256 / groups, tx = threadIdx.x % bx, ty = threadIdx.x / bx;
     unsigned long long mx = 0;
     for (size_t base = (size_t)blockIdx.x * bx; base < n; base += (size_t)gridDim.x * bx) {
         const size_t i = base + tx;
         long long v = 0;
         if (parts) {
-            if (i < n)
-                for (int s = ty; s < num_parts; s += groups) v += (long long)__ldg(parts + (size_t)s * n + i);
+            if (i < n) {
+                // four slices per round: their loads are independent and in flight together
+                int s = ty;
+                for (; s + 3 * groups < num_parts; s += 4 * groups) {
+                    const int32_t a0 = __ldg(parts + (size_t)s * n + i), a1 = __ldg(parts + (size_t)(s + groups) * n + i);
+                    const int32_t a2 = __ldg(parts + (size_t)(s + 2 * groups) * n + i), a3 = __ldg(parts + (size_t)(s + 3 * groups) * n + i);
+                    v += ((long long)a0 + a1) + ((long long)a2 + a3);
+                }
+                for (; s < num_parts; s += groups) v += (long long)__ldg(parts + (size_t)s * n + i);
+            }
             if (groups > 1) {
                 part[threadIdx.x] = v;
                 __syncthreads();
@@ -375,8 +384,13 @@ __global__ void wgrad_finalize_kernel(const int32_t *__restrict__ parts, int num
             v = acc[i];
         }
         if (ty == 0 && i < n) {
-            if (tap_sums)  // index of (oc, tap); a 32-bit division whenever the tensor allows it
-                v += (long long)b1_c * tap_sums[n <= 0xffffffffull ? (size_t)((uint32_t)i / (uint32_t)c_in) : i / (size_t)c_in];
+            if (tap_sums) {  // index of (oc, tap); a 32-bit division whenever the tensor allows it
+                const long long *t = tap_sums + (n <= 0xffffffffull ? (size_t)((uint32_t)i / (uint32_t)c_in) : i / (size_t)c_in);
+                long long ts = 0;
+#pragma unroll
+                for (int r = 0; r < kTapReplicas; ++r) ts += __ldg(t + (size_t)r * replica_stride);
+                v += (long long)b1_c * ts;
+            }
             if (parts || tap_sums) acc[i] = v;
             if (copy_out) copy_out[i] = v;
             const unsigned long long a = (unsigned long long)(v < 0 ? -v : v);
@@ -384,21 +398,29 @@ __global__ void wgrad_finalize_kernel(const int32_t *__restrict__ parts, int num
         }
     }
     mx = block_max_u64(mx);
-    if (threadIdx.x == 0 && mx) atomicMax(&cells->absmax, mx);
+    if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u64, mx);
 }
 
 __global__ void sq_i64_kernel(const long long *__restrict__ src, const int32_t *src_exp, int exp_bias, size_t n,
-                              int8_t *dst, int32_t *dst_exp, const WgradCells *cells, DeviceState *dev)
+                              int8_t *dst, int32_t *dst_exp, DeviceState *dev)
 {
-    const unsigned long long M = cells->absmax;
+    const unsigned long long M = dev->absmax_u64;
     const int t = M ? round_log2_u64(M) : 7;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         const int p_in = (src_exp ? *src_exp : 0) + exp_bias;
         *dst_exp = M ? p_in + t - 7 : p_in;
         if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
     }
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    // four codes per thread and round (one 32-bit store); n is a multiple of 4 for every weight tensor with padded channels
+    const size_t n4 = n / 4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        const longlong2 a = __ldg(reinterpret_cast<const longlong2 *>(src) + 2 * i);
+        const longlong2 b = __ldg(reinterpret_cast<const longlong2 *>(src) + 2 * i + 1);
+        reinterpret_cast<uint32_t *>(dst)[i] = pack4(sq_code64(a.x, t), sq_code64(a.y, t), sq_code64(b.x, t), sq_code64(b.y, t));
+    }
+    for (size_t i = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         dst[i] = (int8_t)sq_code64(src[i], t);
+    if (last_block_done(dev)) dev->absmax_u64 = 0;
 }
 
 // ------------------------------------------------------------------ head of the error chain
@@ -473,10 +495,24 @@ __global__ void prescale_reduce_kernel(const int8_t *__restrict__ e0, const uint
 }
 
 // Pass 2: e3 = Q_e(gamma * e1) under the reduced maximum.
-__global__ void prescale_apply_kernel(const int8_t *__restrict__ e0, const int32_t *e0_exp,
-                                      const uint8_t *__restrict__ mask, size_t n16, int32_t gamma_c, int8_t *e3,
-                                      int32_t *e3_exp, long long *sum_e1, long long *sum_e1x2, DeviceState *dev)
+// gamma of a launch: the host value, or the code read from device memory (clamped to 16 bits, EOQ_DEV_RANGE raised)
+__device__ __forceinline__ int32_t load_gamma(int32_t gamma_c, const int32_t *gamma_dev, DeviceState *dev)
 {
+    if (!gamma_dev) return gamma_c;
+    int32_t g = __ldg(gamma_dev);
+    if (g < -32768 || g > 32767) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(&dev->status, EOQ_DEV_RANGE);
+        g = clampi(g, -32768, 32767);
+    }
+    return g;
+}
+
+__global__ void prescale_apply_kernel(const int8_t *__restrict__ e0, const int32_t *e0_exp,
+                                      const uint8_t *__restrict__ mask, size_t n16, int32_t gamma_c,
+                                      const int32_t *gamma_dev, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
+                                      long long *sum_e1x2, DeviceState *dev)
+{
+    gamma_c = load_gamma(gamma_c, gamma_dev, dev);
     const uint32_t M = dev->absmax_u32 * (uint32_t)abs(gamma_c);  // max |gamma * e1| < 2^7 * 2^15
     const int t = M ? round_log2_u32(M) : 7;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -542,10 +578,12 @@ __global__ void prescale_apply_kernel(const int8_t *__restrict__ e0, const int32
 constexpr int kFusedGroups = 6;
 __global__ void __launch_bounds__(kThreads)
 prescale_fused_kernel(const int8_t *__restrict__ e0, const int32_t *e0_exp, const uint8_t *__restrict__ mask,
-                      const int16_t *__restrict__ x2, size_t n16, int32_t gamma_c, int8_t *e3, int32_t *e3_exp,
-                      long long *sum_e1, long long *sum_e1x2, DeviceState *dev)
+                      const int16_t *__restrict__ x2, size_t n16, int32_t gamma_c, const int32_t *gamma_dev, int8_t *e3,
+                      int32_t *e3_exp, long long *sum_e1, long long *sum_e1x2, DeviceState *dev, unsigned expected_blocks,
+                      uint32_t spin_limit)
 {
     __shared__ unsigned go_s;
+    gamma_c = load_gamma(gamma_c, gamma_dev, dev);
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     const size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     uint32_t e1w[kFusedGroups][4];
@@ -597,8 +635,10 @@ prescale_fused_kernel(const int8_t *__restrict__ e0, const int32_t *e0_exp, cons
         __threadfence();
         atomicAdd(&dev->arrivals, 1u);
         unsigned ok = 0;
-        for (uint32_t it = 0; it < kSpinLimit; ++it) {
-            if (*reinterpret_cast<volatile unsigned *>(&dev->arrivals) >= gridDim.x) { ok = 1; break; }
+        // (expected_blocks is the grid size; a larger value, which only the library's self-test passes, makes this
+        // wait run out)
+        for (uint32_t it = 0; it < spin_limit; ++it) {
+            if (*reinterpret_cast<volatile unsigned *>(&dev->arrivals) >= expected_blocks) { ok = 1; break; }
             __nanosleep(100);
         }
         if (!ok) atomicOr(&dev->status, EOQ_DEV_TIMEOUT);
@@ -725,8 +765,9 @@ __device__ __forceinline__ int update_one(int w, int g, int lr_mant, int t, int 
 
 __global__ void update_apply_kernel(const __grid_constant__ UpdateBatch b, int32_t lr_mant, int32_t lr_exp,
                                     int stochastic, unsigned long long seed, unsigned long long step,
-                                    DeviceState *dev)
+                                    const unsigned long long *step_dev, DeviceState *dev)
 {
+    if (step_dev) step = *step_dev;  // device-resident step counter (bumped by step_bump_kernel behind the call)
     const int k = find_tensor(b, blockIdx.x);
     const UpdateTensor &T = b.t[k];
     const uint32_t M = dev->tensor_absmax[b.tensor_base + k] * (uint32_t)lr_mant;  // max |lr_mant * g| < 2^15
@@ -761,6 +802,8 @@ __global__ void update_apply_kernel(const __grid_constant__ UpdateBatch b, int32
     for (size_t j = tail + threadIdx.x; j < end; j += blockDim.x)
         T.w[j] = (int8_t)update_one(T.w[j], T.g[j], lr_mant, t, d, stochastic, key, j);
 }
+
+__global__ void step_bump_kernel(unsigned long long *step_dev) { *step_dev += 1ull; }
 
 // ------------------------------------------------------------------ layout helpers
 
@@ -838,6 +881,62 @@ __global__ void b1_weight_table_kernel(const int8_t *__restrict__ w, int32_t *ta
     }
 }
 
+// What eoq_weight_prep derives from the weights of several layers in one launch: the b1 table of every layer
+// (as b1_weight_table_kernel builds it) and, for a first layer on the filter-row path, the weights re-packed as
+// [oc][kh][8][c_in] with zero taps.  One block per (layer, output channel).
+__global__ void weight_prep_kernel(const __grid_constant__ PrepBatch b)
+{
+    __shared__ int32_t tap_sum[kMaxTaps];
+    int k = 0;
+    while (k + 1 < b.num && (int)blockIdx.x >= b.first_block[k + 1]) ++k;
+    const PrepItem &it = b.item[k];
+    const eoq_conv_desc_t &d = it.d;
+    const BorderClasses &bc = it.bc;
+    const int oc = blockIdx.x - b.first_block[k];
+    const int taps = d.kh * d.kw;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    for (int t = warp; t < taps; t += nwarps) {
+        const int8_t *p = it.w + ((size_t)oc * taps + t) * d.c_in;
+        int sum = 0;
+        for (int i = lane; i < d.c_in / 16; i += 32) {
+            const int4 v = __ldg(reinterpret_cast<const int4 *>(p) + i);
+            sum = __dp4a(v.x, 0x01010101, sum);
+            sum = __dp4a(v.y, 0x01010101, sum);
+            sum = __dp4a(v.z, 0x01010101, sum);
+            sum = __dp4a(v.w, 0x01010101, sum);
+        }
+        if (d.c_in == 8 && lane == 0) {
+            const int2 v = __ldg(reinterpret_cast<const int2 *>(p));
+            sum = __dp4a(v.x, 0x01010101, sum);
+            sum = __dp4a(v.y, 0x01010101, sum);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == 0) tap_sum[t] = sum;
+    }
+    __syncthreads();
+    for (int cls = threadIdx.x; cls < bc.nrc * bc.ncc; cls += blockDim.x) {
+        const int rc = cls / bc.ncc, cc = cls % bc.ncc;
+        int32_t sum = 0;
+        for (int kh = 0; kh < d.kh; ++kh) {
+            if (!tap_valid(rc, kh, it.ho, d.h, bc.nlo_h, bc.nhi_h, bc.nrc, d.stride, d.pad)) continue;
+            for (int kw = 0; kw < d.kw; ++kw)
+                if (tap_valid(cc, kw, it.wo, d.w, bc.nlo_w, bc.nhi_w, bc.ncc, d.stride, d.pad)) sum += tap_sum[kh * d.kw + kw];
+        }
+        it.table[(size_t)cls * d.c_out + oc] = sum;
+    }
+    if (it.w_rows) {
+        // this output channel's filter rows, each widened to 8 taps (c_in is 16 or 8: 4 or 2 words per tap)
+        const int words = d.c_in / 4;
+        const int32_t *src = reinterpret_cast<const int32_t *>(it.w) + (size_t)oc * taps * words;
+        int32_t *dst = reinterpret_cast<int32_t *>(it.w_rows) + (size_t)oc * d.kh * 8 * words;
+        for (int i = threadIdx.x; i < d.kh * 8 * words; i += blockDim.x) {
+            const int r = i / (8 * words), t = (i / words) % 8, wd = i % words;
+            dst[i] = t < d.kw ? __ldg(src + (r * d.kw + t) * words + wd) : 0;
+        }
+    }
+}
+
 // tap_sums[oc][tap] += sum of e3[n,y,x,oc] over the pixels for which the tap falls inside the image (the weight
 // gradient adds b1 times this to every input channel).  Pixels are summed per border class first (the taps inside
 // the image are the same for all pixels of a class).  A block owns a range of
@@ -845,9 +944,13 @@ __global__ void b1_weight_table_kernel(const int8_t *__restrict__ w, int32_t *ta
 // 32 / (slab / 16) pixels per step.  Interior pixels (one class, almost all of a large image) accumulate in
 // registers, border pixels in shared memory.
 constexpr int kClassSlab = 128;
-__global__ void b1_tap_sums_kernel(const int8_t *__restrict__ e3, long long *tap_sums, int c_out, int ho, int wo,
-                                   size_t pixels, int pixels_per_block, BorderClasses bc, eoq_conv_desc_t d)
+constexpr int kTapUnroll = 8;
+__global__ void b1_tap_sums_kernel(const int8_t *__restrict__ e3, long long *tap_sums, size_t replica_stride, int c_out, int ho,
+                                   int wo, size_t pixels, int pixels_per_block, BorderClasses bc, eoq_conv_desc_t d)
 {
+    // the blocks spread their atomics over kTapReplicas copies of the sums (the consumer adds the copies): all
+    // cells of one copy sit in a few kilobytes, i.e. behind one or two L2 slices, whose atomic rate bounds this kernel
+    tap_sums += (size_t)(blockIdx.x % kTapReplicas) * replica_stride;
     extern __shared__ int32_t cls_acc[];  // [classes][kClassSlab]
     const int classes = bc.nrc * bc.ncc;
     for (int i = threadIdx.x; i < classes * kClassSlab; i += blockDim.x) cls_acc[i] = 0;
@@ -865,27 +968,42 @@ __global__ void b1_tap_sums_kernel(const int8_t *__restrict__ e3, long long *tap
     const size_t end = min(pixels, begin + (size_t)pixels_per_block);
     const bool small = pixels <= 0xffffffffull;
     if (slot < pix_per_step) {
-        for (size_t p = begin + slot; p < end; p += pix_per_step) {
-            int x, y;
-            if (small) {  // 32-bit index arithmetic (a 64-bit division costs more than the rest of the pixel's work)
-                const uint32_t q = (uint32_t)p / (uint32_t)wo;
-                x = (int)((uint32_t)p - q * (uint32_t)wo);
-                y = (int)(q % (uint32_t)ho);
-            } else {
-                x = (int)(p % wo);
-                y = (int)((p / wo) % ho);
+        // kTapUnroll pixels per round: their loads are issued together and are in flight side by side
+        for (size_t p0 = begin + slot; p0 < end; p0 += kTapUnroll * (size_t)pix_per_step) {
+            int4 v[kTapUnroll];
+            int cls[kTapUnroll];
+#pragma unroll
+            for (int u = 0; u < kTapUnroll; ++u) {
+                const size_t p = p0 + (size_t)u * pix_per_step;
+                cls[u] = -2;  // beyond the block's range
+                v[u] = make_int4(0, 0, 0, 0);
+                if (p < end) {
+                    int x, y;
+                    if (small) {  // 32-bit index arithmetic (a 64-bit division costs more than the rest of the pixel's work)
+                        const uint32_t q = (uint32_t)p / (uint32_t)wo;
+                        x = (int)((uint32_t)p - q * (uint32_t)wo);
+                        y = (int)(q % (uint32_t)ho);
+                    } else {
+                        x = (int)(p % wo);
+                        y = (int)((p / wo) % ho);
+                    }
+                    cls[u] = border_class(y, ho, bc.nlo_h, bc.nhi_h, bc.nrc) * bc.ncc + border_class(x, wo, bc.nlo_w, bc.nhi_w, bc.ncc);
+                    v[u] = __ldg(reinterpret_cast<const int4 *>(e3 + p * c_out + ch));
+                }
             }
-            const int cls = border_class(y, ho, bc.nlo_h, bc.nhi_h, bc.nrc) * bc.ncc + border_class(x, wo, bc.nlo_w, bc.nhi_w, bc.ncc);
-            const int4 v = __ldg(reinterpret_cast<const int4 *>(e3 + p * c_out + ch));
-            const int8_t *b = reinterpret_cast<const int8_t *>(&v);
-            if (cls == interior) {
 #pragma unroll
-                for (int k = 0; k < 16; ++k) acc[k] += b[k];
-            } else {
-                int32_t *dst = cls_acc + cls * kClassSlab + sub * 16;
+            for (int u = 0; u < kTapUnroll; ++u) {
+                if (cls[u] == -2) continue;
+                const int8_t *b = reinterpret_cast<const int8_t *>(&v[u]);
+                if (cls[u] == interior) {
 #pragma unroll
-                for (int k = 0; k < 16; ++k)
-                    if (b[k]) atomicAdd(dst + k, (int)b[k]);
+                    for (int k = 0; k < 16; ++k) acc[k] += b[k];
+                } else {
+                    int32_t *dst = cls_acc + cls[u] * kClassSlab + sub * 16;
+#pragma unroll
+                    for (int k = 0; k < 16; ++k)
+                        if (b[k]) atomicAdd(dst + k, (int)b[k]);
+                }
             }
         }
         if (interior >= 0) {
@@ -991,24 +1109,24 @@ cudaError_t launch_sq_i32_scatter(const int32_t *src, const int32_t *src_exp, in
 }
 
 cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
-                          int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int c_in,
-                          const int32_t *parts, int num_parts, WgradCells *cells, DeviceState *dev, int sm_count,
-                          cudaStream_t s)
+                          int32_t *dst_exp, long long *copy_out, const long long *tap_sums, size_t replica_stride,
+                          int32_t b1_c, const int32_t *b1_dev, int c_in, const int32_t *parts, int num_parts,
+                          DeviceState *dev, int sm_count, cudaStream_t s)
 {
-    // the cells were zeroed by the caller's one memset at the head of the weight-gradient call
     const int groups = !parts ? 1 : (num_parts >= 32 ? 8 : (num_parts >= 8 ? 4 : 1));
     const int bx = 256 / groups;
     size_t blocks = (n + bx - 1) / bx;
     if (blocks > (size_t)sm_count * 16) blocks = (size_t)sm_count * 16;
     wgrad_finalize_kernel<<<(unsigned)blocks, 256, 0, s>>>(parts, num_parts, groups, n, const_cast<long long *>(src), tap_sums,
-                                                           b1_c, c_in, copy_out, cells);
-    sq_i64_kernel<<<grid_for(n, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, cells, dev);
+                                                           replica_stride, b1_c, b1_dev, c_in, copy_out, dev);
+    sq_i64_kernel<<<grid_for(n, sm_count, 4), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, dev);
     return cudaGetLastError();
 }
 
 cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const uint8_t *mask, const int16_t *x2,
-                                size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
-                                long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s, int *kernels)
+                                size_t n_el, int32_t gamma_c, const int32_t *gamma_dev, int8_t *e3, int32_t *e3_exp,
+                                long long *sum_e1, long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s,
+                                int *kernels, bool force_timeout)
 {
     const size_t n16 = n_el / 16;
     *kernels = 2;
@@ -1029,8 +1147,12 @@ cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const u
     const size_t max_blocks = (size_t)blocks_per_sm * sm_count;
     const size_t need_blocks = (n16 + (size_t)kThreads * kFusedGroups - 1) / ((size_t)kThreads * kFusedGroups);
     if (coop && n16 > 0 && need_blocks <= max_blocks) {
+        // self-test of the bounded wait: one arrival more than there are blocks and a short limit
+        unsigned expected = (unsigned)need_blocks + (force_timeout ? 1u : 0u);
+        uint32_t spin_limit = force_timeout ? 2048u : kSpinLimit;
         void *args[] = {(void *)&e0, (void *)&e0_exp, (void *)&mask, (void *)&x2, (void *)&n16, (void *)&gamma_c,
-                        (void *)&e3, (void *)&e3_exp, (void *)&sum_e1, (void *)&sum_e1x2, (void *)&dev};
+                        (void *)&gamma_dev, (void *)&e3, (void *)&e3_exp, (void *)&sum_e1, (void *)&sum_e1x2, (void *)&dev,
+                        (void *)&expected, (void *)&spin_limit};
         const cudaError_t e = cudaLaunchCooperativeKernel((const void *)prescale_fused_kernel, dim3((unsigned)need_blocks),
                                                           dim3(kThreads), args, 0, s);
         if (e != cudaErrorCooperativeLaunchTooLarge) {
@@ -1040,13 +1162,14 @@ cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const u
         (void)cudaGetLastError();  // fewer SMs at hand than at start-up (e.g. a partitioned device): two kernels instead
     }
     prescale_reduce_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, mask, x2, n16, dev);
-    prescale_apply_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, e0_exp, mask, n16, gamma_c, e3, e3_exp,
-                                                                       sum_e1, sum_e1x2, dev);
+    prescale_apply_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, e0_exp, mask, n16, gamma_c, gamma_dev, e3,
+                                                                       e3_exp, sum_e1, sum_e1x2, dev);
     return cudaGetLastError();
 }
 
 cudaError_t launch_update(const UpdateTensor *t, int num, int32_t lr_mant, int32_t lr_exp, int stochastic,
-                          uint64_t seed, uint64_t step, DeviceState *dev, int sm_count, cudaStream_t s)
+                          uint64_t seed, uint64_t step, unsigned long long *step_dev, DeviceState *dev, int sm_count,
+                          cudaStream_t s)
 {
     (void)sm_count;
     cudaError_t e = cudaMemsetAsync(dev->tensor_absmax, 0, sizeof(unsigned) * 256, s);
@@ -1077,8 +1200,9 @@ cudaError_t launch_update(const UpdateTensor *t, int num, int32_t lr_mant, int32
         }
         b.first_block[b.num] = blocks;
         if (blocks == 0) continue;
-        update_apply_kernel<<<blocks, kThreads, 0, s>>>(b, lr_mant, lr_exp, stochastic, seed, step, dev);
+        update_apply_kernel<<<blocks, kThreads, 0, s>>>(b, lr_mant, lr_exp, stochastic, seed, step, step_dev, dev);
     }
+    if (step_dev) step_bump_kernel<<<1, 1, 0, s>>>(step_dev);
     return cudaGetLastError();
 }
 
@@ -1109,21 +1233,27 @@ cudaError_t launch_b1_weight_table(const int8_t *w, int32_t *table, const eoq_co
     return cudaGetLastError();
 }
 
-cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, const eoq_conv_desc_t &d, int ho, int wo,
-                                 const BorderClasses &bc, int sm_count, cudaStream_t s)
+cudaError_t launch_weight_prep(const PrepBatch &b, cudaStream_t s)
+{
+    weight_prep_kernel<<<b.first_block[b.num], 128, 0, s>>>(b);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, size_t replica_stride, const eoq_conv_desc_t &d, int ho,
+                                 int wo, const BorderClasses &bc, int sm_count, cudaStream_t s)
 {
     // tap_sums was zeroed by the caller
     const int classes = bc.nrc * bc.ncc;
     const size_t pixels = (size_t)d.n * ho * wo;
     const int slabs = (d.c_out + kClassSlab - 1) / kClassSlab;
-    int blocks = (2 * sm_count + slabs - 1) / slabs;  // more blocks only add contention on the per-tap cells
+    int blocks = (sm_count + slabs - 1) / slabs;  // more blocks only add atomics on the per-tap cells
     size_t ppb = (pixels + blocks - 1) / blocks;
     if (ppb < 64) ppb = 64;
     if (ppb > (1u << 23)) ppb = 1u << 23;  // keeps the int32 class sums exact
     blocks = (int)((pixels + ppb - 1) / ppb);
     dim3 grid(blocks, slabs);
-    b1_tap_sums_kernel<<<grid, 256, sizeof(int32_t) * classes * kClassSlab, s>>>(e3, tap_sums, d.c_out, ho, wo, pixels, (int)ppb,
-                                                                               bc, d);
+    b1_tap_sums_kernel<<<grid, 256, sizeof(int32_t) * classes * kClassSlab, s>>>(e3, tap_sums, replica_stride, d.c_out, ho, wo,
+                                                                               pixels, (int)ppb, bc, d);
     return cudaGetLastError();
 }
 

@@ -85,10 +85,42 @@ __device__ __forceinline__ ForwardOperands forward_operands(const IgemmParams &p
     return o;
 }
 
+// The three scalar codes of the forward chain as the epilogue uses them: the host values of the launch, or the
+// values read from device memory when the caller keeps them there (they then change from one replay of a captured
+// graph to the next without a new capture).
+struct FwdScalars {
+    int32_t b1, gamma, b2;
+};
+
+// Every epilogue thread calls this once per kernel.  Device-resident codes outside their range (16 bits each; b1
+// also bounded by what keeps the accumulator inside int32) raise EOQ_DEV_RANGE and are clamped.
+__device__ __forceinline__ FwdScalars load_fwd_scalars(const IgemmParams &p)
+{
+    FwdScalars s{p.b1_c, p.gamma_c, p.b2_c};
+    if (p.scal_dev) {
+        s.b1 = __ldg(p.scal_dev);
+        s.gamma = __ldg(p.scal_dev + 1);
+        s.b2 = __ldg(p.scal_dev + 2);
+        // |acc| <= k_total * (127 + |b1|) * 127 must stay below 2^31 - 2^24
+        const long long room = (2147483647ll - 16777216ll) / (127ll * (p.k_total > 0 ? p.k_total : 1)) - 127ll;
+        const int32_t b1_lim = (int32_t)(room < 0 ? 0 : (room > 32767 ? 32767 : room));
+        const bool bad = s.b1 < -b1_lim || s.b1 > b1_lim || s.gamma < -32768 || s.gamma > 32767 || s.b2 < -32768 ||
+                         s.b2 > 32767 || (!p.b1_table && s.b1 != 0);
+        if (bad) {
+            if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicOr(&p.dev->status, EOQ_DEV_RANGE);
+            s.b1 = p.b1_table ? clampi(s.b1, -b1_lim, b1_lim) : 0;
+            s.gamma = clampi(s.gamma, -32768, 32767);
+            s.b2 = clampi(s.b2, -32768, 32767);
+        }
+    }
+    return s;
+}
+
 // `acc1` holds the tile's second partial sums when `two` is set; kRelu = a ReLU follows.
 template <bool kShift7, bool kRelu>
-__device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t (&acc)[32], const uint32_t (&acc1)[32],
-                                           bool two, size_t off, const ForwardOperands &ops, int shift)
+__device__ __forceinline__ void forward_16(const IgemmParams &p, const FwdScalars &fs, const uint32_t (&acc)[32],
+                                           const uint32_t (&acc1)[32], bool two, size_t off, const ForwardOperands &ops,
+                                           int shift)
 {
     int32_t a[16];
 #pragma unroll
@@ -104,10 +136,10 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t 
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int4 v = ops.table[i];
-            a[4 * i + 0] += p.b1_c * v.x;
-            a[4 * i + 1] += p.b1_c * v.y;
-            a[4 * i + 2] += p.b1_c * v.z;
-            a[4 * i + 3] += p.b1_c * v.w;
+            a[4 * i + 0] += fs.b1 * v.x;
+            a[4 * i + 1] += fs.b1 * v.y;
+            a[4 * i + 2] += fs.b1 * v.z;
+            a[4 * i + 3] += fs.b1 * v.w;
         }
     }
     if (p.acc_out) {
@@ -147,8 +179,8 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const uint32_t 
     // x4 - 1 = gamma * x2 + (b2 + shortcut) * 2^7 - 1 = gamma * q + add, the bias of q folded into add (mod 2^32).
     // Forming x4 - 1 instead of x4 makes its sign bit [x4 <= 0], the complement of the mask bit, so the mask
     // costs one funnel shift per element; the + 1 rides on the add-min that clamps x4.
-    const uint32_t g = (uint32_t)p.gamma_c;
-    const uint32_t base = ((uint32_t)p.b2_c << 7) - g * q_bias - 1u;
+    const uint32_t g = (uint32_t)fs.gamma;
+    const uint32_t base = ((uint32_t)fs.b2 << 7) - g * q_bias - 1u;
     uint32_t add[16];
     if (p.shortcut) {
         const int4 v = ops.shortcut;

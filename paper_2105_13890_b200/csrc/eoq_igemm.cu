@@ -225,6 +225,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         constexpr int kParts = kEpilogueWarps / 8;
         const int g_begin = (groups * part) / kParts, g_end = (groups * (part + 1)) / kParts;
         const bool fwd = p.epilogue == kEpiForward;
+        const FwdScalars fs = fwd ? load_fwd_scalars(p) : FwdScalars{0, 0, 0};
         int shift = 7;
         if (fwd && p.x_exp) {
             shift = -__ldg(p.x_exp);
@@ -272,11 +273,11 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                     if (fwd) {
                         const bool two = nacc == 2;
                         if (shift == 7) {
-                            if (p.relu) forward_16<true, true>(p, r, r2, two, off, ops, 7);
-                            else forward_16<true, false>(p, r, r2, two, off, ops, 7);
+                            if (p.relu) forward_16<true, true>(p, fs, r, r2, two, off, ops, 7);
+                            else forward_16<true, false>(p, fs, r, r2, two, off, ops, 7);
                         } else {
-                            if (p.relu) forward_16<false, true>(p, r, r2, two, off, ops, shift);
-                            else forward_16<false, false>(p, r, r2, two, off, ops, shift);
+                            if (p.relu) forward_16<false, true>(p, fs, r, r2, two, off, ops, shift);
+                            else forward_16<false, false>(p, fs, r, r2, two, off, ops, shift);
                         }
                     } else {
                         mx = max(mx, dgrad_16(p, r, off));

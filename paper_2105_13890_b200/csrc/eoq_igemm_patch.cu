@@ -266,6 +266,7 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
         const int g_begin = (groups * part) / kParts, g_end = (groups * (part + 1)) / kParts;
         const int yl = row / pl.pw, xx = row % pl.pw;  // position of this thread's row in the patch raster
         const bool fwd = p.epilogue == kEpiForward;
+        const FwdScalars fs = fwd ? load_fwd_scalars(p) : FwdScalars{0, 0, 0};
         uint32_t acc_phase = 0, mx = 0;
         bool ok = true;
         // (column tile, image, row tile in the image) of the current tile, carried from tile to tile: the step
@@ -308,8 +309,8 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                 }
                 if (valid && col < p.N) {
                     if (fwd) {
-                        if (p.relu) forward_16<true, true>(p, r, r2, nacc == 2, off, ops, 7);
-                        else forward_16<true, false>(p, r, r2, nacc == 2, off, ops, 7);
+                        if (p.relu) forward_16<true, true>(p, fs, r, r2, nacc == 2, off, ops, 7);
+                        else forward_16<true, false>(p, fs, r, r2, nacc == 2, off, ops, 7);
                     }
                     else mx = max(mx, dgrad_16(p, r, off));
                 }

@@ -24,6 +24,7 @@ struct DeviceState {
     unsigned tensor_absmax[256];  // per-tensor maxima of the multi-tensor update
     unsigned ticket;       // blocks of the kernel that consumes the cells last count themselves here (see last_block_done)
     unsigned arrivals;     // grid-wide barrier of the one-kernel error head (cooperative launch)
+    unsigned long long probe_cycles;  // eoq_probe_mma_i8: longest issue loop of the last launch, in SM clock cycles
 };
 // Invariant: absmax_u32, absmax_u64, sum0, sum1, ticket and arrivals are zero whenever no call is in flight on the handle.
 // The kernel that reads a call's reductions last puts the cells it used back to zero (its last block does), so
@@ -44,6 +45,8 @@ struct Handle {
     DeviceState *dev;
     unsigned long long launches;  // kernels launched through this handle
     bool profiling;
+    bool gemm_only;               // timing aid: dgrad and wgrad calls launch their GEMM kernel only (eoq_profile_gemm_only)
+    bool force_timeout;           // self-test: the next error-head call makes its grid-wide wait run out
     int num_records;
     ProfRecord *records;          // kMaxProfRecords entries, allocated on first eoq_profile_start
     // Branch stream of the weight-gradient call: the b1 tap sums do not depend on the GEMM, so they are issued
@@ -96,6 +99,8 @@ struct IgemmParams {
     // forward epilogue
     const int32_t *x_exp;     // device exponent of the input or null
     int32_t b1_c, gamma_c, b2_c;
+    const int32_t *scal_dev;  // device {b1_c, gamma_c, b2_c} replacing the three host values, or null
+    int k_total;              // taps * input channels: bounds the accumulator when b1 is only known on the device
     const int32_t *b1_table;  // [classes][N] tap-validity sums of the weights (null when b1_c == 0)
     int b1_nlo_h, b1_nhi_h, b1_nrc, b1_nlo_w, b1_nhi_w, b1_ncc;
     const int8_t *shortcut;
@@ -202,6 +207,10 @@ cudaError_t launch_wgrad_patch(const WgradPatchPlan &pl, const CUtensorMap &map_
 size_t wgrad_smem_bytes(const WgradParams &p);
 cudaError_t launch_wgrad(const WgradParams &p, const CUtensorMap &map_x, const CUtensorMap &map_e, cudaStream_t stream);
 
+// Issue-rate measurement of tcgen05.mma kind::i8 (eoq_probe.cu): `grid` CTAs, each `iters` x 4 MMAs of 128 x n_cols x 32.
+cudaError_t launch_probe_mma_i8(int n_cols, int iters, int grid, DeviceState *dev, unsigned long long *cycles_out,
+                                cudaStream_t s);
+
 // ---------------------------------------------------------------------------------------------
 // Elementwise / reduction kernels
 // ---------------------------------------------------------------------------------------------
@@ -217,30 +226,31 @@ cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bi
                           int sm_count, cudaStream_t s);
 // Q_g of the exact sums.  `src` holds int64 sums; when `parts` is given the sums are first formed from
 // `num_parts` int32 slices of n elements each (and written to src).
-// Reduction cell of one weight-gradient call; it lives in the call's workspace next to the tap sums so that one
-// memset at the head of the call clears everything the call accumulates into.
-struct WgradCells {
-    unsigned long long absmax;  // max |sum| over the weight tensor
-    unsigned long long pad;
-};
 cudaError_t launch_sq_i32_scatter(const int32_t *src, const int32_t *src_exp, int exp_bias, int n_img, int hh, int ww, int c,
                                   int stride, int hq, int wq, int8_t *dst, int32_t *dst_exp, long long *sum_codes,
                                   DeviceState *dev, int sm_count, cudaStream_t s);
+// b1 is b1_c, or the code at b1_dev when that is given.  Two kernels: slice sum + b1 term + max, then Q_g; the maximum
+// travels through the handle's absmax_u64 cell, which the second kernel puts back to zero.
+// tap_sums: kTapReplicas copies, `replica_stride` elements apart, whose sum is the b1 error sum per (oc, tap).
 cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
-                          int32_t *dst_exp, long long *copy_out, const long long *tap_sums, int32_t b1_c, int c_in,
-                          const int32_t *parts, int num_parts, WgradCells *cells, DeviceState *dev, int sm_count,
-                          cudaStream_t s);
+                          int32_t *dst_exp, long long *copy_out, const long long *tap_sums, size_t replica_stride,
+                          int32_t b1_c, const int32_t *b1_dev, int c_in, const int32_t *parts, int num_parts,
+                          DeviceState *dev, int sm_count, cudaStream_t s);
+// gamma is gamma_c, or the code at gamma_dev when that is given.  force_timeout: self-test of the bounded wait.
 cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const uint8_t *mask, const int16_t *x2,
-                                size_t n_el, int32_t gamma_c, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
-                                long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s, int *kernels);
+                                size_t n_el, int32_t gamma_c, const int32_t *gamma_dev, int8_t *e3, int32_t *e3_exp,
+                                long long *sum_e1, long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s,
+                                int *kernels, bool force_timeout);
 struct UpdateTensor {
     int8_t *w;
     const int8_t *g;
     const int32_t *g_exp;
     unsigned long long n;
 };
+// step_dev (device, optional): the step counter is read from it and it is incremented behind the update.
 cudaError_t launch_update(const UpdateTensor *t, int num, int32_t lr_mant, int32_t lr_exp, int stochastic,
-                          uint64_t seed, uint64_t step, DeviceState *dev, int sm_count, cudaStream_t s);
+                          uint64_t seed, uint64_t step, unsigned long long *step_dev, DeviceState *dev, int sm_count,
+                          cudaStream_t s);
 cudaError_t launch_layout_convert(const int8_t *src, int8_t *dst, int n, int c, int h, int w, int to_nhwc,
                                   cudaStream_t s);
 cudaError_t launch_weight_transpose(const int8_t *w, int8_t *wt, int c_out, int taps, int c_in, cudaStream_t s);
@@ -250,8 +260,26 @@ struct BorderClasses {
 };
 cudaError_t launch_b1_weight_table(const int8_t *w, int32_t *table, const eoq_conv_desc_t &d, const BorderClasses &bc,
                                    cudaStream_t s);
-cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, const eoq_conv_desc_t &d, int ho, int wo,
-                                 const BorderClasses &bc, int sm_count, cudaStream_t s);
+constexpr int kTapReplicas = 4;  // copies of the b1 error sums the blocks spread their atomics over
+cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, size_t replica_stride, const eoq_conv_desc_t &d, int ho,
+                                 int wo, const BorderClasses &bc, int sm_count, cudaStream_t s);
 constexpr int kMaxBorderClasses = 64;  // classes (rows x columns) the b1 kernels keep in shared memory
+
+// eoq_weight_prep: one launch derives the b1 tables (and the row-padded first-layer weights) of up to kPrepChunk layers
+struct PrepItem {
+    const int8_t *w;
+    int32_t *table;   // [classes][c_out]
+    int8_t *w_rows;   // [c_out][kh][8][c_in] or null
+    eoq_conv_desc_t d;
+    int ho, wo;
+    BorderClasses bc;
+};
+constexpr int kPrepChunk = 32;
+struct PrepBatch {
+    PrepItem item[kPrepChunk];
+    int first_block[kPrepChunk + 1];
+    int num;
+};
+cudaError_t launch_weight_prep(const PrepBatch &b, cudaStream_t s);
 
 }  // namespace eoq

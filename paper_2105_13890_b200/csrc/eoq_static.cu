@@ -63,6 +63,8 @@ extern "C" int eoq_conv_dgrad_static(const eoq_conv_desc_t *desc, const int8_t *
     h.dev = reinterpret_cast<DeviceState *>(pd.scratch);
     h.launches = 0;
     h.profiling = false;
+    h.force_timeout = false;
+    h.gemm_only = false;
     h.num_records = 0;
     h.records = nullptr;
     h.branch = nullptr;

@@ -25,12 +25,14 @@ EXPORTS = [
     "eoq_create", "eoq_destroy", "eoq_workspace_size", "eoq_conv_fwd", "eoq_conv_dgrad", "eoq_conv_wgrad",
     "eoq_quantize", "eoq_quantize_image", "eoq_err_prescale", "eoq_update", "eoq_layout_convert", "eoq_last_status",
     "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count", "eoq_set_gemm_ctas",
-    "eoq_conv_dgrad_static",
+    "eoq_conv_dgrad_static", "eoq_conv_fwd_dev", "eoq_weight_prep_size", "eoq_weight_prep", "eoq_conv_wgrad_dev",
+    "eoq_err_prescale_dev", "eoq_update_dev", "eoq_describe_plan", "eoq_debug_force_wait_timeout", "eoq_probe_mma_i8", "eoq_profile_gemm_only",
 ]
 EOQ_STATIC_SCRATCH_BYTES = 16 << 20
 EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
-EOQ_PROF_KINDS = 8
-EOQ_PROF_NAMES = ["igemm_fwd", "igemm_dgrad", "wgrad_gemm", "err_head", "dgrad_aux", "wgrad_aux", "fwd_aux", "other"]
+EOQ_PROF_KINDS = 11
+EOQ_PROF_NAMES = ["igemm_fwd", "igemm_dgrad", "wgrad_gemm", "err_head", "dgrad_aux", "wgrad_aux", "fwd_aux", "other", "update",
+                  "input_quantizer", "wgrad_taps"]
 
 
 class EoqError(RuntimeError):
@@ -87,6 +89,17 @@ def lib() -> C.CDLL:
         L.eoq_profile_stop.argtypes = [vp, C.POINTER(C.c_int), C.POINTER(C.c_double)]
         L.eoq_launch_count.argtypes = [vp]
         L.eoq_set_gemm_ctas.argtypes = [vp, C.c_int]
+        L.eoq_conv_fwd_dev.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, C.c_int, vp, vp, vp, vp]
+        L.eoq_weight_prep_size.argtypes = [dp, C.POINTER(sz)]
+        L.eoq_weight_prep.argtypes = [vp, C.c_int, dp, C.POINTER(vp), C.POINTER(vp), vp]
+        L.eoq_conv_wgrad_dev.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.eoq_err_prescale_dev.argtypes = [vp, vp, vp, vp, vp, sz, vp, vp, vp, vp, vp, vp]
+        L.eoq_update_dev.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), i32, i32,
+                                     C.c_int, u64, vp, vp]
+        L.eoq_describe_plan.argtypes = [vp, dp, C.c_int, C.c_char_p, sz]
+        L.eoq_debug_force_wait_timeout.argtypes = [vp]
+        L.eoq_profile_gemm_only.argtypes = [vp, C.c_int]
+        L.eoq_probe_mma_i8.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
         L.eoq_status_string.argtypes = [C.c_int]
         L.eoq_status_string.restype = C.c_char_p
         for name in EXPORTS:
@@ -258,3 +271,86 @@ def eoq_conv_dgrad_static(desc, e3, e3_exp, w, e4, e4_exp, sum_e4=None, status_o
     if check:
         _check(st, "eoq_conv_dgrad_static")
     return st
+
+
+def eoq_conv_fwd_dev(handle, desc, x, x_exp, scalars, w, w_prep, shortcut, relu, x5, x2=None, relu_mask=None, stream=None,
+                     check: bool = True) -> int:
+    """eoq_conv_fwd with the scalars {b1_c, gamma_c, b2_c} in device memory and prepared weights (eoq_weight_prep)."""
+    st = lib().eoq_conv_fwd_dev(handle, C.byref(desc), _ptr(x), _ptr(x_exp), _ptr(scalars), _ptr(w), _ptr(w_prep),
+                                _ptr(shortcut), 1 if relu else 0, _ptr(x5), _ptr(x2), _ptr(relu_mask), _stream(stream))
+    if check:
+        _check(st, "eoq_conv_fwd_dev")
+    return st
+
+
+def eoq_weight_prep_size(desc: eoq_conv_desc_t) -> int:
+    out = C.c_size_t(0)
+    _check(lib().eoq_weight_prep_size(C.byref(desc), C.byref(out)), "eoq_weight_prep_size")
+    return out.value
+
+
+def eoq_weight_prep(handle, descs: Sequence[eoq_conv_desc_t], w: Sequence, prep: Sequence, stream=None,
+                    check: bool = True) -> int:
+    num = len(descs)
+    darr = (eoq_conv_desc_t * num)(*descs)
+    arr = C.c_void_p * num
+    st = lib().eoq_weight_prep(handle, num, darr, arr(*[_ptr(t) for t in w]), arr(*[_ptr(t) for t in prep]),
+                               _stream(stream))
+    if check:
+        _check(st, "eoq_weight_prep")
+    return st
+
+
+def eoq_conv_wgrad_dev(handle, desc, e3, e3_exp, x, b1_c, g, g_exp, workspace=None, stream=None, check: bool = True) -> int:
+    st = lib().eoq_conv_wgrad_dev(handle, C.byref(desc), _ptr(e3), _ptr(e3_exp), _ptr(x), _ptr(b1_c), _ptr(g),
+                                  _ptr(g_exp), _ptr(workspace), _nbytes(workspace), _stream(stream))
+    if check:
+        _check(st, "eoq_conv_wgrad_dev")
+    return st
+
+
+def eoq_err_prescale_dev(handle, e0, e0_exp, relu_mask, x2, n_el, gamma_c, e3, e3_exp, sum_e1=None, sum_e1x2=None,
+                         stream=None, check: bool = True) -> int:
+    st = lib().eoq_err_prescale_dev(handle, _ptr(e0), _ptr(e0_exp), _ptr(relu_mask), _ptr(x2), int(n_el), _ptr(gamma_c),
+                                    _ptr(e3), _ptr(e3_exp), _ptr(sum_e1), _ptr(sum_e1x2), _stream(stream))
+    if check:
+        _check(st, "eoq_err_prescale_dev")
+    return st
+
+
+def eoq_update_dev(handle, w: Sequence, g: Sequence, g_exp: Sequence, lr_mant: int, lr_exp: int, round_mode: int, seed: int,
+                   step, stream=None, check: bool = True) -> int:
+    """eoq_update with the step counter in device memory (a one-element int64/uint64 tensor, bumped by the call)."""
+    num = len(w)
+    arr = C.c_void_p * num
+    sizes = (C.c_size_t * num)(*[t.numel() for t in w])
+    st = lib().eoq_update_dev(handle, num, arr(*[_ptr(t) for t in w]), arr(*[_ptr(t) for t in g]),
+                              arr(*[_ptr(t) for t in g_exp]), sizes, int(lr_mant), int(lr_exp), int(round_mode), int(seed),
+                              _ptr(step), _stream(stream))
+    if check:
+        _check(st, "eoq_update_dev")
+    return st
+
+
+def eoq_describe_plan(handle, desc, pass_: int) -> str:
+    buf = C.create_string_buffer(256)
+    _check(lib().eoq_describe_plan(handle, C.byref(desc), int(pass_), buf, 256), "eoq_describe_plan")
+    return buf.value.decode()
+
+
+def eoq_debug_force_wait_timeout(handle) -> None:
+    """Makes the next one-kernel error-head call on this handle run out at its (bounded) grid-wide wait."""
+    _check(lib().eoq_debug_force_wait_timeout(handle), "eoq_debug_force_wait_timeout")
+
+
+def eoq_probe_mma_i8(handle, n_cols: int, iters: int, launches: int, stream=None):
+    """-> (TOPS over the timed launches, SM cycles per 128 x n_cols x 32 MMA) of tcgen05.mma kind::i8."""
+    tops, cyc = C.c_double(0), C.c_double(0)
+    _check(lib().eoq_probe_mma_i8(handle, int(n_cols), int(iters), int(launches), C.byref(tops), C.byref(cyc), _stream(stream)),
+           "eoq_probe_mma_i8")
+    return tops.value, cyc.value
+
+
+def eoq_profile_gemm_only(handle, on: bool) -> None:
+    """Timing aid: dgrad / wgrad calls launch their GEMM kernel only (their outputs are then not produced)."""
+    _check(lib().eoq_profile_gemm_only(handle, 1 if on else 0), "eoq_profile_gemm_only")

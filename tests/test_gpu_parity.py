@@ -411,3 +411,170 @@ def test_strided_1x1_dgrad_without_sum_dump(d):
         assert G.status_clear() == 0
         assert np.array_equal(G.host(e4).astype(np.int32), ref) and e4_exp.item() == p4
         assert s4.item() == int(ref.astype(np.int64).sum())
+
+
+# ------------------------------------------------------------------ paths that only large problems take
+
+WIDE_CASES = [
+    # (geometry, pass, expected fragment of the plan): a 256-column tile needs at least twice as many tiles as SMs
+    (ConvDesc(13, 56, 56, 64, 256, 1, 1, 1, 0), eoq.EOQ_PASS_FWD, "kernel=igemm tile_n=256"),
+    (ConvDesc(13, 56, 56, 256, 64, 1, 1, 1, 0), eoq.EOQ_PASS_DGRAD, "kernel=igemm classes=1 tile_n=256"),
+    (ConvDesc(148, 14, 14, 256, 256, 3, 3, 1, 1), eoq.EOQ_PASS_FWD, "kernel=igemm_patch tile_n=256 accumulators=1"),
+    (ConvDesc(148, 14, 14, 256, 256, 3, 3, 1, 1), eoq.EOQ_PASS_DGRAD, "kernel=igemm_patch tile_n=256 accumulators=1"),
+]
+
+
+@pytest.mark.parametrize("d,pass_,plan", WIDE_CASES, ids=["igemm_fwd", "igemm_dgrad", "patch_fwd", "patch_dgrad"])
+def test_256_column_tiles(d, pass_, plan):
+    """Both implicit-GEMM kernels with 256-column tiles (one accumulator per tile), which only problems with at
+    least 2 x SMs row tiles take; the plan report confirms the path before the results are compared."""
+    gd = G.gdesc(d)
+    assert plan in eoq.eoq_describe_plan(G.handle(), gd, pass_)
+    x0, w, sc, e3 = layer_data(d, 7300 + d.c_in, wrange=12)
+    if pass_ == eoq.EOQ_PASS_FWD:
+        ref = oracle.layer_forward(d, x0, -3, w, 90, 5, sc, True)
+        shape = ref["x5"].shape
+        x5, x2, acc = G.zeros(shape, torch.int8), G.zeros(shape, torch.int16), G.zeros(shape, torch.int32)
+        mask = G.zeros((ref["x5"].size + 7) // 8, torch.uint8)
+        eoq.eoq_conv_fwd(G.handle(), gd, G.dev(x0), None, -3, G.dev(w), 90, 5, G.dev(sc), True, x5, x2, mask, acc,
+                         G.workspace(gd, eoq.EOQ_PASS_FWD))
+        assert G.status_clear() == 0
+        assert np.array_equal(G.host(acc).astype(np.int64), ref["acc"])
+        assert np.array_equal(G.host(x2).astype(np.int32), ref["x2"])
+        assert np.array_equal(G.host(x5), ref["x5"])
+        assert np.array_equal(G.unpack_mask(mask, shape), ref["mask"])
+    else:
+        B = oracle.conv_dgrad_acc(d, e3, w)
+        e4, p4, _ = oracle.sq_int(B, -11 - 7)
+        e4_d, acc = G.zeros(B.shape, torch.int8), G.zeros(B.shape, torch.int32)
+        e4_exp, s4 = G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+        eoq.eoq_conv_dgrad(G.handle(), gd, G.dev(e3), G.dev(np.array([-11], dtype=np.int32)), G.dev(w), e4_d, e4_exp, s4, acc,
+                           G.workspace(gd, eoq.EOQ_PASS_DGRAD))
+        assert G.status_clear() == 0
+        assert np.array_equal(G.host(acc).astype(np.int64), B) and e4_exp.item() == p4
+        assert np.array_equal(G.host(e4_d).astype(np.int32), e4) and s4.item() == int(e4.astype(np.int64).sum())
+
+
+# ------------------------------------------------------------------ device-resident scalars and prepared weights
+
+DEV_SHAPES = [SHAPES[0], SHAPES[3], SHAPES[5], SHAPES[8], SHAPES[12]]
+
+
+@pytest.mark.parametrize("d", DEV_SHAPES, ids=[IDS[SHAPES.index(d)] for d in DEV_SHAPES])
+def test_device_scalar_entry_points(d):
+    """eoq_weight_prep + eoq_conv_fwd_dev, eoq_err_prescale_dev and eoq_conv_wgrad_dev against the oracle, with the
+    scalars rewritten in device memory between two calls (what a replayed graph sees)."""
+    x0, w, sc, _ = layer_data(d, 8100 + d.c_out)
+    e0 = synth.normal_codes((d.n, d.ho, d.wo, d.c_out), 8101, d.h)
+    gd = G.gdesc(d)
+    h = G.handle()
+    prep = G.zeros(max(eoq.eoq_weight_prep_size(gd), 256), torch.uint8)
+    w_d = G.dev(w)
+    eoq.eoq_weight_prep(h, [gd], [w_d], [prep])
+    scal = G.zeros(3, torch.int32)
+    shape = (d.n, d.ho, d.wo, d.c_out)
+    x5, x2 = G.zeros(shape, torch.int8), G.zeros(shape, torch.int16)
+    mask = G.zeros((int(np.prod(shape)) + 7) // 8, torch.uint8)
+    e3, e3_exp = G.zeros(shape, torch.int8), G.zeros(1, torch.int32)
+    s1, s2 = G.zeros(1, torch.int64), G.zeros(1, torch.int64)
+    g_d, g_exp = G.zeros(w.shape, torch.int8), G.zeros(1, torch.int32)
+    ws = G.workspace(gd, eoq.EOQ_PASS_WGRAD)
+    for b1, gamma, b2 in ((-3, 90, 5), (6, -131, -9), (0, 128, 0)):
+        scal.copy_(torch.tensor([b1, gamma, b2], dtype=torch.int32))
+        ref = oracle.layer_forward(d, x0, b1, w, gamma, b2, sc, True)
+        eoq.eoq_conv_fwd_dev(h, gd, G.dev(x0), None, scal, w_d, prep, G.dev(sc), True, x5, x2, mask)
+        assert G.status_clear() == 0
+        assert np.array_equal(G.host(x5), ref["x5"]) and np.array_equal(G.host(x2).astype(np.int32), ref["x2"])
+        assert np.array_equal(G.unpack_mask(mask, shape), ref["mask"])
+        bwd = oracle.layer_backward(d, e0, -12, ref["mask"], ref["x2"], x0, b1, w, gamma)
+        eoq.eoq_err_prescale_dev(h, G.dev(e0), G.dev(np.array([-12], dtype=np.int32)), mask, x2, e0.size, scal[1:2], e3, e3_exp,
+                                 s1, s2)
+        eoq.eoq_conv_wgrad_dev(h, gd, e3, e3_exp, G.dev(x0), scal[0:1], g_d, g_exp, ws)
+        z = bwd["g_w_zero"]
+        assert G.status_clear() == (eoq.EOQ_DEV_SQ_ZERO if z else 0)
+        assert np.array_equal(G.host(e3), bwd["e3"]) and e3_exp.item() == bwd["p3"]
+        assert s1.item() == bwd["sum_e1"] and s2.item() == bwd["sum_e1x2"]
+        assert np.array_equal(G.host(g_d), bwd["g_w"]) and g_exp.item() == bwd["p_gw"]
+
+
+def test_device_scalars_out_of_range_are_flagged():
+    d = SHAPES[1]
+    x0, w, _, _ = layer_data(d, 8200)
+    gd = G.gdesc(d)
+    prep = G.zeros(max(eoq.eoq_weight_prep_size(gd), 256), torch.uint8)
+    eoq.eoq_weight_prep(G.handle(), [gd], [G.dev(w)], [prep])
+    x5 = G.zeros((d.n, d.ho, d.wo, d.c_out), torch.int8)
+    scal = G.dev(np.array([0, 1 << 20, 0], dtype=np.int32))
+    eoq.eoq_conv_fwd_dev(G.handle(), gd, G.dev(x0), None, scal, G.dev(w), prep, None, True, x5)
+    assert G.status_clear() == eoq.EOQ_DEV_RANGE
+    # a bias without prepared weights cannot be applied: flagged, counted as zero
+    scal = G.dev(np.array([5, 128, 0], dtype=np.int32))
+    eoq.eoq_conv_fwd_dev(G.handle(), gd, G.dev(x0), None, scal, G.dev(w), None, None, True, x5)
+    assert G.status_clear() == eoq.EOQ_DEV_RANGE
+    ref = oracle.layer_forward(d, x0, 0, w, 128, 0)
+    assert np.array_equal(G.host(x5), ref["x5"])
+
+
+def test_update_with_device_step_counter():
+    sizes = [4096, 36864 + 5, 16]
+    ws = [synth.int8_uniform(n, 8301, i) for i, n in enumerate(sizes)]
+    gs = [synth.normal_codes(n, 8302, i, std_codes=40) for i, n in enumerate(sizes)]
+    pgs = [-9, -11, -8]
+    w_d = [G.dev(w) for w in ws]
+    step = G.dev(np.array([5], dtype=np.int64))
+    cur = [w.astype(np.int32) for w in ws]
+    for k in range(3):
+        eoq.eoq_update_dev(G.handle(), w_d, [G.dev(g) for g in gs], [G.dev(np.array([p], dtype=np.int32)) for p in pgs],
+                           37, -8, eoq.EOQ_ROUND_STOCHASTIC, 11, step)
+        assert G.status_clear() == 0
+        for i in range(len(sizes)):
+            cur[i], _, _ = oracle.update(cur[i], gs[i], pgs[i], 37, -8, stochastic=True, seed=11, step=5 + k, tensor_id=i)
+            assert np.array_equal(G.host(w_d[i]).astype(np.int32), cur[i]), (k, i)
+    assert step.item() == 8
+
+
+def test_wgrad_two_kernel_finish_path():
+    """A weight tensor too large for the one-kernel slice sum + Q_g (more sums than a resident grid keeps in
+    registers) takes the finalize + Q_g pair."""
+    d = ConvDesc(1, 6, 6, 1024, 1024, 3, 3, 1, 1)   # 9.4 M weights
+    x0, _, _, e3 = layer_data(d, 8400)
+    Gacc = oracle.conv_wgrad_acc(d, e3, x0, -2)
+    g, pg, _ = oracle.sq_int(Gacc, -9 - 7)
+    gd = G.gdesc(d)
+    g_d, g_exp = G.zeros(Gacc.shape, torch.int8), G.zeros(1, torch.int32)
+    h = G.handle()
+    for _ in range(2):
+        before = eoq.eoq_launch_count(h)
+        eoq.eoq_conv_wgrad(h, gd, G.dev(e3), G.dev(np.array([-9], dtype=np.int32)), G.dev(x0), -2, g_d, g_exp, None,
+                           G.workspace(gd, eoq.EOQ_PASS_WGRAD))
+        assert G.status_clear() == 0
+        assert eoq.eoq_launch_count(h) - before == 4  # tap sums, GEMM, finalize, Q_g
+        assert np.array_equal(G.host(g_d).astype(np.int32), g) and g_exp.item() == pg
+
+
+# ------------------------------------------------------------------ a bounded wait that runs out
+
+def test_wait_that_runs_out_reports_timeout_and_leaves_the_handle_usable():
+    """The grid-wide wait of the one-kernel error head is made to run out (it waits for one block more than
+    exists, with a short limit).  Nothing traps or hangs: the kernel returns, EOQ_DEV_TIMEOUT is reported, no output
+    is written, the reduction cells are clean again, and the next call on the handle is bit-exact."""
+    n_el = 1 << 16
+    e0 = synth.normal_codes(n_el, 8500, 1)
+    mask = synth.bits(n_el, 8501, 0)
+    ref, p3, s1, _, _ = oracle.err_prescale(e0, -12, mask, None, 118)
+    h = eoq.eoq_create(0)
+    try:
+        e3 = torch.full((n_el,), 55, dtype=torch.int8, device="cuda:0")
+        e3_exp, s1_d = torch.full((1,), 1234, dtype=torch.int32, device="cuda:0"), G.zeros(1, torch.int64)
+        args = (G.dev(e0), G.dev(np.array([-12], dtype=np.int32)), G.dev(G.pack_mask(mask)), None, n_el, 118, e3, e3_exp, s1_d, None)
+        eoq.eoq_debug_force_wait_timeout(h)
+        eoq.eoq_err_prescale(h, *args)
+        assert eoq.eoq_last_status(h) == eoq.EOQ_DEV_TIMEOUT
+        assert (G.host(e3) == 55).all() and e3_exp.item() == 1234      # nothing was written
+        assert eoq.eoq_last_status(h) == 0                             # reported once, then clear
+        for _ in range(2):
+            eoq.eoq_err_prescale(h, *args)
+            assert eoq.eoq_last_status(h) == 0
+            assert np.array_equal(G.host(e3), ref) and e3_exp.item() == p3 and s1_d.item() == s1
+    finally:
+        eoq.eoq_destroy(h)

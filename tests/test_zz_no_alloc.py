@@ -2,13 +2,15 @@
 
 eoq_conv_dgrad_static serves callers that may not allocate device memory (no handle, no workspace: its scratch
 is a static device array inside the library).  It must give the same e4 codes, exponent and code sum as
-eoq_conv_dgrad, on a first call and again on a second call that finds the array dirty from the first.
+eoq_conv_dgrad and as the oracle, on a first call and again on a second call that finds the array dirty from the first.
 Collected last on purpose: if it fails, every other test has already run.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
+from oracle import ConvDesc
 from paper_2105_13890_b200 import eoq, synth
 
 pytestmark = pytest.mark.gpu
@@ -48,6 +50,11 @@ def test_static_dgrad_matches_regular_entry_point_twice_in_a_row():
             assert torch.equal(got_e4, ref_e4)          # integer codes: bit for bit
             assert got_exp.item() == ref_exp.item() and got_sum.item() == ref_sum.item()
             assert got_e4.any()
+            # and against the oracle itself
+            od = ConvDesc(desc.n, desc.h, desc.w, desc.c_in, desc.c_out, desc.kh, desc.kw, desc.stride, desc.pad)
+            want, p4, _ = oracle.sq_int(oracle.conv_dgrad_acc(od, e3, wt), -10 - call - 7)
+            assert np.array_equal(got_e4.cpu().numpy().astype(np.int32), want) and got_exp.item() == p4
+            assert got_sum.item() == int(want.astype(np.int64).sum())
     finally:
         eoq.eoq_destroy(handle)
 
