@@ -377,3 +377,162 @@ int eoq_o_update(int32_t *theta, const int8_t *g, int p_g, size_t n, int lr_mant
     __builtin_free(u);
     return z;
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Network glue around the quantized convolution units (conventions of this build where the paper is
+ * silent; every one of them is "parity unpinned" by the paper and pinned here only by exact integer
+ * brute force, invariants and special cases).
+ * ------------------------------------------------------------------------------------------------ */
+
+/*
+ * Max-pooling on int8 codes (the ImageNet networks of Sec. 5.1 pool after the first layer): window
+ * k x k, stride s, padding p; padded positions never win.  idx receives the flat NHWC index of the
+ * first maximum in (kh, kw) scan order, which is where the backward pass routes the error.
+ */
+void eoq_o_maxpool_fwd(const int8_t *x, int n, int h, int w, int c, int k, int s, int p, int8_t *y, int64_t *idx)
+{
+    int ho = out_dim(h, k, s, p), wo = out_dim(w, k, s, p);
+    for (int b = 0; b < n; b++)
+        for (int oy = 0; oy < ho; oy++)
+            for (int ox = 0; ox < wo; ox++)
+                for (int ch = 0; ch < c; ch++) {
+                    int best = -1000;
+                    int64_t arg = -1;
+                    for (int kh = 0; kh < k; kh++)
+                        for (int kw = 0; kw < k; kw++) {
+                            int iy = oy * s + kh - p, ix = ox * s + kw - p;
+                            if (iy < 0 || iy >= h || ix < 0 || ix >= w) continue;
+                            int64_t i = (((int64_t)b * h + iy) * w + ix) * c + ch;
+                            if ((int)x[i] > best) { best = x[i]; arg = i; }
+                        }
+                    int64_t o = (((int64_t)b * ho + oy) * wo + ox) * c + ch;
+                    y[o] = (int8_t)best;
+                    idx[o] = arg;
+                }
+}
+
+/* Backward of max-pooling: every output error code is added at its argmax position (exact sums;
+ * overlapping windows may hit one position several times).  S must hold n_in zeros on entry. */
+void eoq_o_maxpool_bwd(const int8_t *e, const int64_t *idx, size_t n_out, int64_t *S)
+{
+    for (size_t o = 0; o < n_out; o++) S[idx[o]] += e[o];
+}
+
+/* Global average pooling hands the exact integer sum per (sample, channel) to the float head. */
+void eoq_o_avgpool_sum(const int8_t *x, int n, int hw, int c, int64_t *sums)
+{
+    for (int b = 0; b < n; b++)
+        for (int ch = 0; ch < c; ch++) {
+            int64_t acc = 0;
+            for (int i = 0; i < hw; i++) acc += x[((size_t)b * hw + i) * c + ch];
+            sums[(size_t)b * c + ch] = acc;
+        }
+}
+
+/*
+ * Where two error streams meet (block input: branch error a at exponent pa, shortcut error b at pb):
+ * both are brought to the smaller exponent p and added exactly, S = a * 2^(pa - p) + b * 2^(pb - p);
+ * an operand more than 31 octaves below the other is dropped.  The caller applies Q_e = SQ to S.
+ * mask_b (optional, one byte per element) gates operand b (the ReLU derivative at the join).
+ */
+int eoq_o_join(const int8_t *a, int pa, const int8_t *b, int pb, const uint8_t *mask_b, size_t n, int64_t *S)
+{
+    int p = pa < pb ? pa : pb;
+    int sa = pa - p, sb = pb - p;
+    for (size_t i = 0; i < n; i++) {
+        int64_t va = a[i];
+        int64_t vb = (mask_b && !mask_b[i]) ? 0 : b[i];
+        if (sa > 31) S[i] = va;        /* b lies more than 31 octaves below a: dropped, the sum stays at pa */
+        else if (sb > 31) S[i] = vb;   /* a dropped, the sum stays at pb */
+        else S[i] = va * ((int64_t)1 << sa) + vb * ((int64_t)1 << sb);
+    }
+    if (sa > 31) return pa;
+    if (sb > 31) return pb;
+    return p;
+}
+
+/*
+ * exp(x) in fp32 from fused multiply-adds and an exponent adjustment only, so that any IEEE-754
+ * implementation reproduces it bit for bit: x = k ln2 + r with k = nearest integer of x log2(e),
+ * r formed with a two-part ln2, e^r by a degree-7 Taylor polynomial in Horner form (|r| <= 0.35),
+ * then scaled by 2^k.  Inputs below -87 return 0 (the softmax only sees x <= 0).
+ */
+float eoq_o_expf(float x)
+{
+    if (x < -87.0f) return 0.0f;
+    if (x > 88.0f) x = 88.0f;
+    float kf = rintf(x * 1.44269504088896341f);
+    float r = fmaf(-kf, 0.693145751953125f, x);
+    r = fmaf(-kf, 1.42860682030941723212e-6f, r);
+    float p = 1.0f / 5040.0f;
+    p = fmaf(p, r, 1.0f / 720.0f);
+    p = fmaf(p, r, 1.0f / 120.0f);
+    p = fmaf(p, r, 1.0f / 24.0f);
+    p = fmaf(p, r, 1.0f / 6.0f);
+    p = fmaf(p, r, 0.5f);
+    p = fmaf(p, r, 1.0f);
+    p = fmaf(p, r, 1.0f);
+    return ldexpf(p, (int)kf);
+}
+
+/*
+ * The unquantized last layer (Sec. 5.1 keeps it in floating point), written operation by operation
+ * in fp32 so that the result does not depend on the machine:
+ *   pooled[n,c] = (float)sum[n,c] * 2^-7 / hw
+ *   logit[n,j]  = bias[j] + sum over c ascending of fma(W[j,c], pooled[n,c], .)   (one accumulator)
+ *   softmax with the maximum subtracted, exp as above, denominator summed over j ascending
+ *   dlogit[n,j] = (prob - [j == label]) * (1 / n)       (mean cross-entropy over the batch)
+ *   dpooled[n,c] = sum over j ascending of fma(dlogit[n,j], W[j,c], .)          (W before its update)
+ *   W[j,c]  <- fma(-lr, sum over n ascending of fma(dlogit[n,j], pooled[n,c], .), W[j,c]); bias alike
+ * loss = mean over n of (log(denominator) - (logit[label] - max)), reported only.
+ */
+void eoq_o_head(const int64_t *sums, int n, int c, int hw, int classes, float *W, float *bias, const int32_t *labels,
+                float lr, float *loss_out, float *dpooled, float *logits_out)
+{
+    float *pooled = (float *)__builtin_malloc(sizeof(float) * (size_t)n * c);
+    float *dl = (float *)__builtin_malloc(sizeof(float) * (size_t)n * classes);
+    for (size_t i = 0; i < (size_t)n * c; i++) pooled[i] = ((float)sums[i] * 0.0078125f) / (float)hw;
+    float inv_n = 1.0f / (float)n;
+    double loss = 0.0;
+    for (int b = 0; b < n; b++) {
+        float *l = dl + (size_t)b * classes;
+        for (int j = 0; j < classes; j++) {
+            float acc = bias[j];
+            for (int k = 0; k < c; k++) acc = fmaf(W[(size_t)j * c + k], pooled[(size_t)b * c + k], acc);
+            l[j] = acc;
+            if (logits_out) logits_out[(size_t)b * classes + j] = acc;
+        }
+        float m = l[0];
+        for (int j = 1; j < classes; j++) m = l[j] > m ? l[j] : m;
+        float den = 0.0f;
+        float ly = l[labels[b]] - m;
+        for (int j = 0; j < classes; j++) {
+            l[j] = eoq_o_expf(l[j] - m);
+            den = den + l[j];
+        }
+        loss += (double)logf(den) - (double)ly;
+        for (int j = 0; j < classes; j++) {
+            float pr = l[j] / den;
+            l[j] = (pr - (j == labels[b] ? 1.0f : 0.0f)) * inv_n;
+        }
+    }
+    *loss_out = (float)(loss / n);
+    for (int b = 0; b < n; b++)
+        for (int k = 0; k < c; k++) {
+            float acc = 0.0f;
+            for (int j = 0; j < classes; j++) acc = fmaf(dl[(size_t)b * classes + j], W[(size_t)j * c + k], acc);
+            dpooled[(size_t)b * c + k] = acc;
+        }
+    for (int j = 0; j < classes; j++) {
+        for (int k = 0; k < c; k++) {
+            float acc = 0.0f;
+            for (int b = 0; b < n; b++) acc = fmaf(dl[(size_t)b * classes + j], pooled[(size_t)b * c + k], acc);
+            W[(size_t)j * c + k] = fmaf(-lr, acc, W[(size_t)j * c + k]);
+        }
+        float db = 0.0f;
+        for (int b = 0; b < n; b++) db = db + dl[(size_t)b * classes + j];
+        bias[j] = fmaf(-lr, db, bias[j]);
+    }
+    __builtin_free(pooled);
+    __builtin_free(dl);
+}

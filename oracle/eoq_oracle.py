@@ -75,6 +75,9 @@ def _L():
         lib.eoq_o_round_log2_u64.argtypes = [C.c_uint64]
         lib.eoq_o_update_hash.restype = C.c_uint64
         lib.eoq_o_update_hash.argtypes = [C.c_uint64] * 4
+        lib.eoq_o_expf.restype = C.c_float
+        lib.eoq_o_expf.argtypes = [C.c_float]
+        lib.eoq_o_join.restype = C.c_int
         _lib = lib
     return _lib
 
@@ -262,3 +265,66 @@ def q_w(w_f32) -> np.ndarray:
     codes, _, flag = quantize_f32(MODE_CQ, w_f32)
     assert flag == 0
     return codes.astype(np.int8)
+
+
+# --------------------------------------------------------------------------- network glue (conventions of this build)
+
+def maxpool_fwd(x, k: int, s: int, p: int):
+    """Max-pooling on int8 codes -> (codes [n,ho,wo,c], flat NHWC index of the first maximum per output)."""
+    x = _i8(x)
+    n, h, w, c = x.shape
+    ho, wo = (h + 2 * p - k) // s + 1, (w + 2 * p - k) // s + 1
+    y = np.empty((n, ho, wo, c), dtype=np.int8)
+    idx = np.empty((n, ho, wo, c), dtype=np.int64)
+    _L().eoq_o_maxpool_fwd(_p(x), C.c_int(n), C.c_int(h), C.c_int(w), C.c_int(c), C.c_int(k), C.c_int(s), C.c_int(p), _p(y), _p(idx))
+    return y, idx
+
+
+def maxpool_bwd(e, idx, in_shape) -> np.ndarray:
+    """Exact sums of the error codes routed to the argmax positions: int64 [in_shape]."""
+    e = _i8(e)
+    idx = np.ascontiguousarray(idx, dtype=np.int64)
+    S = np.zeros(in_shape, dtype=np.int64)
+    _L().eoq_o_maxpool_bwd(_p(e), _p(idx), C.c_size_t(e.size), _p(S))
+    return S
+
+
+def avgpool_sum(x) -> np.ndarray:
+    """Integer sum over the spatial positions per (sample, channel): int64 [n, c]."""
+    x = _i8(x)
+    n, h, w, c = x.shape
+    sums = np.empty((n, c), dtype=np.int64)
+    _L().eoq_o_avgpool_sum(_p(x), C.c_int(n), C.c_int(h * w), C.c_int(c), _p(sums))
+    return sums
+
+
+def join(a, pa: int, b, pb: int, mask_b=None):
+    """Exact sum of two error tensors at the smaller exponent -> (int64 sums, exponent); mask_b gates b."""
+    a, b = _i8(a), _i8(b)
+    assert a.shape == b.shape
+    S = np.empty(a.shape, dtype=np.int64)
+    m = None if mask_b is None else np.ascontiguousarray(mask_b, dtype=np.uint8)
+    p = _L().eoq_o_join(_p(a), C.c_int(pa), _p(b), C.c_int(pb), _p(m) if m is not None else None, C.c_size_t(a.size), _p(S))
+    return S, int(p)
+
+
+def expf(x: float) -> float:
+    """The head's own exp in fp32 (fused multiply-adds and a power-of-two scaling only)."""
+    return float(_L().eoq_o_expf(C.c_float(x)))
+
+
+def head(sums, hw: int, W, bias, labels, lr: float):
+    """The floating-point last layer: pooling scale, linear layer, softmax cross-entropy (mean), its gradient
+    with respect to the pooled activations, and the SGD step of W and bias (in place).
+    -> (loss, dpooled fp32 [n, c], logits fp32 [n, classes])."""
+    sums = np.ascontiguousarray(sums, dtype=np.int64)
+    n, c = sums.shape
+    classes = W.shape[0]
+    assert W.dtype == np.float32 and bias.dtype == np.float32 and W.flags.c_contiguous and W.shape == (classes, c)
+    labels = np.ascontiguousarray(labels, dtype=np.int32)
+    loss = C.c_float(0)
+    dpooled = np.empty((n, c), dtype=np.float32)
+    logits = np.empty((n, classes), dtype=np.float32)
+    _L().eoq_o_head(_p(sums), C.c_int(n), C.c_int(c), C.c_int(hw), C.c_int(classes), _p(W), _p(bias), _p(labels),
+                    C.c_float(lr), C.byref(loss), _p(dpooled), _p(logits))
+    return float(loss.value), dpooled, logits

@@ -1035,32 +1035,17 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
 
 // ================================================================================= weight gradient
 
-// The b1 tap sums (one pass over e3) next to the weight-gradient GEMM: issued on the handle's branch stream
-// behind a fork event recorded on `s` (everything queued on `s` so far, the clearing memset included, comes
-// first); the caller waits for join_ev on `s` before the kernel that reads the sums.  Without a branch stream
-// (the allocation-free handle) they are issued on `s` itself.
-static cudaError_t launch_tap_sums_beside(Handle *h, const int8_t *e3, long long *tap_sums, size_t tap_bytes,
-                                          const eoq_conv_desc_t &d, int ho, int wo, const BorderClasses &bc,
-                                          cudaStream_t s, bool *joined)
+// The b1 tap sums (one pass over e3), in front of the weight-gradient GEMM on the same stream.  (Issued on a second
+// stream "beside" the GEMM they gain nothing: a GEMM CTA fills its SM, so the blocks of this kernel only start as
+// the GEMM's CTAs leave, and the call pays for a fork and a join on top.)
+static cudaError_t launch_tap_sums(Handle *h, const int8_t *e3, long long *tap_sums, size_t tap_bytes,
+                                   const eoq_conv_desc_t &d, int ho, int wo, const BorderClasses &bc, cudaStream_t s)
 {
     const size_t tap_stride = tap_bytes / kTapReplicas / sizeof(long long);
-    *joined = false;
     count_launches(h, 1);
-    if (!h->branch) {
-        ProfScope prof(h, EOQ_PROF_WGRAD_TAPS, s);
-        cudaError_t e = cudaMemsetAsync(tap_sums, 0, tap_bytes, s);  // the kernel adds into them
-        return e != cudaSuccess ? e : launch_b1_error_sums(e3, tap_sums, tap_stride, d, ho, wo, bc, h->sm_count, s);
-    }
-    cudaError_t e = cudaEventRecord(h->fork_ev, s);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->branch, h->fork_ev, 0);
-    if (e == cudaSuccess) {
-        ProfScope prof(h, EOQ_PROF_WGRAD_TAPS, h->branch);
-        e = cudaMemsetAsync(tap_sums, 0, tap_bytes, h->branch);
-        if (e == cudaSuccess) e = launch_b1_error_sums(e3, tap_sums, tap_stride, d, ho, wo, bc, h->sm_count, h->branch);
-    }
-    if (e == cudaSuccess) e = cudaEventRecord(h->join_ev, h->branch);
-    *joined = e == cudaSuccess;
-    return e;
+    ProfScope prof(h, EOQ_PROF_WGRAD_TAPS, s);
+    cudaError_t e = cudaMemsetAsync(tap_sums, 0, tap_bytes, s);  // the kernel adds into them
+    return e != cudaSuccess ? e : launch_b1_error_sums(e3, tap_sums, tap_stride, d, ho, wo, bc, h->sm_count, s);
 }
 
 // Weight gradient behind eoq_conv_wgrad and eoq_conv_wgrad_dev: b1 is the host code b1_c, or the code at b1_dev.
@@ -1090,7 +1075,6 @@ static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
     long long *acc = reinterpret_cast<long long *>(ws + tap_bytes + 256);
     const size_t acc_bytes = round256(g.w_elems * sizeof(long long));
 
-    bool joined = false;  // the tap sums run on the handle's branch stream and must be waited for
     WgradPatchPlan wp;
     if (plan_wgrad_patch(wp, d, g.ho, g.wo, h->gemm_ctas < kWgradTargetCtas ? h->gemm_ctas : kWgradTargetCtas)) {
         wp.partials = reinterpret_cast<int32_t *>(ws + tap_bytes + 256 + acc_bytes);
@@ -1104,7 +1088,7 @@ static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
             count_launches(h, 1);
             return record(h, launch_wgrad_patch(wp, mx, me, s));
         }
-        e = use_b1 ? launch_tap_sums_beside(h, e3, tap_sums, tap_bytes, d, g.ho, g.wo, bc, s, &joined) : cudaSuccess;
+        e = use_b1 ? launch_tap_sums(h, e3, tap_sums, tap_bytes, d, g.ho, g.wo, bc, s) : cudaSuccess;
         if (e != cudaSuccess) return record(h, e);
         CUtensorMap map_x, map_e;
         if (!make_patch_map(&map_x, x, d.n, d.h, d.w, d.c_in, wp.kc, wp.pw, wp.r_rows + d.kh - 1) ||
@@ -1115,7 +1099,6 @@ static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
             ProfScope prof(h, EOQ_PROF_WGRAD, s);
             e = launch_wgrad_patch(wp, map_x, map_e, s);
         }
-        if (e == cudaSuccess && joined) e = cudaStreamWaitEvent(s, h->join_ev, 0);
         if (e != cudaSuccess) return record(h, e);
         ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
         e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
@@ -1202,7 +1185,7 @@ static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
         ProfScope aux(h, EOQ_PROF_WGRAD_AUX, s);
         e = cudaMemsetAsync(acc, 0, acc_bytes, s);  // the GEMM adds into the int64 sums with atomics
     }
-    if (e == cudaSuccess && use_b1 && !h->gemm_only) e = launch_tap_sums_beside(h, e3, tap_sums, tap_bytes, d, g.ho, g.wo, bc, s, &joined);
+    if (e == cudaSuccess && use_b1 && !h->gemm_only) e = launch_tap_sums(h, e3, tap_sums, tap_bytes, d, g.ho, g.wo, bc, s);
     if (e != cudaSuccess) return record(h, e);
     CUtensorMap map_x, map_e;
     if (!make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage)) return EOQ_ERR_UNSUPPORTED;
@@ -1216,7 +1199,6 @@ static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
         ProfScope prof(h, EOQ_PROF_WGRAD, s);
         e = launch_wgrad(p, map_x, map_e, s);
     }
-    if (e == cudaSuccess && joined) e = cudaStreamWaitEvent(s, h->join_ev, 0);
     if (e != cudaSuccess || h->gemm_only) return record(h, e);
     // the kernel leaves sums as [oc][tap][ic], which is the layout of g
     ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);

@@ -49,9 +49,8 @@ struct Handle {
     bool force_timeout;           // self-test: the next error-head call makes its grid-wide wait run out
     int num_records;
     ProfRecord *records;          // kMaxProfRecords entries, allocated on first eoq_profile_start
-    // Branch stream of the weight-gradient call: the b1 tap sums do not depend on the GEMM, so they are issued
-    // on this stream between a fork and a join event and run beside it (null: everything stays on the caller's
-    // stream).  Under stream capture the fork and join become graph edges.
+    // Fork and join events of the calls that issue independent kernels on the class_branch streams (null branch
+    // streams: everything stays on the caller's stream).  Under stream capture they become graph edges.
     int gemm_ctas;                // most CTAs a GEMM launch of this handle may use (eoq_set_gemm_ctas; default: one per SM)
     cudaStream_t branch;
     cudaEvent_t fork_ev, join_ev;
