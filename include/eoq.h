@@ -258,6 +258,62 @@ EOQ_API int eoq_quantize_image(eoq_handle_t handle, const float *src, int n, int
 EOQ_API int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t *dst, int n, int c, int h, int w,
                        int to_nhwc, void *stream);
 
+/*
+ * Glue between the layer units of a residual network (the paper chains the units in Sec. 3.2.1 -- x0 of a layer is
+ * x5 of the one before, e0 the error its successor hands back -- and keeps the last layer in floating point,
+ * Sec. 5.1; pooling, the shortcut error and the float arithmetic are not specified there and follow the conventions
+ * stated with each call).  All tensors NHWC, channel counts multiples of 16, pointers device unless noted.
+ */
+
+/* Max-pooling of int8 codes, window k x k: y [n,ho,wo,c]; arg (same shape, uint8) = kh * k + kw of the first maximum in
+ * (kh, kw) scan order (padding never wins). */
+EOQ_API int eoq_aux_maxpool_fwd(eoq_handle_t handle, const int8_t *x, int n, int h, int w, int c, int k, int stride, int pad,
+                        int8_t *y, uint8_t *arg, void *stream);
+/* Its backward: every error code e [n,ho,wo,c] (exponent *e_exp) is added at the position its window elected, the
+ * exact sums are requantized with Q_e = SQ: e_in [n,h,w,c], *e_in_exp.  workspace: n*h*w*c int32, 256-byte aligned. */
+EOQ_API int eoq_aux_maxpool_bwd(eoq_handle_t handle, const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int h, int w,
+                        int c, int k, int stride, int pad, int8_t *e_in, int32_t *e_in_exp, void *workspace,
+                        size_t workspace_bytes, void *stream);
+/* Global average pooling hands exact integer sums to the head: sums[n][c] = sum over the hw positions of x. */
+EOQ_API int eoq_aux_avgpool_sum(eoq_handle_t handle, const int8_t *x, int n, int hw, int c, int32_t *sums, void *stream);
+/*
+ * Where the error of a residual branch (a, exponent *a_exp) meets the error arriving through the shortcut (b,
+ * *b_exp; gated by mask_b, bit-packed as eoq_conv_fwd writes it, NULL = no gate): both are brought to the smaller
+ * exponent, added exactly (an operand more than 31 octaves below the other is dropped) and requantized with
+ * Q_e = SQ over the whole tensor.  out, *out_exp; sum_out (optional) = sum of the out codes (for g_b1).
+ * n_el a multiple of 16.
+ */
+EOQ_API int eoq_aux_join(eoq_handle_t handle, const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp,
+                 const uint8_t *mask_b, size_t n_el, int8_t *out, int32_t *out_exp, int64_t *sum_out, void *stream);
+/*
+ * The floating-point last layer, operation by operation in fp32 (every product-sum is one fused multiply-add, sums
+ * run over ascending indices into one accumulator, exp is a fixed polynomial), so that any IEEE-754 machine gives
+ * the same bits: pooled = (float)sums * 2^-7 / hw; logits = W pooled + bias (W [classes][c]); softmax cross-entropy,
+ * mean over the batch; dpooled [n][c] = its gradient with respect to pooled (W before the update); W and bias take
+ * one SGD step with rate lr, in place.  *loss (optional) is reported only (its logarithm is the library's).
+ * labels int32 [n].  workspace: eoq_aux_head_workspace_size bytes, 256-byte aligned.
+ */
+EOQ_API int eoq_aux_head_workspace_size(int n, int c, int classes, size_t *bytes);
+EOQ_API int eoq_aux_head(eoq_handle_t handle, const int32_t *sums, int n, int c, int hw, int classes, float *W, float *bias,
+                 const int32_t *labels, float lr, float *loss, float *dpooled, float *logits, void *workspace,
+                 size_t workspace_bytes, void *stream);
+/* The error the head hands back: SQ over all of dpooled / hw (the gradient of one position of the average), the
+ * code of (sample, channel) written to all hw positions: e [n][hw][c], *e_exp.  workspace: n*c floats. */
+EOQ_API int eoq_aux_head_error(eoq_handle_t handle, const float *dpooled, int n, int c, int hw, int8_t *e, int32_t *e_exp,
+                       void *workspace, size_t workspace_bytes, void *stream);
+/*
+ * Update of `num` scalar parameters (gamma, b1, b2; Sec. 3.2.3 applied to a single value): g = Q_g({total}) with
+ * total the exact sum behind the gradient at exponent *total_exp[i] + exp_bias[i]; u = Q_u(lr g);
+ * theta <- Q(theta - u) saturated to 16 bits, rounding as in eoq_update (the hash counter of scalar i is
+ * tensor_id[i], element 0).  Host arrays of device pointers: theta[i] (int32 code, updated in place), mirror[i]
+ * (optional second copy), total[i] (int64), total_exp[i] (int32), grad_out[i] (optional, receives {code, exponent} of
+ * g).  step: device step counter as in eoq_update_dev (read, not incremented) or NULL for 0.
+ */
+EOQ_API int eoq_aux_scalar_update(eoq_handle_t handle, int num, int32_t *const *theta, int32_t *const *mirror,
+                          const int64_t *const *total, const int32_t *const *total_exp, const int *exp_bias,
+                          const int *tensor_id, int32_t *const *grad_out, int32_t lr_mant, int32_t lr_exp, int round_mode,
+                          uint64_t seed, const uint64_t *step, void *stream);
+
 /* Synchronises `stream`, returns the OR of the EOQ_DEV_* bits raised since the last call, clears them. */
 EOQ_API int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits);
 
@@ -277,8 +333,9 @@ EOQ_API int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits);
 #define EOQ_PROF_OTHER 7         /* eoq_quantize */
 #define EOQ_PROF_UPDATE 8        /* eoq_update */
 #define EOQ_PROF_INPUT_Q 9       /* eoq_quantize_image */
-#define EOQ_PROF_WGRAD_TAPS 10   /* b1 error sums of the weight gradient (on the handle's branch stream) */
-#define EOQ_PROF_KINDS 11
+#define EOQ_PROF_WGRAD_TAPS 10   /* b1 error sums of the weight gradient */
+#define EOQ_PROF_GLUE 11         /* eoq_aux_*: pooling, error join, float head, scalar updates */
+#define EOQ_PROF_KINDS 12
 EOQ_API int eoq_profile_start(eoq_handle_t handle);
 EOQ_API int eoq_profile_stop(eoq_handle_t handle, int launches[EOQ_PROF_KINDS], double milliseconds[EOQ_PROF_KINDS]);
 EOQ_API unsigned long long eoq_launch_count(eoq_handle_t handle);

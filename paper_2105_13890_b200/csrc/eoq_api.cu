@@ -1441,3 +1441,137 @@ extern "C" int eoq_quantize_image(eoq_handle_t handle, const float *src, int n, 
     return record(h, launch_quantize_image(src, n, hh, ww, c_src, c_dst, wmargin, dst, dst_exp, h->dev, h->sm_count,
                                            reinterpret_cast<cudaStream_t>(stream)));
 }
+
+// ================================================================================= network glue
+
+extern "C" int eoq_aux_maxpool_fwd(eoq_handle_t handle, const int8_t *x, int n, int hh, int ww, int c, int k, int stride, int pad,
+                                   int8_t *y, uint8_t *arg, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !x || !y || !arg || n <= 0 || hh <= 0 || ww <= 0 || c <= 0 || k <= 0 || k > 15 || stride <= 0 || pad < 0 || pad >= k)
+        return EOQ_ERR_BAD_ARG;
+    if (c % 16 || !aligned16(x) || !aligned16(y) || !aligned16(arg)) return EOQ_ERR_ALIGNMENT;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 1);
+    ProfScope prof(h, EOQ_PROF_GLUE, s);
+    return record(h, launch_maxpool_fwd(x, n, hh, ww, c, k, stride, pad, y, arg, h->sm_count, s));
+}
+
+extern "C" int eoq_aux_maxpool_bwd(eoq_handle_t handle, const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int hh,
+                                   int ww, int c, int k, int stride, int pad, int8_t *e_in, int32_t *e_in_exp, void *workspace,
+                                   size_t workspace_bytes, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !e || !e_exp || !arg || !e_in || !e_in_exp || n <= 0 || hh <= 0 || ww <= 0 || c <= 0 || k <= 0 || k > 15 ||
+        stride <= 0 || pad < 0 || pad >= k)
+        return EOQ_ERR_BAD_ARG;
+    if (c % 16 || !aligned16(e) || !aligned16(arg) || !aligned16(e_in)) return EOQ_ERR_ALIGNMENT;
+    const size_t n_in = (size_t)n * hh * ww * c;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < n_in * sizeof(int32_t)) return EOQ_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    int32_t *sums = static_cast<int32_t *>(workspace);
+    count_launches(h, 2);
+    ProfScope prof(h, EOQ_PROF_GLUE, s);
+    cudaError_t err = launch_maxpool_bwd(e, arg, n, hh, ww, c, k, stride, pad, sums, h->dev, h->sm_count, s);
+    if (err == cudaSuccess) err = launch_sq_i32(sums, e_exp, 0, n_in, e_in, e_in_exp, nullptr, true, h->dev, h->sm_count, s);
+    return record(h, err);
+}
+
+extern "C" int eoq_aux_avgpool_sum(eoq_handle_t handle, const int8_t *x, int n, int hw, int c, int32_t *sums, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !x || !sums || n <= 0 || hw <= 0 || c <= 0 || hw > (1 << 23)) return EOQ_ERR_BAD_ARG;
+    if (c % 16 || !aligned16(x)) return EOQ_ERR_ALIGNMENT;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 1);
+    ProfScope prof(h, EOQ_PROF_GLUE, s);
+    return record(h, launch_avgpool_sum(x, n, hw, c, sums, s));
+}
+
+extern "C" int eoq_aux_join(eoq_handle_t handle, const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp,
+                            const uint8_t *mask_b, size_t n_el, int8_t *out, int32_t *out_exp, int64_t *sum_out, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !a || !a_exp || !b || !b_exp || !out || !out_exp || n_el == 0 || (n_el % 16)) return EOQ_ERR_BAD_ARG;
+    if (!aligned16(a) || !aligned16(b) || !aligned16(out) || (reinterpret_cast<uintptr_t>(mask_b) & 1)) return EOQ_ERR_ALIGNMENT;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 2);
+    ProfScope prof(h, EOQ_PROF_GLUE, s);
+    return record(h, launch_join(a, a_exp, b, b_exp, mask_b, n_el, out, out_exp, reinterpret_cast<long long *>(sum_out), h->dev,
+                                 h->sm_count, s));
+}
+
+extern "C" int eoq_aux_head_workspace_size(int n, int c, int classes, size_t *bytes)
+{
+    if (!bytes || n <= 0 || c <= 0 || classes <= 0) return EOQ_ERR_BAD_ARG;
+    *bytes = round256((size_t)n * c * sizeof(float)) * 2 + round256((size_t)n * classes * sizeof(float)) + round256((size_t)n * sizeof(double));
+    return EOQ_OK;
+}
+
+extern "C" int eoq_aux_head(eoq_handle_t handle, const int32_t *sums, int n, int c, int hw, int classes, float *W, float *bias,
+                            const int32_t *labels, float lr, float *loss, float *dpooled, float *logits, void *workspace,
+                            size_t workspace_bytes, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !sums || !W || !bias || !labels || !dpooled || !logits || n <= 0 || c <= 0 || hw <= 0 || classes <= 0)
+        return EOQ_ERR_BAD_ARG;
+    size_t need = 0;
+    eoq_aux_head_workspace_size(n, c, classes, &need);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < need) return EOQ_ERR_WORKSPACE;
+    char *ws = static_cast<char *>(workspace);
+    float *pooled = reinterpret_cast<float *>(ws);
+    float *dl = reinterpret_cast<float *>(ws + 2 * round256((size_t)n * c * sizeof(float)));
+    double *loss_n = reinterpret_cast<double *>(ws + 2 * round256((size_t)n * c * sizeof(float)) + round256((size_t)n * classes * sizeof(float)));
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 4);
+    ProfScope prof(h, EOQ_PROF_GLUE, s);
+    return record(h, launch_head(sums, n, c, hw, classes, W, bias, labels, lr, loss, dpooled, logits, pooled, dl, loss_n, s));
+}
+
+extern "C" int eoq_aux_head_error(eoq_handle_t handle, const float *dpooled, int n, int c, int hw, int8_t *e, int32_t *e_exp,
+                                  void *workspace, size_t workspace_bytes, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !dpooled || !e || !e_exp || n <= 0 || c <= 0 || hw <= 0) return EOQ_ERR_BAD_ARG;
+    if (c % 16 || !aligned16(e)) return EOQ_ERR_ALIGNMENT;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < (size_t)n * c * sizeof(float)) return EOQ_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 2);
+    ProfScope prof(h, EOQ_PROF_GLUE, s);
+    return record(h, launch_head_error(dpooled, n, c, hw, static_cast<float *>(workspace), e, e_exp, h->dev, h->sm_count, s));
+}
+
+extern "C" int eoq_aux_scalar_update(eoq_handle_t handle, int num, int32_t *const *theta, int32_t *const *mirror,
+                                     const int64_t *const *total, const int32_t *const *total_exp, const int *exp_bias,
+                                     const int *tensor_id, int32_t *const *grad_out, int32_t lr_mant, int32_t lr_exp,
+                                     int round_mode, uint64_t seed, const uint64_t *step, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || num <= 0 || !theta || !total || !total_exp || !exp_bias || !tensor_id) return EOQ_ERR_BAD_ARG;
+    if (lr_mant < 1 || lr_mant > 255 || lr_exp < -64 || lr_exp > 64) return EOQ_ERR_RANGE;
+    if (round_mode != EOQ_ROUND_RNE && round_mode != EOQ_ROUND_STOCHASTIC) return EOQ_ERR_BAD_ARG;
+    for (int i = 0; i < num; ++i)
+        if (!theta[i] || !total[i] || !total_exp[i]) return EOQ_ERR_BAD_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    ProfScope prof(h, EOQ_PROF_GLUE, s);
+    for (int base = 0; base < num; base += kScalarChunk) {
+        ScalarBatch b;
+        memset(&b, 0, sizeof(b));
+        b.num = num - base < kScalarChunk ? num - base : kScalarChunk;
+        for (int k = 0; k < b.num; ++k) {
+            ScalarItem &it = b.item[k];
+            it.theta = theta[base + k];
+            it.mirror = mirror ? mirror[base + k] : nullptr;
+            it.total = reinterpret_cast<const long long *>(total[base + k]);
+            it.exp = total_exp[base + k];
+            it.exp_bias = exp_bias[base + k];
+            it.tensor_id = tensor_id[base + k];
+            it.grad_out = grad_out ? grad_out[base + k] : nullptr;
+        }
+        cudaError_t e = launch_scalar_update(b, lr_mant, lr_exp, round_mode == EOQ_ROUND_STOCHASTIC, seed,
+                                             reinterpret_cast<const unsigned long long *>(step), 0, s);
+        if (e != cudaSuccess) return record(h, e);
+        count_launches(h, 1);
+    }
+    return EOQ_OK;
+}

@@ -1,0 +1,518 @@
+// Glue between the quantized convolution units of a Fixup residual network (arXiv 2105.13890, Sec. 3.2.1 chains the
+// units: x0 of a layer is x5 of the one before, e0 is the error handed back by its successor): max and average
+// pooling on int8 codes, the exact join of two error streams followed by Q_e, the floating-point last layer
+// (Sec. 5.1 leaves it unquantized) written operation by operation so that it is reproducible bit for bit, the
+// quantized error it hands back, and the update of the scalar parameters (Sec. 3.2.3) on their 16-bit range.
+// All of it is bandwidth- or latency-bound support work; none of it touches the tensor cores.
+#include "eoq_device.cuh"
+#include "eoq_internal.h"
+
+namespace eoq {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d)
+{
+    return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) | ((uint32_t)(d & 0xff) << 24);
+}
+
+inline int blocks_for(size_t items, int sm_count, int per_sm = 8)
+{
+    size_t b = (items + kThreads - 1) / kThreads, cap = (size_t)sm_count * per_sm;
+    if (b > cap) b = cap;
+    return b < 1 ? 1 : (int)b;
+}
+
+// same protocol as in the elementwise kernels: true in thread 0 of the block that arrives last
+__device__ __forceinline__ bool last_block_done(DeviceState *dev)
+{
+    __shared__ unsigned last_s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned t = atomicAdd(&dev->ticket, 1u);
+        last_s = (t == gridDim.x - 1) ? 1u : 0u;
+        if (last_s) {
+            __threadfence();
+            dev->ticket = 0;
+        }
+    }
+    __syncthreads();
+    return last_s != 0 && threadIdx.x == 0;
+}
+
+// ------------------------------------------------------------------ pooling
+
+// One thread per 16 channels of an output pixel.  arg = kh * k + kw of the first maximum in scan order.
+__global__ void maxpool_fwd_kernel(const int8_t *__restrict__ x, int n, int h, int w, int c, int k, int s, int p, int ho, int wo,
+                                   int8_t *__restrict__ y, uint8_t *__restrict__ arg)
+{
+    const int groups = c / 16;
+    const size_t items = (size_t)n * ho * wo * groups;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
+        const int g = (int)(i % groups);
+        size_t pix = i / groups;
+        const int ox = (int)(pix % wo);
+        pix /= wo;
+        const int oy = (int)(pix % ho), b = (int)(pix / ho);
+        int best[16], at[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) { best[q] = -1000; at[q] = 0; }
+        for (int kh = 0; kh < k; ++kh) {
+            const int iy = oy * s + kh - p;
+            if (iy < 0 || iy >= h) continue;
+            for (int kw = 0; kw < k; ++kw) {
+                const int ix = ox * s + kw - p;
+                if (ix < 0 || ix >= w) continue;
+                const int4 v = __ldg(reinterpret_cast<const int4 *>(x + (((size_t)b * h + iy) * w + ix) * c + g * 16));
+                const int8_t *e = reinterpret_cast<const int8_t *>(&v);
+#pragma unroll
+                for (int q = 0; q < 16; ++q)
+                    if ((int)e[q] > best[q]) { best[q] = e[q]; at[q] = kh * k + kw; }
+            }
+        }
+        reinterpret_cast<int4 *>(y)[i] = make_int4((int)pack4(best[0], best[1], best[2], best[3]), (int)pack4(best[4], best[5], best[6], best[7]),
+                                                    (int)pack4(best[8], best[9], best[10], best[11]), (int)pack4(best[12], best[13], best[14], best[15]));
+        reinterpret_cast<int4 *>(arg)[i] = make_int4((int)pack4(at[0], at[1], at[2], at[3]), (int)pack4(at[4], at[5], at[6], at[7]),
+                                                      (int)pack4(at[8], at[9], at[10], at[11]), (int)pack4(at[12], at[13], at[14], at[15]));
+    }
+}
+
+// Backward in gather form: an input position collects the error of every window that elected it (exact int32
+// sums, no atomics), and the block maxima of |sum| go to the handle's cell for the scale quantizer that follows.
+__global__ void maxpool_bwd_kernel(const int8_t *__restrict__ e, const uint8_t *__restrict__ arg, int n, int h, int w, int c, int k,
+                                   int s, int p, int ho, int wo, int32_t *__restrict__ sums, DeviceState *dev)
+{
+    const int groups = c / 16;
+    const size_t items = (size_t)n * h * w * groups;
+    uint32_t mx = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
+        const int g = (int)(i % groups);
+        size_t pix = i / groups;
+        const int ix = (int)(pix % w);
+        pix /= w;
+        const int iy = (int)(pix % h), b = (int)(pix / h);
+        int acc[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) acc[q] = 0;
+        for (int kh = 0; kh < k; ++kh) {
+            const int ty = iy + p - kh;
+            if (ty < 0 || ty % s) continue;
+            const int oy = ty / s;
+            if (oy >= ho) continue;
+            for (int kw = 0; kw < k; ++kw) {
+                const int tx = ix + p - kw;
+                if (tx < 0 || tx % s) continue;
+                const int ox = tx / s;
+                if (ox >= wo) continue;
+                const size_t o = (((size_t)b * ho + oy) * wo + ox) * c + g * 16;
+                const int4 ev = __ldg(reinterpret_cast<const int4 *>(e + o));
+                const int4 av = __ldg(reinterpret_cast<const int4 *>(arg + o));
+                const int8_t *eb = reinterpret_cast<const int8_t *>(&ev);
+                const uint8_t *ab = reinterpret_cast<const uint8_t *>(&av);
+#pragma unroll
+                for (int q = 0; q < 16; ++q)
+                    if (ab[q] == kh * k + kw) acc[q] += eb[q];
+            }
+        }
+        int4 *d = reinterpret_cast<int4 *>(sums + i * 16);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            d[q] = make_int4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+            mx = max(max(mx, (uint32_t)abs(acc[4 * q])), max((uint32_t)abs(acc[4 * q + 1]), max((uint32_t)abs(acc[4 * q + 2]), (uint32_t)abs(acc[4 * q + 3]))));
+        }
+    }
+    mx = (uint32_t)block_max_u64(mx);
+    if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u32, mx);
+}
+
+// sums[b][ch] = sum over the hw positions of x[b][.][ch]; one block per (sample, 16-channel group)
+__global__ void avgpool_sum_kernel(const int8_t *__restrict__ x, int hw, int c, int32_t *__restrict__ sums)
+{
+    __shared__ int part[kThreads][17];
+    const int groups = c / 16, b = blockIdx.x / groups, g = blockIdx.x % groups;
+    int acc[16];
+#pragma unroll
+    for (int q = 0; q < 16; ++q) acc[q] = 0;
+    for (int i = threadIdx.x; i < hw; i += blockDim.x) {
+        const int4 v = __ldg(reinterpret_cast<const int4 *>(x + ((size_t)b * hw + i) * c + g * 16));
+        const int8_t *e = reinterpret_cast<const int8_t *>(&v);
+#pragma unroll
+        for (int q = 0; q < 16; ++q) acc[q] += e[q];
+    }
+#pragma unroll
+    for (int q = 0; q < 16; ++q) part[threadIdx.x][q] = acc[q];
+    __syncthreads();
+    if (threadIdx.x < 16) {
+        int t = 0;
+        for (int i = 0; i < (int)blockDim.x; ++i) t += part[i][threadIdx.x];
+        sums[(size_t)b * c + g * 16 + threadIdx.x] = t;
+    }
+}
+
+// ------------------------------------------------------------------ join of two error streams + Q_e
+
+struct JoinShift {
+    int sa, sb, p;  // left shifts of the two operands (-1: operand dropped) and the exponent of the sums
+};
+__device__ __forceinline__ JoinShift join_shift(int pa, int pb)
+{
+    JoinShift j;
+    const int p = min(pa, pb);
+    j.sa = pa - p;
+    j.sb = pb - p;
+    j.p = p;
+    if (j.sa > 31) { j.sb = -1; j.sa = 0; j.p = pa; }        // b lies more than 31 octaves below a
+    else if (j.sb > 31) { j.sa = -1; j.sb = 0; j.p = pb; }
+    return j;
+}
+__device__ __forceinline__ long long join_one(int a, int b, const JoinShift &j)
+{
+    const long long va = j.sa < 0 ? 0ll : (long long)a * (1ll << j.sa);
+    const long long vb = j.sb < 0 ? 0ll : (long long)b * (1ll << j.sb);
+    return va + vb;
+}
+__device__ __forceinline__ void unpack16(const int4 &v, int (&o)[16])
+{
+    const int8_t *b = reinterpret_cast<const int8_t *>(&v);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) o[k] = b[k];
+}
+
+// pass = 0: max |S| into the handle's 64-bit cell; pass = 1: codes of SQ(S), their sum, exponent; cells back to zero
+template <int kPass>
+__global__ void join_kernel(const int8_t *__restrict__ a, const int32_t *a_exp, const int8_t *__restrict__ b, const int32_t *b_exp,
+                            const uint8_t *__restrict__ mask_b, size_t n16, int8_t *out, int32_t *out_exp, long long *sum_out,
+                            DeviceState *dev)
+{
+    const JoinShift j = join_shift(__ldg(a_exp), __ldg(b_exp));
+    unsigned long long mx = 0;
+    long long sum = 0;
+    int t = 7;
+    if (kPass == 1) {
+        const unsigned long long M = dev->absmax_u64;
+        t = M ? round_log2_u64(M) : 7;
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            *out_exp = M ? j.p + t - 7 : j.p;
+            if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+        }
+    }
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
+        int av[16], bv[16];
+        unpack16(__ldg(reinterpret_cast<const int4 *>(a) + i), av);
+        unpack16(__ldg(reinterpret_cast<const int4 *>(b) + i), bv);
+        const uint32_t m = mask_b ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(mask_b) + i) : 0xffffu;
+        int c[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            const long long s = join_one(av[q], ((m >> q) & 1u) ? bv[q] : 0, j);
+            if (kPass == 0) {
+                const unsigned long long u = (unsigned long long)(s < 0 ? -s : s);
+                mx = u > mx ? u : mx;
+            } else {
+                c[q] = sq_code64(s, t);
+                sum += c[q];
+            }
+        }
+        if (kPass == 1)
+            reinterpret_cast<int4 *>(out)[i] = make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
+                                                          (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+    }
+    if (kPass == 0) {
+        mx = block_max_u64(mx);
+        if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u64, mx);
+    } else {
+        if (sum_out) {
+            sum = block_sum_i64(sum);
+            if (threadIdx.x == 0 && sum) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum0), (unsigned long long)sum);
+        }
+        if (last_block_done(dev)) {
+            if (sum_out) *sum_out = (long long)atomicExch(reinterpret_cast<unsigned long long *>(&dev->sum0), 0ull);
+            dev->absmax_u64 = 0;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ the floating-point last layer
+
+// exp(x) from fused multiply-adds and a power-of-two scaling only (x <= 88): x = k ln2 + r, degree-7 polynomial
+__device__ __forceinline__ float exp_fma(float x)
+{
+    if (x < -87.0f) return 0.0f;
+    if (x > 88.0f) x = 88.0f;
+    const float kf = rintf(__fmul_rn(x, 1.44269504088896341f));
+    float r = __fmaf_rn(-kf, 0.693145751953125f, x);
+    r = __fmaf_rn(-kf, 1.42860682030941723212e-6f, r);
+    float p = 1.0f / 5040.0f;
+    p = __fmaf_rn(p, r, 1.0f / 720.0f);
+    p = __fmaf_rn(p, r, 1.0f / 120.0f);
+    p = __fmaf_rn(p, r, 1.0f / 24.0f);
+    p = __fmaf_rn(p, r, 1.0f / 6.0f);
+    p = __fmaf_rn(p, r, 0.5f);
+    p = __fmaf_rn(p, r, 1.0f);
+    p = __fmaf_rn(p, r, 1.0f);
+    // 2^k with k in [-126, 127] is a normal number and the product is exact short of underflow, which x >= -87 excludes;
+    // p < 2 and k = 127 only for x close to 88, where p * 2^127 stays finite
+    return __fmul_rn(p, __int_as_float(((int)kf + 127) << 23));
+}
+
+// pooled[b][k] = (float)sum * 2^-7 / hw; logits[b][j] = bias[j] + sum_k fma(W[j][k], pooled[b][k], .), k ascending
+__global__ void head_logits_kernel(const int32_t *__restrict__ sums, int n, int c, int hw, int classes, const float *__restrict__ W,
+                                   const float *__restrict__ bias, float *pooled, float *logits)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n * c) pooled[i] = __fdiv_rn(__fmul_rn(__int2float_rn(sums[i]), 0.0078125f), (float)hw);
+    if (i >= n * classes) return;
+    const int b = i / classes, j = i % classes;
+    float acc = bias[j];
+    const int32_t *sb = sums + (size_t)b * c;
+    const float *wj = W + (size_t)j * c;
+    for (int k = 0; k < c; ++k) {
+        const float pk = __fdiv_rn(__fmul_rn(__int2float_rn(sb[k]), 0.0078125f), (float)hw);
+        acc = __fmaf_rn(wj[k], pk, acc);
+    }
+    logits[i] = acc;
+}
+
+// one thread per sample: softmax with the maximum subtracted (denominator summed over j ascending), the gradient
+// of the mean cross-entropy with respect to the logits, the sample's loss
+__global__ void head_softmax_kernel(const float *__restrict__ logits, int n, int classes, const int32_t *__restrict__ labels, float *dl,
+                                    double *loss_n)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= n) return;
+    const float *l = logits + (size_t)b * classes;
+    float *d = dl + (size_t)b * classes;
+    float m = l[0];
+    for (int j = 1; j < classes; ++j) m = l[j] > m ? l[j] : m;
+    const int y = labels[b];
+    const float ly = __fsub_rn(l[y], m);
+    float den = 0.0f;
+    for (int j = 0; j < classes; ++j) {
+        const float ej = exp_fma(__fsub_rn(l[j], m));
+        d[j] = ej;
+        den = __fadd_rn(den, ej);
+    }
+    loss_n[b] = (double)logf(den) - (double)ly;
+    const float inv_n = __fdiv_rn(1.0f, (float)n);
+    for (int j = 0; j < classes; ++j) {
+        const float pr = __fdiv_rn(d[j], den);
+        d[j] = __fmul_rn(__fsub_rn(pr, j == y ? 1.0f : 0.0f), inv_n);
+    }
+}
+
+// dpooled[b][k] = sum_j fma(dl[b][j], W[j][k], .), j ascending (W before its update); thread 0 also forms the mean loss
+__global__ void head_dpooled_kernel(const float *__restrict__ dl, const float *__restrict__ W, int n, int c, int classes, float *dpooled,
+                                    const double *loss_n, float *loss_out)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0 && loss_out) {
+        double s = 0.0;
+        for (int b = 0; b < n; ++b) s += loss_n[b];
+        *loss_out = (float)(s / n);
+    }
+    if (i >= n * c) return;
+    const int b = i / c, k = i % c;
+    float acc = 0.0f;
+    for (int j = 0; j < classes; ++j) acc = __fmaf_rn(dl[(size_t)b * classes + j], W[(size_t)j * c + k], acc);
+    dpooled[i] = acc;
+}
+
+// W[j][k] <- fma(-lr, sum_b fma(dl[b][j], pooled[b][k], .), W[j][k]), b ascending; bias[j] alike (thread k == 0)
+__global__ void head_update_kernel(const float *__restrict__ dl, const float *__restrict__ pooled, int n, int c, int classes, float lr,
+                                   float *W, float *bias)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= classes * c) return;
+    const int j = i / c, k = i % c;
+    float acc = 0.0f;
+    for (int b = 0; b < n; ++b) acc = __fmaf_rn(dl[(size_t)b * classes + j], pooled[(size_t)b * c + k], acc);
+    W[i] = __fmaf_rn(-lr, acc, W[i]);
+    if (k == 0) {
+        float db = 0.0f;
+        for (int b = 0; b < n; ++b) db = __fadd_rn(db, dl[(size_t)b * classes + j]);
+        bias[j] = __fmaf_rn(-lr, db, bias[j]);
+    }
+}
+
+// ------------------------------------------------------------------ error handed back by the head
+
+// ef[i] = dpooled[i] / hw and max |ef| (as float bit patterns) into the handle's cell
+__global__ void head_error_scale_kernel(const float *__restrict__ dpooled, int count, int hw, float *ef, DeviceState *dev)
+{
+    uint32_t mx = 0;
+    bool bad = false;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < count; i += gridDim.x * blockDim.x) {
+        const float v = __fdiv_rn(dpooled[i], (float)hw);
+        ef[i] = v;
+        const uint32_t a = __float_as_uint(v) & 0x7fffffffu;
+        bad |= a >= 0x7f800000u;
+        mx = max(mx, a);
+    }
+    mx = (uint32_t)block_max_u64(mx);
+    bad = __syncthreads_or(bad);
+    if (threadIdx.x == 0) {
+        if (mx) atomicMax(&dev->absmax_u32, mx);
+        if (bad) atomicOr(&dev->status, EOQ_DEV_NONFINITE);
+    }
+}
+
+__device__ __forceinline__ int round_log2_f32bits_aux(uint32_t bits)
+{
+    const int eb = (int)((bits >> 23) & 0xffu);
+    const uint32_t frac = bits & 0x7fffffu;
+    if (eb == 0) return round_log2_u32(frac) - 149;
+    const unsigned long long m = (1ull << 23) | frac;
+    return (eb - 127) + ((m * m >= (1ull << 47)) ? 1 : 0);
+}
+
+// e[b][pos][ch] = SQ code of ef[b][ch] for every position; one thread per 16 channels of a pixel
+__global__ void head_error_spread_kernel(const float *__restrict__ ef, int n, int hw, int c, int8_t *e, int32_t *e_exp, DeviceState *dev)
+{
+    const uint32_t mbits = dev->absmax_u32;
+    const bool usable = mbits != 0 && mbits < 0x7f800000u;
+    const int up = usable ? 7 - round_log2_f32bits_aux(mbits) : 7;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        *e_exp = usable ? -up : -7;
+        if (mbits == 0) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+    }
+    const int groups = c / 16;
+    const size_t items = (size_t)n * hw * groups;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
+        const int g = (int)(i % groups), b = (int)(i / ((size_t)groups * hw));
+        const float *src = ef + (size_t)b * c + g * 16;
+        int q[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const float y = scalbnf(__ldg(src + k), up);
+            q[k] = (fabsf(y) < 1.0e9f) ? clampi(__float2int_rn(y), -127, 127) : (y > 0.f ? 127 : (y < 0.f ? -127 : 0));
+        }
+        reinterpret_cast<int4 *>(e)[i] = make_int4((int)pack4(q[0], q[1], q[2], q[3]), (int)pack4(q[4], q[5], q[6], q[7]),
+                                                    (int)pack4(q[8], q[9], q[10], q[11]), (int)pack4(q[12], q[13], q[14], q[15]));
+    }
+    if (last_block_done(dev)) dev->absmax_u32 = 0;
+}
+
+// ------------------------------------------------------------------ scalar parameters (Sec. 3.2.3 on a single value)
+
+__device__ __forceinline__ unsigned long long mix64_aux(unsigned long long z)
+{
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// One thread per scalar: g = Q_g({total}) (SQ of a single value), u = Q_u(lr g), theta <- Q(theta - u) saturated to 16 bits.
+__global__ void scalar_update_kernel(const __grid_constant__ ScalarBatch b, int32_t lr_mant, int32_t lr_exp, int stochastic,
+                                     unsigned long long seed, const unsigned long long *step_dev, unsigned long long step)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= b.num) return;
+    const ScalarItem &it = b.item[i];
+    if (step_dev) step = *step_dev;
+    const long long total = *it.total;
+    const int p_total = *it.exp + it.exp_bias;
+    int g = 0, pg = p_total;
+    if (total != 0) {
+        const unsigned long long M = (unsigned long long)(total < 0 ? -total : total);
+        const int t = round_log2_u64(M);
+        g = sq_code64(total, t);
+        pg = p_total + t - 7;
+    }
+    if (it.grad_out) { it.grad_out[0] = g; it.grad_out[1] = pg; }
+    int theta = *it.theta;
+    if (g != 0) {
+        const int a = lr_mant * g;  // |a| < 2^15
+        const int tu = round_log2_u32((uint32_t)abs(a));
+        const int u = sq_code32(a, tu);
+        const int d = (pg + lr_exp + tu - 7) + 7;  // exponent of u relative to the grid 2^-7
+        long long next;
+        if (d >= 0) {
+            next = (long long)theta - (long long)u * (1ll << min(d, 40));
+        } else if (-d > 40) {
+            next = theta;
+        } else {
+            const int s = -d;
+            const long long v = (long long)theta * (1ll << s) - u;
+            if (!stochastic) {
+                next = rne_shr64(v, s);
+            } else {
+                unsigned long long key = mix64_aux(seed + 0x9E3779B97F4A7C15ull * (step + 1));
+                key = mix64_aux(key + 0x9E3779B97F4A7C15ull * ((unsigned long long)it.tensor_id + 1));
+                const unsigned long long r = mix64_aux(key + 0x9E3779B97F4A7C15ull) & ((1ull << s) - 1ull);  // element index 0
+                next = (v + (long long)r) >> s;
+            }
+        }
+        theta = (int)(next < -32768 ? -32768 : (next > 32767 ? 32767 : next));
+    }
+    *it.theta = theta;
+    if (it.mirror) *it.mirror = theta;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ launchers
+
+cudaError_t launch_maxpool_fwd(const int8_t *x, int n, int h, int w, int c, int k, int s, int p, int8_t *y, uint8_t *arg,
+                               int sm_count, cudaStream_t st)
+{
+    const int ho = (h + 2 * p - k) / s + 1, wo = (w + 2 * p - k) / s + 1;
+    maxpool_fwd_kernel<<<blocks_for((size_t)n * ho * wo * (c / 16), sm_count), kThreads, 0, st>>>(x, n, h, w, c, k, s, p, ho, wo, y, arg);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_maxpool_bwd(const int8_t *e, const uint8_t *arg, int n, int h, int w, int c, int k, int s, int p, int32_t *sums,
+                               DeviceState *dev, int sm_count, cudaStream_t st)
+{
+    const int ho = (h + 2 * p - k) / s + 1, wo = (w + 2 * p - k) / s + 1;
+    maxpool_bwd_kernel<<<blocks_for((size_t)n * h * w * (c / 16), sm_count), kThreads, 0, st>>>(e, arg, n, h, w, c, k, s, p, ho, wo, sums, dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_avgpool_sum(const int8_t *x, int n, int hw, int c, int32_t *sums, cudaStream_t st)
+{
+    avgpool_sum_kernel<<<n * (c / 16), kThreads, 0, st>>>(x, hw, c, sums);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_join(const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp, const uint8_t *mask_b,
+                        size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, DeviceState *dev, int sm_count,
+                        cudaStream_t st)
+{
+    const size_t n16 = n_el / 16;
+    const int blocks = blocks_for(n16, sm_count, 4);
+    join_kernel<0><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, dev);
+    join_kernel<1><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_head(const int32_t *sums, int n, int c, int hw, int classes, float *W, float *bias, const int32_t *labels,
+                        float lr, float *loss_out, float *dpooled, float *logits, float *pooled, float *dl, double *loss_n,
+                        cudaStream_t st)
+{
+    const int nl = n * (classes > c ? classes : c);
+    head_logits_kernel<<<(nl + 127) / 128, 128, 0, st>>>(sums, n, c, hw, classes, W, bias, pooled, logits);
+    head_softmax_kernel<<<(n + 31) / 32, 32, 0, st>>>(logits, n, classes, labels, dl, loss_n);
+    head_dpooled_kernel<<<(n * c + 127) / 128, 128, 0, st>>>(dl, W, n, c, classes, dpooled, loss_n, loss_out);
+    head_update_kernel<<<(classes * c + 127) / 128, 128, 0, st>>>(dl, pooled, n, c, classes, lr, W, bias);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_head_error(const float *dpooled, int n, int c, int hw, float *ef, int8_t *e, int32_t *e_exp, DeviceState *dev,
+                              int sm_count, cudaStream_t st)
+{
+    head_error_scale_kernel<<<blocks_for((size_t)n * c, sm_count, 1), kThreads, 0, st>>>(dpooled, n * c, hw, ef, dev);
+    head_error_spread_kernel<<<blocks_for((size_t)n * hw * (c / 16), sm_count), kThreads, 0, st>>>(ef, n, hw, c, e, e_exp, dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scalar_update(const ScalarBatch &b, int32_t lr_mant, int32_t lr_exp, int stochastic, uint64_t seed,
+                                 const unsigned long long *step_dev, uint64_t step, cudaStream_t st)
+{
+    scalar_update_kernel<<<(b.num + 63) / 64, 64, 0, st>>>(b, lr_mant, lr_exp, stochastic, seed, step_dev, step);
+    return cudaGetLastError();
+}
+
+}  // namespace eoq

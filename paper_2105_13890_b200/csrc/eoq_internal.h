@@ -281,4 +281,39 @@ struct PrepBatch {
 };
 cudaError_t launch_weight_prep(const PrepBatch &b, cudaStream_t s);
 
+
+// ---------------------------------------------------------------------------------------------
+// Network glue (eoq_aux.cu)
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_maxpool_fwd(const int8_t *x, int n, int h, int w, int c, int k, int s, int p, int8_t *y, uint8_t *arg,
+                               int sm_count, cudaStream_t st);
+// exact int32 sums of the routed errors + max |sum| into dev->absmax_u32 (the scale quantizer that follows reads it)
+cudaError_t launch_maxpool_bwd(const int8_t *e, const uint8_t *arg, int n, int h, int w, int c, int k, int s, int p, int32_t *sums,
+                               DeviceState *dev, int sm_count, cudaStream_t st);
+cudaError_t launch_avgpool_sum(const int8_t *x, int n, int hw, int c, int32_t *sums, cudaStream_t st);
+cudaError_t launch_join(const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp, const uint8_t *mask_b,
+                        size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, DeviceState *dev, int sm_count,
+                        cudaStream_t st);
+cudaError_t launch_head(const int32_t *sums, int n, int c, int hw, int classes, float *W, float *bias, const int32_t *labels,
+                        float lr, float *loss_out, float *dpooled, float *logits, float *pooled, float *dl, double *loss_n,
+                        cudaStream_t st);
+cudaError_t launch_head_error(const float *dpooled, int n, int c, int hw, float *ef, int8_t *e, int32_t *e_exp, DeviceState *dev,
+                              int sm_count, cudaStream_t st);
+struct ScalarItem {
+    int32_t *theta;          // the code to update (device)
+    int32_t *mirror;         // a second place that receives the new code, or null
+    const long long *total;  // exact sum behind the gradient (device)
+    const int32_t *exp;      // its exponent (device) ...
+    int exp_bias;            // ... plus this constant
+    int tensor_id;           // counter of the rounding hash
+    int32_t *grad_out;       // receives {code, exponent} of Q_g(total), or null
+};
+constexpr int kScalarChunk = 64;
+struct ScalarBatch {
+    ScalarItem item[kScalarChunk];
+    int num;
+};
+cudaError_t launch_scalar_update(const ScalarBatch &b, int32_t lr_mant, int32_t lr_exp, int stochastic, uint64_t seed,
+                                 const unsigned long long *step_dev, uint64_t step, cudaStream_t st);
+
 }  // namespace eoq

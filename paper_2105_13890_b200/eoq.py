@@ -26,13 +26,14 @@ EXPORTS = [
     "eoq_quantize", "eoq_quantize_image", "eoq_err_prescale", "eoq_update", "eoq_layout_convert", "eoq_last_status",
     "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count", "eoq_set_gemm_ctas",
     "eoq_conv_dgrad_static", "eoq_conv_fwd_dev", "eoq_weight_prep_size", "eoq_weight_prep", "eoq_conv_wgrad_dev",
-    "eoq_err_prescale_dev", "eoq_update_dev", "eoq_describe_plan", "eoq_debug_force_wait_timeout", "eoq_probe_mma_i8", "eoq_profile_gemm_only",
+    "eoq_err_prescale_dev", "eoq_update_dev", "eoq_describe_plan", "eoq_debug_force_wait_timeout", "eoq_probe_mma_i8", "eoq_profile_gemm_only", "eoq_aux_maxpool_fwd", "eoq_aux_maxpool_bwd",
+    "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_error", "eoq_aux_scalar_update",
 ]
 EOQ_STATIC_SCRATCH_BYTES = 16 << 20
 EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
-EOQ_PROF_KINDS = 11
+EOQ_PROF_KINDS = 12
 EOQ_PROF_NAMES = ["igemm_fwd", "igemm_dgrad", "wgrad_gemm", "err_head", "dgrad_aux", "wgrad_aux", "fwd_aux", "other", "update",
-                  "input_quantizer", "wgrad_taps"]
+                  "input_quantizer", "wgrad_taps", "glue"]
 
 
 class EoqError(RuntimeError):
@@ -98,6 +99,16 @@ def lib() -> C.CDLL:
                                      C.c_int, u64, vp, vp]
         L.eoq_describe_plan.argtypes = [vp, dp, C.c_int, C.c_char_p, sz]
         L.eoq_debug_force_wait_timeout.argtypes = [vp]
+        ci = C.c_int
+        L.eoq_aux_maxpool_fwd.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp]
+        L.eoq_aux_maxpool_bwd.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp, sz, vp]
+        L.eoq_aux_avgpool_sum.argtypes = [vp, vp, ci, ci, ci, vp, vp]
+        L.eoq_aux_join.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp, vp, vp, vp]
+        L.eoq_aux_head_workspace_size.argtypes = [ci, ci, ci, C.POINTER(sz)]
+        L.eoq_aux_head.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp, C.c_float, vp, vp, vp, vp, sz, vp]
+        L.eoq_aux_head_error.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, sz, vp]
+        L.eoq_aux_scalar_update.argtypes = [vp, ci, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(ci),
+                                            C.POINTER(ci), C.POINTER(vp), i32, i32, ci, u64, vp, vp]
         L.eoq_profile_gemm_only.argtypes = [vp, C.c_int]
         L.eoq_probe_mma_i8.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
         L.eoq_status_string.argtypes = [C.c_int]
@@ -354,3 +365,52 @@ def eoq_probe_mma_i8(handle, n_cols: int, iters: int, launches: int, stream=None
 def eoq_profile_gemm_only(handle, on: bool) -> None:
     """Timing aid: dgrad / wgrad calls launch their GEMM kernel only (their outputs are then not produced)."""
     _check(lib().eoq_profile_gemm_only(handle, 1 if on else 0), "eoq_profile_gemm_only")
+
+
+# ------------------------------------------------------------------------------- network glue
+
+def eoq_aux_maxpool_fwd(handle, x, n, h, w, c, k, stride, pad, y, arg, stream=None) -> None:
+    _check(lib().eoq_aux_maxpool_fwd(handle, _ptr(x), n, h, w, c, k, stride, pad, _ptr(y), _ptr(arg), _stream(stream)),
+           "eoq_aux_maxpool_fwd")
+
+
+def eoq_aux_maxpool_bwd(handle, e, e_exp, arg, n, h, w, c, k, stride, pad, e_in, e_in_exp, workspace, stream=None) -> None:
+    _check(lib().eoq_aux_maxpool_bwd(handle, _ptr(e), _ptr(e_exp), _ptr(arg), n, h, w, c, k, stride, pad, _ptr(e_in),
+                                     _ptr(e_in_exp), _ptr(workspace), _nbytes(workspace), _stream(stream)), "eoq_aux_maxpool_bwd")
+
+
+def eoq_aux_avgpool_sum(handle, x, n, hw, c, sums, stream=None) -> None:
+    _check(lib().eoq_aux_avgpool_sum(handle, _ptr(x), n, hw, c, _ptr(sums), _stream(stream)), "eoq_aux_avgpool_sum")
+
+
+def eoq_aux_join(handle, a, a_exp, b, b_exp, mask_b, n_el, out, out_exp, sum_out=None, stream=None) -> None:
+    _check(lib().eoq_aux_join(handle, _ptr(a), _ptr(a_exp), _ptr(b), _ptr(b_exp), _ptr(mask_b), int(n_el), _ptr(out),
+                              _ptr(out_exp), _ptr(sum_out), _stream(stream)), "eoq_aux_join")
+
+
+def eoq_aux_head_workspace_size(n, c, classes) -> int:
+    out = C.c_size_t(0)
+    _check(lib().eoq_aux_head_workspace_size(n, c, classes, C.byref(out)), "eoq_aux_head_workspace_size")
+    return out.value
+
+
+def eoq_aux_head(handle, sums, n, c, hw, classes, W, bias, labels, lr, loss, dpooled, logits, workspace, stream=None) -> None:
+    _check(lib().eoq_aux_head(handle, _ptr(sums), n, c, hw, classes, _ptr(W), _ptr(bias), _ptr(labels), float(lr), _ptr(loss),
+                              _ptr(dpooled), _ptr(logits), _ptr(workspace), _nbytes(workspace), _stream(stream)), "eoq_aux_head")
+
+
+def eoq_aux_head_error(handle, dpooled, n, c, hw, e, e_exp, workspace, stream=None) -> None:
+    _check(lib().eoq_aux_head_error(handle, _ptr(dpooled), n, c, hw, _ptr(e), _ptr(e_exp), _ptr(workspace), _nbytes(workspace),
+                                    _stream(stream)), "eoq_aux_head_error")
+
+
+def eoq_aux_scalar_update(handle, theta: Sequence, mirror: Sequence, total: Sequence, total_exp: Sequence, exp_bias: Sequence[int],
+                          tensor_id: Sequence[int], grad_out: Sequence, lr_mant: int, lr_exp: int, round_mode: int, seed: int,
+                          step=None, stream=None) -> None:
+    num = len(theta)
+    arr = C.c_void_p * num
+    iarr = C.c_int * num
+    _check(lib().eoq_aux_scalar_update(handle, num, arr(*[_ptr(t) for t in theta]), arr(*[_ptr(t) for t in mirror]),
+                                       arr(*[_ptr(t) for t in total]), arr(*[_ptr(t) for t in total_exp]), iarr(*exp_bias),
+                                       iarr(*tensor_id), arr(*[_ptr(t) for t in grad_out]), int(lr_mant), int(lr_exp),
+                                       int(round_mode), int(seed), _ptr(step), _stream(stream)), "eoq_aux_scalar_update")
