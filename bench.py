@@ -1,9 +1,12 @@
 #!/usr/bin/env python
 """Benchmark of the EOQ int8 convolution training path (arXiv 2105.13890) on B200.
 
-One step = one pass of the whole hot path over one synthetic batch: input quantizer, then for every quantized
-convolution of Fixup ResNet-18 (batch 64, 224x224) forward + error head + dgrad + wgrad, then the 8-bit
-update of all weights.  Prints ONE JSON line (rank 0).
+One step = one closed-loop int8 training step of Fixup ResNet-18 (batch 64, 224x224) on synthetic images and
+labels: input quantizer, every quantized convolution unit forward (chained, with max-pooling and shortcuts), global
+average pooling and the floating-point last layer, then back: per unit error head + dgrad + wgrad with the error joins
+at the block inputs, and the 8-bit update of all weights plus the update of the scalars.  --independent times the
+same convolution units fed independent synthetic tensors instead (no glue between them; also the only mode for
+the bottleneck and single-layer workloads).  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet18|resnet20|resnet50|single] [--batch B]
   python bench.py --impl reference ...     # the CPU oracle on host cores, same metric, bounded sample per step
@@ -150,6 +153,34 @@ def oracle_step(wl, seed, scal):
     return time.perf_counter() - t0
 
 
+CHAINED = {"resnet18": ("resnet18", 1000, (3, 2, 1)), "resnet34": ("resnet34", 1000, (3, 2, 1)),
+           "resnet20": ("resnet20", 10, None), "resnet110": ("resnet110", 10, None)}
+
+
+def oracle_chain_step(name, batch, seed):
+    """One closed-loop training step of the same network on the CPU oracle, as it stands.  Returns seconds."""
+    import oracle
+    from oracle import network as N
+    from paper_2105_13890_b200 import synth
+
+    oname, classes, _ = CHAINED[name]
+    net = getattr(N, oname)(batch)
+    N.init(net, lambda s, st: synth.normal_f64(s, seed, st), lambda s, st: synth.normal_f32(s, seed, st), b1=-2, gamma=118, b2=3)
+    f = net.units[0].d
+    img = synth.normal_f32((f.n, f.h, f.w, 3), seed, 0)
+    labels = synth.labels(f.n, classes, seed, 1)
+    t0 = time.perf_counter()
+    N.train_step(net, img, labels, 1, -8, 2.0 ** -6, keep=False)
+    return time.perf_counter() - t0
+
+
+def cpu_step_seconds(args, wl):
+    """The oracle's step for the mode the GPU arm times."""
+    if args.workload in CHAINED and not args.independent:
+        return oracle_chain_step(args.workload, wl.batch, 1)
+    return oracle_step(wl, 1, (-2, 118, 3))
+
+
 def run_reference(args):
     """--impl reference: the oracle timed on the host cores, each step a bounded sample (small batch) of the workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -164,8 +195,8 @@ def run_reference(args):
     full = workloads.get(args.workload, args.batch)
     cores = os.cpu_count() or 1
     for _ in range(args.warmup):
-        oracle_step(wl, 1, (-2, 118, 3))
-    secs = [oracle_step(wl, 1, (-2, 118, 3)) for _ in range(args.steps)]
+        cpu_step_seconds(args, wl)
+    secs = [cpu_step_seconds(args, wl) for _ in range(args.steps)]
     t = sum(secs) / len(secs)
     tops = wl.total_ops / t / 1e12
     line = {
@@ -173,7 +204,8 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "img_per_s": wl.batch / t,
-        "config": {"workload": full.name, "sample": f"batch {sample_batch} of {full.batch} per step, all layers"},
+        "config": {"workload": full.name, "sample": f"batch {sample_batch} of {full.batch} per step, all layers",
+                   "step": "independent layer units" if (args.independent or args.workload not in CHAINED) else "closed loop"},
         "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": cores, "kind": "oracle",
                          "sample": f"{wl.name}: every layer of the workload at batch {sample_batch}"},
         "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -202,6 +234,7 @@ def run_gpu(args):
     import torch
 
     from paper_2105_13890_b200 import eoq, ranks, workloads
+    from paper_2105_13890_b200.chain import ChainedStep
     from paper_2105_13890_b200.step import Scalars, TrainStep
 
     world, rank, local = ranks.world()
@@ -214,7 +247,15 @@ def run_gpu(args):
     wl = workloads.get(args.workload, args.batch)
     handle = eoq.eoq_create(local)
     round_mode = eoq.EOQ_ROUND_STOCHASTIC if args.stochastic else eoq.EOQ_ROUND_RNE
-    step = TrainStep(wl, handle, f"cuda:{local}", scalars=Scalars(), round_mode=round_mode)
+    chained = args.workload in CHAINED and not args.independent
+    if chained:
+        _, classes, pool = CHAINED[args.workload]
+        step = ChainedStep(wl, handle, f"cuda:{local}", scalars=Scalars(), lr_mant=1, lr_exp=-8, classes=classes, pool=pool,
+                           round_mode=round_mode)
+        step.image.copy_(torch.from_numpy(step.host_image(777)))
+        step.labels.copy_(torch.from_numpy(__import__("numpy").arange(wl.batch, dtype="int32") % classes))
+    else:
+        step = TrainStep(wl, handle, f"cuda:{local}", scalars=Scalars(), round_mode=round_mode)
     stream = torch.cuda.current_stream()
 
     # One step = one replay of a CUDA graph of the whole path (the weight-gradient chain of each layer on a side
@@ -344,7 +385,9 @@ def run_gpu(args):
             "pct_of_int8_peak": 100.0 * tops / world / int8_peak,
             "config": {"workload": wl.name, "layers": len(wl.layers), "global_batch": world * wl.batch,
                        "gop_per_step": ops_step / 1e9, "l2": "working set larger than L2; no flush between steps",
-                       "scalars": "b1=-2 gamma=118 b2=3 codes, device-resident",
+                       "step": "closed loop: units chained, pooling, float head, error joins, scalar updates" if chained
+                               else "independent layer units on synthetic tensors",
+                       "scalars": "b1=-2 gamma=118 b2=3 codes at the start, device-resident",
                        "update": "stochastic rounding (extension)" if args.stochastic else "round to nearest even (Sec. 3.2.2)",
                        "parallelism": f"replicas x{world}",
                        "launch": "eager, one stream" if args.eager else "CUDA graph replay, wgrad chains on two side streams"},
@@ -386,7 +429,7 @@ def run_gpu(args):
 
             oracle.build()
             small = workloads.get(args.workload, args.ref_batch if args.ref_batch else wl.batch)
-            secs = oracle_step(small, 1, (-2, 118, 3))
+            secs = cpu_step_seconds(args, small)
             line["cpu_baseline"] = {"value": small.total_ops / secs / 1e12, "unit": "TOPS", "cores": os.cpu_count(),
                                     "kind": "oracle", "seconds": secs,
                                     "sample": f"{small.name}: every layer of the workload at batch {small.batch}, one step"}
@@ -493,6 +536,7 @@ def main():
     ap.add_argument("--ref-arm-batch", type=int, default=1, help="batch of each step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eager", action="store_true", help="launch call by call on one stream instead of replaying a CUDA graph")
+    ap.add_argument("--independent", action="store_true", help="time the layer units on independent synthetic tensors (no glue)")
     ap.add_argument("--stochastic", action="store_true", help="stochastic rounding in the update (an extension; default: nearest even)")
     ap.add_argument("--probe", default=None, choices=["mma_i8"], help="measure the INT8 tensor-pipe figures and exit")
     ap.add_argument("--probe-seconds", type=float, default=2.0, help="length of each sustained probe loop")

@@ -270,10 +270,9 @@ EOQ_API int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t *d
 EOQ_API int eoq_aux_maxpool_fwd(eoq_handle_t handle, const int8_t *x, int n, int h, int w, int c, int k, int stride, int pad,
                         int8_t *y, uint8_t *arg, void *stream);
 /* Its backward: every error code e [n,ho,wo,c] (exponent *e_exp) is added at the position its window elected, the
- * exact sums are requantized with Q_e = SQ: e_in [n,h,w,c], *e_in_exp.  workspace: n*h*w*c int32, 256-byte aligned. */
+ * exact sums are requantized with Q_e = SQ: e_in [n,h,w,c], *e_in_exp. */
 EOQ_API int eoq_aux_maxpool_bwd(eoq_handle_t handle, const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int h, int w,
-                        int c, int k, int stride, int pad, int8_t *e_in, int32_t *e_in_exp, void *workspace,
-                        size_t workspace_bytes, void *stream);
+                        int c, int k, int stride, int pad, int8_t *e_in, int32_t *e_in_exp, void *stream);
 /* Global average pooling hands exact integer sums to the head: sums[n][c] = sum over the hw positions of x. */
 EOQ_API int eoq_aux_avgpool_sum(eoq_handle_t handle, const int8_t *x, int n, int hw, int c, int32_t *sums, void *stream);
 /*

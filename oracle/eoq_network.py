@@ -100,8 +100,16 @@ def resnet18(batch: int, image: int = 224, classes: int = 1000, stem_c: int = 8)
     return resnet_basic(batch, image, (7, 2, 3), stem_c, (3, 2, 1), (64, 128, 256, 512), (2, 2, 2, 2), classes)
 
 
+def resnet34(batch: int, image: int = 224, classes: int = 1000, stem_c: int = 8) -> Net:
+    return resnet_basic(batch, image, (7, 2, 3), stem_c, (3, 2, 1), (64, 128, 256, 512), (3, 4, 6, 3), classes)
+
+
 def resnet20(batch: int, image: int = 32, classes: int = 10, stem_c: int = 16) -> Net:
     return resnet_basic(batch, image, (3, 1, 1), stem_c, None, (16, 32, 64), (3, 3, 3), classes)
+
+
+def resnet110(batch: int, image: int = 32, classes: int = 10, stem_c: int = 16) -> Net:
+    return resnet_basic(batch, image, (3, 1, 1), stem_c, None, (16, 32, 64), (18, 18, 18), classes)
 
 
 def init(net: Net, normal_f64, normal_f32, b1: int = 0, gamma: int = 128, b2: int = 0) -> None:

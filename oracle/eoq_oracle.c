@@ -536,3 +536,71 @@ void eoq_o_head(const int64_t *sums, int n, int c, int hw, int classes, float *W
     __builtin_free(pooled);
     __builtin_free(dl);
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Other bit widths (Sec. 3.2.2 defines Q, CQ and SQ for any k; Sec. 3.2.3 and Sec. 5 compare the 8-bit
+ * update with the 24-bit update of earlier integer-training work).
+ * ------------------------------------------------------------------------------------------------ */
+
+/* SQ(., k) on integer codes at exponent p_a: code = sat(R(a * 2^(k-1-t)), +-(2^(k-1) - 1)), p_out = p_a + t - (k-1). */
+int eoq_o_sq_i64_k(const int64_t *a, size_t n, int p_a, int k, int64_t *codes, int *p_out)
+{
+    uint64_t M = 0;
+    for (size_t i = 0; i < n; i++) {
+        uint64_t m = a[i] < 0 ? (uint64_t)(-a[i]) : (uint64_t)a[i];
+        if (m > M) M = m;
+    }
+    if (M == 0) {
+        for (size_t i = 0; i < n; i++) codes[i] = 0;
+        *p_out = p_a;
+        return 1;
+    }
+    int t = eoq_o_round_log2_u64(M);
+    int64_t lim = ((int64_t)1 << (k - 1)) - 1;
+    for (size_t i = 0; i < n; i++) codes[i] = sat64(eoq_o_rne_shr(a[i], t - (k - 1)), -lim, lim);
+    *p_out = p_a + t - (k - 1);
+    return 0;
+}
+
+/*
+ * The update with an update quantizer of k_u bits and a master copy of the weights on the grid of Q(., k_m):
+ *   u = Q_u(lr g) = SQ(lr g, k_u);   theta <- CQ(theta - u, k_m)   (theta: integer codes at exponent -(k_m - 1));
+ * the layer then works on w = Q_w(theta) = CQ(theta, 8), i.e. code sat(R(theta / 2^(k_m - 8)), +-127).
+ * k_u = k_m = 8 is the paper's 8-bit update (eoq_o_update); k_u = k_m = 24 the wide update it is compared with.
+ * Alignment as in eoq_o_update; shifts beyond 38 bits drop the update (below 2^-38 of a master step).
+ */
+int eoq_o_update_k(int32_t *theta, int8_t *w8, const int8_t *g, int p_g, size_t n, int lr_mant, int lr_exp, int k_u, int k_m,
+                   int stochastic, uint64_t seed, uint64_t step, uint64_t tensor_id, int *p_u_out)
+{
+    int64_t *a = (int64_t *)__builtin_malloc(sizeof(int64_t) * (n ? n : 1));
+    int64_t *u = (int64_t *)__builtin_malloc(sizeof(int64_t) * (n ? n : 1));
+    for (size_t i = 0; i < n; i++) a[i] = (int64_t)lr_mant * g[i];
+    int p_u;
+    int z = eoq_o_sq_i64_k(a, n, p_g + lr_exp, k_u, u, &p_u);
+    int d = p_u + (k_m - 1);
+    int64_t lim = ((int64_t)1 << (k_m - 1)) - 1;
+    for (size_t i = 0; i < n; i++) {
+        int64_t next;
+        if (d >= 0) {
+            next = (int64_t)theta[i] - u[i] * ((int64_t)1 << (d > 38 ? 38 : d));
+        } else if (-d > 38) {
+            next = theta[i];
+        } else {
+            int s = -d;
+            int64_t v = (int64_t)theta[i] * ((int64_t)1 << s) - u[i];
+            if (!stochastic) {
+                next = eoq_o_rne_shr(v, s);
+            } else {
+                uint64_t r = eoq_o_update_hash(seed, step, tensor_id, i) & (((uint64_t)1 << s) - 1);
+                int64_t rem;
+                next = floor_div_pow2(v + (int64_t)r, s, &rem);
+            }
+        }
+        theta[i] = (int32_t)sat64(next, -lim, lim);
+        if (w8) w8[i] = (int8_t)sat64(eoq_o_rne_shr(theta[i], k_m - 8), -127, 127);
+    }
+    *p_u_out = p_u;
+    __builtin_free(a);
+    __builtin_free(u);
+    return z;
+}

@@ -328,3 +328,29 @@ def head(sums, hw: int, W, bias, labels, lr: float):
     _L().eoq_o_head(_p(sums), C.c_int(n), C.c_int(c), C.c_int(hw), C.c_int(classes), _p(W), _p(bias), _p(labels),
                     C.c_float(lr), C.byref(loss), _p(dpooled), _p(logits))
     return float(loss.value), dpooled, logits
+
+
+# --------------------------------------------------------------------------- other bit widths (Sec. 3.2.2 / 3.2.3)
+
+def sq_int_k(a, p_a: int, k: int):
+    """SQ(., k) of integer codes at exponent p_a -> (int64 codes, p_out, zero flag)."""
+    a = np.ascontiguousarray(a, dtype=np.int64)
+    codes = np.empty(a.shape, dtype=np.int64)
+    p_out = C.c_int(0)
+    z = _L().eoq_o_sq_i64_k(_p(a), C.c_size_t(a.size), C.c_int(p_a), C.c_int(k), _p(codes), C.byref(p_out))
+    return codes, p_out.value, int(z)
+
+
+def update_k(theta, g, p_g: int, lr_mant: int, lr_exp: int, k_u: int, k_m: int, stochastic: bool = False, seed: int = 0,
+             step: int = 0, tensor_id: int = 0):
+    """Update with a k_u-bit update quantizer on a k_m-bit master copy (codes at exponent -(k_m - 1)).
+    -> (new master codes int32, 8-bit weight codes Q_w(master), exponent of u, zero flag)."""
+    th = np.array(theta, dtype=np.int32).reshape(-1).copy()
+    g = _i8(g).reshape(-1)
+    assert th.size == g.size
+    w8 = np.empty(th.size, dtype=np.int8)
+    p_u = C.c_int(0)
+    z = _L().eoq_o_update_k(_p(th), _p(w8), _p(g), C.c_int(p_g), C.c_size_t(th.size), C.c_int(lr_mant), C.c_int(lr_exp),
+                            C.c_int(k_u), C.c_int(k_m), C.c_int(1 if stochastic else 0), C.c_uint64(seed), C.c_uint64(step),
+                            C.c_uint64(tensor_id), C.byref(p_u))
+    return th.reshape(np.shape(theta)), w8.reshape(np.shape(theta)), p_u.value, int(z)

@@ -111,6 +111,7 @@ class ChainedStep:
                 blk.proj.x0 = x
             blk.b.x0 = blk.a.x5
             blk.shortcut = blk.proj.x5 if blk.proj else x
+            blk.b.shortcut = blk.shortcut
             x = blk.b.x5
         last = self.blocks[-1].b.layer
         self.hw, self.c_last = last.ho * last.wo, last.c_out
@@ -133,8 +134,6 @@ class ChainedStep:
         for u in self.units:
             for p_ in (eoq.EOQ_PASS_DGRAD, eoq.EOQ_PASS_WGRAD):
                 ws = max(ws, eoq.eoq_workspace_size(u.desc, p_))
-        if pool:
-            ws = max(ws, fl.n * fl.ho * fl.wo * fl.c_out * 4)
         ws = max(ws, n * self.c_last * 4)
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
         dev_index = dev.index if dev.index is not None else 0
@@ -250,7 +249,7 @@ class ChainedStep:
         if self.pool:
             k, s, p = self.pool
             eoq.eoq_aux_maxpool_bwd(h, e_out, e_exp, self.pool_arg, fl.n, fl.ho, fl.wo, fl.c_out, k, s, p, self.stem_e0,
-                                    self.stem_e0_exp, ws)
+                                    self.stem_e0_exp)
             e_out, e_exp = self.stem_e0, self.stem_e0_exp
         eoq.eoq_err_prescale_dev(h, e_out, e_exp, stem.mask, None, stem.n_out, stem.scal[1:2], stem.e3, stem.e3_exp, stem.sum_e1, None)
         wgrad(stem, None)
@@ -282,6 +281,62 @@ class ChainedStep:
 
     def replay(self) -> None:
         self.graph.replay()
+
+    def host_image(self, seed: int) -> np.ndarray:
+        f = self.units[0].layer
+        return synth.normal_f32((f.n, f.h, f.w, self.image_channels), seed, 0)
+
+    def result_tensors(self):
+        """Small per-step results a caller would read back: the loss and the logits."""
+        return [self.loss, self.logits]
+
+    def time_conv_passes(self, replays: int = 5) -> dict:
+        """Milliseconds per step of each convolution pass run alone, as TrainStep.time_conv_passes measures them."""
+        h, ws = self.h, self.workspace
+        s = torch.cuda.Stream(device=self.dev)
+
+        def fwd():
+            for u in self.units:
+                eoq.eoq_conv_fwd_dev(h, u.desc, u.x0, self.image_exp if u.index == 0 else None, u.scal, u.w, u.prep,
+                                     getattr(u, "shortcut", None), u.layer.relu, u.x5, u.x2, u.mask)
+
+        def dgrad():
+            for u in self.units:
+                if u.e4 is not None:
+                    eoq.eoq_conv_dgrad(h, u.desc, u.e3, u.e3_exp, u.w, u.e4, u.e4_exp, u.sum_e4, None, ws)
+
+        def wgrad():
+            for u in self.units:
+                eoq.eoq_conv_wgrad_dev(h, u.desc, u.e3, u.e3_exp, u.x0, None if u.index == 0 else u.scal[0:1], u.g, u.g_exp, ws)
+
+        def timed(fn) -> float:
+            s.wait_stream(torch.cuda.current_stream(self.dev))
+            with torch.cuda.stream(s):
+                fn()
+            torch.cuda.synchronize(self.dev)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                fn()
+            torch.cuda.synchronize(self.dev)
+            with torch.cuda.stream(s):
+                for _ in range(2):
+                    g.replay()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(s)
+                for _ in range(replays):
+                    g.replay()
+                b.record(s)
+            torch.cuda.synchronize(self.dev)
+            return a.elapsed_time(b) / replays
+
+        out = {"fwd": timed(fwd), "dgrad": timed(dgrad), "wgrad": timed(wgrad)}
+        eoq.eoq_profile_gemm_only(h, True)
+        try:
+            out["dgrad_gemm"] = timed(dgrad)
+            out["wgrad_gemm"] = timed(wgrad)
+        finally:
+            eoq.eoq_profile_gemm_only(h, False)
+        return out
 
     def launch_count(self) -> int:
         return sum(eoq.eoq_launch_count(h) for h in [self.h] + self.h_sides)

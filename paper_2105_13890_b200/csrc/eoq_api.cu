@@ -1451,6 +1451,7 @@ extern "C" int eoq_aux_maxpool_fwd(eoq_handle_t handle, const int8_t *x, int n, 
     if (!h || !x || !y || !arg || n <= 0 || hh <= 0 || ww <= 0 || c <= 0 || k <= 0 || k > 15 || stride <= 0 || pad < 0 || pad >= k)
         return EOQ_ERR_BAD_ARG;
     if (c % 16 || !aligned16(x) || !aligned16(y) || !aligned16(arg)) return EOQ_ERR_ALIGNMENT;
+    if ((size_t)n * hh * ww * (c / 16) > 0xffffffffull) return EOQ_ERR_UNSUPPORTED;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     count_launches(h, 1);
     ProfScope prof(h, EOQ_PROF_GLUE, s);
@@ -1458,23 +1459,18 @@ extern "C" int eoq_aux_maxpool_fwd(eoq_handle_t handle, const int8_t *x, int n, 
 }
 
 extern "C" int eoq_aux_maxpool_bwd(eoq_handle_t handle, const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int hh,
-                                   int ww, int c, int k, int stride, int pad, int8_t *e_in, int32_t *e_in_exp, void *workspace,
-                                   size_t workspace_bytes, void *stream)
+                                   int ww, int c, int k, int stride, int pad, int8_t *e_in, int32_t *e_in_exp, void *stream)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
     if (!h || !e || !e_exp || !arg || !e_in || !e_in_exp || n <= 0 || hh <= 0 || ww <= 0 || c <= 0 || k <= 0 || k > 15 ||
         stride <= 0 || pad < 0 || pad >= k)
         return EOQ_ERR_BAD_ARG;
     if (c % 16 || !aligned16(e) || !aligned16(arg) || !aligned16(e_in)) return EOQ_ERR_ALIGNMENT;
-    const size_t n_in = (size_t)n * hh * ww * c;
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < n_in * sizeof(int32_t)) return EOQ_ERR_WORKSPACE;
+    if ((size_t)n * hh * ww * (c / 16) > 0xffffffffull) return EOQ_ERR_UNSUPPORTED;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    int32_t *sums = static_cast<int32_t *>(workspace);
     count_launches(h, 2);
     ProfScope prof(h, EOQ_PROF_GLUE, s);
-    cudaError_t err = launch_maxpool_bwd(e, arg, n, hh, ww, c, k, stride, pad, sums, h->dev, h->sm_count, s);
-    if (err == cudaSuccess) err = launch_sq_i32(sums, e_exp, 0, n_in, e_in, e_in_exp, nullptr, true, h->dev, h->sm_count, s);
-    return record(h, err);
+    return record(h, launch_maxpool_bwd(e, e_exp, arg, n, hh, ww, c, k, stride, pad, e_in, e_in_exp, h->dev, h->sm_count, s));
 }
 
 extern "C" int eoq_aux_avgpool_sum(eoq_handle_t handle, const int8_t *x, int n, int hw, int c, int32_t *sums, void *stream)
@@ -1515,6 +1511,7 @@ extern "C" int eoq_aux_head(eoq_handle_t handle, const int32_t *sums, int n, int
     Handle *h = reinterpret_cast<Handle *>(handle);
     if (!h || !sums || !W || !bias || !labels || !dpooled || !logits || n <= 0 || c <= 0 || hw <= 0 || classes <= 0)
         return EOQ_ERR_BAD_ARG;
+    if (c > 1536) return EOQ_ERR_UNSUPPORTED;  // the pooled activations of 32 samples are kept in shared memory
     size_t need = 0;
     eoq_aux_head_workspace_size(n, c, classes, &need);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < need) return EOQ_ERR_WORKSPACE;
@@ -1523,7 +1520,7 @@ extern "C" int eoq_aux_head(eoq_handle_t handle, const int32_t *sums, int n, int
     float *dl = reinterpret_cast<float *>(ws + 2 * round256((size_t)n * c * sizeof(float)));
     double *loss_n = reinterpret_cast<double *>(ws + 2 * round256((size_t)n * c * sizeof(float)) + round256((size_t)n * classes * sizeof(float)));
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    count_launches(h, 4);
+    count_launches(h, 5);
     ProfScope prof(h, EOQ_PROF_GLUE, s);
     return record(h, launch_head(sums, n, c, hw, classes, W, bias, labels, lr, loss, dpooled, logits, pooled, dl, loss_n, s));
 }

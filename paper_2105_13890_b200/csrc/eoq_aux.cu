@@ -51,12 +51,11 @@ __global__ void maxpool_fwd_kernel(const int8_t *__restrict__ x, int n, int h, i
 {
     const int groups = c / 16;
     const size_t items = (size_t)n * ho * wo * groups;
+    // (the launcher keeps the item count below 2^32: 64-bit divisions would dominate the work of an item)
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
-        const int g = (int)(i % groups);
-        size_t pix = i / groups;
-        const int ox = (int)(pix % wo);
-        pix /= wo;
-        const int oy = (int)(pix % ho), b = (int)(pix / ho);
+        const uint32_t i32 = (uint32_t)i, pix = i32 / (uint32_t)groups, row = pix / (uint32_t)wo;
+        const int g = (int)(i32 - pix * (uint32_t)groups), ox = (int)(pix - row * (uint32_t)wo);
+        const int b = (int)(row / (uint32_t)ho), oy = (int)(row - (uint32_t)b * (uint32_t)ho);
         int best[16], at[16];
 #pragma unroll
         for (int q = 0; q < 16; ++q) { best[q] = -1000; at[q] = 0; }
@@ -80,52 +79,71 @@ __global__ void maxpool_fwd_kernel(const int8_t *__restrict__ x, int n, int h, i
     }
 }
 
-// Backward in gather form: an input position collects the error of every window that elected it (exact int32
-// sums, no atomics), and the block maxima of |sum| go to the handle's cell for the scale quantizer that follows.
-__global__ void maxpool_bwd_kernel(const int8_t *__restrict__ e, const uint8_t *__restrict__ arg, int n, int h, int w, int c, int k,
-                                   int s, int p, int ho, int wo, int32_t *__restrict__ sums, DeviceState *dev)
+// Backward in gather form: an input position collects the error of every window that elected it (exact sums, no
+// atomics; at most k * k windows, so the sums are small).  Q_e needs the maximum over the whole tensor first, so the
+// gather runs twice: pass 0 reduces max |sum| into the handle's cell, pass 1 forms the sums again and codes them.
+// e and arg are a quarter of the output's size and stay in L2; no intermediate tensor is written.
+template <int kPass>
+__global__ void maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *e_exp, const uint8_t *__restrict__ arg, int n, int h,
+                                   int w, int c, int k, int s, int p, int ho, int wo, int8_t *__restrict__ e_in, int32_t *e_in_exp,
+                                   DeviceState *dev)
 {
     const int groups = c / 16;
     const size_t items = (size_t)n * h * w * groups;
     uint32_t mx = 0;
+    int t = 7;
+    if (kPass == 1) {
+        const uint32_t M = dev->absmax_u32;
+        t = M ? round_log2_u32(M) : 7;
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            const int p_in = *e_exp;
+            *e_in_exp = M ? p_in + t - 7 : p_in;
+            if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+        }
+    }
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
-        const int g = (int)(i % groups);
-        size_t pix = i / groups;
-        const int ix = (int)(pix % w);
-        pix /= w;
-        const int iy = (int)(pix % h), b = (int)(pix / h);
+        const uint32_t i32 = (uint32_t)i, pix = i32 / (uint32_t)groups, row = pix / (uint32_t)w;
+        const int g = (int)(i32 - pix * (uint32_t)groups), ix = (int)(pix - row * (uint32_t)w);
+        const int b = (int)(row / (uint32_t)h), iy = (int)(row - (uint32_t)b * (uint32_t)h);
         int acc[16];
 #pragma unroll
         for (int q = 0; q < 16; ++q) acc[q] = 0;
-        for (int kh = 0; kh < k; ++kh) {
-            const int ty = iy + p - kh;
-            if (ty < 0 || ty % s) continue;
-            const int oy = ty / s;
+        // the windows that cover (iy, ix): taps kh congruent to iy + p modulo the stride; the output row falls by
+        // one as kh grows by the stride, so one division per axis serves all of them
+        const int kh0 = (iy + p) % s, kw0 = (ix + p) % s;
+        const int oy0 = (iy + p - kh0) / s, ox0 = (ix + p - kw0) / s;
+        for (int kh = kh0, oy = oy0; kh < k && oy >= 0; kh += s, --oy) {
             if (oy >= ho) continue;
-            for (int kw = 0; kw < k; ++kw) {
-                const int tx = ix + p - kw;
-                if (tx < 0 || tx % s) continue;
-                const int ox = tx / s;
+            for (int kw = kw0, ox = ox0; kw < k && ox >= 0; kw += s, --ox) {
                 if (ox >= wo) continue;
                 const size_t o = (((size_t)b * ho + oy) * wo + ox) * c + g * 16;
                 const int4 ev = __ldg(reinterpret_cast<const int4 *>(e + o));
                 const int4 av = __ldg(reinterpret_cast<const int4 *>(arg + o));
                 const int8_t *eb = reinterpret_cast<const int8_t *>(&ev);
                 const uint8_t *ab = reinterpret_cast<const uint8_t *>(&av);
+                const int tap = kh * k + kw;
 #pragma unroll
                 for (int q = 0; q < 16; ++q)
-                    if (ab[q] == kh * k + kw) acc[q] += eb[q];
+                    if (ab[q] == tap) acc[q] += eb[q];
             }
         }
-        int4 *d = reinterpret_cast<int4 *>(sums + i * 16);
+        if (kPass == 0) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            d[q] = make_int4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
-            mx = max(max(mx, (uint32_t)abs(acc[4 * q])), max((uint32_t)abs(acc[4 * q + 1]), max((uint32_t)abs(acc[4 * q + 2]), (uint32_t)abs(acc[4 * q + 3]))));
+            for (int q = 0; q < 16; ++q) mx = max(mx, (uint32_t)abs(acc[q]));
+        } else {
+            int cd[16];
+#pragma unroll
+            for (int q = 0; q < 16; ++q) cd[q] = sq_code32(acc[q], t);
+            reinterpret_cast<int4 *>(e_in)[i] = make_int4((int)pack4(cd[0], cd[1], cd[2], cd[3]), (int)pack4(cd[4], cd[5], cd[6], cd[7]),
+                                                           (int)pack4(cd[8], cd[9], cd[10], cd[11]), (int)pack4(cd[12], cd[13], cd[14], cd[15]));
         }
     }
-    mx = (uint32_t)block_max_u64(mx);
-    if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u32, mx);
+    if (kPass == 0) {
+        mx = (uint32_t)block_max_u64(mx);
+        if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u32, mx);
+    } else if (last_block_done(dev)) {
+        dev->absmax_u32 = 0;
+    }
 }
 
 // sums[b][ch] = sum over the hw positions of x[b][.][ch]; one block per (sample, 16-channel group)
@@ -199,12 +217,36 @@ __global__ void join_kernel(const int8_t *__restrict__ a, const int32_t *a_exp, 
             if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
         }
     }
+    // exponents a few octaves apart (the usual case) keep every sum inside 32 bits: 127 * 2^23 + 127 < 2^31
+    const bool narrow = j.sa >= 0 && j.sb >= 0 && j.sa <= 23 && j.sb <= 23;
+    const int ma = 1 << (j.sa < 0 ? 0 : min(j.sa, 23)), mb = 1 << (j.sb < 0 ? 0 : min(j.sb, 23));
+    uint32_t mx32 = 0;
+    int sum32 = 0;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
         int av[16], bv[16];
         unpack16(__ldg(reinterpret_cast<const int4 *>(a) + i), av);
         unpack16(__ldg(reinterpret_cast<const int4 *>(b) + i), bv);
         const uint32_t m = mask_b ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(mask_b) + i) : 0xffffu;
         int c[16];
+        if (narrow) {
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+                const int s32 = av[q] * ma + (((m >> q) & 1u) ? bv[q] : 0) * mb;
+                if (kPass == 0) {
+                    mx32 = max(mx32, (uint32_t)abs(s32));
+                } else {
+                    c[q] = sq_code32(s32, t);
+                    sum32 += c[q];
+                }
+            }
+            if (kPass == 1) {
+                sum += sum32;
+                sum32 = 0;
+                reinterpret_cast<int4 *>(out)[i] = make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
+                                                              (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+            }
+            continue;
+        }
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
             const long long s = join_one(av[q], ((m >> q) & 1u) ? bv[q] : 0, j);
@@ -221,7 +263,7 @@ __global__ void join_kernel(const int8_t *__restrict__ a, const int32_t *a_exp, 
                                                           (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
     }
     if (kPass == 0) {
-        mx = block_max_u64(mx);
+        mx = block_max_u64(mx > mx32 ? mx : (unsigned long long)mx32);
         if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u64, mx);
     } else {
         if (sum_out) {
@@ -258,46 +300,79 @@ __device__ __forceinline__ float exp_fma(float x)
     return __fmul_rn(p, __int_as_float(((int)kf + 127) << 23));
 }
 
-// pooled[b][k] = (float)sum * 2^-7 / hw; logits[b][j] = bias[j] + sum_k fma(W[j][k], pooled[b][k], .), k ascending
-__global__ void head_logits_kernel(const int32_t *__restrict__ sums, int n, int c, int hw, int classes, const float *__restrict__ W,
-                                   const float *__restrict__ bias, float *pooled, float *logits)
+// pooled[b][k] = (float)sum * 2^-7 / hw
+__global__ void head_pooled_kernel(const int32_t *__restrict__ sums, int count, int hw, float *pooled)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n * c) pooled[i] = __fdiv_rn(__fmul_rn(__int2float_rn(sums[i]), 0.0078125f), (float)hw);
-    if (i >= n * classes) return;
-    const int b = i / classes, j = i % classes;
-    float acc = bias[j];
-    const int32_t *sb = sums + (size_t)b * c;
-    const float *wj = W + (size_t)j * c;
-    for (int k = 0; k < c; ++k) {
-        const float pk = __fdiv_rn(__fmul_rn(__int2float_rn(sb[k]), 0.0078125f), (float)hw);
-        acc = __fmaf_rn(wj[k], pk, acc);
-    }
-    logits[i] = acc;
+    if (i < count) pooled[i] = __fdiv_rn(__fmul_rn(__int2float_rn(sums[i]), 0.0078125f), (float)hw);
 }
 
-// one thread per sample: softmax with the maximum subtracted (denominator summed over j ascending), the gradient
-// of the mean cross-entropy with respect to the logits, the sample's loss
+// logits[b][j] = bias[j] + sum_k fma(W[j][k], pooled[b][k], .), k ascending into one accumulator per (b, j).
+// A warp owns one class j and 32 samples (one per lane), so all lanes walk k together: 32 consecutive weights are
+// loaded by the warp at once and handed round by shuffle, the pooled activations of the 32 samples sit in shared
+// memory as [k][sample].  Every (b, j) still sees its own strictly sequential chain of fused multiply-adds.
+constexpr int kHeadWarps = 8;
+__global__ void head_logits_kernel(const float *__restrict__ pooled, int n, int c, int classes, const float *__restrict__ W,
+                                   const float *__restrict__ bias, float *logits)
+{
+    extern __shared__ float ps[];  // [c][32]
+    const int b0 = blockIdx.y * 32, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < c * 32; i += blockDim.x) {
+        const int k = i >> 5, sb = i & 31;
+        ps[i] = (b0 + sb < n) ? pooled[(size_t)(b0 + sb) * c + k] : 0.0f;
+    }
+    __syncthreads();
+    const int j = blockIdx.x * kHeadWarps + warp;
+    if (j >= classes) return;
+    float acc = bias[j];
+    const float *wj = W + (size_t)j * c;
+    for (int k0 = 0; k0 < c; k0 += 32) {
+        const float wreg = (k0 + lane < c) ? __ldg(wj + k0 + lane) : 0.0f;
+        const int kn = min(32, c - k0);
+        for (int kk = 0; kk < kn; ++kk) acc = __fmaf_rn(__shfl_sync(0xffffffffu, wreg, kk), ps[(k0 + kk) * 32 + lane], acc);
+    }
+    if (b0 + lane < n) logits[(size_t)(b0 + lane) * classes + j] = acc;
+}
+
+// One block per sample: softmax with the maximum subtracted, the gradient of the mean cross-entropy with respect to
+// the logits, the sample's loss.  The exponentials are formed in parallel; the denominator is then summed by one
+// thread over j ascending into one accumulator, which is the order that makes the result reproducible.
 __global__ void head_softmax_kernel(const float *__restrict__ logits, int n, int classes, const int32_t *__restrict__ labels, float *dl,
                                     double *loss_n)
 {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= n) return;
+    __shared__ float red[32];
+    __shared__ float m_s, den_s;
+    const int b = blockIdx.x;
     const float *l = logits + (size_t)b * classes;
     float *d = dl + (size_t)b * classes;
-    float m = l[0];
-    for (int j = 1; j < classes; ++j) m = l[j] > m ? l[j] : m;
-    const int y = labels[b];
-    const float ly = __fsub_rn(l[y], m);
-    float den = 0.0f;
-    for (int j = 0; j < classes; ++j) {
-        const float ej = exp_fma(__fsub_rn(l[j], m));
-        d[j] = ej;
-        den = __fadd_rn(den, ej);
+    float m = -3.4e38f;
+    for (int j = threadIdx.x; j < classes; j += blockDim.x) m = l[j] > m ? l[j] : m;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float other = __shfl_xor_sync(0xffffffffu, m, o);
+        m = other > m ? other : m;
     }
-    loss_n[b] = (double)logf(den) - (double)ly;
-    const float inv_n = __fdiv_rn(1.0f, (float)n);
-    for (int j = 0; j < classes; ++j) {
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float mm = red[0];
+        for (int i = 1; i < (int)(blockDim.x >> 5); ++i) mm = red[i] > mm ? red[i] : mm;
+        m_s = mm;
+    }
+    __syncthreads();
+    m = m_s;
+    for (int j = threadIdx.x; j < classes; j += blockDim.x) d[j] = exp_fma(__fsub_rn(l[j], m));
+    __syncthreads();
+    const int y = labels[b];
+    if (threadIdx.x == 0) {
+        float den = 0.0f;
+        for (int j = 0; j < classes; ++j) den = __fadd_rn(den, d[j]);
+        den_s = den;
+        loss_n[b] = (double)logf(den) - (double)__fsub_rn(l[y], m);
+    }
+    __syncthreads();
+    const float den = den_s, inv_n = __fdiv_rn(1.0f, (float)n);
+    for (int j = threadIdx.x; j < classes; j += blockDim.x) {
         const float pr = __fdiv_rn(d[j], den);
         d[j] = __fmul_rn(__fsub_rn(pr, j == y ? 1.0f : 0.0f), inv_n);
     }
@@ -463,11 +538,13 @@ cudaError_t launch_maxpool_fwd(const int8_t *x, int n, int h, int w, int c, int 
     return cudaGetLastError();
 }
 
-cudaError_t launch_maxpool_bwd(const int8_t *e, const uint8_t *arg, int n, int h, int w, int c, int k, int s, int p, int32_t *sums,
-                               DeviceState *dev, int sm_count, cudaStream_t st)
+cudaError_t launch_maxpool_bwd(const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int h, int w, int c, int k, int s,
+                               int p, int8_t *e_in, int32_t *e_in_exp, DeviceState *dev, int sm_count, cudaStream_t st)
 {
     const int ho = (h + 2 * p - k) / s + 1, wo = (w + 2 * p - k) / s + 1;
-    maxpool_bwd_kernel<<<blocks_for((size_t)n * h * w * (c / 16), sm_count), kThreads, 0, st>>>(e, arg, n, h, w, c, k, s, p, ho, wo, sums, dev);
+    const int blocks = blocks_for((size_t)n * h * w * (c / 16), sm_count);
+    maxpool_bwd_kernel<0><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, dev);
+    maxpool_bwd_kernel<1><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, dev);
     return cudaGetLastError();
 }
 
@@ -492,9 +569,15 @@ cudaError_t launch_head(const int32_t *sums, int n, int c, int hw, int classes, 
                         float lr, float *loss_out, float *dpooled, float *logits, float *pooled, float *dl, double *loss_n,
                         cudaStream_t st)
 {
-    const int nl = n * (classes > c ? classes : c);
-    head_logits_kernel<<<(nl + 127) / 128, 128, 0, st>>>(sums, n, c, hw, classes, W, bias, pooled, logits);
-    head_softmax_kernel<<<(n + 31) / 32, 32, 0, st>>>(logits, n, classes, labels, dl, loss_n);
+    head_pooled_kernel<<<(n * c + 255) / 256, 256, 0, st>>>(sums, n * c, hw, pooled);
+    {
+        const size_t smem = (size_t)c * 32 * sizeof(float);
+        cudaError_t e = cudaFuncSetAttribute(head_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        dim3 grid((classes + kHeadWarps - 1) / kHeadWarps, (n + 31) / 32);
+        head_logits_kernel<<<grid, 32 * kHeadWarps, smem, st>>>(pooled, n, c, classes, W, bias, logits);
+    }
+    head_softmax_kernel<<<n, 256, 0, st>>>(logits, n, classes, labels, dl, loss_n);
     head_dpooled_kernel<<<(n * c + 127) / 128, 128, 0, st>>>(dl, W, n, c, classes, dpooled, loss_n, loss_out);
     head_update_kernel<<<(classes * c + 127) / 128, 128, 0, st>>>(dl, pooled, n, c, classes, lr, W, bias);
     return cudaGetLastError();

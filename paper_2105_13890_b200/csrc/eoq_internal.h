@@ -287,9 +287,8 @@ cudaError_t launch_weight_prep(const PrepBatch &b, cudaStream_t s);
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_maxpool_fwd(const int8_t *x, int n, int h, int w, int c, int k, int s, int p, int8_t *y, uint8_t *arg,
                                int sm_count, cudaStream_t st);
-// exact int32 sums of the routed errors + max |sum| into dev->absmax_u32 (the scale quantizer that follows reads it)
-cudaError_t launch_maxpool_bwd(const int8_t *e, const uint8_t *arg, int n, int h, int w, int c, int k, int s, int p, int32_t *sums,
-                               DeviceState *dev, int sm_count, cudaStream_t st);
+cudaError_t launch_maxpool_bwd(const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int h, int w, int c, int k, int s,
+                               int p, int8_t *e_in, int32_t *e_in_exp, DeviceState *dev, int sm_count, cudaStream_t st);
 cudaError_t launch_avgpool_sum(const int8_t *x, int n, int hw, int c, int32_t *sums, cudaStream_t st);
 cudaError_t launch_join(const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp, const uint8_t *mask_b,
                         size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, DeviceState *dev, int sm_count,

@@ -101,7 +101,7 @@ def lib() -> C.CDLL:
         L.eoq_debug_force_wait_timeout.argtypes = [vp]
         ci = C.c_int
         L.eoq_aux_maxpool_fwd.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp]
-        L.eoq_aux_maxpool_bwd.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp, sz, vp]
+        L.eoq_aux_maxpool_bwd.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp]
         L.eoq_aux_avgpool_sum.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         L.eoq_aux_join.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp, vp, vp, vp]
         L.eoq_aux_head_workspace_size.argtypes = [ci, ci, ci, C.POINTER(sz)]
@@ -374,9 +374,9 @@ def eoq_aux_maxpool_fwd(handle, x, n, h, w, c, k, stride, pad, y, arg, stream=No
            "eoq_aux_maxpool_fwd")
 
 
-def eoq_aux_maxpool_bwd(handle, e, e_exp, arg, n, h, w, c, k, stride, pad, e_in, e_in_exp, workspace, stream=None) -> None:
+def eoq_aux_maxpool_bwd(handle, e, e_exp, arg, n, h, w, c, k, stride, pad, e_in, e_in_exp, stream=None) -> None:
     _check(lib().eoq_aux_maxpool_bwd(handle, _ptr(e), _ptr(e_exp), _ptr(arg), n, h, w, c, k, stride, pad, _ptr(e_in),
-                                     _ptr(e_in_exp), _ptr(workspace), _nbytes(workspace), _stream(stream)), "eoq_aux_maxpool_bwd")
+                                     _ptr(e_in_exp), _stream(stream)), "eoq_aux_maxpool_bwd")
 
 
 def eoq_aux_avgpool_sum(handle, x, n, hw, c, sums, stream=None) -> None:

@@ -78,3 +78,73 @@ def test_stochastic_rounding_is_unbiased_and_counter_based():
     rne, _, _ = oracle.update(theta, g, -10, 1, 0)
     assert set(np.unique(rne[1:])) == {-12}  # 12.5 ties to even
     assert oracle.update_hash(1, 2, 3, 4) != oracle.update_hash(1, 2, 3, 5)
+
+
+# ------------------------------------------------------------------ other update widths (the 24-bit update the paper compares with)
+
+def brute_update_k(theta, g, p_g, lr_mant, lr_exp, k_u, k_m):
+    lr = Fr(lr_mant) * Fr(2) ** lr_exp
+    vals = [lr * Fr(int(v)) * Fr(2) ** p_g for v in g]
+    m = max(abs(v) for v in vals)
+    if m == 0:
+        return list(theta)
+    t = -300
+    while not (Fr(2) ** (2 * t - 1) <= m * m < Fr(2) ** (2 * t + 1)):
+        t += 1
+    scale, lu, lm = Fr(2) ** t, 2 ** (k_u - 1), 2 ** (k_m - 1)
+    out = []
+    for th, v in zip(theta, vals):
+        u = scale * Fr(max(-(lu - 1), min(lu - 1, round(v / scale * lu))), lu)   # SQ(lr g, k_u)
+        new = Fr(int(th), lm) - u
+        out.append(max(-(lm - 1), min(lm - 1, round(new * lm))))               # CQ(., k_m)
+    return out
+
+
+def test_wide_update_matches_exact_rational_arithmetic():
+    r = synth.rng(33, 0)
+    for k_u, k_m in ((8, 8), (16, 16), (24, 24), (8, 24), (16, 8)):
+        for trial in range(150):
+            n = int(r.integers(1, 8))
+            g = r.integers(-127, 128, size=n).astype(np.int8)
+            lim = 2 ** (k_m - 1) - 1
+            theta = r.integers(-lim, lim + 1, size=n).astype(np.int32)
+            p_g, lr_mant, lr_exp = int(r.integers(-24, 2)), int(r.integers(1, 256)), int(r.integers(-12, 3))
+            new, w8, _, _ = oracle.update_k(theta, g, p_g, lr_mant, lr_exp, k_u, k_m)
+            assert list(new) == brute_update_k(theta, g, p_g, lr_mant, lr_exp, k_u, k_m), (k_u, k_m, trial)
+            assert list(w8) == [max(-127, min(127, round(Fr(int(v), 2 ** (k_m - 8))))) for v in new]
+
+
+def test_eight_bit_case_of_the_wide_update_is_the_paper_update():
+    r = synth.rng(34, 0)
+    g = r.integers(-127, 128, size=300).astype(np.int8)
+    theta = r.integers(-127, 128, size=300).astype(np.int32)
+    for stochastic in (False, True):
+        a, _, pa, _ = oracle.update_k(theta, g, -11, 37, -3, 8, 8, stochastic=stochastic, seed=5, step=2, tensor_id=1)
+        b, pb, _ = oracle.update(theta, g, -11, 37, -3, stochastic=stochastic, seed=5, step=2, tensor_id=1)
+        assert np.array_equal(a, b) and pa == pb
+
+
+def test_generic_width_scale_quantizer_invariants():
+    a = synth.rng(35, 0).integers(-10**9, 10**9, size=500)
+    for k in (4, 8, 16, 24):
+        c, p, _ = oracle.sq_int_k(a, -30, k)
+        lim = 2 ** (k - 1) - 1
+        assert np.abs(c).max() <= lim and np.abs(c).max() >= (lim + 1) / np.sqrt(2) - 1      # largest code in [2^(k-1)/sqrt 2, lim]
+        c2, p2, _ = oracle.sq_int_k(a * 8, -30, k)                                            # power-of-two equivariance
+        assert np.array_equal(c, c2) and p2 == p + 3
+    c8, p8, _ = oracle.sq_int_k(a, -30, 8)
+    ref, pr, _ = oracle.sq_int(a, -30)
+    assert np.array_equal(c8, ref) and p8 == pr
+
+
+def test_wide_master_copy_keeps_updates_the_eight_bit_update_rounds_away():
+    """What the update width changes: steps far below the 8-bit weight grid vanish under nearest rounding with an
+    8-bit master copy, but accumulate in a 24-bit one."""
+    g = np.full(64, 100, dtype=np.int8)
+    g[0] = 127
+    th8, th24 = np.zeros(64, dtype=np.int32), np.zeros(64, dtype=np.int32)
+    for _ in range(40):
+        th8, _, _ = oracle.update(th8, g, -18, 1, 0)                     # u = 100 * 2^-18: a twentieth of a weight step
+        th24, w24, _, _ = oracle.update_k(th24, g, -18, 1, 0, 24, 24)
+    assert not th8.any()
+    assert (th24[1:] == -40 * 100 * 2 ** 5).all() and (w24[1:] == -2).all()   # 40 * 100 * 2^-18 = 1.95 / 128 -> code -2
