@@ -246,6 +246,18 @@ EOQ_API int eoq_update_dev(eoq_handle_t handle, int num, int8_t *const *w, const
                    uint64_t seed, uint64_t *step, void *stream);
 
 /*
+ * The update at other widths (Sec. 3.2.3 sets the paper's 8-bit update against the 24-bit update of earlier integer
+ * training): u = Q_u(lr g) = SQ(lr g, k_u) and a master copy of the weights on the grid of Q(., k_m),
+ *   master <- CQ(master - u, k_m)      (int32 codes at exponent -(k_m - 1), updated in place),
+ *   w      <- Q_w(master) = code sat(R(master / 2^(k_m - 8)), -127, 127)   (what the layer's three passes read).
+ * k_u in [2, 24], k_m in [8, 24]; k_u = k_m = 8 is eoq_update.  Arrays as in eoq_update plus master[i] (device int32,
+ * n[i] codes).  step_dev (optional) as in eoq_update_dev, else the host value `step`.
+ */
+EOQ_API int eoq_update_wide(eoq_handle_t handle, int num, int32_t *const *master, int8_t *const *w, const int8_t *const *g,
+                    const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp, int k_u, int k_m,
+                    int round_mode, uint64_t seed, uint64_t step, uint64_t *step_dev, void *stream);
+
+/*
  * Input quantizer for the network input (Sec. 5.1 quantizes every layer but the last): SQ(., 8) of an fp32
  * NHWC image batch [n][h][w][c_src], written as int8 [n][h][w + 2 wmargin][c_dst] with c_dst >= c_src: the extra
  * channels and the wmargin pixels at both ends of every row are zero (see eoq_conv_desc_t::x_wmargin).

@@ -1396,6 +1396,7 @@ static int update_impl(eoq_handle_t handle, int num, int8_t *const *w, const int
         t[i].g = g[i];
         t[i].g_exp = g_exp[i];
         t[i].n = n[i];
+        t[i].master = nullptr;
     }
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     count_launches(h, 2 * ((num + 63) / 64) + (step_dev ? 1 : 0));
@@ -1417,6 +1418,33 @@ extern "C" int eoq_update_dev(eoq_handle_t handle, int num, int8_t *const *w, co
 {
     if (!step || (reinterpret_cast<uintptr_t>(step) & 7)) return EOQ_ERR_BAD_ARG;
     return update_impl(handle, num, w, g, g_exp, n, lr_mant, lr_exp, round_mode, seed, 0, step, stream);
+}
+
+extern "C" int eoq_update_wide(eoq_handle_t handle, int num, int32_t *const *master, int8_t *const *w, const int8_t *const *g,
+                               const int32_t *const *g_exp, const size_t *n, int32_t lr_mant, int32_t lr_exp, int k_u, int k_m,
+                               int round_mode, uint64_t seed, uint64_t step, uint64_t *step_dev, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || num <= 0 || !master || !w || !g || !g_exp || !n) return EOQ_ERR_BAD_ARG;
+    if (num > 256) return EOQ_ERR_UNSUPPORTED;
+    if (lr_mant < 1 || lr_mant > 255 || lr_exp < -64 || lr_exp > 64) return EOQ_ERR_RANGE;
+    if (k_u < 2 || k_u > 24 || k_m < 8 || k_m > 24) return EOQ_ERR_UNSUPPORTED;
+    if (round_mode != EOQ_ROUND_RNE && round_mode != EOQ_ROUND_STOCHASTIC) return EOQ_ERR_BAD_ARG;
+    if (step_dev && (reinterpret_cast<uintptr_t>(step_dev) & 7)) return EOQ_ERR_BAD_ARG;
+    UpdateTensor t[256];
+    for (int i = 0; i < num; ++i) {
+        if (!master[i] || !w[i] || !g[i] || !g_exp[i] || n[i] == 0) return EOQ_ERR_BAD_ARG;
+        t[i].w = w[i];
+        t[i].g = g[i];
+        t[i].g_exp = g_exp[i];
+        t[i].n = n[i];
+        t[i].master = master[i];
+    }
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 2 * ((num + 63) / 64) + (step_dev ? 1 : 0));
+    ProfScope prof(h, EOQ_PROF_UPDATE, s);
+    return record(h, launch_update_wide(t, num, lr_mant, lr_exp, k_u, k_m, round_mode == EOQ_ROUND_STOCHASTIC, seed, step,
+                                        reinterpret_cast<unsigned long long *>(step_dev), h->dev, s));
 }
 
 extern "C" int eoq_layout_convert(eoq_handle_t handle, const int8_t *src, int8_t *dst, int n, int c, int hh, int ww,

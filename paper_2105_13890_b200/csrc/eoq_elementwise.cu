@@ -803,6 +803,58 @@ __global__ void update_apply_kernel(const __grid_constant__ UpdateBatch b, int32
         T.w[j] = (int8_t)update_one(T.w[j], T.g[j], lr_mant, t, d, stochastic, key, j);
 }
 
+// The update with a k_u-bit update quantizer and k_m-bit master codes (Sec. 3.2.3 compares the 8-bit update with a
+// 24-bit one): u = SQ(lr g, k_u), master <- CQ(master - u, k_m) on the grid 2^-(k_m - 1), w = Q_w(master).
+__global__ void update_wide_apply_kernel(const __grid_constant__ UpdateBatch b, int32_t lr_mant, int32_t lr_exp, int k_u, int k_m,
+                                         int stochastic, unsigned long long seed, unsigned long long step,
+                                         const unsigned long long *step_dev, DeviceState *dev)
+{
+    if (step_dev) step = *step_dev;
+    const int k = find_tensor(b, blockIdx.x);
+    const UpdateTensor &T = b.t[k];
+    const uint32_t M = dev->tensor_absmax[b.tensor_base + k] * (uint32_t)lr_mant;
+    if (M == 0) {
+        if (threadIdx.x == 0 && blockIdx.x == b.first_block[k]) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+        return;
+    }
+    const int t = round_log2_u32(M);
+    const int su = t - (k_u - 1);                                  // u code = R(lr_mant g / 2^su)
+    const int d = (__ldg(T.g_exp) + lr_exp + su) + (k_m - 1);      // exponent of u relative to the master grid
+    const long long lim_u = (1ll << (k_u - 1)) - 1, lim_m = (1ll << (k_m - 1)) - 1;
+    unsigned long long key = 0;
+    if (stochastic) {
+        key = mix64(seed + 0x9E3779B97F4A7C15ull * (step + 1));
+        key = mix64(key + 0x9E3779B97F4A7C15ull * ((unsigned long long)(b.tensor_base + k) + 1));
+    }
+    const size_t begin = (size_t)(blockIdx.x - b.first_block[k]) * kUpdElemsPerBlock;
+    const size_t end = min((size_t)T.n, begin + kUpdElemsPerBlock);
+    for (size_t j = begin + threadIdx.x; j < end; j += blockDim.x) {
+        const long long a = (long long)lr_mant * T.g[j];
+        long long u = su >= 0 ? rne_shr64(a, su) : a * (1ll << (-su));
+        u = u < -lim_u ? -lim_u : (u > lim_u ? lim_u : u);
+        const long long th = T.master[j];
+        long long next;
+        if (d >= 0) {
+            next = th - u * (1ll << min(d, 38));
+        } else if (-d > 38) {
+            next = th;
+        } else {
+            const int s = -d;
+            const long long v = th * (1ll << s) - u;
+            if (!stochastic) {
+                next = rne_shr64(v, s);
+            } else {
+                const unsigned long long r = mix64(key + 0x9E3779B97F4A7C15ull * (j + 1)) & ((1ull << s) - 1ull);
+                next = (v + (long long)r) >> s;
+            }
+        }
+        next = next < -lim_m ? -lim_m : (next > lim_m ? lim_m : next);
+        T.master[j] = (int32_t)next;
+        const long long w8 = rne_shr64(next, k_m - 8);
+        T.w[j] = (int8_t)(w8 < -127 ? -127 : (w8 > 127 ? 127 : w8));
+    }
+}
+
 __global__ void step_bump_kernel(unsigned long long *step_dev) { *step_dev += 1ull; }
 
 // ------------------------------------------------------------------ layout helpers
@@ -1202,6 +1254,31 @@ cudaError_t launch_update(const UpdateTensor *t, int num, int32_t lr_mant, int32
         if (blocks == 0) continue;
         update_apply_kernel<<<blocks, kThreads, 0, s>>>(b, lr_mant, lr_exp, stochastic, seed, step, step_dev, dev);
     }
+    if (step_dev) step_bump_kernel<<<1, 1, 0, s>>>(step_dev);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_update_wide(const UpdateTensor *t, int num, int32_t lr_mant, int32_t lr_exp, int k_u, int k_m, int stochastic,
+                               uint64_t seed, uint64_t step, unsigned long long *step_dev, DeviceState *dev, cudaStream_t s)
+{
+    cudaError_t e = cudaMemsetAsync(dev->tensor_absmax, 0, sizeof(unsigned) * 256, s);
+    if (e != cudaSuccess) return e;
+    for (int pass = 0; pass < 2; ++pass)
+        for (int base = 0; base < num; base += kUpdChunk) {
+            UpdateBatch b;
+            b.num = num - base < kUpdChunk ? num - base : kUpdChunk;
+            b.tensor_base = base;
+            int blocks = 0;
+            for (int k = 0; k < b.num; ++k) {
+                b.t[k] = t[base + k];
+                b.first_block[k] = blocks;
+                blocks += (int)((t[base + k].n + kUpdElemsPerBlock - 1) / kUpdElemsPerBlock);
+            }
+            b.first_block[b.num] = blocks;
+            if (blocks == 0) continue;
+            if (pass == 0) update_absmax_kernel<<<blocks, kThreads, 0, s>>>(b, dev);
+            else update_wide_apply_kernel<<<blocks, kThreads, 0, s>>>(b, lr_mant, lr_exp, k_u, k_m, stochastic, seed, step, step_dev, dev);
+        }
     if (step_dev) step_bump_kernel<<<1, 1, 0, s>>>(step_dev);
     return cudaGetLastError();
 }

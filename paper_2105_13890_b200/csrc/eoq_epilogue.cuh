@@ -62,28 +62,11 @@ __device__ __forceinline__ int32_t sbyte(uint32_t w)
 // The integer pipe bounds this code, so clamps are moved in front of the roundings (both are monotonic, the
 // clamp limits are chosen so that the rounded result is unchanged), roundings run as one FMA each, and the
 // constant offsets of that trick are folded into the multiply-add that forms x4.
-// Global operands of the forward chain for 16 channels of one pixel (b1 table row, shortcut codes).  They do not
-// depend on the accumulator, so the epilogue requests them before it waits for the tile's MMAs: their latency
-// is then hidden behind that wait instead of being added to every tile.
-struct ForwardOperands {
-    int4 table[4];
-    int4 shortcut;
-};
-
-__device__ __forceinline__ ForwardOperands forward_operands(const IgemmParams &p, bool active, size_t off, int col, int cls)
-{
-    ForwardOperands o;
-    if (active && p.b1_table) {
-        const int4 *t = reinterpret_cast<const int4 *>(p.b1_table + (size_t)cls * p.N + col);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) o.table[i] = __ldg(t + i);
-    } else {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) o.table[i] = make_int4(0, 0, 0, 0);
-    }
-    o.shortcut = (active && p.shortcut) ? __ldg(reinterpret_cast<const int4 *>(p.shortcut + off)) : make_int4(0, 0, 0, 0);
-    return o;
-}
+//
+// The b1 term (b1 times the sum of the weights whose taps fall inside the image, per border class and output
+// channel) is read from shared memory, already multiplied by b1: the epilogue warps copy the table there once per
+// kernel (kTableSmemBytes at most; larger tables are read from global memory and multiplied per use).
+constexpr int kTableSmemBytes = 20 * 1024;
 
 // The three scalar codes of the forward chain as the epilogue uses them: the host values of the launch, or the
 // values read from device memory when the caller keeps them there (they then change from one replay of a captured
@@ -116,11 +99,26 @@ __device__ __forceinline__ FwdScalars load_fwd_scalars(const IgemmParams &p)
     return s;
 }
 
+// Filled by the epilogue warps (`nthreads` of them, `tid` = index among them) before their first tile; they meet at
+// named barrier 1 afterwards.  Returns the table's shared-memory address, or null when there is no table or it does
+// not fit (uniform over the kernel).
+__device__ __forceinline__ const int32_t *stage_b1_table(const IgemmParams &p, int32_t b1, uint8_t *smem_table, int tid, int nthreads)
+{
+    const int entries = p.b1_table ? p.b1_nrc * p.b1_ncc * p.N : 0;
+    if (entries == 0 || entries * (int)sizeof(int32_t) > kTableSmemBytes) return nullptr;
+    int32_t *ts = reinterpret_cast<int32_t *>(smem_table);
+    for (int i = tid; i < entries; i += nthreads) ts[i] = b1 * __ldg(p.b1_table + i);
+    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+    return ts;
+}
+
+// `tb`: this pixel's 16 b1 terms in shared memory (already times b1), or null; then `tg` points at the 16 weight
+// sums in global memory (or is null when the layer has no b1 term).  `sc`: the 16 shortcut codes (zero without one).
 // `acc1` holds the tile's second partial sums when `two` is set; kRelu = a ReLU follows.
 template <bool kShift7, bool kRelu>
 __device__ __forceinline__ void forward_16(const IgemmParams &p, const FwdScalars &fs, const uint32_t (&acc)[32],
-                                           const uint32_t (&acc1)[32], bool two, size_t off, const ForwardOperands &ops,
-                                           int shift)
+                                           const uint32_t (&acc1)[32], bool two, size_t off, const int32_t *tb,
+                                           const int32_t *tg, const int4 &sc, int shift)
 {
     int32_t a[16];
 #pragma unroll
@@ -132,10 +130,19 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const FwdScalar
         for (int i = 0; i < 16; ++i) a[i] += (int32_t)acc1[i];
         two = false;
     }
-    if (p.b1_table) {
+    if (tb) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const int4 v = ops.table[i];
+            const int4 v = reinterpret_cast<const int4 *>(tb)[i];
+            a[4 * i + 0] += v.x;
+            a[4 * i + 1] += v.y;
+            a[4 * i + 2] += v.z;
+            a[4 * i + 3] += v.w;
+        }
+    } else if (tg) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int4 v = __ldg(reinterpret_cast<const int4 *>(tg) + i);
             a[4 * i + 0] += fs.b1 * v.x;
             a[4 * i + 1] += fs.b1 * v.y;
             a[4 * i + 2] += fs.b1 * v.z;
@@ -183,7 +190,7 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const FwdScalar
     const uint32_t base = ((uint32_t)fs.b2 << 7) - g * q_bias - 1u;
     uint32_t add[16];
     if (p.shortcut) {
-        const int4 v = ops.shortcut;
+        const int4 v = sc;
         const uint32_t w[4] = {(uint32_t)v.x, (uint32_t)v.y, (uint32_t)v.z, (uint32_t)v.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {

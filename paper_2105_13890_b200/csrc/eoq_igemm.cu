@@ -226,6 +226,10 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         const int g_begin = (groups * part) / kParts, g_end = (groups * (part + 1)) / kParts;
         const bool fwd = p.epilogue == kEpiForward;
         const FwdScalars fs = fwd ? load_fwd_scalars(p) : FwdScalars{0, 0, 0};
+        // the b1 table of the whole layer goes to shared memory (behind the pipeline stages), once, times b1
+        const int32_t *ts = fwd ? stage_b1_table(p, fs.b1, smem_raw + (smem_base - ptx::smem_u32(smem_raw)) + p.num_stages * stage_bytes,
+                                                 (int)threadIdx.x - 128, 32 * kEpilogueWarps)
+                                : nullptr;
         int shift = 7;
         if (fwd && p.x_exp) {
             shift = -__ldg(p.x_exp);
@@ -252,7 +256,11 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
             }
             int col = nt * p.tile_n + g_begin * 16;
             size_t off = pix * p.N + col;
-            ForwardOperands ops = forward_operands(p, fwd && valid && col < p.N, off, col, cls);
+            const int4 zero4 = make_int4(0, 0, 0, 0);
+            // the shortcut codes do not depend on the sums: the first group's are requested before the wait for the MMAs
+            int4 sc = (fwd && valid && col < p.N && p.shortcut) ? __ldg(reinterpret_cast<const int4 *>(p.shortcut + off)) : zero4;
+            const int32_t *tb = ts ? ts + cls * p.N + col : nullptr;
+            const int32_t *tg = (!ts && p.b1_table) ? p.b1_table + (size_t)cls * p.N + col : nullptr;
             if (!(ok = __all_sync(0xffffffffu, wait_bar(tfull_bar(grp), acc_phase, ctx)))) break;  // warp-uniform
             ptx::tc_fence_after();
             const uint32_t t_row = tmem_base + grp * buf_stride + ((uint32_t)(quad * 32) << 16);
@@ -261,9 +269,10 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                 ptx::tmem_ld_32x16(t_row + g * 16, r);
                 uint32_t r2[32];
                 if (nacc == 2) ptx::tmem_ld_32x16(t_row + acc_stride + g * 16, r2);
-                // the next group's operands travel while this group is computed
-                ForwardOperands next = ops;
-                if (g + 1 < g_end) next = forward_operands(p, fwd && valid && col + 16 < p.N, off + 16, col + 16, cls);
+                // the next group's shortcut codes travel while this group is computed
+                int4 sc_next = zero4;
+                if (g + 1 < g_end && fwd && valid && col + 16 < p.N && p.shortcut)
+                    sc_next = __ldg(reinterpret_cast<const int4 *>(p.shortcut + off + 16));
                 ptx::tmem_ld_wait();
                 if (nacc == 2 && !fwd) {
 #pragma unroll
@@ -273,17 +282,19 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                     if (fwd) {
                         const bool two = nacc == 2;
                         if (shift == 7) {
-                            if (p.relu) forward_16<true, true>(p, fs, r, r2, two, off, ops, 7);
-                            else forward_16<true, false>(p, fs, r, r2, two, off, ops, 7);
+                            if (p.relu) forward_16<true, true>(p, fs, r, r2, two, off, tb, tg, sc, 7);
+                            else forward_16<true, false>(p, fs, r, r2, two, off, tb, tg, sc, 7);
                         } else {
-                            if (p.relu) forward_16<false, true>(p, fs, r, r2, two, off, ops, shift);
-                            else forward_16<false, false>(p, fs, r, r2, two, off, ops, shift);
+                            if (p.relu) forward_16<false, true>(p, fs, r, r2, two, off, tb, tg, sc, shift);
+                            else forward_16<false, false>(p, fs, r, r2, two, off, tb, tg, sc, shift);
                         }
                     } else {
                         mx = max(mx, dgrad_16(p, r, off));
                     }
                 }
-                ops = next;
+                sc = sc_next;
+                if (tb) tb += 16;
+                if (tg) tg += 16;
             }
             ptx::tc_fence_before();
             __syncwarp();
@@ -308,14 +319,14 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
 
 size_t igemm_smem_bytes(const IgemmParams &p)
 {
-    return (size_t)p.num_stages * p.subs_per_stage * ((size_t)kTileM + p.tile_n) * p.kc + 1024;
+    return (size_t)p.num_stages * p.subs_per_stage * ((size_t)kTileM + p.tile_n) * p.kc + 1024 + kTableSmemBytes;
 }
 
 cudaError_t launch_igemm(const IgemmParams &p, const CUtensorMap &map_a, const CUtensorMap &map_b, int grid,
                          cudaStream_t stream)
 {
     const size_t smem = igemm_smem_bytes(p);
-    cudaError_t e = cudaFuncSetAttribute(igemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(igemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
     if (e != cudaSuccess) return e;
     igemm_kernel<<<grid, kGemmThreads, smem, stream>>>(p, map_a, map_b);
     return cudaGetLastError();

@@ -37,6 +37,7 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t b_sub = (uint32_t)p.tile_n * p.kc;
     const uint32_t b_region = smem_base + (uint32_t)pl.num_a * pl.a_bytes;
+    const uint32_t table_off = (uint32_t)pl.num_a * pl.a_bytes + (pl.b_resident ? (uint32_t)pl.chunks * p.ntaps : (uint32_t)pl.num_b) * b_sub;
     const uint32_t bar0 = ptx::smem_u32(bars);
     auto a_full = [&](int s) { return bar0 + 8u * s; };
     auto a_empty = [&](int s) { return bar0 + 8u * (kMaxA + s); };
@@ -267,6 +268,10 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
         const int yl = row / pl.pw, xx = row % pl.pw;  // position of this thread's row in the patch raster
         const bool fwd = p.epilogue == kEpiForward;
         const FwdScalars fs = fwd ? load_fwd_scalars(p) : FwdScalars{0, 0, 0};
+        // the b1 table of the whole layer goes to shared memory (behind the operand buffers), once, times b1
+        const int32_t *ts = fwd ? stage_b1_table(p, fs.b1, smem_raw + (smem_base - ptx::smem_u32(smem_raw)) + table_off,
+                                                 (int)threadIdx.x - 128, 32 * kEpilogueWarps)
+                                : nullptr;
         uint32_t acc_phase = 0, mx = 0;
         bool ok = true;
         // (column tile, image, row tile in the image) of the current tile, carried from tile to tile: the step
@@ -290,7 +295,11 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
             }
             int col = nt * p.tile_n + g_begin * 16;
             size_t off = pix * p.N + col;
-            ForwardOperands ops = forward_operands(p, fwd && valid && col < p.N, off, col, cls);
+            const int4 zero4 = make_int4(0, 0, 0, 0);
+            // the shortcut codes do not depend on the sums: the first group's are requested before the wait for the MMAs
+            int4 sc = (fwd && valid && col < p.N && p.shortcut) ? __ldg(reinterpret_cast<const int4 *>(p.shortcut + off)) : zero4;
+            const int32_t *tb = ts ? ts + cls * p.N + col : nullptr;
+            const int32_t *tg = (!ts && p.b1_table) ? p.b1_table + (size_t)cls * p.N + col : nullptr;
             if (!(ok = __all_sync(0xffffffffu, wait_bar<64>(tfull_bar(grp), acc_phase, ctx)))) break;
             ptx::tc_fence_after();
             const uint32_t t_row = tmem_base + grp * buf_stride + ((uint32_t)(quad * 32) << 16);
@@ -299,9 +308,10 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                 ptx::tmem_ld_32x16(t_row + g * 16, r);
                 uint32_t r2[32];
                 if (nacc == 2) ptx::tmem_ld_32x16(t_row + acc_stride + g * 16, r2);
-                // the next group's operands travel while this group is computed
-                ForwardOperands next = ops;
-                if (g + 1 < g_end) next = forward_operands(p, fwd && valid && col + 16 < p.N, off + 16, col + 16, cls);
+                // the next group's shortcut codes travel while this group is computed
+                int4 sc_next = zero4;
+                if (g + 1 < g_end && fwd && valid && col + 16 < p.N && p.shortcut)
+                    sc_next = __ldg(reinterpret_cast<const int4 *>(p.shortcut + off + 16));
                 ptx::tmem_ld_wait();
                 if (nacc == 2 && !fwd) {
 #pragma unroll
@@ -309,12 +319,14 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                 }
                 if (valid && col < p.N) {
                     if (fwd) {
-                        if (p.relu) forward_16<true, true>(p, fs, r, r2, nacc == 2, off, ops, 7);
-                        else forward_16<true, false>(p, fs, r, r2, nacc == 2, off, ops, 7);
+                        if (p.relu) forward_16<true, true>(p, fs, r, r2, nacc == 2, off, tb, tg, sc, 7);
+                        else forward_16<true, false>(p, fs, r, r2, nacc == 2, off, tb, tg, sc, 7);
                     }
                     else mx = max(mx, dgrad_16(p, r, off));
                 }
-                ops = next;
+                sc = sc_next;
+                if (tb) tb += 16;
+                if (tg) tg += 16;
             }
             ptx::tc_fence_before();
             __syncwarp();
@@ -346,13 +358,13 @@ size_t igemm_patch_smem_bytes(const IgemmParams &p, const PatchPlan &pl)
 {
     const size_t b_sub = (size_t)p.tile_n * p.kc;
     const size_t b = pl.b_resident ? (size_t)pl.chunks * p.ntaps * b_sub : (size_t)pl.num_b * b_sub;
-    return (size_t)pl.num_a * pl.a_bytes + b + 1024;
+    return (size_t)pl.num_a * pl.a_bytes + b + 1024 + kTableSmemBytes;
 }
 
 cudaError_t launch_igemm_patch(const IgemmParams &p, const PatchPlan &pl, const CUtensorMap &map_a,
                                const CUtensorMap &map_b, int grid, cudaStream_t stream)
 {
-    cudaError_t e = cudaFuncSetAttribute(igemm_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(igemm_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
     if (e != cudaSuccess) return e;
     igemm_patch_kernel<<<grid, kPatchThreads, igemm_patch_smem_bytes(p, pl), stream>>>(p, pl, map_a, map_b);
     return cudaGetLastError();

@@ -245,11 +245,15 @@ struct UpdateTensor {
     const int8_t *g;
     const int32_t *g_exp;
     unsigned long long n;
+    int32_t *master;  // wide update only: the k_m-bit master codes (w then receives Q_w of them)
 };
 // step_dev (device, optional): the step counter is read from it and it is incremented behind the update.
 cudaError_t launch_update(const UpdateTensor *t, int num, int32_t lr_mant, int32_t lr_exp, int stochastic,
                           uint64_t seed, uint64_t step, unsigned long long *step_dev, DeviceState *dev, int sm_count,
                           cudaStream_t s);
+// The same update with a k_u-bit update quantizer on k_m-bit master codes (t[i].master); t[i].w receives Q_w(master).
+cudaError_t launch_update_wide(const UpdateTensor *t, int num, int32_t lr_mant, int32_t lr_exp, int k_u, int k_m, int stochastic,
+                               uint64_t seed, uint64_t step, unsigned long long *step_dev, DeviceState *dev, cudaStream_t s);
 cudaError_t launch_layout_convert(const int8_t *src, int8_t *dst, int n, int c, int h, int w, int to_nhwc,
                                   cudaStream_t s);
 cudaError_t launch_weight_transpose(const int8_t *w, int8_t *wt, int c_out, int taps, int c_in, cudaStream_t s);

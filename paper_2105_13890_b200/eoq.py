@@ -27,7 +27,7 @@ EXPORTS = [
     "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count", "eoq_set_gemm_ctas",
     "eoq_conv_dgrad_static", "eoq_conv_fwd_dev", "eoq_weight_prep_size", "eoq_weight_prep", "eoq_conv_wgrad_dev",
     "eoq_err_prescale_dev", "eoq_update_dev", "eoq_describe_plan", "eoq_debug_force_wait_timeout", "eoq_probe_mma_i8", "eoq_profile_gemm_only", "eoq_aux_maxpool_fwd", "eoq_aux_maxpool_bwd",
-    "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_error", "eoq_aux_scalar_update",
+    "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide",
 ]
 EOQ_STATIC_SCRATCH_BYTES = 16 << 20
 EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
@@ -97,6 +97,8 @@ def lib() -> C.CDLL:
         L.eoq_err_prescale_dev.argtypes = [vp, vp, vp, vp, vp, sz, vp, vp, vp, vp, vp, vp]
         L.eoq_update_dev.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), i32, i32,
                                      C.c_int, u64, vp, vp]
+        L.eoq_update_wide.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), i32, i32,
+                                      C.c_int, C.c_int, C.c_int, u64, u64, vp, vp]
         L.eoq_describe_plan.argtypes = [vp, dp, C.c_int, C.c_char_p, sz]
         L.eoq_debug_force_wait_timeout.argtypes = [vp]
         ci = C.c_int
@@ -414,3 +416,15 @@ def eoq_aux_scalar_update(handle, theta: Sequence, mirror: Sequence, total: Sequ
                                        arr(*[_ptr(t) for t in total]), arr(*[_ptr(t) for t in total_exp]), iarr(*exp_bias),
                                        iarr(*tensor_id), arr(*[_ptr(t) for t in grad_out]), int(lr_mant), int(lr_exp),
                                        int(round_mode), int(seed), _ptr(step), _stream(stream)), "eoq_aux_scalar_update")
+
+
+def eoq_update_wide(handle, master: Sequence, w: Sequence, g: Sequence, g_exp: Sequence, lr_mant: int, lr_exp: int, k_u: int,
+                    k_m: int, round_mode: int = EOQ_ROUND_RNE, seed: int = 0, step: int = 0, step_dev=None, stream=None) -> None:
+    """The update with a k_u-bit update quantizer on k_m-bit master codes (int32 tensors); w receives Q_w(master)."""
+    num = len(w)
+    arr = C.c_void_p * num
+    sizes = (C.c_size_t * num)(*[t.numel() for t in w])
+    _check(lib().eoq_update_wide(handle, num, arr(*[_ptr(t) for t in master]), arr(*[_ptr(t) for t in w]),
+                                 arr(*[_ptr(t) for t in g]), arr(*[_ptr(t) for t in g_exp]), sizes, int(lr_mant), int(lr_exp),
+                                 int(k_u), int(k_m), int(round_mode), int(seed), int(step), _ptr(step_dev), _stream(stream)),
+           "eoq_update_wide")

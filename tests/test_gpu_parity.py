@@ -578,3 +578,31 @@ def test_wait_that_runs_out_reports_timeout_and_leaves_the_handle_usable():
             assert np.array_equal(G.host(e3), ref) and e3_exp.item() == p3 and s1_d.item() == s1
     finally:
         eoq.eoq_destroy(h)
+
+
+# ------------------------------------------------------------------ other update widths
+
+@pytest.mark.parametrize("k_u,k_m", [(8, 8), (16, 16), (24, 24), (8, 24)])
+@pytest.mark.parametrize("stochastic", [False, True])
+def test_update_at_other_widths(k_u, k_m, stochastic):
+    """Three consecutive updates with a k_u-bit update quantizer on a k_m-bit master copy: master codes and the 8-bit
+    weights derived from them against the oracle; with 24-bit masters, sub-LSB updates accumulate."""
+    sizes = [4096 + 7, 36864, 16]
+    lim = 2 ** (k_m - 1) - 1
+    r = synth.rng(8600, k_m)
+    masters = [r.integers(-lim, lim + 1, size=n).astype(np.int32) for n in sizes]
+    gs = [synth.normal_codes(n, 8601, i, std_codes=40) for i, n in enumerate(sizes)]
+    pgs = [-19, -13, -16]
+    m_d = [G.dev(m) for m in masters]
+    w_d = [G.zeros(n, torch.int8) for n in sizes]
+    step = G.dev(np.array([2], dtype=np.int64))
+    cur = [m.copy() for m in masters]
+    for it in range(3):
+        eoq.eoq_update_wide(G.handle(), m_d, w_d, [G.dev(g) for g in gs], [G.dev(np.array([p], dtype=np.int32)) for p in pgs], 37, -5,
+                            k_u, k_m, eoq.EOQ_ROUND_STOCHASTIC if stochastic else eoq.EOQ_ROUND_RNE, seed=13, step_dev=step)
+        assert G.status_clear() == 0
+        for i in range(len(sizes)):
+            cur[i], w8, _, _ = oracle.update_k(cur[i], gs[i], pgs[i], 37, -5, k_u, k_m, stochastic=stochastic, seed=13, step=2 + it, tensor_id=i)
+            assert np.array_equal(G.host(m_d[i]), cur[i]), (it, i, "master")
+            assert np.array_equal(G.host(w_d[i]), w8), (it, i, "w")
+    assert step.item() == 5
