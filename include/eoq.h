@@ -356,6 +356,26 @@ EOQ_API unsigned long long eoq_launch_count(eoq_handle_t handle);
  * reduction cells back to zero. */
 EOQ_API int eoq_profile_gemm_only(eoq_handle_t handle, int on);
 
+/*
+ * Data-parallel replicas (the paper trains with synchronous SGD on several GPUs, Sec. 5.1).  Every quantizer of the
+ * layer that reduces over the batch -- the maximum behind each SQ (Sec. 3.2.2), the sums behind the scalar gradients,
+ * the exact weight-gradient sums in front of Q_g (Sec. 3.2.1) -- forms its value in one kernel and consumes it in a
+ * later one.  With a hook set, the library calls it on the host between the two, with the device buffer that holds
+ * the local value; the hook enqueues an all-reduce of that buffer on `stream` (ncclAllReduce or the like: in place,
+ * `count` elements, dtype EOQ_REDUCE_I32 or EOQ_REDUCE_I64, op EOQ_REDUCE_MAX over non-negative values or
+ * EOQ_REDUCE_SUM).  Replicas that each hold a share of the batch then continue with the global value and write, bit
+ * for bit, what one device writes on the whole batch: integer maxima and sums do not depend on the order of
+ * reduction.  (One-kernel forms of a call give way to their two-kernel forms while a hook is set.  The float last
+ * layer reduces in a fixed order over the samples: replicas gather sums and labels and each runs eoq_aux_head on
+ * the whole batch.)  fn = NULL removes the hook.
+ */
+#define EOQ_REDUCE_I32 0
+#define EOQ_REDUCE_I64 1
+#define EOQ_REDUCE_MAX 0
+#define EOQ_REDUCE_SUM 1
+typedef void (*eoq_reduce_fn)(void *user, void *device_buffer, size_t count, int dtype, int op, void *stream);
+EOQ_API int eoq_set_reduce_hook(eoq_handle_t handle, eoq_reduce_fn fn, void *user);
+
 /* Caps the CTAs (one per SM) that the GEMM launches of this handle use; 0 = one per SM of the device (the
  * default).  Every GEMM kernel is persistent: with fewer CTAs a launch walks more tiles per CTA and leaves the
  * other SMs free, so that GEMMs issued through two handles on two streams run side by side instead of one after

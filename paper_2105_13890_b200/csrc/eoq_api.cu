@@ -367,6 +367,7 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
     h->profiling = false;
     h->force_timeout = false;
     h->gemm_only = false;
+    h->hook = ReduceHook{nullptr, nullptr};
     h->num_records = 0;
     h->records = nullptr;
     h->branch = nullptr;
@@ -484,6 +485,14 @@ extern "C" int eoq_profile_gemm_only(eoq_handle_t handle, int on)
     }
     h->gemm_only = on != 0;
     return record(h, e);
+}
+
+extern "C" int eoq_set_reduce_hook(eoq_handle_t handle, eoq_reduce_fn fn, void *user)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h) return EOQ_ERR_BAD_ARG;
+    h->hook = ReduceHook{fn, user};
+    return EOQ_OK;
 }
 
 extern "C" int eoq_set_gemm_ctas(eoq_handle_t handle, int ctas)
@@ -864,7 +873,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             {
                 ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
                 e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true,
-                                  h->dev, h->sm_count, s);
+                                  h->dev, h->sm_count, s, h->hook);
             }
             count_launches(h, 1);
             return record(h, e);
@@ -1024,10 +1033,10 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
         if (compact)
             e = launch_sq_i32_scatter(sums, e3_exp, -7, d.n, d.h, d.w, d.c_in, d.stride, (d.h + d.stride - 1) / d.stride,
                                       (d.w + d.stride - 1) / d.stride, e4, e4_exp, reinterpret_cast<long long *>(sum_e4),
-                                      h->dev, h->sm_count, s);
+                                      h->dev, h->sm_count, s, h->hook);
         else
             e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
-                              h->sm_count, s);
+                              h->sm_count, s, h->hook);
     }
     count_launches(h, 1);
     return record(h, e);
@@ -1102,7 +1111,7 @@ static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
         if (e != cudaSuccess) return record(h, e);
         ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
         e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
-                          use_b1 ? tap_sums : nullptr, tap_stride, b1_c, b1_dev, d.c_in, wp.partials, wp.num_splits, h->dev, h->sm_count, s);
+                          use_b1 ? tap_sums : nullptr, tap_stride, b1_c, b1_dev, d.c_in, wp.partials, wp.num_splits, h->dev, h->sm_count, s, h->hook);
         count_launches(h, 2);
         return record(h, e);
     }
@@ -1203,7 +1212,7 @@ static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
     // the kernel leaves sums as [oc][tap][ic], which is the layout of g
     ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
     e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
-                      use_b1 ? tap_sums : nullptr, tap_stride, b1_c, b1_dev, d.c_in, nullptr, 0, h->dev, h->sm_count, s);
+                      use_b1 ? tap_sums : nullptr, tap_stride, b1_c, b1_dev, d.c_in, nullptr, 0, h->dev, h->sm_count, s, h->hook);
     count_launches(h, 2);
     return record(h, e);
 }
@@ -1331,10 +1340,10 @@ extern "C" int eoq_quantize(eoq_handle_t handle, int mode, const void *src, int 
     count_launches(h, mode == EOQ_SQ ? 2 : 1);
     ProfScope prof(h, EOQ_PROF_OTHER, s);
     if (src_is_float)
-        return record(h, launch_quantize_f32(mode, reinterpret_cast<const float *>(src), n, dst, dst_exp, h->dev, h->sm_count, s));
+        return record(h, launch_quantize_f32(mode, reinterpret_cast<const float *>(src), n, dst, dst_exp, h->dev, h->sm_count, s, h->hook));
     if (mode != EOQ_SQ || !src_exp) return EOQ_ERR_UNSUPPORTED;
     return record(h, launch_sq_i32(reinterpret_cast<const int32_t *>(src), src_exp, 0, n, reinterpret_cast<int8_t *>(dst),
-                                   dst_exp, nullptr, false, h->dev, h->sm_count, s));
+                                   dst_exp, nullptr, false, h->dev, h->sm_count, s, h->hook));
 }
 
 static int err_prescale_impl(eoq_handle_t handle, const int8_t *e0, const int32_t *e0_exp, const uint8_t *relu_mask,
@@ -1352,7 +1361,7 @@ static int err_prescale_impl(eoq_handle_t handle, const int8_t *e0, const int32_
     h->force_timeout = false;
     const cudaError_t e = launch_err_prescale(e0, e0_exp, relu_mask, x2, n_el, gamma_c, gamma_dev, e3, e3_exp,
                                               reinterpret_cast<long long *>(sum_e1), reinterpret_cast<long long *>(sum_e1x2),
-                                              h->dev, h->sm_count, s, &kernels, force_timeout);
+                                              h->dev, h->sm_count, s, &kernels, force_timeout, h->hook);
     count_launches(h, kernels);
     return record(h, e);
 }
@@ -1467,7 +1476,7 @@ extern "C" int eoq_quantize_image(eoq_handle_t handle, const float *src, int n, 
     count_launches(h, 2);
     ProfScope prof(h, EOQ_PROF_INPUT_Q, reinterpret_cast<cudaStream_t>(stream));
     return record(h, launch_quantize_image(src, n, hh, ww, c_src, c_dst, wmargin, dst, dst_exp, h->dev, h->sm_count,
-                                           reinterpret_cast<cudaStream_t>(stream)));
+                                           reinterpret_cast<cudaStream_t>(stream), h->hook));
 }
 
 // ================================================================================= network glue
@@ -1498,7 +1507,7 @@ extern "C" int eoq_aux_maxpool_bwd(eoq_handle_t handle, const int8_t *e, const i
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     count_launches(h, 2);
     ProfScope prof(h, EOQ_PROF_GLUE, s);
-    return record(h, launch_maxpool_bwd(e, e_exp, arg, n, hh, ww, c, k, stride, pad, e_in, e_in_exp, h->dev, h->sm_count, s));
+    return record(h, launch_maxpool_bwd(e, e_exp, arg, n, hh, ww, c, k, stride, pad, e_in, e_in_exp, h->dev, h->sm_count, s, h->hook));
 }
 
 extern "C" int eoq_aux_avgpool_sum(eoq_handle_t handle, const int8_t *x, int n, int hw, int c, int32_t *sums, void *stream)
@@ -1522,7 +1531,7 @@ extern "C" int eoq_aux_join(eoq_handle_t handle, const int8_t *a, const int32_t 
     count_launches(h, 2);
     ProfScope prof(h, EOQ_PROF_GLUE, s);
     return record(h, launch_join(a, a_exp, b, b_exp, mask_b, n_el, out, out_exp, reinterpret_cast<long long *>(sum_out), h->dev,
-                                 h->sm_count, s));
+                                 h->sm_count, s, h->hook));
 }
 
 extern "C" int eoq_aux_head_workspace_size(int n, int c, int classes, size_t *bytes)
@@ -1563,7 +1572,7 @@ extern "C" int eoq_aux_head_error(eoq_handle_t handle, const float *dpooled, int
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     count_launches(h, 2);
     ProfScope prof(h, EOQ_PROF_GLUE, s);
-    return record(h, launch_head_error(dpooled, n, c, hw, static_cast<float *>(workspace), e, e_exp, h->dev, h->sm_count, s));
+    return record(h, launch_head_error(dpooled, n, c, hw, static_cast<float *>(workspace), e, e_exp, h->dev, h->sm_count, s, h->hook));
 }
 
 extern "C" int eoq_aux_scalar_update(eoq_handle_t handle, int num, int32_t *const *theta, int32_t *const *mirror,

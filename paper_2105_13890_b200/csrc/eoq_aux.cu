@@ -539,11 +539,13 @@ cudaError_t launch_maxpool_fwd(const int8_t *x, int n, int h, int w, int c, int 
 }
 
 cudaError_t launch_maxpool_bwd(const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int h, int w, int c, int k, int s,
-                               int p, int8_t *e_in, int32_t *e_in_exp, DeviceState *dev, int sm_count, cudaStream_t st)
+                               int p, int8_t *e_in, int32_t *e_in_exp, DeviceState *dev, int sm_count, cudaStream_t st,
+                               const ReduceHook &hook)
 {
     const int ho = (h + 2 * p - k) / s + 1, wo = (w + 2 * p - k) / s + 1;
     const int blocks = blocks_for((size_t)n * h * w * (c / 16), sm_count);
     maxpool_bwd_kernel<0><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, dev);
+    hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, st);
     maxpool_bwd_kernel<1><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, dev);
     return cudaGetLastError();
 }
@@ -556,12 +558,14 @@ cudaError_t launch_avgpool_sum(const int8_t *x, int n, int hw, int c, int32_t *s
 
 cudaError_t launch_join(const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp, const uint8_t *mask_b,
                         size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, DeviceState *dev, int sm_count,
-                        cudaStream_t st)
+                        cudaStream_t st, const ReduceHook &hook)
 {
     const size_t n16 = n_el / 16;
     const int blocks = blocks_for(n16, sm_count, 4);
     join_kernel<0><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, dev);
+    hook(&dev->absmax_u64, 1, EOQ_REDUCE_I64, EOQ_REDUCE_MAX, st);
     join_kernel<1><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, dev);
+    if (sum_out) hook(sum_out, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, st);
     return cudaGetLastError();
 }
 
@@ -584,9 +588,10 @@ cudaError_t launch_head(const int32_t *sums, int n, int c, int hw, int classes, 
 }
 
 cudaError_t launch_head_error(const float *dpooled, int n, int c, int hw, float *ef, int8_t *e, int32_t *e_exp, DeviceState *dev,
-                              int sm_count, cudaStream_t st)
+                              int sm_count, cudaStream_t st, const ReduceHook &hook)
 {
     head_error_scale_kernel<<<blocks_for((size_t)n * c, sm_count, 1), kThreads, 0, st>>>(dpooled, n * c, hw, ef, dev);
+    hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, st);
     head_error_spread_kernel<<<blocks_for((size_t)n * hw * (c / 16), sm_count), kThreads, 0, st>>>(ef, n, hw, c, e, e_exp, dev);
     return cudaGetLastError();
 }

@@ -351,8 +351,9 @@ __global__ void sq_i32_scatter_kernel(const int32_t *__restrict__ src, const int
 // its share of the slices with independent, coalesced loads and the groups meet in shared memory.
 __global__ void wgrad_finalize_kernel(const int32_t *__restrict__ parts, int num_parts, int groups, size_t n, long long *acc,
                                       const long long *__restrict__ tap_sums, size_t replica_stride, int32_t b1_c,
-                                      const int32_t *b1_dev, int c_in, long long *copy_out, DeviceState *dev)
+                                      const int32_t *b1_dev, int c_in, long long *copy_out, DeviceState *dev, int sums_only)
 {
+    // sums_only: the sums are completed elsewhere (an all-reduce over replicas) before their maximum is taken
     __shared__ long long part[256];
     if (b1_dev) b1_c = clampi(__ldg(b1_dev), -32768, 32767);
     const int bx = 256 / groups, tx = threadIdx.x % bx, ty = threadIdx.x / bx;
@@ -396,6 +397,19 @@ __global__ void wgrad_finalize_kernel(const int32_t *__restrict__ parts, int num
             const unsigned long long a = (unsigned long long)(v < 0 ? -v : v);
             mx = a > mx ? a : mx;
         }
+    }
+    mx = block_max_u64(mx);
+    if (threadIdx.x == 0 && mx && !sums_only) atomicMax(&dev->absmax_u64, mx);
+}
+
+// max |.| of int64 sums into the handle's 64-bit cell (used when the sums were completed by an all-reduce)
+__global__ void absmax_i64_kernel(const long long *__restrict__ src, size_t n, DeviceState *dev)
+{
+    unsigned long long mx = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const long long v = src[i];
+        const unsigned long long a = (unsigned long long)(v < 0 ? -v : v);
+        mx = a > mx ? a : mx;
     }
     mx = block_max_u64(mx);
     if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u64, mx);
@@ -1109,20 +1123,22 @@ cudaError_t launch_reset_cells(DeviceState *dev, cudaStream_t s)
 }
 
 cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst, int32_t *dst_exp, DeviceState *dev,
-                                int sm_count, cudaStream_t s)
+                                int sm_count, cudaStream_t s, const ReduceHook &hook)
 {
     if (mode == 2) {
         absmax_f32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
+        hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, s);  // float bit patterns of |x| order like integers
     }
     quantize_f32_kernel<<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(mode, src, n, dst, dst_exp, dev);
     return cudaGetLastError();
 }
 
 cudaError_t launch_quantize_image(const float *src, int n, int h, int w, int c_src, int c_dst, int wmargin, int8_t *dst,
-                                  int32_t *dst_exp, DeviceState *dev, int sm_count, cudaStream_t s)
+                                  int32_t *dst_exp, DeviceState *dev, int sm_count, cudaStream_t s, const ReduceHook &hook)
 {
     const size_t count = (size_t)n * h * w * c_src;
     absmax_f32_kernel<<<grid_for(count / 4 + 1, sm_count), kThreads, 0, s>>>(src, count, dev);
+    hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, s);
     if (c_dst % 16 == 0) {
         const size_t items = (size_t)n * h * (w + 2 * wmargin) * (c_dst / 16);
         quantize_image_kernel<16><<<grid_for(items, sm_count), kThreads, 0, s>>>(src, n * h, w, c_src, c_dst, wmargin, dst, dst_exp, dev);
@@ -1143,34 +1159,48 @@ cudaError_t launch_weight_pad_rows(const int8_t *w, int8_t *wp, int c_out, int k
 
 cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *sum_codes, bool max_already_reduced, DeviceState *dev,
-                          int sm_count, cudaStream_t s)
+                          int sm_count, cudaStream_t s, const ReduceHook &hook)
 {
     if (!max_already_reduced) absmax_i32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
+    hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, s);
     sq_i32_kernel<<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes, dev);
+    if (sum_codes) hook(sum_codes, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, s);
     return cudaGetLastError();
 }
 
 cudaError_t launch_sq_i32_scatter(const int32_t *src, const int32_t *src_exp, int exp_bias, int n_img, int hh, int ww, int c,
                                   int stride, int hq, int wq, int8_t *dst, int32_t *dst_exp, long long *sum_codes,
-                                  DeviceState *dev, int sm_count, cudaStream_t s)
+                                  DeviceState *dev, int sm_count, cudaStream_t s, const ReduceHook &hook)
 {
     const size_t items = (size_t)n_img * hh * ww * (c / 16);
+    hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, s);
     sq_i32_scatter_kernel<<<grid_for(items, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n_img, hh, ww, c, stride, hq, wq,
                                                                         dst, dst_exp, sum_codes, dev);
+    if (sum_codes) hook(sum_codes, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, s);
     return cudaGetLastError();
 }
 
 cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *copy_out, const long long *tap_sums, size_t replica_stride,
                           int32_t b1_c, const int32_t *b1_dev, int c_in, const int32_t *parts, int num_parts,
-                          DeviceState *dev, int sm_count, cudaStream_t s)
+                          DeviceState *dev, int sm_count, cudaStream_t s, const ReduceHook &hook)
 {
     const int groups = !parts ? 1 : (num_parts >= 32 ? 8 : (num_parts >= 8 ? 4 : 1));
     const int bx = 256 / groups;
     size_t blocks = (n + bx - 1) / bx;
     if (blocks > (size_t)sm_count * 16) blocks = (size_t)sm_count * 16;
-    wgrad_finalize_kernel<<<(unsigned)blocks, 256, 0, s>>>(parts, num_parts, groups, n, const_cast<long long *>(src), tap_sums,
-                                                           replica_stride, b1_c, b1_dev, c_in, copy_out, dev);
+    if (hook.fn) {
+        // replicas: local sums (b1 term included, it is linear in the error) -> all-reduce -> maximum of the global sums;
+        // the copy for the caller is taken from the global sums as well
+        wgrad_finalize_kernel<<<(unsigned)blocks, 256, 0, s>>>(parts, num_parts, groups, n, const_cast<long long *>(src), tap_sums,
+                                                               replica_stride, b1_c, b1_dev, c_in, nullptr, dev, 1);
+        hook(const_cast<long long *>(src), n, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, s);
+        absmax_i64_kernel<<<grid_for(n, sm_count, 4), kThreads, 0, s>>>(src, n, dev);
+        if (copy_out) cudaMemcpyAsync(copy_out, src, n * sizeof(long long), cudaMemcpyDeviceToDevice, s);
+    } else {
+        wgrad_finalize_kernel<<<(unsigned)blocks, 256, 0, s>>>(parts, num_parts, groups, n, const_cast<long long *>(src), tap_sums,
+                                                               replica_stride, b1_c, b1_dev, c_in, copy_out, dev, 0);
+    }
     sq_i64_kernel<<<grid_for(n, sm_count, 4), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, dev);
     return cudaGetLastError();
 }
@@ -1178,7 +1208,7 @@ cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_
 cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const uint8_t *mask, const int16_t *x2,
                                 size_t n_el, int32_t gamma_c, const int32_t *gamma_dev, int8_t *e3, int32_t *e3_exp,
                                 long long *sum_e1, long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s,
-                                int *kernels, bool force_timeout)
+                                int *kernels, bool force_timeout, const ReduceHook &hook)
 {
     const size_t n16 = n_el / 16;
     *kernels = 2;
@@ -1198,7 +1228,7 @@ cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const u
     }
     const size_t max_blocks = (size_t)blocks_per_sm * sm_count;
     const size_t need_blocks = (n16 + (size_t)kThreads * kFusedGroups - 1) / ((size_t)kThreads * kFusedGroups);
-    if (coop && n16 > 0 && need_blocks <= max_blocks) {
+    if (coop && !hook.fn && n16 > 0 && need_blocks <= max_blocks) {
         // self-test of the bounded wait: one arrival more than there are blocks and a short limit
         unsigned expected = (unsigned)need_blocks + (force_timeout ? 1u : 0u);
         uint32_t spin_limit = force_timeout ? 2048u : kSpinLimit;
@@ -1214,6 +1244,8 @@ cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const u
         (void)cudaGetLastError();  // fewer SMs at hand than at start-up (e.g. a partitioned device): two kernels instead
     }
     prescale_reduce_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, mask, x2, n16, dev);
+    hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, s);
+    hook(&dev->sum0, 2, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, s);  // sum0 and sum1 are adjacent
     prescale_apply_kernel<<<grid_for(n16, sm_count), kThreads, 0, s>>>(e0, e0_exp, mask, n16, gamma_c, gamma_dev, e3,
                                                                        e3_exp, sum_e1, sum_e1x2, dev);
     return cudaGetLastError();

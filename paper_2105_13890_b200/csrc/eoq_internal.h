@@ -31,6 +31,17 @@ struct DeviceState {
 // no call starts with a memset.  A kernel that gave up on a wait (EOQ_DEV_TIMEOUT) may leave them dirty:
 // eoq_last_status clears them again when it reports that bit.
 
+// eoq_set_reduce_hook: called on the host between the kernel that forms a value reduced over the batch and the kernel
+// that consumes it; it enqueues an all-reduce of the device buffer on the stream (no-op when no hook is set).
+struct ReduceHook {
+    eoq_reduce_fn fn;
+    void *user;
+    void operator()(void *ptr, size_t count, int dtype, int op, cudaStream_t s) const
+    {
+        if (fn) fn(user, ptr, count, dtype, op, reinterpret_cast<void *>(s));
+    }
+};
+
 constexpr int kClassBranches = 3;
 
 struct ProfRecord {
@@ -45,6 +56,7 @@ struct Handle {
     DeviceState *dev;
     unsigned long long launches;  // kernels launched through this handle
     bool profiling;
+    ReduceHook hook;              // all-reduce between the phases of every batch-wide reduction (data-parallel replicas)
     bool gemm_only;               // timing aid: dgrad and wgrad calls launch their GEMM kernel only (eoq_profile_gemm_only)
     bool force_timeout;           // self-test: the next error-head call makes its grid-wide wait run out
     int num_records;
@@ -215,31 +227,31 @@ cudaError_t launch_probe_mma_i8(int n_cols, int iters, int grid, DeviceState *de
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_reset_cells(DeviceState *dev, cudaStream_t s);
 cudaError_t launch_quantize_image(const float *src, int n, int h, int w, int c_src, int c_dst, int wmargin, int8_t *dst,
-                                  int32_t *dst_exp, DeviceState *dev, int sm_count, cudaStream_t s);
+                                  int32_t *dst_exp, DeviceState *dev, int sm_count, cudaStream_t s, const ReduceHook &hook);
 // w[oc][kh][kw][16] -> wp[oc][kh][8][16], zero in the taps kw..7 (weights of the filter-row path)
 cudaError_t launch_weight_pad_rows(const int8_t *w, int8_t *wp, int c_out, int kh, int kw, int c_in, cudaStream_t s);
 cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst, int32_t *dst_exp, DeviceState *dev,
-                                int sm_count, cudaStream_t s);
+                                int sm_count, cudaStream_t s, const ReduceHook &hook);
 cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *sum_codes, bool max_already_reduced, DeviceState *dev,
-                          int sm_count, cudaStream_t s);
+                          int sm_count, cudaStream_t s, const ReduceHook &hook);
 // Q_g of the exact sums.  `src` holds int64 sums; when `parts` is given the sums are first formed from
 // `num_parts` int32 slices of n elements each (and written to src).
 cudaError_t launch_sq_i32_scatter(const int32_t *src, const int32_t *src_exp, int exp_bias, int n_img, int hh, int ww, int c,
                                   int stride, int hq, int wq, int8_t *dst, int32_t *dst_exp, long long *sum_codes,
-                                  DeviceState *dev, int sm_count, cudaStream_t s);
+                                  DeviceState *dev, int sm_count, cudaStream_t s, const ReduceHook &hook);
 // b1 is b1_c, or the code at b1_dev when that is given.  Two kernels: slice sum + b1 term + max, then Q_g; the maximum
 // travels through the handle's absmax_u64 cell, which the second kernel puts back to zero.
 // tap_sums: kTapReplicas copies, `replica_stride` elements apart, whose sum is the b1 error sum per (oc, tap).
 cudaError_t launch_sq_i64(const long long *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *copy_out, const long long *tap_sums, size_t replica_stride,
                           int32_t b1_c, const int32_t *b1_dev, int c_in, const int32_t *parts, int num_parts,
-                          DeviceState *dev, int sm_count, cudaStream_t s);
+                          DeviceState *dev, int sm_count, cudaStream_t s, const ReduceHook &hook);
 // gamma is gamma_c, or the code at gamma_dev when that is given.  force_timeout: self-test of the bounded wait.
 cudaError_t launch_err_prescale(const int8_t *e0, const int32_t *e0_exp, const uint8_t *mask, const int16_t *x2,
                                 size_t n_el, int32_t gamma_c, const int32_t *gamma_dev, int8_t *e3, int32_t *e3_exp,
                                 long long *sum_e1, long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t s,
-                                int *kernels, bool force_timeout);
+                                int *kernels, bool force_timeout, const ReduceHook &hook);
 struct UpdateTensor {
     int8_t *w;
     const int8_t *g;
@@ -292,16 +304,17 @@ cudaError_t launch_weight_prep(const PrepBatch &b, cudaStream_t s);
 cudaError_t launch_maxpool_fwd(const int8_t *x, int n, int h, int w, int c, int k, int s, int p, int8_t *y, uint8_t *arg,
                                int sm_count, cudaStream_t st);
 cudaError_t launch_maxpool_bwd(const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int h, int w, int c, int k, int s,
-                               int p, int8_t *e_in, int32_t *e_in_exp, DeviceState *dev, int sm_count, cudaStream_t st);
+                               int p, int8_t *e_in, int32_t *e_in_exp, DeviceState *dev, int sm_count, cudaStream_t st,
+                               const ReduceHook &hook);
 cudaError_t launch_avgpool_sum(const int8_t *x, int n, int hw, int c, int32_t *sums, cudaStream_t st);
 cudaError_t launch_join(const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp, const uint8_t *mask_b,
                         size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, DeviceState *dev, int sm_count,
-                        cudaStream_t st);
+                        cudaStream_t st, const ReduceHook &hook);
 cudaError_t launch_head(const int32_t *sums, int n, int c, int hw, int classes, float *W, float *bias, const int32_t *labels,
                         float lr, float *loss_out, float *dpooled, float *logits, float *pooled, float *dl, double *loss_n,
                         cudaStream_t st);
 cudaError_t launch_head_error(const float *dpooled, int n, int c, int hw, float *ef, int8_t *e, int32_t *e_exp, DeviceState *dev,
-                              int sm_count, cudaStream_t st);
+                              int sm_count, cudaStream_t st, const ReduceHook &hook);
 struct ScalarItem {
     int32_t *theta;          // the code to update (device)
     int32_t *mirror;         // a second place that receives the new code, or null

@@ -65,6 +65,7 @@ extern "C" int eoq_conv_dgrad_static(const eoq_conv_desc_t *desc, const int8_t *
     h.profiling = false;
     h.force_timeout = false;
     h.gemm_only = false;
+    h.hook = ReduceHook{nullptr, nullptr};
     h.num_records = 0;
     h.records = nullptr;
     h.branch = nullptr;

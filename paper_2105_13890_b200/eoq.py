@@ -27,7 +27,7 @@ EXPORTS = [
     "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count", "eoq_set_gemm_ctas",
     "eoq_conv_dgrad_static", "eoq_conv_fwd_dev", "eoq_weight_prep_size", "eoq_weight_prep", "eoq_conv_wgrad_dev",
     "eoq_err_prescale_dev", "eoq_update_dev", "eoq_describe_plan", "eoq_debug_force_wait_timeout", "eoq_probe_mma_i8", "eoq_profile_gemm_only", "eoq_aux_maxpool_fwd", "eoq_aux_maxpool_bwd",
-    "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide",
+    "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide", "eoq_set_reduce_hook",
 ]
 EOQ_STATIC_SCRATCH_BYTES = 16 << 20
 EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
@@ -59,6 +59,10 @@ def conv_desc(n, h, w, c_in, c_out, kh, kw, stride=1, pad=0, x_wmargin=0) -> eoq
 
 
 _lib = None
+# void fn(void *user, void *device_buffer, size_t count, int dtype, int op, void *stream)
+REDUCE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p, C.c_size_t, C.c_int, C.c_int, C.c_void_p)
+EOQ_REDUCE_I32, EOQ_REDUCE_I64 = 0, 1
+EOQ_REDUCE_MAX, EOQ_REDUCE_SUM = 0, 1
 
 
 def lib() -> C.CDLL:
@@ -99,6 +103,7 @@ def lib() -> C.CDLL:
                                      C.c_int, u64, vp, vp]
         L.eoq_update_wide.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(sz), i32, i32,
                                       C.c_int, C.c_int, C.c_int, u64, u64, vp, vp]
+        L.eoq_set_reduce_hook.argtypes = [vp, REDUCE_FN, vp]
         L.eoq_describe_plan.argtypes = [vp, dp, C.c_int, C.c_char_p, sz]
         L.eoq_debug_force_wait_timeout.argtypes = [vp]
         ci = C.c_int
@@ -428,3 +433,9 @@ def eoq_update_wide(handle, master: Sequence, w: Sequence, g: Sequence, g_exp: S
                                  arr(*[_ptr(t) for t in g]), arr(*[_ptr(t) for t in g_exp]), sizes, int(lr_mant), int(lr_exp),
                                  int(k_u), int(k_m), int(round_mode), int(seed), int(step), _ptr(step_dev), _stream(stream)),
            "eoq_update_wide")
+
+
+def eoq_set_reduce_hook(handle, fn) -> None:
+    """Installs (fn = a REDUCE_FN instance, which the caller keeps alive) or removes (fn = None) the all-reduce hook of
+    a handle: see eoq_set_reduce_hook in eoq.h."""
+    _check(lib().eoq_set_reduce_hook(handle, fn if fn is not None else REDUCE_FN(), None), "eoq_set_reduce_hook")
