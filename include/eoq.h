@@ -173,8 +173,12 @@ EOQ_API int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
  * Limits and rules:
  *   - geometries whose eoq_workspace_size(desc, EOQ_PASS_DGRAD) exceeds EOQ_STATIC_SCRATCH_BYTES are rejected
  *     with EOQ_ERR_WORKSPACE and nothing is launched;
- *   - the first call on a device resolves the array's device address and reads device attributes (no
- *     allocation); make that first call outside any stream capture, with the device current;
+ *   - the first call on a device resolves the array's device address and reads device attributes; make that first
+ *     call outside any stream capture, with the device current.  The call itself allocates nothing, but the array's
+ *     memory is reserved by the CUDA driver when the library's module is loaded on the device, which happens at the
+ *     latest during this first call: on a device whose memory is already taken (a pool that grabbed all of it
+ *     before the library was touched) the call returns EOQ_ERR_CUDA, and eoq_last_cuda_error(NULL) gives the
+ *     driver's code.  Load the library, and make one call, before handing the device's memory to a pool;
  *   - all calls on a device share the one array, which keeps the previous call's contents: the cells that must
  *     start at zero are cleared on the stream at the start of each call, and two calls that overlap on the GPU
  *     (different streams, no ordering between them) race on it -- order them.
@@ -407,7 +411,8 @@ EOQ_API int eoq_describe_plan(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
  * hangs; one call only, then the handle behaves normally again. */
 EOQ_API int eoq_debug_force_wait_timeout(eoq_handle_t handle);
 
-/* The last cudaError_t a call on this handle recorded (0 if none). */
+/* The last cudaError_t a call on this handle recorded (0 if none); handle = NULL: the last one of
+ * eoq_conv_dgrad_static, which has no handle. */
 EOQ_API int eoq_last_cuda_error(eoq_handle_t handle);
 
 EOQ_API const char *eoq_status_string(int status);

@@ -370,7 +370,6 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
     h->hook = ReduceHook{nullptr, nullptr};
     h->num_records = 0;
     h->records = nullptr;
-    h->branch = nullptr;
     h->fork_ev = h->join_ev = nullptr;
     for (int k = 0; k < kClassBranches; ++k) {
         h->class_branch[k] = nullptr;
@@ -388,7 +387,6 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
         e = cudaMalloc(reinterpret_cast<void **>(&h->dev), sizeof(DeviceState));
     }
     if (e == cudaSuccess) e = cudaMemset(h->dev, 0, sizeof(DeviceState));
-    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->branch, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->fork_ev, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->join_ev, cudaEventDisableTiming);
     for (int k = 0; k < kClassBranches && e == cudaSuccess; ++k) {
@@ -403,7 +401,6 @@ extern "C" int eoq_create(eoq_handle_t *handle, int device)
         }
         if (h->join_ev) cudaEventDestroy(h->join_ev);
         if (h->fork_ev) cudaEventDestroy(h->fork_ev);
-        if (h->branch) cudaStreamDestroy(h->branch);
         if (h->dev) cudaFree(h->dev);
         delete h;
         return EOQ_ERR_CUDA;
@@ -424,7 +421,6 @@ extern "C" int eoq_destroy(eoq_handle_t handle)
     }
     if (h->join_ev) cudaEventDestroy(h->join_ev);
     if (h->fork_ev) cudaEventDestroy(h->fork_ev);
-    if (h->branch) cudaStreamDestroy(h->branch);
     if (h->dev) cudaFree(h->dev);
     if (h->records) {
         for (int i = 0; i < h->num_records; ++i) {
@@ -560,7 +556,7 @@ extern "C" int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits
 extern "C" int eoq_last_cuda_error(eoq_handle_t handle)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
-    return h ? h->last_cuda_error : 0;
+    return h ? h->last_cuda_error : static_path_last_cuda_error();
 }
 
 extern "C" const char *eoq_status_string(int status)

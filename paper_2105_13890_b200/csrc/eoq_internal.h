@@ -64,7 +64,6 @@ struct Handle {
     // Fork and join events of the calls that issue independent kernels on the class_branch streams (null branch
     // streams: everything stays on the caller's stream).  Under stream capture they become graph edges.
     int gemm_ctas;                // most CTAs a GEMM launch of this handle may use (eoq_set_gemm_ctas; default: one per SM)
-    cudaStream_t branch;
     cudaEvent_t fork_ev, join_ev;
     // further branch streams: the per-class GEMMs of a strided error back-propagation write disjoint pixels and
     // run side by side, each with its share of the CTAs
@@ -72,6 +71,7 @@ struct Handle {
     cudaEvent_t class_join[kClassBranches];
 };
 constexpr int kMaxProfRecords = 8192;
+int static_path_last_cuda_error();  // last cudaError_t of eoq_conv_dgrad_static (eoq_static.cu)
 
 // Counts `n` kernel launches on the handle.
 inline void count_launches(Handle *h, int n) { h->launches += (unsigned long long)n; }
