@@ -79,18 +79,26 @@ __global__ void maxpool_fwd_kernel(const int8_t *__restrict__ x, int n, int h, i
     }
 }
 
-// Backward in gather form: an input position collects the error of every window that elected it (exact sums, no
-// atomics; at most k * k windows, so the sums are small).  Q_e needs the maximum over the whole tensor first, so the
-// gather runs twice: pass 0 reduces max |sum| into the handle's cell, pass 1 forms the sums again and codes them.
-// e and arg are a quarter of the output's size and stay in L2; no intermediate tensor is written.
+// Backward: every output error code is added at the input position its window elected; the exact sums are then
+// coded with Q_e, which needs their maximum over the whole tensor first.  So the kernel runs twice: pass 0 reduces
+// max |sum| into the handle's cell, pass 1 forms the sums again and codes them (no intermediate tensor is written).
+// A block owns a tile of kPoolTile x kPoolTile input positions of one image and one group of 16 channels: it reads the
+// windows that can reach the tile once (a position is covered by up to ceil(k / stride)^2 windows, so reading per
+// position would fetch every window that many times), adds their codes into shared memory, then walks its tile.
+constexpr int kPoolTile = 16;
 template <int kPass>
-__global__ void maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *e_exp, const uint8_t *__restrict__ arg, int n, int h,
-                                   int w, int c, int k, int s, int p, int ho, int wo, int8_t *__restrict__ e_in, int32_t *e_in_exp,
-                                   DeviceState *dev)
+__global__ void __launch_bounds__(kPoolTile *kPoolTile)
+maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *e_exp, const uint8_t *__restrict__ arg, int n, int h, int w, int c,
+                   int k, int s, int p, int ho, int wo, int tiles_x, int tiles_y, int8_t *__restrict__ e_in, int32_t *e_in_exp,
+                   DeviceState *dev)
 {
+    __shared__ int acc[kPoolTile * kPoolTile][17];   // [position][channel], padded against bank conflicts
     const int groups = c / 16;
-    const size_t items = (size_t)n * h * w * groups;
-    uint32_t mx = 0;
+    int bid = blockIdx.x;
+    const int tx = bid % tiles_x; bid /= tiles_x;
+    const int ty = bid % tiles_y; bid /= tiles_y;
+    const int g = bid % groups, img = bid / groups;
+    const int y0 = ty * kPoolTile, x0 = tx * kPoolTile;
     int t = 7;
     if (kPass == 1) {
         const uint32_t M = dev->absmax_u32;
@@ -101,41 +109,43 @@ __global__ void maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *
             if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
         }
     }
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (size_t)gridDim.x * blockDim.x) {
-        const uint32_t i32 = (uint32_t)i, pix = i32 / (uint32_t)groups, row = pix / (uint32_t)w;
-        const int g = (int)(i32 - pix * (uint32_t)groups), ix = (int)(pix - row * (uint32_t)w);
-        const int b = (int)(row / (uint32_t)h), iy = (int)(row - (uint32_t)b * (uint32_t)h);
-        int acc[16];
 #pragma unroll
-        for (int q = 0; q < 16; ++q) acc[q] = 0;
-        // the windows that cover (iy, ix): taps kh congruent to iy + p modulo the stride; the output row falls by
-        // one as kh grows by the stride, so one division per axis serves all of them
-        const int kh0 = (iy + p) % s, kw0 = (ix + p) % s;
-        const int oy0 = (iy + p - kh0) / s, ox0 = (ix + p - kw0) / s;
-        for (int kh = kh0, oy = oy0; kh < k && oy >= 0; kh += s, --oy) {
-            if (oy >= ho) continue;
-            for (int kw = kw0, ox = ox0; kw < k && ox >= 0; kw += s, --ox) {
-                if (ox >= wo) continue;
-                const size_t o = (((size_t)b * ho + oy) * wo + ox) * c + g * 16;
-                const int4 ev = __ldg(reinterpret_cast<const int4 *>(e + o));
-                const int4 av = __ldg(reinterpret_cast<const int4 *>(arg + o));
-                const int8_t *eb = reinterpret_cast<const int8_t *>(&ev);
-                const uint8_t *ab = reinterpret_cast<const uint8_t *>(&av);
-                const int tap = kh * k + kw;
+    for (int q = 0; q < 16; ++q) acc[threadIdx.x][q] = 0;
+    __syncthreads();
+    // windows whose footprint [o * s - p, o * s - p + k) meets the tile
+    const int oy_lo = max(0, (y0 + p - k + s) / s), oy_hi = min(ho - 1, (y0 + kPoolTile - 1 + p) / s);
+    const int ox_lo = max(0, (x0 + p - k + s) / s), ox_hi = min(wo - 1, (x0 + kPoolTile - 1 + p) / s);
+    const int nwx = ox_hi - ox_lo + 1, nwin = (oy_hi - oy_lo + 1) * nwx;
+    for (int wi = threadIdx.x; wi < nwin; wi += blockDim.x) {
+        const int oy = oy_lo + wi / nwx, ox = ox_lo + wi % nwx;
+        const size_t o = (((size_t)img * ho + oy) * wo + ox) * c + g * 16;
+        const int4 ev = __ldg(reinterpret_cast<const int4 *>(e + o));
+        const int4 av = __ldg(reinterpret_cast<const int4 *>(arg + o));
+        const int8_t *eb = reinterpret_cast<const int8_t *>(&ev);
+        const uint8_t *ab = reinterpret_cast<const uint8_t *>(&av);
 #pragma unroll
-                for (int q = 0; q < 16; ++q)
-                    if (ab[q] == tap) acc[q] += eb[q];
-            }
+        for (int q = 0; q < 16; ++q) {
+            const int kh = ab[q] / k, kw = ab[q] - kh * k;
+            const int ly = oy * s - p + kh - y0, lx = ox * s - p + kw - x0;
+            if (eb[q] && (unsigned)ly < (unsigned)kPoolTile && (unsigned)lx < (unsigned)kPoolTile)
+                atomicAdd(&acc[ly * kPoolTile + lx][q], (int)eb[q]);
         }
+    }
+    __syncthreads();
+    const int ly = threadIdx.x / kPoolTile, lx = threadIdx.x % kPoolTile;
+    const int iy = y0 + ly, ix = x0 + lx;
+    uint32_t mx = 0;
+    if (iy < h && ix < w) {
         if (kPass == 0) {
 #pragma unroll
-            for (int q = 0; q < 16; ++q) mx = max(mx, (uint32_t)abs(acc[q]));
+            for (int q = 0; q < 16; ++q) mx = max(mx, (uint32_t)abs(acc[threadIdx.x][q]));
         } else {
             int cd[16];
 #pragma unroll
-            for (int q = 0; q < 16; ++q) cd[q] = sq_code32(acc[q], t);
-            reinterpret_cast<int4 *>(e_in)[i] = make_int4((int)pack4(cd[0], cd[1], cd[2], cd[3]), (int)pack4(cd[4], cd[5], cd[6], cd[7]),
-                                                           (int)pack4(cd[8], cd[9], cd[10], cd[11]), (int)pack4(cd[12], cd[13], cd[14], cd[15]));
+            for (int q = 0; q < 16; ++q) cd[q] = sq_code32(acc[threadIdx.x][q], t);
+            *reinterpret_cast<int4 *>(e_in + (((size_t)img * h + iy) * w + ix) * c + g * 16) =
+                make_int4((int)pack4(cd[0], cd[1], cd[2], cd[3]), (int)pack4(cd[4], cd[5], cd[6], cd[7]),
+                          (int)pack4(cd[8], cd[9], cd[10], cd[11]), (int)pack4(cd[12], cd[13], cd[14], cd[15]));
         }
     }
     if (kPass == 0) {
@@ -391,7 +401,19 @@ __global__ void head_dpooled_kernel(const float *__restrict__ dl, const float *_
     if (i >= n * c) return;
     const int b = i / c, k = i % c;
     float acc = 0.0f;
-    for (int j = 0; j < classes; ++j) acc = __fmaf_rn(dl[(size_t)b * classes + j], W[(size_t)j * c + k], acc);
+    const float *db = dl + (size_t)b * classes, *wk = W + k;
+    int j = 0;
+    for (; j + 8 <= classes; j += 8) {   // eight independent loads in flight, then the chain in order
+        float w8[8], d8[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            w8[u] = __ldg(wk + (size_t)(j + u) * c);
+            d8[u] = __ldg(db + j + u);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc = __fmaf_rn(d8[u], w8[u], acc);
+    }
+    for (; j < classes; ++j) acc = __fmaf_rn(__ldg(db + j), __ldg(wk + (size_t)j * c), acc);
     dpooled[i] = acc;
 }
 
@@ -403,7 +425,18 @@ __global__ void head_update_kernel(const float *__restrict__ dl, const float *__
     if (i >= classes * c) return;
     const int j = i / c, k = i % c;
     float acc = 0.0f;
-    for (int b = 0; b < n; ++b) acc = __fmaf_rn(dl[(size_t)b * classes + j], pooled[(size_t)b * c + k], acc);
+    int b = 0;
+    for (; b + 8 <= n; b += 8) {
+        float d8[8], p8[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            d8[u] = __ldg(dl + (size_t)(b + u) * classes + j);
+            p8[u] = __ldg(pooled + (size_t)(b + u) * c + k);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc = __fmaf_rn(d8[u], p8[u], acc);
+    }
+    for (; b < n; ++b) acc = __fmaf_rn(__ldg(dl + (size_t)b * classes + j), __ldg(pooled + (size_t)b * c + k), acc);
     W[i] = __fmaf_rn(-lr, acc, W[i]);
     if (k == 0) {
         float db = 0.0f;
@@ -542,11 +575,15 @@ cudaError_t launch_maxpool_bwd(const int8_t *e, const int32_t *e_exp, const uint
                                int p, int8_t *e_in, int32_t *e_in_exp, DeviceState *dev, int sm_count, cudaStream_t st,
                                const ReduceHook &hook)
 {
+    (void)sm_count;
     const int ho = (h + 2 * p - k) / s + 1, wo = (w + 2 * p - k) / s + 1;
-    const int blocks = blocks_for((size_t)n * h * w * (c / 16), sm_count);
-    maxpool_bwd_kernel<0><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, dev);
+    const int tiles_x = (w + kPoolTile - 1) / kPoolTile, tiles_y = (h + kPoolTile - 1) / kPoolTile;
+    const unsigned blocks = (unsigned)((size_t)n * (c / 16) * tiles_x * tiles_y);
+    maxpool_bwd_kernel<0><<<blocks, kPoolTile * kPoolTile, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, tiles_x, tiles_y, e_in,
+                                                                  e_in_exp, dev);
     hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, st);
-    maxpool_bwd_kernel<1><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, dev);
+    maxpool_bwd_kernel<1><<<blocks, kPoolTile * kPoolTile, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, tiles_x, tiles_y, e_in,
+                                                                  e_in_exp, dev);
     return cudaGetLastError();
 }
 
