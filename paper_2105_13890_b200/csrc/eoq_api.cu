@@ -1499,7 +1499,7 @@ extern "C" int eoq_aux_maxpool_bwd(eoq_handle_t handle, const int8_t *e, const i
         stride <= 0 || pad < 0 || pad >= k)
         return EOQ_ERR_BAD_ARG;
     if (c % 16 || !aligned16(e) || !aligned16(arg) || !aligned16(e_in)) return EOQ_ERR_ALIGNMENT;
-    if ((size_t)n * (c / 16) * ((hh + 15) / 16) * ((ww + 15) / 16) > 0x7fffffffull) return EOQ_ERR_UNSUPPORTED;
+    if ((size_t)n * hh * ww * (c / 16) > 0x7fffffffull) return EOQ_ERR_UNSUPPORTED;   // 32-bit item index in the kernel
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     count_launches(h, 2);
     ProfScope prof(h, EOQ_PROF_GLUE, s);

@@ -82,23 +82,17 @@ __global__ void maxpool_fwd_kernel(const int8_t *__restrict__ x, int n, int h, i
 // Backward: every output error code is added at the input position its window elected; the exact sums are then
 // coded with Q_e, which needs their maximum over the whole tensor first.  So the kernel runs twice: pass 0 reduces
 // max |sum| into the handle's cell, pass 1 forms the sums again and codes them (no intermediate tensor is written).
-// A block owns a tile of kPoolTile x kPoolTile input positions of one image and one group of 16 channels: it reads the
-// windows that can reach the tile once (a position is covered by up to ceil(k / stride)^2 windows, so reading per
-// position would fetch every window that many times), adds their codes into shared memory, then walks its tile.
-constexpr int kPoolTile = 16;
+// One thread per 16 channels of an input position gathers from the windows that cover it (at most
+// ceil(k / stride)^2): a window's 16 codes count where its recorded position equals this one.  Four codes are
+// handled per 32-bit word: bytes are compared at once, the chosen codes are kept with an offset of 128 (others as
+// 128 itself) so that they add as unsigned halves of two words without carries between them.
 template <int kPass>
-__global__ void __launch_bounds__(kPoolTile *kPoolTile)
+__global__ void __launch_bounds__(kThreads)
 maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *e_exp, const uint8_t *__restrict__ arg, int n, int h, int w, int c,
-                   int k, int s, int p, int ho, int wo, int tiles_x, int tiles_y, int8_t *__restrict__ e_in, int32_t *e_in_exp,
-                   DeviceState *dev)
+                   int k, int s, int p, int ho, int wo, int8_t *__restrict__ e_in, int32_t *e_in_exp, DeviceState *dev)
 {
-    __shared__ int acc[kPoolTile * kPoolTile][17];   // [position][channel], padded against bank conflicts
     const int groups = c / 16;
-    int bid = blockIdx.x;
-    const int tx = bid % tiles_x; bid /= tiles_x;
-    const int ty = bid % tiles_y; bid /= tiles_y;
-    const int g = bid % groups, img = bid / groups;
-    const int y0 = ty * kPoolTile, x0 = tx * kPoolTile;
+    const uint32_t items = (uint32_t)n * h * w * groups;   // below 2^31 (checked by the caller), so i + stride cannot wrap
     int t = 7;
     if (kPass == 1) {
         const uint32_t M = dev->absmax_u32;
@@ -109,41 +103,49 @@ maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *e_exp, const uin
             if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
         }
     }
-#pragma unroll
-    for (int q = 0; q < 16; ++q) acc[threadIdx.x][q] = 0;
-    __syncthreads();
-    // windows whose footprint [o * s - p, o * s - p + k) meets the tile
-    const int oy_lo = max(0, (y0 + p - k + s) / s), oy_hi = min(ho - 1, (y0 + kPoolTile - 1 + p) / s);
-    const int ox_lo = max(0, (x0 + p - k + s) / s), ox_hi = min(wo - 1, (x0 + kPoolTile - 1 + p) / s);
-    const int nwx = ox_hi - ox_lo + 1, nwin = (oy_hi - oy_lo + 1) * nwx;
-    for (int wi = threadIdx.x; wi < nwin; wi += blockDim.x) {
-        const int oy = oy_lo + wi / nwx, ox = ox_lo + wi % nwx;
-        const size_t o = (((size_t)img * ho + oy) * wo + ox) * c + g * 16;
-        const int4 ev = __ldg(reinterpret_cast<const int4 *>(e + o));
-        const int4 av = __ldg(reinterpret_cast<const int4 *>(arg + o));
-        const int8_t *eb = reinterpret_cast<const int8_t *>(&ev);
-        const uint8_t *ab = reinterpret_cast<const uint8_t *>(&av);
-#pragma unroll
-        for (int q = 0; q < 16; ++q) {
-            const int kh = ab[q] / k, kw = ab[q] - kh * k;
-            const int ly = oy * s - p + kh - y0, lx = ox * s - p + kw - x0;
-            if (eb[q] && (unsigned)ly < (unsigned)kPoolTile && (unsigned)lx < (unsigned)kPoolTile)
-                atomicAdd(&acc[ly * kPoolTile + lx][q], (int)eb[q]);
-        }
-    }
-    __syncthreads();
-    const int ly = threadIdx.x / kPoolTile, lx = threadIdx.x % kPoolTile;
-    const int iy = y0 + ly, ix = x0 + lx;
     uint32_t mx = 0;
-    if (iy < h && ix < w) {
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < items; i += gridDim.x * blockDim.x) {
+        const uint32_t pix = i / (uint32_t)groups, row = pix / (uint32_t)w;
+        const int g = (int)(i - pix * (uint32_t)groups), ix = (int)(pix - row * (uint32_t)w);
+        const int b = (int)(row / (uint32_t)h), iy = (int)(row - (uint32_t)b * (uint32_t)h);
+        // windows o with o * s - p <= i <= o * s - p + k - 1
+        const int oy_lo = max(0, (iy + p - k + s) / s), oy_hi = min(ho - 1, (iy + p) / s);
+        const int ox_lo = max(0, (ix + p - k + s) / s), ox_hi = min(wo - 1, (ix + p) / s);
+        uint32_t even[4] = {0, 0, 0, 0}, odd[4] = {0, 0, 0, 0};
+        int nwin = 0;
+        for (int oy = oy_lo; oy <= oy_hi; ++oy)
+            for (int ox = ox_lo; ox <= ox_hi; ++ox) {
+                const size_t o = (((size_t)b * ho + oy) * wo + ox) * c + g * 16;
+                const int4 ev = __ldg(reinterpret_cast<const int4 *>(e + o));
+                const int4 av = __ldg(reinterpret_cast<const int4 *>(arg + o));
+                const uint32_t me = (uint32_t)((iy - (oy * s - p)) * k + (ix - (ox * s - p))) * 0x01010101u;
+                const uint32_t ew[4] = {(uint32_t)ev.x, (uint32_t)ev.y, (uint32_t)ev.z, (uint32_t)ev.w};
+                const uint32_t aw[4] = {(uint32_t)av.x, (uint32_t)av.y, (uint32_t)av.z, (uint32_t)av.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t hit = __vcmpeq4(aw[q], me);           // 0xff in the bytes this position won
+                    const uint32_t v = (ew[q] & hit) ^ 0x80808080u;      // code + 128 there, 128 elsewhere
+                    even[q] += v & 0x00ff00ffu;
+                    odd[q] += (v >> 8) & 0x00ff00ffu;
+                }
+                ++nwin;
+            }
+        int sum[16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            sum[4 * q + 0] = (int)(even[q] & 0xffffu) - 128 * nwin;
+            sum[4 * q + 1] = (int)(odd[q] & 0xffffu) - 128 * nwin;
+            sum[4 * q + 2] = (int)(even[q] >> 16) - 128 * nwin;
+            sum[4 * q + 3] = (int)(odd[q] >> 16) - 128 * nwin;
+        }
         if (kPass == 0) {
 #pragma unroll
-            for (int q = 0; q < 16; ++q) mx = max(mx, (uint32_t)abs(acc[threadIdx.x][q]));
+            for (int q = 0; q < 16; ++q) mx = max(mx, (uint32_t)abs(sum[q]));
         } else {
             int cd[16];
 #pragma unroll
-            for (int q = 0; q < 16; ++q) cd[q] = sq_code32(acc[threadIdx.x][q], t);
-            *reinterpret_cast<int4 *>(e_in + (((size_t)img * h + iy) * w + ix) * c + g * 16) =
+            for (int q = 0; q < 16; ++q) cd[q] = sq_code32(sum[q], t);
+            reinterpret_cast<int4 *>(e_in)[i] =
                 make_int4((int)pack4(cd[0], cd[1], cd[2], cd[3]), (int)pack4(cd[4], cd[5], cd[6], cd[7]),
                           (int)pack4(cd[8], cd[9], cd[10], cd[11]), (int)pack4(cd[12], cd[13], cd[14], cd[15]));
         }
@@ -575,15 +577,11 @@ cudaError_t launch_maxpool_bwd(const int8_t *e, const int32_t *e_exp, const uint
                                int p, int8_t *e_in, int32_t *e_in_exp, DeviceState *dev, int sm_count, cudaStream_t st,
                                const ReduceHook &hook)
 {
-    (void)sm_count;
     const int ho = (h + 2 * p - k) / s + 1, wo = (w + 2 * p - k) / s + 1;
-    const int tiles_x = (w + kPoolTile - 1) / kPoolTile, tiles_y = (h + kPoolTile - 1) / kPoolTile;
-    const unsigned blocks = (unsigned)((size_t)n * (c / 16) * tiles_x * tiles_y);
-    maxpool_bwd_kernel<0><<<blocks, kPoolTile * kPoolTile, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, tiles_x, tiles_y, e_in,
-                                                                  e_in_exp, dev);
+    const int blocks = blocks_for((size_t)n * h * w * (c / 16), sm_count, 32);
+    maxpool_bwd_kernel<0><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, dev);
     hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, st);
-    maxpool_bwd_kernel<1><<<blocks, kPoolTile * kPoolTile, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, tiles_x, tiles_y, e_in,
-                                                                  e_in_exp, dev);
+    maxpool_bwd_kernel<1><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, dev);
     return cudaGetLastError();
 }
 

@@ -1,0 +1,125 @@
+"""The glue entry points (eoq_aux_*) one by one against the oracle, element by element: pooling over several window
+geometries and ragged image sizes, the error join over exponent gaps that exercise the narrow path, the 64-bit path
+and the dropping rule, the float head bit for bit, and the error it hands back."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2105_13890_b200 import eoq, synth
+
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+def i32(v):
+    return G.dev(np.array([v], dtype=np.int32))
+
+
+POOLS = [  # n, h, w, c, k, stride, pad
+    (2, 12, 12, 16, 3, 2, 1),      # the ImageNet networks' pool
+    (3, 13, 11, 32, 3, 2, 1),      # odd sizes: the last window hangs over the border
+    (2, 8, 8, 48, 2, 2, 0),        # disjoint windows
+    (2, 9, 10, 16, 3, 1, 1),       # every position in nine windows
+    (1, 7, 7, 16, 5, 3, 2),
+    (5, 37, 41, 64, 3, 2, 1),      # several blocks, ragged tail
+]
+
+
+@pytest.mark.parametrize("n,h,w,c,k,s,p", POOLS)
+@pytest.mark.parametrize("ties", [False, True])
+def test_maxpool_forward_and_backward(n, h, w, c, k, s, p, ties):
+    hd = G.handle()
+    x = synth.relu_codes((n, h, w, c), 8100 + h, 0)
+    if ties:
+        x = (x // 32 * 32).astype(np.int8)      # few distinct values: most windows hold their maximum several times
+    y_o, idx = oracle.maxpool_fwd(x, k, s, p)
+    ho, wo = y_o.shape[1:3]
+    e = synth.normal_codes((n, ho, wo, c), 8100 + h, 1)
+    y, arg = G.zeros(y_o.shape, torch.int8), G.zeros(y_o.shape, torch.uint8)
+    eoq.eoq_aux_maxpool_fwd(hd, G.dev(x), n, h, w, c, k, s, p, y, arg)
+    ein, pin = G.zeros(x.shape, torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_aux_maxpool_bwd(hd, G.dev(e), i32(-12), arg, n, h, w, c, k, s, p, ein, pin)
+    torch.cuda.synchronize()
+    assert np.array_equal(G.host(y), y_o)
+    # the recorded position is the oracle's first maximum
+    a = G.host(arg).astype(np.int64)
+    b_, oy, ox, ch = np.meshgrid(np.arange(n), np.arange(ho), np.arange(wo), np.arange(c), indexing="ij")
+    flat = ((b_ * h + (oy * s - p + a // k)) * w + (ox * s - p + a % k)) * c + ch
+    assert np.array_equal(flat, idx)
+    S = oracle.maxpool_bwd(e, idx, x.shape)
+    codes, p_out, _ = oracle.sq_int(S, -12)
+    assert np.array_equal(G.host(ein), codes) and pin.item() == p_out
+    assert eoq.eoq_last_status(hd) == 0
+
+
+def test_maxpool_backward_of_a_zero_error_keeps_the_exponent():
+    hd = G.handle()
+    n, h, w, c = 1, 6, 6, 16
+    x = synth.relu_codes((n, h, w, c), 8200, 0)
+    y, arg = G.zeros((n, 3, 3, c), torch.int8), G.zeros((n, 3, 3, c), torch.uint8)
+    eoq.eoq_aux_maxpool_fwd(hd, G.dev(x), n, h, w, c, 3, 2, 1, y, arg)
+    ein, pin = G.empty((n, h, w, c), torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_aux_maxpool_bwd(hd, G.zeros((n, 3, 3, c), torch.int8), i32(-9), arg, n, h, w, c, 3, 2, 1, ein, pin)
+    torch.cuda.synchronize()
+    assert not G.host(ein).any() and pin.item() == -9
+    assert eoq.eoq_last_status(hd) == eoq.EOQ_DEV_SQ_ZERO
+    G.status_clear()
+
+
+@pytest.mark.parametrize("n,hw,c", [(2, 49, 512), (3, 64, 64), (1, 1, 16), (4, 300, 32)])
+def test_avgpool_sum(n, hw, c):
+    hd = G.handle()
+    x = synth.relu_codes((n, hw, 1, c), 8300 + hw, 0)
+    sums = G.zeros((n, c), torch.int32)
+    eoq.eoq_aux_avgpool_sum(hd, G.dev(x), n, hw, c, sums)
+    torch.cuda.synchronize()
+    assert np.array_equal(G.host(sums).astype(np.int64), oracle.avgpool_sum(x))
+
+
+@pytest.mark.parametrize("pa,pb", [(-12, -12), (-11, -14), (-14, -11), (-10, -33), (-5, -40), (-40, -5), (-20, -51), (-52, -20)])
+@pytest.mark.parametrize("gated", [False, True])
+def test_join(pa, pb, gated):
+    """Equal exponents, small gaps (32-bit path), gaps above 23 octaves (64-bit path) and above 31 (the smaller
+    operand is dropped), with and without the gate bits of operand b."""
+    hd = G.handle()
+    shape = (3, 9, 7, 48)                      # 9072 codes: whole 16-code groups, several blocks, a ragged tail
+    a = synth.normal_codes(shape, 8400, 0)
+    b = synth.normal_codes(shape, 8400, 1)
+    mask01 = (synth.relu_codes(shape, 8400, 2) > 0).astype(np.uint8) if gated else None
+    S, p = oracle.join(a, pa, b, pb, mask01)
+    codes, p_out, _ = oracle.sq_int(S, p)
+    out, pout, ssum = G.zeros(shape, torch.int8), G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+    eoq.eoq_aux_join(hd, G.dev(a), i32(pa), G.dev(b), i32(pb), G.dev(G.pack_mask(mask01)) if gated else None, a.size, out, pout, ssum)
+    torch.cuda.synchronize()
+    assert np.array_equal(G.host(out), codes) and pout.item() == p_out
+    assert ssum.item() == int(codes.astype(np.int64).sum())
+    assert eoq.eoq_last_status(hd) == 0
+
+
+@pytest.mark.parametrize("n,c,hw,classes", [(2, 64, 64, 10), (5, 512, 49, 1000), (33, 64, 64, 10), (64, 512, 49, 1000)])
+def test_float_head_bit_for_bit(n, c, hw, classes):
+    hd = G.handle()
+    sums = (synth.relu_codes((n, c), 8500 + n, 0).astype(np.int64) * hw) // 3
+    W = (synth.normal_f32((classes, c), 8500 + n, 1) / np.float32(np.sqrt(c))).astype(np.float32)
+    bias = (synth.normal_f32((classes,), 8500 + n, 2) * np.float32(0.01)).astype(np.float32)
+    labels = synth.labels(n, classes, 8500 + n, 3).astype(np.int32)
+    W_o, bias_o = W.copy(), bias.copy()
+    loss_o, dpooled_o, logits_o = oracle.head(sums, hw, W_o, bias_o, labels, 2.0 ** -6)
+    W_d, bias_d = G.dev(W), G.dev(bias)
+    loss, dpooled, logits = G.zeros(1, torch.float32), G.zeros((n, c), torch.float32), G.zeros((n, classes), torch.float32)
+    ws = G.zeros(eoq.eoq_aux_head_workspace_size(n, c, classes), torch.uint8)
+    eoq.eoq_aux_head(hd, G.dev(sums.astype(np.int32)), n, c, hw, classes, W_d, bias_d, G.dev(labels), 2.0 ** -6, loss, dpooled, logits, ws)
+    e, pe = G.zeros((n, hw, 1, c), torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_aux_head_error(hd, dpooled, n, c, hw, e, pe, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(G.host(logits), logits_o)
+    assert np.array_equal(G.host(dpooled), dpooled_o)
+    assert np.array_equal(G.host(W_d), W_o) and np.array_equal(G.host(bias_d), bias_o)
+    assert loss.item() == pytest.approx(loss_o, rel=1e-6)
+    # the error handed back: SQ of dpooled / hw, the same code at every position of a (sample, channel)
+    codes, p_e, _ = oracle.quantize_f32(oracle.MODE_SQ, (dpooled_o / np.float32(hw)).astype(np.float32))
+    got = G.host(e).reshape(n, hw, c)
+    assert pe.item() == p_e and all(np.array_equal(got[:, i, :], codes) for i in (0, hw // 2, hw - 1))
+    assert eoq.eoq_last_status(hd) == 0
