@@ -288,6 +288,17 @@ def run_gpu(args):
     if not args.eager:
         launches = step.launches_per_step * args.steps  # graph replays do not pass through the host-side counter
     status |= step.status()
+    if args.step_only:
+        # for a launch list under a profiler: the steps above are all that runs (no end-to-end, per-kernel or per-kind pass)
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "step_only": True, "ms_per_step": ms / args.steps, "steps": args.steps,
+                              "warmup": args.warmup, "gpu_launches": int(launches), "device_status": int(status),
+                              "config": {"workload": wl.name}}), flush=True)
+        if sampler:
+            sampler.stop()
+        eoq.eoq_destroy(handle)
+        ranks.finish()
+        return
 
     # ---- end to end: host image in (pinned), results out, every step
     host_img = torch.from_numpy(step.host_image(12345)).pin_memory()
@@ -541,6 +552,8 @@ def main():
     ap.add_argument("--probe", default=None, choices=["mma_i8"], help="measure the INT8 tensor-pipe figures and exit")
     ap.add_argument("--probe-seconds", type=float, default=2.0, help="length of each sustained probe loop")
     ap.add_argument("--int8-peaks", default=None, help="JSON printed by --probe, to report fractions of those figures too")
+    ap.add_argument("--step-only", action="store_true",
+                    help="run the warm-up and timed steps and nothing else (launch lists under a profiler)")
     ap.add_argument("--dry-run", action="store_true", help="rank plumbing only, on CPU with gloo (tests)")
     args = ap.parse_args()
     if args.warmup < 3:

@@ -114,16 +114,17 @@ __device__ __forceinline__ const int32_t *stage_b1_table(const IgemmParams &p, i
 
 // `tb`: this pixel's 16 b1 terms in shared memory (already times b1), or null; then `tg` points at the 16 weight
 // sums in global memory (or is null when the layer has no b1 term).  `sc`: the 16 shortcut codes (zero without one).
-// `acc1` holds the tile's second partial sums when `two` is set; kRelu = a ReLU follows.
-template <bool kShift7, bool kRelu>
+// `acc1` holds the tile's second partial sums when kTwo is set; kRelu = a ReLU follows.
+template <bool kShift7, bool kRelu, bool kTwo>
 __device__ __forceinline__ void forward_16(const IgemmParams &p, const FwdScalars &fs, const uint32_t (&acc)[32],
-                                           const uint32_t (&acc1)[32], bool two, size_t off, const int32_t *tb,
+                                           const uint32_t (&acc1)[32], size_t off, const int32_t *tb,
                                            const int32_t *tg, const int4 &sc, int shift)
 {
     int32_t a[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) a[i] = (int32_t)acc[i];
-    if (two && (!kShift7 || p.acc_out)) {
+    bool two = kTwo;
+    if (kTwo && (!kShift7 || p.acc_out)) {
         // paths that need the whole sum as a value (the dump, the generic shift) merge the partial sums here;
         // the common path below merges them inside its first clamp
 #pragma unroll

@@ -280,13 +280,22 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                 }
                 if (valid && col < p.N) {
                     if (fwd) {
-                        const bool two = nacc == 2;
                         if (shift == 7) {
-                            if (p.relu) forward_16<true, true>(p, fs, r, r2, two, off, tb, tg, sc, 7);
-                            else forward_16<true, false>(p, fs, r, r2, two, off, tb, tg, sc, 7);
+                            if (nacc == 2) {
+                                if (p.relu) forward_16<true, true, true>(p, fs, r, r2, off, tb, tg, sc, 7);
+                                else forward_16<true, false, true>(p, fs, r, r2, off, tb, tg, sc, 7);
+                            } else {
+                                if (p.relu) forward_16<true, true, false>(p, fs, r, r2, off, tb, tg, sc, 7);
+                                else forward_16<true, false, false>(p, fs, r, r2, off, tb, tg, sc, 7);
+                            }
                         } else {
-                            if (p.relu) forward_16<false, true>(p, fs, r, r2, two, off, tb, tg, sc, shift);
-                            else forward_16<false, false>(p, fs, r, r2, two, off, tb, tg, sc, shift);
+                            // the generic shift (first layer behind the input quantizer) merges the partial sums itself
+                            if (nacc == 2) {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) r[i] += r2[i];
+                            }
+                            if (p.relu) forward_16<false, true, false>(p, fs, r, r2, off, tb, tg, sc, shift);
+                            else forward_16<false, false, false>(p, fs, r, r2, off, tb, tg, sc, shift);
                         }
                     } else {
                         mx = max(mx, dgrad_16(p, r, off));

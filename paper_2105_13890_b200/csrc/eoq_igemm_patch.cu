@@ -319,8 +319,13 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                 }
                 if (valid && col < p.N) {
                     if (fwd) {
-                        if (p.relu) forward_16<true, true>(p, fs, r, r2, nacc == 2, off, tb, tg, sc, 7);
-                        else forward_16<true, false>(p, fs, r, r2, nacc == 2, off, tb, tg, sc, 7);
+                        if (nacc == 2) {
+                            if (p.relu) forward_16<true, true, true>(p, fs, r, r2, off, tb, tg, sc, 7);
+                            else forward_16<true, false, true>(p, fs, r, r2, off, tb, tg, sc, 7);
+                        } else {
+                            if (p.relu) forward_16<true, true, false>(p, fs, r, r2, off, tb, tg, sc, 7);
+                            else forward_16<true, false, false>(p, fs, r, r2, off, tb, tg, sc, 7);
+                        }
                     }
                     else mx = max(mx, dgrad_16(p, r, off));
                 }
