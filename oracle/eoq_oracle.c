@@ -604,3 +604,113 @@ int eoq_o_update_k(int32_t *theta, int8_t *w8, const int8_t *g, int p_g, size_t 
     __builtin_free(u);
     return z;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Batch normalisation behind the same convolution: the comparison the paper draws in its efficiency
+ * discussion (Sec. 5.3, "efficiency comparison of EOQ and traditional BN": the scale-and-bias of
+ * the Fixup block against the mean / standard-deviation normalisation of a mini-batch).  Not part
+ * of the EOQ method; it exists so that the cost of what EOQ removes can be measured beside it.
+ *
+ * Definition (training-mode batch normalisation per channel over all n*h*w positions of the batch):
+ *   a      = A * 2^p                     the convolution output, exact integers A at exponent p
+ *   mean   = sum(a) / P,  var = sum(a^2) / P - mean^2      (biased variance)
+ *   y      = gamma * (a - mean) / sqrt(var + eps) + beta,  x5 = Q_a2(relu(y)),  mask = [y > 0]
+ * Statistics are exact: S1 = sum A (64-bit), S2 = sum A^2 (128-bit), V = P * S2 - S1^2 (128-bit, >= 0).
+ * From there double precision, every operation rounded once, in this order:
+ *   mu = (double)S1 / P;  var_a = (hi(V) * 2^64 + lo(V)) / ((double)P * P)   (in units of A);
+ *   inv = 1 / sqrt(var_a * 4^p + eps);  k = gamma * inv;  scale = (float)(k * 2^p);
+ *   shift = (float)(beta - (k * 2^p) * mu);
+ * then one fused multiply-add per element in single precision: y = fma((float)A, scale, shift), and
+ * x5 = min(rint(y * 128), 127) for y > 0, else 0.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    double mu;      /* mean in units of A */
+    double inv;     /* 1 / sqrt(var + eps), value units */
+    float scale, shift;
+} eoq_o_bn_channel_t;
+
+static double u128_to_double(unsigned __int128 v)
+{
+    double hi = (double)(uint64_t)(v >> 64), lo = (double)(uint64_t)v;
+    return hi * 18446744073709551616.0 + lo;
+}
+
+void eoq_o_bn_forward(const int64_t *A, int p, size_t P, int c, const float *gamma, const float *beta, float eps,
+                      int8_t *x5, uint8_t *mask01, float *y_out, eoq_o_bn_channel_t *ch)
+{
+    for (int k = 0; k < c; k++) {
+        int64_t s1 = 0;
+        unsigned __int128 s2 = 0;
+        for (size_t i = 0; i < P; i++) {
+            int64_t a = A[i * c + k];
+            s1 += a;
+            s2 += (unsigned __int128)((__int128)a * a);
+        }
+        unsigned __int128 V = (unsigned __int128)P * s2 - (unsigned __int128)((__int128)s1 * s1);
+        double Pd = (double)P;
+        double mu = (double)s1 / Pd;
+        double var_a = u128_to_double(V) / (Pd * Pd);
+        double var_v = ldexp(var_a, 2 * p);
+        double inv = 1.0 / sqrt(var_v + (double)eps);
+        double kk = (double)gamma[k] * inv;
+        double ks = ldexp(kk, p);
+        ch[k].mu = mu;
+        ch[k].inv = inv;
+        ch[k].scale = (float)ks;
+        ch[k].shift = (float)((double)beta[k] - ks * mu);
+    }
+    for (size_t i = 0; i < P; i++)
+        for (int k = 0; k < c; k++) {
+            float y = fmaf((float)A[i * c + k], ch[k].scale, ch[k].shift);
+            if (y_out) y_out[i * c + k] = y;
+            int pos = y > 0.0f;
+            float r = rintf(y * 128.0f);
+            x5[i * c + k] = (int8_t)(pos ? (r > 127.0f ? 127 : (int)r) : 0);
+            if (mask01) mask01[i * c + k] = (uint8_t)pos;
+        }
+}
+
+/*
+ * Backward of the same normalisation (e: error codes at exponent p_e arriving at x5; the clamp of Q_a2 is
+ * passed straight through as everywhere else, so dy = e * mask):
+ *   dbeta = sum(dy),  dgamma = sum(dy * xhat),  xhat = (a - mean) * inv
+ *   da    = gamma * inv * (dy - mean(dy) - xhat * mean(dy * xhat))
+ * Exact sums D1 = sum(E * mask), D2 = sum(E * mask * A) (64-bit), then in double, in this order:
+ *   cov = (double)D2 - mu * (double)D1;  g2 = (inv * 2^p) * cov * 2^pe   (= dgamma);  g1 = (double)D1 * 2^pe (= dbeta);
+ *   k = gamma * inv;  ca = (float)(k * 2^pe);  m2 = g2 / P;  cb_d = -(k * m2) * (inv * 2^p);  cb = (float)cb_d;
+ *   cc = (float)(-(k * (g1 / P)) - cb_d * mu);
+ * and per element in single precision da = fma(ca, (float)(E * mask), fma(cb, (float)A, cc)).
+ * The caller quantizes da with Q_e (SQ) like every other error tensor.
+ */
+void eoq_o_bn_backward(const int8_t *E, int p_e, const uint8_t *mask01, const int64_t *A, int p, size_t P, int c,
+                       const float *gamma, const eoq_o_bn_channel_t *ch, float *da, float *dgamma, float *dbeta)
+{
+    float *ca = (float *)__builtin_malloc(sizeof(float) * 3 * (size_t)c), *cb = ca + c, *cc = cb + c;
+    for (int k = 0; k < c; k++) {
+        int64_t d1 = 0, d2 = 0;
+        for (size_t i = 0; i < P; i++) {
+            int64_t dy = mask01[i * c + k] ? (int64_t)E[i * c + k] : 0;
+            d1 += dy;
+            d2 += dy * A[i * c + k];
+        }
+        double Pd = (double)P;
+        double cov = (double)d2 - ch[k].mu * (double)d1;
+        double ip = ldexp(ch[k].inv, p);
+        double g2 = ldexp(ip * cov, p_e);
+        double g1 = ldexp((double)d1, p_e);
+        double kk = (double)gamma[k] * ch[k].inv;
+        double m2 = g2 / Pd;
+        double cb_d = -(kk * m2) * ip;
+        ca[k] = (float)ldexp(kk, p_e);
+        cb[k] = (float)cb_d;
+        cc[k] = (float)(-(kk * (g1 / Pd)) - cb_d * ch[k].mu);
+        dgamma[k] = (float)g2;
+        dbeta[k] = (float)g1;
+    }
+    for (size_t i = 0; i < P; i++)
+        for (int k = 0; k < c; k++) {
+            float dy = mask01[i * c + k] ? (float)E[i * c + k] : 0.0f;
+            da[i * c + k] = fmaf(ca[k], dy, fmaf(cb[k], (float)A[i * c + k], cc[k]));
+        }
+    __builtin_free(ca);
+}

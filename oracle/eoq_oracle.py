@@ -354,3 +354,42 @@ def update_k(theta, g, p_g: int, lr_mant: int, lr_exp: int, k_u: int, k_m: int, 
                             C.c_int(k_u), C.c_int(k_m), C.c_int(1 if stochastic else 0), C.c_uint64(seed), C.c_uint64(step),
                             C.c_uint64(tensor_id), C.byref(p_u))
     return th.reshape(np.shape(theta)), w8.reshape(np.shape(theta)), p_u.value, int(z)
+
+
+# --------------------------------------------------------------------------- batch normalisation (comparison, Sec. 5.3)
+
+BN_CHANNEL = np.dtype([("mu", "f8"), ("inv", "f8"), ("scale", "f4"), ("shift", "f4")])
+
+
+def bn_forward(A, p: int, gamma, beta, eps: float = 1e-5):
+    """Training-mode batch normalisation of a convolution output (exact integers A [n,h,w,c] at exponent p) per
+    channel over the whole batch, then ReLU and Q_a2.
+    -> dict(x5 int8 codes, mask 0/1, y fp32 before the ReLU, ch = per-channel constants for the backward pass)."""
+    A = np.ascontiguousarray(A, dtype=np.int64)
+    c = A.shape[-1]
+    P = A.size // c
+    gamma = np.ascontiguousarray(gamma, dtype=np.float32)
+    beta = np.ascontiguousarray(beta, dtype=np.float32)
+    x5 = np.empty(A.shape, dtype=np.int8)
+    mask = np.empty(A.shape, dtype=np.uint8)
+    y = np.empty(A.shape, dtype=np.float32)
+    ch = np.zeros(c, dtype=BN_CHANNEL)
+    _L().eoq_o_bn_forward(_p(A), C.c_int(p), C.c_size_t(P), C.c_int(c), _p(gamma), _p(beta), C.c_float(eps), _p(x5), _p(mask),
+                          _p(y), _p(ch))
+    return {"x5": x5, "mask": mask, "y": y, "ch": ch}
+
+
+def bn_backward(E, p_e: int, mask01, A, p: int, gamma, ch):
+    """Backward of bn_forward for error codes E at exponent p_e -> (da fp32, dgamma fp32 [c], dbeta fp32 [c])."""
+    E = _i8(E)
+    A = np.ascontiguousarray(A, dtype=np.int64)
+    mask01 = np.ascontiguousarray(mask01, dtype=np.uint8)
+    c = A.shape[-1]
+    P = A.size // c
+    gamma = np.ascontiguousarray(gamma, dtype=np.float32)
+    da = np.empty(A.shape, dtype=np.float32)
+    dgamma = np.empty(c, dtype=np.float32)
+    dbeta = np.empty(c, dtype=np.float32)
+    _L().eoq_o_bn_backward(_p(E), C.c_int(p_e), _p(mask01), _p(A), C.c_int(p), C.c_size_t(P), C.c_int(c), _p(gamma), _p(ch),
+                           _p(da), _p(dgamma), _p(dbeta))
+    return da, dgamma, dbeta
