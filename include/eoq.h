@@ -317,6 +317,30 @@ EOQ_API int eoq_aux_head(eoq_handle_t handle, const int32_t *sums, int n, int c,
 EOQ_API int eoq_aux_head_error(eoq_handle_t handle, const float *dpooled, int n, int c, int hw, int8_t *e, int32_t *e_exp,
                        void *workspace, size_t workspace_bytes, void *stream);
 /*
+ * Comparison case, not on the EOQ path (Sec. 5.3 sets the Fixup scale and bias against "traditional BN"): training-
+ * mode batch normalisation of a convolution output, per channel over all `pixels` = n*ho*wo positions of the batch.
+ *   acc      [pixels][c] exact int32 sums of the convolution (the acc_out of eoq_conv_fwd) at exponent acc_exp
+ *            (-14 for int8 codes at -7 times int8 weights at -7); c a multiple of 16, at most 1024.
+ *   gamma, beta  fp32 [c] (device).  eps added to the biased variance.
+ * eoq_bn_fwd: y = gamma (a - mean) / sqrt(var + eps) + beta; x5 = Q_a2(relu(y)) int8 codes at exponent -7;
+ *   relu_mask bit = [y > 0].  The statistics are exact integer sums; the per-channel constants are formed in double
+ *   precision and each element takes one fp32 fused multiply-add, so the result is reproducible bit for bit.
+ * eoq_bn_bwd: for error codes e at exponent *e_exp arriving at x5 (same shape), dy = e * mask:
+ *   dgamma, dbeta fp32 [c]; da fp32 [pixels][c] = the error with respect to the convolution output (quantize it with
+ *   eoq_quantize(EOQ_SQ) to obtain the int8 error the dgrad and wgrad passes take).  Must follow eoq_bn_fwd on the
+ *   same workspace (it reads the statistics left there).
+ * workspace: eoq_bn_workspace_size(c) bytes, 256-byte aligned, owned by the caller.
+ * Errors: EOQ_ERR_BAD_ARG (null pointer, pixels == 0), EOQ_ERR_ALIGNMENT (c % 16, unaligned pointers),
+ * EOQ_ERR_UNSUPPORTED (c > 1024), EOQ_ERR_WORKSPACE.
+ */
+EOQ_API int eoq_bn_workspace_size(int c, size_t *bytes);
+EOQ_API int eoq_bn_fwd(eoq_handle_t handle, const int32_t *acc, int acc_exp, size_t pixels, int c, const float *gamma,
+               const float *beta, float eps, int8_t *x5, uint8_t *relu_mask, void *workspace, size_t workspace_bytes,
+               void *stream);
+EOQ_API int eoq_bn_bwd(eoq_handle_t handle, const int8_t *e, const int32_t *e_exp, const uint8_t *relu_mask, const int32_t *acc,
+               int acc_exp, size_t pixels, int c, const float *gamma, void *workspace, size_t workspace_bytes, float *da,
+               float *dgamma, float *dbeta, void *stream);
+/*
  * Update of `num` scalar parameters (gamma, b1, b2; Sec. 3.2.3 applied to a single value): g = Q_g({total}) with
  * total the exact sum behind the gradient at exponent *total_exp[i] + exp_bias[i]; u = Q_u(lr g);
  * theta <- Q(theta - u) saturated to 16 bits, rounding as in eoq_update (the hash counter of scalar i is
@@ -345,7 +369,7 @@ EOQ_API int eoq_last_status(eoq_handle_t handle, void *stream, unsigned *bits);
 #define EOQ_PROF_DGRAD_AUX 4     /* Q_e phase 2; weight transpose (only layers with fewer than 32 output channels) */
 #define EOQ_PROF_WGRAD_AUX 5     /* slice sum + b1 term + Q_g behind the weight-gradient GEMM (and the memset in front of it) */
 #define EOQ_PROF_FWD_AUX 6       /* b1 weight table, weight row padding (eoq_weight_prep, or per call without it) */
-#define EOQ_PROF_OTHER 7         /* eoq_quantize */
+#define EOQ_PROF_OTHER 7         /* eoq_quantize, eoq_bn_fwd, eoq_bn_bwd */
 #define EOQ_PROF_UPDATE 8        /* eoq_update */
 #define EOQ_PROF_INPUT_Q 9       /* eoq_quantize_image */
 #define EOQ_PROF_WGRAD_TAPS 10   /* b1 error sums of the weight gradient */

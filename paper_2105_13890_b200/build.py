@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libeoq.so")
-SOURCES = ["eoq_api.cu", "eoq_igemm.cu", "eoq_igemm_patch.cu", "eoq_wgrad_patch.cu", "eoq_wgrad.cu", "eoq_elementwise.cu", "eoq_static.cu", "eoq_probe.cu", "eoq_aux.cu"]
+SOURCES = ["eoq_api.cu", "eoq_igemm.cu", "eoq_igemm_patch.cu", "eoq_wgrad_patch.cu", "eoq_wgrad.cu", "eoq_elementwise.cu", "eoq_static.cu", "eoq_probe.cu", "eoq_aux.cu", "eoq_bn.cu"]
 HEADERS = ["eoq_internal.h", "eoq_device.cuh", "eoq_epilogue.cuh", os.path.join(ROOT, "include", "eoq.h")]
 
 

@@ -1506,6 +1506,55 @@ extern "C" int eoq_aux_maxpool_bwd(eoq_handle_t handle, const int8_t *e, const i
     return record(h, launch_maxpool_bwd(e, e_exp, arg, n, hh, ww, c, k, stride, pad, e_in, e_in_exp, h->dev, h->sm_count, s, h->hook));
 }
 
+extern "C" int eoq_bn_workspace_size(int c, size_t *bytes)
+{
+    if (!bytes || c <= 0) return EOQ_ERR_BAD_ARG;
+    *bytes = (sizeof(BnChannel) * (size_t)c + 255) & ~(size_t)255;
+    return EOQ_OK;
+}
+
+static int bn_check(Handle *h, size_t pixels, int c, const void *ws, size_t ws_bytes)
+{
+    if (!h || !ws || pixels == 0 || c <= 0) return EOQ_ERR_BAD_ARG;
+    if (c % 16 || !aligned16(ws)) return EOQ_ERR_ALIGNMENT;
+    if (c > 1024 || pixels > 0x7fffffffull) return EOQ_ERR_UNSUPPORTED;
+    if (ws_bytes < sizeof(BnChannel) * (size_t)c) return EOQ_ERR_WORKSPACE;
+    return EOQ_OK;
+}
+
+extern "C" int eoq_bn_fwd(eoq_handle_t handle, const int32_t *acc, int acc_exp, size_t pixels, int c, const float *gamma,
+                          const float *beta, float eps, int8_t *x5, uint8_t *relu_mask, void *workspace, size_t workspace_bytes,
+                          void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!acc || !gamma || !beta || !x5 || !relu_mask || !(eps >= 0.0f) || acc_exp < -60 || acc_exp > 60) return EOQ_ERR_BAD_ARG;
+    const int chk = bn_check(h, pixels, c, workspace, workspace_bytes);
+    if (chk != EOQ_OK) return chk;
+    if (!aligned16(acc) || !aligned16(x5) || (reinterpret_cast<uintptr_t>(relu_mask) & 1)) return EOQ_ERR_ALIGNMENT;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 3);
+    ProfScope prof(h, EOQ_PROF_OTHER, s);
+    return record(h, launch_bn_fwd(acc, acc_exp, pixels, c, gamma, beta, eps, x5, relu_mask, reinterpret_cast<BnChannel *>(workspace),
+                                   h->sm_count, s));
+}
+
+extern "C" int eoq_bn_bwd(eoq_handle_t handle, const int8_t *e, const int32_t *e_exp, const uint8_t *relu_mask, const int32_t *acc,
+                          int acc_exp, size_t pixels, int c, const float *gamma, void *workspace, size_t workspace_bytes, float *da,
+                          float *dgamma, float *dbeta, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!e || !e_exp || !relu_mask || !acc || !gamma || !da || !dgamma || !dbeta || acc_exp < -60 || acc_exp > 60)
+        return EOQ_ERR_BAD_ARG;
+    const int chk = bn_check(h, pixels, c, workspace, workspace_bytes);
+    if (chk != EOQ_OK) return chk;
+    if (!aligned16(acc) || !aligned16(e) || !aligned16(da) || (reinterpret_cast<uintptr_t>(relu_mask) & 1)) return EOQ_ERR_ALIGNMENT;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 3);
+    ProfScope prof(h, EOQ_PROF_OTHER, s);
+    return record(h, launch_bn_bwd(e, e_exp, relu_mask, acc, acc_exp, pixels, c, gamma, reinterpret_cast<BnChannel *>(workspace), da,
+                                   dgamma, dbeta, h->sm_count, s));
+}
+
 extern "C" int eoq_aux_avgpool_sum(eoq_handle_t handle, const int8_t *x, int n, int hw, int c, int32_t *sums, void *stream)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);

@@ -329,6 +329,20 @@ struct ScalarBatch {
     ScalarItem item[kScalarChunk];
     int num;
 };
+// Batch normalisation behind the convolution (comparison case, eoq_bn.cu): per-channel record in the workspace
+struct BnChannel {
+    long long s1, shh, shl, sll;   // sum of A; sum of A^2 in three parts (A = h * 2^16 + l): h*h, h*l, l*l
+    long long d1, d2;              // backward: sum of E * mask, sum of E * mask * A
+    double mu, inv;                // mean in units of A; 1 / sqrt(var + eps)
+    float scale, shift;            // y = fma((float)A, scale, shift)
+    float ca, cb, cc, pad;         // da = fma(ca, E * mask, fma(cb, (float)A, cc))
+};
+cudaError_t launch_bn_fwd(const int32_t *acc, int p, size_t pixels, int c, const float *gamma, const float *beta, float eps,
+                          int8_t *x5, uint8_t *relu_mask, BnChannel *ch, int sm_count, cudaStream_t st);
+cudaError_t launch_bn_bwd(const int8_t *e, const int32_t *e_exp, const uint8_t *relu_mask, const int32_t *acc, int p, size_t pixels,
+                          int c, const float *gamma, BnChannel *ch, float *da, float *dgamma, float *dbeta, int sm_count,
+                          cudaStream_t st);
+
 cudaError_t launch_scalar_update(const ScalarBatch &b, int32_t lr_mant, int32_t lr_exp, int stochastic, uint64_t seed,
                                  const unsigned long long *step_dev, uint64_t step, cudaStream_t st);
 

@@ -27,7 +27,7 @@ EXPORTS = [
     "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count", "eoq_set_gemm_ctas",
     "eoq_conv_dgrad_static", "eoq_conv_fwd_dev", "eoq_weight_prep_size", "eoq_weight_prep", "eoq_conv_wgrad_dev",
     "eoq_err_prescale_dev", "eoq_update_dev", "eoq_describe_plan", "eoq_debug_force_wait_timeout", "eoq_probe_mma_i8", "eoq_profile_gemm_only", "eoq_aux_maxpool_fwd", "eoq_aux_maxpool_bwd",
-    "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide", "eoq_set_reduce_hook",
+    "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide", "eoq_set_reduce_hook", "eoq_bn_workspace_size", "eoq_bn_fwd", "eoq_bn_bwd",
 ]
 EOQ_STATIC_SCRATCH_BYTES = 16 << 20
 EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
@@ -116,6 +116,9 @@ def lib() -> C.CDLL:
         L.eoq_aux_head_error.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, sz, vp]
         L.eoq_aux_scalar_update.argtypes = [vp, ci, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(ci),
                                             C.POINTER(ci), C.POINTER(vp), i32, i32, ci, u64, vp, vp]
+        L.eoq_bn_workspace_size.argtypes = [ci, C.POINTER(sz)]
+        L.eoq_bn_fwd.argtypes = [vp, vp, ci, sz, ci, vp, vp, C.c_float, vp, vp, vp, sz, vp]
+        L.eoq_bn_bwd.argtypes = [vp, vp, vp, vp, vp, ci, sz, ci, vp, vp, sz, vp, vp, vp, vp]
         L.eoq_profile_gemm_only.argtypes = [vp, C.c_int]
         L.eoq_probe_mma_i8.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
         L.eoq_status_string.argtypes = [C.c_int]
@@ -384,6 +387,23 @@ def eoq_aux_maxpool_fwd(handle, x, n, h, w, c, k, stride, pad, y, arg, stream=No
 def eoq_aux_maxpool_bwd(handle, e, e_exp, arg, n, h, w, c, k, stride, pad, e_in, e_in_exp, stream=None) -> None:
     _check(lib().eoq_aux_maxpool_bwd(handle, _ptr(e), _ptr(e_exp), _ptr(arg), n, h, w, c, k, stride, pad, _ptr(e_in),
                                      _ptr(e_in_exp), _stream(stream)), "eoq_aux_maxpool_bwd")
+
+
+def eoq_bn_workspace_size(c) -> int:
+    out = C.c_size_t(0)
+    _check(lib().eoq_bn_workspace_size(c, C.byref(out)), "eoq_bn_workspace_size")
+    return out.value
+
+
+def eoq_bn_fwd(handle, acc, acc_exp, pixels, c, gamma, beta, eps, x5, relu_mask, workspace, stream=None) -> None:
+    _check(lib().eoq_bn_fwd(handle, _ptr(acc), acc_exp, int(pixels), c, _ptr(gamma), _ptr(beta), eps, _ptr(x5), _ptr(relu_mask),
+                            _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)), "eoq_bn_fwd")
+
+
+def eoq_bn_bwd(handle, e, e_exp, relu_mask, acc, acc_exp, pixels, c, gamma, workspace, da, dgamma, dbeta, stream=None) -> None:
+    _check(lib().eoq_bn_bwd(handle, _ptr(e), _ptr(e_exp), _ptr(relu_mask), _ptr(acc), acc_exp, int(pixels), c, _ptr(gamma),
+                            _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(da), _ptr(dgamma), _ptr(dbeta),
+                            _stream(stream)), "eoq_bn_bwd")
 
 
 def eoq_aux_avgpool_sum(handle, x, n, hw, c, sums, stream=None) -> None:
