@@ -502,6 +502,102 @@ def run_probe(args):
     print(json.dumps(out), flush=True)
 
 
+# ----------------------------------------------------------------------------------------------- BN comparison
+
+def run_bn_compare(args):
+    """--probe bn_vs_fixup: the paper's second claim restated on this device (Sec. 5.3): on the same int8 convolutions of
+    Fixup ResNet-18, the fused scale-and-bias epilogue of EOQ against training-mode batch normalisation behind the
+    convolution (eoq_bn_fwd / eoq_bn_bwd: two extra passes over the exact sums forward, two more backward, then Q_e).
+    Each variant is replayed from a CUDA graph of ten copies of its calls; times are per call."""
+    import torch
+
+    from paper_2105_13890_b200 import eoq, workloads
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --probe needs a CUDA device")
+    dev = "cuda:0"
+    h = eoq.eoq_create(0)
+    wl = workloads.get("resnet18", args.batch)
+    picks = [l for l in wl.layers if l.name in ("layer1.0.a", "layer2.1.a", "layer3.1.a", "layer4.1.a")]
+    g = torch.Generator(device=dev)
+    g.manual_seed(4242)
+
+    def time_calls(fn, copies=10, replays=5):
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            fn()
+            fn()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            for _ in range(copies):
+                fn()
+        torch.cuda.synchronize()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(replays):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (copies * replays) * 1e3   # microseconds per call
+
+    rows = []
+    for l in picks:
+        d = eoq.conv_desc(l.n, l.h, l.w, l.c_in, l.c_out, l.k, l.k, l.stride, l.pad)
+        shape = (l.n, l.ho, l.wo, l.c_out)
+        n_out = l.n * l.ho * l.wo * l.c_out
+        x0 = torch.randint(0, 100, (l.n, l.h, l.w, l.c_in), dtype=torch.int8, device=dev, generator=g)
+        x0 = torch.where(torch.rand(x0.shape, device=dev, generator=g) < 0.5, torch.zeros_like(x0), x0)
+        w = torch.randint(-6, 7, (l.c_out, l.k, l.k, l.c_in), dtype=torch.int8, device=dev, generator=g)
+        e0 = torch.randint(-90, 91, shape, dtype=torch.int8, device=dev, generator=g)
+        e0_exp = torch.full((1,), -12, dtype=torch.int32, device=dev)
+        x5, x2 = torch.zeros(shape, dtype=torch.int8, device=dev), torch.zeros(shape, dtype=torch.int16, device=dev)
+        mask = torch.zeros((n_out + 7) // 8, dtype=torch.uint8, device=dev)
+        acc = torch.zeros(shape, dtype=torch.int32, device=dev)
+        ws = torch.empty(max(eoq.eoq_workspace_size(d, eoq.EOQ_PASS_FWD), 256), dtype=torch.uint8, device=dev)
+        e3, e3_exp = torch.zeros(shape, dtype=torch.int8, device=dev), torch.zeros(1, dtype=torch.int32, device=dev)
+        s1, s2 = torch.zeros(1, dtype=torch.int64, device=dev), torch.zeros(1, dtype=torch.int64, device=dev)
+        bn_ws = torch.zeros(eoq.eoq_bn_workspace_size(l.c_out), dtype=torch.uint8, device=dev)
+        gamma_f = torch.ones(l.c_out, dtype=torch.float32, device=dev)
+        beta_f = torch.zeros(l.c_out, dtype=torch.float32, device=dev)
+        da = torch.zeros(shape, dtype=torch.float32, device=dev)
+        dg, db = torch.zeros(l.c_out, dtype=torch.float32, device=dev), torch.zeros(l.c_out, dtype=torch.float32, device=dev)
+        pixels = l.n * l.ho * l.wo
+
+        def fwd_eoq():
+            eoq.eoq_conv_fwd(h, d, x0, None, 0, w, 118, 3, None, True, x5, x2, mask, None, ws)
+
+        def fwd_conv_dump():
+            eoq.eoq_conv_fwd(h, d, x0, None, 0, w, 118, 3, None, True, x5, x2, mask, acc, ws)
+
+        def fwd_bn():
+            eoq.eoq_bn_fwd(h, acc, -14, pixels, l.c_out, gamma_f, beta_f, 1e-5, x5, mask, bn_ws)
+
+        def bwd_eoq():
+            eoq.eoq_err_prescale(h, e0, e0_exp, mask, x2, n_out, 118, e3, e3_exp, s1, s2)
+
+        def bwd_bn():
+            eoq.eoq_bn_bwd(h, e0, e0_exp, mask, acc, -14, pixels, l.c_out, gamma_f, bn_ws, da, dg, db)
+            eoq.eoq_quantize(h, eoq.EOQ_SQ, da, True, None, n_out, e3, e3_exp)
+
+        t = {"fwd_eoq_conv_fused_us": time_calls(fwd_eoq), "fwd_conv_with_sum_dump_us": time_calls(fwd_conv_dump),
+             "fwd_bn_passes_us": time_calls(fwd_bn), "bwd_eoq_error_head_us": time_calls(bwd_eoq),
+             "bwd_bn_passes_and_Qe_us": time_calls(bwd_bn)}
+        # BN forward = convolution that writes its exact sums + the BN passes; the dump run here also computes the fused
+        # epilogue, so the lower figure replaces it by the fused convolution's own time
+        t["fwd_bn_total_us"] = [t["fwd_eoq_conv_fused_us"] + t["fwd_bn_passes_us"], t["fwd_conv_with_sum_dump_us"] + t["fwd_bn_passes_us"]]
+        t["fwd_slowdown_with_bn"] = [x / t["fwd_eoq_conv_fused_us"] for x in t["fwd_bn_total_us"]]
+        t["bwd_slowdown_with_bn"] = t["bwd_bn_passes_and_Qe_us"] / t["bwd_eoq_error_head_us"]
+        t["layer"] = f"{l.name} {l.h}x{l.w} {l.c_in}->{l.c_out} k{l.k} batch {l.n}"
+        rows.append(t)
+    assert eoq.eoq_last_status(h) & ~eoq.EOQ_DEV_SQ_ZERO == 0
+    eoq.eoq_destroy(h)
+    print(json.dumps({"probe": "bn_vs_fixup", "unit": "us per call (graph replay)", "layers": rows}), flush=True)
+
+
 # ----------------------------------------------------------------------------------------------- launcher
 
 def launch_ranks(args, argv):
@@ -549,7 +645,8 @@ def main():
     ap.add_argument("--eager", action="store_true", help="launch call by call on one stream instead of replaying a CUDA graph")
     ap.add_argument("--independent", action="store_true", help="time the layer units on independent synthetic tensors (no glue)")
     ap.add_argument("--stochastic", action="store_true", help="stochastic rounding in the update (an extension; default: nearest even)")
-    ap.add_argument("--probe", default=None, choices=["mma_i8"], help="measure the INT8 tensor-pipe figures and exit")
+    ap.add_argument("--probe", default=None, choices=["mma_i8", "bn_vs_fixup"],
+                    help="mma_i8: measure the INT8 tensor-pipe figures; bn_vs_fixup: batch normalisation against the fused Fixup epilogue")
     ap.add_argument("--probe-seconds", type=float, default=2.0, help="length of each sustained probe loop")
     ap.add_argument("--int8-peaks", default=None, help="JSON printed by --probe, to report fractions of those figures too")
     ap.add_argument("--step-only", action="store_true",
@@ -562,6 +659,8 @@ def main():
         sys.exit(launch_ranks(args, sys.argv[1:]))
     if args.dry_run:
         run_dry(args)
+    elif args.probe == "bn_vs_fixup":
+        run_bn_compare(args)
     elif args.probe:
         run_probe(args)
     elif args.impl == "reference":

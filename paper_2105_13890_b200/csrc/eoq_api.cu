@@ -1509,7 +1509,7 @@ extern "C" int eoq_aux_maxpool_bwd(eoq_handle_t handle, const int8_t *e, const i
 extern "C" int eoq_bn_workspace_size(int c, size_t *bytes)
 {
     if (!bytes || c <= 0) return EOQ_ERR_BAD_ARG;
-    *bytes = (sizeof(BnChannel) * (size_t)c + 255) & ~(size_t)255;
+    *bytes = (bn_workspace_bytes(c) + 255) & ~(size_t)255;
     return EOQ_OK;
 }
 
@@ -1518,7 +1518,7 @@ static int bn_check(Handle *h, size_t pixels, int c, const void *ws, size_t ws_b
     if (!h || !ws || pixels == 0 || c <= 0) return EOQ_ERR_BAD_ARG;
     if (c % 16 || !aligned16(ws)) return EOQ_ERR_ALIGNMENT;
     if (c > 1024 || pixels > 0x7fffffffull) return EOQ_ERR_UNSUPPORTED;
-    if (ws_bytes < sizeof(BnChannel) * (size_t)c) return EOQ_ERR_WORKSPACE;
+    if (ws_bytes < bn_workspace_bytes(c)) return EOQ_ERR_WORKSPACE;
     return EOQ_OK;
 }
 

@@ -17,6 +17,8 @@ namespace eoq {
 namespace {
 
 constexpr int kBnThreads = 256;
+constexpr int kBnSplit = 16;       // threads of a finish kernel that share one channel
+constexpr int kBnMaxParts = 296;   // blocks of a statistics kernel (rows of partial sums in the workspace)
 
 __device__ __forceinline__ double u128_to_double(unsigned __int128 v)
 {
@@ -25,27 +27,39 @@ __device__ __forceinline__ double u128_to_double(unsigned __int128 v)
 }
 
 // Every thread owns four consecutive channels (one 16-byte load of sums) and walks pixels with a fixed stride, so
-// that its channels never change; block totals meet in shared memory, one global atomic per cell and block.
-__global__ void __launch_bounds__(kBnThreads) bn_stats_kernel(const int32_t *__restrict__ acc, size_t pixels, int c, BnChannel *ch)
+// that its channels never change; the threads of a block meet in shared memory and the block writes its totals to
+// its own row of `part` ([block][c][4]: s1, hh, hl, ll) - no global atomics; the finish kernel adds the rows.
+constexpr int kBnUnroll = 4;
+__global__ void __launch_bounds__(kBnThreads) bn_stats_kernel(const int32_t *__restrict__ acc, size_t pixels, int c,
+                                                             unsigned long long *__restrict__ part)
 {
-    extern __shared__ unsigned long long cell[];   // [c][4]: s1, hh, hl, ll
+    extern __shared__ unsigned long long cell[];   // [c][4]
     const int cg = c / 4;
     for (int i = threadIdx.x; i < c * 4; i += blockDim.x) cell[i] = 0ull;
     __syncthreads();
     const int g = threadIdx.x % cg, slot = threadIdx.x / cg, slots = blockDim.x / cg;
     long long s1[4] = {0, 0, 0, 0}, hh[4] = {0, 0, 0, 0}, hl[4] = {0, 0, 0, 0};
     unsigned long long ll[4] = {0, 0, 0, 0};
-    for (size_t p = (size_t)blockIdx.x * slots + slot; p < pixels; p += (size_t)gridDim.x * slots) {
-        const int4 v = __ldg(reinterpret_cast<const int4 *>(acc + p * c) + g);
-        const int a[4] = {v.x, v.y, v.z, v.w};
+    const size_t stride = (size_t)gridDim.x * slots;
+    for (size_t p0 = (size_t)blockIdx.x * slots + slot; p0 < pixels; p0 += kBnUnroll * stride) {
+        int4 v[kBnUnroll];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int h = a[q] >> 16;
-            const unsigned l = (unsigned)a[q] & 0xffffu;
-            s1[q] += a[q];
-            hh[q] += h * h;                                   // < 2^30
-            hl[q] += (long long)h * (long long)l;             // |.| < 2^31
-            ll[q] += (unsigned long long)(l * l);             // < 2^32
+        for (int u = 0; u < kBnUnroll; ++u) {
+            const size_t p = p0 + u * stride;
+            v[u] = p < pixels ? __ldg(reinterpret_cast<const int4 *>(acc + p * c) + g) : make_int4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < kBnUnroll; ++u) {
+            const int a[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int h = a[q] >> 16;
+                const unsigned l = (unsigned)a[q] & 0xffffu;
+                s1[q] += a[q];
+                hh[q] += h * h;                                   // < 2^30
+                hl[q] += (long long)h * (long long)l;             // |.| < 2^31
+                ll[q] += (unsigned long long)(l * l);             // < 2^32
+            }
         }
     }
 #pragma unroll
@@ -57,19 +71,36 @@ __global__ void __launch_bounds__(kBnThreads) bn_stats_kernel(const int32_t *__r
         atomicAdd(dst + 3, ll[q]);
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < c * 4; i += blockDim.x) {
-        const unsigned long long v = cell[i];
-        if (v) atomicAdd(reinterpret_cast<unsigned long long *>(&ch[i / 4].s1) + (i % 4), v);
-    }
+    unsigned long long *row = part + (size_t)blockIdx.x * c * 4;
+    for (int i = threadIdx.x; i < c * 4; i += blockDim.x) row[i] = cell[i];
 }
 
-__global__ void bn_finish_kernel(BnChannel *ch, size_t pixels, int c, int p, const float *__restrict__ gamma,
-                                 const float *__restrict__ beta, float eps)
+__global__ void bn_finish_kernel(BnChannel *ch, const unsigned long long *__restrict__ part, int parts, size_t pixels, int c, int p,
+                                 const float *__restrict__ gamma, const float *__restrict__ beta, float eps)
 {
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= c) return;
-    const long long s1 = ch[k].s1;
-    const __int128 s2 = ((__int128)ch[k].shh << 32) + ((__int128)ch[k].shl << 17) + (__int128)(unsigned long long)ch[k].sll;
+    // kBnSplit threads share a channel: each adds every kBnSplit-th row of partial sums, then the lanes meet by shuffle
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x, k = tid / kBnSplit, j = tid % kBnSplit;
+    unsigned long long t[4] = {0, 0, 0, 0};
+    if (k < c)
+        for (int b = j; b < parts; b += kBnSplit) {
+            const ulonglong2 *src = reinterpret_cast<const ulonglong2 *>(part + ((size_t)b * c + k) * 4);
+            const ulonglong2 lo = src[0], hi = src[1];
+            t[0] += lo.x;
+            t[1] += lo.y;
+            t[2] += hi.x;
+            t[3] += hi.y;
+        }
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int d = kBnSplit / 2; d > 0; d >>= 1) t[q] += __shfl_down_sync(0xffffffffu, t[q], d, kBnSplit);
+    if (k >= c || j != 0) return;
+    const long long s1 = (long long)t[0];
+    ch[k].s1 = s1;
+    ch[k].shh = (long long)t[1];
+    ch[k].shl = (long long)t[2];
+    ch[k].sll = (long long)t[3];
+    const __int128 s2 = ((__int128)(long long)t[1] << 32) + ((__int128)(long long)t[2] << 17) + (__int128)t[3];
     const unsigned __int128 V = (unsigned __int128)pixels * (unsigned __int128)s2 - (unsigned __int128)((__int128)s1 * s1);
     const double Pd = __ull2double_rn((unsigned long long)pixels);
     const double mu = __ddiv_rn(__ll2double_rn(s1), Pd);
@@ -119,9 +150,10 @@ __global__ void __launch_bounds__(kBnThreads) bn_apply_kernel(const int32_t *__r
     }
 }
 
-// D1 = sum(E * mask), D2 = sum(E * mask * A) per channel; same thread layout as bn_stats_kernel.
+// D1 = sum(E * mask), D2 = sum(E * mask * A) per channel; same thread layout as bn_stats_kernel, `part` [block][c][2].
 __global__ void __launch_bounds__(kBnThreads) bn_bwd_stats_kernel(const int8_t *__restrict__ e, const uint8_t *__restrict__ relu_mask,
-                                                                 const int32_t *__restrict__ acc, size_t pixels, int c, BnChannel *ch)
+                                                                 const int32_t *__restrict__ acc, size_t pixels, int c,
+                                                                 unsigned long long *__restrict__ part)
 {
     extern __shared__ unsigned long long cell[];   // [c][2]
     const int cg = c / 4;
@@ -129,17 +161,28 @@ __global__ void __launch_bounds__(kBnThreads) bn_bwd_stats_kernel(const int8_t *
     __syncthreads();
     const int g = threadIdx.x % cg, slot = threadIdx.x / cg, slots = blockDim.x / cg;
     long long d1[4] = {0, 0, 0, 0}, d2[4] = {0, 0, 0, 0};
-    for (size_t p = (size_t)blockIdx.x * slots + slot; p < pixels; p += (size_t)gridDim.x * slots) {
-        const size_t i0 = p * c + (size_t)g * 4;
-        const int4 v = __ldg(reinterpret_cast<const int4 *>(acc + i0));
-        const uint32_t ew = __ldg(reinterpret_cast<const uint32_t *>(e + i0));
-        const uint32_t m = (uint32_t)__ldg(relu_mask + (i0 >> 3)) >> (i0 & 7);
-        const int a[4] = {v.x, v.y, v.z, v.w};
+    const size_t stride = (size_t)gridDim.x * slots;
+    for (size_t p0 = (size_t)blockIdx.x * slots + slot; p0 < pixels; p0 += kBnUnroll * stride) {
+        int4 v[kBnUnroll];
+        uint32_t ew[kBnUnroll], m[kBnUnroll];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int dy = ((m >> q) & 1u) ? (int)(int8_t)(ew >> (8 * q)) : 0;
-            d1[q] += dy;
-            d2[q] += (long long)dy * a[q];
+        for (int u = 0; u < kBnUnroll; ++u) {
+            const size_t p = p0 + u * stride;
+            const size_t i0 = p * c + (size_t)g * 4;
+            const bool in = p < pixels;
+            v[u] = in ? __ldg(reinterpret_cast<const int4 *>(acc + i0)) : make_int4(0, 0, 0, 0);
+            ew[u] = in ? __ldg(reinterpret_cast<const uint32_t *>(e + i0)) : 0u;
+            m[u] = in ? (uint32_t)__ldg(relu_mask + (i0 >> 3)) >> (i0 & 7) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < kBnUnroll; ++u) {
+            const int a[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int dy = ((m[u] >> q) & 1u) ? (int)(int8_t)(ew[u] >> (8 * q)) : 0;
+                d1[q] += dy;
+                d2[q] += (long long)dy * a[q];
+            }
         }
     }
 #pragma unroll
@@ -148,21 +191,33 @@ __global__ void __launch_bounds__(kBnThreads) bn_bwd_stats_kernel(const int8_t *
         atomicAdd(cell + (size_t)(g * 4 + q) * 2 + 1, (unsigned long long)d2[q]);
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < c * 2; i += blockDim.x) {
-        const unsigned long long v = cell[i];
-        if (v) atomicAdd(reinterpret_cast<unsigned long long *>(&ch[i / 2].d1) + (i % 2), v);
-    }
+    unsigned long long *row = part + (size_t)blockIdx.x * c * 2;
+    for (int i = threadIdx.x; i < c * 2; i += blockDim.x) row[i] = cell[i];
 }
 
-__global__ void bn_bwd_finish_kernel(BnChannel *ch, size_t pixels, int c, int p, const int32_t *e_exp, const float *__restrict__ gamma,
-                                     float *dgamma, float *dbeta)
+__global__ void bn_bwd_finish_kernel(BnChannel *ch, const unsigned long long *__restrict__ part, int parts, size_t pixels, int c, int p,
+                                     const int32_t *e_exp, const float *__restrict__ gamma, float *dgamma, float *dbeta)
 {
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= c) return;
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x, k = tid / kBnSplit, j = tid % kBnSplit;
+    unsigned long long t0 = 0, t1 = 0;
+    if (k < c)
+        for (int b = j; b < parts; b += kBnSplit) {
+            const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(part + ((size_t)b * c + k) * 2);
+            t0 += v.x;
+            t1 += v.y;
+        }
+#pragma unroll
+    for (int d = kBnSplit / 2; d > 0; d >>= 1) {
+        t0 += __shfl_down_sync(0xffffffffu, t0, d, kBnSplit);
+        t1 += __shfl_down_sync(0xffffffffu, t1, d, kBnSplit);
+    }
+    if (k >= c || j != 0) return;
+    ch[k].d1 = (long long)t0;
+    ch[k].d2 = (long long)t1;
     const int p_e = *e_exp;
     const double Pd = __ull2double_rn((unsigned long long)pixels);
     const double mu = ch[k].mu, inv = ch[k].inv;
-    const double d1 = __ll2double_rn(ch[k].d1), d2 = __ll2double_rn(ch[k].d2);
+    const double d1 = __ll2double_rn((long long)t0), d2 = __ll2double_rn((long long)t1);
     const double cov = __dsub_rn(d2, __dmul_rn(mu, d1));
     const double ip = ldexp(inv, p);
     const double g2 = ldexp(__dmul_rn(ip, cov), p_e);
@@ -213,7 +268,8 @@ inline int stats_threads(int c) { return (kBnThreads / (c / 4)) * (c / 4); }
 
 inline int stats_grid(size_t pixels, int slots, int sm_count)
 {
-    size_t b = (pixels + slots - 1) / slots, cap = (size_t)sm_count * 4;
+    size_t b = (pixels + (size_t)slots * kBnUnroll - 1) / ((size_t)slots * kBnUnroll), cap = (size_t)(2 * sm_count);
+    if (cap > (size_t)kBnMaxParts) cap = kBnMaxParts;
     if (b > cap) b = cap;
     return b < 1 ? 1 : (int)b;
 }
@@ -227,14 +283,15 @@ inline int grid_for(size_t items, int sm_count, int per_sm)
 
 }  // namespace
 
+size_t bn_workspace_bytes(int c) { return sizeof(BnChannel) * (size_t)c + sizeof(unsigned long long) * 4 * (size_t)c * kBnMaxParts; }
+
 cudaError_t launch_bn_fwd(const int32_t *acc, int p, size_t pixels, int c, const float *gamma, const float *beta, float eps,
                           int8_t *x5, uint8_t *relu_mask, BnChannel *ch, int sm_count, cudaStream_t st)
 {
-    cudaError_t e = cudaMemsetAsync(ch, 0, sizeof(BnChannel) * (size_t)c, st);
-    if (e != cudaSuccess) return e;
-    const int threads = stats_threads(c), slots = threads / (c / 4);
-    bn_stats_kernel<<<stats_grid(pixels, slots, sm_count), threads, sizeof(unsigned long long) * 4 * c, st>>>(acc, pixels, c, ch);
-    bn_finish_kernel<<<(c + 127) / 128, 128, 0, st>>>(ch, pixels, c, p, gamma, beta, eps);
+    unsigned long long *part = reinterpret_cast<unsigned long long *>(ch + c);
+    const int threads = stats_threads(c), slots = threads / (c / 4), parts = stats_grid(pixels, slots, sm_count);
+    bn_stats_kernel<<<parts, threads, sizeof(unsigned long long) * 4 * c, st>>>(acc, pixels, c, part);
+    bn_finish_kernel<<<(c * kBnSplit + 127) / 128, 128, 0, st>>>(ch, part, parts, pixels, c, p, gamma, beta, eps);
     const size_t groups = pixels * (size_t)(c / 16);
     bn_apply_kernel<<<grid_for(groups, sm_count, 8), kBnThreads, sizeof(float2) * c, st>>>(acc, groups, c, ch, x5, relu_mask);
     return cudaGetLastError();
@@ -244,13 +301,10 @@ cudaError_t launch_bn_bwd(const int8_t *e, const int32_t *e_exp, const uint8_t *
                           int c, const float *gamma, BnChannel *ch, float *da, float *dgamma, float *dbeta, int sm_count,
                           cudaStream_t st)
 {
-    const int threads = stats_threads(c), slots = threads / (c / 4);
-    // d1 and d2 start from zero on every call; they sit side by side in the record of a channel
-    cudaError_t err = cudaMemset2DAsync(&ch[0].d1, sizeof(BnChannel), 0, 2 * sizeof(long long), (size_t)c, st);
-    if (err != cudaSuccess) return err;
-    bn_bwd_stats_kernel<<<stats_grid(pixels, slots, sm_count), threads, sizeof(unsigned long long) * 2 * c, st>>>(e, relu_mask, acc,
-                                                                                                                     pixels, c, ch);
-    bn_bwd_finish_kernel<<<(c + 127) / 128, 128, 0, st>>>(ch, pixels, c, p, e_exp, gamma, dgamma, dbeta);
+    unsigned long long *part = reinterpret_cast<unsigned long long *>(ch + c);
+    const int threads = stats_threads(c), slots = threads / (c / 4), parts = stats_grid(pixels, slots, sm_count);
+    bn_bwd_stats_kernel<<<parts, threads, sizeof(unsigned long long) * 2 * c, st>>>(e, relu_mask, acc, pixels, c, part);
+    bn_bwd_finish_kernel<<<(c * kBnSplit + 127) / 128, 128, 0, st>>>(ch, part, parts, pixels, c, p, e_exp, gamma, dgamma, dbeta);
     const size_t groups = pixels * (size_t)(c / 16);
     bn_bwd_apply_kernel<<<grid_for(groups, sm_count, 8), kBnThreads, sizeof(float4) * c, st>>>(e, relu_mask, acc, groups, c, ch, da);
     return cudaGetLastError();

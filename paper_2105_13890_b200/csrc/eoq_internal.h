@@ -337,6 +337,7 @@ struct BnChannel {
     float scale, shift;            // y = fma((float)A, scale, shift)
     float ca, cb, cc, pad;         // da = fma(ca, E * mask, fma(cb, (float)A, cc))
 };
+size_t bn_workspace_bytes(int c);   // records + per-block partial sums
 cudaError_t launch_bn_fwd(const int32_t *acc, int p, size_t pixels, int c, const float *gamma, const float *beta, float eps,
                           int8_t *x5, uint8_t *relu_mask, BnChannel *ch, int sm_count, cudaStream_t st);
 cudaError_t launch_bn_bwd(const int8_t *e, const int32_t *e_exp, const uint8_t *relu_mask, const int32_t *acc, int p, size_t pixels,
