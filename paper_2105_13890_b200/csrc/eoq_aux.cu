@@ -390,33 +390,63 @@ __global__ void head_softmax_kernel(const float *__restrict__ logits, int n, int
     }
 }
 
-// dpooled[b][k] = sum_j fma(dl[b][j], W[j][k], .), j ascending (W before its update); thread 0 also forms the mean loss
-__global__ void head_dpooled_kernel(const float *__restrict__ dl, const float *__restrict__ W, int n, int c, int classes, float *dpooled,
-                                    const double *loss_n, float *loss_out)
+// dpooled[b][k] = sum_j fma(dl[b][j], W[j][k], .), j ascending (W before its update); one thread also forms the mean loss.
+// Every output is one chain of `classes` dependent multiply-adds, so the only parallelism is across outputs (n * c of
+// them) and the only thing to hide is the memory traffic: a block owns kDpCh channels x kDpN samples, all its threads
+// fetch the next kDpK rows of W (and of dl) together into registers while the chains run on the current rows in
+// shared memory.
+constexpr int kDpCh = 64, kDpN = 4, kDpK = 32;
+__global__ void __launch_bounds__(kDpCh *kDpN)
+head_dpooled_kernel(const float *__restrict__ dl, const float *__restrict__ W, int n, int c, int classes, float *dpooled,
+                    const double *loss_n, float *loss_out)
 {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i == 0 && loss_out) {
+    __shared__ float w_s[2][kDpK][kDpCh];
+    __shared__ float d_s[2][kDpN][kDpK];
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && loss_out) {
         double s = 0.0;
         for (int b = 0; b < n; ++b) s += loss_n[b];
         *loss_out = (float)(s / n);
     }
-    if (i >= n * c) return;
-    const int b = i / c, k = i % c;
-    float acc = 0.0f;
-    const float *db = dl + (size_t)b * classes, *wk = W + k;
-    int j = 0;
-    for (; j + 8 <= classes; j += 8) {   // eight independent loads in flight, then the chain in order
-        float w8[8], d8[8];
+    const int cl = threadIdx.x % kDpCh, nl = threadIdx.x / kDpCh;
+    const int k = blockIdx.x * kDpCh + cl, b = blockIdx.y * kDpN + nl;
+    const bool kin = k < c;
+    constexpr int kRowsPerThread = kDpK / kDpN;   // rows of the W tile one thread fetches
+    float wr[kRowsPerThread], dr = 0.0f;
+    auto fetch = [&](int j0) {
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            w8[u] = __ldg(wk + (size_t)(j + u) * c);
-            d8[u] = __ldg(db + j + u);
+        for (int r = 0; r < kRowsPerThread; ++r) {
+            const int j = j0 + nl + r * kDpN;
+            wr[r] = (kin && j < classes) ? __ldg(W + (size_t)j * c + k) : 0.0f;
         }
+        if (threadIdx.x < kDpN * kDpK) {
+            const int bb = blockIdx.y * kDpN + threadIdx.x / kDpK, j = j0 + threadIdx.x % kDpK;
+            dr = (bb < n && j < classes) ? __ldg(dl + (size_t)bb * classes + j) : 0.0f;
+        }
+    };
+    auto stash = [&](int buf) {
 #pragma unroll
-        for (int u = 0; u < 8; ++u) acc = __fmaf_rn(d8[u], w8[u], acc);
+        for (int r = 0; r < kRowsPerThread; ++r) w_s[buf][nl + r * kDpN][cl] = wr[r];
+        if (threadIdx.x < kDpN * kDpK) d_s[buf][threadIdx.x / kDpK][threadIdx.x % kDpK] = dr;
+    };
+    fetch(0);
+    stash(0);
+    __syncthreads();
+    float acc = 0.0f;
+    int buf = 0;
+    for (int j0 = 0; j0 < classes; j0 += kDpK, buf ^= 1) {
+        const bool more = j0 + kDpK < classes;
+        if (more) fetch(j0 + kDpK);
+        const int len = min(kDpK, classes - j0);
+        if (len == kDpK) {
+#pragma unroll
+            for (int jj = 0; jj < kDpK; ++jj) acc = __fmaf_rn(d_s[buf][nl][jj], w_s[buf][jj][cl], acc);
+        } else {
+            for (int jj = 0; jj < len; ++jj) acc = __fmaf_rn(d_s[buf][nl][jj], w_s[buf][jj][cl], acc);
+        }
+        if (more) stash(buf ^ 1);
+        __syncthreads();
     }
-    for (; j < classes; ++j) acc = __fmaf_rn(__ldg(db + j), __ldg(wk + (size_t)j * c), acc);
-    dpooled[i] = acc;
+    if (kin && b < n) dpooled[(size_t)b * c + k] = acc;
 }
 
 // W[j][k] <- fma(-lr, sum_b fma(dl[b][j], pooled[b][k], .), W[j][k]), b ascending; bias[j] alike (thread k == 0)
@@ -596,7 +626,7 @@ cudaError_t launch_join(const int8_t *a, const int32_t *a_exp, const int8_t *b, 
                         cudaStream_t st, const ReduceHook &hook)
 {
     const size_t n16 = n_el / 16;
-    const int blocks = blocks_for(n16, sm_count, 4);
+    const int blocks = blocks_for(n16, sm_count, 8);
     join_kernel<0><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, dev);
     hook(&dev->absmax_u64, 1, EOQ_REDUCE_I64, EOQ_REDUCE_MAX, st);
     join_kernel<1><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, dev);
@@ -617,7 +647,8 @@ cudaError_t launch_head(const int32_t *sums, int n, int c, int hw, int classes, 
         head_logits_kernel<<<grid, 32 * kHeadWarps, smem, st>>>(pooled, n, c, classes, W, bias, logits);
     }
     head_softmax_kernel<<<n, 256, 0, st>>>(logits, n, classes, labels, dl, loss_n);
-    head_dpooled_kernel<<<(n * c + 127) / 128, 128, 0, st>>>(dl, W, n, c, classes, dpooled, loss_n, loss_out);
+    head_dpooled_kernel<<<dim3((c + kDpCh - 1) / kDpCh, (n + kDpN - 1) / kDpN), kDpCh * kDpN, 0, st>>>(dl, W, n, c, classes, dpooled,
+                                                                                                   loss_n, loss_out);
     head_update_kernel<<<(classes * c + 127) / 128, 128, 0, st>>>(dl, pooled, n, c, classes, lr, W, bias);
     return cudaGetLastError();
 }
