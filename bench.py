@@ -355,6 +355,8 @@ def run_gpu(args):
         torch.cuda._sleep(12_000_000)
         step.run()
     prof_n, prof_ms = eoq.eoq_profile_stop(handle)
+    # the tensor pipe's own INT8 figure, measured on the spot (issue-rate probe, N = 256, about ten milliseconds)
+    probe_tops, _ = eoq.eoq_probe_mma_i8(handle, 256, 2048, 10)
     t_wall2 = time.time()
     # clocks while the GPU was under this load: the timed steps first, the whole loaded span if that is too short
     clocks = None
@@ -416,6 +418,7 @@ def run_gpu(args):
                 "timing": "graph replay of the launches back to back, CUDA events around the run",
                 "frac_of_nominal_4500": achieved / NOMINAL_INT8_TOPS,
                 "frac_of_sustained_bf16_x2": achieved / (pk["bf16_sustained"] * INT8_OVER_BF16),
+                "mma_i8_probe_tops": probe_tops, "frac_of_mma_i8_probe": achieved / probe_tops,
             },
             "kernels": {
                 "igemm_fwd": {"launches": n_fwd, "ms": conv_ms["fwd"], "tops": fwd_ops / (conv_ms["fwd"] / 1e3) / 1e12},
