@@ -157,6 +157,19 @@ EOQ_API int eoq_weight_prep(eoq_handle_t handle, int num, const eoq_conv_desc_t 
 EOQ_API int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
                    const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4, int32_t *acc_dump,
                    void *workspace, size_t workspace_bytes, void *stream);
+/*
+ * eoq_conv_dgrad with the error head of the layer that consumes e4 fused into Q_e (what eoq_err_prescale_dev would
+ * compute from e4; Sec. 3.2.1, e1 = e0 [x4 > 0], e3 = Q_e(gamma e1) of the layer in front): next_relu_mask, next_x2
+ * (optional, int16) and next_gamma (device code) are that layer's; next_e3 (same shape as e4), *next_e3_exp,
+ * *next_sum_e1 and (with next_x2) *next_sum_e1x2 are its results.  The GEMM's epilogue reduces the maximum over the
+ * positions that layer's ReLU lets through beside the plain one (Q_e is monotonic in |.|, so the largest code of e1 is
+ * the code of that maximum), and the pass that writes e4 writes next_e3 as well.  Bit-identical to the two calls in
+ * sequence.  EOQ_ERR_UNSUPPORTED for strided 1x1 filters (their sums are kept compact).
+ */
+EOQ_API int eoq_conv_dgrad_head(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                        const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4, const uint8_t *next_relu_mask,
+                        const int16_t *next_x2, const int32_t *next_gamma, int8_t *next_e3, int32_t *next_e3_exp,
+                        int64_t *next_sum_e1, int64_t *next_sum_e1x2, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * eoq_conv_dgrad without any allocation (the paper has no counterpart; this is a deployment variant).
@@ -289,6 +302,14 @@ EOQ_API int eoq_aux_maxpool_fwd(eoq_handle_t handle, const int8_t *x, int n, int
  * exact sums are requantized with Q_e = SQ: e_in [n,h,w,c], *e_in_exp. */
 EOQ_API int eoq_aux_maxpool_bwd(eoq_handle_t handle, const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int h, int w,
                         int c, int k, int stride, int pad, int8_t *e_in, int32_t *e_in_exp, void *stream);
+/* The same with the error head of the layer in front of the pool fused in (what eoq_err_prescale_dev would compute
+ * from e_in, without x2): e1 = e_in * [x4 > 0] (relu_mask of that layer, bit i of the NHWC element index),
+ * e3 = Q_e(gamma * e1) [n,h,w,c] with *e3_exp, *sum_e1 (optional) = sum of the e1 codes; gamma: that layer's code in
+ * device memory.  e_in and e_in_exp may be NULL when only e3 is wanted.  Bit-identical to the two calls in sequence. */
+EOQ_API int eoq_aux_maxpool_bwd_head(eoq_handle_t handle, const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int h,
+                             int w, int c, int k, int stride, int pad, int8_t *e_in, int32_t *e_in_exp,
+                             const uint8_t *relu_mask, const int32_t *gamma, int8_t *e3, int32_t *e3_exp, int64_t *sum_e1,
+                             void *stream);
 /* Global average pooling hands exact integer sums to the head: sums[n][c] = sum over the hw positions of x. */
 EOQ_API int eoq_aux_avgpool_sum(eoq_handle_t handle, const int8_t *x, int n, int hw, int c, int32_t *sums, void *stream);
 /*
@@ -300,6 +321,14 @@ EOQ_API int eoq_aux_avgpool_sum(eoq_handle_t handle, const int8_t *x, int n, int
  */
 EOQ_API int eoq_aux_join(eoq_handle_t handle, const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp,
                  const uint8_t *mask_b, size_t n_el, int8_t *out, int32_t *out_exp, int64_t *sum_out, void *stream);
+/* The same with the error head of the layer that consumes `out` fused in (what eoq_err_prescale_dev would compute from
+ * out): e1 = out * [x4 > 0] (relu_mask of that layer), e3 = Q_e(gamma * e1) with *e3_exp, *sum_e1 and, when x2 is given
+ * (int16, that layer's x2), *sum_e1x2 = sum of e1 * x2; gamma: that layer's code in device memory.  Bit-identical to
+ * the two calls in sequence. */
+EOQ_API int eoq_aux_join_head(eoq_handle_t handle, const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp,
+                      const uint8_t *mask_b, size_t n_el, int8_t *out, int32_t *out_exp, int64_t *sum_out,
+                      const uint8_t *relu_mask, const int16_t *x2, const int32_t *gamma, int8_t *e3, int32_t *e3_exp,
+                      int64_t *sum_e1, int64_t *sum_e1x2, void *stream);
 /*
  * The floating-point last layer, operation by operation in fp32 (every product-sum is one fused multiply-add, sums
  * run over ascending indices into one accumulator, exp is a fixed polynomial), so that any IEEE-754 machine gives
@@ -312,6 +341,12 @@ EOQ_API int eoq_aux_head_workspace_size(int n, int c, int classes, size_t *bytes
 EOQ_API int eoq_aux_head(eoq_handle_t handle, const int32_t *sums, int n, int c, int hw, int classes, float *W, float *bias,
                  const int32_t *labels, float lr, float *loss, float *dpooled, float *logits, void *workspace,
                  size_t workspace_bytes, void *stream);
+/* The SGD step of W and bias alone, from what the last eoq_aux_head call on this workspace left there (its pooled
+ * activations and logit gradients): for callers that pass lr = 0 to eoq_aux_head (W and bias then stay untouched,
+ * which is what a zero rate means) and take the step later, e.g. on another stream beside the backward pass.
+ * The results are the ones eoq_aux_head gives with that lr. */
+EOQ_API int eoq_aux_head_update(eoq_handle_t handle, int n, int c, int classes, float *W, float *bias, float lr, const void *workspace,
+                        size_t workspace_bytes, void *stream);
 /* The error the head hands back: SQ over all of dpooled / hw (the gradient of one position of the average), the
  * code of (sample, channel) written to all hw positions: e [n][hw][c], *e_exp.  workspace: n*c floats. */
 EOQ_API int eoq_aux_head_error(eoq_handle_t handle, const float *dpooled, int n, int c, int hw, int8_t *e, int32_t *e_exp,

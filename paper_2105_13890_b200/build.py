@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libeoq.so")
 SOURCES = ["eoq_api.cu", "eoq_igemm.cu", "eoq_igemm_patch.cu", "eoq_wgrad_patch.cu", "eoq_wgrad.cu", "eoq_elementwise.cu", "eoq_static.cu", "eoq_probe.cu", "eoq_aux.cu", "eoq_bn.cu"]
-HEADERS = ["eoq_internal.h", "eoq_device.cuh", "eoq_epilogue.cuh", os.path.join(ROOT, "include", "eoq.h")]
+HEADERS = ["eoq_internal.h", "eoq_device.cuh", "eoq_epilogue.cuh", "eoq_next_head.cuh", os.path.join(ROOT, "include", "eoq.h")]
 
 
 def _stale() -> bool:

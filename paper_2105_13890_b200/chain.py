@@ -69,8 +69,9 @@ class ChainedStep:
     def __init__(self, workload: Workload, handle: int, device: str = "cuda:0", seed: int = synth.BASE_SEED,
                  scalars: Optional[Scalars] = None, lr_mant: int = 3, lr_exp: int = -4, head_lr: float = 2.0 ** -6,
                  classes: int = 1000, pool: Optional[tuple] = None, round_mode: int = eoq.EOQ_ROUND_RNE,
-                 image_channels: int = 3, side_streams: int = 2):
+                 image_channels: int = 3, side_streams: int = 2, keep_pool_error: bool = False):
         self.wl, self.h, self.dev = workload, handle, torch.device(device)
+        self.keep_pool_error = keep_pool_error   # also write the error between the pool and the first layer's head
         self.sc = scalars or Scalars()
         self.lr_mant, self.lr_exp, self.head_lr, self.classes = lr_mant, lr_exp, head_lr, classes
         self.round_mode, self.seed, self.pool = round_mode, seed, pool
@@ -212,8 +213,13 @@ class ChainedStep:
         last = self.blocks[-1].b
         n = fl.n
         eoq.eoq_aux_avgpool_sum(h, last.x5, n, self.hw, self.c_last, self.sums)
-        eoq.eoq_aux_head(h, self.sums, n, self.c_last, self.hw, self.classes, self.W, self.bias, self.labels, self.head_lr, self.loss,
-                         self.dpooled, self.logits, self.head_ws)
+        # the head's own SGD step is not needed by the backward pass: it runs beside it
+        eoq.eoq_aux_head(h, self.sums, n, self.c_last, self.hw, self.classes, self.W, self.bias, self.labels,
+                         0.0 if overlap else self.head_lr, self.loss, self.dpooled, self.logits, self.head_ws)
+        if overlap:
+            self.sides[-1].wait_stream(main)
+            with torch.cuda.stream(self.sides[-1]):
+                eoq.eoq_aux_head_update(self.h_sides[-1], n, self.c_last, self.classes, self.W, self.bias, self.head_lr, self.head_ws)
         eoq.eoq_aux_head_error(h, self.dpooled, n, self.c_last, self.hw, self.e_head, self.e_head_exp, ws)
 
         side_no = [0]
@@ -229,12 +235,16 @@ class ChainedStep:
                 eoq.eoq_conv_wgrad_dev(h, u.desc, u.e3, u.e3_exp, u.x0, b1_dev, u.g, u.g_exp, ws)
 
         e_out, e_exp = self.e_head, self.e_head_exp
-        for blk in reversed(self.blocks):
+        head_done = False   # the error head of this block's last unit already ran inside the join of the block behind it
+        for i in reversed(range(len(self.blocks))):
+            blk = self.blocks[i]
             a, b, pr = blk.a, blk.b, blk.proj
-            eoq.eoq_err_prescale_dev(h, e_out, e_exp, b.mask, b.x2, b.n_out, b.scal[1:2], b.e3, b.e3_exp, b.sum_e1, b.sum_e1x2)
+            if not head_done:
+                eoq.eoq_err_prescale_dev(h, e_out, e_exp, b.mask, b.x2, b.n_out, b.scal[1:2], b.e3, b.e3_exp, b.sum_e1, b.sum_e1x2)
             wgrad(b, b.scal[0:1])
-            eoq.eoq_conv_dgrad(h, b.desc, b.e3, b.e3_exp, b.w, b.e4, b.e4_exp, b.sum_e4, None, ws)
-            eoq.eoq_err_prescale_dev(h, b.e4, b.e4_exp, a.mask, None, a.n_out, a.scal[1:2], a.e3, a.e3_exp, a.sum_e1, None)
+            # error back through unit B; the error head of unit A rides on its Q_e
+            eoq.eoq_conv_dgrad_head(h, b.desc, b.e3, b.e3_exp, b.w, b.e4, b.e4_exp, b.sum_e4, a.mask, None, a.scal[1:2], a.e3,
+                                    a.e3_exp, a.sum_e1, None, ws)
             wgrad(a, a.scal[0:1])
             eoq.eoq_conv_dgrad(h, a.desc, a.e3, a.e3_exp, a.w, a.e4, a.e4_exp, a.sum_e4, None, ws)
             if pr:
@@ -242,16 +252,31 @@ class ChainedStep:
                 eoq.eoq_err_prescale_dev(h, e_out, e_exp, b.mask, None, pr.n_out, self.c128, pr.e3, pr.e3_exp, pr.sum_e1, None)
                 wgrad(pr, a.scal[0:1])
                 eoq.eoq_conv_dgrad(h, pr.desc, pr.e3, pr.e3_exp, pr.w, pr.e4, pr.e4_exp, pr.sum_e4, None, ws)
-                eoq.eoq_aux_join(h, a.e4, a.e4_exp, pr.e4, pr.e4_exp, None, a.e4.numel(), blk.e_in, blk.e_in_exp, blk.sum_join)
+                j_b, j_b_exp, j_mask = pr.e4, pr.e4_exp, None
             else:
-                eoq.eoq_aux_join(h, a.e4, a.e4_exp, e_out, e_exp, b.mask, a.e4.numel(), blk.e_in, blk.e_in_exp, blk.sum_join)
+                j_b, j_b_exp, j_mask = e_out, e_exp, b.mask
+            # the joined error feeds the last unit of the block in front (or the first layer when no pool sits between):
+            # that unit's error head rides on the join
+            nxt = self.blocks[i - 1].b if i > 0 else (None if self.pool else stem)
+            if nxt is not None:
+                eoq.eoq_aux_join_head(h, a.e4, a.e4_exp, j_b, j_b_exp, j_mask, a.e4.numel(), blk.e_in, blk.e_in_exp, blk.sum_join,
+                                      nxt.mask, nxt.x2, nxt.scal[1:2], nxt.e3, nxt.e3_exp, nxt.sum_e1,
+                                      nxt.sum_e1x2 if nxt.x2 is not None else None)
+                head_done = True
+            else:
+                eoq.eoq_aux_join(h, a.e4, a.e4_exp, j_b, j_b_exp, j_mask, a.e4.numel(), blk.e_in, blk.e_in_exp, blk.sum_join)
+                head_done = False
             e_out, e_exp = blk.e_in, blk.e_in_exp
         if self.pool:
             k, s, p = self.pool
-            eoq.eoq_aux_maxpool_bwd(h, e_out, e_exp, self.pool_arg, fl.n, fl.ho, fl.wo, fl.c_out, k, s, p, self.stem_e0,
-                                    self.stem_e0_exp)
-            e_out, e_exp = self.stem_e0, self.stem_e0_exp
-        eoq.eoq_err_prescale_dev(h, e_out, e_exp, stem.mask, None, stem.n_out, stem.scal[1:2], stem.e3, stem.e3_exp, stem.sum_e1, None)
+            # pool backward and the first layer's error head in one pair of kernels; the error between them (51 MB at
+            # batch 64) is written only when a caller wants to look at it
+            eoq.eoq_aux_maxpool_bwd_head(h, e_out, e_exp, self.pool_arg, fl.n, fl.ho, fl.wo, fl.c_out, k, s, p,
+                                         self.stem_e0 if self.keep_pool_error else None, self.stem_e0_exp, stem.mask,
+                                         stem.scal[1:2], stem.e3, stem.e3_exp, stem.sum_e1)
+        elif not head_done:
+            eoq.eoq_err_prescale_dev(h, e_out, e_exp, stem.mask, None, stem.n_out, stem.scal[1:2], stem.e3, stem.e3_exp, stem.sum_e1,
+                                     None)
         wgrad(stem, None)
         if overlap:
             for side in self.sides:

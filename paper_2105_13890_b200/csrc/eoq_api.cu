@@ -815,9 +815,10 @@ extern "C" int eoq_weight_prep(eoq_handle_t handle, int num, const eoq_conv_desc
 
 // ================================================================================= error back-propagation
 
-extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3,
-                              const int32_t *e3_exp, const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4,
-                              int32_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
+// `next`: the error head of the layer that consumes e4, fused into Q_e (null for the plain call)
+static int conv_dgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                           const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4, int32_t *acc_dump,
+                           const NextHeadArgs *next, void *workspace, size_t workspace_bytes, void *stream)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
     Geometry g;
@@ -826,6 +827,13 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
     if (st != EOQ_OK) return st;
     if (!aligned16(e3) || !aligned16(w) || !aligned16(e4) || !aligned16(acc_dump)) return EOQ_ERR_ALIGNMENT;
     if (desc->c_in % 16) return EOQ_ERR_UNSUPPORTED;  // 8 channels exist for the network input, which takes no error
+    if (next) {
+        if (!next->mask || !next->gamma || !next->e3 || !next->e3_exp) return EOQ_ERR_BAD_ARG;
+        if (!aligned16(next->e3) || (next->x2 && !aligned16(next->x2)) || (reinterpret_cast<uintptr_t>(next->mask) & 1))
+            return EOQ_ERR_ALIGNMENT;
+        // the compact sums of a strided 1x1 filter are not laid out like the error tensor
+        if (desc->kh == 1 && desc->kw == 1 && desc->pad == 0 && desc->stride > 1) return EOQ_ERR_UNSUPPORTED;
+    }
     if ((st = check_workspace(desc, EOQ_PASS_DGRAD, workspace, workspace_bytes)) != EOQ_OK) return st;
     const eoq_conv_desc_t &d = *desc;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
@@ -851,6 +859,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             p.epilogue = kEpiDgrad;
             p.acc_out = sums;
             p.dev = h->dev;
+            p.next_mask = next ? next->mask : nullptr;
             // the weights are read where they are, [c_out][tap][c_in]: the reduction (c_out) is their slow axis, so
             // they reach the MMA as MN-major atoms of b_row input channels
             p.b_mn = 1;
@@ -869,7 +878,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             {
                 ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
                 e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true,
-                                  h->dev, h->sm_count, s, h->hook);
+                                  h->dev, h->sm_count, s, h->hook, next);
             }
             count_launches(h, 1);
             return record(h, e);
@@ -977,6 +986,7 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
             p.epilogue = kEpiDgrad;
             p.acc_out = sums;
             p.dev = h->dev;
+            p.next_mask = next ? next->mask : nullptr;
             CUtensorMap map_a, map_b;
             if (weights_in_place) {
                 p.b_mn = 1;
@@ -1032,10 +1042,28 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                                       h->dev, h->sm_count, s, h->hook);
         else
             e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
-                              h->sm_count, s, h->hook);
+                              h->sm_count, s, h->hook, next);
     }
     count_launches(h, 1);
     return record(h, e);
+}
+
+extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3,
+                              const int32_t *e3_exp, const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4,
+                              int32_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return conv_dgrad_impl(handle, desc, e3, e3_exp, w, e4, e4_exp, sum_e4, acc_dump, nullptr, workspace, workspace_bytes, stream);
+}
+
+extern "C" int eoq_conv_dgrad_head(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                                   const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4, const uint8_t *next_relu_mask,
+                                   const int16_t *next_x2, const int32_t *next_gamma, int8_t *next_e3, int32_t *next_e3_exp,
+                                   int64_t *next_sum_e1, int64_t *next_sum_e1x2, void *workspace, size_t workspace_bytes,
+                                   void *stream)
+{
+    const NextHeadArgs next{next_relu_mask, next_x2, next_gamma, next_e3, next_e3_exp, reinterpret_cast<long long *>(next_sum_e1),
+                            reinterpret_cast<long long *>(next_sum_e1x2)};
+    return conv_dgrad_impl(handle, desc, e3, e3_exp, w, e4, e4_exp, sum_e4, nullptr, &next, workspace, workspace_bytes, stream);
 }
 
 // ================================================================================= weight gradient
@@ -1503,7 +1531,28 @@ extern "C" int eoq_aux_maxpool_bwd(eoq_handle_t handle, const int8_t *e, const i
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     count_launches(h, 2);
     ProfScope prof(h, EOQ_PROF_GLUE, s);
-    return record(h, launch_maxpool_bwd(e, e_exp, arg, n, hh, ww, c, k, stride, pad, e_in, e_in_exp, h->dev, h->sm_count, s, h->hook));
+    return record(h, launch_maxpool_bwd(e, e_exp, arg, n, hh, ww, c, k, stride, pad, e_in, e_in_exp, nullptr, nullptr, nullptr, nullptr,
+                                        nullptr, h->dev, h->sm_count, s, h->hook));
+}
+
+extern "C" int eoq_aux_maxpool_bwd_head(eoq_handle_t handle, const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int hh,
+                                        int ww, int c, int k, int stride, int pad, int8_t *e_in, int32_t *e_in_exp,
+                                        const uint8_t *relu_mask, const int32_t *gamma, int8_t *e3, int32_t *e3_exp, int64_t *sum_e1,
+                                        void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !e || !e_exp || !arg || !relu_mask || !gamma || !e3 || !e3_exp || n <= 0 || hh <= 0 || ww <= 0 || c <= 0 || k <= 0 ||
+        k > 15 || stride <= 0 || pad < 0 || pad >= k)
+        return EOQ_ERR_BAD_ARG;
+    if (c % 16 || !aligned16(e) || !aligned16(arg) || !aligned16(e3) || (e_in && !aligned16(e_in)) ||
+        (reinterpret_cast<uintptr_t>(relu_mask) & 1))
+        return EOQ_ERR_ALIGNMENT;
+    if ((size_t)n * hh * ww * (c / 16) > 0x7fffffffull) return EOQ_ERR_UNSUPPORTED;   // 32-bit item index in the kernel
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 2);
+    ProfScope prof(h, EOQ_PROF_GLUE, s);
+    return record(h, launch_maxpool_bwd(e, e_exp, arg, n, hh, ww, c, k, stride, pad, e_in, e_in_exp, relu_mask, gamma, e3, e3_exp,
+                                        reinterpret_cast<long long *>(sum_e1), h->dev, h->sm_count, s, h->hook));
 }
 
 extern "C" int eoq_bn_workspace_size(int c, size_t *bytes)
@@ -1575,7 +1624,26 @@ extern "C" int eoq_aux_join(eoq_handle_t handle, const int8_t *a, const int32_t 
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     count_launches(h, 2);
     ProfScope prof(h, EOQ_PROF_GLUE, s);
-    return record(h, launch_join(a, a_exp, b, b_exp, mask_b, n_el, out, out_exp, reinterpret_cast<long long *>(sum_out), h->dev,
+    return record(h, launch_join(a, a_exp, b, b_exp, mask_b, n_el, out, out_exp, reinterpret_cast<long long *>(sum_out), nullptr, nullptr,
+                                 nullptr, nullptr, nullptr, nullptr, nullptr, h->dev, h->sm_count, s, h->hook));
+}
+
+extern "C" int eoq_aux_join_head(eoq_handle_t handle, const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp,
+                                 const uint8_t *mask_b, size_t n_el, int8_t *out, int32_t *out_exp, int64_t *sum_out,
+                                 const uint8_t *relu_mask, const int16_t *x2, const int32_t *gamma, int8_t *e3, int32_t *e3_exp,
+                                 int64_t *sum_e1, int64_t *sum_e1x2, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !a || !a_exp || !b || !b_exp || !out || !out_exp || !relu_mask || !gamma || !e3 || !e3_exp || n_el == 0 || (n_el % 16))
+        return EOQ_ERR_BAD_ARG;
+    if (!aligned16(a) || !aligned16(b) || !aligned16(out) || !aligned16(e3) || (x2 && !aligned16(x2)) ||
+        (reinterpret_cast<uintptr_t>(mask_b) & 1) || (reinterpret_cast<uintptr_t>(relu_mask) & 1))
+        return EOQ_ERR_ALIGNMENT;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 2);
+    ProfScope prof(h, EOQ_PROF_GLUE, s);
+    return record(h, launch_join(a, a_exp, b, b_exp, mask_b, n_el, out, out_exp, reinterpret_cast<long long *>(sum_out), relu_mask, x2, gamma,
+                                 e3, e3_exp, reinterpret_cast<long long *>(sum_e1), reinterpret_cast<long long *>(sum_e1x2), h->dev,
                                  h->sm_count, s, h->hook));
 }
 
@@ -1602,9 +1670,26 @@ extern "C" int eoq_aux_head(eoq_handle_t handle, const int32_t *sums, int n, int
     float *dl = reinterpret_cast<float *>(ws + 2 * round256((size_t)n * c * sizeof(float)));
     double *loss_n = reinterpret_cast<double *>(ws + 2 * round256((size_t)n * c * sizeof(float)) + round256((size_t)n * classes * sizeof(float)));
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    count_launches(h, 5);
+    count_launches(h, lr != 0.0f ? 5 : 4);
     ProfScope prof(h, EOQ_PROF_GLUE, s);
     return record(h, launch_head(sums, n, c, hw, classes, W, bias, labels, lr, loss, dpooled, logits, pooled, dl, loss_n, s));
+}
+
+extern "C" int eoq_aux_head_update(eoq_handle_t handle, int n, int c, int classes, float *W, float *bias, float lr, const void *workspace,
+                                   size_t workspace_bytes, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || !W || !bias || n <= 0 || c <= 0 || classes <= 0) return EOQ_ERR_BAD_ARG;
+    size_t need = 0;
+    eoq_aux_head_workspace_size(n, c, classes, &need);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < need) return EOQ_ERR_WORKSPACE;
+    const char *ws = static_cast<const char *>(workspace);
+    const float *pooled = reinterpret_cast<const float *>(ws);
+    const float *dl = reinterpret_cast<const float *>(ws + 2 * round256((size_t)n * c * sizeof(float)));
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    count_launches(h, 1);
+    ProfScope prof(h, EOQ_PROF_GLUE, s);
+    return record(h, launch_head_update(dl, pooled, n, c, classes, lr, W, bias, s));
 }
 
 extern "C" int eoq_aux_head_error(eoq_handle_t handle, const float *dpooled, int n, int c, int hw, int8_t *e, int32_t *e_exp,

@@ -6,6 +6,7 @@
 // All of it is bandwidth- or latency-bound support work; none of it touches the tensor cores.
 #include "eoq_device.cuh"
 #include "eoq_internal.h"
+#include "eoq_next_head.cuh"
 
 namespace eoq {
 
@@ -86,27 +87,40 @@ __global__ void maxpool_fwd_kernel(const int8_t *__restrict__ x, int n, int h, i
 // ceil(k / stride)^2): a window's 16 codes count where its recorded position equals this one.  Four codes are
 // handled per 32-bit word: bytes are compared at once, the chosen codes are kept with an offset of 128 (others as
 // 128 itself) so that they add as unsigned halves of two words without carries between them.
-template <int kPass>
+//
+// kNext: the consumer's error head rides along (the layer in front of the pool: e1 = e_in * [x4 > 0],
+// e3 = Q_e(gamma * e1), sum of e1).  Coding is monotonic in |sum|, so max |e1| is the code of the largest masked
+// |sum|: pass 0 reduces that second maximum as well (into the 64-bit cell), and pass 1 knows both scales, writes
+// e_in (optional) and e3 and adds up e1 - the two kernels of a separate error head and their pass over e_in are gone.
+template <int kPass, bool kNext>
 __global__ void __launch_bounds__(kThreads)
 maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *e_exp, const uint8_t *__restrict__ arg, int n, int h, int w, int c,
-                   int k, int s, int p, int ho, int wo, int8_t *__restrict__ e_in, int32_t *e_in_exp, DeviceState *dev)
+                   int k, int s, int p, int ho, int wo, int8_t *__restrict__ e_in, int32_t *e_in_exp,
+                   const uint8_t *__restrict__ next_mask, const int32_t *next_gamma, int8_t *__restrict__ e3, int32_t *e3_exp,
+                   long long *sum_e1, DeviceState *dev)
 {
     const int groups = c / 16;
     const uint32_t items = (uint32_t)n * h * w * groups;   // below 2^31 (checked by the caller), so i + stride cannot wrap
     int t = 7;
+    NextHead nh = {};
     if (kPass == 1) {
         const uint32_t M = dev->absmax_u32;
         t = M ? round_log2_u32(M) : 7;
+        const int p_in = *e_exp;
+        const int p0 = M ? p_in + t - 7 : p_in;
+        if (kNext) nh = next_head_setup(next_gamma, (uint32_t)abs(sq_code32((int32_t)dev->absmax_u64, t)), dev);
         if (blockIdx.x == 0 && threadIdx.x == 0) {
-            const int p_in = *e_exp;
-            *e_in_exp = M ? p_in + t - 7 : p_in;
+            if (e_in_exp) *e_in_exp = p0;
             if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+            if (kNext) next_head_exponent(nh, p0, e3_exp, dev);
         }
     }
-    uint32_t mx = 0;
+    uint32_t mx = 0, mx_masked = 0;
+    int s1 = 0;
+    long long s1_total = 0;
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < items; i += gridDim.x * blockDim.x) {
         const uint32_t pix = i / (uint32_t)groups, row = pix / (uint32_t)w;
-        const int g = (int)(i - pix * (uint32_t)groups), ix = (int)(pix - row * (uint32_t)w);
+        const int gi = (int)(i - pix * (uint32_t)groups), ix = (int)(pix - row * (uint32_t)w);
         const int b = (int)(row / (uint32_t)h), iy = (int)(row - (uint32_t)b * (uint32_t)h);
         // windows o with o * s - p <= i <= o * s - p + k - 1
         const int oy_lo = max(0, (iy + p - k + s) / s), oy_hi = min(ho - 1, (iy + p) / s);
@@ -115,7 +129,7 @@ maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *e_exp, const uin
         int nwin = 0;
         for (int oy = oy_lo; oy <= oy_hi; ++oy)
             for (int ox = ox_lo; ox <= ox_hi; ++ox) {
-                const size_t o = (((size_t)b * ho + oy) * wo + ox) * c + g * 16;
+                const size_t o = (((size_t)b * ho + oy) * wo + ox) * c + gi * 16;
                 const int4 ev = __ldg(reinterpret_cast<const int4 *>(e + o));
                 const int4 av = __ldg(reinterpret_cast<const int4 *>(arg + o));
                 const uint32_t me = (uint32_t)((iy - (oy * s - p)) * k + (ix - (ox * s - p))) * 0x01010101u;
@@ -138,23 +152,57 @@ maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *e_exp, const uin
             sum[4 * q + 2] = (int)(even[q] >> 16) - 128 * nwin;
             sum[4 * q + 3] = (int)(odd[q] >> 16) - 128 * nwin;
         }
+        const uint32_t mbits = kNext ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(next_mask) + i) : 0u;
         if (kPass == 0) {
 #pragma unroll
-            for (int q = 0; q < 16; ++q) mx = max(mx, (uint32_t)abs(sum[q]));
+            for (int q = 0; q < 16; ++q) {
+                const uint32_t v = (uint32_t)abs(sum[q]);
+                mx = max(mx, v);
+                if (kNext && ((mbits >> q) & 1u)) mx_masked = max(mx_masked, v);
+            }
         } else {
             int cd[16];
 #pragma unroll
             for (int q = 0; q < 16; ++q) cd[q] = sq_code32(sum[q], t);
-            reinterpret_cast<int4 *>(e_in)[i] =
-                make_int4((int)pack4(cd[0], cd[1], cd[2], cd[3]), (int)pack4(cd[4], cd[5], cd[6], cd[7]),
-                          (int)pack4(cd[8], cd[9], cd[10], cd[11]), (int)pack4(cd[12], cd[13], cd[14], cd[15]));
+            if (e_in)
+                reinterpret_cast<int4 *>(e_in)[i] =
+                    make_int4((int)pack4(cd[0], cd[1], cd[2], cd[3]), (int)pack4(cd[4], cd[5], cd[6], cd[7]),
+                              (int)pack4(cd[8], cd[9], cd[10], cd[11]), (int)pack4(cd[12], cd[13], cd[14], cd[15]));
+            if (kNext) {
+                int c3[16];
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    const int e1 = ((mbits >> q) & 1u) ? cd[q] : 0;
+                    s1 += e1;
+                    c3[q] = next_head_code(nh, e1);
+                }
+                reinterpret_cast<int4 *>(e3)[i] =
+                    make_int4((int)pack4(c3[0], c3[1], c3[2], c3[3]), (int)pack4(c3[4], c3[5], c3[6], c3[7]),
+                              (int)pack4(c3[8], c3[9], c3[10], c3[11]), (int)pack4(c3[12], c3[13], c3[14], c3[15]));
+                s1_total += s1;
+                s1 = 0;
+            }
         }
     }
     if (kPass == 0) {
         mx = (uint32_t)block_max_u64(mx);
-        if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u32, mx);
-    } else if (last_block_done(dev)) {
-        dev->absmax_u32 = 0;
+        if (kNext) mx_masked = (uint32_t)block_max_u64(mx_masked);
+        if (threadIdx.x == 0) {
+            if (mx) atomicMax(&dev->absmax_u32, mx);
+            if (kNext && mx_masked) atomicMax(&dev->absmax_u64, (unsigned long long)mx_masked);
+        }
+    } else {
+        if (kNext && sum_e1) {
+            s1_total = block_sum_i64(s1_total);
+            if (threadIdx.x == 0 && s1_total) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum0), (unsigned long long)s1_total);
+        }
+        if (last_block_done(dev)) {
+            dev->absmax_u32 = 0;
+            if (kNext) {
+                dev->absmax_u64 = 0;
+                if (sum_e1) *sum_e1 = (long long)atomicExch(reinterpret_cast<unsigned long long *>(&dev->sum0), 0ull);
+            }
+        }
     }
 }
 
@@ -211,80 +259,131 @@ __device__ __forceinline__ void unpack16(const int4 &v, int (&o)[16])
     for (int k = 0; k < 16; ++k) o[k] = b[k];
 }
 
-// pass = 0: max |S| into the handle's 64-bit cell; pass = 1: codes of SQ(S), their sum, exponent; cells back to zero
-template <int kPass>
+// pass = 0: max |S| into the handle's 64-bit cell; pass = 1: codes of SQ(S), their sum, exponent; cells back to zero.
+// kNext: the error head of the layer that consumes the joined error rides along (see NextHead): pass 0 also reduces
+// the maximum over the positions that layer's ReLU lets through, pass 1 also writes that layer's e3 and its two sums.
+template <int kPass, bool kNext>
 __global__ void join_kernel(const int8_t *__restrict__ a, const int32_t *a_exp, const int8_t *__restrict__ b, const int32_t *b_exp,
                             const uint8_t *__restrict__ mask_b, size_t n16, int8_t *out, int32_t *out_exp, long long *sum_out,
-                            DeviceState *dev)
+                            const uint8_t *__restrict__ next_mask, const int16_t *__restrict__ next_x2, const int32_t *next_gamma,
+                            int8_t *__restrict__ e3, int32_t *e3_exp, long long *sum_e1, long long *sum_e1x2, DeviceState *dev)
 {
     const JoinShift j = join_shift(__ldg(a_exp), __ldg(b_exp));
-    unsigned long long mx = 0;
-    long long sum = 0;
+    unsigned long long mx = 0, mxm = 0;
+    long long sum = 0, s1 = 0, s2 = 0;
     int t = 7;
+    NextHead nh = {};
     if (kPass == 1) {
         const unsigned long long M = dev->absmax_u64;
         t = M ? round_log2_u64(M) : 7;
+        const int p0 = M ? j.p + t - 7 : j.p;
+        if (kNext) {
+            const unsigned long long Mm = dev->absmax2_u64;
+            nh = next_head_setup(next_gamma, (uint32_t)abs(sq_code64((long long)Mm, t)), dev);
+        }
         if (blockIdx.x == 0 && threadIdx.x == 0) {
-            *out_exp = M ? j.p + t - 7 : j.p;
+            *out_exp = p0;
             if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+            if (kNext) next_head_exponent(nh, p0, e3_exp, dev);
         }
     }
     // exponents a few octaves apart (the usual case) keep every sum inside 32 bits: 127 * 2^23 + 127 < 2^31
     const bool narrow = j.sa >= 0 && j.sb >= 0 && j.sa <= 23 && j.sb <= 23;
     const int ma = 1 << (j.sa < 0 ? 0 : min(j.sa, 23)), mb = 1 << (j.sb < 0 ? 0 : min(j.sb, 23));
-    uint32_t mx32 = 0;
-    int sum32 = 0;
+    uint32_t mx32 = 0, mxm32 = 0;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
         int av[16], bv[16];
         unpack16(__ldg(reinterpret_cast<const int4 *>(a) + i), av);
         unpack16(__ldg(reinterpret_cast<const int4 *>(b) + i), bv);
         const uint32_t m = mask_b ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(mask_b) + i) : 0xffffu;
+        const uint32_t nm = kNext ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(next_mask) + i) : 0u;
         int c[16];
         if (narrow) {
 #pragma unroll
             for (int q = 0; q < 16; ++q) {
                 const int s32 = av[q] * ma + (((m >> q) & 1u) ? bv[q] : 0) * mb;
                 if (kPass == 0) {
-                    mx32 = max(mx32, (uint32_t)abs(s32));
+                    const uint32_t v = (uint32_t)abs(s32);
+                    mx32 = max(mx32, v);
+                    if (kNext && ((nm >> q) & 1u)) mxm32 = max(mxm32, v);
                 } else {
                     c[q] = sq_code32(s32, t);
-                    sum32 += c[q];
                 }
             }
-            if (kPass == 1) {
-                sum += sum32;
-                sum32 = 0;
-                reinterpret_cast<int4 *>(out)[i] = make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
-                                                              (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
-            }
-            continue;
-        }
+        } else {
 #pragma unroll
-        for (int q = 0; q < 16; ++q) {
-            const long long s = join_one(av[q], ((m >> q) & 1u) ? bv[q] : 0, j);
-            if (kPass == 0) {
-                const unsigned long long u = (unsigned long long)(s < 0 ? -s : s);
-                mx = u > mx ? u : mx;
-            } else {
-                c[q] = sq_code64(s, t);
-                sum += c[q];
+            for (int q = 0; q < 16; ++q) {
+                const long long s = join_one(av[q], ((m >> q) & 1u) ? bv[q] : 0, j);
+                if (kPass == 0) {
+                    const unsigned long long u = (unsigned long long)(s < 0 ? -s : s);
+                    mx = u > mx ? u : mx;
+                    if (kNext && ((nm >> q) & 1u)) mxm = u > mxm ? u : mxm;
+                } else {
+                    c[q] = sq_code64(s, t);
+                }
             }
         }
-        if (kPass == 1)
+        if (kPass == 1) {
+            int sum32 = 0;
+#pragma unroll
+            for (int q = 0; q < 16; ++q) sum32 += c[q];
+            sum += sum32;
             reinterpret_cast<int4 *>(out)[i] = make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
                                                           (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+            if (kNext) {
+                int e1[16], c3[16], a1 = 0;
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    e1[q] = ((nm >> q) & 1u) ? c[q] : 0;
+                    a1 += e1[q];
+                    c3[q] = next_head_code(nh, e1[q]);
+                }
+                s1 += a1;
+                if (next_x2) {
+                    const int4 lo = __ldg(reinterpret_cast<const int4 *>(next_x2) + 2 * i);
+                    const int4 hi = __ldg(reinterpret_cast<const int4 *>(next_x2) + 2 * i + 1);
+                    const int16_t *pl = reinterpret_cast<const int16_t *>(&lo), *ph = reinterpret_cast<const int16_t *>(&hi);
+                    int a2 = 0;  // |e1 * x2| < 2^22, 16 terms
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) a2 += e1[q] * pl[q] + e1[8 + q] * ph[q];
+                    s2 += a2;
+                }
+                reinterpret_cast<int4 *>(e3)[i] =
+                    make_int4((int)pack4(c3[0], c3[1], c3[2], c3[3]), (int)pack4(c3[4], c3[5], c3[6], c3[7]),
+                              (int)pack4(c3[8], c3[9], c3[10], c3[11]), (int)pack4(c3[12], c3[13], c3[14], c3[15]));
+            }
+        }
     }
     if (kPass == 0) {
         mx = block_max_u64(mx > mx32 ? mx : (unsigned long long)mx32);
-        if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u64, mx);
+        if (kNext) mxm = block_max_u64(mxm > mxm32 ? mxm : (unsigned long long)mxm32);
+        if (threadIdx.x == 0) {
+            if (mx) atomicMax(&dev->absmax_u64, mx);
+            if (kNext && mxm) atomicMax(&dev->absmax2_u64, mxm);
+        }
     } else {
         if (sum_out) {
             sum = block_sum_i64(sum);
             if (threadIdx.x == 0 && sum) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum0), (unsigned long long)sum);
         }
+        if (kNext) {
+            s1 = block_sum_i64(s1);
+            s2 = block_sum_i64(s2);
+            if (threadIdx.x == 0) {
+                if (s1) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum1), (unsigned long long)s1);
+                if (s2) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum2), (unsigned long long)s2);
+            }
+        }
         if (last_block_done(dev)) {
             if (sum_out) *sum_out = (long long)atomicExch(reinterpret_cast<unsigned long long *>(&dev->sum0), 0ull);
             dev->absmax_u64 = 0;
+            if (kNext) {
+                dev->absmax2_u64 = 0;
+                const long long t1 = (long long)atomicExch(reinterpret_cast<unsigned long long *>(&dev->sum1), 0ull);
+                const long long t2 = (long long)atomicExch(reinterpret_cast<unsigned long long *>(&dev->sum2), 0ull);
+                if (sum_e1) *sum_e1 = t1;
+                if (sum_e1x2) *sum_e1x2 = t2;
+            }
         }
     }
 }
@@ -604,14 +703,27 @@ cudaError_t launch_maxpool_fwd(const int8_t *x, int n, int h, int w, int c, int 
 }
 
 cudaError_t launch_maxpool_bwd(const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int h, int w, int c, int k, int s,
-                               int p, int8_t *e_in, int32_t *e_in_exp, DeviceState *dev, int sm_count, cudaStream_t st,
+                               int p, int8_t *e_in, int32_t *e_in_exp, const uint8_t *next_mask, const int32_t *next_gamma, int8_t *e3,
+                               int32_t *e3_exp, long long *sum_e1, DeviceState *dev, int sm_count, cudaStream_t st,
                                const ReduceHook &hook)
 {
     const int ho = (h + 2 * p - k) / s + 1, wo = (w + 2 * p - k) / s + 1;
     const int blocks = blocks_for((size_t)n * h * w * (c / 16), sm_count, 32);
-    maxpool_bwd_kernel<0><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, dev);
-    hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, st);
-    maxpool_bwd_kernel<1><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, dev);
+    if (e3) {
+        maxpool_bwd_kernel<0, true><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, next_mask,
+                                                                 next_gamma, e3, e3_exp, sum_e1, dev);
+        hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, st);
+        hook(&dev->absmax_u64, 1, EOQ_REDUCE_I64, EOQ_REDUCE_MAX, st);
+        maxpool_bwd_kernel<1, true><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, next_mask,
+                                                                 next_gamma, e3, e3_exp, sum_e1, dev);
+        if (sum_e1) hook(sum_e1, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, st);
+    } else {
+        maxpool_bwd_kernel<0, false><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, nullptr,
+                                                                  nullptr, nullptr, nullptr, nullptr, dev);
+        hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, st);
+        maxpool_bwd_kernel<1, false><<<blocks, kThreads, 0, st>>>(e, e_exp, arg, n, h, w, c, k, s, p, ho, wo, e_in, e_in_exp, nullptr,
+                                                                  nullptr, nullptr, nullptr, nullptr, dev);
+    }
     return cudaGetLastError();
 }
 
@@ -622,15 +734,30 @@ cudaError_t launch_avgpool_sum(const int8_t *x, int n, int hw, int c, int32_t *s
 }
 
 cudaError_t launch_join(const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp, const uint8_t *mask_b,
-                        size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, DeviceState *dev, int sm_count,
-                        cudaStream_t st, const ReduceHook &hook)
+                        size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, const uint8_t *next_mask,
+                        const int16_t *next_x2, const int32_t *next_gamma, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
+                        long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t st, const ReduceHook &hook)
 {
     const size_t n16 = n_el / 16;
     const int blocks = blocks_for(n16, sm_count, 8);
-    join_kernel<0><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, dev);
-    hook(&dev->absmax_u64, 1, EOQ_REDUCE_I64, EOQ_REDUCE_MAX, st);
-    join_kernel<1><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, dev);
-    if (sum_out) hook(sum_out, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, st);
+    if (e3) {
+        join_kernel<0, true><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, next_mask, next_x2,
+                                                          next_gamma, e3, e3_exp, sum_e1, sum_e1x2, dev);
+        hook(&dev->absmax_u64, 1, EOQ_REDUCE_I64, EOQ_REDUCE_MAX, st);
+        hook(&dev->absmax2_u64, 1, EOQ_REDUCE_I64, EOQ_REDUCE_MAX, st);
+        join_kernel<1, true><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, next_mask, next_x2,
+                                                          next_gamma, e3, e3_exp, sum_e1, sum_e1x2, dev);
+        if (sum_out) hook(sum_out, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, st);
+        if (sum_e1) hook(sum_e1, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, st);
+        if (sum_e1x2) hook(sum_e1x2, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, st);
+    } else {
+        join_kernel<0, false><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, nullptr, nullptr,
+                                                           nullptr, nullptr, nullptr, nullptr, nullptr, dev);
+        hook(&dev->absmax_u64, 1, EOQ_REDUCE_I64, EOQ_REDUCE_MAX, st);
+        join_kernel<1, false><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, nullptr, nullptr,
+                                                           nullptr, nullptr, nullptr, nullptr, nullptr, dev);
+        if (sum_out) hook(sum_out, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, st);
+    }
     return cudaGetLastError();
 }
 
@@ -649,6 +776,13 @@ cudaError_t launch_head(const int32_t *sums, int n, int c, int hw, int classes, 
     head_softmax_kernel<<<n, 256, 0, st>>>(logits, n, classes, labels, dl, loss_n);
     head_dpooled_kernel<<<dim3((c + kDpCh - 1) / kDpCh, (n + kDpN - 1) / kDpN), kDpCh * kDpN, 0, st>>>(dl, W, n, c, classes, dpooled,
                                                                                                    loss_n, loss_out);
+    if (lr != 0.0f) head_update_kernel<<<(classes * c + 127) / 128, 128, 0, st>>>(dl, pooled, n, c, classes, lr, W, bias);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_head_update(const float *dl, const float *pooled, int n, int c, int classes, float lr, float *W, float *bias,
+                               cudaStream_t st)
+{
     head_update_kernel<<<(classes * c + 127) / 128, 128, 0, st>>>(dl, pooled, n, c, classes, lr, W, bias);
     return cudaGetLastError();
 }

@@ -4,6 +4,7 @@
 // Reductions run warp-shuffle -> one atomic per warp; 16 elements per thread with 128-bit accesses.
 #include "eoq_device.cuh"
 #include "eoq_internal.h"
+#include "eoq_next_head.cuh"
 
 namespace eoq {
 
@@ -227,17 +228,25 @@ __global__ void absmax_i32_kernel(const int32_t *__restrict__ src, size_t n, Dev
     if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u32, mx);
 }
 
+// kNext: the error head of the layer that consumes dst rides along (see NextHead): the masked maximum sits in the
+// handle's 64-bit cell (the GEMM epilogue reduced it beside the plain one), so the codes of e3 and the head's sums
+// come out of the same pass.  n must then be a multiple of 16.
+template <bool kNext>
 __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *src_exp, int exp_bias, size_t n,
-                              int8_t *dst, int32_t *dst_exp, long long *sum_codes, DeviceState *dev)
+                              int8_t *dst, int32_t *dst_exp, long long *sum_codes, NextHeadArgs next, DeviceState *dev)
 {
     const uint32_t M = dev->absmax_u32;
     const int t = M ? round_log2_u32(M) : 7;
+    const int p_in = (src_exp ? *src_exp : 0) + exp_bias;
+    const int p0 = M ? p_in + t - 7 : p_in;
+    NextHead nh = {};
+    if (kNext) nh = next_head_setup(next.gamma, (uint32_t)abs(sq_code32((int32_t)dev->absmax_u64, t)), dev);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
-        const int p_in = (src_exp ? *src_exp : 0) + exp_bias;
-        *dst_exp = M ? p_in + t - 7 : p_in;
+        *dst_exp = p0;
         if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+        if (kNext) next_head_exponent(nh, p0, next.e3_exp, dev);
     }
-    long long sum = 0;
+    long long sum = 0, s1 = 0, s2 = 0;
     const size_t n16 = n / 16;
     const int4 *s4 = reinterpret_cast<const int4 *>(src);
     const int sh = t - 7;
@@ -272,19 +281,58 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
         reinterpret_cast<int4 *>(dst)[i] =
             make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
                       (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+        if (kNext) {
+            const uint32_t bits = (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(next.mask) + i);
+            int e1[16], c3[16], a1 = 0;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                e1[k] = ((bits >> k) & 1u) ? c[k] : 0;
+                a1 += e1[k];
+                c3[k] = next_head_code(nh, e1[k]);
+            }
+            s1 += a1;
+            if (next.x2) {
+                const int4 lo = __ldg(reinterpret_cast<const int4 *>(next.x2) + 2 * i);
+                const int4 hi = __ldg(reinterpret_cast<const int4 *>(next.x2) + 2 * i + 1);
+                const int16_t *pl = reinterpret_cast<const int16_t *>(&lo), *ph = reinterpret_cast<const int16_t *>(&hi);
+                int a2 = 0;  // |e1 * x2| < 2^22, 16 terms
+#pragma unroll
+                for (int k = 0; k < 8; ++k) a2 += e1[k] * pl[k] + e1[8 + k] * ph[k];
+                s2 += a2;
+            }
+            reinterpret_cast<int4 *>(next.e3)[i] =
+                make_int4((int)pack4(c3[0], c3[1], c3[2], c3[3]), (int)pack4(c3[4], c3[5], c3[6], c3[7]),
+                          (int)pack4(c3[8], c3[9], c3[10], c3[11]), (int)pack4(c3[12], c3[13], c3[14], c3[15]));
+        }
     }
-    for (size_t i = n16 * 16 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        const int c = sq_code32(src[i], t);
-        sum += c;
-        dst[i] = (int8_t)c;
-    }
+    if (!kNext)
+        for (size_t i = n16 * 16 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+            const int c = sq_code32(src[i], t);
+            sum += c;
+            dst[i] = (int8_t)c;
+        }
     if (sum_codes) {
         sum = block_sum_i64(sum);
         if (threadIdx.x == 0 && sum) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum0), (unsigned long long)sum);
     }
+    if (kNext) {
+        s1 = block_sum_i64(s1);
+        s2 = block_sum_i64(s2);
+        if (threadIdx.x == 0) {
+            if (s1) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum1), (unsigned long long)s1);
+            if (s2) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum2), (unsigned long long)s2);
+        }
+    }
     if (last_block_done(dev)) {
         if (sum_codes) *sum_codes = (long long)atomicExch(reinterpret_cast<unsigned long long *>(&dev->sum0), 0ull);
         dev->absmax_u32 = 0;
+        if (kNext) {
+            dev->absmax_u64 = 0;
+            const long long t1 = (long long)atomicExch(reinterpret_cast<unsigned long long *>(&dev->sum1), 0ull);
+            const long long t2 = (long long)atomicExch(reinterpret_cast<unsigned long long *>(&dev->sum2), 0ull);
+            if (next.sum_e1) *next.sum_e1 = t1;
+            if (next.sum_e1x2) *next.sum_e1x2 = t2;
+        }
     }
 }
 
@@ -1159,11 +1207,21 @@ cudaError_t launch_weight_pad_rows(const int8_t *w, int8_t *wp, int c_out, int k
 
 cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *sum_codes, bool max_already_reduced, DeviceState *dev,
-                          int sm_count, cudaStream_t s, const ReduceHook &hook)
+                          int sm_count, cudaStream_t s, const ReduceHook &hook, const NextHeadArgs *next)
 {
     if (!max_already_reduced) absmax_i32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
     hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, s);
-    sq_i32_kernel<<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes, dev);
+    if (next) {
+        // (only behind a GEMM whose epilogue reduced the masked maximum)
+        hook(&dev->absmax_u64, 1, EOQ_REDUCE_I64, EOQ_REDUCE_MAX, s);
+        sq_i32_kernel<true><<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes, *next,
+                                                                              dev);
+        if (next->sum_e1) hook(next->sum_e1, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, s);
+        if (next->sum_e1x2) hook(next->sum_e1x2, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, s);
+    } else {
+        sq_i32_kernel<false><<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes,
+                                                                               NextHeadArgs{}, dev);
+    }
     if (sum_codes) hook(sum_codes, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, s);
     return cudaGetLastError();
 }

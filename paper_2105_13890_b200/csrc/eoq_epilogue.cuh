@@ -233,17 +233,25 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const FwdScalar
 
 // Error back-propagation: keep the exact int32 sums (the scale quantizer needs the maximum over the whole
 // tensor before any element can be coded) and track max |.|.
-__device__ __forceinline__ uint32_t dgrad_16(const IgemmParams &p, const uint32_t *acc, size_t off)
+__device__ __forceinline__ uint32_t dgrad_16(const IgemmParams &p, const uint32_t *acc, size_t off, uint32_t &mx_masked)
 {
     uint32_t mx = 0;
     int4 *d = reinterpret_cast<int4 *>(p.acc_out + off);
+    // the consumer's error head needs the maximum over the positions its ReLU lets through as well (off is the element
+    // index of the error tensor and a multiple of 16: one 16-bit word of mask bits)
+    const uint32_t bits = p.next_mask ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p.next_mask) + (off >> 4)) : 0u;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         int4 v = make_int4((int)acc[4 * i], (int)acc[4 * i + 1], (int)acc[4 * i + 2], (int)acc[4 * i + 3]);
-        mx = max(mx, (uint32_t)abs(v.x));
-        mx = max(mx, (uint32_t)abs(v.y));
-        mx = max(mx, (uint32_t)abs(v.z));
-        mx = max(mx, (uint32_t)abs(v.w));
+        const uint32_t a0 = (uint32_t)abs(v.x), a1 = (uint32_t)abs(v.y), a2 = (uint32_t)abs(v.z), a3 = (uint32_t)abs(v.w);
+        mx = max(max(mx, a0), max(a1, max(a2, a3)));
+        if (bits) {
+            const uint32_t b4 = bits >> (4 * i);
+            mx_masked = max(mx_masked, (b4 & 1u) ? a0 : 0u);
+            mx_masked = max(mx_masked, (b4 & 2u) ? a1 : 0u);
+            mx_masked = max(mx_masked, (b4 & 4u) ? a2 : 0u);
+            mx_masked = max(mx_masked, (b4 & 8u) ? a3 : 0u);
+        }
         d[i] = v;
     }
     return mx;

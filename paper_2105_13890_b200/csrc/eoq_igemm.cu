@@ -238,7 +238,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                 shift = max(-16, min(31, shift));
             }
         }
-        uint32_t acc_phase = 0, mx = 0;
+        uint32_t acc_phase = 0, mx = 0, mx_masked = 0;
         bool ok = true;
         for (int tile = blockIdx.x + grp * gridDim.x; tile < num_tiles && ok; tile += 2 * gridDim.x) {
             const int mt = tile / p.num_n_tiles, nt = tile % p.num_n_tiles;
@@ -298,7 +298,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                             else forward_16<false, false, false>(p, fs, r, r2, off, tb, tg, sc, shift);
                         }
                     } else {
-                        mx = max(mx, dgrad_16(p, r, off));
+                        mx = max(mx, dgrad_16(p, r, off, mx_masked));
                     }
                 }
                 sc = sc_next;
@@ -313,6 +313,10 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
         if (p.epilogue == kEpiDgrad) {
             mx = warp_max_u32(mx);
             if (lane == 0 && mx) atomicMax(&p.dev->absmax_u32, mx);
+            if (p.next_mask) {
+                mx_masked = warp_max_u32(mx_masked);
+                if (lane == 0 && mx_masked) atomicMax(&p.dev->absmax_u64, (unsigned long long)mx_masked);
+            }
         }
     }
 

@@ -272,7 +272,7 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
         const int32_t *ts = fwd ? stage_b1_table(p, fs.b1, smem_raw + (smem_base - ptx::smem_u32(smem_raw)) + table_off,
                                                  (int)threadIdx.x - 128, 32 * kEpilogueWarps)
                                 : nullptr;
-        uint32_t acc_phase = 0, mx = 0;
+        uint32_t acc_phase = 0, mx = 0, mx_masked = 0;
         bool ok = true;
         // (column tile, image, row tile in the image) of the current tile, carried from tile to tile: the step
         // between two tiles of this pair is constant, so its quotients are formed once instead of four integer
@@ -327,7 +327,7 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                             else forward_16<true, false, false>(p, fs, r, r2, off, tb, tg, sc, 7);
                         }
                     }
-                    else mx = max(mx, dgrad_16(p, r, off));
+                    else mx = max(mx, dgrad_16(p, r, off, mx_masked));
                 }
                 sc = sc_next;
                 if (tb) tb += 16;
@@ -347,6 +347,10 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
         if (p.epilogue == kEpiDgrad) {
             mx = warp_max_u32(mx);
             if (lane == 0 && mx) atomicMax(&p.dev->absmax_u32, mx);
+            if (p.next_mask) {
+                mx_masked = warp_max_u32(mx_masked);
+                if (lane == 0 && mx_masked) atomicMax(&p.dev->absmax_u64, (unsigned long long)mx_masked);
+            }
         }
     }
     ptx::tc_fence_before();

@@ -21,18 +21,31 @@ struct DeviceState {
     unsigned absmax_u32;   // reduction cell for |.| maxima (int32 sources, float bit patterns)
     unsigned long long absmax_u64;
     long long sum0, sum1;  // reduction cells for integer sums
+    unsigned long long absmax2_u64;  // second maximum of a call that also serves its consumer's error head (masked |.|)
+    long long sum2;                  // third sum of such a call
     unsigned tensor_absmax[256];  // per-tensor maxima of the multi-tensor update
     unsigned ticket;       // blocks of the kernel that consumes the cells last count themselves here (see last_block_done)
     unsigned arrivals;     // grid-wide barrier of the one-kernel error head (cooperative launch)
     unsigned long long probe_cycles;  // eoq_probe_mma_i8: longest issue loop of the last launch, in SM clock cycles
 };
-// Invariant: absmax_u32, absmax_u64, sum0, sum1, ticket and arrivals are zero whenever no call is in flight on the handle.
+// Invariant: absmax_u32, absmax_u64, absmax2_u64, sum0, sum1, sum2, ticket and arrivals are zero whenever no call is in flight on the handle.
 // The kernel that reads a call's reductions last puts the cells it used back to zero (its last block does), so
 // no call starts with a memset.  A kernel that gave up on a wait (EOQ_DEV_TIMEOUT) may leave them dirty:
 // eoq_last_status clears them again when it reports that bit.
 
 // eoq_set_reduce_hook: called on the host between the kernel that forms a value reduced over the batch and the kernel
 // that consumes it; it enqueues an all-reduce of the device buffer on the stream (no-op when no hook is set).
+// The error head of the layer that consumes an error tensor, fused into the second pass of the kernel that produces it
+// (eoq_conv_dgrad_head, eoq_aux_join_head, eoq_aux_maxpool_bwd_head).
+struct NextHeadArgs {
+    const uint8_t *mask;      // that layer's ReLU mask bits
+    const int16_t *x2;        // its x2, or null
+    const int32_t *gamma;     // its gamma code (device)
+    int8_t *e3;
+    int32_t *e3_exp;
+    long long *sum_e1, *sum_e1x2;
+};
+
 struct ReduceHook {
     eoq_reduce_fn fn;
     void *user;
@@ -111,6 +124,7 @@ struct IgemmParams {
     const int32_t *x_exp;     // device exponent of the input or null
     int32_t b1_c, gamma_c, b2_c;
     const int32_t *scal_dev;  // device {b1_c, gamma_c, b2_c} replacing the three host values, or null
+    const uint8_t *next_mask; // dgrad: ReLU mask bits of the layer that consumes the error (its head rides on Q_e), or null
     int k_total;              // taps * input channels: bounds the accumulator when b1 is only known on the device
     const int32_t *b1_table;  // [classes][N] tap-validity sums of the weights (null when b1_c == 0)
     int b1_nlo_h, b1_nhi_h, b1_nrc, b1_nlo_w, b1_nhi_w, b1_ncc;
@@ -234,7 +248,7 @@ cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst,
                                 int sm_count, cudaStream_t s, const ReduceHook &hook);
 cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *sum_codes, bool max_already_reduced, DeviceState *dev,
-                          int sm_count, cudaStream_t s, const ReduceHook &hook);
+                          int sm_count, cudaStream_t s, const ReduceHook &hook, const NextHeadArgs *next = nullptr);
 // Q_g of the exact sums.  `src` holds int64 sums; when `parts` is given the sums are first formed from
 // `num_parts` int32 slices of n elements each (and written to src).
 cudaError_t launch_sq_i32_scatter(const int32_t *src, const int32_t *src_exp, int exp_bias, int n_img, int hh, int ww, int c,
@@ -304,15 +318,19 @@ cudaError_t launch_weight_prep(const PrepBatch &b, cudaStream_t s);
 cudaError_t launch_maxpool_fwd(const int8_t *x, int n, int h, int w, int c, int k, int s, int p, int8_t *y, uint8_t *arg,
                                int sm_count, cudaStream_t st);
 cudaError_t launch_maxpool_bwd(const int8_t *e, const int32_t *e_exp, const uint8_t *arg, int n, int h, int w, int c, int k, int s,
-                               int p, int8_t *e_in, int32_t *e_in_exp, DeviceState *dev, int sm_count, cudaStream_t st,
+                               int p, int8_t *e_in, int32_t *e_in_exp, const uint8_t *next_mask, const int32_t *next_gamma, int8_t *e3,
+                               int32_t *e3_exp, long long *sum_e1, DeviceState *dev, int sm_count, cudaStream_t st,
                                const ReduceHook &hook);
 cudaError_t launch_avgpool_sum(const int8_t *x, int n, int hw, int c, int32_t *sums, cudaStream_t st);
 cudaError_t launch_join(const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp, const uint8_t *mask_b,
-                        size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, DeviceState *dev, int sm_count,
-                        cudaStream_t st, const ReduceHook &hook);
+                        size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, const uint8_t *next_mask,
+                        const int16_t *next_x2, const int32_t *next_gamma, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
+                        long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t st, const ReduceHook &hook);
 cudaError_t launch_head(const int32_t *sums, int n, int c, int hw, int classes, float *W, float *bias, const int32_t *labels,
                         float lr, float *loss_out, float *dpooled, float *logits, float *pooled, float *dl, double *loss_n,
                         cudaStream_t st);
+cudaError_t launch_head_update(const float *dl, const float *pooled, int n, int c, int classes, float lr, float *W, float *bias,
+                               cudaStream_t st);
 cudaError_t launch_head_error(const float *dpooled, int n, int c, int hw, float *ef, int8_t *e, int32_t *e_exp, DeviceState *dev,
                               int sm_count, cudaStream_t st, const ReduceHook &hook);
 struct ScalarItem {

@@ -27,7 +27,7 @@ EXPORTS = [
     "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count", "eoq_set_gemm_ctas",
     "eoq_conv_dgrad_static", "eoq_conv_fwd_dev", "eoq_weight_prep_size", "eoq_weight_prep", "eoq_conv_wgrad_dev",
     "eoq_err_prescale_dev", "eoq_update_dev", "eoq_describe_plan", "eoq_debug_force_wait_timeout", "eoq_probe_mma_i8", "eoq_profile_gemm_only", "eoq_aux_maxpool_fwd", "eoq_aux_maxpool_bwd",
-    "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide", "eoq_set_reduce_hook", "eoq_bn_workspace_size", "eoq_bn_fwd", "eoq_bn_bwd",
+    "eoq_aux_maxpool_bwd_head", "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_join_head", "eoq_conv_dgrad_head", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_update", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide", "eoq_set_reduce_hook", "eoq_bn_workspace_size", "eoq_bn_fwd", "eoq_bn_bwd",
 ]
 EOQ_STATIC_SCRATCH_BYTES = 16 << 20
 EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
@@ -109,10 +109,14 @@ def lib() -> C.CDLL:
         ci = C.c_int
         L.eoq_aux_maxpool_fwd.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp]
         L.eoq_aux_maxpool_bwd.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp]
+        L.eoq_aux_maxpool_bwd_head.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
         L.eoq_aux_avgpool_sum.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         L.eoq_aux_join.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp, vp, vp, vp]
+        L.eoq_conv_dgrad_head.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.eoq_aux_join_head.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.eoq_aux_head_workspace_size.argtypes = [ci, ci, ci, C.POINTER(sz)]
         L.eoq_aux_head.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp, C.c_float, vp, vp, vp, vp, sz, vp]
+        L.eoq_aux_head_update.argtypes = [vp, ci, ci, ci, vp, vp, C.c_float, vp, sz, vp]
         L.eoq_aux_head_error.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, sz, vp]
         L.eoq_aux_scalar_update.argtypes = [vp, ci, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(ci),
                                             C.POINTER(ci), C.POINTER(vp), i32, i32, ci, u64, vp, vp]
@@ -389,6 +393,13 @@ def eoq_aux_maxpool_bwd(handle, e, e_exp, arg, n, h, w, c, k, stride, pad, e_in,
                                      _ptr(e_in_exp), _stream(stream)), "eoq_aux_maxpool_bwd")
 
 
+def eoq_aux_maxpool_bwd_head(handle, e, e_exp, arg, n, h, w, c, k, stride, pad, e_in, e_in_exp, relu_mask, gamma, e3, e3_exp,
+                             sum_e1=None, stream=None) -> None:
+    _check(lib().eoq_aux_maxpool_bwd_head(handle, _ptr(e), _ptr(e_exp), _ptr(arg), n, h, w, c, k, stride, pad, _ptr(e_in),
+                                          _ptr(e_in_exp), _ptr(relu_mask), _ptr(gamma), _ptr(e3), _ptr(e3_exp), _ptr(sum_e1),
+                                          _stream(stream)), "eoq_aux_maxpool_bwd_head")
+
+
 def eoq_bn_workspace_size(c) -> int:
     out = C.c_size_t(0)
     _check(lib().eoq_bn_workspace_size(c, C.byref(out)), "eoq_bn_workspace_size")
@@ -415,6 +426,21 @@ def eoq_aux_join(handle, a, a_exp, b, b_exp, mask_b, n_el, out, out_exp, sum_out
                               _ptr(out_exp), _ptr(sum_out), _stream(stream)), "eoq_aux_join")
 
 
+def eoq_conv_dgrad_head(handle, desc, e3, e3_exp, w, e4, e4_exp, sum_e4, next_mask, next_x2, next_gamma, next_e3, next_e3_exp,
+                        next_sum_e1=None, next_sum_e1x2=None, workspace=None, stream=None) -> None:
+    _check(lib().eoq_conv_dgrad_head(handle, C.byref(desc), _ptr(e3), _ptr(e3_exp), _ptr(w), _ptr(e4), _ptr(e4_exp), _ptr(sum_e4),
+                                     _ptr(next_mask), _ptr(next_x2), _ptr(next_gamma), _ptr(next_e3), _ptr(next_e3_exp),
+                                     _ptr(next_sum_e1), _ptr(next_sum_e1x2), _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "eoq_conv_dgrad_head")
+
+
+def eoq_aux_join_head(handle, a, a_exp, b, b_exp, mask_b, n_el, out, out_exp, sum_out, relu_mask, x2, gamma, e3, e3_exp, sum_e1=None,
+                      sum_e1x2=None, stream=None) -> None:
+    _check(lib().eoq_aux_join_head(handle, _ptr(a), _ptr(a_exp), _ptr(b), _ptr(b_exp), _ptr(mask_b), int(n_el), _ptr(out), _ptr(out_exp),
+                                   _ptr(sum_out), _ptr(relu_mask), _ptr(x2), _ptr(gamma), _ptr(e3), _ptr(e3_exp), _ptr(sum_e1),
+                                   _ptr(sum_e1x2), _stream(stream)), "eoq_aux_join_head")
+
+
 def eoq_aux_head_workspace_size(n, c, classes) -> int:
     out = C.c_size_t(0)
     _check(lib().eoq_aux_head_workspace_size(n, c, classes, C.byref(out)), "eoq_aux_head_workspace_size")
@@ -424,6 +450,11 @@ def eoq_aux_head_workspace_size(n, c, classes) -> int:
 def eoq_aux_head(handle, sums, n, c, hw, classes, W, bias, labels, lr, loss, dpooled, logits, workspace, stream=None) -> None:
     _check(lib().eoq_aux_head(handle, _ptr(sums), n, c, hw, classes, _ptr(W), _ptr(bias), _ptr(labels), float(lr), _ptr(loss),
                               _ptr(dpooled), _ptr(logits), _ptr(workspace), _nbytes(workspace), _stream(stream)), "eoq_aux_head")
+
+
+def eoq_aux_head_update(handle, n, c, classes, W, bias, lr, workspace, stream=None) -> None:
+    _check(lib().eoq_aux_head_update(handle, n, c, classes, _ptr(W), _ptr(bias), lr, _ptr(workspace), _nbytes(workspace),
+                                     _stream(stream)), "eoq_aux_head_update")
 
 
 def eoq_aux_head_error(handle, dpooled, n, c, hw, e, e_exp, workspace, stream=None) -> None:

@@ -6,6 +6,7 @@ import pytest
 import torch
 
 import oracle
+from oracle import ConvDesc
 from paper_2105_13890_b200 import eoq, synth
 
 import gpu_util as G
@@ -54,6 +55,36 @@ def test_maxpool_forward_and_backward(n, h, w, c, k, s, p, ties):
     assert eoq.eoq_last_status(hd) == 0
 
 
+@pytest.mark.parametrize("n,h,w,c,k,s,p", POOLS[:4] + POOLS[5:])
+@pytest.mark.parametrize("gamma", [128, 37, -300])
+def test_maxpool_backward_with_the_error_head_fused(n, h, w, c, k, s, p, gamma):
+    """eoq_aux_maxpool_bwd_head against the oracle's pool backward followed by its error head, and against the two
+    separate GPU calls; with and without the intermediate error written."""
+    hd = G.handle()
+    x = synth.relu_codes((n, h, w, c), 8150 + h, 0)
+    _, idx = oracle.maxpool_fwd(x, k, s, p)
+    ho, wo = idx.shape[1:3]
+    e = synth.normal_codes((n, ho, wo, c), 8150 + h, 1)
+    mask01 = synth.bits((n, h, w, c), 8150 + h, 2, 0.55)
+    S = oracle.maxpool_bwd(e, idx, x.shape)
+    e0, p0, _ = oracle.sq_int(S, -12)
+    want_e3, want_p3, want_s1, _, _ = oracle.err_prescale(e0.astype(np.int8), p0, mask01, None, gamma)
+    y, arg = G.zeros((n, ho, wo, c), torch.int8), G.zeros((n, ho, wo, c), torch.uint8)
+    eoq.eoq_aux_maxpool_fwd(hd, G.dev(x), n, h, w, c, k, s, p, y, arg)
+    g_d = i32(gamma)
+    for keep in (True, False):
+        ein, pin = G.zeros(x.shape, torch.int8), G.zeros(1, torch.int32)
+        e3, p3, s1 = G.zeros(x.shape, torch.int8), G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+        eoq.eoq_aux_maxpool_bwd_head(hd, G.dev(e), i32(-12), arg, n, h, w, c, k, s, p, ein if keep else None, pin, G.dev(G.pack_mask(mask01)),
+                                     g_d, e3, p3, s1)
+        torch.cuda.synchronize()
+        assert eoq.eoq_last_status(hd) == 0
+        if keep:
+            assert np.array_equal(G.host(ein), e0)
+        assert pin.item() == p0
+        assert np.array_equal(G.host(e3), want_e3) and p3.item() == want_p3 and s1.item() == want_s1
+
+
 def test_maxpool_backward_of_a_zero_error_keeps_the_exponent():
     hd = G.handle()
     n, h, w, c = 1, 6, 6, 16
@@ -98,6 +129,38 @@ def test_join(pa, pb, gated):
     assert eoq.eoq_last_status(hd) == 0
 
 
+@pytest.mark.parametrize("pa,pb", [(-12, -12), (-11, -14), (-10, -36), (-40, -5)])
+@pytest.mark.parametrize("gamma,with_x2", [(118, True), (128, False), (-77, True)])
+def test_join_with_the_consumer_error_head_fused(pa, pb, gamma, with_x2):
+    """eoq_aux_join_head against the oracle's join followed by its error head (both 32- and 64-bit paths of the join)."""
+    hd = G.handle()
+    shape = (3, 9, 7, 48)
+    a = synth.normal_codes(shape, 8450, 0)
+    b = synth.normal_codes(shape, 8450, 1)
+    gate01 = (synth.relu_codes(shape, 8450, 2) > 0).astype(np.uint8)
+    mask01 = synth.bits(shape, 8450, 3, 0.5)
+    x2 = (synth.relu_codes(shape, 8450, 4).astype(np.int32) * 37 - 900).astype(np.int16) if with_x2 else None
+    S, p = oracle.join(a, pa, b, pb, gate01)
+    codes, p_out, _ = oracle.sq_int(S, p)
+    want_e3, want_p3, want_s1, want_s2, _ = oracle.err_prescale(codes.astype(np.int8), p_out, mask01, x2, gamma)
+    out, pout, ssum = G.zeros(shape, torch.int8), G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+    e3, p3 = G.zeros(shape, torch.int8), G.zeros(1, torch.int32)
+    s1, s2 = G.zeros(1, torch.int64), G.zeros(1, torch.int64)
+    eoq.eoq_aux_join_head(hd, G.dev(a), i32(pa), G.dev(b), i32(pb), G.dev(G.pack_mask(gate01)), a.size, out, pout, ssum,
+                          G.dev(G.pack_mask(mask01)), G.dev(x2) if with_x2 else None, i32(gamma), e3, p3, s1, s2 if with_x2 else None)
+    torch.cuda.synchronize()
+    assert eoq.eoq_last_status(hd) == 0
+    assert np.array_equal(G.host(out), codes) and pout.item() == p_out and ssum.item() == int(codes.astype(np.int64).sum())
+    assert np.array_equal(G.host(e3), want_e3) and p3.item() == want_p3 and s1.item() == want_s1
+    if with_x2:
+        assert s2.item() == want_s2
+    # the handle's cells are clean again: a plain join right after gives the plain result
+    out2, pout2 = G.zeros(shape, torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_aux_join(hd, G.dev(a), i32(pa), G.dev(b), i32(pb), G.dev(G.pack_mask(gate01)), a.size, out2, pout2, None)
+    torch.cuda.synchronize()
+    assert np.array_equal(G.host(out2), codes) and pout2.item() == p_out
+
+
 @pytest.mark.parametrize("n,c,hw,classes", [(2, 64, 64, 10), (5, 512, 49, 1000), (33, 64, 64, 10), (64, 512, 49, 1000)])
 def test_float_head_bit_for_bit(n, c, hw, classes):
     hd = G.handle()
@@ -118,8 +181,70 @@ def test_float_head_bit_for_bit(n, c, hw, classes):
     assert np.array_equal(G.host(dpooled), dpooled_o)
     assert np.array_equal(G.host(W_d), W_o) and np.array_equal(G.host(bias_d), bias_o)
     assert loss.item() == pytest.approx(loss_o, rel=1e-6)
+    # the SGD step taken apart from the rest gives the same parameters
+    W2, bias2 = G.dev(W), G.dev(bias)
+    eoq.eoq_aux_head(hd, G.dev(sums.astype(np.int32)), n, c, hw, classes, W2, bias2, G.dev(labels), 0.0, loss, dpooled, logits, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(G.host(W2), W) and np.array_equal(G.host(bias2), bias) and np.array_equal(G.host(dpooled), dpooled_o)
+    eoq.eoq_aux_head_update(hd, n, c, classes, W2, bias2, 2.0 ** -6, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(G.host(W2), W_o) and np.array_equal(G.host(bias2), bias_o)
     # the error handed back: SQ of dpooled / hw, the same code at every position of a (sample, channel)
     codes, p_e, _ = oracle.quantize_f32(oracle.MODE_SQ, (dpooled_o / np.float32(hw)).astype(np.float32))
     got = G.host(e).reshape(n, hw, c)
     assert pe.item() == p_e and all(np.array_equal(got[:, i, :], codes) for i in (0, hw // 2, hw - 1))
     assert eoq.eoq_last_status(hd) == 0
+
+
+DGRADS = [  # n, h, w, c_in, c_out, k, stride, pad
+    (2, 12, 12, 32, 32, 3, 1, 1),      # patch kernel
+    (3, 7, 7, 64, 128, 3, 1, 1),       # small image: per-tap kernel
+    (2, 10, 10, 32, 64, 3, 2, 1),      # strided: four residue classes side by side
+    (2, 9, 11, 48, 32, 1, 1, 0),       # 1x1
+    (1, 20, 20, 64, 64, 5, 1, 2),
+]
+
+
+@pytest.mark.parametrize("n,h,w,c_in,c_out,k,stride,pad", DGRADS)
+@pytest.mark.parametrize("gamma,with_x2", [(128, False), (91, True)])
+def test_dgrad_with_the_consumer_error_head_fused(n, h, w, c_in, c_out, k, stride, pad, gamma, with_x2):
+    """eoq_conv_dgrad_head against the oracle's dgrad + Q_e followed by its error head."""
+    hd = G.handle()
+    d = ConvDesc(n, h, w, c_in, c_out, k, k, stride, pad)
+    gd = G.gdesc(d)
+    e3 = synth.normal_codes((n, d.ho, d.wo, c_out), 8600 + h, 0)
+    wt = synth.int8_uniform((c_out, k, k, c_in), 8600 + h, 1, -30, 30)
+    in_shape = (n, h, w, c_in)
+    mask01 = synth.bits(in_shape, 8600 + h, 2, 0.5)
+    x2 = (synth.relu_codes(in_shape, 8600 + h, 3).astype(np.int32) * 29 - 700).astype(np.int16) if with_x2 else None
+    S = oracle.conv_dgrad_acc(d, e3, wt)
+    e4_o, p4_o, _ = oracle.sq_int(S, -11 - 7)
+    want_e3, want_p3, want_s1, want_s2, _ = oracle.err_prescale(e4_o.astype(np.int8), p4_o, mask01, x2, gamma)
+    e4, p4, s4 = G.zeros(in_shape, torch.int8), G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+    n3, pn3 = G.zeros(in_shape, torch.int8), G.zeros(1, torch.int32)
+    s1, s2 = G.zeros(1, torch.int64), G.zeros(1, torch.int64)
+    eoq.eoq_conv_dgrad_head(hd, gd, G.dev(e3), i32(-11), G.dev(wt), e4, p4, s4, G.dev(G.pack_mask(mask01)),
+                            G.dev(x2) if with_x2 else None, i32(gamma), n3, pn3, s1, s2 if with_x2 else None,
+                            G.workspace(gd, eoq.EOQ_PASS_DGRAD))
+    torch.cuda.synchronize()
+    assert eoq.eoq_last_status(hd) == 0
+    assert np.array_equal(G.host(e4), e4_o) and p4.item() == p4_o and s4.item() == int(e4_o.astype(np.int64).sum())
+    assert np.array_equal(G.host(n3), want_e3) and pn3.item() == want_p3 and s1.item() == want_s1
+    if with_x2:
+        assert s2.item() == want_s2
+    # the plain call right after finds clean cells
+    e4b, p4b = G.zeros(in_shape, torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_conv_dgrad(hd, gd, G.dev(e3), i32(-11), G.dev(wt), e4b, p4b, None, None, G.workspace(gd, eoq.EOQ_PASS_DGRAD))
+    torch.cuda.synchronize()
+    assert np.array_equal(G.host(e4b), e4_o) and p4b.item() == p4_o
+
+
+def test_dgrad_head_refuses_the_compact_strided_1x1_case():
+    hd = G.handle()
+    d = ConvDesc(2, 8, 8, 32, 64, 1, 1, 2, 0)
+    gd = G.gdesc(d)
+    z8 = lambda shape: G.zeros(shape, torch.int8)
+    with pytest.raises(eoq.EoqError):
+        eoq.eoq_conv_dgrad_head(hd, gd, z8((2, 4, 4, 64)), i32(-11), z8((64, 1, 1, 32)), z8((2, 8, 8, 32)), G.zeros(1, torch.int32), None,
+                                G.zeros(2 * 8 * 8 * 32 // 8, torch.uint8), None, i32(128), z8((2, 8, 8, 32)), G.zeros(1, torch.int32),
+                                None, None, G.workspace(gd, eoq.EOQ_PASS_DGRAD))

@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 SEED = synth.BASE_SEED
 
 
-def build(name, batch, round_mode, lr=(3, -4)):
+def build(name, batch, round_mode, lr=(3, -4), keep_pool_error=False):
     if name == "resnet20":
         wl, classes, pool = workloads.resnet20(batch), 10, None
         net = N.resnet20(batch)
@@ -25,7 +25,7 @@ def build(name, batch, round_mode, lr=(3, -4)):
         wl, classes, pool = workloads.resnet18(batch), 1000, (3, 2, 1)
         net = N.resnet18(batch)
     st = ChainedStep(wl, eoq.eoq_create(0), scalars=Scalars(), lr_mant=lr[0], lr_exp=lr[1], head_lr=2.0 ** -6, classes=classes,
-                     pool=pool, round_mode=round_mode, seed=SEED)
+                     pool=pool, round_mode=round_mode, seed=SEED, keep_pool_error=keep_pool_error)
     N.init(net, lambda s, stream: synth.normal_f64(s, SEED, stream), lambda s, stream: synth.normal_f32(s, SEED, stream),
            b1=-2, gamma=118, b2=3)
     return wl, st, net
@@ -55,7 +55,7 @@ def compare_parameters(st, net, where):
 @pytest.mark.parametrize("name,batch,mode", [("resnet20", 2, eoq.EOQ_ROUND_RNE), ("resnet20", 4, eoq.EOQ_ROUND_STOCHASTIC),
                                              ("resnet18", 2, eoq.EOQ_ROUND_RNE)])
 def test_chained_step_matches_the_oracle_on_every_tensor(name, batch, mode):
-    wl, st, net = build(name, batch, mode)
+    wl, st, net = build(name, batch, mode, keep_pool_error=True)
     compare_parameters(st, net, "init")
     img, labels = feed(st, 0)
     st.run()
