@@ -127,23 +127,41 @@ maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *e_exp, const uin
         const int ox_lo = max(0, (ix + p - k + s) / s), ox_hi = min(wo - 1, (ix + p) / s);
         uint32_t even[4] = {0, 0, 0, 0}, odd[4] = {0, 0, 0, 0};
         int nwin = 0;
-        for (int oy = oy_lo; oy <= oy_hi; ++oy)
-            for (int ox = ox_lo; ox <= ox_hi; ++ox) {
-                const size_t o = (((size_t)b * ho + oy) * wo + ox) * c + gi * 16;
-                const int4 ev = __ldg(reinterpret_cast<const int4 *>(e + o));
-                const int4 av = __ldg(reinterpret_cast<const int4 *>(arg + o));
-                const uint32_t me = (uint32_t)((iy - (oy * s - p)) * k + (ix - (ox * s - p))) * 0x01010101u;
-                const uint32_t ew[4] = {(uint32_t)ev.x, (uint32_t)ev.y, (uint32_t)ev.z, (uint32_t)ev.w};
-                const uint32_t aw[4] = {(uint32_t)av.x, (uint32_t)av.y, (uint32_t)av.z, (uint32_t)av.w};
+        auto take = [&](const int4 &ev, const int4 &av, int oy, int ox) {
+            const uint32_t me = (uint32_t)((iy - (oy * s - p)) * k + (ix - (ox * s - p))) * 0x01010101u;
+            const uint32_t ew[4] = {(uint32_t)ev.x, (uint32_t)ev.y, (uint32_t)ev.z, (uint32_t)ev.w};
+            const uint32_t aw[4] = {(uint32_t)av.x, (uint32_t)av.y, (uint32_t)av.z, (uint32_t)av.w};
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint32_t hit = __vcmpeq4(aw[q], me);           // 0xff in the bytes this position won
-                    const uint32_t v = (ew[q] & hit) ^ 0x80808080u;      // code + 128 there, 128 elsewhere
-                    even[q] += v & 0x00ff00ffu;
-                    odd[q] += (v >> 8) & 0x00ff00ffu;
-                }
-                ++nwin;
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t hit = __vcmpeq4(aw[q], me);           // 0xff in the bytes this position won
+                const uint32_t v = (ew[q] & hit) ^ 0x80808080u;      // code + 128 there, 128 elsewhere
+                even[q] += v & 0x00ff00ffu;
+                odd[q] += (v >> 8) & 0x00ff00ffu;
             }
+            ++nwin;
+        };
+        if (oy_hi - oy_lo <= 1 && ox_hi - ox_lo <= 1) {
+            // the usual case (window at most twice the stride): at most 2 x 2 windows, all eight loads issued together
+            int4 ev[4], av[4];
+            bool in[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int oy = oy_lo + (u >> 1), ox = ox_lo + (u & 1);
+                in[u] = oy <= oy_hi && ox <= ox_hi;
+                const size_t o = (((size_t)b * ho + oy) * wo + ox) * c + gi * 16;
+                ev[u] = in[u] ? __ldg(reinterpret_cast<const int4 *>(e + o)) : make_int4(0, 0, 0, 0);
+                av[u] = in[u] ? __ldg(reinterpret_cast<const int4 *>(arg + o)) : make_int4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (in[u]) take(ev[u], av[u], oy_lo + (u >> 1), ox_lo + (u & 1));
+        } else {
+            for (int oy = oy_lo; oy <= oy_hi; ++oy)
+                for (int ox = ox_lo; ox <= ox_hi; ++ox) {
+                    const size_t o = (((size_t)b * ho + oy) * wo + ox) * c + gi * 16;
+                    take(__ldg(reinterpret_cast<const int4 *>(e + o)), __ldg(reinterpret_cast<const int4 *>(arg + o)), oy, ox);
+                }
+        }
         int sum[16];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -162,8 +180,14 @@ maxpool_bwd_kernel(const int8_t *__restrict__ e, const int32_t *e_exp, const uin
             }
         } else {
             int cd[16];
+            if (t >= 8) {   // a right shift by t - 7 >= 1 (sums are below 2^15, nothing can wrap)
+                const int sh = t - 7, half_m1 = (1 << (sh - 1)) - 1;
 #pragma unroll
-            for (int q = 0; q < 16; ++q) cd[q] = sq_code32(sum[q], t);
+                for (int q = 0; q < 16; ++q) cd[q] = sq_code32_shr(sum[q], sh, half_m1);
+            } else {
+#pragma unroll
+                for (int q = 0; q < 16; ++q) cd[q] = sq_code32(sum[q], t);
+            }
             if (e_in)
                 reinterpret_cast<int4 *>(e_in)[i] =
                     make_int4((int)pack4(cd[0], cd[1], cd[2], cd[3]), (int)pack4(cd[4], cd[5], cd[6], cd[7]),
@@ -426,21 +450,28 @@ constexpr int kHeadWarps = 8;
 __global__ void head_logits_kernel(const float *__restrict__ pooled, int n, int c, int classes, const float *__restrict__ W,
                                    const float *__restrict__ bias, float *logits)
 {
-    extern __shared__ float ps[];  // [c][32]
+    extern __shared__ float ps[];  // [c][33]: row k holds the 32 samples' activations (padded: the fill walks k, the chains walk samples)
     const int b0 = blockIdx.y * 32, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int i = threadIdx.x; i < c * 32; i += blockDim.x) {
-        const int k = i >> 5, sb = i & 31;
-        ps[i] = (b0 + sb < n) ? pooled[(size_t)(b0 + sb) * c + k] : 0.0f;
+        const int sb = i / c, k = i - sb * c;   // consecutive threads read consecutive k of one sample
+        ps[k * 33 + sb] = (b0 + sb < n) ? pooled[(size_t)(b0 + sb) * c + k] : 0.0f;
     }
     __syncthreads();
     const int j = blockIdx.x * kHeadWarps + warp;
     if (j >= classes) return;
     float acc = bias[j];
     const float *wj = W + (size_t)j * c;
+    float wnext = lane < c ? __ldg(wj + lane) : 0.0f;
     for (int k0 = 0; k0 < c; k0 += 32) {
-        const float wreg = (k0 + lane < c) ? __ldg(wj + k0 + lane) : 0.0f;
+        const float wreg = wnext;
+        if (k0 + 32 < c) wnext = (k0 + 32 + lane < c) ? __ldg(wj + k0 + 32 + lane) : 0.0f;   // the next 32 weights travel meanwhile
         const int kn = min(32, c - k0);
-        for (int kk = 0; kk < kn; ++kk) acc = __fmaf_rn(__shfl_sync(0xffffffffu, wreg, kk), ps[(k0 + kk) * 32 + lane], acc);
+        if (kn == 32) {
+#pragma unroll
+            for (int kk = 0; kk < 32; ++kk) acc = __fmaf_rn(__shfl_sync(0xffffffffu, wreg, kk), ps[(k0 + kk) * 33 + lane], acc);
+        } else {
+            for (int kk = 0; kk < kn; ++kk) acc = __fmaf_rn(__shfl_sync(0xffffffffu, wreg, kk), ps[(k0 + kk) * 33 + lane], acc);
+        }
     }
     if (b0 + lane < n) logits[(size_t)(b0 + lane) * classes + j] = acc;
 }
@@ -767,7 +798,7 @@ cudaError_t launch_head(const int32_t *sums, int n, int c, int hw, int classes, 
 {
     head_pooled_kernel<<<(n * c + 255) / 256, 256, 0, st>>>(sums, n * c, hw, pooled);
     {
-        const size_t smem = (size_t)c * 32 * sizeof(float);
+        const size_t smem = (size_t)c * 33 * sizeof(float);
         cudaError_t e = cudaFuncSetAttribute(head_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         dim3 grid((classes + kHeadWarps - 1) / kHeadWarps, (n + 31) / 32);
