@@ -215,12 +215,20 @@ def run_reference(args):
 
 # ----------------------------------------------------------------------------------------------- GPU arm
 
-def bandwidth_bytes(wl):
-    """Algorithmic bytes per step of the bandwidth-bound kernel groups (what the method itself must move)."""
+def bandwidth_bytes(wl, chained=False):
+    """Algorithmic bytes per step of the bandwidth-bound kernel groups (what the method itself must move).
+    In the closed-loop step most error heads ride on the kernel that produces their input error: the head of a block's
+    first unit on the Q_e pass behind the second unit's dgrad (its bytes are counted there), the others on joins and the
+    pool's backward (glue, not listed); only the last block's and the projection shortcuts' heads run on their own."""
     head = dq = fin = upd = 0
-    for l in wl.layers:
+    last_b = max((i for i, l in enumerate(wl.layers) if l.name.endswith(".b")), default=-1)
+    for i, l in enumerate(wl.layers):
         n_out = l.n * l.ho * l.wo * l.c_out
-        head += n_out * (1 + 1 + 0.125 + (2 if l.gamma_trainable else 0))   # e0 in, e3 out, mask, x2 for g_gamma
+        own = n_out * (1 + 1 + 0.125 + (2 if l.gamma_trainable else 0))    # e0 in, e3 out, mask, x2 for g_gamma
+        if not chained or l.name.endswith(".proj") or i == last_b:
+            head += own
+        elif l.name.endswith(".a"):
+            dq += n_out * (1 + 0.125)                                       # e3 out and mask bits, on the Q_e pass of unit B
         if l.has_dgrad:
             dq += l.n * l.h * l.w * l.c_in * (4 + 1)                        # exact int32 sums in, e4 codes out
         fin += l.weight_elems * (4 + 1)                                     # exact sums in, g codes out
@@ -386,7 +394,7 @@ def run_gpu(args):
         names = eoq.EOQ_PROF_NAMES
         by_kind = {name: prof_ms[i] / prof_steps for i, name in enumerate(names)}
         bw = {}
-        for kind, nbytes in bandwidth_bytes(wl).items():
+        for kind, nbytes in bandwidth_bytes(wl, chained).items():
             t_ms = by_kind.get(kind, 0.0)
             gbs = nbytes / (t_ms / 1e3) / 1e9 if t_ms > 0 else None
             bw[kind] = {"algorithmic_bytes": nbytes, "ms": t_ms, "gbs": gbs, "frac_of_hbm": gbs / pk["hbm_gbs"] if gbs else None}

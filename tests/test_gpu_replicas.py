@@ -113,6 +113,9 @@ def test_join_pooling_and_input_quantizer_through_the_hook():
         x = synth.relu_codes((n, hh, ww, c), 9200, 2)
         e = synth.normal_codes((n, 5, 5, c), 9200, 3)
         img = synth.normal_f32((n, 12, 12, 3), 9200, 4)
+        m01 = synth.bits((n, hh, ww, c), 9200, 5, 0.5)
+        x2 = (synth.relu_codes((n, hh, ww, c), 9200, 6).astype(np.int32) * 31).astype(np.int16)
+        gam = G.dev(np.array([109], dtype=np.int32))
 
         def run(sl):
             m = sl.stop - sl.start
@@ -126,8 +129,19 @@ def test_join_pooling_and_input_quantizer_through_the_hook():
             eoq.eoq_aux_maxpool_bwd(h, G.dev(e[sl]), G.dev(np.array([-13], dtype=np.int32)), arg, m, hh, ww, c, 3, 2, 1, ein, pin)
             q, pq = G.zeros((m, 12, 12, 16), torch.int8), G.zeros(1, torch.int32)
             eoq.eoq_quantize_image(h, G.dev(img[sl]), m, 12, 12, 3, 16, 0, q, pq)
+            # the same producers with their consumer's error head fused in: two maxima and up to three sums to exchange
+            mk, x2d = G.dev(G.pack_mask(m01[sl])), G.dev(x2[sl])
+            j2, pj2, sj2 = G.zeros((m, hh, ww, c), torch.int8), G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+            h3, ph3, hs1, hs2 = G.zeros((m, hh, ww, c), torch.int8), G.zeros(1, torch.int32), G.zeros(1, torch.int64), G.zeros(1, torch.int64)
+            eoq.eoq_aux_join_head(h, G.dev(a[sl]), G.dev(np.array([-11], dtype=np.int32)), G.dev(b[sl]), G.dev(np.array([-14], dtype=np.int32)),
+                                  None, j2.numel(), j2, pj2, sj2, mk, x2d, gam, h3, ph3, hs1, hs2)
+            ein2, pin2 = G.zeros((m, hh, ww, c), torch.int8), G.zeros(1, torch.int32)
+            p3, pp3, ps1 = G.zeros((m, hh, ww, c), torch.int8), G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+            eoq.eoq_aux_maxpool_bwd_head(h, G.dev(e[sl]), G.dev(np.array([-13], dtype=np.int32)), arg, m, hh, ww, c, 3, 2, 1, ein2, pin2, mk,
+                                         gam, p3, pp3, ps1)
             torch.cuda.synchronize()
-            return {"j": j, "pj": pj, "sj": sj, "ein": ein, "pin": pin, "q": q, "pq": pq}
+            return {"j": j, "pj": pj, "sj": sj, "ein": ein, "pin": pin, "q": q, "pq": pq, "j2": j2, "pj2": pj2, "sj2": sj2, "h3": h3,
+                    "ph3": ph3, "hs1": hs1, "hs2": hs2, "ein2": ein2, "pin2": pin2, "p3": p3, "pp3": pp3, "ps1": ps1}
 
         whole = run(slice(0, n))
         parts = [slice(0, 2), slice(2, 4)]
@@ -144,11 +158,12 @@ def test_join_pooling_and_input_quantizer_through_the_hook():
             eoq.eoq_set_reduce_hook(h, inj.fn)
             reps.append(run(sl))
         eoq.eoq_set_reduce_hook(h, None)
-        for key in ("j", "ein", "q"):
+        for key in ("j", "ein", "q", "j2", "h3", "ein2", "p3"):
             assert torch.equal(torch.cat([reps[0][key], reps[1][key]]), whole[key]), key
         for r in reps:
-            for key in ("pj", "sj", "pin", "pq"):
+            for key in ("pj", "sj", "pin", "pq", "pj2", "sj2", "ph3", "hs1", "hs2", "pin2", "pp3", "ps1"):
                 assert torch.equal(r[key], whole[key]), key
+        assert torch.equal(whole["j2"], whole["j"]) and torch.equal(whole["ein2"], whole["ein"])
         S, p = oracle.join(a, -11, b, -14)
         ref, pr, _ = oracle.sq_int(S, p)
         assert np.array_equal(G.host(whole["j"]).astype(np.int32), ref) and whole["pj"].item() == pr
