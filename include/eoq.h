@@ -215,6 +215,22 @@ EOQ_API int eoq_conv_wgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
 EOQ_API int eoq_conv_wgrad_dev(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
                        const int8_t *x, const int32_t *b1_c, int8_t *g, int32_t *g_exp, void *workspace,
                        size_t workspace_bytes, void *stream);
+/*
+ * The weight gradient in two parts, for training loops that finish the gradients of all layers together.
+ * eoq_conv_wgrad_gemm: the GEMM of eoq_conv_wgrad_dev alone; the exact sums stay in `workspace` (which must then stay
+ *   untouched until the finish) and *num_parts (host) receives what the finish needs to read them.
+ * eoq_wgrad_finish: for `num` layers at once (host arrays of length num; device pointers inside): the b1 error sums
+ *   (b1_c[i]: the layer's code in device memory, or NULL for a layer without a bias in front of its convolution), the
+ *   sum of the split-K slices plus the b1 term, and Q_g -> gq[i], *g_exp[i].  Four launches per 16 layers instead of
+ *   four per layer.  workspace[i], workspace_bytes[i], num_parts[i]: as given to / returned by eoq_conv_wgrad_gemm
+ *   for that layer; descs[i], e3[i], e3_exp[i] likewise.  Results are those of eoq_conv_wgrad_dev, bit for bit.
+ * EOQ_ERR_UNSUPPORTED while a reduce hook is installed (replicas exchange per layer).
+ */
+EOQ_API int eoq_conv_wgrad_gemm(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                        const int8_t *x, void *workspace, size_t workspace_bytes, int *num_parts, void *stream);
+EOQ_API int eoq_wgrad_finish(eoq_handle_t handle, int num, const eoq_conv_desc_t *descs, const int8_t *const *e3,
+                     const int32_t *const *e3_exp, const int32_t *const *b1_c, int8_t *const *gq, int32_t *const *g_exp,
+                     void *const *workspace, const size_t *workspace_bytes, const int *num_parts, void *stream);
 
 /*
  * The three quantization functions (Sec. 3.2.2) on a flat tensor of n elements.

@@ -69,9 +69,12 @@ class ChainedStep:
     def __init__(self, workload: Workload, handle: int, device: str = "cuda:0", seed: int = synth.BASE_SEED,
                  scalars: Optional[Scalars] = None, lr_mant: int = 3, lr_exp: int = -4, head_lr: float = 2.0 ** -6,
                  classes: int = 1000, pool: Optional[tuple] = None, round_mode: int = eoq.EOQ_ROUND_RNE,
-                 image_channels: int = 3, side_streams: int = 2, keep_pool_error: bool = False):
+                 image_channels: int = 3, side_streams: int = 2, keep_pool_error: bool = False, finish_together: bool = True):
         self.wl, self.h, self.dev = workload, handle, torch.device(device)
         self.keep_pool_error = keep_pool_error   # also write the error between the pool and the first layer's head
+        # weight gradients: only the GEMMs run per layer beside the backward chain; the b1 sums, slice sums and Q_g of all
+        # layers follow in four launches at the end (each layer then keeps its sums in a workspace of its own)
+        self.finish_together = finish_together
         self.sc = scalars or Scalars()
         self.lr_mant, self.lr_exp, self.head_lr, self.classes = lr_mant, lr_exp, head_lr, classes
         self.round_mode, self.seed, self.pool = round_mode, seed, pool
@@ -144,6 +147,11 @@ class ChainedStep:
         for hs in self.h_sides:
             eoq.eoq_set_gemm_ctas(hs, half)
         self.sides = [torch.cuda.Stream(device=dev) for _ in range(side_streams)]
+        if finish_together:
+            for u in self.units:
+                u.wgrad_ws = torch.empty(max(256, eoq.eoq_workspace_size(u.desc, eoq.EOQ_PASS_WGRAD)), dtype=torch.uint8, device=dev)
+                u.wgrad_parts = 0
+                u.b1_dev = None
         self.graph = None
         self._init_parameters(seed)
         self._scalar_items()
@@ -224,21 +232,50 @@ class ChainedStep:
 
         side_no = [0]
 
+        def wgrad_call(hh, u: UnitBuffers, b1_dev, wsp) -> None:
+            if self.finish_together:
+                u.b1_dev = b1_dev
+                u.wgrad_parts = eoq.eoq_conv_wgrad_gemm(hh, u.desc, u.e3, u.e3_exp, u.x0, u.wgrad_ws)
+            else:
+                eoq.eoq_conv_wgrad_dev(hh, u.desc, u.e3, u.e3_exp, u.x0, b1_dev, u.g, u.g_exp, wsp)
+
         def wgrad(u: UnitBuffers, b1_dev) -> None:
             if overlap:
                 k = side_no[0] % len(self.sides)
                 side_no[0] += 1
                 self.sides[k].wait_stream(main)
                 with torch.cuda.stream(self.sides[k]):
-                    eoq.eoq_conv_wgrad_dev(self.h_sides[k], u.desc, u.e3, u.e3_exp, u.x0, b1_dev, u.g, u.g_exp, self.workspace_sides[k])
+                    wgrad_call(self.h_sides[k], u, b1_dev, self.workspace_sides[k])
             else:
-                eoq.eoq_conv_wgrad_dev(h, u.desc, u.e3, u.e3_exp, u.x0, b1_dev, u.g, u.g_exp, ws)
+                wgrad_call(h, u, b1_dev, ws)
+
+        def finish(us) -> None:
+            """b1 sums, slice sums and Q_g of the units whose GEMMs have been issued: a few launches for all of them,
+            behind those GEMMs on a side stream (so that they run beside the rest of the backward chain)."""
+            if not self.finish_together or not us:
+                return
+            args = ([u.desc for u in us], [u.e3 for u in us], [u.e3_exp for u in us], [u.b1_dev for u in us], [u.g for u in us],
+                    [u.g_exp for u in us], [u.wgrad_ws for u in us], [u.wgrad_parts for u in us])
+            if overlap:
+                for side in self.sides[1:]:
+                    self.sides[0].wait_stream(side)
+                with torch.cuda.stream(self.sides[0]):
+                    eoq.eoq_wgrad_finish(self.h_sides[0], *args)
+            else:
+                eoq.eoq_wgrad_finish(h, *args)
 
         e_out, e_exp = self.e_head, self.e_head_exp
         head_done = False   # the error head of this block's last unit already ran inside the join of the block behind it
+        pending = []        # units whose weight-gradient GEMM is issued and not yet finished
+        stage = None
         for i in reversed(range(len(self.blocks))):
             blk = self.blocks[i]
             a, b, pr = blk.a, blk.b, blk.proj
+            if stage is not None and a.layer.name.split(".")[0] != stage:
+                finish(pending)     # a stage of the network is through: its gradients are finished together
+                pending = []
+            stage = a.layer.name.split(".")[0]
+            pending += [b, a] + ([pr] if pr else [])
             if not head_done:
                 eoq.eoq_err_prescale_dev(h, e_out, e_exp, b.mask, b.x2, b.n_out, b.scal[1:2], b.e3, b.e3_exp, b.sum_e1, b.sum_e1x2)
             wgrad(b, b.scal[0:1])
@@ -267,6 +304,7 @@ class ChainedStep:
                 eoq.eoq_aux_join(h, a.e4, a.e4_exp, j_b, j_b_exp, j_mask, a.e4.numel(), blk.e_in, blk.e_in_exp, blk.sum_join)
                 head_done = False
             e_out, e_exp = blk.e_in, blk.e_in_exp
+        finish(pending)
         if self.pool:
             k, s, p = self.pool
             # pool backward and the first layer's error head in one pair of kernels; the error between them (51 MB at
@@ -278,6 +316,7 @@ class ChainedStep:
             eoq.eoq_err_prescale_dev(h, e_out, e_exp, stem.mask, None, stem.n_out, stem.scal[1:2], stem.e3, stem.e3_exp, stem.sum_e1,
                                      None)
         wgrad(stem, None)
+        finish([stem])
         if overlap:
             for side in self.sides:
                 main.wait_stream(side)

@@ -1082,13 +1082,16 @@ static cudaError_t launch_tap_sums(Handle *h, const int8_t *e3, long long *tap_s
 }
 
 // Weight gradient behind eoq_conv_wgrad and eoq_conv_wgrad_dev: b1 is the host code b1_c, or the code at b1_dev.
+// num_parts_out (eoq_conv_wgrad_gemm): the GEMM alone; the sums stay in the workspace for eoq_wgrad_finish and
+// *num_parts_out tells it how many int32 slices there are (0: the GEMM added into the int64 sums).
 static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
                            const int8_t *x, int32_t b1_c, const int32_t *b1_dev, int8_t *gq, int32_t *g_exp,
-                           int64_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
+                           int64_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream, int *num_parts_out = nullptr)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
     Geometry g;
-    if (!h || !e3 || !e3_exp || !x || !gq || !g_exp) return EOQ_ERR_BAD_ARG;
+    const bool gemm_only = num_parts_out != nullptr || (h && h->gemm_only);
+    if (!h || !e3 || !e3_exp || !x || (!num_parts_out && (!gq || !g_exp))) return EOQ_ERR_BAD_ARG;
     int st = check_desc(desc, &g);
     if (st != EOQ_OK) return st;
     if (!aligned16(e3) || !aligned16(x) || !aligned16(gq) || !aligned16(acc_dump)) return EOQ_ERR_ALIGNMENT;
@@ -1113,12 +1116,14 @@ static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
         wp.partials = reinterpret_cast<int32_t *>(ws + tap_bytes + 256 + acc_bytes);
         wp.dev = h->dev;
         cudaError_t e;
-        if (h->gemm_only) {
+        if (gemm_only) {
             CUtensorMap mx, me;
             if (!make_patch_map(&mx, x, d.n, d.h, d.w, d.c_in, wp.kc, wp.pw, wp.r_rows + d.kh - 1) ||
                 !make_patch_map(&me, e3, d.n, g.ho, g.wo, d.c_out, wp.tile_n, wp.pw, wp.r_rows))
                 return EOQ_ERR_UNSUPPORTED;
             count_launches(h, 1);
+            if (num_parts_out) *num_parts_out = wp.num_splits;
+            ProfScope prof(h, EOQ_PROF_WGRAD, s);
             return record(h, launch_wgrad_patch(wp, mx, me, s));
         }
         e = use_b1 ? launch_tap_sums(h, e3, tap_sums, tap_bytes, d, g.ho, g.wo, bc, s) : cudaSuccess;
@@ -1218,7 +1223,7 @@ static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
         ProfScope aux(h, EOQ_PROF_WGRAD_AUX, s);
         e = cudaMemsetAsync(acc, 0, acc_bytes, s);  // the GEMM adds into the int64 sums with atomics
     }
-    if (e == cudaSuccess && use_b1 && !h->gemm_only) e = launch_tap_sums(h, e3, tap_sums, tap_bytes, d, g.ho, g.wo, bc, s);
+    if (e == cudaSuccess && use_b1 && !gemm_only) e = launch_tap_sums(h, e3, tap_sums, tap_bytes, d, g.ho, g.wo, bc, s);
     if (e != cudaSuccess) return record(h, e);
     CUtensorMap map_x, map_e;
     if (!make_matrix_map(&map_e, e3, (size_t)p.P, d.c_out, p.nc, p.pixels_per_stage)) return EOQ_ERR_UNSUPPORTED;
@@ -1232,7 +1237,8 @@ static int conv_wgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
         ProfScope prof(h, EOQ_PROF_WGRAD, s);
         e = launch_wgrad(p, map_x, map_e, s);
     }
-    if (e != cudaSuccess || h->gemm_only) return record(h, e);
+    if (num_parts_out) *num_parts_out = 0;
+    if (e != cudaSuccess || gemm_only) return record(h, e);
     // the kernel leaves sums as [oc][tap][ic], which is the layout of g
     ProfScope prof_q(h, EOQ_PROF_WGRAD_AUX, s);
     e = launch_sq_i64(acc, e3_exp, -7, g.w_elems, gq, g_exp, reinterpret_cast<long long *>(acc_dump),
@@ -1254,6 +1260,78 @@ extern "C" int eoq_conv_wgrad_dev(eoq_handle_t handle, const eoq_conv_desc_t *de
 {
     // b1_c null: the layer has no bias in front of its convolution (the first layer of a network)
     return conv_wgrad_impl(handle, desc, e3, e3_exp, x, 0, b1_c, gq, g_exp, nullptr, workspace, workspace_bytes, stream);
+}
+
+extern "C" int eoq_conv_wgrad_gemm(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                                   const int8_t *x, void *workspace, size_t workspace_bytes, int *num_parts, void *stream)
+{
+    if (!num_parts) return EOQ_ERR_BAD_ARG;
+    return conv_wgrad_impl(handle, desc, e3, e3_exp, x, 0, nullptr, nullptr, nullptr, nullptr, workspace, workspace_bytes, stream,
+                           num_parts);
+}
+
+extern "C" int eoq_wgrad_finish(eoq_handle_t handle, int num, const eoq_conv_desc_t *descs, const int8_t *const *e3,
+                                const int32_t *const *e3_exp, const int32_t *const *b1_c, int8_t *const *gq, int32_t *const *g_exp,
+                                void *const *workspace, const size_t *workspace_bytes, const int *num_parts, void *stream)
+{
+    Handle *h = reinterpret_cast<Handle *>(handle);
+    if (!h || num <= 0 || !descs || !e3 || !e3_exp || !b1_c || !gq || !g_exp || !workspace || !workspace_bytes || !num_parts)
+        return EOQ_ERR_BAD_ARG;
+    if (h->hook.fn) return EOQ_ERR_UNSUPPORTED;  // replicas exchange per layer: eoq_conv_wgrad_dev
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    for (int i = 0; i < num; ++i) {
+        Geometry g;
+        int st = check_desc(&descs[i], &g);
+        if (st != EOQ_OK) return st;
+        if (!e3[i] || !e3_exp[i] || !gq[i] || !g_exp[i] || num_parts[i] < 0) return EOQ_ERR_BAD_ARG;
+        if (!aligned16(e3[i]) || !aligned16(gq[i])) return EOQ_ERR_ALIGNMENT;
+        if ((st = check_workspace(&descs[i], EOQ_PASS_WGRAD, workspace[i], workspace_bytes[i])) != EOQ_OK) return st;
+        const BorderClasses bc = border_classes(descs[i], g);
+        if (b1_c[i] && bc.nrc * bc.ncc > kMaxBorderClasses) return EOQ_ERR_UNSUPPORTED;
+    }
+    for (int base = 0; base < num; base += kFinishChunk) {
+        FinishBatch b;
+        memset(&b, 0, sizeof(b));
+        b.num = num - base < kFinishChunk ? num - base : kFinishChunk;
+        for (int k = 0; k < b.num; ++k) {
+            const eoq_conv_desc_t &d = descs[base + k];
+            Geometry g;
+            check_desc(&d, &g);
+            FinishItem &it = b.item[k];
+            // the workspace as eoq_conv_wgrad_gemm laid it out: [tap sums][256 spare bytes][int64 sums][split-K slices]
+            char *ws = reinterpret_cast<char *>(workspace[base + k]);
+            const size_t tap_stride = round256((size_t)d.c_out * g.taps * sizeof(long long)) / sizeof(long long);
+            const size_t tap_bytes = kTapReplicas * tap_stride * sizeof(long long);
+            const size_t acc_bytes = round256(g.w_elems * sizeof(long long));
+            it.e3 = e3[base + k];
+            it.e3_exp = e3_exp[base + k];
+            it.b1_dev = b1_c[base + k];
+            it.tap_sums = reinterpret_cast<long long *>(ws);
+            it.tap_stride = tap_stride;
+            it.zero_bytes = tap_bytes + 256;
+            it.max_cell = reinterpret_cast<unsigned long long *>(ws + tap_bytes);
+            it.acc = reinterpret_cast<long long *>(ws + tap_bytes + 256);
+            it.num_parts = num_parts[base + k];
+            it.parts = it.num_parts > 0 ? reinterpret_cast<const int32_t *>(ws + tap_bytes + 256 + acc_bytes) : nullptr;
+            it.g = gq[base + k];
+            it.g_exp = g_exp[base + k];
+            it.n = g.w_elems;
+            it.pixels = (unsigned long long)d.n * g.ho * g.wo;
+            it.d = d;
+            it.bc = border_classes(d, g);
+            it.ho = g.ho;
+            it.wo = g.wo;
+            plan_finish_item(it, h->sm_count);
+            b.tap_first[k + 1] = b.tap_first[k] + it.tap_grid_x * it.tap_grid_y;
+            b.fin_first[k + 1] = b.fin_first[k] + it.fin_blocks;
+            b.sq_first[k + 1] = b.sq_first[k] + it.sq_blocks;
+        }
+        ProfScope prof(h, EOQ_PROF_WGRAD_AUX, s);
+        const cudaError_t e = launch_wgrad_finish(b, &h->dev->status, s);
+        count_launches(h, 4);
+        if (e != cudaSuccess) return record(h, e);
+    }
+    return EOQ_OK;
 }
 
 // ================================================================================= tensor-pipe probe

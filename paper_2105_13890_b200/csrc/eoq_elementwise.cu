@@ -397,16 +397,17 @@ __global__ void sq_i32_scatter_kernel(const int32_t *__restrict__ src, const int
 // sum of the error over the pixels whose tap falls inside the image); optionally copies the exact sums out; and
 // reduces max |.|.  A block of 256 threads is (256 / groups) elements x `groups` slice groups: every thread adds
 // its share of the slices with independent, coalesced loads and the groups meet in shared memory.
-__global__ void wgrad_finalize_kernel(const int32_t *__restrict__ parts, int num_parts, int groups, size_t n, long long *acc,
-                                      const long long *__restrict__ tap_sums, size_t replica_stride, int32_t b1_c,
-                                      const int32_t *b1_dev, int c_in, long long *copy_out, DeviceState *dev, int sums_only)
+// (bx of nblocks): the block's place among the blocks of its tensor; max_cell: where max |.| is reduced (null: not at all)
+__device__ __forceinline__ void wgrad_finalize_body(const int32_t *__restrict__ parts, int num_parts, int groups, size_t n, long long *acc,
+                                                    const long long *__restrict__ tap_sums, size_t replica_stride, int32_t b1_c,
+                                                    const int32_t *b1_dev, int c_in, long long *copy_out,
+                                                    unsigned long long *max_cell, int bx, int nblocks)
 {
-    // sums_only: the sums are completed elsewhere (an all-reduce over replicas) before their maximum is taken
     __shared__ long long part[256];
     if (b1_dev) b1_c = clampi(__ldg(b1_dev), -32768, 32767);
-    const int bx = 256 / groups, tx = threadIdx.x % bx, ty = threadIdx.x / bx;
+    const int bw = 256 / groups, tx = threadIdx.x % bw, ty = threadIdx.x / bw;
     unsigned long long mx = 0;
-    for (size_t base = (size_t)blockIdx.x * bx; base < n; base += (size_t)gridDim.x * bx) {
+    for (size_t base = (size_t)bx * bw; base < n; base += (size_t)nblocks * bw) {
         const size_t i = base + tx;
         long long v = 0;
         if (parts) {
@@ -425,7 +426,7 @@ __global__ void wgrad_finalize_kernel(const int32_t *__restrict__ parts, int num
                 __syncthreads();
                 if (ty == 0) {
                     v = 0;
-                    for (int k = 0; k < groups; ++k) v += part[k * bx + tx];
+                    for (int k = 0; k < groups; ++k) v += part[k * bw + tx];
                 }
                 __syncthreads();
             }
@@ -447,7 +448,16 @@ __global__ void wgrad_finalize_kernel(const int32_t *__restrict__ parts, int num
         }
     }
     mx = block_max_u64(mx);
-    if (threadIdx.x == 0 && mx && !sums_only) atomicMax(&dev->absmax_u64, mx);
+    if (threadIdx.x == 0 && mx && max_cell) atomicMax(max_cell, mx);
+}
+
+__global__ void wgrad_finalize_kernel(const int32_t *__restrict__ parts, int num_parts, int groups, size_t n, long long *acc,
+                                      const long long *__restrict__ tap_sums, size_t replica_stride, int32_t b1_c,
+                                      const int32_t *b1_dev, int c_in, long long *copy_out, DeviceState *dev, int sums_only)
+{
+    // sums_only: the sums are completed elsewhere (an all-reduce over replicas) before their maximum is taken
+    wgrad_finalize_body(parts, num_parts, groups, n, acc, tap_sums, replica_stride, b1_c, b1_dev, c_in, copy_out,
+                        sums_only ? nullptr : &dev->absmax_u64, (int)blockIdx.x, (int)gridDim.x);
 }
 
 // max |.| of int64 sums into the handle's 64-bit cell (used when the sums were completed by an all-reduce)
@@ -463,25 +473,31 @@ __global__ void absmax_i64_kernel(const long long *__restrict__ src, size_t n, D
     if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u64, mx);
 }
 
-__global__ void sq_i64_kernel(const long long *__restrict__ src, const int32_t *src_exp, int exp_bias, size_t n,
-                              int8_t *dst, int32_t *dst_exp, DeviceState *dev)
+// (bx of nblocks) as above; M: the tensor's max |.|; status: where a zero tensor is flagged
+__device__ __forceinline__ void sq_i64_body(const long long *__restrict__ src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
+                                            int32_t *dst_exp, unsigned long long M, unsigned *status, int bx, int nblocks)
 {
-    const unsigned long long M = dev->absmax_u64;
     const int t = M ? round_log2_u64(M) : 7;
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (bx == 0 && threadIdx.x == 0) {
         const int p_in = (src_exp ? *src_exp : 0) + exp_bias;
         *dst_exp = M ? p_in + t - 7 : p_in;
-        if (!M) atomicOr(&dev->status, EOQ_DEV_SQ_ZERO);
+        if (!M) atomicOr(status, EOQ_DEV_SQ_ZERO);
     }
     // four codes per thread and round (one 32-bit store); n is a multiple of 4 for every weight tensor with padded channels
     const size_t n4 = n / 4;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    for (size_t i = (size_t)bx * blockDim.x + threadIdx.x; i < n4; i += (size_t)nblocks * blockDim.x) {
         const longlong2 a = __ldg(reinterpret_cast<const longlong2 *>(src) + 2 * i);
         const longlong2 b = __ldg(reinterpret_cast<const longlong2 *>(src) + 2 * i + 1);
         reinterpret_cast<uint32_t *>(dst)[i] = pack4(sq_code64(a.x, t), sq_code64(a.y, t), sq_code64(b.x, t), sq_code64(b.y, t));
     }
-    for (size_t i = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    for (size_t i = n4 * 4 + (size_t)bx * blockDim.x + threadIdx.x; i < n; i += (size_t)nblocks * blockDim.x)
         dst[i] = (int8_t)sq_code64(src[i], t);
+}
+
+__global__ void sq_i64_kernel(const long long *__restrict__ src, const int32_t *src_exp, int exp_bias, size_t n,
+                              int8_t *dst, int32_t *dst_exp, DeviceState *dev)
+{
+    sq_i64_body(src, src_exp, exp_bias, n, dst, dst_exp, dev->absmax_u64, &dev->status, (int)blockIdx.x, (int)gridDim.x);
     if (last_block_done(dev)) dev->absmax_u64 = 0;
 }
 
@@ -1059,26 +1075,28 @@ __global__ void weight_prep_kernel(const __grid_constant__ PrepBatch b)
 // registers, border pixels in shared memory.
 constexpr int kClassSlab = 128;
 constexpr int kTapUnroll = 8;
-__global__ void b1_tap_sums_kernel(const int8_t *__restrict__ e3, long long *tap_sums, size_t replica_stride, int c_out, int ho,
-                                   int wo, size_t pixels, int pixels_per_block, BorderClasses bc, eoq_conv_desc_t d)
+// (bx, by): the block's place in the grid of its layer (pixel range, channel slab)
+__device__ __forceinline__ void b1_tap_sums_body(const int8_t *__restrict__ e3, long long *tap_sums, size_t replica_stride, int c_out,
+                                                 int ho, int wo, size_t pixels, int pixels_per_block, const BorderClasses &bc,
+                                                 const eoq_conv_desc_t &d, int bx, int by)
 {
     // the blocks spread their atomics over kTapReplicas copies of the sums (the consumer adds the copies): all
     // cells of one copy sit in a few kilobytes, i.e. behind one or two L2 slices, whose atomic rate bounds this kernel
-    tap_sums += (size_t)(blockIdx.x % kTapReplicas) * replica_stride;
+    tap_sums += (size_t)(bx % kTapReplicas) * replica_stride;
     extern __shared__ int32_t cls_acc[];  // [classes][kClassSlab]
     const int classes = bc.nrc * bc.ncc;
     for (int i = threadIdx.x; i < classes * kClassSlab; i += blockDim.x) cls_acc[i] = 0;
     __syncthreads();
-    const int slab_ch = min(kClassSlab, c_out - (int)blockIdx.y * kClassSlab);  // channels of this slab (multiple of 16)
+    const int slab_ch = min(kClassSlab, c_out - by * kClassSlab);  // channels of this slab (multiple of 16)
     const int lanes_per_pix = slab_ch / 16;
     const int pix_per_step = blockDim.x / lanes_per_pix;
     const int sub = threadIdx.x % lanes_per_pix, slot = threadIdx.x / lanes_per_pix;
-    const int ch = blockIdx.y * kClassSlab + sub * 16;
+    const int ch = by * kClassSlab + sub * 16;
     const int interior = (bc.nrc != ho && bc.ncc != wo) ? bc.nlo_h * bc.ncc + bc.nlo_w : -1;
     int acc[16];
 #pragma unroll
     for (int k = 0; k < 16; ++k) acc[k] = 0;
-    const size_t begin = (size_t)blockIdx.x * pixels_per_block;
+    const size_t begin = (size_t)bx * pixels_per_block;
     const size_t end = min(pixels, begin + (size_t)pixels_per_block);
     const bool small = pixels <= 0xffffffffull;
     if (slot < pix_per_step) {
@@ -1154,9 +1172,61 @@ __global__ void b1_tap_sums_kernel(const int8_t *__restrict__ e3, long long *tap
             for (unsigned long long cm = cols; cm; cm &= cm - 1) sum += row[(__ffsll((long long)cm) - 1) * kClassSlab];
         }
         if (sum)
-            atomicAdd(reinterpret_cast<unsigned long long *>(tap_sums + (size_t)(blockIdx.y * kClassSlab + c) * taps + tap),
+            atomicAdd(reinterpret_cast<unsigned long long *>(tap_sums + (size_t)(by * kClassSlab + c) * taps + tap),
                       (unsigned long long)sum);
     }
+}
+
+
+__global__ void b1_tap_sums_kernel(const int8_t *__restrict__ e3, long long *tap_sums, size_t replica_stride, int c_out, int ho,
+                                   int wo, size_t pixels, int pixels_per_block, BorderClasses bc, eoq_conv_desc_t d)
+{
+    b1_tap_sums_body(e3, tap_sums, replica_stride, c_out, ho, wo, pixels, pixels_per_block, bc, d, (int)blockIdx.x, (int)blockIdx.y);
+}
+
+// ------------------------------------------------------------------ weight-gradient finish of many layers at once
+// A block finds the layer it works for by its index (first[] holds the first block of every item).
+__device__ __forceinline__ int finish_item_of(const int *first, int num, int block)
+{
+    int k = 0;
+    while (k + 1 < num && block >= first[k + 1]) ++k;
+    return k;
+}
+
+// zeroes what the finish accumulates into: the tap sums of every layer and its maximum cell (one block per layer)
+__global__ void finish_zero_kernel(FinishBatch b)
+{
+    const FinishItem &it = b.item[blockIdx.x];
+    int4 *dst = reinterpret_cast<int4 *>(it.tap_sums);
+    const size_t n16 = it.zero_bytes / 16;
+    for (size_t i = threadIdx.x; i < n16; i += blockDim.x) dst[i] = make_int4(0, 0, 0, 0);
+}
+
+__global__ void finish_taps_kernel(FinishBatch b)
+{
+    const int k = finish_item_of(b.tap_first, b.num, (int)blockIdx.x);
+    const FinishItem &it = b.item[k];
+    if (!it.b1_dev) return;
+    const int local = (int)blockIdx.x - b.tap_first[k];
+    b1_tap_sums_body(it.e3, it.tap_sums, (size_t)it.tap_stride, it.d.c_out, it.ho, it.wo, (size_t)it.pixels, it.pixels_per_block, it.bc,
+                     it.d, local % it.tap_grid_x, local / it.tap_grid_x);
+}
+
+__global__ void finish_sums_kernel(FinishBatch b)
+{
+    const int k = finish_item_of(b.fin_first, b.num, (int)blockIdx.x);
+    const FinishItem &it = b.item[k];
+    wgrad_finalize_body(it.parts, it.num_parts, it.groups, (size_t)it.n, it.acc, it.b1_dev ? it.tap_sums : nullptr,
+                        (size_t)it.tap_stride, 0, it.b1_dev, it.d.c_in, nullptr, it.max_cell, (int)blockIdx.x - b.fin_first[k],
+                        it.fin_blocks);
+}
+
+__global__ void finish_code_kernel(FinishBatch b, unsigned *status)
+{
+    const int k = finish_item_of(b.sq_first, b.num, (int)blockIdx.x);
+    const FinishItem &it = b.item[k];
+    sq_i64_body(it.acc, it.e3_exp, -7, (size_t)it.n, it.g, it.g_exp, *it.max_cell, status, (int)blockIdx.x - b.sq_first[k],
+                it.sq_blocks);
 }
 
 }  // namespace
@@ -1421,6 +1491,47 @@ cudaError_t launch_b1_error_sums(const int8_t *e3, long long *tap_sums, size_t r
     dim3 grid(blocks, slabs);
     b1_tap_sums_kernel<<<grid, 256, sizeof(int32_t) * classes * kClassSlab, s>>>(e3, tap_sums, replica_stride, d.c_out, ho, wo,
                                                                                pixels, (int)ppb, bc, d);
+    return cudaGetLastError();
+}
+
+void plan_finish_item(FinishItem &it, int sm_count)
+{
+    // the b1 error sums: as launch_b1_error_sums lays them out
+    const int slabs = (it.d.c_out + kClassSlab - 1) / kClassSlab;
+    int blocks = (sm_count + slabs - 1) / slabs;
+    size_t ppb = ((size_t)it.pixels + blocks - 1) / blocks;
+    if (ppb < 64) ppb = 64;
+    if (ppb > (1u << 23)) ppb = 1u << 23;
+    it.pixels_per_block = (int)ppb;
+    it.tap_grid_x = (int)(((size_t)it.pixels + ppb - 1) / ppb);
+    it.tap_grid_y = slabs;
+    // slice sums and codes: as launch_sq_i64 sizes them, with a smaller cap (many tensors share the device)
+    it.groups = !it.parts ? 1 : (it.num_parts >= 32 ? 8 : (it.num_parts >= 8 ? 4 : 1));
+    const int bw = 256 / it.groups;
+    size_t fb = ((size_t)it.n + bw - 1) / bw;
+    if (fb > (size_t)sm_count * 4) fb = (size_t)sm_count * 4;
+    it.fin_blocks = (int)(fb < 1 ? 1 : fb);
+    size_t qb = ((size_t)it.n / 4 + kThreads - 1) / kThreads;
+    if (qb > (size_t)sm_count * 2) qb = (size_t)sm_count * 2;
+    it.sq_blocks = (int)(qb < 1 ? 1 : qb);
+}
+
+cudaError_t launch_wgrad_finish(const FinishBatch &b, unsigned *status, cudaStream_t s)
+{
+    int max_classes = 1;
+    for (int k = 0; k < b.num; ++k) {
+        const int c = b.item[k].bc.nrc * b.item[k].bc.ncc;
+        if (b.item[k].b1_dev && c > max_classes) max_classes = c;
+    }
+    const size_t smem = sizeof(int32_t) * max_classes * kClassSlab;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(finish_taps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    finish_zero_kernel<<<b.num, 256, 0, s>>>(b);
+    finish_taps_kernel<<<b.tap_first[b.num], 256, smem, s>>>(b);
+    finish_sums_kernel<<<b.fin_first[b.num], 256, 0, s>>>(b);
+    finish_code_kernel<<<b.sq_first[b.num], kThreads, 0, s>>>(b, status);
     return cudaGetLastError();
 }
 

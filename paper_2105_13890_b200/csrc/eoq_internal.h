@@ -347,6 +347,36 @@ struct ScalarBatch {
     ScalarItem item[kScalarChunk];
     int num;
 };
+// Finish of the weight gradients of many layers in a few launches (eoq_wgrad_finish): per layer the b1 error sums,
+// the sum of the split-K slices plus the b1 term, and Q_g.  One item per layer; blocks find their item by their index.
+constexpr int kFinishChunk = 16;
+struct FinishItem {
+    const int8_t *e3;
+    const int32_t *e3_exp;
+    const int32_t *b1_dev;         // null: no b1 term (then the tap sums are neither formed nor read)
+    long long *tap_sums;           // kTapReplicas copies, tap_stride elements apart; zeroed by the finish itself
+    unsigned long long *max_cell;  // max |sum| of the layer (in the spare bytes behind the tap sums)
+    long long *acc;                // exact sums [oc][tap][ic]
+    const int32_t *parts;          // int32 split-K slices, or null when the GEMM added into acc
+    int8_t *g;
+    int32_t *g_exp;
+    unsigned long long n;          // weights
+    unsigned long long tap_stride, zero_bytes;
+    unsigned long long pixels;
+    eoq_conv_desc_t d;
+    BorderClasses bc;
+    int ho, wo, pixels_per_block, tap_grid_x, tap_grid_y;
+    int num_parts, groups, fin_blocks, sq_blocks;
+};
+struct FinishBatch {
+    int num;
+    int tap_first[kFinishChunk + 1], fin_first[kFinishChunk + 1], sq_first[kFinishChunk + 1];
+    FinishItem item[kFinishChunk];
+};
+// fills the launch geometry of an item (tap grid, block counts) from its sizes
+void plan_finish_item(FinishItem &it, int sm_count);
+cudaError_t launch_wgrad_finish(const FinishBatch &b, unsigned *status, cudaStream_t s);
+
 // Batch normalisation behind the convolution (comparison case, eoq_bn.cu): per-channel record in the workspace
 struct BnChannel {
     long long s1, shh, shl, sll;   // sum of A; sum of A^2 in three parts (A = h * 2^16 + l): h*h, h*l, l*l

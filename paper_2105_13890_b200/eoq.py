@@ -27,7 +27,7 @@ EXPORTS = [
     "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count", "eoq_set_gemm_ctas",
     "eoq_conv_dgrad_static", "eoq_conv_fwd_dev", "eoq_weight_prep_size", "eoq_weight_prep", "eoq_conv_wgrad_dev",
     "eoq_err_prescale_dev", "eoq_update_dev", "eoq_describe_plan", "eoq_debug_force_wait_timeout", "eoq_probe_mma_i8", "eoq_profile_gemm_only", "eoq_aux_maxpool_fwd", "eoq_aux_maxpool_bwd",
-    "eoq_aux_maxpool_bwd_head", "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_join_head", "eoq_conv_dgrad_head", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_update", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide", "eoq_set_reduce_hook", "eoq_bn_workspace_size", "eoq_bn_fwd", "eoq_bn_bwd",
+    "eoq_aux_maxpool_bwd_head", "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_join_head", "eoq_conv_dgrad_head", "eoq_conv_wgrad_gemm", "eoq_wgrad_finish", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_update", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide", "eoq_set_reduce_hook", "eoq_bn_workspace_size", "eoq_bn_fwd", "eoq_bn_bwd",
 ]
 EOQ_STATIC_SCRATCH_BYTES = 16 << 20
 EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
@@ -112,6 +112,9 @@ def lib() -> C.CDLL:
         L.eoq_aux_maxpool_bwd_head.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
         L.eoq_aux_avgpool_sum.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         L.eoq_aux_join.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp, vp, vp, vp]
+        L.eoq_conv_wgrad_gemm.argtypes = [vp, dp, vp, vp, vp, vp, sz, C.POINTER(ci), vp]
+        L.eoq_wgrad_finish.argtypes = [vp, ci, dp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
+                                       C.POINTER(vp), C.POINTER(sz), C.POINTER(ci), vp]
         L.eoq_conv_dgrad_head.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.eoq_aux_join_head.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.eoq_aux_head_workspace_size.argtypes = [ci, ci, ci, C.POINTER(sz)]
@@ -324,6 +327,25 @@ def eoq_weight_prep(handle, descs: Sequence[eoq_conv_desc_t], w: Sequence, prep:
     if check:
         _check(st, "eoq_weight_prep")
     return st
+
+
+def eoq_conv_wgrad_gemm(handle, desc, e3, e3_exp, x, workspace, stream=None) -> int:
+    """The weight-gradient GEMM alone; returns the slice count eoq_wgrad_finish needs for this layer."""
+    parts = C.c_int(0)
+    _check(lib().eoq_conv_wgrad_gemm(handle, C.byref(desc), _ptr(e3), _ptr(e3_exp), _ptr(x), _ptr(workspace), _nbytes(workspace),
+                                     C.byref(parts), _stream(stream)), "eoq_conv_wgrad_gemm")
+    return parts.value
+
+
+def eoq_wgrad_finish(handle, descs: Sequence[eoq_conv_desc_t], e3: Sequence, e3_exp: Sequence, b1_c: Sequence, g: Sequence,
+                     g_exp: Sequence, workspace: Sequence, num_parts: Sequence[int], stream=None) -> None:
+    num = len(descs)
+    darr = (eoq_conv_desc_t * num)(*descs)
+    arr = C.c_void_p * num
+    _check(lib().eoq_wgrad_finish(handle, num, darr, arr(*[_ptr(t) for t in e3]), arr(*[_ptr(t) for t in e3_exp]),
+                                  arr(*[_ptr(t) for t in b1_c]), arr(*[_ptr(t) for t in g]), arr(*[_ptr(t) for t in g_exp]),
+                                  arr(*[_ptr(t) for t in workspace]), (C.c_size_t * num)(*[_nbytes(t) for t in workspace]),
+                                  (C.c_int * num)(*[int(v) for v in num_parts]), _stream(stream)), "eoq_wgrad_finish")
 
 
 def eoq_conv_wgrad_dev(handle, desc, e3, e3_exp, x, b1_c, g, g_exp, workspace=None, stream=None, check: bool = True) -> int:
