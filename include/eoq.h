@@ -170,6 +170,18 @@ EOQ_API int eoq_conv_dgrad_head(eoq_handle_t handle, const eoq_conv_desc_t *desc
                         const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4, const uint8_t *next_relu_mask,
                         const int16_t *next_x2, const int32_t *next_gamma, int8_t *next_e3, int32_t *next_e3_exp,
                         int64_t *next_sum_e1, int64_t *next_sum_e1x2, void *workspace, size_t workspace_bytes, void *stream);
+/*
+ * eoq_conv_dgrad followed by the error join that takes e4 as its first operand (eoq_aux_join: out = Q_e(e4 + b), b
+ * gated by mask_b when given) and, when next_relu_mask is not NULL, by the error head of the layer that consumes `out`
+ * (eoq_aux_join_head's arguments).  Three kernels instead of five: the join's first pass (its two maxima) rides on the
+ * Q_e pass that writes e4.  Bit-identical to the separate calls.  EOQ_ERR_UNSUPPORTED for strided 1x1 filters.
+ */
+EOQ_API int eoq_conv_dgrad_join_head(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                             const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4, const int8_t *b, const int32_t *b_exp,
+                             const uint8_t *mask_b, int8_t *out, int32_t *out_exp, int64_t *sum_out,
+                             const uint8_t *next_relu_mask, const int16_t *next_x2, const int32_t *next_gamma, int8_t *next_e3,
+                             int32_t *next_e3_exp, int64_t *next_sum_e1, int64_t *next_sum_e1x2, void *workspace,
+                             size_t workspace_bytes, void *stream);
 
 /*
  * eoq_conv_dgrad without any allocation (the paper has no counterpart; this is a deployment variant).

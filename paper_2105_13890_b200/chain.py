@@ -283,7 +283,6 @@ class ChainedStep:
             eoq.eoq_conv_dgrad_head(h, b.desc, b.e3, b.e3_exp, b.w, b.e4, b.e4_exp, b.sum_e4, a.mask, None, a.scal[1:2], a.e3,
                                     a.e3_exp, a.sum_e1, None, ws)
             wgrad(a, a.scal[0:1])
-            eoq.eoq_conv_dgrad(h, a.desc, a.e3, a.e3_exp, a.w, a.e4, a.e4_exp, a.sum_e4, None, ws)
             if pr:
                 # the error entering the shortcut is e1 of unit B: e_out gated by unit B's ReLU mask
                 eoq.eoq_err_prescale_dev(h, e_out, e_exp, b.mask, None, pr.n_out, self.c128, pr.e3, pr.e3_exp, pr.sum_e1, None)
@@ -292,16 +291,17 @@ class ChainedStep:
                 j_b, j_b_exp, j_mask = pr.e4, pr.e4_exp, None
             else:
                 j_b, j_b_exp, j_mask = e_out, e_exp, b.mask
-            # the joined error feeds the last unit of the block in front (or the first layer when no pool sits between):
-            # that unit's error head rides on the join
+            # error back through unit A, joined with the shortcut's error; the joined error feeds the last unit of the
+            # block in front (or the first layer when no pool sits between), whose error head rides on the join
             nxt = self.blocks[i - 1].b if i > 0 else (None if self.pool else stem)
             if nxt is not None:
-                eoq.eoq_aux_join_head(h, a.e4, a.e4_exp, j_b, j_b_exp, j_mask, a.e4.numel(), blk.e_in, blk.e_in_exp, blk.sum_join,
-                                      nxt.mask, nxt.x2, nxt.scal[1:2], nxt.e3, nxt.e3_exp, nxt.sum_e1,
-                                      nxt.sum_e1x2 if nxt.x2 is not None else None)
+                eoq.eoq_conv_dgrad_join_head(h, a.desc, a.e3, a.e3_exp, a.w, a.e4, a.e4_exp, a.sum_e4, j_b, j_b_exp, j_mask, blk.e_in,
+                                             blk.e_in_exp, blk.sum_join, nxt.mask, nxt.x2, nxt.scal[1:2], nxt.e3, nxt.e3_exp,
+                                             nxt.sum_e1, nxt.sum_e1x2 if nxt.x2 is not None else None, ws)
                 head_done = True
             else:
-                eoq.eoq_aux_join(h, a.e4, a.e4_exp, j_b, j_b_exp, j_mask, a.e4.numel(), blk.e_in, blk.e_in_exp, blk.sum_join)
+                eoq.eoq_conv_dgrad_join_head(h, a.desc, a.e3, a.e3_exp, a.w, a.e4, a.e4_exp, a.sum_e4, j_b, j_b_exp, j_mask, blk.e_in,
+                                             blk.e_in_exp, blk.sum_join, workspace=ws)
                 head_done = False
             e_out, e_exp = blk.e_in, blk.e_in_exp
         finish(pending)

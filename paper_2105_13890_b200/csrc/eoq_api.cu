@@ -815,10 +815,23 @@ extern "C" int eoq_weight_prep(eoq_handle_t handle, int num, const eoq_conv_desc
 
 // ================================================================================= error back-propagation
 
-// `next`: the error head of the layer that consumes e4, fused into Q_e (null for the plain call)
+// The error join that takes e4 as its first operand, run behind the dgrad (eoq_conv_dgrad_join_head): the join's first
+// pass rides on Q_e, its second pass follows; `next` there is the head of the layer that consumes the joined error.
+struct JoinCall {
+    const int8_t *b;
+    const int32_t *b_exp;
+    const uint8_t *mask_b;
+    int8_t *out;
+    int32_t *out_exp;
+    long long *sum_out;
+    const NextHeadArgs *next;
+};
+
+// `next`: the error head of the layer that consumes e4, fused into Q_e (null for the plain call); `jc`: see JoinCall
 static int conv_dgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
                            const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4, int32_t *acc_dump,
-                           const NextHeadArgs *next, void *workspace, size_t workspace_bytes, void *stream)
+                           const NextHeadArgs *next, void *workspace, size_t workspace_bytes, void *stream,
+                           const JoinCall *jc = nullptr)
 {
     Handle *h = reinterpret_cast<Handle *>(handle);
     Geometry g;
@@ -834,6 +847,39 @@ static int conv_dgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
         // the compact sums of a strided 1x1 filter are not laid out like the error tensor
         if (desc->kh == 1 && desc->kw == 1 && desc->pad == 0 && desc->stride > 1) return EOQ_ERR_UNSUPPORTED;
     }
+    JoinStatArgs jstat{};
+    const JoinStatArgs *jstat_p = nullptr;
+    if (jc) {
+        if (!jc->b || !jc->b_exp || !jc->out || !jc->out_exp || (g.in_elems % 16)) return EOQ_ERR_BAD_ARG;
+        if (!aligned16(jc->b) || !aligned16(jc->out) || (reinterpret_cast<uintptr_t>(jc->mask_b) & 1)) return EOQ_ERR_ALIGNMENT;
+        if (jc->next) {
+            if (!jc->next->mask || !jc->next->gamma || !jc->next->e3 || !jc->next->e3_exp) return EOQ_ERR_BAD_ARG;
+            if (!aligned16(jc->next->e3) || (jc->next->x2 && !aligned16(jc->next->x2)) ||
+                (reinterpret_cast<uintptr_t>(jc->next->mask) & 1))
+                return EOQ_ERR_ALIGNMENT;
+        }
+        if (desc->kh == 1 && desc->kw == 1 && desc->pad == 0 && desc->stride > 1) return EOQ_ERR_UNSUPPORTED;
+        if (!h->hook.fn) {   // with replicas the join runs as its own two passes, each followed by its exchange
+            jstat = JoinStatArgs{jc->b, jc->b_exp, jc->mask_b, jc->next ? jc->next->mask : nullptr};
+            jstat_p = &jstat;
+        }
+    }
+    // what follows Q_e when a join was asked for
+    auto join_after = [&](cudaError_t e, cudaStream_t st) -> int {
+        if (e != cudaSuccess || !jc) return record(h, e);
+        ProfScope prof(h, EOQ_PROF_GLUE, st);
+        if (jstat_p) {
+            count_launches(h, 1);
+            return record(h, launch_join_second(e4, e4_exp, jc->b, jc->b_exp, jc->mask_b, g.in_elems, jc->out, jc->out_exp, jc->sum_out,
+                                                jc->next, h->dev, h->sm_count, st));
+        }
+        count_launches(h, 2);
+        const NextHeadArgs *n = jc->next;
+        return record(h, launch_join(e4, e4_exp, jc->b, jc->b_exp, jc->mask_b, g.in_elems, jc->out, jc->out_exp, jc->sum_out,
+                                     n ? n->mask : nullptr, n ? n->x2 : nullptr, n ? n->gamma : nullptr, n ? n->e3 : nullptr,
+                                     n ? n->e3_exp : nullptr, n ? n->sum_e1 : nullptr, n ? n->sum_e1x2 : nullptr, h->dev, h->sm_count,
+                                     st, h->hook));
+    };
     if ((st = check_workspace(desc, EOQ_PASS_DGRAD, workspace, workspace_bytes)) != EOQ_OK) return st;
     const eoq_conv_desc_t &d = *desc;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
@@ -878,10 +924,10 @@ static int conv_dgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
             {
                 ProfScope prof(h, EOQ_PROF_DGRAD_AUX, s);
                 e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true,
-                                  h->dev, h->sm_count, s, h->hook, next);
+                                  h->dev, h->sm_count, s, h->hook, next, jstat_p);
             }
             count_launches(h, 1);
-            return record(h, e);
+            return join_after(e, s);
         }
     }
     // With at least 32 output channels per K chunk the per-class GEMMs read the weights in place as MN-major atoms
@@ -1042,10 +1088,10 @@ static int conv_dgrad_impl(eoq_handle_t handle, const eoq_conv_desc_t *desc, con
                                       h->dev, h->sm_count, s, h->hook);
         else
             e = launch_sq_i32(sums, e3_exp, -7, g.in_elems, e4, e4_exp, reinterpret_cast<long long *>(sum_e4), true, h->dev,
-                              h->sm_count, s, h->hook, next);
+                              h->sm_count, s, h->hook, next, jstat_p);
     }
     count_launches(h, 1);
-    return record(h, e);
+    return join_after(e, s);
 }
 
 extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3,
@@ -1053,6 +1099,19 @@ extern "C" int eoq_conv_dgrad(eoq_handle_t handle, const eoq_conv_desc_t *desc, 
                               int32_t *acc_dump, void *workspace, size_t workspace_bytes, void *stream)
 {
     return conv_dgrad_impl(handle, desc, e3, e3_exp, w, e4, e4_exp, sum_e4, acc_dump, nullptr, workspace, workspace_bytes, stream);
+}
+
+extern "C" int eoq_conv_dgrad_join_head(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,
+                                        const int8_t *w, int8_t *e4, int32_t *e4_exp, int64_t *sum_e4, const int8_t *b,
+                                        const int32_t *b_exp, const uint8_t *mask_b, int8_t *out, int32_t *out_exp, int64_t *sum_out,
+                                        const uint8_t *next_relu_mask, const int16_t *next_x2, const int32_t *next_gamma,
+                                        int8_t *next_e3, int32_t *next_e3_exp, int64_t *next_sum_e1, int64_t *next_sum_e1x2,
+                                        void *workspace, size_t workspace_bytes, void *stream)
+{
+    const NextHeadArgs next{next_relu_mask, next_x2, next_gamma, next_e3, next_e3_exp, reinterpret_cast<long long *>(next_sum_e1),
+                            reinterpret_cast<long long *>(next_sum_e1x2)};
+    const JoinCall jc{b, b_exp, mask_b, out, out_exp, reinterpret_cast<long long *>(sum_out), next_relu_mask ? &next : nullptr};
+    return conv_dgrad_impl(handle, desc, e3, e3_exp, w, e4, e4_exp, sum_e4, nullptr, nullptr, workspace, workspace_bytes, stream, &jc);
 }
 
 extern "C" int eoq_conv_dgrad_head(eoq_handle_t handle, const eoq_conv_desc_t *desc, const int8_t *e3, const int32_t *e3_exp,

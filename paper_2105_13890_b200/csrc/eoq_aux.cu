@@ -256,26 +256,6 @@ __global__ void avgpool_sum_kernel(const int8_t *__restrict__ x, int hw, int c, 
 
 // ------------------------------------------------------------------ join of two error streams + Q_e
 
-struct JoinShift {
-    int sa, sb, p;  // left shifts of the two operands (-1: operand dropped) and the exponent of the sums
-};
-__device__ __forceinline__ JoinShift join_shift(int pa, int pb)
-{
-    JoinShift j;
-    const int p = min(pa, pb);
-    j.sa = pa - p;
-    j.sb = pb - p;
-    j.p = p;
-    if (j.sa > 31) { j.sb = -1; j.sa = 0; j.p = pa; }        // b lies more than 31 octaves below a
-    else if (j.sb > 31) { j.sa = -1; j.sb = 0; j.p = pb; }
-    return j;
-}
-__device__ __forceinline__ long long join_one(int a, int b, const JoinShift &j)
-{
-    const long long va = j.sa < 0 ? 0ll : (long long)a * (1ll << j.sa);
-    const long long vb = j.sb < 0 ? 0ll : (long long)b * (1ll << j.sb);
-    return va + vb;
-}
 __device__ __forceinline__ void unpack16(const int4 &v, int (&o)[16])
 {
     const int8_t *b = reinterpret_cast<const int8_t *>(&v);
@@ -789,6 +769,21 @@ cudaError_t launch_join(const int8_t *a, const int32_t *a_exp, const int8_t *b, 
                                                            nullptr, nullptr, nullptr, nullptr, nullptr, dev);
         if (sum_out) hook(sum_out, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, st);
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_join_second(const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp, const uint8_t *mask_b,
+                               size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, const NextHeadArgs *next,
+                               DeviceState *dev, int sm_count, cudaStream_t st)
+{
+    const size_t n16 = n_el / 16;
+    const int blocks = blocks_for(n16, sm_count, 8);
+    if (next)
+        join_kernel<1, true><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, next->mask, next->x2,
+                                                          next->gamma, next->e3, next->e3_exp, next->sum_e1, next->sum_e1x2, dev);
+    else
+        join_kernel<1, false><<<blocks, kThreads, 0, st>>>(a, a_exp, b, b_exp, mask_b, n16, out, out_exp, sum_out, nullptr, nullptr,
+                                                           nullptr, nullptr, nullptr, nullptr, nullptr, dev);
     return cudaGetLastError();
 }
 

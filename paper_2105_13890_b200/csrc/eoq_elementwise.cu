@@ -231,9 +231,12 @@ __global__ void absmax_i32_kernel(const int32_t *__restrict__ src, size_t n, Dev
 // kNext: the error head of the layer that consumes dst rides along (see NextHead): the masked maximum sits in the
 // handle's 64-bit cell (the GEMM epilogue reduced it beside the plain one), so the codes of e3 and the head's sums
 // come out of the same pass.  n must then be a multiple of 16.
-template <bool kNext>
+// kJoin: dst is the first operand of an error join; the join's first pass rides along: max |dst * 2^sa + b * 2^sb|
+// over all positions (64-bit cell) and over those the consumer's ReLU lets through (second 64-bit cell).
+template <bool kNext, bool kJoin>
 __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *src_exp, int exp_bias, size_t n,
-                              int8_t *dst, int32_t *dst_exp, long long *sum_codes, NextHeadArgs next, DeviceState *dev)
+                              int8_t *dst, int32_t *dst_exp, long long *sum_codes, NextHeadArgs next, JoinStatArgs join,
+                              DeviceState *dev)
 {
     const uint32_t M = dev->absmax_u32;
     const int t = M ? round_log2_u32(M) : 7;
@@ -250,6 +253,16 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
     const size_t n16 = n / 16;
     const int4 *s4 = reinterpret_cast<const int4 *>(src);
     const int sh = t - 7;
+    JoinShift js = {0, 0, 0};
+    bool j_narrow = true;
+    int j_ma = 1, j_mb = 1;
+    unsigned long long jmx = 0, jmxm = 0;
+    if (kJoin) {
+        js = join_shift(p0, __ldg(join.b_exp));
+        j_narrow = js.sa >= 0 && js.sb >= 0 && js.sa <= 23 && js.sb <= 23;
+        j_ma = 1 << (js.sa < 0 ? 0 : min(js.sa, 23));
+        j_mb = 1 << (js.sb < 0 ? 0 : min(js.sb, 23));
+    }
     // the maximum bounds every element, so |a| + 2^(sh-1) cannot wrap as long as M + M / 2^7 < 2^31
     const bool fast = sh >= 1 && M < 0x7e000000u;
     const int32_t half_m1 = fast ? (1 << (sh - 1)) - 1 : 0;
@@ -281,6 +294,25 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
         reinterpret_cast<int4 *>(dst)[i] =
             make_int4((int)pack4(c[0], c[1], c[2], c[3]), (int)pack4(c[4], c[5], c[6], c[7]),
                       (int)pack4(c[8], c[9], c[10], c[11]), (int)pack4(c[12], c[13], c[14], c[15]));
+        if (kJoin) {
+            const int4 bq = __ldg(reinterpret_cast<const int4 *>(join.b) + i);
+            const int8_t *bb = reinterpret_cast<const int8_t *>(&bq);
+            const uint32_t gate = join.mask_b ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(join.mask_b) + i) : 0xffffu;
+            const uint32_t nm = join.next_mask ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(join.next_mask) + i) : 0u;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const int bv = ((gate >> k) & 1u) ? (int)bb[k] : 0;
+                unsigned long long u;
+                if (j_narrow) {
+                    u = (unsigned long long)(uint32_t)abs(c[k] * j_ma + bv * j_mb);
+                } else {
+                    const long long v = join_one(c[k], bv, js);
+                    u = (unsigned long long)(v < 0 ? -v : v);
+                }
+                jmx = u > jmx ? u : jmx;
+                if ((nm >> k) & 1u) jmxm = u > jmxm ? u : jmxm;
+            }
+        }
         if (kNext) {
             const uint32_t bits = (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(next.mask) + i);
             int e1[16], c3[16], a1 = 0;
@@ -305,7 +337,7 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
                           (int)pack4(c3[8], c3[9], c3[10], c3[11]), (int)pack4(c3[12], c3[13], c3[14], c3[15]));
         }
     }
-    if (!kNext)
+    if (!kNext && !kJoin)
         for (size_t i = n16 * 16 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
             const int c = sq_code32(src[i], t);
             sum += c;
@@ -321,6 +353,15 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
         if (threadIdx.x == 0) {
             if (s1) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum1), (unsigned long long)s1);
             if (s2) atomicAdd(reinterpret_cast<unsigned long long *>(&dev->sum2), (unsigned long long)s2);
+        }
+    }
+    if (kJoin) {
+        // the join's second pass (the next kernel on the stream) reads these cells and puts them back to zero
+        jmx = block_max_u64(jmx);
+        jmxm = block_max_u64(jmxm);
+        if (threadIdx.x == 0) {
+            if (jmx) atomicMax(&dev->absmax_u64, jmx);
+            if (jmxm) atomicMax(&dev->absmax2_u64, jmxm);
         }
     }
     if (last_block_done(dev)) {
@@ -1277,20 +1318,23 @@ cudaError_t launch_weight_pad_rows(const int8_t *w, int8_t *wp, int c_out, int k
 
 cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *sum_codes, bool max_already_reduced, DeviceState *dev,
-                          int sm_count, cudaStream_t s, const ReduceHook &hook, const NextHeadArgs *next)
+                          int sm_count, cudaStream_t s, const ReduceHook &hook, const NextHeadArgs *next, const JoinStatArgs *join)
 {
     if (!max_already_reduced) absmax_i32_kernel<<<grid_for(n / 4 + 1, sm_count), kThreads, 0, s>>>(src, n, dev);
     hook(&dev->absmax_u32, 1, EOQ_REDUCE_I32, EOQ_REDUCE_MAX, s);
-    if (next) {
+    const int grid = grid_for(n / 16 + 1, sm_count);
+    if (join) {
+        // (no hook in this form: callers with replicas take the separate calls)
+        sq_i32_kernel<false, true><<<grid, kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes, NextHeadArgs{}, *join, dev);
+    } else if (next) {
         // (only behind a GEMM whose epilogue reduced the masked maximum)
         hook(&dev->absmax_u64, 1, EOQ_REDUCE_I64, EOQ_REDUCE_MAX, s);
-        sq_i32_kernel<true><<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes, *next,
-                                                                              dev);
+        sq_i32_kernel<true, false><<<grid, kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes, *next, JoinStatArgs{}, dev);
         if (next->sum_e1) hook(next->sum_e1, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, s);
         if (next->sum_e1x2) hook(next->sum_e1x2, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, s);
     } else {
-        sq_i32_kernel<false><<<grid_for(n / 16 + 1, sm_count), kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes,
-                                                                               NextHeadArgs{}, dev);
+        sq_i32_kernel<false, false><<<grid, kThreads, 0, s>>>(src, src_exp, exp_bias, n, dst, dst_exp, sum_codes, NextHeadArgs{},
+                                                              JoinStatArgs{}, dev);
     }
     if (sum_codes) hook(sum_codes, 1, EOQ_REDUCE_I64, EOQ_REDUCE_SUM, s);
     return cudaGetLastError();

@@ -46,6 +46,15 @@ struct NextHeadArgs {
     long long *sum_e1, *sum_e1x2;
 };
 
+// The first pass of an error join (its two maxima) riding on the Q_e pass that writes the join's first operand
+// (eoq_conv_dgrad_join_head): operand b with its exponent and gate bits, and the consumer's mask for the masked maximum.
+struct JoinStatArgs {
+    const int8_t *b;
+    const int32_t *b_exp;
+    const uint8_t *mask_b;     // gate bits of b, or null
+    const uint8_t *next_mask;  // ReLU mask of the layer that consumes the joined error, or null
+};
+
 struct ReduceHook {
     eoq_reduce_fn fn;
     void *user;
@@ -248,7 +257,8 @@ cudaError_t launch_quantize_f32(int mode, const float *src, size_t n, void *dst,
                                 int sm_count, cudaStream_t s, const ReduceHook &hook);
 cudaError_t launch_sq_i32(const int32_t *src, const int32_t *src_exp, int exp_bias, size_t n, int8_t *dst,
                           int32_t *dst_exp, long long *sum_codes, bool max_already_reduced, DeviceState *dev,
-                          int sm_count, cudaStream_t s, const ReduceHook &hook, const NextHeadArgs *next = nullptr);
+                          int sm_count, cudaStream_t s, const ReduceHook &hook, const NextHeadArgs *next = nullptr,
+                          const JoinStatArgs *join = nullptr);
 // Q_g of the exact sums.  `src` holds int64 sums; when `parts` is given the sums are first formed from
 // `num_parts` int32 slices of n elements each (and written to src).
 cudaError_t launch_sq_i32_scatter(const int32_t *src, const int32_t *src_exp, int exp_bias, int n_img, int hh, int ww, int c,
@@ -326,6 +336,10 @@ cudaError_t launch_join(const int8_t *a, const int32_t *a_exp, const int8_t *b, 
                         size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, const uint8_t *next_mask,
                         const int16_t *next_x2, const int32_t *next_gamma, int8_t *e3, int32_t *e3_exp, long long *sum_e1,
                         long long *sum_e1x2, DeviceState *dev, int sm_count, cudaStream_t st, const ReduceHook &hook);
+// the second pass of launch_join alone: the maxima are already in the handle's cells (see JoinStatArgs)
+cudaError_t launch_join_second(const int8_t *a, const int32_t *a_exp, const int8_t *b, const int32_t *b_exp, const uint8_t *mask_b,
+                               size_t n_el, int8_t *out, int32_t *out_exp, long long *sum_out, const NextHeadArgs *next,
+                               DeviceState *dev, int sm_count, cudaStream_t st);
 cudaError_t launch_head(const int32_t *sums, int n, int c, int hw, int classes, float *W, float *bias, const int32_t *labels,
                         float lr, float *loss_out, float *dpooled, float *logits, float *pooled, float *dl, double *loss_n,
                         cudaStream_t st);

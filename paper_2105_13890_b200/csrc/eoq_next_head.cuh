@@ -47,4 +47,27 @@ __device__ __forceinline__ void next_head_exponent(const NextHead &nh, int p0, i
 }
 
 
+// Join of two error streams: both at the smaller exponent, added exactly; an operand more than 31 octaves below the
+// other is dropped.
+struct JoinShift {
+    int sa, sb, p;  // left shifts of the two operands (-1: operand dropped) and the exponent of the sums
+};
+__device__ __forceinline__ JoinShift join_shift(int pa, int pb)
+{
+    JoinShift j;
+    const int p = min(pa, pb);
+    j.sa = pa - p;
+    j.sb = pb - p;
+    j.p = p;
+    if (j.sa > 31) { j.sb = -1; j.sa = 0; j.p = pa; }        // b lies more than 31 octaves below a
+    else if (j.sb > 31) { j.sa = -1; j.sb = 0; j.p = pb; }
+    return j;
+}
+__device__ __forceinline__ long long join_one(int a, int b, const JoinShift &j)
+{
+    const long long va = j.sa < 0 ? 0ll : (long long)a * (1ll << j.sa);
+    const long long vb = j.sb < 0 ? 0ll : (long long)b * (1ll << j.sb);
+    return va + vb;
+}
+
 }  // namespace eoq

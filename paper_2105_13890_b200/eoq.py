@@ -27,7 +27,7 @@ EXPORTS = [
     "eoq_last_cuda_error", "eoq_status_string", "eoq_profile_start", "eoq_profile_stop", "eoq_launch_count", "eoq_set_gemm_ctas",
     "eoq_conv_dgrad_static", "eoq_conv_fwd_dev", "eoq_weight_prep_size", "eoq_weight_prep", "eoq_conv_wgrad_dev",
     "eoq_err_prescale_dev", "eoq_update_dev", "eoq_describe_plan", "eoq_debug_force_wait_timeout", "eoq_probe_mma_i8", "eoq_profile_gemm_only", "eoq_aux_maxpool_fwd", "eoq_aux_maxpool_bwd",
-    "eoq_aux_maxpool_bwd_head", "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_join_head", "eoq_conv_dgrad_head", "eoq_conv_wgrad_gemm", "eoq_wgrad_finish", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_update", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide", "eoq_set_reduce_hook", "eoq_bn_workspace_size", "eoq_bn_fwd", "eoq_bn_bwd",
+    "eoq_aux_maxpool_bwd_head", "eoq_aux_avgpool_sum", "eoq_aux_join", "eoq_aux_join_head", "eoq_conv_dgrad_head", "eoq_conv_dgrad_join_head", "eoq_conv_wgrad_gemm", "eoq_wgrad_finish", "eoq_aux_head_workspace_size", "eoq_aux_head", "eoq_aux_head_update", "eoq_aux_head_error", "eoq_aux_scalar_update", "eoq_update_wide", "eoq_set_reduce_hook", "eoq_bn_workspace_size", "eoq_bn_fwd", "eoq_bn_bwd",
 ]
 EOQ_STATIC_SCRATCH_BYTES = 16 << 20
 EOQ_PROF_IGEMM_FWD, EOQ_PROF_IGEMM_DGRAD, EOQ_PROF_WGRAD = 0, 1, 2
@@ -115,6 +115,7 @@ def lib() -> C.CDLL:
         L.eoq_conv_wgrad_gemm.argtypes = [vp, dp, vp, vp, vp, vp, sz, C.POINTER(ci), vp]
         L.eoq_wgrad_finish.argtypes = [vp, ci, dp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
                                        C.POINTER(vp), C.POINTER(sz), C.POINTER(ci), vp]
+        L.eoq_conv_dgrad_join_head.argtypes = [vp, dp] + [vp] * 19 + [vp, sz, vp]
         L.eoq_conv_dgrad_head.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.eoq_aux_join_head.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.eoq_aux_head_workspace_size.argtypes = [ci, ci, ci, C.POINTER(sz)]
@@ -446,6 +447,16 @@ def eoq_aux_avgpool_sum(handle, x, n, hw, c, sums, stream=None) -> None:
 def eoq_aux_join(handle, a, a_exp, b, b_exp, mask_b, n_el, out, out_exp, sum_out=None, stream=None) -> None:
     _check(lib().eoq_aux_join(handle, _ptr(a), _ptr(a_exp), _ptr(b), _ptr(b_exp), _ptr(mask_b), int(n_el), _ptr(out),
                               _ptr(out_exp), _ptr(sum_out), _stream(stream)), "eoq_aux_join")
+
+
+def eoq_conv_dgrad_join_head(handle, desc, e3, e3_exp, w, e4, e4_exp, sum_e4, b, b_exp, mask_b, out, out_exp, sum_out, next_mask=None,
+                             next_x2=None, next_gamma=None, next_e3=None, next_e3_exp=None, next_sum_e1=None, next_sum_e1x2=None,
+                             workspace=None, stream=None) -> None:
+    _check(lib().eoq_conv_dgrad_join_head(handle, C.byref(desc), _ptr(e3), _ptr(e3_exp), _ptr(w), _ptr(e4), _ptr(e4_exp), _ptr(sum_e4),
+                                          _ptr(b), _ptr(b_exp), _ptr(mask_b), _ptr(out), _ptr(out_exp), _ptr(sum_out), _ptr(next_mask),
+                                          _ptr(next_x2), _ptr(next_gamma), _ptr(next_e3), _ptr(next_e3_exp), _ptr(next_sum_e1),
+                                          _ptr(next_sum_e1x2), _ptr(workspace), _nbytes(workspace), _stream(stream)),
+           "eoq_conv_dgrad_join_head")
 
 
 def eoq_conv_dgrad_head(handle, desc, e3, e3_exp, w, e4, e4_exp, sum_e4, next_mask, next_x2, next_gamma, next_e3, next_e3_exp,

@@ -248,3 +248,46 @@ def test_dgrad_head_refuses_the_compact_strided_1x1_case():
         eoq.eoq_conv_dgrad_head(hd, gd, z8((2, 4, 4, 64)), i32(-11), z8((64, 1, 1, 32)), z8((2, 8, 8, 32)), G.zeros(1, torch.int32), None,
                                 G.zeros(2 * 8 * 8 * 32 // 8, torch.uint8), None, i32(128), z8((2, 8, 8, 32)), G.zeros(1, torch.int32),
                                 None, None, G.workspace(gd, eoq.EOQ_PASS_DGRAD))
+
+
+@pytest.mark.parametrize("n,h,w,c_in,c_out,k,stride,pad", DGRADS)
+@pytest.mark.parametrize("pb,gated,with_head", [(-17, True, True), (-20, False, True), (-50, True, False), (-3, True, True)])
+def test_dgrad_join_and_head_in_one_call(n, h, w, c_in, c_out, k, stride, pad, pb, gated, with_head):
+    """eoq_conv_dgrad_join_head against the oracle's dgrad + Q_e, join + Q_e and error head (join exponents that take the
+    32-bit path, the 64-bit path and the dropping rule in both directions)."""
+    hd = G.handle()
+    d = ConvDesc(n, h, w, c_in, c_out, k, k, stride, pad)
+    gd = G.gdesc(d)
+    e3 = synth.normal_codes((n, d.ho, d.wo, c_out), 8650 + h, 0)
+    wt = synth.int8_uniform((c_out, k, k, c_in), 8650 + h, 1, -30, 30)
+    in_shape = (n, h, w, c_in)
+    b = synth.normal_codes(in_shape, 8650 + h, 2)
+    gate01 = synth.bits(in_shape, 8650 + h, 3, 0.6) if gated else None
+    mask01 = synth.bits(in_shape, 8650 + h, 4, 0.5)
+    x2 = (synth.relu_codes(in_shape, 8650 + h, 5).astype(np.int32) * 23 - 500).astype(np.int16)
+    S = oracle.conv_dgrad_acc(d, e3, wt)
+    e4_o, p4_o, _ = oracle.sq_int(S, -11 - 7)
+    J, pj = oracle.join(e4_o.astype(np.int8), p4_o, b, pb, gate01)
+    out_o, pout_o, _ = oracle.sq_int(J, pj)
+    want_e3, want_p3, want_s1, want_s2, _ = oracle.err_prescale(out_o.astype(np.int8), pout_o, mask01, x2, 97)
+    e4, p4, s4 = G.zeros(in_shape, torch.int8), G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+    out, pout, sout = G.zeros(in_shape, torch.int8), G.zeros(1, torch.int32), G.zeros(1, torch.int64)
+    n3, pn3 = G.zeros(in_shape, torch.int8), G.zeros(1, torch.int32)
+    s1, s2 = G.zeros(1, torch.int64), G.zeros(1, torch.int64)
+    head = (G.dev(G.pack_mask(mask01)), G.dev(x2), i32(97), n3, pn3, s1, s2) if with_head else (None,) * 7
+    eoq.eoq_conv_dgrad_join_head(hd, gd, G.dev(e3), i32(-11), G.dev(wt), e4, p4, s4, G.dev(b), i32(pb),
+                                 G.dev(G.pack_mask(gate01)) if gated else None, out, pout, sout, *head,
+                                 workspace=G.workspace(gd, eoq.EOQ_PASS_DGRAD))
+    torch.cuda.synchronize()
+    assert eoq.eoq_last_status(hd) == 0
+    assert np.array_equal(G.host(e4), e4_o) and p4.item() == p4_o and s4.item() == int(e4_o.astype(np.int64).sum())
+    assert np.array_equal(G.host(out), out_o) and pout.item() == pout_o and sout.item() == int(out_o.astype(np.int64).sum())
+    if with_head:
+        assert np.array_equal(G.host(n3), want_e3) and pn3.item() == want_p3 and s1.item() == want_s1 and s2.item() == want_s2
+    # every cell of the handle is clean again: the plain calls give the plain results
+    e4b, p4b = G.zeros(in_shape, torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_conv_dgrad(hd, gd, G.dev(e3), i32(-11), G.dev(wt), e4b, p4b, None, None, G.workspace(gd, eoq.EOQ_PASS_DGRAD))
+    out2, pout2 = G.zeros(in_shape, torch.int8), G.zeros(1, torch.int32)
+    eoq.eoq_aux_join(hd, e4b, p4b, G.dev(b), i32(pb), G.dev(G.pack_mask(gate01)) if gated else None, b.size, out2, pout2, None)
+    torch.cuda.synchronize()
+    assert np.array_equal(G.host(out2), out_o) and pout2.item() == pout_o
