@@ -97,6 +97,32 @@ def test_chained_step_matches_the_oracle_on_every_tensor(name, batch, mode):
     compare_parameters(st, net, "after the step")
 
 
+def test_closed_loop_step_at_the_benchmark_size():
+    """Fixup ResNet-18 at batch 64, 224x224, in the configuration the benchmark times (one captured graph with the
+    weight-gradient work on side streams, replayed): every unit's error codes and weight gradient, the joined errors,
+    the head's results and every updated parameter against the oracle (which needs about a minute for this step)."""
+    wl, st, net = build("resnet18", 64, eoq.EOQ_ROUND_RNE, lr=(1, -8))
+    saved = st.save()
+    feed(st, 0)
+    st.capture(overlap=True)
+    st.restore(saved)
+    img, labels = feed(st, 1)
+    st.replay()
+    torch.cuda.synchronize()
+    assert st.status() & ~eoq.EOQ_DEV_SQ_ZERO == 0
+    log = N.train_step(net, img, labels, st.lr_mant, st.lr_exp, st.head_lr, stochastic=False, seed=SEED)
+    for u, ou in zip(st.units, net.units):
+        fw, bw = log[ou.name]["fwd"], log[ou.name]["bwd"]
+        assert np.array_equal(host(u.x5), fw["x5"]), (ou.name, "x5")
+        assert np.array_equal(host(u.e3), bw["e3"]) and u.e3_exp.item() == bw["p3"], (ou.name, "e3")
+        assert np.array_equal(host(u.g), bw["g_w"]) and u.g_exp.item() == bw["p_gw"], (ou.name, "g_w")
+    for blk, ob in zip(st.blocks, net.blocks):
+        bw = log[net.units[ob.a].name]["bwd"]
+        assert np.array_equal(host(blk.e_in), bw["join"]) and blk.e_in_exp.item() == bw["p_join"], (blk.a.layer.name, "join")
+    assert np.array_equal(host(st.logits), log["head"]["logits"]) and np.array_equal(host(st.dpooled), log["head"]["dpooled"])
+    compare_parameters(st, net, "after the step")
+
+
 def run_trajectory(name, batch, steps, mode, full_at):
     """`steps` consecutive closed-loop steps replayed from one captured graph, a fresh image and labels every step:
     checksum of the parameters every step, full tensors at the steps in `full_at`."""
