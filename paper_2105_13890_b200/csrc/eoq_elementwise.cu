@@ -228,6 +228,14 @@ __global__ void absmax_i32_kernel(const int32_t *__restrict__ src, size_t n, Dev
     if (threadIdx.x == 0 && mx) atomicMax(&dev->absmax_u32, mx);
 }
 
+// One 256-bit streaming load (sm_100); ptr must be 32-byte aligned.
+__device__ __forceinline__ void ld_global_256_stream(const int32_t *ptr, int *v)
+{
+    asm volatile("ld.global.cs.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "l"(ptr));
+}
+
 // kNext: the error head of the layer that consumes dst rides along (see NextHead): the masked maximum sits in the
 // handle's 64-bit cell (the GEMM epilogue reduced it beside the plain one), so the codes of e3 and the head's sums
 // come out of the same pass.  n must then be a multiple of 16.
@@ -266,26 +274,28 @@ __global__ void sq_i32_kernel(const int32_t *__restrict__ src, const int32_t *sr
     // the maximum bounds every element, so |a| + 2^(sh-1) cannot wrap as long as M + M / 2^7 < 2^31
     const bool fast = sh >= 1 && M < 0x7e000000u;
     const int32_t half_m1 = fast ? (1 << (sh - 1)) - 1 : 0;
+    const bool wide_in = (reinterpret_cast<uintptr_t>(src) & 31) == 0;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
-        int c[16];
-        if (fast) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                int4 v = __ldcs(s4 + i * 4 + k);
-                c[4 * k + 0] = sq_code32_shr(v.x, sh, half_m1);
-                c[4 * k + 1] = sq_code32_shr(v.y, sh, half_m1);
-                c[4 * k + 2] = sq_code32_shr(v.z, sh, half_m1);
-                c[4 * k + 3] = sq_code32_shr(v.w, sh, half_m1);
-            }
+        int c[16], a[16];
+        if (wide_in) {   // two 256-bit loads: whole 32-byte sectors per lane
+            ld_global_256_stream(src + i * 16, a);
+            ld_global_256_stream(src + i * 16 + 8, a + 8);
         } else {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                int4 v = __ldcs(s4 + i * 4 + k);
-                c[4 * k + 0] = sq_code32(v.x, t);
-                c[4 * k + 1] = sq_code32(v.y, t);
-                c[4 * k + 2] = sq_code32(v.z, t);
-                c[4 * k + 3] = sq_code32(v.w, t);
+                const int4 v = __ldcs(s4 + i * 4 + k);
+                a[4 * k + 0] = v.x;
+                a[4 * k + 1] = v.y;
+                a[4 * k + 2] = v.z;
+                a[4 * k + 3] = v.w;
             }
+        }
+        if (fast) {
+#pragma unroll
+            for (int k = 0; k < 16; ++k) c[k] = sq_code32_shr(a[k], sh, half_m1);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 16; ++k) c[k] = sq_code32(a[k], t);
         }
         int s = 0;
 #pragma unroll

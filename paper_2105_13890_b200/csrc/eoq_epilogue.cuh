@@ -68,6 +68,14 @@ __device__ __forceinline__ int32_t sbyte(uint32_t w)
 // kernel (kTableSmemBytes at most; larger tables are read from global memory and multiplied per use).
 constexpr int kTableSmemBytes = 20 * 1024;
 
+// One 256-bit store (sm_100): a whole 32-byte sector per lane instead of two half sectors.  ptr must be 32-byte aligned.
+__device__ __forceinline__ void st_global_256(void *ptr, const uint32_t *v)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+                 "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
+
 // The three scalar codes of the forward chain as the epilogue uses them: the host values of the launch, or the
 // values read from device memory when the caller keeps them there (they then change from one replay of a captured
 // graph to the next without a new capture).
@@ -223,27 +231,33 @@ __device__ __forceinline__ void forward_16(const IgemmParams &p, const FwdScalar
     *reinterpret_cast<int4 *>(p.x5 + off) = o;
     if (p.relu_mask) *reinterpret_cast<uint16_t *>(p.relu_mask + (off >> 3)) = (uint16_t)~nbits;
     if (p.x2) {
-        int4 *d = reinterpret_cast<int4 *>(p.x2 + off);
-        d[0] = make_int4((int)__byte_perm(q[0], q[1], 0x5410), (int)__byte_perm(q[2], q[3], 0x5410),
-                         (int)__byte_perm(q[4], q[5], 0x5410), (int)__byte_perm(q[6], q[7], 0x5410));
-        d[1] = make_int4((int)__byte_perm(q[8], q[9], 0x5410), (int)__byte_perm(q[10], q[11], 0x5410),
-                         (int)__byte_perm(q[12], q[13], 0x5410), (int)__byte_perm(q[14], q[15], 0x5410));
+        uint32_t h[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) h[i] = __byte_perm(q[2 * i], q[2 * i + 1], 0x5410);
+        if ((reinterpret_cast<uintptr_t>(p.x2) & 31) == 0) {   // (uniform) the 16 codes of x2 are one 32-byte sector
+            st_global_256(p.x2 + off, h);
+        } else {
+            int4 *d = reinterpret_cast<int4 *>(p.x2 + off);
+            d[0] = make_int4((int)h[0], (int)h[1], (int)h[2], (int)h[3]);
+            d[1] = make_int4((int)h[4], (int)h[5], (int)h[6], (int)h[7]);
+        }
     }
 }
 
 // Error back-propagation: keep the exact int32 sums (the scale quantizer needs the maximum over the whole
 // tensor before any element can be coded) and track max |.|.
+// kWide: the destination is 32-byte aligned (the launch checks the base; off is a multiple of 16 elements)
+template <bool kWide>
 __device__ __forceinline__ uint32_t dgrad_16(const IgemmParams &p, const uint32_t *acc, size_t off, uint32_t &mx_masked)
 {
     uint32_t mx = 0;
-    int4 *d = reinterpret_cast<int4 *>(p.acc_out + off);
     // the consumer's error head needs the maximum over the positions its ReLU lets through as well (off is the element
     // index of the error tensor and a multiple of 16: one 16-bit word of mask bits)
     const uint32_t bits = p.next_mask ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p.next_mask) + (off >> 4)) : 0u;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        int4 v = make_int4((int)acc[4 * i], (int)acc[4 * i + 1], (int)acc[4 * i + 2], (int)acc[4 * i + 3]);
-        const uint32_t a0 = (uint32_t)abs(v.x), a1 = (uint32_t)abs(v.y), a2 = (uint32_t)abs(v.z), a3 = (uint32_t)abs(v.w);
+        const uint32_t a0 = (uint32_t)abs((int)acc[4 * i]), a1 = (uint32_t)abs((int)acc[4 * i + 1]);
+        const uint32_t a2 = (uint32_t)abs((int)acc[4 * i + 2]), a3 = (uint32_t)abs((int)acc[4 * i + 3]);
         mx = max(max(mx, a0), max(a1, max(a2, a3)));
         if (bits) {
             const uint32_t b4 = bits >> (4 * i);
@@ -252,7 +266,14 @@ __device__ __forceinline__ uint32_t dgrad_16(const IgemmParams &p, const uint32_
             mx_masked = max(mx_masked, (b4 & 4u) ? a2 : 0u);
             mx_masked = max(mx_masked, (b4 & 8u) ? a3 : 0u);
         }
-        d[i] = v;
+    }
+    if (kWide) {
+        st_global_256(p.acc_out + off, acc);
+        st_global_256(p.acc_out + off + 8, acc + 8);
+    } else {
+        int4 *d = reinterpret_cast<int4 *>(p.acc_out + off);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) d[i] = make_int4((int)acc[4 * i], (int)acc[4 * i + 1], (int)acc[4 * i + 2], (int)acc[4 * i + 3]);
     }
     return mx;
 }

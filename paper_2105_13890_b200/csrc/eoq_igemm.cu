@@ -239,6 +239,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
             }
         }
         uint32_t acc_phase = 0, mx = 0, mx_masked = 0;
+        const bool wide_out = (reinterpret_cast<uintptr_t>(p.acc_out) & 31) == 0;   // 256-bit stores of the exact sums
         bool ok = true;
         for (int tile = blockIdx.x + grp * gridDim.x; tile < num_tiles && ok; tile += 2 * gridDim.x) {
             const int mt = tile / p.num_n_tiles, nt = tile % p.num_n_tiles;
@@ -298,7 +299,7 @@ igemm_kernel(const __grid_constant__ IgemmParams p, const __grid_constant__ CUte
                             else forward_16<false, false, false>(p, fs, r, r2, off, tb, tg, sc, shift);
                         }
                     } else {
-                        mx = max(mx, dgrad_16(p, r, off, mx_masked));
+                        mx = max(mx, wide_out ? dgrad_16<true>(p, r, off, mx_masked) : dgrad_16<false>(p, r, off, mx_masked));
                     }
                 }
                 sc = sc_next;

@@ -273,6 +273,7 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                                                  (int)threadIdx.x - 128, 32 * kEpilogueWarps)
                                 : nullptr;
         uint32_t acc_phase = 0, mx = 0, mx_masked = 0;
+        const bool wide_out = (reinterpret_cast<uintptr_t>(p.acc_out) & 31) == 0;   // 256-bit stores of the exact sums
         bool ok = true;
         // (column tile, image, row tile in the image) of the current tile, carried from tile to tile: the step
         // between two tiles of this pair is constant, so its quotients are formed once instead of four integer
@@ -327,7 +328,7 @@ igemm_patch_kernel(const __grid_constant__ IgemmParams p, const __grid_constant_
                             else forward_16<true, false, false>(p, fs, r, r2, off, tb, tg, sc, 7);
                         }
                     }
-                    else mx = max(mx, dgrad_16(p, r, off, mx_masked));
+                    else mx = max(mx, wide_out ? dgrad_16<true>(p, r, off, mx_masked) : dgrad_16<false>(p, r, off, mx_masked));
                 }
                 sc = sc_next;
                 if (tb) tb += 16;
